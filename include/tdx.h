@@ -1,0 +1,193 @@
+/*
+ * tdx -- dense contractions for B200 (sm_100a): matmul with optionally transposed operands and a
+ * fused negate/scale, and zero-padded 2-D convolution with fused bias + ReLU.
+ *
+ * These are the payload computations that the schedules of "The MLIR Transform Dialect"
+ * (arXiv 2409.03864) exist to speed up; each entry point cites the passage that states its operation.
+ *
+ * Conventions (all entry points)
+ *  - Every function returns a tdx_status (int); 0 is success.  Nothing throws, aborts or exits.
+ *  - Statuses below 16 are "silenceable" in the sense of the paper's Section 3 error model:
+ *    nothing was launched, outputs are untouched, and the caller may try an alternative
+ *    (Case Study 4's `alternatives` construct).  Statuses >= 16 are definite errors: the state
+ *    of the outputs is unspecified.
+ *  - Unless a parameter says "host", every data pointer is DEVICE memory on the current CUDA device,
+ *    owned by the caller, and must stay valid until the work enqueued on `stream` has finished.
+ *    Inputs are read-only; outputs must not alias inputs.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls enqueue work
+ *    and return; device-detected conditions (a bounded wait that ran out) are reported by
+ *    tdx_check_device_status.
+ *  - All matrices are dense row-major; bf16 values are the upper 16 bits of the fp32 pattern.
+ *  - tdx_last_error() returns a thread-local, library-owned description of the last failure.
+ */
+#ifndef TDX_H_
+#define TDX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    TDX_OK = 0,
+    /* silenceable: nothing launched, outputs untouched */
+    TDX_ERR_INVALID_ARG = 1, /* negative size, bad flag, NULL pointer, unknown dtype              */
+    TDX_ERR_UNSUPPORTED = 2, /* valid request that no kernel here implements                       */
+    TDX_ERR_ALIGNMENT = 3,   /* a pointer or pitch breaks the alignment the chosen kernel needs    */
+    TDX_ERR_CONFIG = 4,      /* an explicit tdx_config is infeasible for this problem              */
+    TDX_ERR_WORKSPACE = 5,   /* workspace missing or too small                                     */
+    /* definite */
+    TDX_ERR_CUDA = 16,      /* a CUDA runtime / driver call failed                                 */
+    TDX_ERR_TIMEOUT = 17,   /* a kernel gave up on a bounded wait (see tdx_check_device_status)    */
+    TDX_ERR_NO_DEVICE = 18  /* no usable sm_100 device / driver                                    */
+} tdx_status;
+
+typedef enum {
+    TDX_F32 = 0, /* A, B, C fp32; fp32 FMA on CUDA cores                     */
+    TDX_BF16 = 1 /* A, B bf16; fp32 accumulate (tensor cores); C bf16        */
+} tdx_dtype;
+
+typedef enum {
+    TDX_KERNEL_AUTO = 0,
+    TDX_KERNEL_UMMA = 1,    /* tcgen05 tensor-core pipeline (bf16 only, needs 16-byte aligned pitches) */
+    TDX_KERNEL_SIMT = 2,    /* tiled fp32 CUDA-core GEMM (fp32 GEMM only)                              */
+    TDX_KERNEL_GENERIC = 3  /* one thread per output; any dtype, shape and alignment                   */
+} tdx_kernel;
+
+/*
+ * Tile configuration: the knobs the paper's Case Study 5 hands to its autotuner (tile sizes per
+ * loop, vectorise or not) restated for this hardware.  A zero field means "choose for me".
+ */
+typedef struct {
+    int kernel;     /* tdx_kernel                                                              */
+    int tile_m;     /* 128                                                                     */
+    int tile_n;     /* 32, 64, 96, ..., 256 (multiple of 32; multiple of 64 when transB = 0)    */
+    int tile_k;     /* 64                                                                      */
+    int stages;     /* depth of the TMA/mbarrier ring, 2..8, bounded by shared memory          */
+    int cta_pair;   /* 1 (one CTA per tile)                                                    */
+    int split_k;    /* >= 1; > 1 needs a workspace and runs a fixed-order reduction afterwards  */
+    int store_mode; /* 0 = 16-byte stores from registers                                       */
+    int raster;     /* width, in tiles along M, of the panels the tile order walks; 0 = all     */
+    int patch_w;    /* conv only: output-pixel patch that forms the rows of a tile (w x h,      */
+    int patch_h;    /*   w*h a power of two <= 128, w >= 8); 0 = choose                         */
+} tdx_config;
+
+/*
+ * C[M x N] = alpha * op(A)[M x K] . op(B)[K x N]     (C overwritten; no accumulate)
+ *
+ * The operation is the matmul loop nest of the paper's Case Study 4 (the OpenMP tiling figure),
+ * one batch, without the accumulate.  transA / transB are the "matmul that supports transposed
+ * operands" of Case Study 3's matmul_of_transpose pattern: the transpose is a property of how the
+ * operand is read, never a copy.  The negate of negate_of_transpose commutes with the transpose
+ * and the product, so it is alpha = -1.
+ *
+ *   transA = 0: A stored M x K;  transA = 1: A stored K x M.
+ *   transB = 0: B stored K x N;  transB = 1: B stored N x K.
+ *   dtype: TDX_F32 (all fp32) or TDX_BF16 (bf16 in, fp32 accumulate, bf16 out, one rounding of alpha*acc).
+ *   M or N = 0: no-op.  K = 0: C is zero-filled.
+ * Errors: INVALID_ARG (negative size, flag not 0/1, NULL pointer with non-empty problem, unknown dtype,
+ *         non-finite alpha is allowed), CUDA.  Shapes that miss the tensor-core path's alignment rules
+ *         are served by the generic GPU kernel, not rejected.  There is no CPU fallback.
+ */
+int tdx_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype,
+             const void* A, const void* B, void* C, void* stream);
+
+/*
+ * Same as tdx_gemm with an explicit configuration and caller-owned split-K workspace.
+ * cfg = NULL or cfg->split_k = 0: the library chooses split_k (tuning cache, else heuristic); then
+ * `workspace` may be NULL and the library uses an internal, lazily grown buffer.  With an explicit
+ * cfg->split_k > 1 the caller must pass at least tdx_gemm_workspace_size bytes (256-byte aligned)
+ * -> else WORKSPACE.
+ * An infeasible cfg -> CONFIG with C untouched (the paper's `alternatives`: a failed alternative
+ * leaves the payload unchanged).
+ */
+int tdx_gemm_ex(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype,
+                const void* A, const void* B, void* C, void* stream,
+                const tdx_config* cfg, void* workspace, size_t workspace_bytes);
+
+/* Bytes of workspace tdx_gemm_ex needs for cfg (0 when cfg->split_k <= 1). */
+int tdx_gemm_workspace_size(int64_t M, int64_t N, int64_t K, int dtype, const tdx_config* cfg, size_t* bytes);
+
+/*
+ * y[n,p,q,k] = relu?( bias[k] + sum_{r,s,c} X(n, p*stride + r - pad, q*stride + s - pad, c) * w[k,r,s,c] )
+ * with X = x inside the image and 0 outside: the zero padding is never materialised and padded
+ * elements are never added (the add_of_zero_pad pattern of Case Study 3).  The paper states no
+ * convolution formula; this is the standard cross-correlation of the ResNet-50 layers its Case
+ * Study 4 draws its loop nest from.
+ *
+ *   x: N x H x W x Cin (NHWC);  w: Cout x R x S x Cin (KRSC);  bias: fp32 [Cout] or NULL;
+ *   y: N x P x Q x Cout with P = floor((H + 2 pad - R) / stride) + 1, Q likewise (0 if negative).
+ *   dtype: TDX_BF16 (x, w, y bf16; fp32 accumulate) or TDX_F32 (all fp32).  relu in {0, 1}.
+ * Errors: INVALID_ARG (size <= 0 for Cin/R/S, negative N/H/W/Cout/pad, stride < 1, NULL pointers), CUDA.
+ * Empty outputs (N, Cout, P or Q = 0) are a no-op.
+ */
+int tdx_conv2d_bias_relu(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
+                         int pad, int stride, int dtype, const void* x, const void* w, const float* bias,
+                         int relu, void* y, void* stream);
+
+/* As above with an explicit configuration (split_k must be 1).  Infeasible cfg -> CONFIG, y untouched. */
+int tdx_conv2d_bias_relu_ex(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
+                            int pad, int stride, int dtype, const void* x, const void* w, const float* bias,
+                            int relu, void* y, void* stream, const tdx_config* cfg);
+
+/*
+ * Host-buffer variants: A, B, C (x, w, bias, y) are HOST pointers (pinned memory gives the best
+ * copy rate).  The call copies the inputs to device staging buffers owned by the library, runs the
+ * same kernels as above, copies the result back and returns after the stream has drained.
+ */
+int tdx_gemm_host(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype,
+                  const void* A_host, const void* B_host, void* C_host, void* stream);
+int tdx_conv2d_bias_relu_host(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
+                              int pad, int stride, int dtype, const void* x_host, const void* w_host,
+                              const float* bias_host, int relu, void* y_host, void* stream);
+
+/*
+ * Tile-configuration search: the stand-in for the autotuner integration of the paper's Case Study 5.
+ * Enumerates the configurations that pass the static constraints (the analogue of "tile sizes must
+ * divide their dimension, vectorise only if divisible": shared-memory and TMEM budgets, layout
+ * divisibility), times each on the device with CUDA events on scratch operands the call allocates,
+ * returns the fastest and records it in the in-process tuning cache used by the automatic choice.
+ *   iters: timed launches per candidate (>= 1).  best / best_us: outputs (best_us = mean microseconds).
+ *   tried / tried_us / cap / n_tried: optional (NULL / 0) list of every candidate with its time.
+ */
+int tdx_tune_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, int iters,
+                  tdx_config* best, float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried,
+                  void* stream);
+int tdx_tune_conv2d(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
+                    int pad, int stride, int dtype, int iters, tdx_config* best, float* best_us,
+                    tdx_config* tried, float* tried_us, int cap, int* n_tried, void* stream);
+
+/* The statically feasible search space (no device needed).  Writes up to cap configs, *n = total count. */
+int tdx_enum_gemm_configs(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype,
+                          tdx_config* out, int cap, int* n);
+int tdx_enum_conv2d_configs(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
+                            int pad, int stride, int dtype, tdx_config* out, int cap, int* n);
+
+/* The configuration the automatic choice would use right now (tuning cache, else heuristic). */
+int tdx_default_gemm_config(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, tdx_config* out);
+int tdx_default_conv2d_config(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
+                              int pad, int stride, int dtype, tdx_config* out);
+
+/* Persist / restore the tuning cache (a small JSON text file). */
+int tdx_tune_save(const char* json_path);
+int tdx_tune_load(const char* json_path);
+int tdx_tune_clear(void);
+
+/*
+ * Synchronises `stream`, reads and clears the device status word.  TDX_OK, or TDX_ERR_TIMEOUT if a
+ * kernel abandoned a bounded wait since the last check (its outputs are then unspecified).
+ */
+int tdx_check_device_status(void* stream);
+
+/* Number of kernels this library has launched in this process (all threads). */
+int64_t tdx_kernel_launch_count(void);
+
+const char* tdx_last_error(void);
+const char* tdx_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TDX_H_ */

@@ -1,0 +1,254 @@
+"""ctypes binding of libtdx.so: argument marshalling only, same names as include/tdx.h.
+
+Pointers may be given as torch tensors (their data_ptr() is used), numpy arrays (for the *_host
+entry points), integers or None.  Streams may be a torch.cuda.Stream, an integer handle or None.
+Every function returns the library's status code unless stated otherwise; `check()` turns a
+non-zero status into a TdxError carrying tdx_last_error().
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+_LIB_PATH = Path(__file__).resolve().parent / "libtdx.so"
+
+TDX_OK = 0
+TDX_ERR_INVALID_ARG = 1
+TDX_ERR_UNSUPPORTED = 2
+TDX_ERR_ALIGNMENT = 3
+TDX_ERR_CONFIG = 4
+TDX_ERR_WORKSPACE = 5
+TDX_ERR_CUDA = 16
+TDX_ERR_TIMEOUT = 17
+TDX_ERR_NO_DEVICE = 18
+
+TDX_F32 = 0
+TDX_BF16 = 1
+
+TDX_KERNEL_AUTO = 0
+TDX_KERNEL_UMMA = 1
+TDX_KERNEL_SIMT = 2
+TDX_KERNEL_GENERIC = 3
+
+
+class TdxError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"tdx status {status}: {message}")
+        self.status = status
+
+
+class tdx_config(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in
+                ("kernel", "tile_m", "tile_n", "tile_k", "stages", "cta_pair", "split_k", "store_mode", "raster",
+                 "patch_w", "patch_h")]
+
+    def as_dict(self) -> dict:
+        return {n: int(getattr(self, n)) for n, _ in self._fields_}
+
+    def __repr__(self) -> str:
+        return "tdx_config(" + ", ".join(f"{k}={v}" for k, v in self.as_dict().items()) + ")"
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libtdx.so (built in-tree by paper_2409_03864_b200.build).  Fails loudly if it is missing."""
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise FileNotFoundError(
+                f"{_LIB_PATH} is missing: run `python -m paper_2409_03864_b200.build` (there is no fallback path)")
+        L = ctypes.CDLL(str(_LIB_PATH))
+        i64, ci, cf, vp, sz = ctypes.c_int64, ctypes.c_int, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t
+        cfgp = ctypes.POINTER(tdx_config)
+        fp = ctypes.POINTER(ctypes.c_float)
+        ip = ctypes.POINTER(ctypes.c_int)
+        gemm_args = [i64, i64, i64, ci, ci, cf, ci, vp, vp, vp, vp]
+        conv_args = [i64] * 7 + [ci, ci, ci, vp, vp, vp, ci, vp, vp]
+        L.tdx_gemm.argtypes = gemm_args
+        L.tdx_gemm_ex.argtypes = gemm_args + [cfgp, vp, sz]
+        L.tdx_gemm_workspace_size.argtypes = [i64, i64, i64, ci, cfgp, ctypes.POINTER(sz)]
+        L.tdx_conv2d_bias_relu.argtypes = conv_args
+        L.tdx_conv2d_bias_relu_ex.argtypes = conv_args + [cfgp]
+        L.tdx_gemm_host.argtypes = gemm_args
+        L.tdx_conv2d_bias_relu_host.argtypes = conv_args
+        L.tdx_tune_gemm.argtypes = [i64, i64, i64, ci, ci, ci, ci, cfgp, fp, cfgp, fp, ci, ip, vp]
+        L.tdx_tune_conv2d.argtypes = [i64] * 7 + [ci, ci, ci, ci, cfgp, fp, cfgp, fp, ci, ip, vp]
+        L.tdx_enum_gemm_configs.argtypes = [i64, i64, i64, ci, ci, ci, cfgp, ci, ip]
+        L.tdx_enum_conv2d_configs.argtypes = [i64] * 7 + [ci, ci, ci, cfgp, ci, ip]
+        L.tdx_default_gemm_config.argtypes = [i64, i64, i64, ci, ci, ci, cfgp]
+        L.tdx_default_conv2d_config.argtypes = [i64] * 7 + [ci, ci, ci, cfgp]
+        L.tdx_tune_save.argtypes = [ctypes.c_char_p]
+        L.tdx_tune_load.argtypes = [ctypes.c_char_p]
+        L.tdx_tune_clear.argtypes = []
+        L.tdx_check_device_status.argtypes = [vp]
+        L.tdx_kernel_launch_count.argtypes = []
+        L.tdx_kernel_launch_count.restype = i64
+        L.tdx_last_error.restype = ctypes.c_char_p
+        L.tdx_version.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            fn = getattr(L, name)
+            if name not in ("tdx_kernel_launch_count", "tdx_last_error", "tdx_version"):
+                fn.restype = ci
+        _lib = L
+    return _lib
+
+
+# every symbol include/tdx.h declares
+EXPORTS = (
+    "tdx_gemm", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_relu_ex",
+    "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
+    "tdx_enum_conv2d_configs", "tdx_default_gemm_config", "tdx_default_conv2d_config", "tdx_tune_save",
+    "tdx_tune_load", "tdx_tune_clear", "tdx_check_device_status", "tdx_kernel_launch_count", "tdx_last_error",
+    "tdx_version",
+)
+
+
+def _ptr(x):
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    if hasattr(x, "ctypes"):
+        return x.ctypes.data
+    raise TypeError(f"cannot take a pointer from {type(x)}")
+
+
+def _stream(s):
+    if s is None:
+        return None
+    if isinstance(s, int):
+        return s
+    return s.cuda_stream
+
+
+def _cfg(c):
+    return None if c is None else ctypes.byref(c)
+
+
+def tdx_last_error() -> str:
+    return lib().tdx_last_error().decode()
+
+
+def tdx_version() -> str:
+    return lib().tdx_version().decode()
+
+
+def check(status: int) -> int:
+    if status != TDX_OK:
+        raise TdxError(status, tdx_last_error())
+    return status
+
+
+def tdx_gemm(M, N, K, transA, transB, alpha, dtype, A, B, C, stream=None) -> int:
+    return lib().tdx_gemm(M, N, K, transA, transB, alpha, dtype, _ptr(A), _ptr(B), _ptr(C), _stream(stream))
+
+
+def tdx_gemm_ex(M, N, K, transA, transB, alpha, dtype, A, B, C, stream=None, cfg=None, workspace=None,
+                workspace_bytes=0) -> int:
+    return lib().tdx_gemm_ex(M, N, K, transA, transB, alpha, dtype, _ptr(A), _ptr(B), _ptr(C), _stream(stream),
+                             _cfg(cfg), _ptr(workspace), workspace_bytes)
+
+
+def tdx_gemm_workspace_size(M, N, K, dtype, cfg):
+    """Returns (status, bytes)."""
+    out = ctypes.c_size_t(0)
+    st = lib().tdx_gemm_workspace_size(M, N, K, dtype, _cfg(cfg), ctypes.byref(out))
+    return st, int(out.value)
+
+
+def tdx_conv2d_bias_relu(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, relu, y, stream=None) -> int:
+    return lib().tdx_conv2d_bias_relu(N, H, W, Cin, Cout, R, S, pad, stride, dtype, _ptr(x), _ptr(w), _ptr(bias),
+                                      relu, _ptr(y), _stream(stream))
+
+
+def tdx_conv2d_bias_relu_ex(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, relu, y, stream=None,
+                            cfg=None) -> int:
+    return lib().tdx_conv2d_bias_relu_ex(N, H, W, Cin, Cout, R, S, pad, stride, dtype, _ptr(x), _ptr(w), _ptr(bias),
+                                         relu, _ptr(y), _stream(stream), _cfg(cfg))
+
+
+def tdx_gemm_host(M, N, K, transA, transB, alpha, dtype, A_host, B_host, C_host, stream=None) -> int:
+    return lib().tdx_gemm_host(M, N, K, transA, transB, alpha, dtype, _ptr(A_host), _ptr(B_host), _ptr(C_host),
+                               _stream(stream))
+
+
+def tdx_conv2d_bias_relu_host(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x_host, w_host, bias_host, relu, y_host,
+                              stream=None) -> int:
+    return lib().tdx_conv2d_bias_relu_host(N, H, W, Cin, Cout, R, S, pad, stride, dtype, _ptr(x_host), _ptr(w_host),
+                                           _ptr(bias_host), relu, _ptr(y_host), _stream(stream))
+
+
+def _tune(call, cap):
+    best, best_us = tdx_config(), ctypes.c_float(0)
+    tried = (tdx_config * cap)()
+    tried_us = (ctypes.c_float * cap)()
+    n = ctypes.c_int(0)
+    st = call(ctypes.byref(best), ctypes.byref(best_us), tried, tried_us, cap, ctypes.byref(n))
+    k = min(int(n.value), cap)
+    return st, best, float(best_us.value), [(tried[i].as_dict(), float(tried_us[i])) for i in range(k)]
+
+
+def tdx_tune_gemm(M, N, K, transA, transB, dtype, iters=20, stream=None, cap=512):
+    """Returns (status, best tdx_config, best microseconds, [(config dict, microseconds), ...])."""
+    L = lib()
+    return _tune(lambda b, bu, t, tu, c, n: L.tdx_tune_gemm(M, N, K, transA, transB, dtype, iters, b, bu, t, tu, c, n,
+                                                            _stream(stream)), cap)
+
+
+def tdx_tune_conv2d(N, H, W, Cin, Cout, R, S, pad, stride, dtype, iters=20, stream=None, cap=512):
+    L = lib()
+    return _tune(lambda b, bu, t, tu, c, n: L.tdx_tune_conv2d(N, H, W, Cin, Cout, R, S, pad, stride, dtype, iters, b,
+                                                              bu, t, tu, c, n, _stream(stream)), cap)
+
+
+def _enum(call, cap=1024):
+    out = (tdx_config * cap)()
+    n = ctypes.c_int(0)
+    st = call(out, cap, ctypes.byref(n))
+    return st, [out[i].as_dict() for i in range(min(cap, int(n.value)))]
+
+
+def tdx_enum_gemm_configs(M, N, K, transA, transB, dtype):
+    """Returns (status, [config dict, ...])."""
+    L = lib()
+    return _enum(lambda o, c, n: L.tdx_enum_gemm_configs(M, N, K, transA, transB, dtype, o, c, n))
+
+
+def tdx_enum_conv2d_configs(N, H, W, Cin, Cout, R, S, pad, stride, dtype):
+    L = lib()
+    return _enum(lambda o, c, n: L.tdx_enum_conv2d_configs(N, H, W, Cin, Cout, R, S, pad, stride, dtype, o, c, n))
+
+
+def tdx_default_gemm_config(M, N, K, transA, transB, dtype):
+    """Returns (status, tdx_config)."""
+    c = tdx_config()
+    return lib().tdx_default_gemm_config(M, N, K, transA, transB, dtype, ctypes.byref(c)), c
+
+
+def tdx_default_conv2d_config(N, H, W, Cin, Cout, R, S, pad, stride, dtype):
+    c = tdx_config()
+    return lib().tdx_default_conv2d_config(N, H, W, Cin, Cout, R, S, pad, stride, dtype, ctypes.byref(c)), c
+
+
+def tdx_tune_save(path: str) -> int:
+    return lib().tdx_tune_save(str(path).encode())
+
+
+def tdx_tune_load(path: str) -> int:
+    return lib().tdx_tune_load(str(path).encode())
+
+
+def tdx_tune_clear() -> int:
+    return lib().tdx_tune_clear()
+
+
+def tdx_check_device_status(stream=None) -> int:
+    return lib().tdx_check_device_status(_stream(stream))
+
+
+def tdx_kernel_launch_count() -> int:
+    return int(lib().tdx_kernel_launch_count())

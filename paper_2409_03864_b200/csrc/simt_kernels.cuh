@@ -1,0 +1,193 @@
+// CUDA-core kernels: the fp32 tiled GEMM, the generic (any shape / alignment) GEMM and
+// convolution used when the tensor-core path's layout constraints do not hold, and the
+// fixed-order split-K reduction.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace tdx {
+
+__device__ __forceinline__ float ld_as_float(const float* p, long long i) { return __ldg(p + i); }
+__device__ __forceinline__ float ld_as_float(const __nv_bfloat16* p, long long i) {
+    return __bfloat162float(p[i]);
+}
+__device__ __forceinline__ void st_from_float(float* p, long long i, float v) { p[i] = v; }
+__device__ __forceinline__ void st_from_float(__nv_bfloat16* p, long long i, float v) {
+    p[i] = __float2bfloat16_rn(v);
+}
+
+// ---------------------------------------------------------------------------
+// fp32 tiled GEMM: C = alpha * op(A) op(B), element (i,k) of op(A) at A[i*sa_i + k*sa_k],
+// element (k,j) of op(B) at B[k*sb_k + j*sb_j].  Each thread owns a TM x TN register tile;
+// the reduction runs k = 0..K-1 in order with fp32 FMAs.
+// ---------------------------------------------------------------------------
+template <int BM, int BN, int BK, int TM, int TN>
+__global__ void __launch_bounds__((BM / TM) * (BN / TN))
+sgemm_tiled_kernel(int M, int N, int K, long long sa_i, long long sa_k, long long sb_k, long long sb_j, float alpha,
+                   const float* __restrict__ A, const float* __restrict__ B, float* __restrict__ C) {
+    constexpr int NT = (BM / TM) * (BN / TN);
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Bs[BK][BN + 4];
+    const int tid = threadIdx.x;
+    const int tx = tid % (BN / TN);
+    const int ty = tid / (BN / TN);
+    const int m0 = blockIdx.y * BM;
+    const int n0 = blockIdx.x * BN;
+    float acc[TM][TN];
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) acc[i][j] = 0.0f;
+
+    for (int k0 = 0; k0 < K; k0 += BK) {
+        for (int idx = tid; idx < BM * BK; idx += NT) {
+            int i, k;
+            if (sa_k == 1) { i = idx / BK; k = idx % BK; } else { i = idx % BM; k = idx / BM; }
+            const int gi = m0 + i, gk = k0 + k;
+            As[k][i] = (gi < M && gk < K) ? __ldg(A + gi * sa_i + gk * sa_k) : 0.0f;
+        }
+        for (int idx = tid; idx < BN * BK; idx += NT) {
+            int j, k;
+            if (sb_j == 1) { k = idx / BN; j = idx % BN; } else { j = idx / BK; k = idx % BK; }
+            const int gj = n0 + j, gk = k0 + k;
+            Bs[k][j] = (gj < N && gk < K) ? __ldg(B + gk * sb_k + gj * sb_j) : 0.0f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < BK; ++k) {
+            float a[TM], b[TN];
+#pragma unroll
+            for (int i = 0; i < TM; ++i) a[i] = As[k][ty * TM + i];
+#pragma unroll
+            for (int j = 0; j < TN; ++j) b[j] = Bs[k][tx * TN + j];
+#pragma unroll
+            for (int i = 0; i < TM; ++i)
+#pragma unroll
+                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+        const int gi = m0 + ty * TM + i;
+        if (gi >= M) continue;
+#pragma unroll
+        for (int j = 0; j < TN; ++j) {
+            const int gj = n0 + tx * TN + j;
+            if (gj < N) C[static_cast<long long>(gi) * N + gj] = alpha * acc[i][j];
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Generic GEMM, one thread per output element (no layout or alignment constraints).
+// ---------------------------------------------------------------------------
+template <typename TIn, typename TOut>
+__global__ void gemm_generic_kernel(long long M, long long N, long long K, long long sa_i, long long sa_k,
+                                    long long sb_k, long long sb_j, float alpha, const TIn* __restrict__ A,
+                                    const TIn* __restrict__ B, TOut* __restrict__ C) {
+    const long long total = M * N;
+    for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < total;
+         e += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const long long i = e / N, j = e - i * N;
+        float acc = 0.0f;
+        for (long long k = 0; k < K; ++k)
+            acc = fmaf(ld_as_float(A, i * sa_i + k * sa_k), ld_as_float(B, k * sb_k + j * sb_j), acc);
+        st_from_float(C, e, alpha * acc);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Generic convolution + bias + ReLU, one thread per output element.  x NHWC, w KRSC.
+// Taps that fall into the zero padding are skipped (they would add zero).
+// ---------------------------------------------------------------------------
+template <typename TIn, typename TOut>
+__global__ void conv2d_generic_kernel(int Nimg, int H, int W, int Cin, int Cout, int R, int S, int pad, int stride,
+                                      int P, int Q, const TIn* __restrict__ x, const TIn* __restrict__ w,
+                                      const float* __restrict__ bias, int relu, TOut* __restrict__ y) {
+    const long long total = static_cast<long long>(Nimg) * P * Q * Cout;
+    for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < total;
+         e += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const int k = static_cast<int>(e % Cout);
+        long long row = e / Cout;
+        const int q = static_cast<int>(row % Q);
+        row /= Q;
+        const int p = static_cast<int>(row % P);
+        const int n = static_cast<int>(row / P);
+        float acc = 0.0f;
+        for (int r = 0; r < R; ++r) {
+            const int h = p * stride + r - pad;
+            if (h < 0 || h >= H) continue;
+            for (int s = 0; s < S; ++s) {
+                const int ww = q * stride + s - pad;
+                if (ww < 0 || ww >= W) continue;
+                const long long xo = ((static_cast<long long>(n) * H + h) * W + ww) * Cin;
+                const long long wo = ((static_cast<long long>(k) * R + r) * S + s) * Cin;
+                for (int c = 0; c < Cin; ++c) acc = fmaf(ld_as_float(x, xo + c), ld_as_float(w, wo + c), acc);
+            }
+        }
+        if (bias != nullptr) acc += __ldg(bias + k);
+        if (relu) acc = fmaxf(acc, 0.0f);
+        st_from_float(y, e, acc);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Split-K reduction: out[i,j] = epilogue( sum_{s = 0..split-1, ascending} partial[s][i][j] ).
+// The order is fixed, so results do not depend on scheduling.
+// ---------------------------------------------------------------------------
+__global__ void splitk_reduce_kernel(long long MN, int N, int split, const float* __restrict__ partial, float alpha,
+                                     const float* __restrict__ bias, int relu, __nv_bfloat16* __restrict__ out,
+                                     int vec8) {
+    if (vec8) {
+        const long long groups = MN / 8;
+        for (long long g = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; g < groups;
+             g += static_cast<long long>(gridDim.x) * blockDim.x) {
+            const long long e = g * 8;
+            float acc[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
+            for (int s = 0; s < split; ++s) {
+                const float4* src = reinterpret_cast<const float4*>(partial + s * MN + e);
+                const float4 v0 = __ldg(src), v1 = __ldg(src + 1);
+                acc[0] += v0.x; acc[1] += v0.y; acc[2] += v0.z; acc[3] += v0.w;
+                acc[4] += v1.x; acc[5] += v1.y; acc[6] += v1.z; acc[7] += v1.w;
+            }
+            const int col = static_cast<int>(e % N);
+            uint32_t pk[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float a = alpha * acc[2 * j], b = alpha * acc[2 * j + 1];
+                if (bias != nullptr) { a += __ldg(bias + col + 2 * j); b += __ldg(bias + col + 2 * j + 1); }
+                if (relu) { a = fmaxf(a, 0.0f); b = fmaxf(b, 0.0f); }
+                __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+                pk[j] = *reinterpret_cast<uint32_t*>(&h);
+            }
+            *reinterpret_cast<uint4*>(out + e) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        }
+    } else {
+        for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < MN;
+             e += static_cast<long long>(gridDim.x) * blockDim.x) {
+            float acc = 0.0f;
+            for (int s = 0; s < split; ++s) acc += __ldg(partial + s * MN + e);
+            float v = alpha * acc;
+            if (bias != nullptr) v += __ldg(bias + e % N);
+            if (relu) v = fmaxf(v, 0.0f);
+            out[e] = __float2bfloat16_rn(v);
+        }
+    }
+}
+
+// Deterministic pseudo-random fill used only by the tuner's scratch operands.
+__global__ void fill_pattern_bf16_kernel(__nv_bfloat16* p, long long n, uint32_t seed) {
+    for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < n;
+         e += static_cast<long long>(gridDim.x) * blockDim.x) {
+        uint32_t h = static_cast<uint32_t>(e) * 2654435761u + seed;
+        h ^= h >> 15; h *= 2246822519u; h ^= h >> 13;
+        const float v = (static_cast<float>(h & 0xFFFF) - 32768.0f) * (1.0f / 16384.0f);
+        p[e] = __float2bfloat16_rn(v);
+    }
+}
+
+}  // namespace tdx

@@ -1,0 +1,1206 @@
+// C-ABI of the tdx library: argument validation, kernel choice, TMA descriptor cache,
+// launches, the tile-configuration search and its cache.  See include/tdx.h for the contract.
+#include "tdx.h"
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "simt_kernels.cuh"
+#include "umma_kernel.cuh"
+
+namespace {
+
+using tdx::UmmaParams;
+
+// ------------------------------------------------------------------ errors
+thread_local std::string g_err;
+
+int fail(int status, const char* fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    g_err = buf;
+    return status;
+}
+
+#define TDX_CUDA(expr)                                                                                   \
+    do {                                                                                                 \
+        cudaError_t e_ = (expr);                                                                         \
+        if (e_ != cudaSuccess) return fail(TDX_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_)); \
+    } while (0)
+
+std::atomic<int64_t> g_launches{0};
+
+__device__ int g_device_status_word = 0;
+
+// ------------------------------------------------------------------ per-device state
+constexpr int kSmemLimitDefault = 232448;  // 227 KiB opt-in limit of sm_100
+constexpr int kStaticSmemReserve = 512;    // barriers and flags declared statically in the kernel
+constexpr int kDefaultSmCount = 148;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct DeviceCtx {
+    int dev = -1;
+    int sm_count = kDefaultSmCount;
+    int smem_optin = kSmemLimitDefault;
+    int* status_ptr = nullptr;
+    EncodeTiledFn encode = nullptr;
+    void* ws = nullptr;          // internal split-K workspace
+    size_t ws_bytes = 0;
+    void* staging[4] = {nullptr, nullptr, nullptr, nullptr};  // host-variant device copies
+    size_t staging_bytes[4] = {0, 0, 0, 0};
+};
+
+std::mutex g_mu;
+std::map<int, DeviceCtx> g_ctx;
+
+int get_ctx(DeviceCtx** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(TDX_ERR_NO_DEVICE, "no CUDA device: %s", cudaGetErrorString(e));
+    }
+    std::lock_guard<std::mutex> lk(g_mu);
+    auto it = g_ctx.find(dev);
+    if (it != g_ctx.end()) {
+        *out = &it->second;
+        return TDX_OK;
+    }
+    cudaDeviceProp prop;
+    e = cudaGetDeviceProperties(&prop, dev);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(TDX_ERR_NO_DEVICE, "cudaGetDeviceProperties: %s", cudaGetErrorString(e));
+    }
+    if (prop.major != 10) return fail(TDX_ERR_NO_DEVICE, "device %d is sm_%d%d, this library is built for sm_100a", dev, prop.major, prop.minor);
+    DeviceCtx c;
+    c.dev = dev;
+    c.sm_count = prop.multiProcessorCount;
+    c.smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
+    void* sym = nullptr;
+    e = cudaGetSymbolAddress(&sym, g_device_status_word);
+    if (e != cudaSuccess) return fail(TDX_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+    c.status_ptr = static_cast<int*>(sym);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess)
+        return fail(TDX_ERR_NO_DEVICE, "driver does not export cuTensorMapEncodeTiled");
+    c.encode = reinterpret_cast<EncodeTiledFn>(fn);
+    e = cudaFuncSetAttribute(tdx::umma_contract_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             c.smem_optin - kStaticSmemReserve);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tdx::umma_contract_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 c.smem_optin - kStaticSmemReserve);
+    if (e != cudaSuccess) return fail(TDX_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
+    auto ins = g_ctx.emplace(dev, c);
+    *out = &ins.first->second;
+    return TDX_OK;
+}
+
+// ------------------------------------------------------------------ TMA descriptor cache
+struct MapKey {
+    const void* ptr;
+    int rank;
+    uint64_t dims[4];
+    uint64_t strides[3];
+    uint32_t box[4];
+    bool operator<(const MapKey& o) const { return std::memcmp(this, &o, sizeof(MapKey)) < 0; }
+};
+std::map<MapKey, CUtensorMap> g_maps;
+
+// bf16 tensor, 128-byte swizzle, zero fill outside the tensor.
+int get_tensor_map(DeviceCtx* ctx, const void* ptr, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                   const uint32_t* box, CUtensorMap* out) {
+    MapKey key;
+    std::memset(&key, 0, sizeof key);
+    key.ptr = ptr;
+    key.rank = rank;
+    for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+    for (int i = 0; i + 1 < rank; ++i) key.strides[i] = strides_bytes[i];
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        auto it = g_maps.find(key);
+        if (it != g_maps.end()) { *out = it->second; return TDX_OK; }
+    }
+    cuuint64_t gdim[4], gstr[3];
+    cuuint32_t gbox[4], estr[4];
+    for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; gbox[i] = box[i]; estr[i] = 1; }
+    for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_bytes[i];
+    CUtensorMap m;
+    CUresult r = ctx->encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank),
+                             const_cast<void*>(ptr), gdim, gstr, gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS)
+        return fail(TDX_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) rank %d dims %llu %llu box %u %u", (int)r, rank,
+                    (unsigned long long)dims[0], (unsigned long long)(rank > 1 ? dims[1] : 0), box[0],
+                    rank > 1 ? box[1] : 0);
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        if (g_maps.size() > 4096) g_maps.clear();
+        g_maps[key] = m;
+    }
+    *out = m;
+    return TDX_OK;
+}
+
+// ------------------------------------------------------------------ tuning cache
+struct TuneEntry { tdx_config cfg; float us; };
+std::map<std::string, TuneEntry> g_tune;
+
+std::string gemm_key(int64_t M, int64_t N, int64_t K, int tA, int tB, int dtype) {
+    char b[160];
+    snprintf(b, sizeof b, "gemm:%lld:%lld:%lld:%d:%d:%d", (long long)M, (long long)N, (long long)K, tA, tB, dtype);
+    return b;
+}
+std::string conv_key(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
+                     int stride, int dtype) {
+    char b[200];
+    snprintf(b, sizeof b, "conv:%lld:%lld:%lld:%lld:%lld:%lld:%lld:%d:%d:%d", (long long)N, (long long)H, (long long)W,
+             (long long)Cin, (long long)Cout, (long long)R, (long long)S, pad, stride, dtype);
+    return b;
+}
+bool tune_lookup(const std::string& key, tdx_config* out) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    auto it = g_tune.find(key);
+    if (it == g_tune.end()) return false;
+    *out = it->second.cfg;
+    return true;
+}
+void cfg_to_ints(const tdx_config& c, int* v) {
+    v[0] = c.kernel; v[1] = c.tile_m; v[2] = c.tile_n; v[3] = c.tile_k; v[4] = c.stages; v[5] = c.cta_pair;
+    v[6] = c.split_k; v[7] = c.store_mode; v[8] = c.raster; v[9] = c.patch_w; v[10] = c.patch_h;
+}
+void ints_to_cfg(const int* v, tdx_config* c) {
+    c->kernel = v[0]; c->tile_m = v[1]; c->tile_n = v[2]; c->tile_k = v[3]; c->stages = v[4]; c->cta_pair = v[5];
+    c->split_k = v[6]; c->store_mode = v[7]; c->raster = v[8]; c->patch_w = v[9]; c->patch_h = v[10];
+}
+
+// ------------------------------------------------------------------ problem descriptions
+struct GemmProblem {
+    int64_t M, N, K;
+    int transA, transB, dtype;
+};
+struct ConvProblem {
+    int64_t N, H, W, Cin, Cout, R, S;
+    int pad, stride, dtype;
+    int64_t P, Q;
+};
+
+int64_t conv_out_dim(int64_t H, int64_t R, int64_t pad, int64_t stride) {
+    const int64_t span = H + 2 * pad - R;
+    return span < 0 ? 0 : span / stride + 1;
+}
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// Layout rules of the tensor-core GEMM path: every TMA row pitch must be a multiple of 16 bytes.
+bool gemm_umma_layout_ok(const GemmProblem& g) {
+    if (g.dtype != TDX_BF16) return false;
+    if (g.M >= (1LL << 31) || g.N >= (1LL << 31) || g.K >= (1LL << 31)) return false;
+    if (g.transA ? (g.M % 8) : (g.K % 8)) return false;
+    if (g.transB ? (g.K % 8) : (g.N % 8)) return false;
+    if (ceil_div(g.M, 128) * ceil_div(g.N, 32) * 64 >= (1LL << 31)) return false;
+    return true;
+}
+bool conv_umma_layout_ok(const ConvProblem& c) {
+    if (c.dtype != TDX_BF16 || c.stride != 1) return false;
+    if (c.Cin % 8) return false;
+    if (c.N * c.P * c.Q >= (1LL << 31) || c.H * c.W * c.Cin * 2 >= (1LL << 40)) return false;
+    if (c.R * c.S >= (1LL << 15) || c.Cout >= (1LL << 31)) return false;
+    return true;
+}
+
+int umma_max_stages(int tile_n, int smem_limit) {
+    const int stage = tdx::kABytes + tile_n * 128;
+    int s = (smem_limit - kStaticSmemReserve - 1024) / stage;
+    return std::min(s, tdx::kMaxStages);
+}
+
+int tmem_cols_for(int bn) {
+    int c = 32;
+    while (c < 2 * bn) c *= 2;
+    return c;
+}
+
+// Static feasibility of a fully specified tensor-core configuration (the search-space constraints).
+// Returns 0 when feasible, else a short reason.
+const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num_kb, int smem_limit, bool conv) {
+    if (c.tile_m != 128) return "tile_m must be 128";
+    if (c.tile_k != 64) return "tile_k must be 64";
+    if (c.cta_pair != 1) return "cta_pair must be 1";
+    if (c.store_mode != 0) return "store_mode must be 0";
+    if (c.tile_n < 32 || c.tile_n > 256 || c.tile_n % 32) return "tile_n must be a multiple of 32 in [32, 256]";
+    if (b_mn_major && c.tile_n % 64) return "tile_n must be a multiple of 64 when B is read N-major";
+    if (c.stages < 2 || c.stages > umma_max_stages(c.tile_n, smem_limit)) return "stages outside the shared-memory budget";
+    if (c.split_k < 1) return "split_k must be >= 1";
+    if (conv && c.split_k != 1) return "conv has no split-K";
+    if (c.split_k > 1) {
+        const int64_t per = ceil_div(num_kb, c.split_k);
+        if ((c.split_k - 1) * per >= num_kb) return "split_k leaves an empty K slice";
+    }
+    if (c.raster < 0) return "raster must be >= 0";
+    return nullptr;
+}
+
+bool patch_ok(int bw, int bh) {
+    const int a = bw * bh;
+    return bw >= 8 && bw <= 128 && bh >= 1 && a <= 128 && (a & (a - 1)) == 0 && (bw & (bw - 1)) == 0;
+}
+
+void choose_patch(int64_t P, int64_t Q, int* bw_out, int* bh_out) {
+    int64_t best_cost = -1;
+    int best_bw = 8, best_bh = 1;
+    for (int bw = 8; bw <= 128; bw *= 2) {
+        for (int bh = 1; bw * bh <= 128; bh *= 2) {
+            const int64_t cost = ceil_div(Q, bw) * bw * ceil_div(P, bh) * bh;
+            const bool better = best_cost < 0 || cost < best_cost ||
+                                (cost == best_cost && (bw * bh > best_bw * best_bh ||
+                                                       (bw * bh == best_bw * best_bh && bw > best_bw)));
+            if (better) { best_cost = cost; best_bw = bw; best_bh = bh; }
+        }
+    }
+    *bw_out = best_bw;
+    *bh_out = best_bh;
+}
+
+// Heuristic default (used when neither the caller nor the tuning cache gives a configuration).
+void default_umma_config(int64_t tiles_m, int64_t N, int64_t num_kb, bool b_mn_major, int sm_count, int smem_limit,
+                         bool allow_split, tdx_config* c) {
+    std::memset(c, 0, sizeof *c);
+    c->kernel = TDX_KERNEL_UMMA;
+    c->tile_m = 128;
+    c->tile_k = 64;
+    c->cta_pair = 1;
+    c->store_mode = 0;
+    c->split_k = 1;
+    const int min_bn = b_mn_major ? 64 : 32;
+    int bn = 0;
+    const int64_t n_cap = ceil_div(N, min_bn) * min_bn;   // narrowest tile that covers N at once
+    for (int cand : {256, 128, 64, 32}) {
+        if (cand < min_bn) continue;
+        if (cand > n_cap && cand / 2 >= n_cap) continue;  // a narrower tile covers N just as well
+        if (tiles_m * ceil_div(N, cand) >= sm_count) { bn = cand; break; }
+    }
+    if (bn == 0) {
+        bn = N > 64 ? 128 : (N > 32 ? 64 : min_bn);
+        const int64_t tiles = tiles_m * ceil_div(N, bn);
+        if (allow_split && tiles < sm_count) {
+            int64_t s = std::min<int64_t>(ceil_div(sm_count, tiles), std::max<int64_t>(1, num_kb / 4));
+            s = std::min<int64_t>(s, 32);
+            while (s > 1 && (s - 1) * ceil_div(num_kb, s) >= num_kb) --s;
+            c->split_k = static_cast<int>(std::max<int64_t>(1, s));
+        }
+    }
+    c->tile_n = bn;
+    c->stages = std::max(2, umma_max_stages(bn, smem_limit));
+    c->raster = 8;
+}
+
+// ------------------------------------------------------------------ launches
+int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensorMap& mb, const UmmaParams& p,
+                cudaStream_t st) {
+    const long long items = static_cast<long long>(p.tiles_m) * p.tiles_n * p.split_k;
+    const int grid = static_cast<int>(std::min<long long>(items, ctx->sm_count));
+    const size_t smem = static_cast<size_t>(p.stages) * (tdx::kABytes + p.bn * 128) + 1024;
+    if (conv)
+        tdx::umma_contract_kernel<true><<<grid, tdx::kUmmaThreads, smem, st>>>(ma, mb, p);
+    else
+        tdx::umma_contract_kernel<false><<<grid, tdx::kUmmaThreads, smem, st>>>(ma, mb, p);
+    TDX_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return TDX_OK;
+}
+
+int ensure_ws(DeviceCtx* ctx, size_t bytes, void** out) {
+    if (ctx->ws_bytes < bytes) {
+        if (ctx->ws) TDX_CUDA(cudaFree(ctx->ws));
+        ctx->ws = nullptr;
+        ctx->ws_bytes = 0;
+        TDX_CUDA(cudaMalloc(&ctx->ws, bytes));
+        ctx->ws_bytes = bytes;
+    }
+    *out = ctx->ws;
+    return TDX_OK;
+}
+
+int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
+                  const tdx_config& cfg, void* ws, size_t ws_bytes, bool internal_ws, cudaStream_t st) {
+    const int64_t num_kb = ceil_div(g.K, 64);
+    UmmaParams p;
+    std::memset(&p, 0, sizeof p);
+    p.M = static_cast<int>(g.M);
+    p.N = static_cast<int>(g.N);
+    p.num_kb = static_cast<int>(num_kb);
+    p.tiles_m = static_cast<int>(ceil_div(g.M, 128));
+    p.tiles_n = static_cast<int>(ceil_div(g.N, cfg.tile_n));
+    p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
+    p.split_k = cfg.split_k;
+    p.kb_per_split = static_cast<int>(ceil_div(num_kb, cfg.split_k));
+    p.bn = cfg.tile_n;
+    p.stages = cfg.stages;
+    p.tmem_cols = tmem_cols_for(cfg.tile_n);
+    p.a_mn_major = g.transA ? 1 : 0;   // A stored K x M: M contiguous
+    p.b_mn_major = g.transB ? 0 : 1;   // B stored K x N: N contiguous
+    p.alpha = alpha;
+    p.bias = nullptr;
+    p.relu = 0;
+    p.C = static_cast<__nv_bfloat16*>(C);
+    p.ldc = g.N;
+    p.status = ctx->status_ptr;
+    p.vec_store = (g.N % 8 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+
+    if (cfg.split_k > 1) {
+        const size_t need = static_cast<size_t>(cfg.split_k) * g.M * g.N * sizeof(float);
+        if (internal_ws) {
+            int rc = ensure_ws(ctx, need, &ws);
+            if (rc) return rc;
+        } else if (ws == nullptr || ws_bytes < need || reinterpret_cast<uintptr_t>(ws) % 256) {
+            return fail(TDX_ERR_WORKSPACE, "split_k=%d needs %zu bytes of 256-byte aligned workspace", cfg.split_k, need);
+        }
+        p.partial = static_cast<float*>(ws);
+    }
+
+    CUtensorMap ma, mb;
+    int rc;
+    if (p.a_mn_major) {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.M), static_cast<uint64_t>(g.K)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.M) * 2};
+        uint32_t box[2] = {64, 64};
+        rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
+    } else {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.M)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
+        uint32_t box[2] = {64, 128};
+        rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
+    }
+    if (rc) return rc;
+    if (p.b_mn_major) {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.K)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
+        uint32_t box[2] = {64, 64};
+        rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
+    } else {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.N)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
+        uint32_t box[2] = {64, static_cast<uint32_t>(cfg.tile_n)};
+        rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
+    }
+    if (rc) return rc;
+
+    rc = launch_umma(ctx, false, ma, mb, p, st);
+    if (rc) return rc;
+    if (cfg.split_k > 1) {
+        const long long MN = static_cast<long long>(g.M) * g.N;
+        const int vec8 = p.vec_store ? 1 : 0;
+        const long long work = vec8 ? MN / 8 : MN;
+        const int grid = static_cast<int>(std::min<long long>(ceil_div(work, 256), 148LL * 16));
+        tdx::splitk_reduce_kernel<<<std::max(grid, 1), 256, 0, st>>>(MN, static_cast<int>(g.N), cfg.split_k, p.partial,
+                                                                     alpha, nullptr, 0, p.C, vec8);
+        TDX_CUDA(cudaGetLastError());
+        g_launches.fetch_add(1);
+    }
+    return TDX_OK;
+}
+
+int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const void* w, const float* bias, int relu,
+                  void* y, const tdx_config& cfg, cudaStream_t st) {
+    const int cchunks = static_cast<int>(ceil_div(c.Cin, 64));
+    UmmaParams p;
+    std::memset(&p, 0, sizeof p);
+    p.bw = cfg.patch_w;
+    p.bh = cfg.patch_h;
+    p.nb = 128 / (p.bw * p.bh);
+    p.patches_w = static_cast<int>(ceil_div(c.Q, p.bw));
+    p.patches_h = static_cast<int>(ceil_div(c.P, p.bh));
+    const int64_t total_patches = c.N * p.patches_w * p.patches_h;
+    p.M = static_cast<int>(c.N * c.P * c.Q);
+    p.N = static_cast<int>(c.Cout);
+    p.num_kb = static_cast<int>(c.R * c.S * cchunks);
+    p.tiles_m = static_cast<int>(ceil_div(total_patches, p.nb));
+    p.tiles_n = static_cast<int>(ceil_div(c.Cout, cfg.tile_n));
+    p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
+    p.split_k = 1;
+    p.kb_per_split = p.num_kb;
+    p.bn = cfg.tile_n;
+    p.stages = cfg.stages;
+    p.tmem_cols = tmem_cols_for(cfg.tile_n);
+    p.a_mn_major = 0;
+    p.b_mn_major = 0;
+    p.alpha = 1.0f;
+    p.bias = bias;
+    p.relu = relu;
+    p.C = static_cast<__nv_bfloat16*>(y);
+    p.ldc = c.Cout;
+    p.vec_store = (c.Cout % 8 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
+    p.P = static_cast<int>(c.P);
+    p.Q = static_cast<int>(c.Q);
+    p.Nimg = static_cast<int>(c.N);
+    p.S = static_cast<int>(c.S);
+    p.pad = c.pad;
+    p.cchunks = cchunks;
+    p.status = ctx->status_ptr;
+
+    CUtensorMap ma, mb;
+    {
+        uint64_t dims[4] = {static_cast<uint64_t>(c.Cin), static_cast<uint64_t>(c.W), static_cast<uint64_t>(c.H),
+                            static_cast<uint64_t>(c.N)};
+        uint64_t str[3] = {static_cast<uint64_t>(c.Cin) * 2, static_cast<uint64_t>(c.W * c.Cin) * 2,
+                           static_cast<uint64_t>(c.H * c.W * c.Cin) * 2};
+        uint32_t box[4] = {64, static_cast<uint32_t>(p.bw), static_cast<uint32_t>(p.bh), 1};
+        int rc = get_tensor_map(ctx, x, 4, dims, str, box, &ma);
+        if (rc) return rc;
+    }
+    {
+        uint64_t dims[3] = {static_cast<uint64_t>(c.Cin), static_cast<uint64_t>(c.R * c.S),
+                            static_cast<uint64_t>(c.Cout)};
+        uint64_t str[2] = {static_cast<uint64_t>(c.Cin) * 2, static_cast<uint64_t>(c.R * c.S * c.Cin) * 2};
+        uint32_t box[3] = {64, 1, static_cast<uint32_t>(cfg.tile_n)};
+        int rc = get_tensor_map(ctx, w, 3, dims, str, box, &mb);
+        if (rc) return rc;
+    }
+    return launch_umma(ctx, true, ma, mb, p, st);
+}
+
+void gemm_strides(const GemmProblem& g, long long* sa_i, long long* sa_k, long long* sb_k, long long* sb_j) {
+    *sa_i = g.transA ? 1 : g.K;
+    *sa_k = g.transA ? g.M : 1;
+    *sb_k = g.transB ? 1 : g.N;
+    *sb_j = g.transB ? g.K : 1;
+}
+
+int run_gemm_simt_f32(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
+                      cudaStream_t st) {
+    if (g.M >= (1LL << 31) || g.N >= (1LL << 31) || g.K >= (1LL << 31))
+        return fail(TDX_ERR_UNSUPPORTED, "fp32 tiled GEMM needs dimensions below 2^31");
+    long long sa_i, sa_k, sb_k, sb_j;
+    gemm_strides(g, &sa_i, &sa_k, &sb_k, &sb_j);
+    const float* a = static_cast<const float*>(A);
+    const float* b = static_cast<const float*>(B);
+    float* c = static_cast<float*>(C);
+    if (ceil_div(g.M, 64) * ceil_div(g.N, 64) >= ctx->sm_count) {
+        dim3 grid(static_cast<unsigned>(ceil_div(g.N, 64)), static_cast<unsigned>(ceil_div(g.M, 64)));
+        tdx::sgemm_tiled_kernel<64, 64, 16, 4, 4><<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k,
+                                                                       sb_j, alpha, a, b, c);
+    } else {
+        dim3 grid(static_cast<unsigned>(ceil_div(g.N, 32)), static_cast<unsigned>(ceil_div(g.M, 32)));
+        tdx::sgemm_tiled_kernel<32, 32, 16, 2, 2><<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k,
+                                                                       sb_j, alpha, a, b, c);
+    }
+    TDX_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return TDX_OK;
+}
+
+int run_gemm_generic(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
+                     cudaStream_t st) {
+    long long sa_i, sa_k, sb_k, sb_j;
+    gemm_strides(g, &sa_i, &sa_k, &sb_k, &sb_j);
+    const long long total = g.M * g.N;
+    const int grid = static_cast<int>(std::min<long long>(ceil_div(total, 256), static_cast<long long>(ctx->sm_count) * 32));
+    if (g.dtype == TDX_F32)
+        tdx::gemm_generic_kernel<float, float><<<grid, 256, 0, st>>>(g.M, g.N, g.K, sa_i, sa_k, sb_k, sb_j, alpha,
+                                                                    static_cast<const float*>(A),
+                                                                    static_cast<const float*>(B), static_cast<float*>(C));
+    else
+        tdx::gemm_generic_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
+            g.M, g.N, g.K, sa_i, sa_k, sb_k, sb_j, alpha, static_cast<const __nv_bfloat16*>(A),
+            static_cast<const __nv_bfloat16*>(B), static_cast<__nv_bfloat16*>(C));
+    TDX_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return TDX_OK;
+}
+
+int run_conv_generic(DeviceCtx* ctx, const ConvProblem& c, const void* x, const void* w, const float* bias, int relu,
+                     void* y, cudaStream_t st) {
+    if (c.N >= (1LL << 31) || c.H >= (1LL << 31) || c.W >= (1LL << 31) || c.Cin >= (1LL << 31) ||
+        c.Cout >= (1LL << 31) || c.R >= (1LL << 31) || c.S >= (1LL << 31))
+        return fail(TDX_ERR_UNSUPPORTED, "conv dimensions must be below 2^31");
+    const long long total = c.N * c.P * c.Q * c.Cout;
+    const int grid = static_cast<int>(std::min<long long>(ceil_div(total, 256), static_cast<long long>(ctx->sm_count) * 32));
+    if (c.dtype == TDX_F32)
+        tdx::conv2d_generic_kernel<float, float><<<grid, 256, 0, st>>>(
+            (int)c.N, (int)c.H, (int)c.W, (int)c.Cin, (int)c.Cout, (int)c.R, (int)c.S, c.pad, c.stride, (int)c.P,
+            (int)c.Q, static_cast<const float*>(x), static_cast<const float*>(w), bias, relu, static_cast<float*>(y));
+    else
+        tdx::conv2d_generic_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
+            (int)c.N, (int)c.H, (int)c.W, (int)c.Cin, (int)c.Cout, (int)c.R, (int)c.S, c.pad, c.stride, (int)c.P,
+            (int)c.Q, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w), bias, relu,
+            static_cast<__nv_bfloat16*>(y));
+    TDX_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return TDX_OK;
+}
+
+// ------------------------------------------------------------------ validation
+int validate_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const void* A, const void* B,
+                  const void* C, bool need_ptrs) {
+    if (M < 0 || N < 0 || K < 0) return fail(TDX_ERR_INVALID_ARG, "negative dimension (M=%lld N=%lld K=%lld)", (long long)M, (long long)N, (long long)K);
+    if ((transA != 0 && transA != 1) || (transB != 0 && transB != 1)) return fail(TDX_ERR_INVALID_ARG, "transA/transB must be 0 or 1");
+    if (dtype != TDX_F32 && dtype != TDX_BF16) return fail(TDX_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    if (need_ptrs && M > 0 && N > 0) {
+        if (C == nullptr) return fail(TDX_ERR_INVALID_ARG, "C is NULL");
+        if (K > 0 && (A == nullptr || B == nullptr)) return fail(TDX_ERR_INVALID_ARG, "A or B is NULL");
+        const uintptr_t el = dtype == TDX_F32 ? 4 : 2;
+        if (reinterpret_cast<uintptr_t>(A) % el || reinterpret_cast<uintptr_t>(B) % el || reinterpret_cast<uintptr_t>(C) % el)
+            return fail(TDX_ERR_ALIGNMENT, "pointer not aligned to its element size");
+    }
+    return TDX_OK;
+}
+
+int validate_conv(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
+                  int stride, int dtype, const void* x, const void* w, const void* y, int relu, bool need_ptrs,
+                  ConvProblem* out) {
+    if (N < 0 || H < 0 || W < 0 || Cout < 0 || pad < 0) return fail(TDX_ERR_INVALID_ARG, "negative dimension or pad");
+    if (Cin <= 0 || R <= 0 || S <= 0) return fail(TDX_ERR_INVALID_ARG, "Cin, R and S must be positive");
+    if (stride < 1) return fail(TDX_ERR_INVALID_ARG, "stride must be >= 1");
+    if (dtype != TDX_F32 && dtype != TDX_BF16) return fail(TDX_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    if (relu != 0 && relu != 1) return fail(TDX_ERR_INVALID_ARG, "relu must be 0 or 1");
+    ConvProblem c{N, H, W, Cin, Cout, R, S, pad, stride, dtype, conv_out_dim(H, R, pad, stride), conv_out_dim(W, S, pad, stride)};
+    if (need_ptrs && N > 0 && Cout > 0 && c.P > 0 && c.Q > 0) {
+        if (x == nullptr || w == nullptr || y == nullptr) return fail(TDX_ERR_INVALID_ARG, "x, w or y is NULL");
+        const uintptr_t el = dtype == TDX_F32 ? 4 : 2;
+        if (reinterpret_cast<uintptr_t>(x) % el || reinterpret_cast<uintptr_t>(w) % el || reinterpret_cast<uintptr_t>(y) % el)
+            return fail(TDX_ERR_ALIGNMENT, "pointer not aligned to its element size");
+    }
+    *out = c;
+    return TDX_OK;
+}
+
+// Fill the zero fields of a (possibly partial) GEMM config and check it.  smem_limit / sm_count come from the
+// device when there is one, else from the sm_100 defaults, so the search space can be listed without a GPU.
+int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_count, int smem_limit, tdx_config* out) {
+    const bool layout_ok = gemm_umma_layout_ok(g);
+    tdx_config c;
+    std::memset(&c, 0, sizeof c);
+    if (user) c = *user;
+    if (c.kernel < 0 || c.kernel > 3) return fail(TDX_ERR_CONFIG, "unknown kernel %d", c.kernel);
+    bool from_cache = false;
+    if (c.kernel == TDX_KERNEL_AUTO) {
+        if (!user) {
+            tdx_config cached;
+            if (tune_lookup(gemm_key(g.M, g.N, g.K, g.transA, g.transB, g.dtype), &cached)) { c = cached; from_cache = true; }
+        }
+        if (!from_cache) c.kernel = g.dtype == TDX_F32 ? TDX_KERNEL_SIMT : (layout_ok ? TDX_KERNEL_UMMA : TDX_KERNEL_GENERIC);
+    }
+    if (c.kernel == TDX_KERNEL_SIMT) {
+        if (g.dtype != TDX_F32) return fail(TDX_ERR_CONFIG, "the tiled SIMT kernel is fp32 only");
+        *out = c;
+        return TDX_OK;
+    }
+    if (c.kernel == TDX_KERNEL_GENERIC) { *out = c; return TDX_OK; }
+    // tensor-core path
+    if (g.dtype != TDX_BF16) return fail(TDX_ERR_CONFIG, "the tensor-core kernel is bf16 only");
+    if (!layout_ok) return fail(TDX_ERR_ALIGNMENT, "tensor-core path needs 16-byte aligned row pitches (contiguous dims %% 8 == 0)");
+    const int64_t num_kb = ceil_div(g.K, 64);
+    const bool b_mn = g.transB == 0;
+    tdx_config d;
+    default_umma_config(ceil_div(g.M, 128), g.N, num_kb, b_mn, sm_count, smem_limit, true, &d);
+    if (c.tile_m == 0) c.tile_m = d.tile_m;
+    if (c.tile_k == 0) c.tile_k = d.tile_k;
+    if (c.cta_pair == 0) c.cta_pair = d.cta_pair;
+    if (c.tile_n == 0) c.tile_n = d.tile_n;
+    if (c.split_k == 0) c.split_k = (user && user->tile_n != 0 && user->tile_n != d.tile_n) ? 1 : d.split_k;
+    if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_n, smem_limit));
+    if (!user && !from_cache) c.raster = d.raster;
+    const char* why = umma_config_reason(c, b_mn, num_kb, smem_limit, false);
+    if (why) return fail(TDX_ERR_CONFIG, "infeasible config: %s", why);
+    *out = c;
+    return TDX_OK;
+}
+
+int resolve_conv_config(const ConvProblem& cp, const tdx_config* user, int sm_count, int smem_limit, tdx_config* out) {
+    const bool layout_ok = conv_umma_layout_ok(cp);
+    tdx_config c;
+    std::memset(&c, 0, sizeof c);
+    if (user) c = *user;
+    if (c.kernel < 0 || c.kernel > 3) return fail(TDX_ERR_CONFIG, "unknown kernel %d", c.kernel);
+    if (c.kernel == TDX_KERNEL_SIMT) return fail(TDX_ERR_CONFIG, "conv has no tiled SIMT kernel");
+    bool from_cache = false;
+    if (c.kernel == TDX_KERNEL_AUTO) {
+        if (!user) {
+            tdx_config cached;
+            if (tune_lookup(conv_key(cp.N, cp.H, cp.W, cp.Cin, cp.Cout, cp.R, cp.S, cp.pad, cp.stride, cp.dtype), &cached)) { c = cached; from_cache = true; }
+        }
+        if (!from_cache) c.kernel = layout_ok ? TDX_KERNEL_UMMA : TDX_KERNEL_GENERIC;
+    }
+    if (c.kernel == TDX_KERNEL_GENERIC) { *out = c; return TDX_OK; }
+    if (cp.dtype != TDX_BF16) return fail(TDX_ERR_CONFIG, "the tensor-core kernel is bf16 only");
+    if (!layout_ok) return fail(TDX_ERR_ALIGNMENT, "tensor-core conv needs stride 1 and Cin %% 8 == 0");
+    if (c.patch_w == 0 && c.patch_h == 0) choose_patch(cp.P, cp.Q, &c.patch_w, &c.patch_h);
+    if (!patch_ok(c.patch_w, c.patch_h)) return fail(TDX_ERR_CONFIG, "infeasible config: patch %dx%d", c.patch_w, c.patch_h);
+    const int nb = 128 / (c.patch_w * c.patch_h);
+    const int64_t tiles_m = ceil_div(cp.N * ceil_div(cp.Q, c.patch_w) * ceil_div(cp.P, c.patch_h), nb);
+    const int64_t num_kb = cp.R * cp.S * ceil_div(cp.Cin, 64);
+    tdx_config d;
+    default_umma_config(tiles_m, cp.Cout, num_kb, false, sm_count, smem_limit, false, &d);
+    if (c.tile_m == 0) c.tile_m = d.tile_m;
+    if (c.tile_k == 0) c.tile_k = d.tile_k;
+    if (c.cta_pair == 0) c.cta_pair = d.cta_pair;
+    if (c.tile_n == 0) c.tile_n = d.tile_n;
+    if (c.split_k == 0) c.split_k = 1;
+    if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_n, smem_limit));
+    if (!user && !from_cache) c.raster = d.raster;
+    const char* why = umma_config_reason(c, false, num_kb, smem_limit, true);
+    if (why) return fail(TDX_ERR_CONFIG, "infeasible config: %s", why);
+    *out = c;
+    return TDX_OK;
+}
+
+void device_limits(int* sm_count, int* smem_limit) {
+    *sm_count = kDefaultSmCount;
+    *smem_limit = kSmemLimitDefault;
+    int dev;
+    if (cudaGetDevice(&dev) == cudaSuccess) {
+        std::lock_guard<std::mutex> lk(g_mu);
+        auto it = g_ctx.find(dev);
+        if (it != g_ctx.end()) { *sm_count = it->second.sm_count; *smem_limit = it->second.smem_optin; }
+    } else {
+        cudaGetLastError();
+    }
+}
+
+int gemm_dispatch(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype, const void* A,
+                  const void* B, void* C, void* stream, const tdx_config* cfg, void* ws, size_t ws_bytes,
+                  bool internal_ws) {
+    int rc = validate_gemm(M, N, K, transA, transB, dtype, A, B, C, true);
+    if (rc) return rc;
+    if (M == 0 || N == 0) return TDX_OK;
+    GemmProblem g{M, N, K, transA, transB, dtype};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (K == 0) {
+        DeviceCtx* ctx0;
+        rc = get_ctx(&ctx0);
+        if (rc) return rc;
+        TDX_CUDA(cudaMemsetAsync(C, 0, static_cast<size_t>(M) * N * (dtype == TDX_F32 ? 4 : 2), st));
+        return TDX_OK;
+    }
+    int sm_count, smem_limit;
+    device_limits(&sm_count, &smem_limit);
+    // configuration errors are reported before anything touches the device
+    tdx_config pre;
+    if (cfg) {
+        rc = resolve_gemm_config(g, cfg, sm_count, smem_limit, &pre);
+        if (rc) return rc;
+    }
+    DeviceCtx* ctx;
+    rc = get_ctx(&ctx);
+    if (rc) return rc;
+    tdx_config c;
+    rc = resolve_gemm_config(g, cfg, ctx->sm_count, ctx->smem_optin, &c);
+    if (rc) return rc;
+    switch (c.kernel) {
+        case TDX_KERNEL_SIMT: return run_gemm_simt_f32(ctx, g, alpha, A, B, C, st);
+        case TDX_KERNEL_GENERIC: return run_gemm_generic(ctx, g, alpha, A, B, C, st);
+        default:
+            if (reinterpret_cast<uintptr_t>(A) % 16 || reinterpret_cast<uintptr_t>(B) % 16) {
+                if (cfg && cfg->kernel == TDX_KERNEL_UMMA)
+                    return fail(TDX_ERR_ALIGNMENT, "tensor-core path needs 16-byte aligned A and B");
+                return run_gemm_generic(ctx, g, alpha, A, B, C, st);
+            }
+            return run_gemm_umma(ctx, g, alpha, A, B, C, c, ws, ws_bytes, internal_ws, st);
+    }
+}
+
+int conv_dispatch(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad, int stride,
+                  int dtype, const void* x, const void* w, const float* bias, int relu, void* y, void* stream,
+                  const tdx_config* cfg) {
+    ConvProblem cp;
+    int rc = validate_conv(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, y, relu, true, &cp);
+    if (rc) return rc;
+    if (N == 0 || Cout == 0 || cp.P == 0 || cp.Q == 0) return TDX_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int sm_count, smem_limit;
+    device_limits(&sm_count, &smem_limit);
+    tdx_config pre;
+    if (cfg) {
+        rc = resolve_conv_config(cp, cfg, sm_count, smem_limit, &pre);
+        if (rc) return rc;
+    }
+    DeviceCtx* ctx;
+    rc = get_ctx(&ctx);
+    if (rc) return rc;
+    tdx_config c;
+    rc = resolve_conv_config(cp, cfg, ctx->sm_count, ctx->smem_optin, &c);
+    if (rc) return rc;
+    if (c.kernel == TDX_KERNEL_GENERIC) return run_conv_generic(ctx, cp, x, w, bias, relu, y, st);
+    if (reinterpret_cast<uintptr_t>(x) % 16 || reinterpret_cast<uintptr_t>(w) % 16) {
+        if (cfg && cfg->kernel == TDX_KERNEL_UMMA) return fail(TDX_ERR_ALIGNMENT, "tensor-core path needs 16-byte aligned x and w");
+        return run_conv_generic(ctx, cp, x, w, bias, relu, y, st);
+    }
+    return run_conv_umma(ctx, cp, x, w, bias, relu, y, c, st);
+}
+
+// ------------------------------------------------------------------ search space
+void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int sm_count, int smem_limit, bool conv,
+                     std::vector<tdx_config>* out) {
+    for (int bn : {256, 128, 64, 32}) {
+        if (b_mn && bn % 64) continue;
+        if (bn > 32 && bn / 2 >= N + 31) continue;   // a tile more than twice as wide as the problem only wastes work
+        const int max_st = umma_max_stages(bn, smem_limit);
+        std::vector<int> stage_opts;
+        stage_opts.push_back(max_st);
+        if (max_st - 2 >= 3) stage_opts.push_back(max_st - 2);
+        const int64_t tiles = tiles_m * ceil_div(N, bn);
+        std::vector<int> splits{1};
+        if (!conv && tiles < 2LL * sm_count)
+            for (int s : {2, 3, 4, 6, 8, 16})
+                if (num_kb / s >= 2 && tiles * s <= 4LL * sm_count) splits.push_back(s);
+        for (int st : stage_opts)
+            for (int sk : splits)
+                for (int raster : {0, 8, 2}) {
+                    if (raster != 0 && tiles_m <= raster) continue;
+                    tdx_config c;
+                    std::memset(&c, 0, sizeof c);
+                    c.kernel = TDX_KERNEL_UMMA;
+                    c.tile_m = 128; c.tile_n = bn; c.tile_k = 64; c.stages = st; c.cta_pair = 1;
+                    c.split_k = sk; c.store_mode = 0; c.raster = raster;
+                    if (umma_config_reason(c, b_mn, num_kb, smem_limit, conv) == nullptr) out->push_back(c);
+                }
+    }
+}
+
+int write_configs(const std::vector<tdx_config>& v, tdx_config* out, int cap, int* n) {
+    if (n) *n = static_cast<int>(v.size());
+    if (out)
+        for (int i = 0; i < cap && i < static_cast<int>(v.size()); ++i) out[i] = v[i];
+    return TDX_OK;
+}
+
+int enum_gemm(const GemmProblem& g, int sm_count, int smem_limit, std::vector<tdx_config>* v) {
+    if (g.dtype == TDX_F32) {
+        tdx_config c;
+        std::memset(&c, 0, sizeof c);
+        c.kernel = TDX_KERNEL_SIMT;
+        v->push_back(c);
+        return TDX_OK;
+    }
+    if (!gemm_umma_layout_ok(g)) {
+        tdx_config c;
+        std::memset(&c, 0, sizeof c);
+        c.kernel = TDX_KERNEL_GENERIC;
+        v->push_back(c);
+        return TDX_OK;
+    }
+    enum_umma_space(g.transB == 0, ceil_div(g.M, 128), g.N, ceil_div(g.K, 64), sm_count, smem_limit, false, v);
+    return TDX_OK;
+}
+
+int enum_conv(const ConvProblem& cp, int sm_count, int smem_limit, std::vector<tdx_config>* v) {
+    if (!conv_umma_layout_ok(cp)) {
+        tdx_config c;
+        std::memset(&c, 0, sizeof c);
+        c.kernel = TDX_KERNEL_GENERIC;
+        v->push_back(c);
+        return TDX_OK;
+    }
+    // patch shapes: every shape whose padded area is within 15 % of the best one
+    int bbw, bbh;
+    choose_patch(cp.P, cp.Q, &bbw, &bbh);
+    const int64_t best_cost = ceil_div(cp.Q, bbw) * bbw * ceil_div(cp.P, bbh) * bbh;
+    for (int bw = 8; bw <= 128; bw *= 2)
+        for (int bh = 1; bw * bh <= 128; bh *= 2) {
+            if (bw * bh < 32 && !(bw == bbw && bh == bbh)) continue;
+            const int64_t cost = ceil_div(cp.Q, bw) * bw * ceil_div(cp.P, bh) * bh;
+            if (cost * 100 > best_cost * 115) continue;
+            const int nb = 128 / (bw * bh);
+            const int64_t tiles_m = ceil_div(cp.N * ceil_div(cp.Q, bw) * ceil_div(cp.P, bh), nb);
+            std::vector<tdx_config> sub;
+            enum_umma_space(false, tiles_m, cp.Cout, cp.R * cp.S * ceil_div(cp.Cin, 64), sm_count, smem_limit, true, &sub);
+            for (auto& c : sub) { c.patch_w = bw; c.patch_h = bh; v->push_back(c); }
+        }
+    return TDX_OK;
+}
+
+struct ScratchGuard {
+    std::vector<void*> ptrs;
+    ~ScratchGuard() { for (void* p : ptrs) if (p) cudaFree(p); }
+    int alloc(void** p, size_t bytes) {
+        cudaError_t e = cudaMalloc(p, std::max<size_t>(bytes, 256));
+        if (e != cudaSuccess) { cudaGetLastError(); return fail(TDX_ERR_CUDA, "cudaMalloc(%zu): %s", bytes, cudaGetErrorString(e)); }
+        ptrs.push_back(*p);
+        return TDX_OK;
+    }
+};
+
+int fill_scratch(void* p, size_t elems, uint32_t seed, cudaStream_t st) {
+    tdx::fill_pattern_bf16_kernel<<<1184, 256, 0, st>>>(static_cast<__nv_bfloat16*>(p), static_cast<long long>(elems), seed);
+    TDX_CUDA(cudaGetLastError());
+    return TDX_OK;
+}
+
+template <typename Launch>
+int time_candidates(const std::vector<tdx_config>& cands, int iters, cudaStream_t st, Launch&& launch, tdx_config* best,
+                    float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried) {
+    cudaEvent_t e0, e1;
+    TDX_CUDA(cudaEventCreate(&e0));
+    TDX_CUDA(cudaEventCreate(&e1));
+    float best_t = -1.0f;
+    int count = 0;
+    int rc = TDX_OK;
+    for (const tdx_config& c : cands) {
+        rc = launch(c);              // warm-up (also validates the configuration)
+        if (rc == TDX_ERR_CONFIG || rc == TDX_ERR_WORKSPACE) { rc = TDX_OK; continue; }
+        if (rc) break;
+        rc = launch(c);
+        if (rc) break;
+        cudaEventRecord(e0, st);
+        for (int i = 0; i < iters && rc == TDX_OK; ++i) rc = launch(c);
+        cudaEventRecord(e1, st);
+        if (rc) break;
+        cudaError_t e = cudaEventSynchronize(e1);
+        if (e != cudaSuccess) { rc = fail(TDX_ERR_CUDA, "tuning launch failed: %s", cudaGetErrorString(e)); break; }
+        float ms = 0.0f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        const float us = ms * 1000.0f / iters;
+        if (tried && tried_us && count < cap) { tried[count] = c; tried_us[count] = us; }
+        ++count;
+        if (best_t < 0 || us < best_t) { best_t = us; *best = c; }
+    }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (rc) return rc;
+    if (best_t < 0) return fail(TDX_ERR_UNSUPPORTED, "no feasible configuration");
+    if (best_us) *best_us = best_t;
+    if (n_tried) *n_tried = count;
+    return TDX_OK;
+}
+
+int ensure_staging(DeviceCtx* ctx, int slot, size_t bytes, void** out) {
+    bytes = std::max<size_t>(bytes, 256);
+    if (ctx->staging_bytes[slot] < bytes) {
+        if (ctx->staging[slot]) TDX_CUDA(cudaFree(ctx->staging[slot]));
+        ctx->staging[slot] = nullptr;
+        ctx->staging_bytes[slot] = 0;
+        TDX_CUDA(cudaMalloc(&ctx->staging[slot], bytes));
+        ctx->staging_bytes[slot] = bytes;
+    }
+    *out = ctx->staging[slot];
+    return TDX_OK;
+}
+
+}  // namespace
+
+// ====================================================================== C ABI
+extern "C" {
+
+int tdx_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype, const void* A,
+             const void* B, void* C, void* stream) {
+    return gemm_dispatch(M, N, K, transA, transB, alpha, dtype, A, B, C, stream, nullptr, nullptr, 0, true);
+}
+
+int tdx_gemm_ex(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype, const void* A,
+                const void* B, void* C, void* stream, const tdx_config* cfg, void* workspace, size_t workspace_bytes) {
+    // the library's own workspace serves every split-K it chose itself
+    const bool internal = (workspace == nullptr) && (cfg == nullptr || cfg->split_k == 0);
+    return gemm_dispatch(M, N, K, transA, transB, alpha, dtype, A, B, C, stream, cfg, workspace, workspace_bytes, internal);
+}
+
+int tdx_gemm_workspace_size(int64_t M, int64_t N, int64_t K, int dtype, const tdx_config* cfg, size_t* bytes) {
+    if (bytes == nullptr) return fail(TDX_ERR_INVALID_ARG, "bytes is NULL");
+    if (M < 0 || N < 0 || K < 0) return fail(TDX_ERR_INVALID_ARG, "negative dimension");
+    if (dtype != TDX_F32 && dtype != TDX_BF16) return fail(TDX_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    const int split = cfg ? std::max(cfg->split_k, 1) : 1;
+    *bytes = split > 1 ? static_cast<size_t>(split) * M * N * sizeof(float) : 0;
+    return TDX_OK;
+}
+
+int tdx_conv2d_bias_relu(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
+                         int stride, int dtype, const void* x, const void* w, const float* bias, int relu, void* y,
+                         void* stream) {
+    return conv_dispatch(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, relu, y, stream, nullptr);
+}
+
+int tdx_conv2d_bias_relu_ex(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
+                            int stride, int dtype, const void* x, const void* w, const float* bias, int relu, void* y,
+                            void* stream, const tdx_config* cfg) {
+    return conv_dispatch(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, relu, y, stream, cfg);
+}
+
+int tdx_gemm_host(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype, const void* A_host,
+                  const void* B_host, void* C_host, void* stream) {
+    int rc = validate_gemm(M, N, K, transA, transB, dtype, A_host, B_host, C_host, true);
+    if (rc) return rc;
+    if (M == 0 || N == 0) return TDX_OK;
+    DeviceCtx* ctx;
+    rc = get_ctx(&ctx);
+    if (rc) return rc;
+    const size_t el = dtype == TDX_F32 ? 4 : 2;
+    const size_t a_bytes = static_cast<size_t>(M) * K * el, b_bytes = static_cast<size_t>(K) * N * el,
+                 c_bytes = static_cast<size_t>(M) * N * el;
+    void *dA, *dB, *dC;
+    if ((rc = ensure_staging(ctx, 0, a_bytes, &dA))) return rc;
+    if ((rc = ensure_staging(ctx, 1, b_bytes, &dB))) return rc;
+    if ((rc = ensure_staging(ctx, 2, c_bytes, &dC))) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (a_bytes) TDX_CUDA(cudaMemcpyAsync(dA, A_host, a_bytes, cudaMemcpyHostToDevice, st));
+    if (b_bytes) TDX_CUDA(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, st));
+    rc = gemm_dispatch(M, N, K, transA, transB, alpha, dtype, dA, dB, dC, stream, nullptr, nullptr, 0, true);
+    if (rc) return rc;
+    TDX_CUDA(cudaMemcpyAsync(C_host, dC, c_bytes, cudaMemcpyDeviceToHost, st));
+    TDX_CUDA(cudaStreamSynchronize(st));
+    return TDX_OK;
+}
+
+int tdx_conv2d_bias_relu_host(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
+                              int stride, int dtype, const void* x_host, const void* w_host, const float* bias_host,
+                              int relu, void* y_host, void* stream) {
+    ConvProblem cp;
+    int rc = validate_conv(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x_host, w_host, y_host, relu, true, &cp);
+    if (rc) return rc;
+    if (N == 0 || Cout == 0 || cp.P == 0 || cp.Q == 0) return TDX_OK;
+    DeviceCtx* ctx;
+    rc = get_ctx(&ctx);
+    if (rc) return rc;
+    const size_t el = dtype == TDX_F32 ? 4 : 2;
+    const size_t x_bytes = static_cast<size_t>(N) * H * W * Cin * el, w_bytes = static_cast<size_t>(Cout) * R * S * Cin * el,
+                 y_bytes = static_cast<size_t>(N) * cp.P * cp.Q * Cout * el, b_bytes = static_cast<size_t>(Cout) * 4;
+    void *dx, *dw, *dy, *db = nullptr;
+    if ((rc = ensure_staging(ctx, 0, x_bytes, &dx))) return rc;
+    if ((rc = ensure_staging(ctx, 1, w_bytes, &dw))) return rc;
+    if ((rc = ensure_staging(ctx, 2, y_bytes, &dy))) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (x_bytes) TDX_CUDA(cudaMemcpyAsync(dx, x_host, x_bytes, cudaMemcpyHostToDevice, st));
+    TDX_CUDA(cudaMemcpyAsync(dw, w_host, w_bytes, cudaMemcpyHostToDevice, st));
+    if (bias_host) {
+        if ((rc = ensure_staging(ctx, 3, b_bytes, &db))) return rc;
+        TDX_CUDA(cudaMemcpyAsync(db, bias_host, b_bytes, cudaMemcpyHostToDevice, st));
+    }
+    rc = conv_dispatch(N, H, W, Cin, Cout, R, S, pad, stride, dtype, dx, dw, static_cast<const float*>(db), relu, dy,
+                       stream, nullptr);
+    if (rc) return rc;
+    TDX_CUDA(cudaMemcpyAsync(y_host, dy, y_bytes, cudaMemcpyDeviceToHost, st));
+    TDX_CUDA(cudaStreamSynchronize(st));
+    return TDX_OK;
+}
+
+int tdx_enum_gemm_configs(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, tdx_config* out, int cap,
+                          int* n) {
+    int rc = validate_gemm(M, N, K, transA, transB, dtype, nullptr, nullptr, nullptr, false);
+    if (rc) return rc;
+    if (cap < 0 || (cap > 0 && out == nullptr)) return fail(TDX_ERR_INVALID_ARG, "bad output list");
+    int sm_count, smem_limit;
+    device_limits(&sm_count, &smem_limit);
+    std::vector<tdx_config> v;
+    if (M > 0 && N > 0 && K > 0) enum_gemm(GemmProblem{M, N, K, transA, transB, dtype}, sm_count, smem_limit, &v);
+    return write_configs(v, out, cap, n);
+}
+
+int tdx_enum_conv2d_configs(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
+                            int stride, int dtype, tdx_config* out, int cap, int* n) {
+    ConvProblem cp;
+    int rc = validate_conv(N, H, W, Cin, Cout, R, S, pad, stride, dtype, nullptr, nullptr, nullptr, 0, false, &cp);
+    if (rc) return rc;
+    if (cap < 0 || (cap > 0 && out == nullptr)) return fail(TDX_ERR_INVALID_ARG, "bad output list");
+    int sm_count, smem_limit;
+    device_limits(&sm_count, &smem_limit);
+    std::vector<tdx_config> v;
+    if (N > 0 && Cout > 0 && cp.P > 0 && cp.Q > 0) enum_conv(cp, sm_count, smem_limit, &v);
+    return write_configs(v, out, cap, n);
+}
+
+int tdx_default_gemm_config(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, tdx_config* out) {
+    int rc = validate_gemm(M, N, K, transA, transB, dtype, nullptr, nullptr, nullptr, false);
+    if (rc) return rc;
+    if (out == nullptr) return fail(TDX_ERR_INVALID_ARG, "out is NULL");
+    if (M == 0 || N == 0 || K == 0) { std::memset(out, 0, sizeof *out); return TDX_OK; }
+    int sm_count, smem_limit;
+    device_limits(&sm_count, &smem_limit);
+    return resolve_gemm_config(GemmProblem{M, N, K, transA, transB, dtype}, nullptr, sm_count, smem_limit, out);
+}
+
+int tdx_default_conv2d_config(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
+                              int stride, int dtype, tdx_config* out) {
+    ConvProblem cp;
+    int rc = validate_conv(N, H, W, Cin, Cout, R, S, pad, stride, dtype, nullptr, nullptr, nullptr, 0, false, &cp);
+    if (rc) return rc;
+    if (out == nullptr) return fail(TDX_ERR_INVALID_ARG, "out is NULL");
+    if (N == 0 || Cout == 0 || cp.P == 0 || cp.Q == 0) { std::memset(out, 0, sizeof *out); return TDX_OK; }
+    int sm_count, smem_limit;
+    device_limits(&sm_count, &smem_limit);
+    return resolve_conv_config(cp, nullptr, sm_count, smem_limit, out);
+}
+
+int tdx_tune_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, int iters, tdx_config* best,
+                  float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried, void* stream) {
+    int rc = validate_gemm(M, N, K, transA, transB, dtype, nullptr, nullptr, nullptr, false);
+    if (rc) return rc;
+    if (best == nullptr || iters < 1 || cap < 0) return fail(TDX_ERR_INVALID_ARG, "best is NULL, iters < 1 or cap < 0");
+    if (M == 0 || N == 0 || K == 0) return fail(TDX_ERR_INVALID_ARG, "empty problem");
+    DeviceCtx* ctx;
+    rc = get_ctx(&ctx);
+    if (rc) return rc;
+    GemmProblem g{M, N, K, transA, transB, dtype};
+    std::vector<tdx_config> cands;
+    enum_gemm(g, ctx->sm_count, ctx->smem_optin, &cands);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t el = dtype == TDX_F32 ? 4 : 2;
+    ScratchGuard guard;
+    void *A, *B, *C, *ws;
+    size_t ws_bytes = 0;
+    for (const auto& c : cands) ws_bytes = std::max(ws_bytes, c.split_k > 1 ? static_cast<size_t>(c.split_k) * M * N * 4 : 0);
+    if ((rc = guard.alloc(&A, M * K * el))) return rc;
+    if ((rc = guard.alloc(&B, K * N * el))) return rc;
+    if ((rc = guard.alloc(&C, M * N * el))) return rc;
+    if ((rc = guard.alloc(&ws, ws_bytes))) return rc;
+    // fp32 buffers are filled as pairs of bf16 patterns: finite, varied values either way
+    if ((rc = fill_scratch(A, M * K * el / 2, 1u, st))) return rc;
+    if ((rc = fill_scratch(B, K * N * el / 2, 2u, st))) return rc;
+    auto launch = [&](const tdx_config& c) {
+        return gemm_dispatch(M, N, K, transA, transB, 1.0f, dtype, A, B, C, stream, &c, ws, ws_bytes, false);
+    };
+    rc = time_candidates(cands, iters, st, launch, best, best_us, tried, tried_us, cap, n_tried);
+    cudaStreamSynchronize(st);
+    if (rc) return rc;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        g_tune[gemm_key(M, N, K, transA, transB, dtype)] = TuneEntry{*best, best_us ? *best_us : 0.0f};
+    }
+    return TDX_OK;
+}
+
+int tdx_tune_conv2d(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
+                    int stride, int dtype, int iters, tdx_config* best, float* best_us, tdx_config* tried,
+                    float* tried_us, int cap, int* n_tried, void* stream) {
+    ConvProblem cp;
+    int rc = validate_conv(N, H, W, Cin, Cout, R, S, pad, stride, dtype, nullptr, nullptr, nullptr, 0, false, &cp);
+    if (rc) return rc;
+    if (best == nullptr || iters < 1 || cap < 0) return fail(TDX_ERR_INVALID_ARG, "best is NULL, iters < 1 or cap < 0");
+    if (N == 0 || Cout == 0 || cp.P == 0 || cp.Q == 0) return fail(TDX_ERR_INVALID_ARG, "empty problem");
+    DeviceCtx* ctx;
+    rc = get_ctx(&ctx);
+    if (rc) return rc;
+    std::vector<tdx_config> cands;
+    enum_conv(cp, ctx->sm_count, ctx->smem_optin, &cands);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t el = dtype == TDX_F32 ? 4 : 2;
+    ScratchGuard guard;
+    void *x, *w, *y, *b;
+    if ((rc = guard.alloc(&x, N * H * W * Cin * el))) return rc;
+    if ((rc = guard.alloc(&w, Cout * R * S * Cin * el))) return rc;
+    if ((rc = guard.alloc(&y, N * cp.P * cp.Q * Cout * el))) return rc;
+    if ((rc = guard.alloc(&b, Cout * 4))) return rc;
+    if ((rc = fill_scratch(x, N * H * W * Cin * el / 2, 3u, st))) return rc;
+    if ((rc = fill_scratch(w, Cout * R * S * Cin * el / 2, 4u, st))) return rc;
+    TDX_CUDA(cudaMemsetAsync(b, 0, Cout * 4, st));
+    auto launch = [&](const tdx_config& c) {
+        return conv_dispatch(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, static_cast<const float*>(b), 1, y, stream, &c);
+    };
+    rc = time_candidates(cands, iters, st, launch, best, best_us, tried, tried_us, cap, n_tried);
+    cudaStreamSynchronize(st);
+    if (rc) return rc;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        g_tune[conv_key(N, H, W, Cin, Cout, R, S, pad, stride, dtype)] = TuneEntry{*best, best_us ? *best_us : 0.0f};
+    }
+    return TDX_OK;
+}
+
+int tdx_tune_save(const char* json_path) {
+    if (json_path == nullptr) return fail(TDX_ERR_INVALID_ARG, "path is NULL");
+    FILE* f = fopen(json_path, "w");
+    if (!f) return fail(TDX_ERR_INVALID_ARG, "cannot open %s for writing", json_path);
+    std::lock_guard<std::mutex> lk(g_mu);
+    fprintf(f, "{\"version\": 1, \"entries\": [\n");
+    size_t i = 0;
+    for (const auto& kv : g_tune) {
+        int v[11];
+        cfg_to_ints(kv.second.cfg, v);
+        fprintf(f, "  {\"key\": \"%s\", \"cfg\": [", kv.first.c_str());
+        for (int j = 0; j < 11; ++j) fprintf(f, "%d%s", v[j], j < 10 ? ", " : "");
+        fprintf(f, "], \"us\": %.3f}%s\n", kv.second.us, ++i < g_tune.size() ? "," : "");
+    }
+    fprintf(f, "]}\n");
+    fclose(f);
+    return TDX_OK;
+}
+
+int tdx_tune_load(const char* json_path) {
+    if (json_path == nullptr) return fail(TDX_ERR_INVALID_ARG, "path is NULL");
+    FILE* f = fopen(json_path, "r");
+    if (!f) return fail(TDX_ERR_INVALID_ARG, "cannot open %s", json_path);
+    std::string text;
+    char buf[4096];
+    size_t got;
+    while ((got = fread(buf, 1, sizeof buf, f)) > 0) text.append(buf, got);
+    fclose(f);
+    std::map<std::string, TuneEntry> loaded;
+    size_t pos = 0;
+    while ((pos = text.find("\"key\"", pos)) != std::string::npos) {
+        const size_t q0 = text.find('"', text.find(':', pos) + 1);
+        const size_t q1 = q0 == std::string::npos ? q0 : text.find('"', q0 + 1);
+        const size_t b0 = q1 == std::string::npos ? q1 : text.find('[', q1);
+        const size_t b1 = b0 == std::string::npos ? b0 : text.find(']', b0);
+        if (b1 == std::string::npos) return fail(TDX_ERR_INVALID_ARG, "malformed tuning cache %s", json_path);
+        const std::string key = text.substr(q0 + 1, q1 - q0 - 1);
+        int v[11];
+        int n = 0;
+        const char* s = text.c_str() + b0 + 1;
+        const char* end = text.c_str() + b1;
+        while (s < end && n < 11) {
+            char* next;
+            long val = strtol(s, &next, 10);
+            if (next == s) break;
+            v[n++] = static_cast<int>(val);
+            s = next;
+            while (s < end && (*s == ',' || *s == ' ')) ++s;
+        }
+        if (n != 11) return fail(TDX_ERR_INVALID_ARG, "malformed cfg list in %s", json_path);
+        TuneEntry e;
+        ints_to_cfg(v, &e.cfg);
+        e.us = 0.0f;
+        const size_t u = text.find("\"us\"", b1);
+        const size_t nextkey = text.find("\"key\"", b1);
+        if (u != std::string::npos && (nextkey == std::string::npos || u < nextkey))
+            e.us = static_cast<float>(atof(text.c_str() + text.find(':', u) + 1));
+        loaded[key] = e;
+        pos = b1;
+    }
+    std::lock_guard<std::mutex> lk(g_mu);
+    for (auto& kv : loaded) g_tune[kv.first] = kv.second;
+    return TDX_OK;
+}
+
+int tdx_tune_clear(void) {
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_tune.clear();
+    return TDX_OK;
+}
+
+int tdx_check_device_status(void* stream) {
+    DeviceCtx* ctx;
+    int rc = get_ctx(&ctx);
+    if (rc) return rc;
+    TDX_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    int v = 0;
+    TDX_CUDA(cudaMemcpy(&v, ctx->status_ptr, sizeof v, cudaMemcpyDeviceToHost));
+    if (v != 0) {
+        TDX_CUDA(cudaMemset(ctx->status_ptr, 0, sizeof v));
+        return fail(TDX_ERR_TIMEOUT, "a kernel abandoned a bounded wait (role code %d)", v);
+    }
+    return TDX_OK;
+}
+
+int64_t tdx_kernel_launch_count(void) { return g_launches.load(); }
+
+const char* tdx_last_error(void) { return g_err.c_str(); }
+
+const char* tdx_version(void) { return "tdx 0.1.0 (sm_100a)"; }
+
+}  // extern "C"

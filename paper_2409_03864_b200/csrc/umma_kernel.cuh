@@ -1,0 +1,353 @@
+// Persistent, warp-specialised tcgen05 contraction kernel (bf16 x bf16 -> fp32 in TMEM).
+//
+// One CTA owns a stream of 128 x BN output tiles.  Roles:
+//   warp 0 (one lane)  TMA producer: fills a ring of shared-memory stages, each holding a
+//                      128 x 64 slice of op(A) and a 64 x BN slice of op(B), 128-byte swizzled.
+//   warp 1 (one lane)  MMA issuer: per stage four tcgen05.mma (K = 16 each) into one of two
+//                      TMEM accumulators; tcgen05.commit releases the stage / publishes the tile.
+//   warps 2..5         epilogue: tcgen05.ld the accumulator (one row per thread), apply
+//                      alpha / bias / ReLU, convert, store 16 bytes at a time.
+// The second accumulator lets the epilogue of tile t overlap the main loop of tile t+1.
+//
+// Operand transposes are never materialised: a K-major operand is loaded as one box of
+// (64 k) x (rows); an MN-major operand as boxes of (64 mn) x (64 k), and the MMA
+// descriptors say which one it is.  For the convolution the A slice of K-step (r, s, c-chunk)
+// is the input window shifted by (r - pad, s - pad); out-of-range coordinates are zero-filled
+// by the copy engine, which is all the padding there is.
+//
+// Every wait is bounded: a wait that runs out records a code in the device status word,
+// raises a CTA-wide abort flag and all roles leave their loops and free TMEM.
+#pragma once
+#include <cuda_bf16.h>
+
+#include "ptx_sm100.cuh"
+
+namespace tdx {
+
+constexpr int kBM = 128;          // tile rows = TMEM lanes
+constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int kUmmaK = 16;        // K of one tcgen05.mma for 16-bit inputs
+constexpr int kUmmaThreads = 192;
+constexpr int kMaxStages = 8;
+constexpr int kABytes = kBM * kBK * 2;                 // 16 KiB
+constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at boost clock
+
+enum : int { kTimeoutProducer = 1, kTimeoutMma = 2, kTimeoutEpilogue = 3 };
+
+struct UmmaParams {
+    int M, N;                 // logical output rows / columns
+    int num_kb;               // K blocks of 64 in the whole reduction
+    int tiles_m, tiles_n, panel;
+    int split_k, kb_per_split;
+    int bn, stages, tmem_cols;
+    int a_mn_major, b_mn_major;
+    float alpha;
+    const float* bias;        // [N] or nullptr
+    int relu;
+    __nv_bfloat16* C;         // bf16 output, row pitch ldc elements
+    long long ldc;
+    float* partial;           // split-K: [split][M][N] fp32
+    int vec_store;            // rows of C / partial are 16-byte aligned and N % 8 == 0
+    // convolution geometry (kConv only)
+    int bw, bh, nb;           // spatial patch (bw x bh output pixels), patches per tile
+    int patches_w, patches_h; // patches per image along Q and P
+    int P, Q, Nimg, S, pad, cchunks;
+    int* status;              // device status word
+};
+
+__device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, volatile int* s_abort, int* g_status,
+                                             int code) {
+    if (ptx::mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    for (;;) {
+        if (ptx::mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 63u) == 0u) {
+            if (*s_abort) return false;
+            if (clock64() - t0 > kWaitLimitCycles) {
+                *s_abort = 1;
+                atomicCAS(g_status, 0, code);
+                return false;
+            }
+        }
+    }
+}
+
+struct TileCoord {
+    int m_blk, n_blk, kb0, kb1, split;
+};
+
+__device__ __forceinline__ TileCoord decode_item(const UmmaParams& p, int item) {
+    TileCoord t;
+    const int tile = item / p.split_k;
+    t.split = item - tile * p.split_k;
+    const int per_panel = p.panel * p.tiles_n;
+    const int pidx = tile / per_panel;
+    const int rem = tile - pidx * per_panel;
+    const int m_first = pidx * p.panel;
+    const int w = min(p.panel, p.tiles_m - m_first);
+    t.n_blk = rem / w;
+    t.m_blk = m_first + (rem - t.n_blk * w);
+    t.kb0 = t.split * p.kb_per_split;
+    t.kb1 = min(p.num_kb, t.kb0 + p.kb_per_split);
+    return t;
+}
+
+template <bool kConv>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                     const UmmaParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t tfull_bar[2];
+    __shared__ __align__(8) uint64_t tempty_bar[2];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t b_bytes = static_cast<uint32_t>(p.bn) * 128u;
+    const uint32_t stage_bytes = kABytes + b_bytes;
+    volatile int* abort_flag = &s_abort;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; ++s) {
+            ptx::mbar_init(&full_bar[s], 1);
+            ptx::mbar_init(&empty_bar[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(&tfull_bar[b], 1);
+            ptx::mbar_init(&tempty_bar[b], 4);
+        }
+        s_abort = 0;
+        ptx::fence_barrier_init();
+        ptx::tma_prefetch_desc(&tmA);
+        ptx::tma_prefetch_desc(&tmB);
+    }
+    if (warp == 1) {
+        __syncwarp();
+        ptx::tmem_alloc(&s_tmem_base, static_cast<uint32_t>(p.tmem_cols));
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = s_tmem_base;
+    const int total_items = p.tiles_m * p.tiles_n * p.split_k;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
+                const TileCoord t = decode_item(p, item);
+                for (int kb = t.kb0; kb < t.kb1; ++kb) {
+                    if (!wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) {
+                        ok = false;
+                        break;
+                    }
+                    uint64_t* bar = &full_bar[stage];
+                    ptx::mbar_arrive_expect_tx(bar, stage_bytes);
+                    uint8_t* a_dst = smem + static_cast<size_t>(stage) * stage_bytes;
+                    uint8_t* b_dst = a_dst + kABytes;
+                    if (kConv) {
+                        const int tap = kb / p.cchunks;
+                        const int cc = kb - tap * p.cchunks;
+                        const int r = tap / p.S;
+                        const int s = tap - r * p.S;
+                        const int ppi = p.patches_w * p.patches_h;
+                        const uint32_t patch_bytes = static_cast<uint32_t>(p.bw * p.bh) * 128u;
+                        for (int i = 0; i < p.nb; ++i) {
+                            const int patch = t.m_blk * p.nb + i;
+                            const int n = patch / ppi;
+                            const int rem = patch - n * ppi;
+                            const int ph = rem / p.patches_w;
+                            const int pw = rem - ph * p.patches_w;
+                            ptx::tma_load_4d(a_dst + i * patch_bytes, &tmA, bar, cc * kBK, pw * p.bw + s - p.pad,
+                                             ph * p.bh + r - p.pad, n);
+                        }
+                        ptx::tma_load_3d(b_dst, &tmB, bar, cc * kBK, tap, t.n_blk * p.bn);
+                    } else {
+                        if (p.a_mn_major) {
+                            ptx::tma_load_2d(a_dst, &tmA, bar, t.m_blk * kBM, kb * kBK);
+                            ptx::tma_load_2d(a_dst + 8192, &tmA, bar, t.m_blk * kBM + 64, kb * kBK);
+                        } else {
+                            ptx::tma_load_2d(a_dst, &tmA, bar, kb * kBK, t.m_blk * kBM);
+                        }
+                        if (p.b_mn_major) {
+                            for (int i = 0; i < p.bn / 64; ++i)
+                                ptx::tma_load_2d(b_dst + i * 8192, &tmB, bar, t.n_blk * p.bn + i * 64, kb * kBK);
+                        } else {
+                            ptx::tma_load_2d(b_dst, &tmB, bar, kb * kBK, t.n_blk * p.bn);
+                        }
+                    }
+                    if (++stage == p.stages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+            if (!ok) {
+                // let copies that are still in flight land before the CTA goes away
+                for (int i = 0; i < 64; ++i) __nanosleep(2000);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = ptx::make_idesc_bf16_f32(kBM, p.bn, p.a_mn_major, p.b_mn_major);
+            // K-major: 8-row groups are 1024 B apart (SBO); K advances 32 B inside the swizzle row.
+            // MN-major: 64-element groups along MN are one 64 x 64 box (8192 B) apart (LBO),
+            //           8-k groups are 1024 B apart (SBO); K advances 16 rows = 2048 B.
+            const uint32_t a_lbo = p.a_mn_major ? 8192u : 16u;
+            const uint32_t b_lbo = p.b_mn_major ? 8192u : 16u;
+            const uint32_t a_kstep = p.a_mn_major ? 2048u : 32u;
+            const uint32_t b_kstep = p.b_mn_major ? 2048u : 32u;
+            int stage = 0;
+            uint32_t phase = 0;
+            int local = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++local) {
+                const TileCoord t = decode_item(p, item);
+                const int buf = local & 1;
+                const uint32_t aphase = (local >> 1) & 1;
+                if (!wait_bounded(&tempty_bar[buf], aphase ^ 1u, abort_flag, p.status, kTimeoutMma)) break;
+                ptx::tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * p.bn);
+                for (int kb = t.kb0; kb < t.kb1; ++kb) {
+                    if (!wait_bounded(&full_bar[stage], phase, abort_flag, p.status, kTimeoutMma)) {
+                        ok = false;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t a_addr = ptx::smem_u32(smem + static_cast<size_t>(stage) * stage_bytes);
+                    const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+                    for (int j = 0; j < kBK / kUmmaK; ++j) {
+                        const uint64_t adesc = ptx::make_smem_desc_sw128(a_addr + j * a_kstep, a_lbo, 1024u);
+                        const uint64_t bdesc = ptx::make_smem_desc_sw128(b_addr + j * b_kstep, b_lbo, 1024u);
+                        ptx::umma_bf16(d_tmem, adesc, bdesc, idesc, (kb > t.kb0 || j > 0) ? 1u : 0u);
+                    }
+                    ptx::umma_commit(&empty_bar[stage]);
+                    if (++stage == p.stages) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (ok) ptx::umma_commit(&tfull_bar[buf]);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (4 warps)
+        const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
+        const int row_in_tile = quarter * 32 + lane;
+        int local = 0;
+        for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++local) {
+            const TileCoord t = decode_item(p, item);
+            const int buf = local & 1;
+            const uint32_t aphase = (local >> 1) & 1;
+            if (!wait_bounded(&tfull_bar[buf], aphase, abort_flag, p.status, kTimeoutEpilogue)) break;
+            ptx::tc_fence_after_sync();
+
+            long long grow;
+            bool valid;
+            if (kConv) {
+                const int per_patch = p.bw * p.bh;
+                const int pl = row_in_tile / per_patch;
+                const int within = row_in_tile - pl * per_patch;
+                const int hl = within / p.bw;
+                const int wl = within - hl * p.bw;
+                const int patch = t.m_blk * p.nb + pl;
+                const int ppi = p.patches_w * p.patches_h;
+                const int n = patch / ppi;
+                const int rem = patch - n * ppi;
+                const int ph = rem / p.patches_w;
+                const int pw = rem - ph * p.patches_w;
+                const int pp = ph * p.bh + hl;
+                const int qq = pw * p.bw + wl;
+                valid = (n < p.Nimg) && (pp < p.P) && (qq < p.Q);
+                grow = (static_cast<long long>(n) * p.P + pp) * p.Q + qq;
+            } else {
+                grow = static_cast<long long>(t.m_blk) * kBM + row_in_tile;
+                valid = grow < p.M;
+            }
+
+            for (int c0 = 0; c0 < p.bn; c0 += 32) {
+                uint32_t r[32];
+                const uint32_t taddr =
+                    tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * p.bn + c0);
+                ptx::tmem_ld_32x32b_x32(taddr, r);
+                ptx::tmem_ld_wait();
+                const int col0 = t.n_blk * p.bn + c0;
+                if (valid && col0 < p.N) {
+                if (p.split_k > 1) {
+                    float* dst = p.partial + (static_cast<long long>(t.split) * p.M + grow) * p.N + col0;
+                    if (p.vec_store) {
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            if (col0 + g * 4 < p.N) {
+                                float4 v = make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]),
+                                                       __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
+                                *reinterpret_cast<float4*>(dst + g * 4) = v;
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col0 + j < p.N) dst[j] = __uint_as_float(r[j]);
+                    }
+                } else {
+                    float v[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        float x = p.alpha * __uint_as_float(r[j]);
+                        if (p.bias != nullptr && col0 + j < p.N) x += __ldg(p.bias + col0 + j);
+                        if (p.relu) x = fmaxf(x, 0.0f);
+                        v[j] = x;
+                    }
+                    __nv_bfloat16* dst = p.C + grow * p.ldc + col0;
+                    if (p.vec_store) {
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            if (col0 + g * 8 < p.N) {
+                                uint4 pk;
+                                __nv_bfloat162 h0 = __floats2bfloat162_rn(v[g * 8 + 0], v[g * 8 + 1]);
+                                __nv_bfloat162 h1 = __floats2bfloat162_rn(v[g * 8 + 2], v[g * 8 + 3]);
+                                __nv_bfloat162 h2 = __floats2bfloat162_rn(v[g * 8 + 4], v[g * 8 + 5]);
+                                __nv_bfloat162 h3 = __floats2bfloat162_rn(v[g * 8 + 6], v[g * 8 + 7]);
+                                pk.x = *reinterpret_cast<uint32_t*>(&h0);
+                                pk.y = *reinterpret_cast<uint32_t*>(&h1);
+                                pk.z = *reinterpret_cast<uint32_t*>(&h2);
+                                pk.w = *reinterpret_cast<uint32_t*>(&h3);
+                                *reinterpret_cast<uint4*>(dst + g * 8) = pk;
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(v[j]);
+                    }
+                }
+                }
+                __syncwarp();   // reconverge before the next warp-aligned TMEM load
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&tempty_bar[buf]);
+        }
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        __syncwarp();
+        ptx::tmem_dealloc(tmem_base, static_cast<uint32_t>(p.tmem_cols));
+    }
+}
+
+}  // namespace tdx

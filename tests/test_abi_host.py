@@ -1,0 +1,167 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol the
+header declares, validates arguments before touching a device, and lists a search space that
+obeys the static constraints."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import paper_2409_03864_b200 as tdx
+from paper_2409_03864_b200 import build as tdx_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    tdx_build.build()
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "tdx.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(tdx_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = declared_symbols()
+    assert len(names) >= 18
+    L = ctypes.CDLL(str(tdx_build.LIB))
+    for n in names:
+        assert hasattr(L, n), f"{n} declared in tdx.h but not exported"
+    assert set(names) == set(tdx.binding.EXPORTS)
+    assert tdx.tdx_version().startswith("tdx ")
+
+
+def test_gemm_argument_validation_is_silenceable_and_precedes_cuda():
+    bad = [
+        dict(M=-1), dict(N=-3), dict(K=-1), dict(transA=2), dict(transB=-1), dict(dtype=7),
+        dict(A=None), dict(B=None), dict(C=None),
+    ]
+    base = dict(M=8, N=8, K=8, transA=0, transB=0, alpha=1.0, dtype=tdx.TDX_BF16, A=256, B=512, C=1024)
+    for b in bad:
+        a = dict(base, **b)
+        st = tdx.tdx_gemm(**a)
+        assert st == tdx.TDX_ERR_INVALID_ARG, (b, st)
+        assert tdx.tdx_last_error()
+    # misaligned element pointer
+    assert tdx.tdx_gemm(**dict(base, A=257)) == tdx.TDX_ERR_ALIGNMENT
+    # empty problems are a no-op even without a device
+    assert tdx.tdx_gemm(**dict(base, M=0, A=None, B=None, C=None)) == tdx.TDX_OK
+    assert tdx.tdx_gemm(**dict(base, N=0)) == tdx.TDX_OK
+
+
+def test_conv_argument_validation():
+    base = dict(N=1, H=8, W=8, Cin=8, Cout=8, R=3, S=3, pad=1, stride=1, dtype=tdx.TDX_BF16, x=256, w=512, bias=None,
+                relu=1, y=1024)
+    for b in [dict(N=-1), dict(Cin=0), dict(R=0), dict(S=-1), dict(pad=-1), dict(stride=0), dict(dtype=5),
+              dict(relu=2), dict(x=None), dict(w=None), dict(y=None)]:
+        st = tdx.tdx_conv2d_bias_relu(**dict(base, **b))
+        assert st == tdx.TDX_ERR_INVALID_ARG, (b, st)
+    # filter larger than the padded image: empty output, no-op
+    assert tdx.tdx_conv2d_bias_relu(**dict(base, H=1, W=1, pad=0)) == tdx.TDX_OK
+    assert tdx.tdx_conv2d_bias_relu(**dict(base, Cout=0)) == tdx.TDX_OK
+
+
+def test_infeasible_explicit_config_is_reported_before_any_device_work():
+    base = dict(M=256, N=256, K=256, transA=0, transB=1, alpha=1.0, dtype=tdx.TDX_BF16, A=256, B=512, C=1024)
+    for kw in [dict(tile_n=48), dict(tile_n=512), dict(stages=9), dict(tile_m=64), dict(split_k=7),
+               dict(tile_k=32), dict(cta_pair=3), dict(kernel=9), dict(kernel=tdx.TDX_KERNEL_SIMT)]:
+        cfg = tdx.tdx_config(kernel=kw.pop("kernel", tdx.TDX_KERNEL_UMMA), **kw)
+        assert tdx.tdx_gemm_ex(**base, cfg=cfg) == tdx.TDX_ERR_CONFIG, kw
+    # N-major B (transB=0) needs tile_n % 64 == 0
+    cfg = tdx.tdx_config(kernel=tdx.TDX_KERNEL_UMMA, tile_n=32)
+    assert tdx.tdx_gemm_ex(**dict(base, transB=0), cfg=cfg) == tdx.TDX_ERR_CONFIG
+    # forcing the tensor-core kernel on a pitch that is not a multiple of 16 bytes
+    cfg = tdx.tdx_config(kernel=tdx.TDX_KERNEL_UMMA)
+    assert tdx.tdx_gemm_ex(**dict(base, K=100), cfg=cfg) == tdx.TDX_ERR_ALIGNMENT
+    # conv: split-K and bad patches
+    cbase = dict(N=1, H=16, W=16, Cin=64, Cout=64, R=3, S=3, pad=1, stride=1, dtype=tdx.TDX_BF16, x=256, w=512,
+                 bias=None, relu=1, y=1024)
+    for kw in [dict(split_k=2), dict(patch_w=4, patch_h=4), dict(patch_w=24, patch_h=2), dict(patch_w=64, patch_h=4)]:
+        cfg = tdx.tdx_config(kernel=tdx.TDX_KERNEL_UMMA, **kw)
+        assert tdx.tdx_conv2d_bias_relu_ex(**cbase, cfg=cfg) == tdx.TDX_ERR_CONFIG, kw
+
+
+def test_workspace_size():
+    st, b = tdx.tdx_gemm_workspace_size(128, 8192, 8192, tdx.TDX_BF16, tdx.tdx_config(split_k=4))
+    assert st == tdx.TDX_OK and b == 4 * 128 * 8192 * 4
+    st, b = tdx.tdx_gemm_workspace_size(128, 8192, 8192, tdx.TDX_BF16, tdx.tdx_config(split_k=1))
+    assert st == tdx.TDX_OK and b == 0
+    assert tdx.tdx_gemm_workspace_size(-1, 1, 1, tdx.TDX_BF16, None)[0] == tdx.TDX_ERR_INVALID_ARG
+
+
+SMEM_LIMIT = 232448
+
+
+@pytest.mark.parametrize("shape", [(1024, 1024, 1024), (8192, 8192, 8192), (128, 8192, 8192), (8192, 128, 8192),
+                                   (4096, 4096, 512)])
+def test_gemm_search_space_obeys_constraints(shape):
+    M, N, K = shape
+    st, cfgs = tdx.tdx_enum_gemm_configs(M, N, K, 0, 0, tdx.TDX_BF16)
+    assert st == tdx.TDX_OK and len(cfgs) >= 4
+    num_kb = -(-K // 64)
+    seen = set()
+    for c in cfgs:
+        key = tuple(c.values())
+        assert key not in seen
+        seen.add(key)
+        assert c["kernel"] == tdx.TDX_KERNEL_UMMA and c["tile_m"] == 128 and c["tile_k"] == 64
+        assert c["tile_n"] % 64 == 0                          # B is read N-major here
+        assert 2 <= c["stages"] <= 8
+        assert c["stages"] * (16384 + c["tile_n"] * 128) + 1024 + 512 <= SMEM_LIMIT
+        assert 2 * c["tile_n"] <= 512                          # two TMEM accumulators
+        per = -(-num_kb // c["split_k"])
+        assert (c["split_k"] - 1) * per < num_kb               # no empty K slice
+    if M * N <= 128 * 8192:
+        assert any(c["split_k"] > 1 for c in cfgs)             # skinny shapes get split-K candidates
+    if shape == (8192, 8192, 8192):
+        assert all(c["split_k"] == 1 for c in cfgs)
+
+
+def test_search_space_for_other_kernels():
+    st, cfgs = tdx.tdx_enum_gemm_configs(256, 256, 256, 0, 0, tdx.TDX_F32)
+    assert st == tdx.TDX_OK and [c["kernel"] for c in cfgs] == [tdx.TDX_KERNEL_SIMT]
+    st, cfgs = tdx.tdx_enum_gemm_configs(196, 256, 2305, 0, 0, tdx.TDX_BF16)   # K pitch not 16-byte aligned
+    assert st == tdx.TDX_OK and [c["kernel"] for c in cfgs] == [tdx.TDX_KERNEL_GENERIC]
+    st, cfgs = tdx.tdx_enum_conv2d_configs(32, 56, 56, 256, 256, 3, 3, 1, 1, tdx.TDX_BF16)
+    assert st == tdx.TDX_OK and cfgs
+    for c in cfgs:
+        a = c["patch_w"] * c["patch_h"]
+        assert c["patch_w"] >= 8 and a <= 128 and a & (a - 1) == 0 and c["split_k"] == 1
+    st, cfgs = tdx.tdx_enum_conv2d_configs(1, 8, 8, 8, 8, 3, 3, 1, 2, tdx.TDX_BF16)  # stride 2
+    assert [c["kernel"] for c in cfgs] == [tdx.TDX_KERNEL_GENERIC]
+
+
+def test_default_configs():
+    st, c = tdx.tdx_default_gemm_config(4096, 4096, 4096, 0, 1, tdx.TDX_BF16)
+    assert st == tdx.TDX_OK and c.kernel == tdx.TDX_KERNEL_UMMA and c.tile_n == 256 and c.split_k == 1
+    st, c = tdx.tdx_default_gemm_config(128, 8192, 8192, 0, 0, tdx.TDX_BF16)
+    assert st == tdx.TDX_OK and c.split_k > 1
+    st, c = tdx.tdx_default_gemm_config(256, 256, 256, 0, 0, tdx.TDX_F32)
+    assert st == tdx.TDX_OK and c.kernel == tdx.TDX_KERNEL_SIMT
+    st, c = tdx.tdx_default_conv2d_config(32, 56, 56, 256, 256, 3, 3, 1, 1, tdx.TDX_BF16)
+    assert st == tdx.TDX_OK and (c.patch_w, c.patch_h) == (8, 8) and c.tile_n == 256
+    st, c = tdx.tdx_default_conv2d_config(4, 128, 128, 64, 64, 3, 3, 1, 1, tdx.TDX_BF16)
+    assert st == tdx.TDX_OK and (c.patch_w, c.patch_h) == (128, 1) and c.tile_n == 64
+
+
+def test_tuning_cache_round_trip(tmp_path):
+    path = tmp_path / "cache.json"
+    path.write_text('{"version": 1, "entries": [\n  {"key": "gemm:640:640:640:0:1:1", '
+                    '"cfg": [1, 128, 64, 64, 3, 1, 2, 0, 2, 0, 0], "us": 12.500}\n]}\n')
+    assert tdx.tdx_tune_clear() == tdx.TDX_OK
+    assert tdx.tdx_tune_load(str(path)) == tdx.TDX_OK
+    st, c = tdx.tdx_default_gemm_config(640, 640, 640, 0, 1, tdx.TDX_BF16)
+    assert st == tdx.TDX_OK and (c.tile_n, c.stages, c.split_k, c.raster) == (64, 3, 2, 2)
+    out = tmp_path / "out.json"
+    assert tdx.tdx_tune_save(str(out)) == tdx.TDX_OK
+    assert "gemm:640:640:640:0:1:1" in out.read_text() and "[1, 128, 64, 64, 3, 1, 2, 0, 2, 0, 0]" in out.read_text()
+    assert tdx.tdx_tune_clear() == tdx.TDX_OK
+    st, c = tdx.tdx_default_gemm_config(640, 640, 640, 0, 1, tdx.TDX_BF16)
+    assert c.tile_n != 64 or c.split_k != 2
+    assert tdx.tdx_tune_load(str(tmp_path / "missing.json")) == tdx.TDX_ERR_INVALID_ARG
+    bad = tmp_path / "bad.json"
+    bad.write_text('{"entries": [{"key": "gemm:1:1:1:0:0:1", "cfg": [1, 2, 3]}]}')
+    assert tdx.tdx_tune_load(str(bad)) == tdx.TDX_ERR_INVALID_ARG

@@ -1,0 +1,151 @@
+"""GPU parity of tdx_conv2d_bias_relu against the CPU oracle (through the C ABI)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2409_03864_b200 as tdx
+import seeded_inputs as si
+from gpu_util import TIGHT, TOL, conv_error, run_conv, structured_rows
+
+pytestmark = pytest.mark.gpu
+
+
+def umma(**kw):
+    return tdx.tdx_config(kernel=tdx.TDX_KERNEL_UMMA, **kw)
+
+
+def test_conv_delta_filter_is_exact_shifted_copy():
+    # w[k, r0, s0, c] = delta(c, k): the output is the input shifted by (r0 - pad, s0 - pad) with zeros
+    # shifted in from the padding -- exact in bf16, so the comparison is bitwise.
+    N, H, W, C, pad = 2, 12, 20, 64, 1
+    x = si.normal(70, 0, (N, H, W, C), "bf16")
+    for r0, s0 in [(0, 0), (1, 1), (2, 0), (0, 2)]:
+        w = np.zeros((C, 3, 3, C), dtype=np.float32)
+        for k in range(C):
+            w[k, r0, s0, k] = 1.0
+        wb = si.f32_to_bf16_bits(w)
+        st, y, ok = run_conv(N, H, W, C, C, 3, 3, pad, 1, "bf16", x, wb, None, 0, cfg=umma())
+        assert st == 0 and ok, tdx.tdx_last_error()
+        exp = np.zeros((N, H, W, C), dtype=np.uint16)
+        dh, dw = r0 - pad, s0 - pad
+        hs, ws = slice(max(0, -dh), min(H, H - dh)), slice(max(0, -dw), min(W, W - dw))
+        hd, wd = slice(max(0, dh), min(H, H + dh)), slice(max(0, dw), min(W, W + dw))
+        exp[:, hs, ws, :] = x[:, hd, wd, :]
+        y = y.reshape(N, H, W, C)
+        nz = (exp & 0x7FFF) != 0
+        assert np.array_equal(y[nz], exp[nz]) and ((y[~nz] & 0x7FFF) == 0).all(), (r0, s0)
+
+
+CASES = [
+    # N, H,  W,  Cin, Cout, R, S, pad
+    (1, 8, 8, 64, 64, 3, 3, 1),
+    (2, 14, 14, 128, 96, 3, 3, 1),       # 14 x 14 maps: ragged 8 x 8 patches; tile_n = 96 or 128 with a tail
+    (3, 7, 7, 64, 32, 3, 3, 1),          # patches spanning several images in one tile
+    (1, 20, 36, 72, 40, 3, 3, 1),        # Cin not a multiple of 64: zero-filled channel tail
+    (2, 9, 17, 8, 8, 1, 1, 0),           # 1 x 1 filter, tiny channel count
+    (1, 16, 16, 64, 64, 5, 5, 2),
+    (1, 16, 24, 64, 72, 3, 5, 0),        # no padding, non-square filter
+    (1, 10, 130, 64, 64, 3, 3, 1),       # wide rows: 128-wide patches with a ragged tail
+    (1, 6, 6, 64, 36, 3, 3, 2),          # pad larger than the usual (R - 1) / 2; Cout % 8 != 0 -> scalar stores
+]
+
+
+@pytest.mark.parametrize("case", CASES)
+@pytest.mark.parametrize("bias_relu", [(True, 1), (False, 0)])
+def test_conv_small_cases_vs_oracle(case, bias_relu):
+    N, H, W, Cin, Cout, R, S, pad = case
+    use_bias, relu = bias_relu
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, R, S, seed=71)
+    bias = b if use_bias else None
+    st, y, ok = run_conv(N, H, W, Cin, Cout, R, S, pad, 1, "bf16", x, w, bias, relu, cfg=umma())
+    assert st == 0 and ok, tdx.tdx_last_error()
+    err = conv_error(N, H, W, Cin, Cout, R, S, pad, 1, "bf16", x, w, bias, relu, y)
+    assert err < TOL["bf16"] and err < TIGHT["bf16"], err
+
+
+@pytest.mark.parametrize("patch", [(8, 8), (16, 8), (8, 16), (32, 4), (128, 1), (8, 1), (16, 2)])
+def test_conv_patch_shapes(patch):
+    N, H, W, Cin, Cout = 2, 24, 40, 64, 64
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=72)
+    st, y, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1,
+                         cfg=umma(patch_w=patch[0], patch_h=patch[1], tile_n=64, stages=3))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y) < TIGHT["bf16"]
+
+
+def test_conv_padding_equals_explicit_zero_padded_copy_bitwise():
+    # the copy engine's zero fill and explicit zeros feed the same products in the same order
+    N, H, W, Cin, Cout, pad = 2, 16, 24, 64, 64, 1
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=73)
+    _, y1, _ = run_conv(N, H, W, Cin, Cout, 3, 3, pad, 1, "bf16", x, w, b, 1, cfg=umma(patch_w=8, patch_h=8))
+    xp = np.zeros((N, H + 2 * pad, W + 2 * pad, Cin), dtype=np.uint16)
+    xp[:, pad:pad + H, pad:pad + W, :] = x
+    _, y2, _ = run_conv(N, H + 2 * pad, W + 2 * pad, Cin, Cout, 3, 3, 0, 1, "bf16", xp, w, b, 1,
+                        cfg=umma(patch_w=8, patch_h=8))
+    assert np.array_equal(y1, y2)
+
+
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("stride", [1, 2])
+def test_conv_generic_kernel(dtype, stride):
+    N, H, W, Cin, Cout = 2, 11, 13, 5, 7
+    xb, wb, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=74)
+    if dtype == "f32":
+        x, w = si.bf16_bits_to_f32(xb), si.bf16_bits_to_f32(wb)
+    else:
+        x, w = xb, wb
+    st, y, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, stride, dtype, x, w, b, 1)
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert conv_error(N, H, W, Cin, Cout, 3, 3, 1, stride, dtype, x, w, b, 1, y) < TOL[dtype]
+
+
+def test_conv_infeasible_config_leaves_output_untouched():
+    N, H, W, Cin, Cout = 1, 8, 8, 64, 64
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=75)
+    st, _, untouched = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, cfg=umma(patch_w=4, patch_h=4))
+    assert st == tdx.TDX_ERR_CONFIG and untouched
+    st, _, untouched = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 2, "bf16", x, w, b, 1, cfg=umma())   # stride 2
+    assert st == tdx.TDX_ERR_ALIGNMENT and untouched
+
+
+def test_conv_host_buffer_entry_point():
+    N, H, W, Cin, Cout = 1, 16, 16, 64, 64
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=76)
+    y = np.zeros((N * H * W, Cout), dtype=np.uint16)
+    st = tdx.tdx_conv2d_bias_relu_host(N, H, W, Cin, Cout, 3, 3, 1, 1, tdx.TDX_BF16, x, w, b, 1, y)
+    assert st == 0, tdx.tdx_last_error()
+    assert conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y) < TIGHT["bf16"]
+
+
+# ------------------------------------------------------------------ full-size workloads
+
+def test_full_size_conv_128x128x64():
+    # N=4, H=W=128, Cin=Cout=64, 3x3, stride 1, pad 1, bias + ReLU, seed 2 -- full oracle
+    N, H, W, Cin, Cout = 4, 128, 128, 64, 64
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=2)
+    st, y, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1)
+    assert st == 0 and ok, tdx.tdx_last_error()
+    err = conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y)
+    assert err < TOL["bf16"] and err < TIGHT["bf16"], err
+    assert (oracle.decode(y, "bf16") >= 0).all()
+    assert tdx.tdx_check_device_status() == 0
+
+
+def test_full_size_conv_56x56x256():
+    # N=32, H=W=56, Cin=Cout=256, seed 3 -- rows sampled from every part of the image batch
+    N, H, W, Cin, Cout = 32, 56, 56, 256, 256
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=3)
+    st, y, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1)
+    assert st == 0 and ok, tdx.tdx_last_error()
+    M = N * H * W
+    rows = structured_rows(M, extra=2, max_blocks=24)
+    # image corners and edges of the first and last image
+    for n in (0, N - 1):
+        for p, q in [(0, 0), (0, W - 1), (H - 1, 0), (H - 1, W - 1), (0, 7), (8, 0), (27, 55)]:
+            rows = np.append(rows, (n * H + p) * W + q)
+    rows = np.unique(rows)
+    err = conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y, rows=rows)
+    assert err < TOL["bf16"] and err < TIGHT["bf16"], err
+    assert (oracle.decode(y[::53], "bf16") >= 0).all()
+    assert tdx.tdx_check_device_status() == 0
