@@ -62,7 +62,7 @@ typedef enum {
  */
 typedef struct {
     int kernel;     /* tdx_kernel                                                              */
-    int tile_m;     /* 128                                                                     */
+    int tile_m;     /* 128 or 256 (two 128-row halves that share each B slice)                 */
     int tile_n;     /* 32, 64, 96, ..., 256 (multiple of 32; multiple of 64 when transB = 0)    */
     int tile_k;     /* 64                                                                      */
     int stages;     /* depth of the TMA/mbarrier ring, 2..8, bounded by shared memory          */
@@ -71,7 +71,7 @@ typedef struct {
     int store_mode; /* 0 = 16-byte stores from registers                                       */
     int raster;     /* width, in tiles along M, of the panels the tile order walks; 0 = all     */
     int patch_w;    /* conv only: output-pixel patch that forms the rows of a tile (w x h,      */
-    int patch_h;    /*   w*h a power of two <= 128, w >= 8); 0 = choose                         */
+    int patch_h;    /*   w*h a power of two <= 128, w >= 8; tile_m / (w*h) patches per tile); 0 = choose */
 } tdx_config;
 
 /*

@@ -227,28 +227,31 @@ bool conv_umma_layout_ok(const ConvProblem& c) {
     return true;
 }
 
-int umma_max_stages(int tile_n, int smem_limit) {
-    const int stage = tdx::kABytes + tile_n * 128;
+int umma_max_stages(int tile_m, int tile_n, int smem_limit) {
+    const int stage = (tile_m + tile_n) * 128;
     int s = (smem_limit - kStaticSmemReserve - 1024) / stage;
     return std::min(s, tdx::kMaxStages);
 }
 
-int tmem_cols_for(int bn) {
+// Accumulator slots (128 x tile_n each) kept in TMEM: a 256-row tile uses two per tile, and gets four
+// when they fit so that the epilogue still overlaps the next tile's main loop.
+int tmem_slots_for(int tile_m, int bn) { return (tile_m == 256 && bn <= 128) ? 4 : 2; }
+int tmem_cols_for(int tile_m, int bn) {
     int c = 32;
-    while (c < 2 * bn) c *= 2;
+    while (c < tmem_slots_for(tile_m, bn) * bn) c *= 2;
     return c;
 }
 
 // Static feasibility of a fully specified tensor-core configuration (the search-space constraints).
 // Returns 0 when feasible, else a short reason.
 const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num_kb, int smem_limit, bool conv) {
-    if (c.tile_m != 128) return "tile_m must be 128";
+    if (c.tile_m != 128 && c.tile_m != 256) return "tile_m must be 128 or 256";
     if (c.tile_k != 64) return "tile_k must be 64";
     if (c.cta_pair != 1) return "cta_pair must be 1";
     if (c.store_mode != 0) return "store_mode must be 0";
     if (c.tile_n < 32 || c.tile_n > 256 || c.tile_n % 32) return "tile_n must be a multiple of 32 in [32, 256]";
     if (b_mn_major && c.tile_n % 64) return "tile_n must be a multiple of 64 when B is read N-major";
-    if (c.stages < 2 || c.stages > umma_max_stages(c.tile_n, smem_limit)) return "stages outside the shared-memory budget";
+    if (c.stages < 2 || c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit)) return "stages outside the shared-memory budget";
     if (c.split_k < 1) return "split_k must be >= 1";
     if (conv && c.split_k != 1) return "conv has no split-K";
     if (c.split_k > 1) {
@@ -291,12 +294,17 @@ void default_umma_config(int64_t tiles_m, int64_t N, int64_t num_kb, bool b_mn_m
     c->store_mode = 0;
     c->split_k = 1;
     const int min_bn = b_mn_major ? 64 : 32;
-    int bn = 0;
+    int bn = 0, tm = 128;
     const int64_t n_cap = ceil_div(N, min_bn) * min_bn;   // narrowest tile that covers N at once
-    for (int cand : {256, 128, 64, 32}) {
-        if (cand < min_bn) continue;
-        if (cand > n_cap && cand / 2 >= n_cap) continue;  // a narrower tile covers N just as well
-        if (tiles_m * ceil_div(N, cand) >= sm_count) { bn = cand; break; }
+    // widest tile that still gives every SM at least one tile; 256-row tiles first (fewest L2 bytes per flop)
+    for (int cand_m : {256, 128}) {
+        if (bn) break;
+        for (int cand : {256, 128, 64, 32}) {
+            if (cand < min_bn) continue;
+            if (cand_m == 256 && cand < 128) continue;
+            if (cand > n_cap && cand / 2 >= n_cap) continue;  // a narrower tile covers N just as well
+            if (ceil_div(tiles_m, cand_m / 128) * ceil_div(N, cand) >= sm_count) { bn = cand; tm = cand_m; break; }
+        }
     }
     if (bn == 0) {
         bn = N > 64 ? 128 : (N > 32 ? 64 : min_bn);
@@ -308,8 +316,9 @@ void default_umma_config(int64_t tiles_m, int64_t N, int64_t num_kb, bool b_mn_m
             c->split_k = static_cast<int>(std::max<int64_t>(1, s));
         }
     }
+    c->tile_m = tm;
     c->tile_n = bn;
-    c->stages = std::max(2, umma_max_stages(bn, smem_limit));
+    c->stages = std::max(2, umma_max_stages(tm, bn, smem_limit));
     c->raster = 8;
 }
 
@@ -318,11 +327,12 @@ int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensor
                 cudaStream_t st) {
     const long long items = static_cast<long long>(p.tiles_m) * p.tiles_n * p.split_k;
     const int grid = static_cast<int>(std::min<long long>(items, ctx->sm_count));
-    const size_t smem = static_cast<size_t>(p.stages) * (tdx::kABytes + p.bn * 128) + 1024;
+    const size_t smem = static_cast<size_t>(p.stages) * ((p.bm + p.bn) * 128) + 1024;
+    const int threads = p.bm == 256 ? 320 : 192;   // producer warp, MMA warp, 4 epilogue warps per 128-row half
     if (conv)
-        tdx::umma_contract_kernel<true><<<grid, tdx::kUmmaThreads, smem, st>>>(ma, mb, p);
+        tdx::umma_contract_kernel<true><<<grid, threads, smem, st>>>(ma, mb, p);
     else
-        tdx::umma_contract_kernel<false><<<grid, tdx::kUmmaThreads, smem, st>>>(ma, mb, p);
+        tdx::umma_contract_kernel<false><<<grid, threads, smem, st>>>(ma, mb, p);
     TDX_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     return TDX_OK;
@@ -348,14 +358,16 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     p.M = static_cast<int>(g.M);
     p.N = static_cast<int>(g.N);
     p.num_kb = static_cast<int>(num_kb);
-    p.tiles_m = static_cast<int>(ceil_div(g.M, 128));
+    p.bm = cfg.tile_m;
+    p.slots = tmem_slots_for(cfg.tile_m, cfg.tile_n);
+    p.tiles_m = static_cast<int>(ceil_div(g.M, cfg.tile_m));
     p.tiles_n = static_cast<int>(ceil_div(g.N, cfg.tile_n));
     p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
     p.split_k = cfg.split_k;
     p.kb_per_split = static_cast<int>(ceil_div(num_kb, cfg.split_k));
     p.bn = cfg.tile_n;
     p.stages = cfg.stages;
-    p.tmem_cols = tmem_cols_for(cfg.tile_n);
+    p.tmem_cols = tmem_cols_for(cfg.tile_m, cfg.tile_n);
     p.a_mn_major = g.transA ? 1 : 0;   // A stored K x M: M contiguous
     p.b_mn_major = g.transB ? 0 : 1;   // B stored K x N: N contiguous
     p.alpha = alpha;
@@ -426,7 +438,9 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     std::memset(&p, 0, sizeof p);
     p.bw = cfg.patch_w;
     p.bh = cfg.patch_h;
-    p.nb = 128 / (p.bw * p.bh);
+    p.bm = cfg.tile_m;
+    p.slots = tmem_slots_for(cfg.tile_m, cfg.tile_n);
+    p.nb = cfg.tile_m / (p.bw * p.bh);
     p.patches_w = static_cast<int>(ceil_div(c.Q, p.bw));
     p.patches_h = static_cast<int>(ceil_div(c.P, p.bh));
     const int64_t total_patches = c.N * p.patches_w * p.patches_h;
@@ -440,7 +454,7 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     p.kb_per_split = p.num_kb;
     p.bn = cfg.tile_n;
     p.stages = cfg.stages;
-    p.tmem_cols = tmem_cols_for(cfg.tile_n);
+    p.tmem_cols = tmem_cols_for(cfg.tile_m, cfg.tile_n);
     p.a_mn_major = 0;
     p.b_mn_major = 0;
     p.alpha = 1.0f;
@@ -612,12 +626,12 @@ int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_cou
     const bool b_mn = g.transB == 0;
     tdx_config d;
     default_umma_config(ceil_div(g.M, 128), g.N, num_kb, b_mn, sm_count, smem_limit, true, &d);
-    if (c.tile_m == 0) c.tile_m = d.tile_m;
+    if (c.tile_m == 0) c.tile_m = (c.tile_n == 0 || c.tile_n == d.tile_n) ? d.tile_m : 128;
     if (c.tile_k == 0) c.tile_k = d.tile_k;
     if (c.cta_pair == 0) c.cta_pair = d.cta_pair;
     if (c.tile_n == 0) c.tile_n = d.tile_n;
     if (c.split_k == 0) c.split_k = (user && user->tile_n != 0 && user->tile_n != d.tile_n) ? 1 : d.split_k;
-    if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_n, smem_limit));
+    if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit));
     if (!user && !from_cache) c.raster = d.raster;
     const char* why = umma_config_reason(c, b_mn, num_kb, smem_limit, false);
     if (why) return fail(TDX_ERR_CONFIG, "infeasible config: %s", why);
@@ -650,12 +664,12 @@ int resolve_conv_config(const ConvProblem& cp, const tdx_config* user, int sm_co
     const int64_t num_kb = cp.R * cp.S * ceil_div(cp.Cin, 64);
     tdx_config d;
     default_umma_config(tiles_m, cp.Cout, num_kb, false, sm_count, smem_limit, false, &d);
-    if (c.tile_m == 0) c.tile_m = d.tile_m;
+    if (c.tile_m == 0) c.tile_m = (c.tile_n == 0 || c.tile_n == d.tile_n) ? d.tile_m : 128;
     if (c.tile_k == 0) c.tile_k = d.tile_k;
     if (c.cta_pair == 0) c.cta_pair = d.cta_pair;
     if (c.tile_n == 0) c.tile_n = d.tile_n;
     if (c.split_k == 0) c.split_k = 1;
-    if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_n, smem_limit));
+    if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit));
     if (!user && !from_cache) c.raster = d.raster;
     const char* why = umma_config_reason(c, false, num_kb, smem_limit, true);
     if (why) return fail(TDX_ERR_CONFIG, "infeasible config: %s", why);
@@ -750,29 +764,36 @@ int conv_dispatch(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, in
 // ------------------------------------------------------------------ search space
 void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int sm_count, int smem_limit, bool conv,
                      std::vector<tdx_config>* out) {
-    for (int bn : {256, 128, 64, 32}) {
-        if (b_mn && bn % 64) continue;
-        if (bn > 32 && bn / 2 >= N + 31) continue;   // a tile more than twice as wide as the problem only wastes work
-        const int max_st = umma_max_stages(bn, smem_limit);
-        std::vector<int> stage_opts;
-        stage_opts.push_back(max_st);
-        if (max_st - 2 >= 3) stage_opts.push_back(max_st - 2);
-        const int64_t tiles = tiles_m * ceil_div(N, bn);
-        std::vector<int> splits{1};
-        if (!conv && tiles < 2LL * sm_count)
-            for (int s : {2, 3, 4, 6, 8, 16})
-                if (num_kb / s >= 2 && tiles * s <= 4LL * sm_count) splits.push_back(s);
-        for (int st : stage_opts)
-            for (int sk : splits)
-                for (int raster : {0, 8, 2}) {
-                    if (raster != 0 && tiles_m <= raster) continue;
-                    tdx_config c;
-                    std::memset(&c, 0, sizeof c);
-                    c.kernel = TDX_KERNEL_UMMA;
-                    c.tile_m = 128; c.tile_n = bn; c.tile_k = 64; c.stages = st; c.cta_pair = 1;
-                    c.split_k = sk; c.store_mode = 0; c.raster = raster;
-                    if (umma_config_reason(c, b_mn, num_kb, smem_limit, conv) == nullptr) out->push_back(c);
-                }
+    for (int tm : {256, 128}) {
+        const int64_t tiles_m_t = ceil_div(tiles_m, tm / 128);
+        for (int bn = 256; bn >= 32; bn -= 32) {
+            if (b_mn && bn % 64) continue;
+            if (bn > 32 && bn - 32 >= N) continue;        // a narrower tile already covers N
+            if (bn != 256 && bn != 128 && bn != 64 && bn != 32 && N % bn && ceil_div(N, bn) == ceil_div(N, bn + 32))
+                continue;                                 // odd widths only where they change the tile count
+            const int max_st = umma_max_stages(tm, bn, smem_limit);
+            if (max_st < 2) continue;
+            std::vector<int> stage_opts;
+            stage_opts.push_back(max_st);
+            if (max_st - 2 >= 3) stage_opts.push_back(max_st - 2);
+            const int64_t tiles = tiles_m_t * ceil_div(N, bn);
+            if (tm == 256 && tiles < sm_count / 2) continue;   // too few tiles to be worth the taller tile
+            std::vector<int> splits{1};
+            if (!conv && tiles < 2LL * sm_count)
+                for (int s : {2, 3, 4, 6, 8, 16})
+                    if (num_kb / s >= 2 && tiles * s <= 4LL * sm_count) splits.push_back(s);
+            for (int st : stage_opts)
+                for (int sk : splits)
+                    for (int raster : {0, 8, 2, 4, 16}) {
+                        if (raster != 0 && tiles_m_t <= raster) continue;
+                        tdx_config c;
+                        std::memset(&c, 0, sizeof c);
+                        c.kernel = TDX_KERNEL_UMMA;
+                        c.tile_m = tm; c.tile_n = bn; c.tile_k = 64; c.stages = st; c.cta_pair = 1;
+                        c.split_k = sk; c.store_mode = 0; c.raster = raster;
+                        if (umma_config_reason(c, b_mn, num_kb, smem_limit, conv) == nullptr) out->push_back(c);
+                    }
+        }
     }
 }
 

@@ -1,13 +1,17 @@
 // Persistent, warp-specialised tcgen05 contraction kernel (bf16 x bf16 -> fp32 in TMEM).
 //
-// One CTA owns a stream of 128 x BN output tiles.  Roles:
+// One CTA owns a stream of BM x BN output tiles (BM = 128 or 256).  Roles:
 //   warp 0 (one lane)  TMA producer: fills a ring of shared-memory stages, each holding a
-//                      128 x 64 slice of op(A) and a 64 x BN slice of op(B), 128-byte swizzled.
-//   warp 1 (one lane)  MMA issuer: per stage four tcgen05.mma (K = 16 each) into one of two
-//                      TMEM accumulators; tcgen05.commit releases the stage / publishes the tile.
-//   warps 2..5         epilogue: tcgen05.ld the accumulator (one row per thread), apply
-//                      alpha / bias / ReLU, convert, store 16 bytes at a time.
-// The second accumulator lets the epilogue of tile t overlap the main loop of tile t+1.
+//                      BM x 64 slice of op(A) and a 64 x BN slice of op(B), 128-byte swizzled.
+//   warp 1 (one lane)  MMA issuer: per stage and per 128-row half four tcgen05.mma (K = 16
+//                      each) into a TMEM accumulator slot; tcgen05.commit releases the stage /
+//                      publishes the tile.
+//   warps 2..5 (6..9)  epilogue of the first (second) 128-row half: tcgen05.ld the accumulator
+//                      (one row per thread), apply alpha / bias / ReLU, convert, store 16 bytes
+//                      at a time.
+// TMEM holds 2 or 4 accumulator slots of 128 x BN; when a tile leaves slots free, the epilogue
+// of tile t overlaps the main loop of tile t+1.  A 256-row tile halves the operand bytes fetched
+// from L2 per flop (the B slice is shared by both halves), which is what bounds the 128-row tile.
 //
 // Operand transposes are never materialised: a K-major operand is loaded as one box of
 // (64 k) x (rows); an MN-major operand as boxes of (64 mn) x (64 k), and the MMA
@@ -24,12 +28,12 @@
 
 namespace tdx {
 
-constexpr int kBM = 128;          // tile rows = TMEM lanes
+constexpr int kHalfM = 128;       // rows of one MMA / one accumulator slot = TMEM lanes
 constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaK = 16;        // K of one tcgen05.mma for 16-bit inputs
-constexpr int kUmmaThreads = 192;
 constexpr int kMaxStages = 8;
-constexpr int kABytes = kBM * kBK * 2;                 // 16 KiB
+constexpr int kMaxSlots = 4;
+constexpr int kHalfABytes = kHalfM * kBK * 2;          // 16 KiB: one 128-row half of the A slice
 constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at boost clock
 
 enum : int { kTimeoutProducer = 1, kTimeoutMma = 2, kTimeoutEpilogue = 3 };
@@ -39,7 +43,8 @@ struct UmmaParams {
     int num_kb;               // K blocks of 64 in the whole reduction
     int tiles_m, tiles_n, panel;
     int split_k, kb_per_split;
-    int bn, stages, tmem_cols;
+    int bm, bn, stages, tmem_cols;   // bm = 128 or 256
+    int slots;                        // accumulator slots of 128 x bn in TMEM (2 or 4)
     int a_mn_major, b_mn_major;
     float alpha;
     const float* bias;        // [N] or nullptr
@@ -49,7 +54,7 @@ struct UmmaParams {
     float* partial;           // split-K: [split][M][N] fp32
     int vec_store;            // rows of C / partial are 16-byte aligned and N % 8 == 0
     // convolution geometry (kConv only)
-    int bw, bh, nb;           // spatial patch (bw x bh output pixels), patches per tile
+    int bw, bh, nb;           // spatial patch (bw x bh output pixels), patches per tile = bm / (bw*bh)
     int patches_w, patches_h; // patches per image along Q and P
     int P, Q, Nimg, S, pad, cchunks;
     int* status;              // device status word
@@ -94,14 +99,14 @@ __device__ __forceinline__ TileCoord decode_item(const UmmaParams& p, int item) 
 }
 
 template <bool kConv>
-__global__ void __launch_bounds__(kUmmaThreads, 1)
+__global__ void __launch_bounds__(320, 1)
 umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
     __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
-    __shared__ __align__(8) uint64_t tfull_bar[2];
-    __shared__ __align__(8) uint64_t tempty_bar[2];
+    __shared__ __align__(8) uint64_t tfull_bar[kMaxSlots];
+    __shared__ __align__(8) uint64_t tempty_bar[kMaxSlots];
     __shared__ uint32_t s_tmem_base;
     __shared__ int s_abort;
 
@@ -109,7 +114,9 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t b_bytes = static_cast<uint32_t>(p.bn) * 128u;
-    const uint32_t stage_bytes = kABytes + b_bytes;
+    const int mh = p.bm / kHalfM;                      // 128-row halves per tile
+    const uint32_t a_bytes = static_cast<uint32_t>(mh) * kHalfABytes;
+    const uint32_t stage_bytes = a_bytes + b_bytes;
     volatile int* abort_flag = &s_abort;
 
     if (threadIdx.x == 0) {
@@ -117,7 +124,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             ptx::mbar_init(&full_bar[s], 1);
             ptx::mbar_init(&empty_bar[s], 1);
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < p.slots; ++b) {
             ptx::mbar_init(&tfull_bar[b], 1);
             ptx::mbar_init(&tempty_bar[b], 4);
         }
@@ -153,7 +160,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     uint64_t* bar = &full_bar[stage];
                     ptx::mbar_arrive_expect_tx(bar, stage_bytes);
                     uint8_t* a_dst = smem + static_cast<size_t>(stage) * stage_bytes;
-                    uint8_t* b_dst = a_dst + kABytes;
+                    uint8_t* b_dst = a_dst + a_bytes;
                     if (kConv) {
                         const int tap = kb / p.cchunks;
                         const int cc = kb - tap * p.cchunks;
@@ -173,10 +180,12 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         ptx::tma_load_3d(b_dst, &tmB, bar, cc * kBK, tap, t.n_blk * p.bn);
                     } else {
                         if (p.a_mn_major) {
-                            ptx::tma_load_2d(a_dst, &tmA, bar, t.m_blk * kBM, kb * kBK);
-                            ptx::tma_load_2d(a_dst + 8192, &tmA, bar, t.m_blk * kBM + 64, kb * kBK);
+                            for (int i = 0; i < 2 * mh; ++i)
+                                ptx::tma_load_2d(a_dst + i * 8192, &tmA, bar, t.m_blk * p.bm + i * 64, kb * kBK);
                         } else {
-                            ptx::tma_load_2d(a_dst, &tmA, bar, kb * kBK, t.m_blk * kBM);
+                            for (int h = 0; h < mh; ++h)
+                                ptx::tma_load_2d(a_dst + h * kHalfABytes, &tmA, bar, kb * kBK,
+                                                 t.m_blk * p.bm + h * kHalfM);
                         }
                         if (p.b_mn_major) {
                             for (int i = 0; i < p.bn / 64; ++i)
@@ -199,7 +208,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = ptx::make_idesc_bf16_f32(kBM, p.bn, p.a_mn_major, p.b_mn_major);
+            const uint32_t idesc = ptx::make_idesc_bf16_f32(kHalfM, p.bn, p.a_mn_major, p.b_mn_major);
             // K-major: 8-row groups are 1024 B apart (SBO); K advances 32 B inside the swizzle row.
             // MN-major: 64-element groups along MN are one 64 x 64 box (8192 B) apart (LBO),
             //           8-k groups are 1024 B apart (SBO); K advances 16 rows = 2048 B.
@@ -213,11 +222,22 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             bool ok = true;
             for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++local) {
                 const TileCoord t = decode_item(p, item);
-                const int buf = local & 1;
-                const uint32_t aphase = (local >> 1) & 1;
-                if (!wait_bounded(&tempty_bar[buf], aphase ^ 1u, abort_flag, p.status, kTimeoutMma)) break;
+                // accumulator slots of this tile: use number u of slot s has barrier phase (u & 1)
+                uint32_t d_tmem[2] = {0u, 0u};
+                int slot[2] = {0, 0};
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (h < mh && ok) {
+                        const int idx = local * mh + h;
+                        slot[h] = idx % p.slots;
+                        const uint32_t aphase = (idx / p.slots) & 1;
+                        d_tmem[h] = tmem_base + static_cast<uint32_t>(slot[h] * p.bn);
+                        if (!wait_bounded(&tempty_bar[slot[h]], aphase ^ 1u, abort_flag, p.status, kTimeoutMma))
+                            ok = false;
+                    }
+                }
+                if (!ok) break;
                 ptx::tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(buf * p.bn);
                 for (int kb = t.kb0; kb < t.kb1; ++kb) {
                     if (!wait_bounded(&full_bar[stage], phase, abort_flag, p.status, kTimeoutMma)) {
                         ok = false;
@@ -225,12 +245,18 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     }
                     ptx::tc_fence_after_sync();
                     const uint32_t a_addr = ptx::smem_u32(smem + static_cast<size_t>(stage) * stage_bytes);
-                    const uint32_t b_addr = a_addr + kABytes;
+                    const uint32_t b_addr = a_addr + a_bytes;
 #pragma unroll
-                    for (int j = 0; j < kBK / kUmmaK; ++j) {
-                        const uint64_t adesc = ptx::make_smem_desc_sw128(a_addr + j * a_kstep, a_lbo, 1024u);
-                        const uint64_t bdesc = ptx::make_smem_desc_sw128(b_addr + j * b_kstep, b_lbo, 1024u);
-                        ptx::umma_bf16(d_tmem, adesc, bdesc, idesc, (kb > t.kb0 || j > 0) ? 1u : 0u);
+                    for (int h = 0; h < 2; ++h) {
+                        if (h < mh) {
+#pragma unroll
+                            for (int j = 0; j < kBK / kUmmaK; ++j) {
+                                const uint64_t adesc =
+                                    ptx::make_smem_desc_sw128(a_addr + h * kHalfABytes + j * a_kstep, a_lbo, 1024u);
+                                const uint64_t bdesc = ptx::make_smem_desc_sw128(b_addr + j * b_kstep, b_lbo, 1024u);
+                                ptx::umma_bf16(d_tmem[h], adesc, bdesc, idesc, (kb > t.kb0 || j > 0) ? 1u : 0u);
+                            }
+                        }
                     }
                     ptx::umma_commit(&empty_bar[stage]);
                     if (++stage == p.stages) {
@@ -238,18 +264,23 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         phase ^= 1u;
                     }
                 }
-                if (ok) ptx::umma_commit(&tfull_bar[buf]);
+                if (ok) {
+                    ptx::umma_commit(&tfull_bar[slot[0]]);
+                    if (mh == 2) ptx::umma_commit(&tfull_bar[slot[1]]);
+                }
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (4 warps)
+        // ------------------------------------------------------------ epilogue (4 warps per 128-row half)
+        const int half = (warp - 2) >> 2;             // which 128-row half of the tile this warp group drains
         const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
-        const int row_in_tile = quarter * 32 + lane;
+        const int row_in_tile = half * kHalfM + quarter * 32 + lane;
         int local = 0;
         for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++local) {
             const TileCoord t = decode_item(p, item);
-            const int buf = local & 1;
-            const uint32_t aphase = (local >> 1) & 1;
+            const int sidx = local * mh + half;
+            const int buf = sidx % p.slots;
+            const uint32_t aphase = (sidx / p.slots) & 1;
             if (!wait_bounded(&tfull_bar[buf], aphase, abort_flag, p.status, kTimeoutEpilogue)) break;
             ptx::tc_fence_after_sync();
 
@@ -272,7 +303,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 valid = (n < p.Nimg) && (pp < p.P) && (qq < p.Q);
                 grow = (static_cast<long long>(n) * p.P + pp) * p.Q + qq;
             } else {
-                grow = static_cast<long long>(t.m_blk) * kBM + row_in_tile;
+                grow = static_cast<long long>(t.m_blk) * p.bm + row_in_tile;
                 valid = grow < p.M;
             }
 

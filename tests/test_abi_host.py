@@ -66,7 +66,8 @@ def test_conv_argument_validation():
 
 def test_infeasible_explicit_config_is_reported_before_any_device_work():
     base = dict(M=256, N=256, K=256, transA=0, transB=1, alpha=1.0, dtype=tdx.TDX_BF16, A=256, B=512, C=1024)
-    for kw in [dict(tile_n=48), dict(tile_n=512), dict(stages=9), dict(tile_m=64), dict(split_k=7),
+    for kw in [dict(tile_n=48), dict(tile_n=512), dict(stages=9), dict(tile_m=64), dict(tile_m=384), dict(tile_m=256, tile_n=256, stages=4),
+               dict(split_k=7),
                dict(tile_k=32), dict(cta_pair=3), dict(kernel=9), dict(kernel=tdx.TDX_KERNEL_SIMT)]:
         cfg = tdx.tdx_config(kernel=kw.pop("kernel", tdx.TDX_KERNEL_UMMA), **kw)
         assert tdx.tdx_gemm_ex(**base, cfg=cfg) == tdx.TDX_ERR_CONFIG, kw
@@ -107,11 +108,11 @@ def test_gemm_search_space_obeys_constraints(shape):
         key = tuple(c.values())
         assert key not in seen
         seen.add(key)
-        assert c["kernel"] == tdx.TDX_KERNEL_UMMA and c["tile_m"] == 128 and c["tile_k"] == 64
+        assert c["kernel"] == tdx.TDX_KERNEL_UMMA and c["tile_m"] in (128, 256) and c["tile_k"] == 64
         assert c["tile_n"] % 64 == 0                          # B is read N-major here
         assert 2 <= c["stages"] <= 8
-        assert c["stages"] * (16384 + c["tile_n"] * 128) + 1024 + 512 <= SMEM_LIMIT
-        assert 2 * c["tile_n"] <= 512                          # two TMEM accumulators
+        assert c["stages"] * (c["tile_m"] + c["tile_n"]) * 128 + 1024 + 512 <= SMEM_LIMIT
+        assert (c["tile_m"] // 128) * c["tile_n"] <= 512      # one tile's accumulators fit in TMEM
         per = -(-num_kb // c["split_k"])
         assert (c["split_k"] - 1) * per < num_kb               # no empty K slice
     if M * N <= 128 * 8192:
@@ -137,6 +138,7 @@ def test_search_space_for_other_kernels():
 def test_default_configs():
     st, c = tdx.tdx_default_gemm_config(4096, 4096, 4096, 0, 1, tdx.TDX_BF16)
     assert st == tdx.TDX_OK and c.kernel == tdx.TDX_KERNEL_UMMA and c.tile_n == 256 and c.split_k == 1
+    assert c.tile_m == 256 and c.stages == 3                 # 3 x 64 KiB stages fit in shared memory
     st, c = tdx.tdx_default_gemm_config(128, 8192, 8192, 0, 0, tdx.TDX_BF16)
     assert st == tdx.TDX_OK and c.split_k > 1
     st, c = tdx.tdx_default_gemm_config(256, 256, 256, 0, 0, tdx.TDX_F32)

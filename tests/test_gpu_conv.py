@@ -74,6 +74,16 @@ def test_conv_patch_shapes(patch):
     assert conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y) < TIGHT["bf16"]
 
 
+@pytest.mark.parametrize("cfgkw", [dict(tile_n=64, patch_w=8, patch_h=8), dict(tile_n=128, patch_w=16, patch_h=8),
+                                   dict(tile_n=256, patch_w=128, patch_h=1)])
+def test_conv_256_row_tiles(cfgkw):
+    N, H, W, Cin, Cout = 3, 24, 40, 128, 200
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=77)
+    st, y, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, cfg=umma(tile_m=256, **cfgkw))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y) < TIGHT["bf16"]
+
+
 def test_conv_padding_equals_explicit_zero_padded_copy_bitwise():
     # the copy engine's zero fill and explicit zeros feed the same products in the same order
     N, H, W, Cin, Cout, pad = 2, 16, 24, 64, 64, 1

@@ -95,6 +95,31 @@ def test_umma_explicit_tile_configs(cfgkw):
     assert err < TIGHT["bf16"], err
 
 
+@pytest.mark.parametrize("transA,transB", [(0, 1), (0, 0), (1, 1), (1, 0)])
+@pytest.mark.parametrize("cfgkw", [dict(tile_n=256, stages=3), dict(tile_n=128, stages=2), dict(tile_n=64, stages=5),
+                                   dict(tile_n=192, stages=2, raster=2)])
+def test_umma_256_row_tiles(cfgkw, transA, transB):
+    # 256-row tiles: two 128-row halves share each B slice; 2 or 4 TMEM accumulator slots
+    M, N, K = 904, 520, 328          # 4 row tiles with a ragged last one, ragged N and K tails
+    A, B = si.gemm_bf16_normal(M, N, K, seed=62, transA=transA, transB=transB)
+    st, C, ok = run_gemm(M, N, K, transA, transB, 1.0, "bf16", A, B, cfg=umma(tile_m=256, **cfgkw))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    err = gemm_error(M, N, K, transA, transB, 1.0, "bf16", A, B, C)
+    assert err < TIGHT["bf16"], err
+
+
+def test_umma_256_row_tiles_exact_integers_many_tiles_per_cta():
+    # more tiles than SMs, so every CTA walks several tiles and the accumulator slots wrap around
+    M, N, K = 256 * 20, 64 * 16, 128
+    A = si.small_integers(63, 0, (M, K), "bf16", -1, 1)
+    B = si.small_integers(63, 1, (N, K), "bf16", -1, 1)
+    for cfgkw in (dict(tile_m=256, tile_n=64), dict(tile_m=256, tile_n=256), dict(tile_m=128, tile_n=32)):
+        st, C, ok = run_gemm(M, N, K, 0, 1, 1.0, "bf16", A, B, cfg=umma(**cfgkw))
+        assert st == 0 and ok, tdx.tdx_last_error()
+        ref = oracle.gemm(M, N, K, 0, 1, 1.0, "bf16", A, B)
+        assert np.array_equal(oracle.decode(C, "bf16"), ref), cfgkw
+
+
 @pytest.mark.parametrize("split", [2, 3, 5])
 @pytest.mark.parametrize("transB", [0, 1])
 def test_umma_split_k_with_workspace(split, transB):
