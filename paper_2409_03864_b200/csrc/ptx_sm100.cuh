@@ -46,7 +46,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 
 // ---------------------------------------------------------------- TMA loads
 // Tile-mode bulk tensor loads global -> shared, completion signalled on an
-// mbarrier as transferred bytes.  No multicast is used anywhere.
+// mbarrier as transferred bytes.  Every load targets the issuing CTA only.
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
