@@ -181,6 +181,39 @@ int tdx_tune_clear(void);
  */
 int tdx_check_device_status(void* stream);
 
+/*
+ * Split-K GEMM for callers that must not allocate device memory.  (The paper has no counterpart to
+ * this entry point; it exists for integration reasons only.)
+ *
+ * Who needs it: code that runs where a device allocation is off limits -- a serving loop whose memory
+ * was sized and handed out once at start-up, a plug-in living inside another framework's memory pool
+ * (a raw cudaMalloc there bypasses the pool's accounting and, like cudaFree, stalls every stream of
+ * the device while it runs), or a latency-critical step that cannot afford that stall.  tdx_gemm
+ * may grow an internal split-K workspace with cudaMalloc and tdx_gemm_ex wants a workspace from the
+ * caller; this call needs neither.
+ *
+ * It computes exactly what tdx_gemm_ex computes for dtype TDX_BF16 with cfg = {kernel = UMMA,
+ * tile_m = 128, tile_n as given (0 = choose), split_k as given}: C = alpha * op(A) . op(B), partial
+ * sums of the split_k K-slices reduced in a fixed order.  The partials live in a fixed array of
+ * TDX_STATIC_SCRATCH_BYTES that is part of the library image: every GPU that loads the library holds
+ * those bytes until the process exits, whether or not this function is ever called.
+ *
+ *   split_k >= 1;  split_k * M * N * 4 bytes must not exceed TDX_STATIC_SCRATCH_BYTES, else
+ *   TDX_ERR_WORKSPACE (nothing launched, C untouched).  Layout rules are those of the tensor-core
+ *   path (16-byte aligned pointers, contiguous dimensions multiples of 8): a shape that misses them
+ *   gets TDX_ERR_ALIGNMENT rather than another kernel.
+ *   The first call on each device looks up the array's device address (no allocation); make that
+ *   first call outside any stream capture.
+ *   The call itself performs no cudaMalloc / cudaFree and uses no allocating library routine.
+ *   All calls share the one array and it keeps whatever the previous call left there.  Nothing in it
+ *   needs to start at zero: each call writes every partial it later reads.  Two calls whose kernels
+ *   may overlap on the GPU (different streams, no dependency between them) race on the array --
+ *   order them on one stream or with events.
+ */
+#define TDX_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
+int tdx_gemm_splitk_static(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha,
+                           const void* A, const void* B, void* C, int tile_n, int split_k, void* stream);
+
 /* Number of kernels this library has launched in this process (all threads). */
 int64_t tdx_kernel_launch_count(void);
 

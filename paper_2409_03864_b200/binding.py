@@ -82,6 +82,7 @@ def lib() -> ctypes.CDLL:
         L.tdx_tune_save.argtypes = [ctypes.c_char_p]
         L.tdx_tune_load.argtypes = [ctypes.c_char_p]
         L.tdx_tune_clear.argtypes = []
+        L.tdx_gemm_splitk_static.argtypes = [i64, i64, i64, ci, ci, cf, vp, vp, vp, ci, ci, vp]
         L.tdx_check_device_status.argtypes = [vp]
         L.tdx_kernel_launch_count.argtypes = []
         L.tdx_kernel_launch_count.restype = i64
@@ -100,7 +101,7 @@ EXPORTS = (
     "tdx_gemm", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_relu_ex",
     "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
     "tdx_enum_conv2d_configs", "tdx_default_gemm_config", "tdx_default_conv2d_config", "tdx_tune_save",
-    "tdx_tune_load", "tdx_tune_clear", "tdx_check_device_status", "tdx_kernel_launch_count", "tdx_last_error",
+    "tdx_tune_load", "tdx_tune_clear", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_kernel_launch_count", "tdx_last_error",
     "tdx_version",
 )
 
@@ -244,6 +245,18 @@ def tdx_tune_load(path: str) -> int:
 
 def tdx_tune_clear() -> int:
     return lib().tdx_tune_clear()
+
+
+TDX_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
+
+
+def tdx_gemm_splitk_static(M, N, K, transA, transB, alpha, A, B, C, tile_n=0, split_k=2, stream=None) -> int:
+    """bf16 split-K GEMM that allocates no device memory: its partial sums live in a fixed
+    TDX_STATIC_SCRATCH_BYTES array inside the library, for callers that may not call cudaMalloc
+    (fixed memory budgets, code living inside another allocator's pool).  Calls that can overlap
+    on the GPU race on that array; keep them ordered on one stream."""
+    return lib().tdx_gemm_splitk_static(M, N, K, transA, transB, alpha, _ptr(A), _ptr(B), _ptr(C), tile_n, split_k,
+                                        _stream(stream))
 
 
 def tdx_check_device_status(stream=None) -> int:

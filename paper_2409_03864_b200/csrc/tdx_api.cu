@@ -1220,6 +1220,140 @@ int tdx_check_device_status(void* stream) {
 
 int64_t tdx_kernel_launch_count(void) { return g_launches.load(); }
 
+}  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// tdx_gemm_splitk_static: split-K GEMM whose partial sums live in an array that is part of the
+// library image, for callers that must not allocate device memory (see include/tdx.h).
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+// The scratch itself.  In host code this name is only a handle for the runtime's symbol table, not
+// an address a kernel can use; the device address is fetched once per device below.
+static __device__ __align__(256) float g_static_splitk_scratch[TDX_STATIC_SCRATCH_BYTES / sizeof(float)];
+
+constexpr int kMaxStaticDevices = 64;
+float* g_static_scratch_ptr[kMaxStaticDevices] = {};   // device address of the array, per device ordinal
+std::mutex g_static_mu;
+
+// Device address of the scratch array on the current device (looked up on first use, then cached).
+int static_scratch_address(int dev, float** out) {
+    if (dev < 0 || dev >= kMaxStaticDevices) return fail(TDX_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    if (g_static_scratch_ptr[dev] == nullptr) {
+        float* ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_splitk_scratch);
+        if (e != cudaSuccess || ptr == nullptr)
+            return fail(TDX_ERR_CUDA, "cudaGetSymbolAddress(static scratch): %s", cudaGetErrorString(e));
+        g_static_scratch_ptr[dev] = ptr;
+    }
+    *out = g_static_scratch_ptr[dev];
+    return TDX_OK;
+}
+
+// bf16 2-D tensor map, built on the spot (no cache, no heap).
+int encode_map_2d(DeviceCtx* ctx, const void* ptr, uint64_t inner, uint64_t outer, uint32_t box_inner,
+                  uint32_t box_outer, CUtensorMap* out) {
+    cuuint64_t gdim[2] = {inner, outer};
+    cuuint64_t gstr[1] = {inner * 2};
+    cuuint32_t gbox[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstr, gbox, estr,
+                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(TDX_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d)", static_cast<int>(r));
+    return TDX_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int tdx_gemm_splitk_static(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, const void* A,
+                           const void* B, void* C, int tile_n, int split_k, void* stream) {
+    int rc = validate_gemm(M, N, K, transA, transB, TDX_BF16, A, B, C, true);
+    if (rc) return rc;
+    if (split_k < 1 || tile_n < 0) return fail(TDX_ERR_INVALID_ARG, "split_k must be >= 1 and tile_n >= 0");
+    if (M == 0 || N == 0) return TDX_OK;
+    if (K == 0) return fail(TDX_ERR_UNSUPPORTED, "K = 0: use tdx_gemm");
+    // size check first: it needs no device
+    const double need = static_cast<double>(split_k) * static_cast<double>(M) * static_cast<double>(N) * 4.0;
+    if (split_k > 1 && need > static_cast<double>(TDX_STATIC_SCRATCH_BYTES))
+        return fail(TDX_ERR_WORKSPACE,
+                    "split_k * M * N * 4 = %.0f bytes exceeds the static scratch of %u bytes (TDX_STATIC_SCRATCH_BYTES)",
+                    need, TDX_STATIC_SCRATCH_BYTES);
+    GemmProblem g{M, N, K, transA, transB, TDX_BF16};
+    if (!gemm_umma_layout_ok(g) || reinterpret_cast<uintptr_t>(A) % 16 || reinterpret_cast<uintptr_t>(B) % 16)
+        return fail(TDX_ERR_ALIGNMENT, "static split-K GEMM needs 16-byte aligned A, B and contiguous dims %% 8 == 0");
+    tdx_config want;
+    std::memset(&want, 0, sizeof want);
+    want.kernel = TDX_KERNEL_UMMA;
+    want.tile_m = 128;
+    want.tile_n = tile_n;
+    want.split_k = split_k;
+    int sm_count, smem_limit;
+    device_limits(&sm_count, &smem_limit);
+    tdx_config cfg;
+    rc = resolve_gemm_config(g, &want, sm_count, smem_limit, &cfg);
+    if (rc) return rc;
+    DeviceCtx* ctx;
+    rc = get_ctx(&ctx);
+    if (rc) return rc;
+    rc = resolve_gemm_config(g, &want, ctx->sm_count, ctx->smem_optin, &cfg);
+    if (rc) return rc;
+    float* scratch = nullptr;
+    rc = static_scratch_address(ctx->dev, &scratch);
+    if (rc) return rc;
+
+    const int64_t num_kb = ceil_div(K, 64);
+    UmmaParams p;
+    std::memset(&p, 0, sizeof p);
+    p.M = static_cast<int>(M);
+    p.N = static_cast<int>(N);
+    p.num_kb = static_cast<int>(num_kb);
+    p.bm = cfg.tile_m;
+    p.slots = tmem_slots_for(cfg.tile_m, cfg.tile_n);
+    p.tiles_m = static_cast<int>(ceil_div(M, cfg.tile_m));
+    p.tiles_n = static_cast<int>(ceil_div(N, cfg.tile_n));
+    p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
+    p.split_k = cfg.split_k;
+    p.kb_per_split = static_cast<int>(ceil_div(num_kb, cfg.split_k));
+    p.bn = cfg.tile_n;
+    p.stages = cfg.stages;
+    p.tmem_cols = tmem_cols_for(cfg.tile_m, cfg.tile_n);
+    p.a_mn_major = transA ? 1 : 0;
+    p.b_mn_major = transB ? 0 : 1;
+    p.alpha = alpha;
+    p.C = static_cast<__nv_bfloat16*>(C);
+    p.ldc = N;
+    p.status = ctx->status_ptr;
+    p.vec_store = (N % 8 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+    p.partial = cfg.split_k > 1 ? scratch : nullptr;
+
+    CUtensorMap ma, mb;
+    rc = p.a_mn_major ? encode_map_2d(ctx, A, static_cast<uint64_t>(M), static_cast<uint64_t>(K), 64, 64, &ma)
+                      : encode_map_2d(ctx, A, static_cast<uint64_t>(K), static_cast<uint64_t>(M), 64, 128, &ma);
+    if (rc) return rc;
+    rc = p.b_mn_major ? encode_map_2d(ctx, B, static_cast<uint64_t>(N), static_cast<uint64_t>(K), 64, 64, &mb)
+                      : encode_map_2d(ctx, B, static_cast<uint64_t>(K), static_cast<uint64_t>(N), 64,
+                                      static_cast<uint32_t>(cfg.tile_n), &mb);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = launch_umma(ctx, false, ma, mb, p, st);
+    if (rc) return rc;
+    if (cfg.split_k > 1) {
+        const long long MN = static_cast<long long>(M) * N;
+        const int vec8 = p.vec_store ? 1 : 0;
+        const long long work = vec8 ? MN / 8 : MN;
+        const int grid = static_cast<int>(std::min<long long>(ceil_div(work, 256), 148LL * 16));
+        tdx::splitk_reduce_kernel<<<std::max(grid, 1), 256, 0, st>>>(MN, static_cast<int>(N), cfg.split_k, scratch, alpha,
+                                                                     nullptr, 0, p.C, vec8);
+        TDX_CUDA(cudaGetLastError());
+        g_launches.fetch_add(1);
+    }
+    return TDX_OK;
+}
+
 const char* tdx_last_error(void) { return g_err.c_str(); }
 
 const char* tdx_version(void) { return "tdx 0.1.0 (sm_100a)"; }
