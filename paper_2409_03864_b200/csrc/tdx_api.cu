@@ -186,11 +186,12 @@ bool tune_lookup(const std::string& key, tdx_config* out) {
 }
 void cfg_to_ints(const tdx_config& c, int* v) {
     v[0] = c.kernel; v[1] = c.tile_m; v[2] = c.tile_n; v[3] = c.tile_k; v[4] = c.stages; v[5] = c.cta_pair;
-    v[6] = c.split_k; v[7] = c.store_mode; v[8] = c.raster; v[9] = c.patch_w; v[10] = c.patch_h;
+    v[6] = c.split_k; v[7] = c.store_mode; v[8] = c.raster; v[9] = c.patch_w; v[10] = c.patch_h; v[11] = c.k_stagger;
 }
 void ints_to_cfg(const int* v, tdx_config* c) {
     c->kernel = v[0]; c->tile_m = v[1]; c->tile_n = v[2]; c->tile_k = v[3]; c->stages = v[4]; c->cta_pair = v[5];
     c->split_k = v[6]; c->store_mode = v[7]; c->raster = v[8]; c->patch_w = v[9]; c->patch_h = v[10];
+    c->k_stagger = v[11];
 }
 
 // ------------------------------------------------------------------ problem descriptions
@@ -227,9 +228,12 @@ bool conv_umma_layout_ok(const ConvProblem& c) {
     return true;
 }
 
-int umma_max_stages(int tile_m, int tile_n, int smem_limit) {
+// Shared memory the staged (TMA-store) epilogue needs: one 32 x 64 bf16 block per epilogue warp.
+int staging_bytes_for(int tile_m, int store_mode) { return store_mode == 2 ? (tile_m / 128) * 4 * 4096 : 0; }
+
+int umma_max_stages(int tile_m, int tile_n, int smem_limit, int store_mode) {
     const int stage = (tile_m + tile_n) * 128;
-    int s = (smem_limit - kStaticSmemReserve - 1024) / stage;
+    int s = (smem_limit - kStaticSmemReserve - 1024 - staging_bytes_for(tile_m, store_mode)) / stage;
     return std::min(s, tdx::kMaxStages);
 }
 
@@ -244,14 +248,21 @@ int tmem_cols_for(int tile_m, int bn) {
 
 // Static feasibility of a fully specified tensor-core configuration (the search-space constraints).
 // Returns 0 when feasible, else a short reason.
-const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num_kb, int smem_limit, bool conv) {
+const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num_kb, int smem_limit, bool conv,
+                               int64_t N) {
     if (c.tile_m != 128 && c.tile_m != 256) return "tile_m must be 128 or 256";
     if (c.tile_k != 64) return "tile_k must be 64";
     if (c.cta_pair != 1) return "cta_pair must be 1";
-    if (c.store_mode != 0) return "store_mode must be 0";
+    if (c.store_mode != 1 && c.store_mode != 2) return "store_mode must be 1 (direct) or 2 (TMA store)";
+    if (c.store_mode == 2) {
+        if (c.tile_n % 64) return "the TMA-store epilogue needs tile_n % 64 == 0";
+        if (N % 8) return "the TMA-store epilogue needs an output row pitch that is a multiple of 16 bytes";
+        if (c.split_k > 1) return "split-K writes fp32 partials directly: use store_mode 1";
+        if (conv && c.patch_w * c.patch_h < 32) return "the TMA-store epilogue needs patches of at least 32 pixels";
+    }
     if (c.tile_n < 32 || c.tile_n > 256 || c.tile_n % 32) return "tile_n must be a multiple of 32 in [32, 256]";
     if (b_mn_major && c.tile_n % 64) return "tile_n must be a multiple of 64 when B is read N-major";
-    if (c.stages < 2 || c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit)) return "stages outside the shared-memory budget";
+    if (c.stages < 2 || c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode)) return "stages outside the shared-memory budget";
     if (c.split_k < 1) return "split_k must be >= 1";
     if (conv && c.split_k != 1) return "conv has no split-K";
     if (c.split_k > 1) {
@@ -259,6 +270,7 @@ const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num
         if ((c.split_k - 1) * per >= num_kb) return "split_k leaves an empty K slice";
     }
     if (c.raster < 0) return "raster must be >= 0";
+    if (c.k_stagger != 0 && c.k_stagger != 1) return "k_stagger must be 0 or 1";
     return nullptr;
 }
 
@@ -291,7 +303,7 @@ void default_umma_config(int64_t tiles_m, int64_t N, int64_t num_kb, bool b_mn_m
     c->tile_m = 128;
     c->tile_k = 64;
     c->cta_pair = 1;
-    c->store_mode = 0;
+    c->store_mode = 1;
     c->split_k = 1;
     const int min_bn = b_mn_major ? 64 : 32;
     int bn = 0, tm = 128;
@@ -318,21 +330,24 @@ void default_umma_config(int64_t tiles_m, int64_t N, int64_t num_kb, bool b_mn_m
     }
     c->tile_m = tm;
     c->tile_n = bn;
-    c->stages = std::max(2, umma_max_stages(tm, bn, smem_limit));
+    // staged epilogue whenever the layout allows it (whole-line writes instead of 16-byte pieces)
+    if (c->split_k == 1 && bn % 64 == 0 && N % 8 == 0) c->store_mode = 2;
+    c->stages = std::max(2, umma_max_stages(tm, bn, smem_limit, c->store_mode));
     c->raster = 8;
 }
 
 // ------------------------------------------------------------------ launches
-int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensorMap& mb, const UmmaParams& p,
-                cudaStream_t st) {
+int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
+                const UmmaParams& p, cudaStream_t st) {
     const long long items = static_cast<long long>(p.tiles_m) * p.tiles_n * p.split_k;
     const int grid = static_cast<int>(std::min<long long>(items, ctx->sm_count));
-    const size_t smem = static_cast<size_t>(p.stages) * ((p.bm + p.bn) * 128) + 1024;
+    const size_t smem = static_cast<size_t>(p.stages) * ((p.bm + p.bn) * 128) + 1024 +
+                        staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
     const int threads = p.bm == 256 ? 320 : 192;   // producer warp, MMA warp, 4 epilogue warps per 128-row half
     if (conv)
-        tdx::umma_contract_kernel<true><<<grid, threads, smem, st>>>(ma, mb, p);
+        tdx::umma_contract_kernel<true><<<grid, threads, smem, st>>>(ma, mb, mc, p);
     else
-        tdx::umma_contract_kernel<false><<<grid, threads, smem, st>>>(ma, mb, p);
+        tdx::umma_contract_kernel<false><<<grid, threads, smem, st>>>(ma, mb, mc, p);
     TDX_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     return TDX_OK;
@@ -365,6 +380,7 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
     p.split_k = cfg.split_k;
     p.kb_per_split = static_cast<int>(ceil_div(num_kb, cfg.split_k));
+    p.k_stagger = cfg.k_stagger;
     p.bn = cfg.tile_n;
     p.stages = cfg.stages;
     p.tmem_cols = tmem_cols_for(cfg.tile_m, cfg.tile_n);
@@ -416,7 +432,16 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     }
     if (rc) return rc;
 
-    rc = launch_umma(ctx, false, ma, mb, p, st);
+    CUtensorMap mc = ma;   // unused unless the staged epilogue is on
+    p.tma_store = (cfg.store_mode == 2 && cfg.split_k == 1 && p.vec_store) ? 1 : 0;
+    if (p.tma_store) {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.M)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
+        uint32_t box[2] = {64, 32};
+        rc = get_tensor_map(ctx, C, 2, dims, str, box, &mc);
+        if (rc) return rc;
+    }
+    rc = launch_umma(ctx, false, ma, mb, mc, p, st);
     if (rc) return rc;
     if (cfg.split_k > 1) {
         const long long MN = static_cast<long long>(g.M) * g.N;
@@ -452,6 +477,7 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
     p.split_k = 1;
     p.kb_per_split = p.num_kb;
+    p.k_stagger = cfg.k_stagger;
     p.bn = cfg.tile_n;
     p.stages = cfg.stages;
     p.tmem_cols = tmem_cols_for(cfg.tile_m, cfg.tile_n);
@@ -489,7 +515,20 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
         int rc = get_tensor_map(ctx, w, 3, dims, str, box, &mb);
         if (rc) return rc;
     }
-    return launch_umma(ctx, true, ma, mb, p, st);
+    CUtensorMap mc = ma;
+    p.tma_store = (cfg.store_mode == 2 && p.vec_store && p.bw * p.bh >= 32) ? 1 : 0;
+    if (p.tma_store) {
+        p.sbx = std::min(p.bw, 32);
+        p.sby = 32 / p.sbx;
+        uint64_t dims[4] = {static_cast<uint64_t>(c.Cout), static_cast<uint64_t>(c.Q), static_cast<uint64_t>(c.P),
+                            static_cast<uint64_t>(c.N)};
+        uint64_t str[3] = {static_cast<uint64_t>(c.Cout) * 2, static_cast<uint64_t>(c.Q * c.Cout) * 2,
+                           static_cast<uint64_t>(c.P * c.Q * c.Cout) * 2};
+        uint32_t box[4] = {64, static_cast<uint32_t>(p.sbx), static_cast<uint32_t>(p.sby), 1};
+        int rc = get_tensor_map(ctx, y, 4, dims, str, box, &mc);
+        if (rc) return rc;
+    }
+    return launch_umma(ctx, true, ma, mb, mc, p, st);
 }
 
 void gemm_strides(const GemmProblem& g, long long* sa_i, long long* sa_k, long long* sb_k, long long* sb_j) {
@@ -631,9 +670,13 @@ int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_cou
     if (c.cta_pair == 0) c.cta_pair = d.cta_pair;
     if (c.tile_n == 0) c.tile_n = d.tile_n;
     if (c.split_k == 0) c.split_k = (user && user->tile_n != 0 && user->tile_n != d.tile_n) ? 1 : d.split_k;
-    if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit));
+    if (c.store_mode == 0) {
+        c.store_mode = (c.split_k == 1 && c.tile_n % 64 == 0 && g.N % 8 == 0) ? 2 : 1;
+        if (c.store_mode == 2 && c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, 2)) c.store_mode = 1;
+    }
+    if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode));
     if (!user && !from_cache) c.raster = d.raster;
-    const char* why = umma_config_reason(c, b_mn, num_kb, smem_limit, false);
+    const char* why = umma_config_reason(c, b_mn, num_kb, smem_limit, false, g.N);
     if (why) return fail(TDX_ERR_CONFIG, "infeasible config: %s", why);
     *out = c;
     return TDX_OK;
@@ -669,9 +712,13 @@ int resolve_conv_config(const ConvProblem& cp, const tdx_config* user, int sm_co
     if (c.cta_pair == 0) c.cta_pair = d.cta_pair;
     if (c.tile_n == 0) c.tile_n = d.tile_n;
     if (c.split_k == 0) c.split_k = 1;
-    if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit));
+    if (c.store_mode == 0) {
+        c.store_mode = (c.tile_n % 64 == 0 && cp.Cout % 8 == 0 && c.patch_w * c.patch_h >= 32) ? 2 : 1;
+        if (c.store_mode == 2 && c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, 2)) c.store_mode = 1;
+    }
+    if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode));
     if (!user && !from_cache) c.raster = d.raster;
-    const char* why = umma_config_reason(c, false, num_kb, smem_limit, true);
+    const char* why = umma_config_reason(c, false, num_kb, smem_limit, true, cp.Cout);
     if (why) return fail(TDX_ERR_CONFIG, "infeasible config: %s", why);
     *out = c;
     return TDX_OK;
@@ -763,7 +810,7 @@ int conv_dispatch(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, in
 
 // ------------------------------------------------------------------ search space
 void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int sm_count, int smem_limit, bool conv,
-                     std::vector<tdx_config>* out) {
+                     int patch_w, int patch_h, std::vector<tdx_config>* out) {
     for (int tm : {256, 128}) {
         const int64_t tiles_m_t = ceil_div(tiles_m, tm / 128);
         for (int bn = 256; bn >= 32; bn -= 32) {
@@ -771,28 +818,35 @@ void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int 
             if (bn > 32 && bn - 32 >= N) continue;        // a narrower tile already covers N
             if (bn != 256 && bn != 128 && bn != 64 && bn != 32 && N % bn && ceil_div(N, bn) == ceil_div(N, bn + 32))
                 continue;                                 // odd widths only where they change the tile count
-            const int max_st = umma_max_stages(tm, bn, smem_limit);
-            if (max_st < 2) continue;
-            std::vector<int> stage_opts;
-            stage_opts.push_back(max_st);
-            if (max_st - 2 >= 3) stage_opts.push_back(max_st - 2);
             const int64_t tiles = tiles_m_t * ceil_div(N, bn);
             if (tm == 256 && tiles < sm_count / 2) continue;   // too few tiles to be worth the taller tile
             std::vector<int> splits{1};
             if (!conv && tiles < 2LL * sm_count)
                 for (int s : {2, 3, 4, 6, 8, 16})
                     if (num_kb / s >= 2 && tiles * s <= 4LL * sm_count) splits.push_back(s);
-            for (int st : stage_opts)
-                for (int sk : splits)
-                    for (int raster : {0, 8, 2, 4, 16}) {
-                        if (raster != 0 && tiles_m_t <= raster) continue;
-                        tdx_config c;
-                        std::memset(&c, 0, sizeof c);
-                        c.kernel = TDX_KERNEL_UMMA;
-                        c.tile_m = tm; c.tile_n = bn; c.tile_k = 64; c.stages = st; c.cta_pair = 1;
-                        c.split_k = sk; c.store_mode = 0; c.raster = raster;
-                        if (umma_config_reason(c, b_mn, num_kb, smem_limit, conv) == nullptr) out->push_back(c);
-                    }
+            for (int sk : splits)
+                for (int sm : {2, 1}) {
+                    if (sm == 2 && (sk > 1 || bn % 64 || N % 8)) continue;
+                    if (sm == 1 && sk == 1 && bn % 64 == 0 && N % 8 == 0 && tiles * tm * bn > (1 << 22))
+                        continue;                          // large outputs: 16-byte scattered stores never win
+                    const int max_st = umma_max_stages(tm, bn, smem_limit, sm);
+                    if (max_st < 2) continue;
+                    std::vector<int> stage_opts;
+                    stage_opts.push_back(max_st);
+                    if (max_st - 2 >= 3) stage_opts.push_back(max_st - 2);
+                    for (int st : stage_opts)
+                        for (int raster : {0, 8, 2, 4, 16})
+                            for (int stagger : {0, 1}) {
+                                if (raster != 0 && tiles_m_t <= raster) continue;
+                                tdx_config c;
+                                std::memset(&c, 0, sizeof c);
+                                c.kernel = TDX_KERNEL_UMMA;
+                                c.tile_m = tm; c.tile_n = bn; c.tile_k = 64; c.stages = st; c.cta_pair = 1;
+                                c.split_k = sk; c.store_mode = sm; c.raster = raster; c.k_stagger = stagger;
+                                c.patch_w = patch_w; c.patch_h = patch_h;
+                                if (umma_config_reason(c, b_mn, num_kb, smem_limit, conv, N) == nullptr) out->push_back(c);
+                            }
+                }
         }
     }
 }
@@ -819,7 +873,7 @@ int enum_gemm(const GemmProblem& g, int sm_count, int smem_limit, std::vector<td
         v->push_back(c);
         return TDX_OK;
     }
-    enum_umma_space(g.transB == 0, ceil_div(g.M, 128), g.N, ceil_div(g.K, 64), sm_count, smem_limit, false, v);
+    enum_umma_space(g.transB == 0, ceil_div(g.M, 128), g.N, ceil_div(g.K, 64), sm_count, smem_limit, false, 0, 0, v);
     return TDX_OK;
 }
 
@@ -842,9 +896,8 @@ int enum_conv(const ConvProblem& cp, int sm_count, int smem_limit, std::vector<t
             if (cost * 100 > best_cost * 115) continue;
             const int nb = 128 / (bw * bh);
             const int64_t tiles_m = ceil_div(cp.N * ceil_div(cp.Q, bw) * ceil_div(cp.P, bh), nb);
-            std::vector<tdx_config> sub;
-            enum_umma_space(false, tiles_m, cp.Cout, cp.R * cp.S * ceil_div(cp.Cin, 64), sm_count, smem_limit, true, &sub);
-            for (auto& c : sub) { c.patch_w = bw; c.patch_h = bh; v->push_back(c); }
+            enum_umma_space(false, tiles_m, cp.Cout, cp.R * cp.S * ceil_div(cp.Cin, 64), sm_count, smem_limit, true, bw, bh,
+                            v);
         }
     return TDX_OK;
 }
@@ -1141,10 +1194,10 @@ int tdx_tune_save(const char* json_path) {
     fprintf(f, "{\"version\": 1, \"entries\": [\n");
     size_t i = 0;
     for (const auto& kv : g_tune) {
-        int v[11];
+        int v[12];
         cfg_to_ints(kv.second.cfg, v);
         fprintf(f, "  {\"key\": \"%s\", \"cfg\": [", kv.first.c_str());
-        for (int j = 0; j < 11; ++j) fprintf(f, "%d%s", v[j], j < 10 ? ", " : "");
+        for (int j = 0; j < 12; ++j) fprintf(f, "%d%s", v[j], j < 11 ? ", " : "");
         fprintf(f, "], \"us\": %.3f}%s\n", kv.second.us, ++i < g_tune.size() ? "," : "");
     }
     fprintf(f, "]}\n");
@@ -1170,11 +1223,11 @@ int tdx_tune_load(const char* json_path) {
         const size_t b1 = b0 == std::string::npos ? b0 : text.find(']', b0);
         if (b1 == std::string::npos) return fail(TDX_ERR_INVALID_ARG, "malformed tuning cache %s", json_path);
         const std::string key = text.substr(q0 + 1, q1 - q0 - 1);
-        int v[11];
+        int v[12] = {0};
         int n = 0;
         const char* s = text.c_str() + b0 + 1;
         const char* end = text.c_str() + b1;
-        while (s < end && n < 11) {
+        while (s < end && n < 12) {
             char* next;
             long val = strtol(s, &next, 10);
             if (next == s) break;
@@ -1182,7 +1235,7 @@ int tdx_tune_load(const char* json_path) {
             s = next;
             while (s < end && (*s == ',' || *s == ' ')) ++s;
         }
-        if (n != 11) return fail(TDX_ERR_INVALID_ARG, "malformed cfg list in %s", json_path);
+        if (n != 11 && n != 12) return fail(TDX_ERR_INVALID_ARG, "malformed cfg list in %s", json_path);
         TuneEntry e;
         ints_to_cfg(v, &e.cfg);
         e.us = 0.0f;
@@ -1291,6 +1344,7 @@ int tdx_gemm_splitk_static(int64_t M, int64_t N, int64_t K, int transA, int tran
     want.tile_m = 128;
     want.tile_n = tile_n;
     want.split_k = split_k;
+    want.store_mode = 1;
     int sm_count, smem_limit;
     device_limits(&sm_count, &smem_limit);
     tdx_config cfg;
@@ -1318,6 +1372,7 @@ int tdx_gemm_splitk_static(int64_t M, int64_t N, int64_t K, int transA, int tran
     p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
     p.split_k = cfg.split_k;
     p.kb_per_split = static_cast<int>(ceil_div(num_kb, cfg.split_k));
+    p.k_stagger = cfg.k_stagger;
     p.bn = cfg.tile_n;
     p.stages = cfg.stages;
     p.tmem_cols = tmem_cols_for(cfg.tile_m, cfg.tile_n);
@@ -1339,7 +1394,7 @@ int tdx_gemm_splitk_static(int64_t M, int64_t N, int64_t K, int transA, int tran
                                       static_cast<uint32_t>(cfg.tile_n), &mb);
     if (rc) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    rc = launch_umma(ctx, false, ma, mb, p, st);
+    rc = launch_umma(ctx, false, ma, mb, ma, p, st);   // direct stores: the third map is unused
     if (rc) return rc;
     if (cfg.split_k > 1) {
         const long long MN = static_cast<long long>(M) * N;

@@ -7,8 +7,9 @@
 //                      each) into a TMEM accumulator slot; tcgen05.commit releases the stage /
 //                      publishes the tile.
 //   warps 2..5 (6..9)  epilogue of the first (second) 128-row half: tcgen05.ld the accumulator
-//                      (one row per thread), apply alpha / bias / ReLU, convert, store 16 bytes
-//                      at a time.
+//                      (one row per thread), apply alpha / bias / ReLU, convert, and either store
+//                      16 bytes at a time from registers or stage 32 x 64 blocks in shared memory
+//                      (128-byte swizzled) and let the copy engine write whole lines (TMA store).
 // TMEM holds 2 or 4 accumulator slots of 128 x BN; when a tile leaves slots free, the epilogue
 // of tile t overlaps the main loop of tile t+1.  A 256-row tile halves the operand bytes fetched
 // from L2 per flop (the B slice is shared by both halves), which is what bounds the 128-row tile.
@@ -43,6 +44,7 @@ struct UmmaParams {
     int num_kb;               // K blocks of 64 in the whole reduction
     int tiles_m, tiles_n, panel;
     int split_k, kb_per_split;
+    int k_stagger;            // CTAs start their K loop at different blocks (same products, rotated order)
     int bm, bn, stages, tmem_cols;   // bm = 128 or 256
     int slots;                        // accumulator slots of 128 x bn in TMEM (2 or 4)
     int a_mn_major, b_mn_major;
@@ -53,6 +55,8 @@ struct UmmaParams {
     long long ldc;
     float* partial;           // split-K: [split][M][N] fp32
     int vec_store;            // rows of C / partial are 16-byte aligned and N % 8 == 0
+    int tma_store;            // final output leaves through shared memory + TMA store (needs bn % 64 == 0)
+    int sbx, sby;             // conv TMA-store box: sbx x sby output pixels (sbx * sby = 32)
     // convolution geometry (kConv only)
     int bw, bh, nb;           // spatial patch (bw x bh output pixels), patches per tile = bm / (bw*bh)
     int patches_w, patches_h; // patches per image along Q and P
@@ -101,7 +105,7 @@ __device__ __forceinline__ TileCoord decode_item(const UmmaParams& p, int item) 
 template <bool kConv>
 __global__ void __launch_bounds__(320, 1)
 umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                     const UmmaParams p) {
+                     const __grid_constant__ CUtensorMap tmC, const UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kMaxStages];
     __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
@@ -132,6 +136,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         ptx::fence_barrier_init();
         ptx::tma_prefetch_desc(&tmA);
         ptx::tma_prefetch_desc(&tmB);
+        if (p.tma_store) ptx::tma_prefetch_desc(&tmC);
     }
     if (warp == 1) {
         __syncwarp();
@@ -152,7 +157,9 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             bool ok = true;
             for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
                 const TileCoord t = decode_item(p, item);
-                for (int kb = t.kb0; kb < t.kb1; ++kb) {
+                const int nkb = t.kb1 - t.kb0;
+                int kb = t.kb0 + (p.k_stagger ? static_cast<int>((static_cast<long long>(blockIdx.x) * nkb) / gridDim.x) : 0);
+                for (int i = 0; i < nkb; ++i, kb = (kb + 1 == t.kb1) ? t.kb0 : kb + 1) {
                     if (!wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) {
                         ok = false;
                         break;
@@ -238,7 +245,8 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 }
                 if (!ok) break;
                 ptx::tc_fence_after_sync();
-                for (int kb = t.kb0; kb < t.kb1; ++kb) {
+                const int nkb = t.kb1 - t.kb0;
+                for (int i = 0; i < nkb; ++i) {
                     if (!wait_bounded(&full_bar[stage], phase, abort_flag, p.status, kTimeoutMma)) {
                         ok = false;
                         break;
@@ -254,7 +262,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                                 const uint64_t adesc =
                                     ptx::make_smem_desc_sw128(a_addr + h * kHalfABytes + j * a_kstep, a_lbo, 1024u);
                                 const uint64_t bdesc = ptx::make_smem_desc_sw128(b_addr + j * b_kstep, b_lbo, 1024u);
-                                ptx::umma_bf16(d_tmem[h], adesc, bdesc, idesc, (kb > t.kb0 || j > 0) ? 1u : 0u);
+                                ptx::umma_bf16(d_tmem[h], adesc, bdesc, idesc, (i > 0 || j > 0) ? 1u : 0u);
                             }
                         }
                     }
@@ -307,6 +315,78 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 valid = grow < p.M;
             }
 
+            if (p.tma_store && p.split_k == 1) {
+                // ---- staged path: 32 rows x 64 columns per warp and step, written by the copy engine
+                uint8_t* stage_buf = smem + static_cast<size_t>(p.stages) * stage_bytes + (warp - 2) * 4096;
+                const int wrow0 = half * kHalfM + quarter * 32;      // first tile row of this warp
+                int sc1 = 0, sc2 = 0, sc3 = 0;                       // store coordinates above the column
+                bool box_ok;
+                if (kConv) {
+                    const int per_patch = p.bw * p.bh;
+                    const int pl = wrow0 / per_patch;
+                    const int within = wrow0 - pl * per_patch;
+                    const int hl0 = within / p.bw;
+                    const int wl0 = within - hl0 * p.bw;
+                    const int patch = t.m_blk * p.nb + pl;
+                    const int ppi = p.patches_w * p.patches_h;
+                    const int n = patch / ppi;
+                    const int rem = patch - n * ppi;
+                    const int ph = rem / p.patches_w;
+                    const int pw = rem - ph * p.patches_w;
+                    sc1 = pw * p.bw + wl0;
+                    sc2 = ph * p.bh + hl0;
+                    sc3 = n;
+                    box_ok = (n < p.Nimg) && (sc2 < p.P) && (sc1 < p.Q);
+                } else {
+                    sc1 = t.m_blk * p.bm + wrow0;
+                    box_ok = sc1 < p.M;
+                }
+                for (int c0 = 0; c0 < p.bn; c0 += 64) {
+                    uint32_t r0[32], r1[32];
+                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                                           static_cast<uint32_t>(buf * p.bn + c0);
+                    ptx::tmem_ld_32x32b_x32(taddr, r0);
+                    ptx::tmem_ld_32x32b_x32(taddr + 32, r1);
+                    ptx::tmem_ld_wait();
+                    const int col0 = t.n_blk * p.bn + c0;
+                    // the previous store of this warp must have finished reading the staging buffer
+                    if (lane == 0) ptx::tma_store_wait_read<0>();
+                    __syncwarp();
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int j = g * 8 + e * 2;
+                            float x0 = p.alpha * __uint_as_float(j < 32 ? r0[j & 31] : r1[j & 31]);
+                            float x1 = p.alpha * __uint_as_float(j + 1 < 32 ? r0[(j + 1) & 31] : r1[(j + 1) & 31]);
+                            if (p.bias != nullptr) {
+                                if (col0 + j < p.N) x0 += __ldg(p.bias + col0 + j);
+                                if (col0 + j + 1 < p.N) x1 += __ldg(p.bias + col0 + j + 1);
+                            }
+                            if (p.relu) {
+                                x0 = fmaxf(x0, 0.0f);
+                                x1 = fmaxf(x1, 0.0f);
+                            }
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
+                            pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+                        }
+                        // 128-byte swizzle: 16-byte slot g of row `lane` lives at slot g ^ (lane % 8)
+                        *reinterpret_cast<uint4*>(stage_buf + lane * 128 + ((g ^ (lane & 7)) << 4)) =
+                            make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                    ptx::fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0 && box_ok && col0 < p.N) {
+                        if (kConv)
+                            ptx::tma_store_4d(&tmC, stage_buf, col0, sc1, sc2, sc3);
+                        else
+                            ptx::tma_store_2d(&tmC, stage_buf, col0, sc1);
+                        ptx::tma_store_commit();
+                    }
+                    __syncwarp();
+                }
+            } else
             for (int c0 = 0; c0 < p.bn; c0 += 32) {
                 uint32_t r[32];
                 const uint32_t taddr =
@@ -370,6 +450,8 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&tempty_bar[buf]);
         }
+        // shared memory must stay alive until the copy engine has drained this warp's last store
+        if (p.tma_store && lane == 0) ptx::tma_store_wait_all<0>();
     }
 
     ptx::tc_fence_before_sync();

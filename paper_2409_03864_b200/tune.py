@@ -47,14 +47,14 @@ def tune_one(spec, iters):
     f = spec.split(":")
     v = [int(x) for x in f[1:]]
     if f[0] == "gemm":
-        return tdx.tdx_tune_gemm(*v, tdx.TDX_BF16, iters=iters, cap=2048)
+        return tdx.tdx_tune_gemm(*v, tdx.TDX_BF16, iters=iters, cap=8192)
     if f[0] == "conv":
-        return tdx.tdx_tune_conv2d(*v, tdx.TDX_BF16, iters=iters, cap=2048)
+        return tdx.tdx_tune_conv2d(*v, tdx.TDX_BF16, iters=iters, cap=8192)
     raise SystemExit(f"unknown workload {spec!r}")
 
 
 def brief(c):
-    s = f"m{c['tile_m']} n{c['tile_n']} st{c['stages']} sk{c['split_k']} r{c['raster']}"
+    s = f"m{c['tile_m']} n{c['tile_n']} st{c['stages']} sk{c['split_k']} r{c['raster']} ks{c['k_stagger']} sm{c['store_mode']}"
     if c["patch_w"]:
         s += f" p{c['patch_w']}x{c['patch_h']}"
     return s

@@ -68,7 +68,8 @@ def test_infeasible_explicit_config_is_reported_before_any_device_work():
     base = dict(M=256, N=256, K=256, transA=0, transB=1, alpha=1.0, dtype=tdx.TDX_BF16, A=256, B=512, C=1024)
     for kw in [dict(tile_n=48), dict(tile_n=512), dict(stages=9), dict(tile_m=64), dict(tile_m=384), dict(tile_m=256, tile_n=256, stages=4),
                dict(split_k=7),
-               dict(tile_k=32), dict(cta_pair=3), dict(kernel=9), dict(kernel=tdx.TDX_KERNEL_SIMT)]:
+               dict(tile_k=32), dict(cta_pair=3), dict(store_mode=3), dict(store_mode=2, tile_n=96),
+               dict(store_mode=2, split_k=2), dict(store_mode=2, tile_m=256, tile_n=256, stages=4), dict(kernel=9), dict(kernel=tdx.TDX_KERNEL_SIMT)]:
         cfg = tdx.tdx_config(kernel=kw.pop("kernel", tdx.TDX_KERNEL_UMMA), **kw)
         assert tdx.tdx_gemm_ex(**base, cfg=cfg) == tdx.TDX_ERR_CONFIG, kw
     # N-major B (transB=0) needs tile_n % 64 == 0
@@ -111,7 +112,11 @@ def test_gemm_search_space_obeys_constraints(shape):
         assert c["kernel"] == tdx.TDX_KERNEL_UMMA and c["tile_m"] in (128, 256) and c["tile_k"] == 64
         assert c["tile_n"] % 64 == 0                          # B is read N-major here
         assert 2 <= c["stages"] <= 8
-        assert c["stages"] * (c["tile_m"] + c["tile_n"]) * 128 + 1024 + 512 <= SMEM_LIMIT
+        assert c["store_mode"] in (1, 2)
+        staging = (c["tile_m"] // 128) * 4 * 4096 if c["store_mode"] == 2 else 0
+        assert c["stages"] * (c["tile_m"] + c["tile_n"]) * 128 + 1024 + 512 + staging <= SMEM_LIMIT
+        if c["store_mode"] == 2:
+            assert c["split_k"] == 1 and c["tile_n"] % 64 == 0
         assert (c["tile_m"] // 128) * c["tile_n"] <= 512      # one tile's accumulators fit in TMEM
         per = -(-num_kb // c["split_k"])
         assert (c["split_k"] - 1) * per < num_kb               # no empty K slice
@@ -152,14 +157,14 @@ def test_default_configs():
 def test_tuning_cache_round_trip(tmp_path):
     path = tmp_path / "cache.json"
     path.write_text('{"version": 1, "entries": [\n  {"key": "gemm:640:640:640:0:1:1", '
-                    '"cfg": [1, 128, 64, 64, 3, 1, 2, 0, 2, 0, 0], "us": 12.500}\n]}\n')
+                    '"cfg": [1, 128, 64, 64, 3, 1, 2, 1, 2, 0, 0], "us": 12.500}\n]}\n')
     assert tdx.tdx_tune_clear() == tdx.TDX_OK
     assert tdx.tdx_tune_load(str(path)) == tdx.TDX_OK
     st, c = tdx.tdx_default_gemm_config(640, 640, 640, 0, 1, tdx.TDX_BF16)
     assert st == tdx.TDX_OK and (c.tile_n, c.stages, c.split_k, c.raster) == (64, 3, 2, 2)
     out = tmp_path / "out.json"
     assert tdx.tdx_tune_save(str(out)) == tdx.TDX_OK
-    assert "gemm:640:640:640:0:1:1" in out.read_text() and "[1, 128, 64, 64, 3, 1, 2, 0, 2, 0, 0]" in out.read_text()
+    assert "gemm:640:640:640:0:1:1" in out.read_text() and "[1, 128, 64, 64, 3, 1, 2, 1, 2, 0, 0, 0]" in out.read_text()
     assert tdx.tdx_tune_clear() == tdx.TDX_OK
     st, c = tdx.tdx_default_gemm_config(640, 640, 640, 0, 1, tdx.TDX_BF16)
     assert c.tile_n != 64 or c.split_k != 2

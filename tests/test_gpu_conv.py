@@ -84,6 +84,30 @@ def test_conv_256_row_tiles(cfgkw):
     assert conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y) < TIGHT["bf16"]
 
 
+@pytest.mark.parametrize("patch", [(8, 8), (32, 1), (16, 4), (64, 2), (128, 1), (8, 4)])
+def test_conv_store_modes_agree(patch):
+    # ragged 30 x 44 maps: patches hang over the right and bottom edges and over the last image
+    N, H, W, Cin, Cout = 3, 30, 44, 64, 128
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=79)
+    outs = []
+    for sm in (1, 2):
+        st, y, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1,
+                             cfg=umma(patch_w=patch[0], patch_h=patch[1], tile_n=64, store_mode=sm))
+        assert st == 0 and ok, tdx.tdx_last_error()
+        assert conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y) < TIGHT["bf16"]
+        outs.append(y)
+    assert np.array_equal(outs[0], outs[1])
+
+
+def test_conv_staggered_k_order():
+    N, H, W, Cin, Cout = 8, 28, 28, 192, 128
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=78)
+    for tm in (128, 256):
+        st, y, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, cfg=umma(tile_m=tm, k_stagger=1))
+        assert st == 0 and ok, tdx.tdx_last_error()
+        assert conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y) < TIGHT["bf16"]
+
+
 def test_conv_padding_equals_explicit_zero_padded_copy_bitwise():
     # the copy engine's zero fill and explicit zeros feed the same products in the same order
     N, H, W, Cin, Cout, pad = 2, 16, 24, 64, 64, 1

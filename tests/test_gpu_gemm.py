@@ -120,6 +120,39 @@ def test_umma_256_row_tiles_exact_integers_many_tiles_per_cta():
         assert np.array_equal(oracle.decode(C, "bf16"), ref), cfgkw
 
 
+@pytest.mark.parametrize("store_mode", [1, 2])
+@pytest.mark.parametrize("cfgkw", [dict(tile_m=128, tile_n=64), dict(tile_m=128, tile_n=256), dict(tile_m=256, tile_n=128),
+                                   dict(tile_m=256, tile_n=256)])
+def test_umma_store_modes(cfgkw, store_mode):
+    # 1 = 16-byte stores from registers, 2 = staged in shared memory and written by the copy engine;
+    # ragged M and N tails exercise the predicated stores / the copy engine's clipping
+    M, N, K = 1000, 840, 264
+    A, B = si.gemm_bf16_normal(M, N, K, seed=66, transB=1)
+    st, C, ok = run_gemm(M, N, K, 0, 1, -1.0, "bf16", A, B, cfg=umma(store_mode=store_mode, **cfgkw))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert gemm_error(M, N, K, 0, 1, -1.0, "bf16", A, B, C) < TIGHT["bf16"]
+    if store_mode == 2:
+        st, C1, _ = run_gemm(M, N, K, 0, 1, -1.0, "bf16", A, B, cfg=umma(store_mode=1, **cfgkw))
+        assert np.array_equal(C, C1)                             # same arithmetic, different way out
+
+
+@pytest.mark.parametrize("cfgkw", [dict(tile_m=128, tile_n=64, stages=3), dict(tile_m=256, tile_n=128, stages=2)])
+def test_umma_staggered_k_order(cfgkw):
+    # each CTA starts its K loop at a different block: same products, rotated order
+    M, N, K = 1536, 1280, 712
+    A, B = si.gemm_bf16_normal(M, N, K, seed=64, transB=1)
+    st, C, ok = run_gemm(M, N, K, 0, 1, 1.0, "bf16", A, B, cfg=umma(k_stagger=1, **cfgkw))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert gemm_error(M, N, K, 0, 1, 1.0, "bf16", A, B, C) < TIGHT["bf16"]
+    st, C2, _ = run_gemm(M, N, K, 0, 1, 1.0, "bf16", A, B, cfg=umma(k_stagger=1, **cfgkw))
+    assert np.array_equal(C, C2)                                  # still deterministic
+    Ai = si.small_integers(65, 0, (M, K), "bf16", -1, 1)
+    Bi = si.small_integers(65, 1, (N, K), "bf16", -1, 1)
+    st, Ci, ok = run_gemm(M, N, K, 0, 1, 1.0, "bf16", Ai, Bi, cfg=umma(k_stagger=1, split_k=0, **cfgkw))
+    assert st == 0 and ok
+    assert np.array_equal(oracle.decode(Ci, "bf16"), oracle.gemm(M, N, K, 0, 1, 1.0, "bf16", Ai, Bi))
+
+
 @pytest.mark.parametrize("split", [2, 3, 5])
 @pytest.mark.parametrize("transB", [0, 1])
 def test_umma_split_k_with_workspace(split, transB):
