@@ -68,9 +68,9 @@ typedef struct {
     int stages;     /* depth of the TMA/mbarrier ring, 2..8, bounded by shared memory          */
     int cta_pair;   /* 1 (one CTA per tile)                                                    */
     int split_k;    /* >= 1; > 1 needs a workspace and runs a fixed-order reduction afterwards  */
-    int store_mode; /* 1 = 16-byte stores from registers; 2 = 32 x 64 blocks staged in shared     */
-                    /*     memory and written by TMA store (needs tile_n % 64 == 0, N % 8 == 0,    */
-                    /*     split_k = 1, 16-byte aligned C; falls back to 1 if C is misaligned)      */
+    int store_mode; /* 1 = 16-byte stores from registers; 2 = 32 x 32 blocks staged in shared     */
+                    /*     memory and written by TMA store (needs N % 8 == 0, split_k = 1,         */
+                    /*     16-byte aligned C; falls back to 1 if C is misaligned)                  */
     int raster;     /* width, in tiles along M, of the panels the tile order walks; 0 = all     */
     int patch_w;    /* conv only: output-pixel patch that forms the rows of a tile (w x h,      */
     int patch_h;    /*   w*h a power of two <= 128, w >= 8; tile_m / (w*h) patches per tile); 0 = choose */

@@ -121,17 +121,19 @@ struct MapKey {
     uint64_t dims[4];
     uint64_t strides[3];
     uint32_t box[4];
+    int swizzle;
     bool operator<(const MapKey& o) const { return std::memcmp(this, &o, sizeof(MapKey)) < 0; }
 };
 std::map<MapKey, CUtensorMap> g_maps;
 
-// bf16 tensor, 128-byte swizzle, zero fill outside the tensor.
+// bf16 tensor, 128-byte (or 64-byte) swizzle, zero fill outside the tensor.
 int get_tensor_map(DeviceCtx* ctx, const void* ptr, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                   const uint32_t* box, CUtensorMap* out) {
+                   const uint32_t* box, CUtensorMap* out, int swizzle_bytes = 128) {
     MapKey key;
     std::memset(&key, 0, sizeof key);
     key.ptr = ptr;
     key.rank = rank;
+    key.swizzle = swizzle_bytes;
     for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
     for (int i = 0; i + 1 < rank; ++i) key.strides[i] = strides_bytes[i];
     {
@@ -146,8 +148,8 @@ int get_tensor_map(DeviceCtx* ctx, const void* ptr, int rank, const uint64_t* di
     CUtensorMap m;
     CUresult r = ctx->encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank),
                              const_cast<void*>(ptr), gdim, gstr, gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                             swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS)
         return fail(TDX_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) rank %d dims %llu %llu box %u %u", (int)r, rank,
                     (unsigned long long)dims[0], (unsigned long long)(rank > 1 ? dims[1] : 0), box[0],
@@ -228,8 +230,8 @@ bool conv_umma_layout_ok(const ConvProblem& c) {
     return true;
 }
 
-// Shared memory the staged (TMA-store) epilogue needs: one 32 x 64 bf16 block per epilogue warp.
-int staging_bytes_for(int tile_m, int store_mode) { return store_mode == 2 ? (tile_m / 128) * 4 * 4096 : 0; }
+// Shared memory the staged (TMA-store) epilogue needs: one 32 x 32 bf16 block for each of its 16 warps.
+int staging_bytes_for(int /*tile_m*/, int store_mode) { return store_mode == 2 ? 16 * 2048 : 0; }
 
 int umma_max_stages(int tile_m, int tile_n, int smem_limit, int store_mode) {
     const int stage = (tile_m + tile_n) * 128;
@@ -255,7 +257,6 @@ const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num
     if (c.cta_pair != 1) return "cta_pair must be 1";
     if (c.store_mode != 1 && c.store_mode != 2) return "store_mode must be 1 (direct) or 2 (TMA store)";
     if (c.store_mode == 2) {
-        if (c.tile_n % 64) return "the TMA-store epilogue needs tile_n % 64 == 0";
         if (N % 8) return "the TMA-store epilogue needs an output row pitch that is a multiple of 16 bytes";
         if (c.split_k > 1) return "split-K writes fp32 partials directly: use store_mode 1";
         if (conv && c.patch_w * c.patch_h < 32) return "the TMA-store epilogue needs patches of at least 32 pixels";
@@ -331,7 +332,7 @@ void default_umma_config(int64_t tiles_m, int64_t N, int64_t num_kb, bool b_mn_m
     c->tile_m = tm;
     c->tile_n = bn;
     // staged epilogue whenever the layout allows it (whole-line writes instead of 16-byte pieces)
-    if (c->split_k == 1 && bn % 64 == 0 && N % 8 == 0) c->store_mode = 2;
+    if (c->split_k == 1 && N % 8 == 0) c->store_mode = 2;
     c->stages = std::max(2, umma_max_stages(tm, bn, smem_limit, c->store_mode));
     c->raster = 8;
 }
@@ -343,7 +344,8 @@ int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensor
     const int grid = static_cast<int>(std::min<long long>(items, ctx->sm_count));
     const size_t smem = static_cast<size_t>(p.stages) * ((p.bm + p.bn) * 128) + 1024 +
                         staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
-    const int threads = p.bm == 256 ? 320 : 192;   // producer warp, MMA warp, 4 epilogue warps per 128-row half
+    // producer warp, MMA warp, then 16 epilogue warps (staged epilogue) or 4 per 128-row half (direct)
+    const int threads = p.tma_store ? 576 : (p.bm == 256 ? 320 : 192);
     if (conv)
         tdx::umma_contract_kernel<true><<<grid, threads, smem, st>>>(ma, mb, mc, p);
     else
@@ -437,8 +439,8 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     if (p.tma_store) {
         uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.M)};
         uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
-        uint32_t box[2] = {64, 32};
-        rc = get_tensor_map(ctx, C, 2, dims, str, box, &mc);
+        uint32_t box[2] = {32, 32};
+        rc = get_tensor_map(ctx, C, 2, dims, str, box, &mc, 64);
         if (rc) return rc;
     }
     rc = launch_umma(ctx, false, ma, mb, mc, p, st);
@@ -524,8 +526,8 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
                             static_cast<uint64_t>(c.N)};
         uint64_t str[3] = {static_cast<uint64_t>(c.Cout) * 2, static_cast<uint64_t>(c.Q * c.Cout) * 2,
                            static_cast<uint64_t>(c.P * c.Q * c.Cout) * 2};
-        uint32_t box[4] = {64, static_cast<uint32_t>(p.sbx), static_cast<uint32_t>(p.sby), 1};
-        int rc = get_tensor_map(ctx, y, 4, dims, str, box, &mc);
+        uint32_t box[4] = {32, static_cast<uint32_t>(p.sbx), static_cast<uint32_t>(p.sby), 1};
+        int rc = get_tensor_map(ctx, y, 4, dims, str, box, &mc, 64);
         if (rc) return rc;
     }
     return launch_umma(ctx, true, ma, mb, mc, p, st);
@@ -671,7 +673,7 @@ int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_cou
     if (c.tile_n == 0) c.tile_n = d.tile_n;
     if (c.split_k == 0) c.split_k = (user && user->tile_n != 0 && user->tile_n != d.tile_n) ? 1 : d.split_k;
     if (c.store_mode == 0) {
-        c.store_mode = (c.split_k == 1 && c.tile_n % 64 == 0 && g.N % 8 == 0) ? 2 : 1;
+        c.store_mode = (c.split_k == 1 && g.N % 8 == 0) ? 2 : 1;
         if (c.store_mode == 2 && c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, 2)) c.store_mode = 1;
     }
     if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode));
@@ -713,7 +715,7 @@ int resolve_conv_config(const ConvProblem& cp, const tdx_config* user, int sm_co
     if (c.tile_n == 0) c.tile_n = d.tile_n;
     if (c.split_k == 0) c.split_k = 1;
     if (c.store_mode == 0) {
-        c.store_mode = (c.tile_n % 64 == 0 && cp.Cout % 8 == 0 && c.patch_w * c.patch_h >= 32) ? 2 : 1;
+        c.store_mode = (cp.Cout % 8 == 0 && c.patch_w * c.patch_h >= 32) ? 2 : 1;
         if (c.store_mode == 2 && c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, 2)) c.store_mode = 1;
     }
     if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode));
@@ -826,8 +828,8 @@ void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int 
                     if (num_kb / s >= 2 && tiles * s <= 4LL * sm_count) splits.push_back(s);
             for (int sk : splits)
                 for (int sm : {2, 1}) {
-                    if (sm == 2 && (sk > 1 || bn % 64 || N % 8)) continue;
-                    if (sm == 1 && sk == 1 && bn % 64 == 0 && N % 8 == 0 && tiles * tm * bn > (1 << 22))
+                    if (sm == 2 && (sk > 1 || N % 8)) continue;
+                    if (sm == 1 && sk == 1 && N % 8 == 0 && tiles * tm * bn > (1 << 22))
                         continue;                          // large outputs: 16-byte scattered stores never win
                     const int max_st = umma_max_stages(tm, bn, smem_limit, sm);
                     if (max_st < 2) continue;

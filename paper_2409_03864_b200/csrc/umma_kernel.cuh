@@ -6,10 +6,11 @@
 //   warp 1 (one lane)  MMA issuer: per stage and per 128-row half four tcgen05.mma (K = 16
 //                      each) into a TMEM accumulator slot; tcgen05.commit releases the stage /
 //                      publishes the tile.
-//   warps 2..5 (6..9)  epilogue of the first (second) 128-row half: tcgen05.ld the accumulator
-//                      (one row per thread), apply alpha / bias / ReLU, convert, and either store
-//                      16 bytes at a time from registers or stage 32 x 64 blocks in shared memory
-//                      (128-byte swizzled) and let the copy engine write whole lines (TMA store).
+//   warps 2..         epilogue: tcgen05.ld the accumulator (one row per thread), apply alpha /
+//                      bias / ReLU, convert, and either store 16 bytes at a time from registers
+//                      (one warp per 32 rows) or stage 32 x 32 blocks in shared memory (64-byte
+//                      swizzled) and let the copy engine write them (TMA store; 16 warps, four per
+//                      TMEM lane quarter, so that TMEM-load and store latencies overlap).
 // TMEM holds 2 or 4 accumulator slots of 128 x BN; when a tile leaves slots free, the epilogue
 // of tile t overlaps the main loop of tile t+1.  A 256-row tile halves the operand bytes fetched
 // from L2 per flop (the B slice is shared by both halves), which is what bounds the 128-row tile.
@@ -103,7 +104,7 @@ __device__ __forceinline__ TileCoord decode_item(const UmmaParams& p, int item) 
 }
 
 template <bool kConv>
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(576, 1)
 umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                      const __grid_constant__ CUtensorMap tmC, const UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -130,7 +131,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
         for (int b = 0; b < p.slots; ++b) {
             ptx::mbar_init(&tfull_bar[b], 1);
-            ptx::mbar_init(&tempty_bar[b], 4);
+            ptx::mbar_init(&tempty_bar[b], static_cast<uint32_t>(((blockDim.x >> 5) - 2) / mh));
         }
         s_abort = 0;
         ptx::fence_barrier_init();
@@ -280,7 +281,14 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
     } else {
         // ------------------------------------------------------------ epilogue (4 warps per 128-row half)
-        const int half = (warp - 2) >> 2;             // which 128-row half of the tile this warp group drains
+        // epilogue warp e = warp - 2: with the staged epilogue there are 16 of them (4 per TMEM lane
+        // quarter) and the warps of a quarter take the 32-column steps round robin; the direct
+        // epilogue has one warp per quarter and 128-row half.
+        const int ew = warp - 2;
+        const int nwarps_epi = (static_cast<int>(blockDim.x) >> 5) - 2;
+        const int ncgrp = nwarps_epi / (4 * mh);      // warps sharing one (half, quarter)
+        const int half = (ew >> 2) % mh;              // which 128-row half of the tile this warp drains
+        const int cgrp = (ew >> 2) / mh;              // which share of the columns
         const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
         const int row_in_tile = half * kHalfM + quarter * 32 + lane;
         int local = 0;
@@ -316,8 +324,8 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             }
 
             if (p.tma_store && p.split_k == 1) {
-                // ---- staged path: 32 rows x 64 columns per warp and step, written by the copy engine
-                uint8_t* stage_buf = smem + static_cast<size_t>(p.stages) * stage_bytes + (warp - 2) * 4096;
+                // ---- staged path: 32 rows x 32 columns per warp and step, written by the copy engine
+                uint8_t* stage_buf = smem + static_cast<size_t>(p.stages) * stage_bytes + (warp - 2) * 2048;
                 const int wrow0 = half * kHalfM + quarter * 32;      // first tile row of this warp
                 int sc1 = 0, sc2 = 0, sc3 = 0;                       // store coordinates above the column
                 bool box_ok;
@@ -341,39 +349,55 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     sc1 = t.m_blk * p.bm + wrow0;
                     box_ok = sc1 < p.M;
                 }
-                for (int c0 = 0; c0 < p.bn; c0 += 64) {
-                    uint32_t r0[32], r1[32];
+                // 64-byte swizzle of the staging block: 16-byte slot c of row `lane` lives at slot c ^ ((lane / 2) % 4)
+                uint8_t* my_row = stage_buf + lane * 64;
+                const int sw = (lane >> 1) & 3;
+                const bool plain = (p.bias == nullptr) && (p.relu == 0);
+                for (int c0 = cgrp * 32; c0 < p.bn; c0 += ncgrp * 32) {
+                    uint32_t r[32];
                     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                            static_cast<uint32_t>(buf * p.bn + c0);
-                    ptx::tmem_ld_32x32b_x32(taddr, r0);
-                    ptx::tmem_ld_32x32b_x32(taddr + 32, r1);
+                    ptx::tmem_ld_32x32b_x32(taddr, r);
                     ptx::tmem_ld_wait();
                     const int col0 = t.n_blk * p.bn + c0;
-                    // the previous store of this warp must have finished reading the staging buffer
+                    // the previous store of this warp must have finished reading the staging block
                     if (lane == 0) ptx::tma_store_wait_read<0>();
                     __syncwarp();
+                    if (plain) {
 #pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        uint32_t pk[4];
+                        for (int g = 0; g < 4; ++g) {
+                            uint32_t pk[4];
 #pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int j = g * 8 + e * 2;
-                            float x0 = p.alpha * __uint_as_float(j < 32 ? r0[j & 31] : r1[j & 31]);
-                            float x1 = p.alpha * __uint_as_float(j + 1 < 32 ? r0[(j + 1) & 31] : r1[(j + 1) & 31]);
-                            if (p.bias != nullptr) {
-                                if (col0 + j < p.N) x0 += __ldg(p.bias + col0 + j);
-                                if (col0 + j + 1 < p.N) x1 += __ldg(p.bias + col0 + j + 1);
+                            for (int e = 0; e < 4; ++e) {
+                                __nv_bfloat162 h2 = __floats2bfloat162_rn(p.alpha * __uint_as_float(r[g * 8 + e * 2]),
+                                                                          p.alpha * __uint_as_float(r[g * 8 + e * 2 + 1]));
+                                pk[e] = *reinterpret_cast<uint32_t*>(&h2);
                             }
-                            if (p.relu) {
-                                x0 = fmaxf(x0, 0.0f);
-                                x1 = fmaxf(x1, 0.0f);
-                            }
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
-                            pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+                            *reinterpret_cast<uint4*>(my_row + ((g ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                         }
-                        // 128-byte swizzle: 16-byte slot g of row `lane` lives at slot g ^ (lane % 8)
-                        *reinterpret_cast<uint4*>(stage_buf + lane * 128 + ((g ^ (lane & 7)) << 4)) =
-                            make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    } else {
+                        const int last = p.N - 1;    // columns past N are clipped by the store; keep the bias index in range
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            uint32_t pk[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const int j = g * 8 + e * 2;
+                                float x0 = p.alpha * __uint_as_float(r[j]);
+                                float x1 = p.alpha * __uint_as_float(r[j + 1]);
+                                if (p.bias != nullptr) {
+                                    x0 += __ldg(p.bias + min(col0 + j, last));
+                                    x1 += __ldg(p.bias + min(col0 + j + 1, last));
+                                }
+                                if (p.relu) {
+                                    x0 = fmaxf(x0, 0.0f);
+                                    x1 = fmaxf(x1, 0.0f);
+                                }
+                                __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
+                                pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+                            }
+                            *reinterpret_cast<uint4*>(my_row + ((g ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        }
                     }
                     ptx::fence_proxy_async_smem();
                     __syncwarp();

@@ -122,7 +122,7 @@ def test_umma_256_row_tiles_exact_integers_many_tiles_per_cta():
 
 @pytest.mark.parametrize("store_mode", [1, 2])
 @pytest.mark.parametrize("cfgkw", [dict(tile_m=128, tile_n=64), dict(tile_m=128, tile_n=256), dict(tile_m=256, tile_n=128),
-                                   dict(tile_m=256, tile_n=256)])
+                                   dict(tile_m=256, tile_n=256), dict(tile_m=128, tile_n=32), dict(tile_m=256, tile_n=96)])
 def test_umma_store_modes(cfgkw, store_mode):
     # 1 = 16-byte stores from registers, 2 = staged in shared memory and written by the copy engine;
     # ragged M and N tails exercise the predicated stores / the copy engine's clipping
