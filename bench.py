@@ -4,9 +4,10 @@
 A step is one call of the headline workload: C = -(A . B^T), bf16 in / fp32 accumulate / bf16 out,
 M = N = K = 4096, N(0,1) operands (seed 1), B stored N x K.  Inputs are resident in HBM; the step
 rotates over several buffer sets whose total footprint exceeds L2, so operands are not served from
-a warm cache.  One JSON line is printed by rank 0.
+a warm cache.  One JSON line is printed by rank 0.  --workload selects one of the other
+configurations (c1, c3, c4, c5a..c5e), measured the same way.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl tdx|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl tdx|reference] [--workload c2]
 
 With N > 1 (launched by torch.distributed.run) every rank runs an independent replica on its own
 GPU -- the path has no exchange step, so there is no data-path collective; the reported value is
@@ -30,14 +31,82 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-M = N = K = 4096
-SEED = 1
-FLOP_PER_STEP = 2.0 * M * N * K
-ALGO_BYTES_PER_STEP = 3 * M * N * 2          # each operand read once, the output written once (bf16)
 METRIC = "GEMM/conv2d TFLOP/s at 1 B200 and fraction of dense bf16 (fp32) peak"
-WORKLOAD = "gemm_bf16_negated_transB_4096"
-BUFFER_SETS = 8                              # 8 x 96 MiB = 805 MB of operands and outputs > 126 MB of L2
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
+L2_BYTES = 126e6
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel from the ncu capture of the same
+# workload (see profiles/); None where no capture of the current kernel exists.
+TRAFFIC = {}
+
+# name: (kind, dims..., seed, bound).  The default (headline) workload is c2; the others are the remaining
+# configurations, selectable with --workload so that every one can be measured the same way.
+WORKLOADS = {
+    "c1": dict(kind="gemm", dtype="f32", M=256, N=256, K=256, tA=0, tB=0, alpha=1.0, seed=0, bound="alu",
+               label="gemm_f32_256"),
+    "c2": dict(kind="gemm", dtype="bf16", M=4096, N=4096, K=4096, tA=0, tB=1, alpha=-1.0, seed=1, bound="tensor",
+               label="gemm_bf16_negated_transB_4096"),
+    "c3": dict(kind="conv", N=4, H=128, W=128, Cin=64, Cout=64, R=3, S=3, pad=1, stride=1, seed=2, bound="tensor",
+               label="conv_bf16_4x128x128x64_k3"),
+    "c4": dict(kind="conv", N=32, H=56, W=56, Cin=256, Cout=256, R=3, S=3, pad=1, stride=1, seed=3, bound="tensor",
+               label="conv_bf16_32x56x56x256_k3"),
+    "c5a": dict(kind="gemm", dtype="bf16", M=1024, N=1024, K=1024, tA=0, tB=0, alpha=1.0, seed=4, bound="tensor",
+                label="gemm_bf16_1024"),
+    "c5b": dict(kind="gemm", dtype="bf16", M=8192, N=8192, K=8192, tA=0, tB=0, alpha=1.0, seed=4, bound="tensor",
+                label="gemm_bf16_8192"),
+    "c5c": dict(kind="gemm", dtype="bf16", M=128, N=8192, K=8192, tA=0, tB=0, alpha=1.0, seed=4, bound="hbm",
+                label="gemm_bf16_128x8192x8192"),
+    "c5d": dict(kind="gemm", dtype="bf16", M=8192, N=128, K=8192, tA=0, tB=0, alpha=1.0, seed=4, bound="hbm",
+                label="gemm_bf16_8192x128x8192"),
+    "c5e": dict(kind="gemm", dtype="bf16", M=4096, N=4096, K=512, tA=0, tB=0, alpha=1.0, seed=4, bound="tensor",
+                label="gemm_bf16_4096x4096x512"),
+}
+
+
+class Workload:
+    """Shapes, algorithmic flops/bytes, seeded host inputs and launchers of one configuration."""
+
+    def __init__(self, name):
+        self.name, self.w = name, WORKLOADS[name]
+        w = self.w
+        if w["kind"] == "gemm":
+            self.el = 4 if w["dtype"] == "f32" else 2
+            self.flops = 2.0 * w["M"] * w["N"] * w["K"]
+            self.in_bytes = (w["M"] * w["K"] + w["K"] * w["N"]) * self.el
+            self.out_bytes = w["M"] * w["N"] * self.el
+            self.rows = w["M"]
+        else:
+            self.el = 2
+            self.P = (w["H"] + 2 * w["pad"] - w["R"]) // w["stride"] + 1
+            self.Q = (w["W"] + 2 * w["pad"] - w["S"]) // w["stride"] + 1
+            self.rows = w["N"] * self.P * self.Q
+            self.flops = 2.0 * self.rows * w["Cout"] * w["R"] * w["S"] * w["Cin"]
+            self.in_bytes = (w["N"] * w["H"] * w["W"] * w["Cin"] + w["Cout"] * w["R"] * w["S"] * w["Cin"]) * 2 + w["Cout"] * 4
+            self.out_bytes = self.rows * w["Cout"] * 2
+        self.algo_bytes = self.in_bytes + self.out_bytes       # each operand read once, the output written once
+        self.dtype = w.get("dtype", "bf16")
+
+    def host_inputs(self):
+        import seeded_inputs as si
+        w = self.w
+        if w["kind"] == "gemm":
+            if w["dtype"] == "f32":
+                return si.gemm_f32_uniform(w["M"], w["N"], w["K"], seed=w["seed"])
+            return si.gemm_bf16_normal(w["M"], w["N"], w["K"], seed=w["seed"], transA=w["tA"], transB=w["tB"])
+        return si.conv_bf16(w["N"], w["H"], w["W"], w["Cin"], w["Cout"], w["R"], w["S"], seed=w["seed"])
+
+    def config_dict(self):
+        return {k: v for k, v in self.w.items() if k not in ("kind", "seed", "bound", "label")}
+
+    def oracle_rows(self, host, rows):
+        import oracle
+        w = self.w
+        if w["kind"] == "gemm":
+            return oracle.gemm(w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], w["dtype"], host[0], host[1], rows=rows)
+        return oracle.conv2d(w["N"], w["H"], w["W"], w["Cin"], w["Cout"], w["R"], w["S"], w["pad"], w["stride"], "bf16",
+                             host[0], host[1], host[2], 1, rows=rows)
+
+    def flops_for_rows(self, n_rows):
+        return self.flops * n_rows / self.rows
 
 
 def measured_peaks():
@@ -98,27 +167,24 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def oracle_sample(rows_target_seconds: float = 12.0):
-    """Times the CPU oracle on a row sample of the workload; returns (tflops, cores, description)."""
+def oracle_sample(wl, host, target_seconds=12.0):
+    """Times the CPU oracle on a row sample of the workload; returns (TFLOP/s, threads, description)."""
     import numpy as np
 
     import oracle
-    import seeded_inputs as si
 
-    A, B = si.gemm_bf16_normal(M, N, K, seed=SEED, transB=1)
-    oracle.gemm(8, N, K, 0, 1, -1.0, "bf16", A[:8], B)                 # page in, spin up the thread pool
-    rows = np.arange(0, M, M // 16, dtype=np.int64)                      # 16 rows
+    wl.oracle_rows(host, np.arange(min(8, wl.rows), dtype=np.int64))            # page in, spin up the thread pool
+    probe = np.linspace(0, wl.rows - 1, min(16, wl.rows)).astype(np.int64)
     t0 = time.perf_counter()
-    oracle.gemm(M, N, K, 0, 1, -1.0, "bf16", A, B, rows=rows)
+    wl.oracle_rows(host, probe)
     t = time.perf_counter() - t0
-    n_rows = int(min(M, max(16, 16 * rows_target_seconds / max(t, 1e-3))))
-    n_rows -= n_rows % 8
-    rows = np.linspace(0, M - 1, n_rows).astype(np.int64)
+    n_rows = int(min(wl.rows, max(len(probe), len(probe) * target_seconds / max(t, 1e-4))))
+    rows = np.linspace(0, wl.rows - 1, n_rows).astype(np.int64)
     t0 = time.perf_counter()
-    oracle.gemm(M, N, K, 0, 1, -1.0, "bf16", A, B, rows=rows)
+    wl.oracle_rows(host, rows)
     t = time.perf_counter() - t0
-    tflops = 2.0 * n_rows * N * K / t / 1e12
-    return tflops, oracle.num_threads(), f"{n_rows} of {M} output rows (all {N} columns), {t:.1f} s", t, n_rows
+    return (wl.flops_for_rows(n_rows) / t / 1e12, oracle.num_threads(),
+            f"{n_rows} of {wl.rows} output rows (all columns), {t:.1f} s")
 
 
 def run_reference(args):
@@ -128,30 +194,30 @@ def run_reference(args):
     import numpy as np
 
     import oracle
-    import seeded_inputs as si
 
-    A, B = si.gemm_bf16_normal(M, N, K, seed=SEED, transB=1)
+    wl = Workload(args.workload)
+    host = wl.host_inputs()
     # size the per-step sample from a short probe so that the whole run takes about a minute
-    oracle.gemm(M, N, K, 0, 1, -1.0, "bf16", A, B, rows=np.arange(8, dtype=np.int64))
+    wl.oracle_rows(host, np.arange(min(8, wl.rows), dtype=np.int64))
+    probe = np.linspace(0, wl.rows - 1, min(16, wl.rows)).astype(np.int64)
     t0 = time.perf_counter()
-    oracle.gemm(M, N, K, 0, 1, -1.0, "bf16", A, B, rows=np.arange(16, dtype=np.int64))
-    rows_per_s = 16.0 / max(time.perf_counter() - t0, 1e-4)
-    rows_per_step = int(max(1, min(256, rows_per_s * 60.0 / max(1, args.steps + args.warmup))))
-    rows = np.linspace(0, M - 1, rows_per_step).astype(np.int64)
+    wl.oracle_rows(host, probe)
+    rows_per_s = len(probe) / max(time.perf_counter() - t0, 1e-5)
+    rows_per_step = int(max(1, min(wl.rows, rows_per_s * 60.0 / max(1, args.steps + args.warmup))))
+    rows = np.linspace(0, wl.rows - 1, rows_per_step).astype(np.int64)
     for _ in range(args.warmup):
-        oracle.gemm(M, N, K, 0, 1, -1.0, "bf16", A, B, rows=rows)
+        wl.oracle_rows(host, rows)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        oracle.gemm(M, N, K, 0, 1, -1.0, "bf16", A, B, rows=rows)
+        wl.oracle_rows(host, rows)
     t = time.perf_counter() - t0
-    flops = 2.0 * rows_per_step * N * K * args.steps
-    value = flops / t / 1e12
-    sample = f"each step = {rows_per_step} of {M} output rows (all columns) of the workload"
+    value = wl.flops_for_rows(rows_per_step) * args.steps / t / 1e12
+    sample = f"each step = {rows_per_step} of {wl.rows} output rows (all columns) of the workload"
+    cfg = dict(wl.config_dict(), workload=wl.w["label"], sample=sample)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "M": M, "N": N, "K": K, "transB": 1, "alpha": -1.0, "sample": sample},
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic", "config": cfg,
         "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -166,7 +232,6 @@ def run_tdx(args):
     import torch
 
     import paper_2409_03864_b200 as tdx
-    import seeded_inputs as si
 
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -179,27 +244,52 @@ def run_tdx(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     tdx.lib()
+    wl = Workload(args.workload)
+    w = wl.w
+    host = wl.host_inputs()
 
     # CPU baseline first (rank 0, single-GPU runs only), before the GPU is busy
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, cores, desc, _, _ = oracle_sample()
+        v, cores, desc = oracle_sample(wl, host)
         cpu_baseline = {"value": v, "unit": "TFLOP/s", "cores": cores, "kind": "oracle", "sample": desc}
 
-    A, B = si.gemm_bf16_normal(M, N, K, seed=SEED, transB=1)
-    hA = torch.from_numpy(A.view(np.int16)).pin_memory()
-    hB = torch.from_numpy(B.view(np.int16)).pin_memory()
-    hC = torch.empty(M * N, dtype=torch.int16).pin_memory()
-    sets = []
-    for _ in range(BUFFER_SETS):
-        sets.append((hA.cuda(non_blocking=True), hB.cuda(non_blocking=True),
-                     torch.empty(M * N, dtype=torch.int16, device="cuda")))
+    def pinned(a):
+        a = np.ascontiguousarray(a)
+        return torch.from_numpy(a.view(np.int16) if a.dtype == np.uint16 else a).pin_memory()
+
+    h_in = [pinned(a) for a in host]
+    out_dtype = torch.float32 if wl.dtype == "f32" else torch.int16
+    h_out = torch.empty(wl.out_bytes // wl.el, dtype=out_dtype).pin_memory()
+    # rotate over enough buffer sets that the cycled footprint exceeds L2 several times
+    n_sets = int(min(512, max(2, -(-int(6 * L2_BYTES) // wl.algo_bytes))))
+    sets = [([h.cuda(non_blocking=True) for h in h_in], torch.empty_like(h_out, device="cuda")) for _ in range(n_sets)]
     stream = torch.cuda.current_stream()
-    st_cfg, cfg = tdx.tdx_default_gemm_config(M, N, K, 0, 1, tdx.TDX_BF16)
+    DT = tdx.TDX_F32 if wl.dtype == "f32" else tdx.TDX_BF16
+    if w["kind"] == "gemm":
+        st_cfg, cfg = tdx.tdx_default_gemm_config(w["M"], w["N"], w["K"], w["tA"], w["tB"], DT)
+
+        def launch(ins, out):
+            return tdx.tdx_gemm(w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], DT, ins[0], ins[1], out, stream)
+
+        def launch_host():
+            return tdx.tdx_gemm_host(w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], DT, h_in[0], h_in[1], h_out,
+                                     stream)
+        kernel_name = "sgemm_tiled_kernel" if wl.dtype == "f32" else "umma_contract_kernel<false>"
+    else:
+        cargs = (w["N"], w["H"], w["W"], w["Cin"], w["Cout"], w["R"], w["S"], w["pad"], w["stride"], DT)
+        st_cfg, cfg = tdx.tdx_default_conv2d_config(*cargs)
+
+        def launch(ins, out):
+            return tdx.tdx_conv2d_bias_relu(*cargs, ins[0], ins[1], ins[2], 1, out, stream)
+
+        def launch_host():
+            return tdx.tdx_conv2d_bias_relu_host(*cargs, h_in[0], h_in[1], h_in[2], 1, h_out, stream)
+        kernel_name = "umma_contract_kernel<true>"
 
     def step(i):
-        a, b, c = sets[i % BUFFER_SETS]
-        tdx.check(tdx.tdx_gemm(M, N, K, 0, 1, -1.0, tdx.TDX_BF16, a, b, c, stream))
+        ins, out = sets[i % n_sets]
+        tdx.check(launch(ins, out))
 
     for i in range(args.warmup):
         step(i)
@@ -222,16 +312,19 @@ def run_tdx(args):
     launches = tdx.tdx_kernel_launch_count() - n0
     ms_total = e0.elapsed_time(e1)
 
-    # per-launch durations of the dominant kernel (CUDA events on the launching stream)
-    n_k = min(args.steps, 200)
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_k)]
-    for i, (a, b) in enumerate(evs):
+    # launch duration of the dominant kernel: CUDA events on the launching stream around groups of 10 launches
+    group = 10
+    n_groups = max(1, min(args.steps // group, 50))
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_groups)]
+    for gidx, (a, b) in enumerate(evs):
         a.record(stream)
-        step(i)
+        for i in range(group):
+            step(gidx * group + i)
         b.record(stream)
     torch.cuda.synchronize()
     clocks = sampler.stop() if rank == 0 else None
-    kernel_ms = statistics.mean(a.elapsed_time(b) for a, b in evs)
+    launches_per_step = launches / args.steps
+    kernel_ms = statistics.mean(a.elapsed_time(b) for a, b in evs) / group
     tdx.check(tdx.tdx_check_device_status(stream))
 
     if distributed:
@@ -239,47 +332,58 @@ def run_tdx(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms_total = float(t.item())
         dist.barrier()
-    value = world * FLOP_PER_STEP * args.steps / (ms_total * 1e-3) / 1e12
+    value = world * wl.flops * args.steps / (ms_total * 1e-3) / 1e12
 
-    # end to end through the host-buffer entry point: H2D of A and B, the GEMM, D2H of C, every step
+    # end to end through the host-buffer entry point: H2D of the inputs, the kernels, D2H of the result, every step
     e2e_steps = max(3, min(args.steps, 20))
     for _ in range(3):
-        tdx.check(tdx.tdx_gemm_host(M, N, K, 0, 1, -1.0, tdx.TDX_BF16, hA, hB, hC, stream))
+        tdx.check(launch_host())
     torch.cuda.synchronize()
     if distributed:
         dist.barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
-        tdx.check(tdx.tdx_gemm_host(M, N, K, 0, 1, -1.0, tdx.TDX_BF16, hA, hB, hC, stream))
+        tdx.check(launch_host())
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     if distributed:
         t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         e2e_s = float(t.item())
-    e2e_value = world * FLOP_PER_STEP * e2e_steps / e2e_s / 1e12
+    e2e_value = world * wl.flops * e2e_steps / e2e_s / 1e12
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
-        peak = float(peaks["bf16_tflops"])
-        achieved = FLOP_PER_STEP / (kernel_ms * 1e-3) / 1e12
+        sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+        if w["bound"] == "tensor":
+            achieved, unit = wl.flops / (kernel_ms * 1e-3) / 1e12, "TFLOP/s"
+            peak, src = float(peaks["bf16_tflops"]), f"{peak_kind} bf16_tflops (burst)"
+        elif w["bound"] == "hbm":
+            achieved, unit = wl.algo_bytes / (kernel_ms * 1e-3) / 1e9, "GB/s"
+            peak, src = float(peaks["hbm_gbs"]), f"{peak_kind} hbm_gbs"
+        else:   # fp32 CUDA-core path: 2 flops x 128 lanes x SMs x max SM clock
+            achieved, unit = wl.flops / (kernel_ms * 1e-3) / 1e12, "TFLOP/s"
+            peak = 2 * 128 * sm_count * float(peaks.get("sm_max_mhz", 1965.0)) * 1e6 / 1e12
+            src = "derived: 2 x 128 fp32 lanes x SMs x max SM clock"
+        roof = {"bound": w["bound"], "achieved": achieved, "peak": peak, "unit": unit, "frac": achieved / peak,
+                "traffic": TRAFFIC.get(args.workload), "kernel": kernel_name, "kernel_ms": kernel_ms, "peak_source": src,
+                "launches_per_step": launches_per_step,
+                "hbm_gbs_algorithmic": wl.algo_bytes / (kernel_ms * 1e-3) / 1e9}
+        if w["bound"] == "tensor":
+            roof["frac_of_sustained_peak"] = achieved / float(peaks.get("bf16_tflops_sustained", peak))
         line = {
             "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "M": M, "N": N, "K": K, "transA": 0, "transB": 1, "alpha": -1.0,
-                       "accumulate": "fp32", "out": "bf16", "parallelism": f"replicas x{world}",
-                       "l2": f"rotating {BUFFER_SETS} buffer sets ({BUFFER_SETS * ALGO_BYTES_PER_STEP / 1e6:.0f} MB) larger than L2",
-                       "tile_config": cfg.as_dict() if st_cfg == 0 else None},
+            "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": dict(wl.config_dict(), workload=w["label"], accumulate="fp32", parallelism=f"replicas x{world}",
+                           l2=f"rotating {n_sets} buffer sets ({n_sets * wl.algo_bytes / 1e6:.0f} MB) larger than L2",
+                           tile_config=cfg.as_dict() if st_cfg == 0 else None),
             "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": 2 * M * K * 2,
-                    "d2h_bytes_per_step": M * N * 2, "steps": e2e_steps, "api": "tdx_gemm_host (pinned host buffers)"},
+            "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": int(wl.in_bytes),
+                    "d2h_bytes_per_step": int(wl.out_bytes), "steps": e2e_steps,
+                    "api": "tdx_gemm_host / tdx_conv2d_bias_relu_host (pinned host buffers)"},
             "gpu_launches": int(launches),
-            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                         "frac": achieved / peak, "traffic": None, "kernel": "umma_contract_kernel<false>",
-                         "kernel_ms": kernel_ms, "peak_source": f"{peak_kind} bf16_tflops (burst)",
-                         "frac_of_sustained_peak": achieved / float(peaks.get("bf16_tflops_sustained", peak)),
-                         "hbm_gbs_algorithmic": ALGO_BYTES_PER_STEP / (kernel_ms * 1e-3) / 1e9},
+            "roofline": roof,
             "cpu_baseline": cpu_baseline,
         }
         print(json.dumps(line))
@@ -295,6 +399,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="tdx", choices=["tdx", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS),
+                    help="c2 (default) is the headline workload; the others are the remaining configurations")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -8,6 +8,7 @@ non-zero status into a TdxError carrying tdx_last_error().
 from __future__ import annotations
 
 import ctypes
+import os
 from pathlib import Path
 
 _LIB_PATH = Path(__file__).resolve().parent / "libtdx.so"
@@ -93,6 +94,11 @@ def lib() -> ctypes.CDLL:
             if name not in ("tdx_kernel_launch_count", "tdx_last_error", "tdx_version"):
                 fn.restype = ci
         _lib = L
+        # Tuned tile configurations measured on B200 ship next to the library; TDX_TUNE_CACHE names another
+        # file, or "0" for none.  A missing or unreadable file only means the heuristic defaults are used.
+        cache = os.environ.get("TDX_TUNE_CACHE", str(_LIB_PATH.parent / "tuned_b200.json"))
+        if cache != "0" and os.path.exists(cache):
+            L.tdx_tune_load(cache.encode())
     return _lib
 
 

@@ -18,6 +18,27 @@ def built():
     tdx_build.build()
 
 
+@pytest.fixture(autouse=True)
+def heuristics_only():
+    """These tests look at the heuristic defaults: run them without the shipped tuning cache, restore it after."""
+    tdx.tdx_tune_clear()
+    yield
+    tdx.tdx_tune_clear()
+    shipped = os.path.join(ROOT, "paper_2409_03864_b200", "tuned_b200.json")
+    if os.path.exists(shipped):
+        tdx.tdx_tune_load(shipped)
+
+
+def test_shipped_tuning_cache_loads_and_is_feasible():
+    shipped = os.path.join(ROOT, "paper_2409_03864_b200", "tuned_b200.json")
+    assert os.path.exists(shipped)
+    assert tdx.tdx_tune_load(shipped) == tdx.TDX_OK
+    st, c = tdx.tdx_default_gemm_config(4096, 4096, 4096, 0, 1, tdx.TDX_BF16)
+    assert st == tdx.TDX_OK and c.kernel == tdx.TDX_KERNEL_UMMA and c.tile_m in (128, 256)
+    st, c = tdx.tdx_default_conv2d_config(32, 56, 56, 256, 256, 3, 3, 1, 1, tdx.TDX_BF16)
+    assert st == tdx.TDX_OK and c.patch_w * c.patch_h >= 8
+
+
 def declared_symbols():
     text = open(os.path.join(ROOT, "include", "tdx.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
