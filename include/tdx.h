@@ -76,6 +76,9 @@ typedef struct {
     int patch_h;    /*   w*h a power of two <= 128, w >= 8; tile_m / (w*h) patches per tile); 0 = choose */
     int k_stagger;  /* 1 = each CTA starts its K loop at a different block (rotated order, same terms),  */
                     /*     so that CTAs do not all fetch the same operand lines at the same moment       */
+    int halo;       /* conv only: 1 = the input window is fetched again for every filter tap; 2 = it is   */
+                    /*     loaded once per 64-channel chunk into shared memory and all taps read it there  */
+                    /*     (8 x 16 patches, stride 1, more than one tap); 0 = choose                      */
 } tdx_config;
 
 /*

@@ -41,7 +41,7 @@ class TdxError(RuntimeError):
 class tdx_config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in
                 ("kernel", "tile_m", "tile_n", "tile_k", "stages", "cta_pair", "split_k", "store_mode", "raster",
-                 "patch_w", "patch_h", "k_stagger")]
+                 "patch_w", "patch_h", "k_stagger", "halo")]
 
     def as_dict(self) -> dict:
         return {n: int(getattr(self, n)) for n, _ in self._fields_}

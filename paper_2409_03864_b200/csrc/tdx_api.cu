@@ -16,6 +16,7 @@
 #include <vector>
 
 #include "simt_kernels.cuh"
+#include "umma_conv_halo.cuh"
 #include "umma_kernel.cuh"
 
 namespace {
@@ -108,6 +109,9 @@ int get_ctx(DeviceCtx** out) {
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(tdx::umma_contract_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  c.smem_optin - kStaticSmemReserve);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tdx::umma_conv_halo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 c.smem_optin - kStaticSmemReserve);
     if (e != cudaSuccess) return fail(TDX_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     auto ins = g_ctx.emplace(dev, c);
     *out = &ins.first->second;
@@ -189,11 +193,13 @@ bool tune_lookup(const std::string& key, tdx_config* out) {
 void cfg_to_ints(const tdx_config& c, int* v) {
     v[0] = c.kernel; v[1] = c.tile_m; v[2] = c.tile_n; v[3] = c.tile_k; v[4] = c.stages; v[5] = c.cta_pair;
     v[6] = c.split_k; v[7] = c.store_mode; v[8] = c.raster; v[9] = c.patch_w; v[10] = c.patch_h; v[11] = c.k_stagger;
+    v[12] = c.halo;
 }
 void ints_to_cfg(const int* v, tdx_config* c) {
     c->kernel = v[0]; c->tile_m = v[1]; c->tile_n = v[2]; c->tile_k = v[3]; c->stages = v[4]; c->cta_pair = v[5];
     c->split_k = v[6]; c->store_mode = v[7]; c->raster = v[8]; c->patch_w = v[9]; c->patch_h = v[10];
     c->k_stagger = v[11];
+    c->halo = v[12];
 }
 
 // ------------------------------------------------------------------ problem descriptions
@@ -241,6 +247,18 @@ int umma_max_stages(int tile_m, int tile_n, int smem_limit, int store_mode) {
 
 // Accumulator slots (128 x tile_n each) kept in TMEM: a 256-row tile uses two per tile, and gets four
 // when they fit so that the epilogue still overlaps the next tile's main loop.
+// Halo-reuse convolution: 8 x 16 output-pixel patches, input window kept in shared memory across the taps.
+constexpr int kHaloPatchW = 8, kHaloPatchH = 16, kHaloAStages = 2;
+int halo_tile_bytes(int64_t R, int64_t S) {
+    const int64_t b = (kHaloPatchW + S - 1) * (kHaloPatchH + R - 1) * 128;
+    return static_cast<int>((b + 1023) / 1024 * 1024);
+}
+int halo_max_stages(int tile_m, int tile_n, int64_t R, int64_t S, int smem_limit, int store_mode) {
+    const int a = kHaloAStages * (tile_m / 128) * halo_tile_bytes(R, S);
+    const int left = smem_limit - kStaticSmemReserve - 1024 - staging_bytes_for(tile_m, store_mode) - a;
+    return left <= 0 ? 0 : std::min(left / (tile_n * 128), tdx::kMaxStages);
+}
+
 int tmem_slots_for(int tile_m, int bn) { return (tile_m == 256 && bn <= 128) ? 4 : 2; }
 int tmem_cols_for(int tile_m, int bn) {
     int c = 32;
@@ -251,7 +269,7 @@ int tmem_cols_for(int tile_m, int bn) {
 // Static feasibility of a fully specified tensor-core configuration (the search-space constraints).
 // Returns 0 when feasible, else a short reason.
 const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num_kb, int smem_limit, bool conv,
-                               int64_t N) {
+                               int64_t N, int64_t R = 1, int64_t S = 1) {
     if (c.tile_m != 128 && c.tile_m != 256) return "tile_m must be 128 or 256";
     if (c.tile_k != 64) return "tile_k must be 64";
     if (c.cta_pair != 1) return "cta_pair must be 1";
@@ -263,6 +281,15 @@ const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num
     }
     if (c.tile_n < 32 || c.tile_n > 256 || c.tile_n % 32) return "tile_n must be a multiple of 32 in [32, 256]";
     if (b_mn_major && c.tile_n % 64) return "tile_n must be a multiple of 64 when B is read N-major";
+    if (!conv && c.halo > 1) return "halo applies to the convolution only";
+    if (conv && c.halo != 1 && c.halo != 2) return "halo must be 1 (per-tap loads) or 2 (halo tile kept in shared memory)";
+    if (conv && c.halo == 2) {
+        if (R * S < 2) return "halo reuse needs a filter with more than one tap";
+        if (c.patch_w != kHaloPatchW || c.patch_h != kHaloPatchH) return "halo reuse works on 8 x 16 patches";
+        if (kHaloPatchW + S - 1 > 256 || kHaloPatchH + R - 1 > 256) return "filter too large for a halo tile";
+        if (c.stages < 2 || c.stages > halo_max_stages(c.tile_m, c.tile_n, R, S, smem_limit, c.store_mode))
+            return "stages outside the shared-memory budget";
+    } else
     if (c.stages < 2 || c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode)) return "stages outside the shared-memory budget";
     if (c.split_k < 1) return "split_k must be >= 1";
     if (conv && c.split_k != 1) return "conv has no split-K";
@@ -339,14 +366,19 @@ void default_umma_config(int64_t tiles_m, int64_t N, int64_t num_kb, bool b_mn_m
 
 // ------------------------------------------------------------------ launches
 int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
-                const UmmaParams& p, cudaStream_t st) {
+                const UmmaParams& p, cudaStream_t st, bool halo = false) {
     const long long items = static_cast<long long>(p.tiles_m) * p.tiles_n * p.split_k;
     const int grid = static_cast<int>(std::min<long long>(items, ctx->sm_count));
-    const size_t smem = static_cast<size_t>(p.stages) * ((p.bm + p.bn) * 128) + 1024 +
-                        staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
+    size_t smem = static_cast<size_t>(p.stages) * ((p.bm + p.bn) * 128) + 1024 +
+                  staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
+    if (halo)
+        smem = static_cast<size_t>(p.a_stages) * (p.bm / 128) * p.halo_bytes + static_cast<size_t>(p.stages) * p.bn * 128 +
+               1024 + staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
     // producer warp, MMA warp, then 16 epilogue warps (staged epilogue) or 4 per 128-row half (direct)
     const int threads = p.tma_store ? 576 : (p.bm == 256 ? 320 : 192);
-    if (conv)
+    if (halo)
+        tdx::umma_conv_halo_kernel<<<grid, threads, smem, st>>>(ma, mb, mc, p);
+    else if (conv)
         tdx::umma_contract_kernel<true><<<grid, threads, smem, st>>>(ma, mb, mc, p);
     else
         tdx::umma_contract_kernel<false><<<grid, threads, smem, st>>>(ma, mb, mc, p);
@@ -468,6 +500,14 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     p.bm = cfg.tile_m;
     p.slots = tmem_slots_for(cfg.tile_m, cfg.tile_n);
     p.nb = cfg.tile_m / (p.bw * p.bh);
+    const bool halo = cfg.halo == 2;
+    if (halo) {
+        p.R = static_cast<int>(c.R);
+        p.hpitch = static_cast<int>(kHaloPatchW + c.S - 1);
+        p.hrows = static_cast<int>(kHaloPatchH + c.R - 1);
+        p.halo_bytes = halo_tile_bytes(c.R, c.S);
+        p.a_stages = kHaloAStages;
+    }
     p.patches_w = static_cast<int>(ceil_div(c.Q, p.bw));
     p.patches_h = static_cast<int>(ceil_div(c.P, p.bh));
     const int64_t total_patches = c.N * p.patches_w * p.patches_h;
@@ -505,7 +545,7 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
                             static_cast<uint64_t>(c.N)};
         uint64_t str[3] = {static_cast<uint64_t>(c.Cin) * 2, static_cast<uint64_t>(c.W * c.Cin) * 2,
                            static_cast<uint64_t>(c.H * c.W * c.Cin) * 2};
-        uint32_t box[4] = {64, static_cast<uint32_t>(p.bw), static_cast<uint32_t>(p.bh), 1};
+        uint32_t box[4] = {64, static_cast<uint32_t>(halo ? p.hpitch : p.bw), static_cast<uint32_t>(halo ? p.hrows : p.bh), 1};
         int rc = get_tensor_map(ctx, x, 4, dims, str, box, &ma);
         if (rc) return rc;
     }
@@ -530,7 +570,7 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
         int rc = get_tensor_map(ctx, y, 4, dims, str, box, &mc, 64);
         if (rc) return rc;
     }
-    return launch_umma(ctx, true, ma, mb, mc, p, st);
+    return launch_umma(ctx, true, ma, mb, mc, p, st, halo);
 }
 
 void gemm_strides(const GemmProblem& g, long long* sa_i, long long* sa_k, long long* sb_k, long long* sb_j) {
@@ -702,6 +742,8 @@ int resolve_conv_config(const ConvProblem& cp, const tdx_config* user, int sm_co
     if (c.kernel == TDX_KERNEL_GENERIC) { *out = c; return TDX_OK; }
     if (cp.dtype != TDX_BF16) return fail(TDX_ERR_CONFIG, "the tensor-core kernel is bf16 only");
     if (!layout_ok) return fail(TDX_ERR_ALIGNMENT, "tensor-core conv needs stride 1 and Cin %% 8 == 0");
+    if (c.halo == 0) c.halo = 1;
+    if (c.halo == 2 && c.patch_w == 0 && c.patch_h == 0) { c.patch_w = kHaloPatchW; c.patch_h = kHaloPatchH; }
     if (c.patch_w == 0 && c.patch_h == 0) choose_patch(cp.P, cp.Q, &c.patch_w, &c.patch_h);
     if (!patch_ok(c.patch_w, c.patch_h)) return fail(TDX_ERR_CONFIG, "infeasible config: patch %dx%d", c.patch_w, c.patch_h);
     const int nb = 128 / (c.patch_w * c.patch_h);
@@ -716,11 +758,13 @@ int resolve_conv_config(const ConvProblem& cp, const tdx_config* user, int sm_co
     if (c.split_k == 0) c.split_k = 1;
     if (c.store_mode == 0) {
         c.store_mode = (cp.Cout % 8 == 0 && c.patch_w * c.patch_h >= 32) ? 2 : 1;
-        if (c.store_mode == 2 && c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, 2)) c.store_mode = 1;
+        if (c.store_mode == 2 && c.halo != 2 && c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, 2)) c.store_mode = 1;
     }
-    if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode));
+    if (c.stages == 0)
+        c.stages = c.halo == 2 ? std::max(2, halo_max_stages(c.tile_m, c.tile_n, cp.R, cp.S, smem_limit, c.store_mode))
+                               : std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode));
     if (!user && !from_cache) c.raster = d.raster;
-    const char* why = umma_config_reason(c, false, num_kb, smem_limit, true, cp.Cout);
+    const char* why = umma_config_reason(c, false, num_kb, smem_limit, true, cp.Cout, cp.R, cp.S);
     if (why) return fail(TDX_ERR_CONFIG, "infeasible config: %s", why);
     *out = c;
     return TDX_OK;
@@ -846,7 +890,8 @@ void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int 
                                 c.tile_m = tm; c.tile_n = bn; c.tile_k = 64; c.stages = st; c.cta_pair = 1;
                                 c.split_k = sk; c.store_mode = sm; c.raster = raster; c.k_stagger = stagger;
                                 c.patch_w = patch_w; c.patch_h = patch_h;
-                                if (umma_config_reason(c, b_mn, num_kb, smem_limit, conv, N) == nullptr) out->push_back(c);
+                                c.halo = conv ? 1 : 0;
+                                if (umma_config_reason(c, b_mn, num_kb, smem_limit, conv, N, 3, 3) == nullptr) out->push_back(c);
                             }
                 }
         }
@@ -886,6 +931,28 @@ int enum_conv(const ConvProblem& cp, int sm_count, int smem_limit, std::vector<t
         c.kernel = TDX_KERNEL_GENERIC;
         v->push_back(c);
         return TDX_OK;
+    }
+    // halo-reuse candidates (8 x 16 patches)
+    if (cp.R * cp.S > 1) {
+        const int64_t num_kb = cp.R * cp.S * ceil_div(cp.Cin, 64);
+        for (int tm : {256, 128})
+            for (int bn = 256; bn >= 32; bn -= 32) {
+                if (bn > 32 && bn - 32 >= cp.Cout) continue;
+                if (bn != 256 && bn != 128 && bn != 64 && bn != 32 && cp.Cout % bn) continue;
+                const int sm = cp.Cout % 8 == 0 ? 2 : 1;
+                const int max_st = halo_max_stages(tm, bn, cp.R, cp.S, smem_limit, sm);
+                for (int st : {max_st, max_st - 1, max_st - 2}) {
+                    if (st < 2) continue;
+                    for (int raster : {0, 8, 2}) {
+                        tdx_config c;
+                        std::memset(&c, 0, sizeof c);
+                        c.kernel = TDX_KERNEL_UMMA;
+                        c.tile_m = tm; c.tile_n = bn; c.tile_k = 64; c.stages = st; c.cta_pair = 1; c.split_k = 1;
+                        c.store_mode = sm; c.raster = raster; c.patch_w = kHaloPatchW; c.patch_h = kHaloPatchH; c.halo = 2;
+                        if (umma_config_reason(c, false, num_kb, smem_limit, true, cp.Cout, cp.R, cp.S) == nullptr) v->push_back(c);
+                    }
+                }
+            }
     }
     // patch shapes: every shape whose padded area is within 15 % of the best one
     int bbw, bbh;
@@ -1196,10 +1263,10 @@ int tdx_tune_save(const char* json_path) {
     fprintf(f, "{\"version\": 1, \"entries\": [\n");
     size_t i = 0;
     for (const auto& kv : g_tune) {
-        int v[12];
+        int v[13];
         cfg_to_ints(kv.second.cfg, v);
         fprintf(f, "  {\"key\": \"%s\", \"cfg\": [", kv.first.c_str());
-        for (int j = 0; j < 12; ++j) fprintf(f, "%d%s", v[j], j < 11 ? ", " : "");
+        for (int j = 0; j < 13; ++j) fprintf(f, "%d%s", v[j], j < 12 ? ", " : "");
         fprintf(f, "], \"us\": %.3f}%s\n", kv.second.us, ++i < g_tune.size() ? "," : "");
     }
     fprintf(f, "]}\n");
@@ -1225,11 +1292,11 @@ int tdx_tune_load(const char* json_path) {
         const size_t b1 = b0 == std::string::npos ? b0 : text.find(']', b0);
         if (b1 == std::string::npos) return fail(TDX_ERR_INVALID_ARG, "malformed tuning cache %s", json_path);
         const std::string key = text.substr(q0 + 1, q1 - q0 - 1);
-        int v[12] = {0};
+        int v[13] = {0};
         int n = 0;
         const char* s = text.c_str() + b0 + 1;
         const char* end = text.c_str() + b1;
-        while (s < end && n < 12) {
+        while (s < end && n < 13) {
             char* next;
             long val = strtol(s, &next, 10);
             if (next == s) break;
@@ -1237,7 +1304,7 @@ int tdx_tune_load(const char* json_path) {
             s = next;
             while (s < end && (*s == ',' || *s == ' ')) ++s;
         }
-        if (n != 11 && n != 12) return fail(TDX_ERR_INVALID_ARG, "malformed cfg list in %s", json_path);
+        if (n < 11 || n > 13) return fail(TDX_ERR_INVALID_ARG, "malformed cfg list in %s", json_path);
         TuneEntry e;
         ints_to_cfg(v, &e.cfg);
         e.us = 0.0f;

@@ -1,0 +1,214 @@
+// Convolution kernel that keeps the input halo tile in shared memory across the filter taps.
+//
+// The per-tap kernel (umma_contract_kernel<true>) fetches the shifted input window again for every
+// filter tap: R*S fetches of the same pixels from L2.  Here a 128-row MMA tile is an 8-wide, 16-high
+// patch of output pixels; its (8 + S - 1) x (16 + R - 1) input window for one 64-channel chunk is loaded
+// ONCE (one TMA box, zero fill outside the image), and tap (r, s) is read straight out of it: output
+// pixel (h, w) of the patch needs window pixel (h + r, w + s), i.e. the 8-row groups of the A operand
+// start at window row r, column s and are one window row (hpitch * 128 bytes) apart -- exactly what
+// the shared-memory descriptor's start address and stride-dimension offset express.  The 128-byte
+// swizzle is a function of the shared-memory address, so a start that is not 1024-byte aligned reads
+// consistently what the copy engine wrote.
+//
+// Two rings: halo tiles (a_stages deep, one per channel chunk and 128-row half) and filter slices
+// (stages deep, one per (chunk, tap)).  Roles, accumulator slots, epilogue and bounded waits are those
+// of umma_contract_kernel.
+#pragma once
+#include "umma_kernel.cuh"
+
+namespace tdx {
+
+constexpr int kMaxAStages = 3;
+
+// output patch of 128-row half `half` of tile `m_blk`: image n and top-left output pixel (p0, q0)
+__device__ __forceinline__ void halo_patch_origin(const UmmaParams& p, int m_blk, int half, int mh, int* n, int* p0,
+                                                  int* q0) {
+    const int patch = m_blk * mh + half;
+    const int ppi = p.patches_w * p.patches_h;
+    *n = patch / ppi;
+    const int rem = patch - *n * ppi;
+    const int ph = rem / p.patches_w;
+    *p0 = ph * p.bh;
+    *q0 = (rem - ph * p.patches_w) * p.bw;
+}
+
+__global__ void __launch_bounds__(576, 1)
+umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                      const __grid_constant__ CUtensorMap tmC, const UmmaParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t afull_bar[kMaxAStages];
+    __shared__ __align__(8) uint64_t aempty_bar[kMaxAStages];
+    __shared__ __align__(8) uint64_t bfull_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t bempty_bar[kMaxStages];
+    __shared__ __align__(8) uint64_t tfull_bar[kMaxSlots];
+    __shared__ __align__(8) uint64_t tempty_bar[kMaxSlots];
+    __shared__ uint32_t s_tmem_base;
+    __shared__ int s_abort;
+
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int mh = p.bm / kHalfM;
+    const uint32_t b_bytes = static_cast<uint32_t>(p.bn) * 128u;
+    const uint32_t a_stage_bytes = static_cast<uint32_t>(mh * p.halo_bytes);
+    uint8_t* a_ring = smem;
+    uint8_t* b_ring = smem + static_cast<size_t>(p.a_stages) * a_stage_bytes;
+    uint8_t* staging = b_ring + static_cast<size_t>(p.stages) * b_bytes;
+    volatile int* abort_flag = &s_abort;
+    const int taps = p.R * p.S;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.a_stages; ++s) {
+            ptx::mbar_init(&afull_bar[s], 1);
+            ptx::mbar_init(&aempty_bar[s], 1);
+        }
+        for (int s = 0; s < p.stages; ++s) {
+            ptx::mbar_init(&bfull_bar[s], 1);
+            ptx::mbar_init(&bempty_bar[s], 1);
+        }
+        for (int b = 0; b < p.slots; ++b) {
+            ptx::mbar_init(&tfull_bar[b], 1);
+            ptx::mbar_init(&tempty_bar[b], static_cast<uint32_t>(((blockDim.x >> 5) - 2) / mh));
+        }
+        s_abort = 0;
+        ptx::fence_barrier_init();
+        ptx::tma_prefetch_desc(&tmA);
+        ptx::tma_prefetch_desc(&tmB);
+        if (p.tma_store) ptx::tma_prefetch_desc(&tmC);
+    }
+    if (warp == 1) {
+        __syncwarp();
+        ptx::tmem_alloc(&s_tmem_base, static_cast<uint32_t>(p.tmem_cols));
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = s_tmem_base;
+    const int total_items = p.tiles_m * p.tiles_n;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer: two cursors, halo tiles ahead of slices
+        if (lane == 0) {
+            int a_item = blockIdx.x, a_cc = 0, a_buf = 0;     // next halo load to issue
+            uint32_t a_phase = 0;
+            long long a_issued = 0, b_chunk = 0;             // halo loads issued / channel chunks started by the slice cursor
+            int b_stage = 0;
+            uint32_t b_phase = 0;
+            bool ok = true;
+            const uint32_t halo_tx = static_cast<uint32_t>(mh * p.hpitch * p.hrows) * 128u;
+
+            auto issue_halo = [&]() {
+                const TileCoord t = decode_item(p, a_item);
+                uint64_t* bar = &afull_bar[a_buf];
+                ptx::mbar_arrive_expect_tx(bar, halo_tx);
+                for (int h = 0; h < mh; ++h) {
+                    int n, p0, q0;
+                    halo_patch_origin(p, t.m_blk, h, mh, &n, &p0, &q0);
+                    ptx::tma_load_4d(a_ring + static_cast<size_t>(a_buf) * a_stage_bytes + h * p.halo_bytes, &tmA, bar,
+                                     a_cc * kBK, q0 - p.pad, p0 - p.pad, n);
+                }
+                if (++a_buf == p.a_stages) { a_buf = 0; a_phase ^= 1u; }
+                if (++a_cc == p.cchunks) { a_cc = 0; a_item += gridDim.x; }
+                ++a_issued;
+            };
+
+            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
+                const TileCoord t = decode_item(p, item);
+                for (int cc = 0; ok && cc < p.cchunks; ++cc, ++b_chunk) {
+                    // the halo tile of this chunk must be on its way before its filter slices queue up behind it
+                    while (ok && a_issued <= b_chunk) {
+                        if (!wait_bounded(&aempty_bar[a_buf], a_phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) ok = false;
+                        else issue_halo();
+                    }
+                    for (int tap = 0; ok && tap < taps; ++tap) {
+                        // run ahead with halo tiles whenever a buffer is free
+                        if (a_item < total_items && ptx::mbar_try_wait(&aempty_bar[a_buf], a_phase ^ 1u)) issue_halo();
+                        if (!wait_bounded(&bempty_bar[b_stage], b_phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) {
+                            ok = false;
+                            break;
+                        }
+                        uint64_t* bar = &bfull_bar[b_stage];
+                        ptx::mbar_arrive_expect_tx(bar, b_bytes);
+                        ptx::tma_load_3d(b_ring + static_cast<size_t>(b_stage) * b_bytes, &tmB, bar, cc * kBK, tap,
+                                         t.n_blk * p.bn);
+                        if (++b_stage == p.stages) { b_stage = 0; b_phase ^= 1u; }
+                    }
+                }
+            }
+            if (!ok) {
+                for (int i = 0; i < 64; ++i) __nanosleep(2000);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = ptx::make_idesc_bf16_f32(kHalfM, p.bn, 0, 0);
+            const uint32_t a_sbo = static_cast<uint32_t>(p.hpitch) * 128u;     // one window row between 8-row groups
+            int a_buf = 0, b_stage = 0, local = 0;
+            uint32_t a_phase = 0, b_phase = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++local) {
+                uint32_t d_tmem[2] = {0u, 0u};
+                int slot[2] = {0, 0};
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (h < mh && ok) {
+                        const int idx = local * mh + h;
+                        slot[h] = idx % p.slots;
+                        const uint32_t aphase = (idx / p.slots) & 1;
+                        d_tmem[h] = tmem_base + static_cast<uint32_t>(slot[h] * p.bn);
+                        if (!wait_bounded(&tempty_bar[slot[h]], aphase ^ 1u, abort_flag, p.status, kTimeoutMma)) ok = false;
+                    }
+                }
+                if (!ok) break;
+                ptx::tc_fence_after_sync();
+                for (int cc = 0; ok && cc < p.cchunks; ++cc) {
+                    if (!wait_bounded(&afull_bar[a_buf], a_phase, abort_flag, p.status, kTimeoutMma)) { ok = false; break; }
+                    const uint32_t halo_addr = ptx::smem_u32(a_ring + static_cast<size_t>(a_buf) * a_stage_bytes);
+                    for (int tap = 0; tap < taps; ++tap) {
+                        if (!wait_bounded(&bfull_bar[b_stage], b_phase, abort_flag, p.status, kTimeoutMma)) { ok = false; break; }
+                        ptx::tc_fence_after_sync();
+                        const int r = tap / p.S;
+                        const int s = tap - r * p.S;
+                        const uint32_t a_off = static_cast<uint32_t>(r * p.hpitch + s) * 128u;
+                        const uint32_t b_addr = ptx::smem_u32(b_ring + static_cast<size_t>(b_stage) * b_bytes);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            if (h < mh) {
+#pragma unroll
+                                for (int j = 0; j < kBK / kUmmaK; ++j) {
+                                    const uint64_t adesc = ptx::make_smem_desc_sw128(
+                                        halo_addr + h * p.halo_bytes + a_off + j * 32u, 16u, a_sbo);
+                                    const uint64_t bdesc = ptx::make_smem_desc_sw128(b_addr + j * 32u, 16u, 1024u);
+                                    ptx::umma_bf16(d_tmem[h], adesc, bdesc, idesc, (cc > 0 || tap > 0 || j > 0) ? 1u : 0u);
+                                }
+                            }
+                        }
+                        ptx::umma_commit(&bempty_bar[b_stage]);
+                        if (++b_stage == p.stages) { b_stage = 0; b_phase ^= 1u; }
+                    }
+                    if (!ok) break;
+                    ptx::umma_commit(&aempty_bar[a_buf]);
+                    if (++a_buf == p.a_stages) { a_buf = 0; a_phase ^= 1u; }
+                }
+                if (ok) {
+                    ptx::umma_commit(&tfull_bar[slot[0]]);
+                    if (mh == 2) ptx::umma_commit(&tfull_bar[slot[1]]);
+                }
+            }
+        }
+    } else {
+        epilogue_role<true>(p, &tmC, staging, tmem_base, tfull_bar, tempty_bar, abort_flag, mh, warp, lane, total_items);
+    }
+
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        __syncwarp();
+        ptx::tmem_dealloc(tmem_base, static_cast<uint32_t>(p.tmem_cols));
+    }
+}
+
+}  // namespace tdx

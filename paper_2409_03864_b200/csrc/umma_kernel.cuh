@@ -62,6 +62,12 @@ struct UmmaParams {
     int bw, bh, nb;           // spatial patch (bw x bh output pixels), patches per tile = bm / (bw*bh)
     int patches_w, patches_h; // patches per image along Q and P
     int P, Q, Nimg, S, pad, cchunks;
+    // halo-reuse convolution (umma_conv_halo_kernel): the input window of an 8 x 16 pixel patch is loaded once
+    // per channel chunk and shared by all filter taps
+    int R;                    // filter rows (taps = R * S)
+    int hpitch, hrows;        // halo tile: (8 + S - 1) pixels wide, (16 + R - 1) pixels high
+    int halo_bytes;           // hpitch * hrows * 128 rounded up to 1024
+    int a_stages;             // halo tiles in flight per 128-row half
     int* status;              // device status word
 };
 
@@ -101,6 +107,207 @@ __device__ __forceinline__ TileCoord decode_item(const UmmaParams& p, int item) 
     t.kb0 = t.split * p.kb_per_split;
     t.kb1 = min(p.num_kb, t.kb0 + p.kb_per_split);
     return t;
+}
+
+// Epilogue role (all warps from the third on).  With the staged epilogue there are 16 of them (4 per TMEM
+// lane quarter) and the warps of a quarter take the 32-column steps round robin; the direct epilogue has one
+// warp per quarter and 128-row half.
+template <bool kConv>
+__device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtensorMap* tmC, uint8_t* staging_base,
+                                              uint32_t tmem_base, uint64_t* tfull_bar, uint64_t* tempty_bar,
+                                              volatile int* abort_flag, int mh, int warp, int lane, int total_items) {
+    const int ew = warp - 2;
+    const int nwarps_epi = (static_cast<int>(blockDim.x) >> 5) - 2;
+    const int ncgrp = nwarps_epi / (4 * mh);      // warps sharing one (half, quarter)
+    const int half = (ew >> 2) % mh;              // which 128-row half of the tile this warp drains
+    const int cgrp = (ew >> 2) / mh;              // which share of the columns
+    const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
+    const int row_in_tile = half * kHalfM + quarter * 32 + lane;
+    int local = 0;
+    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++local) {
+        const TileCoord t = decode_item(p, item);
+        const int sidx = local * mh + half;
+        const int buf = sidx % p.slots;
+        const uint32_t aphase = (sidx / p.slots) & 1;
+        if (!wait_bounded(&tfull_bar[buf], aphase, abort_flag, p.status, kTimeoutEpilogue)) break;
+        ptx::tc_fence_after_sync();
+
+        long long grow;
+        bool valid;
+        if (kConv) {
+            const int per_patch = p.bw * p.bh;
+            const int pl = row_in_tile / per_patch;
+            const int within = row_in_tile - pl * per_patch;
+            const int hl = within / p.bw;
+            const int wl = within - hl * p.bw;
+            const int patch = t.m_blk * p.nb + pl;
+            const int ppi = p.patches_w * p.patches_h;
+            const int n = patch / ppi;
+            const int rem = patch - n * ppi;
+            const int ph = rem / p.patches_w;
+            const int pw = rem - ph * p.patches_w;
+            const int pp = ph * p.bh + hl;
+            const int qq = pw * p.bw + wl;
+            valid = (n < p.Nimg) && (pp < p.P) && (qq < p.Q);
+            grow = (static_cast<long long>(n) * p.P + pp) * p.Q + qq;
+        } else {
+            grow = static_cast<long long>(t.m_blk) * p.bm + row_in_tile;
+            valid = grow < p.M;
+        }
+
+        if (p.tma_store && p.split_k == 1) {
+            // ---- staged path: 32 rows x 32 columns per warp and step, written by the copy engine
+            uint8_t* stage_buf = staging_base + (warp - 2) * 2048;
+            const int wrow0 = half * kHalfM + quarter * 32;      // first tile row of this warp
+            int sc1 = 0, sc2 = 0, sc3 = 0;                       // store coordinates above the column
+            bool box_ok;
+            if (kConv) {
+                const int per_patch = p.bw * p.bh;
+                const int pl = wrow0 / per_patch;
+                const int within = wrow0 - pl * per_patch;
+                const int hl0 = within / p.bw;
+                const int wl0 = within - hl0 * p.bw;
+                const int patch = t.m_blk * p.nb + pl;
+                const int ppi = p.patches_w * p.patches_h;
+                const int n = patch / ppi;
+                const int rem = patch - n * ppi;
+                const int ph = rem / p.patches_w;
+                const int pw = rem - ph * p.patches_w;
+                sc1 = pw * p.bw + wl0;
+                sc2 = ph * p.bh + hl0;
+                sc3 = n;
+                box_ok = (n < p.Nimg) && (sc2 < p.P) && (sc1 < p.Q);
+            } else {
+                sc1 = t.m_blk * p.bm + wrow0;
+                box_ok = sc1 < p.M;
+            }
+            // 64-byte swizzle of the staging block: 16-byte slot c of row `lane` lives at slot c ^ ((lane / 2) % 4)
+            uint8_t* my_row = stage_buf + lane * 64;
+            const int sw = (lane >> 1) & 3;
+            const bool plain = (p.bias == nullptr) && (p.relu == 0);
+            for (int c0 = cgrp * 32; c0 < p.bn; c0 += ncgrp * 32) {
+                uint32_t r[32];
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                                       static_cast<uint32_t>(buf * p.bn + c0);
+                ptx::tmem_ld_32x32b_x32(taddr, r);
+                ptx::tmem_ld_wait();
+                const int col0 = t.n_blk * p.bn + c0;
+                // the previous store of this warp must have finished reading the staging block
+                if (lane == 0) ptx::tma_store_wait_read<0>();
+                __syncwarp();
+                if (plain) {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(p.alpha * __uint_as_float(r[g * 8 + e * 2]),
+                                                                      p.alpha * __uint_as_float(r[g * 8 + e * 2 + 1]));
+                            pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+                        }
+                        *reinterpret_cast<uint4*>(my_row + ((g ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                } else {
+                    const int last = p.N - 1;    // columns past N are clipped by the store; keep the bias index in range
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        uint32_t pk[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const int j = g * 8 + e * 2;
+                            float x0 = p.alpha * __uint_as_float(r[j]);
+                            float x1 = p.alpha * __uint_as_float(r[j + 1]);
+                            if (p.bias != nullptr) {
+                                x0 += __ldg(p.bias + min(col0 + j, last));
+                                x1 += __ldg(p.bias + min(col0 + j + 1, last));
+                            }
+                            if (p.relu) {
+                                x0 = fmaxf(x0, 0.0f);
+                                x1 = fmaxf(x1, 0.0f);
+                            }
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
+                            pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+                        }
+                        *reinterpret_cast<uint4*>(my_row + ((g ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    }
+                }
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0 && box_ok && col0 < p.N) {
+                    if (kConv)
+                        ptx::tma_store_4d(tmC, stage_buf, col0, sc1, sc2, sc3);
+                    else
+                        ptx::tma_store_2d(tmC, stage_buf, col0, sc1);
+                    ptx::tma_store_commit();
+                }
+                __syncwarp();
+            }
+        } else
+        for (int c0 = 0; c0 < p.bn; c0 += 32) {
+            uint32_t r[32];
+            const uint32_t taddr =
+                tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * p.bn + c0);
+            ptx::tmem_ld_32x32b_x32(taddr, r);
+            ptx::tmem_ld_wait();
+            const int col0 = t.n_blk * p.bn + c0;
+            if (valid && col0 < p.N) {
+            if (p.split_k > 1) {
+                float* dst = p.partial + (static_cast<long long>(t.split) * p.M + grow) * p.N + col0;
+                if (p.vec_store) {
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        if (col0 + g * 4 < p.N) {
+                            float4 v = make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]),
+                                                   __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
+                            *reinterpret_cast<float4*>(dst + g * 4) = v;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (col0 + j < p.N) dst[j] = __uint_as_float(r[j]);
+                }
+            } else {
+                float v[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    float x = p.alpha * __uint_as_float(r[j]);
+                    if (p.bias != nullptr && col0 + j < p.N) x += __ldg(p.bias + col0 + j);
+                    if (p.relu) x = fmaxf(x, 0.0f);
+                    v[j] = x;
+                }
+                __nv_bfloat16* dst = p.C + grow * p.ldc + col0;
+                if (p.vec_store) {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        if (col0 + g * 8 < p.N) {
+                            uint4 pk;
+                            __nv_bfloat162 h0 = __floats2bfloat162_rn(v[g * 8 + 0], v[g * 8 + 1]);
+                            __nv_bfloat162 h1 = __floats2bfloat162_rn(v[g * 8 + 2], v[g * 8 + 3]);
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(v[g * 8 + 4], v[g * 8 + 5]);
+                            __nv_bfloat162 h3 = __floats2bfloat162_rn(v[g * 8 + 6], v[g * 8 + 7]);
+                            pk.x = *reinterpret_cast<uint32_t*>(&h0);
+                            pk.y = *reinterpret_cast<uint32_t*>(&h1);
+                            pk.z = *reinterpret_cast<uint32_t*>(&h2);
+                            pk.w = *reinterpret_cast<uint32_t*>(&h3);
+                            *reinterpret_cast<uint4*>(dst + g * 8) = pk;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(v[j]);
+                }
+            }
+            }
+            __syncwarp();   // reconverge before the next warp-aligned TMEM load
+        }
+        ptx::tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&tempty_bar[buf]);
+    }
+    // shared memory must stay alive until the copy engine has drained this warp's last store
+    if (p.tma_store && lane == 0) ptx::tma_store_wait_all<0>();
 }
 
 template <bool kConv>
@@ -280,202 +487,8 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (4 warps per 128-row half)
-        // epilogue warp e = warp - 2: with the staged epilogue there are 16 of them (4 per TMEM lane
-        // quarter) and the warps of a quarter take the 32-column steps round robin; the direct
-        // epilogue has one warp per quarter and 128-row half.
-        const int ew = warp - 2;
-        const int nwarps_epi = (static_cast<int>(blockDim.x) >> 5) - 2;
-        const int ncgrp = nwarps_epi / (4 * mh);      // warps sharing one (half, quarter)
-        const int half = (ew >> 2) % mh;              // which 128-row half of the tile this warp drains
-        const int cgrp = (ew >> 2) / mh;              // which share of the columns
-        const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
-        const int row_in_tile = half * kHalfM + quarter * 32 + lane;
-        int local = 0;
-        for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++local) {
-            const TileCoord t = decode_item(p, item);
-            const int sidx = local * mh + half;
-            const int buf = sidx % p.slots;
-            const uint32_t aphase = (sidx / p.slots) & 1;
-            if (!wait_bounded(&tfull_bar[buf], aphase, abort_flag, p.status, kTimeoutEpilogue)) break;
-            ptx::tc_fence_after_sync();
-
-            long long grow;
-            bool valid;
-            if (kConv) {
-                const int per_patch = p.bw * p.bh;
-                const int pl = row_in_tile / per_patch;
-                const int within = row_in_tile - pl * per_patch;
-                const int hl = within / p.bw;
-                const int wl = within - hl * p.bw;
-                const int patch = t.m_blk * p.nb + pl;
-                const int ppi = p.patches_w * p.patches_h;
-                const int n = patch / ppi;
-                const int rem = patch - n * ppi;
-                const int ph = rem / p.patches_w;
-                const int pw = rem - ph * p.patches_w;
-                const int pp = ph * p.bh + hl;
-                const int qq = pw * p.bw + wl;
-                valid = (n < p.Nimg) && (pp < p.P) && (qq < p.Q);
-                grow = (static_cast<long long>(n) * p.P + pp) * p.Q + qq;
-            } else {
-                grow = static_cast<long long>(t.m_blk) * p.bm + row_in_tile;
-                valid = grow < p.M;
-            }
-
-            if (p.tma_store && p.split_k == 1) {
-                // ---- staged path: 32 rows x 32 columns per warp and step, written by the copy engine
-                uint8_t* stage_buf = smem + static_cast<size_t>(p.stages) * stage_bytes + (warp - 2) * 2048;
-                const int wrow0 = half * kHalfM + quarter * 32;      // first tile row of this warp
-                int sc1 = 0, sc2 = 0, sc3 = 0;                       // store coordinates above the column
-                bool box_ok;
-                if (kConv) {
-                    const int per_patch = p.bw * p.bh;
-                    const int pl = wrow0 / per_patch;
-                    const int within = wrow0 - pl * per_patch;
-                    const int hl0 = within / p.bw;
-                    const int wl0 = within - hl0 * p.bw;
-                    const int patch = t.m_blk * p.nb + pl;
-                    const int ppi = p.patches_w * p.patches_h;
-                    const int n = patch / ppi;
-                    const int rem = patch - n * ppi;
-                    const int ph = rem / p.patches_w;
-                    const int pw = rem - ph * p.patches_w;
-                    sc1 = pw * p.bw + wl0;
-                    sc2 = ph * p.bh + hl0;
-                    sc3 = n;
-                    box_ok = (n < p.Nimg) && (sc2 < p.P) && (sc1 < p.Q);
-                } else {
-                    sc1 = t.m_blk * p.bm + wrow0;
-                    box_ok = sc1 < p.M;
-                }
-                // 64-byte swizzle of the staging block: 16-byte slot c of row `lane` lives at slot c ^ ((lane / 2) % 4)
-                uint8_t* my_row = stage_buf + lane * 64;
-                const int sw = (lane >> 1) & 3;
-                const bool plain = (p.bias == nullptr) && (p.relu == 0);
-                for (int c0 = cgrp * 32; c0 < p.bn; c0 += ncgrp * 32) {
-                    uint32_t r[32];
-                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
-                                           static_cast<uint32_t>(buf * p.bn + c0);
-                    ptx::tmem_ld_32x32b_x32(taddr, r);
-                    ptx::tmem_ld_wait();
-                    const int col0 = t.n_blk * p.bn + c0;
-                    // the previous store of this warp must have finished reading the staging block
-                    if (lane == 0) ptx::tma_store_wait_read<0>();
-                    __syncwarp();
-                    if (plain) {
-#pragma unroll
-                        for (int g = 0; g < 4; ++g) {
-                            uint32_t pk[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                __nv_bfloat162 h2 = __floats2bfloat162_rn(p.alpha * __uint_as_float(r[g * 8 + e * 2]),
-                                                                          p.alpha * __uint_as_float(r[g * 8 + e * 2 + 1]));
-                                pk[e] = *reinterpret_cast<uint32_t*>(&h2);
-                            }
-                            *reinterpret_cast<uint4*>(my_row + ((g ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                        }
-                    } else {
-                        const int last = p.N - 1;    // columns past N are clipped by the store; keep the bias index in range
-#pragma unroll
-                        for (int g = 0; g < 4; ++g) {
-                            uint32_t pk[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const int j = g * 8 + e * 2;
-                                float x0 = p.alpha * __uint_as_float(r[j]);
-                                float x1 = p.alpha * __uint_as_float(r[j + 1]);
-                                if (p.bias != nullptr) {
-                                    x0 += __ldg(p.bias + min(col0 + j, last));
-                                    x1 += __ldg(p.bias + min(col0 + j + 1, last));
-                                }
-                                if (p.relu) {
-                                    x0 = fmaxf(x0, 0.0f);
-                                    x1 = fmaxf(x1, 0.0f);
-                                }
-                                __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
-                                pk[e] = *reinterpret_cast<uint32_t*>(&h2);
-                            }
-                            *reinterpret_cast<uint4*>(my_row + ((g ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                        }
-                    }
-                    ptx::fence_proxy_async_smem();
-                    __syncwarp();
-                    if (lane == 0 && box_ok && col0 < p.N) {
-                        if (kConv)
-                            ptx::tma_store_4d(&tmC, stage_buf, col0, sc1, sc2, sc3);
-                        else
-                            ptx::tma_store_2d(&tmC, stage_buf, col0, sc1);
-                        ptx::tma_store_commit();
-                    }
-                    __syncwarp();
-                }
-            } else
-            for (int c0 = 0; c0 < p.bn; c0 += 32) {
-                uint32_t r[32];
-                const uint32_t taddr =
-                    tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * p.bn + c0);
-                ptx::tmem_ld_32x32b_x32(taddr, r);
-                ptx::tmem_ld_wait();
-                const int col0 = t.n_blk * p.bn + c0;
-                if (valid && col0 < p.N) {
-                if (p.split_k > 1) {
-                    float* dst = p.partial + (static_cast<long long>(t.split) * p.M + grow) * p.N + col0;
-                    if (p.vec_store) {
-#pragma unroll
-                        for (int g = 0; g < 8; ++g) {
-                            if (col0 + g * 4 < p.N) {
-                                float4 v = make_float4(__uint_as_float(r[g * 4]), __uint_as_float(r[g * 4 + 1]),
-                                                       __uint_as_float(r[g * 4 + 2]), __uint_as_float(r[g * 4 + 3]));
-                                *reinterpret_cast<float4*>(dst + g * 4) = v;
-                            }
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (col0 + j < p.N) dst[j] = __uint_as_float(r[j]);
-                    }
-                } else {
-                    float v[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        float x = p.alpha * __uint_as_float(r[j]);
-                        if (p.bias != nullptr && col0 + j < p.N) x += __ldg(p.bias + col0 + j);
-                        if (p.relu) x = fmaxf(x, 0.0f);
-                        v[j] = x;
-                    }
-                    __nv_bfloat16* dst = p.C + grow * p.ldc + col0;
-                    if (p.vec_store) {
-#pragma unroll
-                        for (int g = 0; g < 4; ++g) {
-                            if (col0 + g * 8 < p.N) {
-                                uint4 pk;
-                                __nv_bfloat162 h0 = __floats2bfloat162_rn(v[g * 8 + 0], v[g * 8 + 1]);
-                                __nv_bfloat162 h1 = __floats2bfloat162_rn(v[g * 8 + 2], v[g * 8 + 3]);
-                                __nv_bfloat162 h2 = __floats2bfloat162_rn(v[g * 8 + 4], v[g * 8 + 5]);
-                                __nv_bfloat162 h3 = __floats2bfloat162_rn(v[g * 8 + 6], v[g * 8 + 7]);
-                                pk.x = *reinterpret_cast<uint32_t*>(&h0);
-                                pk.y = *reinterpret_cast<uint32_t*>(&h1);
-                                pk.z = *reinterpret_cast<uint32_t*>(&h2);
-                                pk.w = *reinterpret_cast<uint32_t*>(&h3);
-                                *reinterpret_cast<uint4*>(dst + g * 8) = pk;
-                            }
-                        }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (col0 + j < p.N) dst[j] = __float2bfloat16_rn(v[j]);
-                    }
-                }
-                }
-                __syncwarp();   // reconverge before the next warp-aligned TMEM load
-            }
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&tempty_bar[buf]);
-        }
-        // shared memory must stay alive until the copy engine has drained this warp's last store
-        if (p.tma_store && lane == 0) ptx::tma_store_wait_all<0>();
+        epilogue_role<kConv>(p, &tmC, smem + static_cast<size_t>(p.stages) * stage_bytes, tmem_base, tfull_bar,
+                             tempty_bar, abort_flag, mh, warp, lane, total_items);
     }
 
     ptx::tc_fence_before_sync();

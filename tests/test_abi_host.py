@@ -185,7 +185,7 @@ def test_tuning_cache_round_trip(tmp_path):
     assert st == tdx.TDX_OK and (c.tile_n, c.stages, c.split_k, c.raster) == (64, 3, 2, 2)
     out = tmp_path / "out.json"
     assert tdx.tdx_tune_save(str(out)) == tdx.TDX_OK
-    assert "gemm:640:640:640:0:1:1" in out.read_text() and "[1, 128, 64, 64, 3, 1, 2, 1, 2, 0, 0, 0]" in out.read_text()
+    assert "gemm:640:640:640:0:1:1" in out.read_text() and "[1, 128, 64, 64, 3, 1, 2, 1, 2, 0, 0, 0, 0]" in out.read_text()
     assert tdx.tdx_tune_clear() == tdx.TDX_OK
     st, c = tdx.tdx_default_gemm_config(640, 640, 640, 0, 1, tdx.TDX_BF16)
     assert c.tile_n != 64 or c.split_k != 2

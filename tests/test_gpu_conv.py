@@ -99,6 +99,44 @@ def test_conv_store_modes_agree(patch):
     assert np.array_equal(outs[0], outs[1])
 
 
+HALO_CASES = [
+    # N, H,  W,  Cin, Cout, R, S, pad
+    (2, 16, 8, 64, 64, 3, 3, 1),          # exactly one 8 x 16 patch per image
+    (3, 56, 56, 128, 96, 3, 3, 1),        # 56 = 3.5 patches high: ragged last patch row
+    (1, 20, 36, 72, 40, 3, 3, 1),         # channel tail, ragged both ways
+    (2, 30, 44, 64, 128, 5, 5, 2),        # 5 x 5 window
+    (1, 24, 24, 64, 64, 3, 5, 0),         # no padding, non-square filter
+    (1, 7, 7, 256, 256, 3, 3, 1),         # image smaller than a patch
+    (1, 33, 17, 64, 72, 1, 3, 1),         # single filter row
+]
+
+
+@pytest.mark.parametrize("case", HALO_CASES)
+@pytest.mark.parametrize("tile_m", [128, 256])
+def test_conv_halo_reuse_vs_oracle(case, tile_m):
+    # the input window of a patch is loaded once per channel chunk and every filter tap reads it from shared memory
+    N, H, W, Cin, Cout, R, S, pad = case
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, R, S, seed=80)
+    st, y, ok = run_conv(N, H, W, Cin, Cout, R, S, pad, 1, "bf16", x, w, b, 1, cfg=umma(halo=2, tile_m=tile_m))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    err = conv_error(N, H, W, Cin, Cout, R, S, pad, 1, "bf16", x, w, b, 1, y)
+    assert err < TOL["bf16"] and err < TIGHT["bf16"], err
+
+
+def test_conv_halo_reuse_equals_per_tap_loads_bitwise_for_one_channel_chunk():
+    # with Cin <= 64 both kernels add the taps in the same order
+    N, H, W, Cin, Cout = 2, 40, 24, 64, 64
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=81)
+    _, y1, _ = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, cfg=umma(halo=1, patch_w=8, patch_h=16))
+    st, y2, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, cfg=umma(halo=2, tile_n=64, stages=2))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert np.array_equal(y1, y2)
+    # a 1 x 1 filter has nothing to reuse: the halo kernel is refused, output untouched
+    st, _, untouched = run_conv(N, H, W, Cin, Cout, 1, 1, 0, 1, "bf16", x, si.normal(82, 1, (Cout, 1, 1, Cin), "bf16"), b, 1,
+                                cfg=umma(halo=2))
+    assert st == tdx.TDX_ERR_CONFIG and untouched
+
+
 def test_conv_staggered_k_order():
     N, H, W, Cin, Cout = 8, 28, 28, 192, 128
     x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=78)
