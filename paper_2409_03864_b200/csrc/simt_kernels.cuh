@@ -81,6 +81,161 @@ sgemm_tiled_kernel(int M, int N, int K, long long sa_i, long long sa_k, long lon
 }
 
 // ---------------------------------------------------------------------------
+// fp32 GEMM for small problems: 32 x 32 tiles, 2 x 2 outputs per thread, and a 4-stage cp.async ring so
+// that the global-load latency of K-tile t+3 hides behind the FMAs of tile t (a small problem has too few
+// CTAs per SM to hide it any other way).  Same index maps and the same k-ascending fp32 FMA order as
+// sgemm_tiled_kernel.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void cp_async_f32(float* smem_dst, const float* gmem_src, bool valid) {
+    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+    const int src_bytes = valid ? 4 : 0;   // 0 source bytes: the destination is zero-filled
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(gmem_src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+__global__ void __launch_bounds__(256)
+sgemm_small_kernel(int M, int N, int K, long long sa_i, long long sa_k, long long sb_k, long long sb_j, float alpha,
+                   const float* __restrict__ A, const float* __restrict__ B, float* __restrict__ C) {
+    constexpr int BM = 32, BN = 32, BK = 32, ST = 4, LD = BM + 2;
+    __shared__ __align__(16) float As[ST][BK][LD];
+    __shared__ __align__(16) float Bs[ST][BK][LD];
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;          // 16 x 16 threads, 2 x 2 outputs each
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int ktiles = (K + BK - 1) / BK;
+
+    auto load_tile = [&](int kt, int st) {
+        const int k0 = kt * BK;
+#pragma unroll
+        for (int e = 0; e < (BM * BK) / 256; ++e) {
+            const int idx = tid + e * 256;
+            int i, k;
+            if (sa_k == 1) { i = idx / BK; k = idx % BK; } else { i = idx % BM; k = idx / BM; }
+            const int gi = m0 + i, gk = k0 + k;
+            const bool ok = gi < M && gk < K;
+            cp_async_f32(&As[st][k][i], A + (ok ? gi * sa_i + gk * sa_k : 0), ok);
+        }
+#pragma unroll
+        for (int e = 0; e < (BN * BK) / 256; ++e) {
+            const int idx = tid + e * 256;
+            int j, k;
+            if (sb_j == 1) { k = idx / BN; j = idx % BN; } else { j = idx / BK; k = idx % BK; }
+            const int gj = n0 + j, gk = k0 + k;
+            const bool ok = gj < N && gk < K;
+            cp_async_f32(&Bs[st][k][j], B + (ok ? gk * sb_k + gj * sb_j : 0), ok);
+        }
+    };
+
+    for (int s = 0; s < ST - 1; ++s) {
+        if (s < ktiles) load_tile(s, s);
+        cp_async_commit();
+    }
+    float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+    for (int kt = 0; kt < ktiles; ++kt) {
+        cp_async_wait<ST - 2>();
+        __syncthreads();                               // tile kt has landed; everyone is done with tile kt-1
+        if (kt + ST - 1 < ktiles) load_tile(kt + ST - 1, (kt + ST - 1) % ST);
+        cp_async_commit();
+        const int st = kt % ST;
+#pragma unroll
+        for (int k = 0; k < BK; ++k) {
+            const float2 a = *reinterpret_cast<const float2*>(&As[st][k][ty * 2]);
+            const float2 b = *reinterpret_cast<const float2*>(&Bs[st][k][tx * 2]);
+            acc[0][0] = fmaf(a.x, b.x, acc[0][0]);
+            acc[0][1] = fmaf(a.x, b.y, acc[0][1]);
+            acc[1][0] = fmaf(a.y, b.x, acc[1][0]);
+            acc[1][1] = fmaf(a.y, b.y, acc[1][1]);
+        }
+    }
+    cp_async_wait<0>();
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int gi = m0 + ty * 2 + i;
+        if (gi >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int gj = n0 + tx * 2 + j;
+            if (gj < N) C[static_cast<long long>(gi) * N + gj] = alpha * acc[i][j];
+        }
+    }
+}
+
+// Same tiling for the plain row-major case (A is M x K, B is K x N, K and N multiples of 4, 16-byte aligned
+// bases): both operands move with 16-byte cp.async, A stays k-contiguous in shared memory.
+__device__ __forceinline__ void cp_async_16(float* smem_dst, const float* gmem_src, bool valid) {
+    const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+    const int src_bytes = valid ? 16 : 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(gmem_src), "r"(src_bytes) : "memory");
+}
+
+__global__ void __launch_bounds__(256)
+sgemm_small_rowmajor_kernel(int M, int N, int K, float alpha, const float* __restrict__ A, const float* __restrict__ B,
+                            float* __restrict__ C) {
+    constexpr int BM = 32, BN = 32, BK = 32, ST = 4, LDA = BK + 4, LDB = BN + 4;
+    __shared__ __align__(16) float As[ST][BM][LDA];   // [m][k]
+    __shared__ __align__(16) float Bs[ST][BK][LDB];   // [k][n]
+    const int tid = threadIdx.x;
+    const int tx = tid & 15, ty = tid >> 4;
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int ktiles = (K + BK - 1) / BK;
+    const int lr = tid >> 3, lc = (tid & 7) * 4;     // 32 rows x 8 groups of 4 floats: one 16-byte copy per thread and operand
+
+    auto load_tile = [&](int kt, int st) {
+        const int k0 = kt * BK;
+        {
+            const int gi = m0 + lr, gk = k0 + lc;
+            const bool ok = gi < M && gk < K;            // K % 4 == 0: a group is all in or all out
+            cp_async_16(&As[st][lr][lc], A + (ok ? static_cast<long long>(gi) * K + gk : 0), ok);
+        }
+        {
+            const int gk = k0 + lr, gj = n0 + lc;
+            const bool ok = gk < K && gj < N;
+            cp_async_16(&Bs[st][lr][lc], B + (ok ? static_cast<long long>(gk) * N + gj : 0), ok);
+        }
+    };
+
+    for (int s = 0; s < ST - 1; ++s) {
+        if (s < ktiles) load_tile(s, s);
+        cp_async_commit();
+    }
+    float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+    for (int kt = 0; kt < ktiles; ++kt) {
+        cp_async_wait<ST - 2>();
+        __syncthreads();
+        if (kt + ST - 1 < ktiles) load_tile(kt + ST - 1, (kt + ST - 1) % ST);
+        cp_async_commit();
+        const int st = kt % ST;
+#pragma unroll
+        for (int k4 = 0; k4 < BK; k4 += 4) {
+            const float4 a0 = *reinterpret_cast<const float4*>(&As[st][ty * 2][k4]);
+            const float4 a1 = *reinterpret_cast<const float4*>(&As[st][ty * 2 + 1][k4]);
+            const float av0[4] = {a0.x, a0.y, a0.z, a0.w}, av1[4] = {a1.x, a1.y, a1.z, a1.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float2 b = *reinterpret_cast<const float2*>(&Bs[st][k4 + k][tx * 2]);
+                acc[0][0] = fmaf(av0[k], b.x, acc[0][0]);
+                acc[0][1] = fmaf(av0[k], b.y, acc[0][1]);
+                acc[1][0] = fmaf(av1[k], b.x, acc[1][0]);
+                acc[1][1] = fmaf(av1[k], b.y, acc[1][1]);
+            }
+        }
+    }
+    cp_async_wait<0>();
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+        const int gi = m0 + ty * 2 + i;
+        if (gi >= M) continue;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int gj = n0 + tx * 2 + j;
+            if (gj < N) C[static_cast<long long>(gi) * N + gj] = alpha * acc[i][j];
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
 // Generic GEMM, one thread per output element (no layout or alignment constraints).
 // ---------------------------------------------------------------------------
 template <typename TIn, typename TOut>

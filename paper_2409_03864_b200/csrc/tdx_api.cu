@@ -595,8 +595,12 @@ int run_gemm_simt_f32(DeviceCtx* ctx, const GemmProblem& g, float alpha, const v
                                                                        sb_j, alpha, a, b, c);
     } else {
         dim3 grid(static_cast<unsigned>(ceil_div(g.N, 32)), static_cast<unsigned>(ceil_div(g.M, 32)));
-        tdx::sgemm_tiled_kernel<32, 32, 16, 2, 2><<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k,
-                                                                       sb_j, alpha, a, b, c);
+        const bool rowmajor16 = !g.transA && !g.transB && g.K % 4 == 0 && g.N % 4 == 0 &&
+                                reinterpret_cast<uintptr_t>(A) % 16 == 0 && reinterpret_cast<uintptr_t>(B) % 16 == 0;
+        if (rowmajor16)
+            tdx::sgemm_small_rowmajor_kernel<<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, alpha, a, b, c);
+        else
+            tdx::sgemm_small_kernel<<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k, sb_j, alpha, a, b, c);
     }
     TDX_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);

@@ -28,7 +28,7 @@ def test_fp32_gemm_256_cubed_uniform():
 
 
 @pytest.mark.parametrize("transA,transB", [(0, 0), (0, 1), (1, 0), (1, 1)])
-@pytest.mark.parametrize("shape", [(1, 1, 1), (33, 65, 17), (130, 70, 257), (64, 64, 64), (300, 500, 40)])
+@pytest.mark.parametrize("shape", [(1, 1, 1), (33, 65, 17), (130, 70, 257), (64, 64, 64), (300, 500, 40), (100, 76, 204)])
 def test_fp32_gemm_shapes_and_transposes(shape, transA, transB):
     M, N, K = shape
     A = si.uniform(10, 0, (K, M) if transA else (M, K), "f32")
