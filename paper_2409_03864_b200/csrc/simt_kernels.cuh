@@ -295,6 +295,9 @@ __global__ void conv2d_generic_kernel(int Nimg, int H, int W, int Cin, int Cout,
 __global__ void splitk_reduce_kernel(long long MN, int N, int split, const float* __restrict__ partial, float alpha,
                                      const float* __restrict__ bias, int relu, __nv_bfloat16* __restrict__ out,
                                      int vec8) {
+    // launched with programmatic stream serialization: this grid may start while the GEMM drains; wait here
+    // until the GEMM grid has completed and its partial sums are visible (a no-op for an ordinary launch)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (vec8) {
         const long long groups = MN / 8;
         for (long long g = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; g < groups;

@@ -387,6 +387,28 @@ int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensor
     return TDX_OK;
 }
 
+// The reduction is launched with programmatic stream serialization so that its launch latency hides behind
+// the tail of the GEMM kernel; it waits on the device for the GEMM grid to complete before reading partials.
+int launch_splitk_reduce(int grid, cudaStream_t st, long long MN, int N, int split, const float* partial, float alpha,
+                         __nv_bfloat16* out, int vec8) {
+    cudaLaunchConfig_t lc;
+    std::memset(&lc, 0, sizeof lc);
+    lc.gridDim = dim3(static_cast<unsigned>(grid));
+    lc.blockDim = dim3(256);
+    lc.dynamicSmemBytes = 0;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    const float* bias = nullptr;
+    int relu = 0;
+    TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::splitk_reduce_kernel, MN, N, split, partial, alpha, bias, relu, out, vec8));
+    g_launches.fetch_add(1);
+    return TDX_OK;
+}
+
 int ensure_ws(DeviceCtx* ctx, size_t bytes, void** out) {
     if (ctx->ws_bytes < bytes) {
         if (ctx->ws) TDX_CUDA(cudaFree(ctx->ws));
@@ -482,10 +504,8 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         const int vec8 = p.vec_store ? 1 : 0;
         const long long work = vec8 ? MN / 8 : MN;
         const int grid = static_cast<int>(std::min<long long>(ceil_div(work, 256), 148LL * 16));
-        tdx::splitk_reduce_kernel<<<std::max(grid, 1), 256, 0, st>>>(MN, static_cast<int>(g.N), cfg.split_k, p.partial,
-                                                                     alpha, nullptr, 0, p.C, vec8);
-        TDX_CUDA(cudaGetLastError());
-        g_launches.fetch_add(1);
+        rc = launch_splitk_reduce(std::max(grid, 1), st, MN, static_cast<int>(g.N), cfg.split_k, p.partial, alpha, p.C, vec8);
+        if (rc) return rc;
     }
     return TDX_OK;
 }
@@ -746,7 +766,19 @@ int resolve_conv_config(const ConvProblem& cp, const tdx_config* user, int sm_co
     if (c.kernel == TDX_KERNEL_GENERIC) { *out = c; return TDX_OK; }
     if (cp.dtype != TDX_BF16) return fail(TDX_ERR_CONFIG, "the tensor-core kernel is bf16 only");
     if (!layout_ok) return fail(TDX_ERR_ALIGNMENT, "tensor-core conv needs stride 1 and Cin %% 8 == 0");
-    if (c.halo == 0) c.halo = 1;
+    const bool halo_auto = c.halo == 0 && !from_cache;
+    if (c.halo == 0) {
+        // halo reuse unless its fixed 8 x 16 patches waste much more of the image than the best free patch shape
+        c.halo = 1;
+        if (cp.R * cp.S > 1 && c.patch_w == 0 && c.patch_h == 0) {
+            int bw, bh;
+            choose_patch(cp.P, cp.Q, &bw, &bh);
+            const int64_t best = ceil_div(cp.Q, bw) * bw * ceil_div(cp.P, bh) * bh;
+            const int64_t mine = ceil_div(cp.Q, kHaloPatchW) * kHaloPatchW * ceil_div(cp.P, kHaloPatchH) * kHaloPatchH;
+            const int tm = c.tile_m ? c.tile_m : 128, tn = c.tile_n ? c.tile_n : 64;
+            if (mine * 100 <= best * 120 && halo_max_stages(tm, tn, cp.R, cp.S, smem_limit, 2) >= 2) c.halo = 2;
+        }
+    }
     if (c.halo == 2 && c.patch_w == 0 && c.patch_h == 0) { c.patch_w = kHaloPatchW; c.patch_h = kHaloPatchH; }
     if (c.patch_w == 0 && c.patch_h == 0) choose_patch(cp.P, cp.Q, &c.patch_w, &c.patch_h);
     if (!patch_ok(c.patch_w, c.patch_h)) return fail(TDX_ERR_CONFIG, "infeasible config: patch %dx%d", c.patch_w, c.patch_h);
@@ -769,6 +801,14 @@ int resolve_conv_config(const ConvProblem& cp, const tdx_config* user, int sm_co
                                : std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode));
     if (!user && !from_cache) c.raster = d.raster;
     const char* why = umma_config_reason(c, false, num_kb, smem_limit, true, cp.Cout, cp.R, cp.S);
+    if (why && halo_auto && c.halo == 2) {
+        // the automatic choice of halo reuse did not fit (large filter): fall back to per-tap loads
+        tdx_config retry;
+        std::memset(&retry, 0, sizeof retry);
+        if (user) retry = *user;
+        retry.halo = 1;
+        return resolve_conv_config(cp, &retry, sm_count, smem_limit, out);
+    }
     if (why) return fail(TDX_ERR_CONFIG, "infeasible config: %s", why);
     *out = c;
     return TDX_OK;
