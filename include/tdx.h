@@ -66,7 +66,9 @@ typedef struct {
     int tile_n;     /* 32, 64, 96, ..., 256 (multiple of 32; multiple of 64 when transB = 0)    */
     int tile_k;     /* 64                                                                      */
     int stages;     /* depth of the TMA/mbarrier ring, 2..8, bounded by shared memory          */
-    int cta_pair;   /* 1 (one CTA per tile)                                                    */
+    int cta_pair;   /* 1 = one CTA per tile; 2 = a cluster of two CTAs per 256-row tile (GEMM only): each  */
+                    /*     CTA stages its 128 rows of A and half of the B slice, one thread issues MMAs    */
+                    /*     over both, and each CTA keeps a 128 x tile_n accumulator half                  */
     int split_k;    /* >= 1; > 1 needs a workspace and runs a fixed-order reduction afterwards  */
     int store_mode; /* 1 = 16-byte stores from registers; 2 = 32 x 32 blocks staged in shared     */
                     /*     memory and written by TMA store (needs N % 8 == 0, split_k = 1,         */

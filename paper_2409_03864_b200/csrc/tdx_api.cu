@@ -18,6 +18,7 @@
 #include "simt_kernels.cuh"
 #include "umma_conv_halo.cuh"
 #include "umma_kernel.cuh"
+#include "umma_pair.cuh"
 
 namespace {
 
@@ -108,6 +109,9 @@ int get_ctx(DeviceCtx** out) {
                              c.smem_optin - kStaticSmemReserve);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(tdx::umma_contract_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 c.smem_optin - kStaticSmemReserve);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tdx::umma_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  c.smem_optin - kStaticSmemReserve);
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(tdx::umma_conv_halo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -259,6 +263,13 @@ int halo_max_stages(int tile_m, int tile_n, int64_t R, int64_t S, int smem_limit
     return left <= 0 ? 0 : std::min(left / (tile_n * 128), tdx::kMaxStages);
 }
 
+// CTA pair (256 x tile_n per pair): each CTA stages its 128 rows of A and tile_n / 2 columns of B
+int pair_max_stages(int tile_n, int smem_limit, int store_mode) {
+    const int stage = (128 + tile_n / 2) * 128;
+    const int s = (smem_limit - kStaticSmemReserve - 1024 - staging_bytes_for(128, store_mode)) / stage;
+    return std::min(s, tdx::kMaxStages);
+}
+
 int tmem_slots_for(int tile_m, int bn) { return (tile_m == 256 && bn <= 128) ? 4 : 2; }
 int tmem_cols_for(int tile_m, int bn) {
     int c = 32;
@@ -272,7 +283,14 @@ const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num
                                int64_t N, int64_t R = 1, int64_t S = 1) {
     if (c.tile_m != 128 && c.tile_m != 256) return "tile_m must be 128 or 256";
     if (c.tile_k != 64) return "tile_k must be 64";
-    if (c.cta_pair != 1) return "cta_pair must be 1";
+    if (c.cta_pair != 1 && c.cta_pair != 2) return "cta_pair must be 1 or 2";
+    if (c.cta_pair == 2) {
+        if (conv) return "CTA pairs are implemented for the GEMM only";
+        if (c.tile_m != 256) return "a CTA pair works on 256-row tiles";
+        if (c.split_k != 1) return "CTA pairs have no split-K";
+        if (b_mn_major && c.tile_n % 128) return "tile_n must be a multiple of 128 for a CTA pair when B is read N-major";
+        if (c.k_stagger) return "CTA pairs have no k_stagger";
+    }
     if (c.store_mode != 1 && c.store_mode != 2) return "store_mode must be 1 (direct) or 2 (TMA store)";
     if (c.store_mode == 2) {
         if (N % 8) return "the TMA-store epilogue needs an output row pitch that is a multiple of 16 bytes";
@@ -289,6 +307,8 @@ const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num
         if (kHaloPatchW + S - 1 > 256 || kHaloPatchH + R - 1 > 256) return "filter too large for a halo tile";
         if (c.stages < 2 || c.stages > halo_max_stages(c.tile_m, c.tile_n, R, S, smem_limit, c.store_mode))
             return "stages outside the shared-memory budget";
+    } else if (c.cta_pair == 2) {
+        if (c.stages < 2 || c.stages > pair_max_stages(c.tile_n, smem_limit, c.store_mode)) return "stages outside the shared-memory budget";
     } else
     if (c.stages < 2 || c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode)) return "stages outside the shared-memory budget";
     if (c.split_k < 1) return "split_k must be >= 1";
@@ -507,6 +527,90 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         rc = launch_splitk_reduce(std::max(grid, 1), st, MN, static_cast<int>(g.N), cfg.split_k, p.partial, alpha, p.C, vec8);
         if (rc) return rc;
     }
+    return TDX_OK;
+}
+
+// GEMM on CTA pairs: 256 x tile_n per pair, each CTA loads its 128 rows of A and tile_n / 2 columns of B.
+int run_gemm_pair(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
+                  const tdx_config& cfg, cudaStream_t st) {
+    const int64_t num_kb = ceil_div(g.K, 64);
+    UmmaParams p;
+    std::memset(&p, 0, sizeof p);
+    p.M = static_cast<int>(g.M);
+    p.N = static_cast<int>(g.N);
+    p.num_kb = static_cast<int>(num_kb);
+    p.bm = 128;                                      // what one CTA of the pair owns (epilogue geometry)
+    p.slots = 2 * cfg.tile_n <= 256 ? 4 : 2;
+    p.tiles_m = static_cast<int>(ceil_div(g.M, 256));
+    p.tiles_n = static_cast<int>(ceil_div(g.N, cfg.tile_n));
+    p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
+    p.split_k = 1;
+    p.kb_per_split = p.num_kb;
+    p.bn = cfg.tile_n;
+    p.stages = cfg.stages;
+    p.tmem_cols = 32;
+    while (p.tmem_cols < p.slots * cfg.tile_n) p.tmem_cols *= 2;
+    p.a_mn_major = g.transA ? 1 : 0;
+    p.b_mn_major = g.transB ? 0 : 1;
+    p.alpha = alpha;
+    p.C = static_cast<__nv_bfloat16*>(C);
+    p.ldc = g.N;
+    p.status = ctx->status_ptr;
+    p.vec_store = (g.N % 8 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+    p.tma_store = (cfg.store_mode == 2 && p.vec_store) ? 1 : 0;
+
+    CUtensorMap ma, mb, mc;
+    int rc;
+    if (p.a_mn_major) {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.M), static_cast<uint64_t>(g.K)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.M) * 2};
+        uint32_t box[2] = {64, 64};
+        rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
+    } else {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.M)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
+        uint32_t box[2] = {64, 128};
+        rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
+    }
+    if (rc) return rc;
+    if (p.b_mn_major) {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.K)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
+        uint32_t box[2] = {64, 64};
+        rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
+    } else {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.N)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
+        uint32_t box[2] = {64, static_cast<uint32_t>(cfg.tile_n / 2)};
+        rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
+    }
+    if (rc) return rc;
+    mc = ma;
+    if (p.tma_store) {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.M)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
+        uint32_t box[2] = {32, 32};
+        rc = get_tensor_map(ctx, C, 2, dims, str, box, &mc, 64);
+        if (rc) return rc;
+    }
+    const long long pair_tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
+    const int pairs = static_cast<int>(std::min<long long>(pair_tiles, ctx->sm_count / 2));
+    cudaLaunchConfig_t lc;
+    std::memset(&lc, 0, sizeof lc);
+    lc.gridDim = dim3(static_cast<unsigned>(2 * pairs));
+    lc.blockDim = dim3(p.tma_store ? 576 : 192);
+    lc.dynamicSmemBytes = static_cast<size_t>(p.stages) * ((128 + p.bn / 2) * 128) + 1024 +
+                          staging_bytes_for(128, p.tma_store ? 2 : 1);
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_pair_kernel, ma, mb, mc, p));
+    g_launches.fetch_add(1);
     return TDX_OK;
 }
 
@@ -731,16 +835,18 @@ int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_cou
     const bool b_mn = g.transB == 0;
     tdx_config d;
     default_umma_config(ceil_div(g.M, 128), g.N, num_kb, b_mn, sm_count, smem_limit, true, &d);
-    if (c.tile_m == 0) c.tile_m = (c.tile_n == 0 || c.tile_n == d.tile_n) ? d.tile_m : 128;
+    if (c.tile_m == 0) c.tile_m = c.cta_pair == 2 ? 256 : ((c.tile_n == 0 || c.tile_n == d.tile_n) ? d.tile_m : 128);
     if (c.tile_k == 0) c.tile_k = d.tile_k;
     if (c.cta_pair == 0) c.cta_pair = d.cta_pair;
     if (c.tile_n == 0) c.tile_n = d.tile_n;
-    if (c.split_k == 0) c.split_k = (user && user->tile_n != 0 && user->tile_n != d.tile_n) ? 1 : d.split_k;
+    if (c.split_k == 0) c.split_k = (user && user->cta_pair == 2) ? 1 : (user && user->tile_n != 0 && user->tile_n != d.tile_n) ? 1 : d.split_k;
     if (c.store_mode == 0) {
         c.store_mode = (c.split_k == 1 && g.N % 8 == 0) ? 2 : 1;
-        if (c.store_mode == 2 && c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, 2)) c.store_mode = 1;
+        if (c.store_mode == 2 && c.cta_pair != 2 && c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, 2)) c.store_mode = 1;
     }
-    if (c.stages == 0) c.stages = std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode));
+    if (c.stages == 0)
+        c.stages = c.cta_pair == 2 ? std::max(2, pair_max_stages(c.tile_n, smem_limit, c.store_mode))
+                                   : std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode));
     if (!user && !from_cache) c.raster = d.raster;
     const char* why = umma_config_reason(c, b_mn, num_kb, smem_limit, false, g.N);
     if (why) return fail(TDX_ERR_CONFIG, "infeasible config: %s", why);
@@ -865,6 +971,7 @@ int gemm_dispatch(int64_t M, int64_t N, int64_t K, int transA, int transB, float
                     return fail(TDX_ERR_ALIGNMENT, "tensor-core path needs 16-byte aligned A and B");
                 return run_gemm_generic(ctx, g, alpha, A, B, C, st);
             }
+            if (c.cta_pair == 2) return run_gemm_pair(ctx, g, alpha, A, B, C, c, st);
             return run_gemm_umma(ctx, g, alpha, A, B, C, c, ws, ws_bytes, internal_ws, st);
     }
 }
@@ -965,6 +1072,26 @@ int enum_gemm(const GemmProblem& g, int sm_count, int smem_limit, std::vector<td
         return TDX_OK;
     }
     enum_umma_space(g.transB == 0, ceil_div(g.M, 128), g.N, ceil_div(g.K, 64), sm_count, smem_limit, false, 0, 0, v);
+    // CTA-pair candidates: 256 x tile_n per pair
+    const bool b_mn = g.transB == 0;
+    const int64_t pair_tiles_m = ceil_div(g.M, 256);
+    for (int bn : {256, 192, 128}) {
+        if (b_mn && bn % 128) continue;
+        if (bn - 64 >= g.N) continue;
+        if (pair_tiles_m * ceil_div(g.N, bn) < sm_count / 4) continue;
+        const int sm = g.N % 8 == 0 ? 2 : 1;
+        const int max_st = pair_max_stages(bn, smem_limit, sm);
+        for (int stg : {max_st, max_st - 2})
+            for (int raster : {0, 8, 2, 4, 16}) {
+                if (stg < 2 || (raster != 0 && pair_tiles_m <= raster)) continue;
+                tdx_config c;
+                std::memset(&c, 0, sizeof c);
+                c.kernel = TDX_KERNEL_UMMA;
+                c.tile_m = 256; c.tile_n = bn; c.tile_k = 64; c.stages = stg; c.cta_pair = 2; c.split_k = 1;
+                c.store_mode = sm; c.raster = raster;
+                if (umma_config_reason(c, b_mn, ceil_div(g.K, 64), smem_limit, false, g.N) == nullptr) v->push_back(c);
+            }
+    }
     return TDX_OK;
 }
 

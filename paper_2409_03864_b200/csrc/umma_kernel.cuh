@@ -115,7 +115,15 @@ __device__ __forceinline__ TileCoord decode_item(const UmmaParams& p, int item) 
 template <bool kConv>
 __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtensorMap* tmC, uint8_t* staging_base,
                                               uint32_t tmem_base, uint64_t* tfull_bar, uint64_t* tempty_bar,
-                                              volatile int* abort_flag, int mh, int warp, int lane, int total_items) {
+                                              volatile int* abort_flag, int mh, int warp, int lane, int total_items,
+                                              int first_item = -1, int item_stride = 0, int m_mul = 1, int m_add = 0,
+                                              uint32_t tempty_cluster_addr = 0) {
+    // CTA pairs: the pair walks tiles of 256 rows, this CTA owns rows [128 * (2 m + rank), +128) of tile m, and the
+    // accumulator-free signal goes to the leader CTA's barrier (tempty_cluster_addr, a shared::cluster address)
+    if (first_item < 0) {
+        first_item = blockIdx.x;
+        item_stride = gridDim.x;
+    }
     const int ew = warp - 2;
     const int nwarps_epi = (static_cast<int>(blockDim.x) >> 5) - 2;
     const int ncgrp = nwarps_epi / (4 * mh);      // warps sharing one (half, quarter)
@@ -124,8 +132,9 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
     const int row_in_tile = half * kHalfM + quarter * 32 + lane;
     int local = 0;
-    for (int item = blockIdx.x; item < total_items; item += gridDim.x, ++local) {
-        const TileCoord t = decode_item(p, item);
+    for (int item = first_item; item < total_items; item += item_stride, ++local) {
+        TileCoord t = decode_item(p, item);
+        t.m_blk = t.m_blk * m_mul + m_add;
         const int sidx = local * mh + half;
         const int buf = sidx % p.slots;
         const uint32_t aphase = (sidx / p.slots) & 1;
@@ -304,7 +313,12 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
         }
         ptx::tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&tempty_bar[buf]);
+        if (lane == 0) {
+            if (tempty_cluster_addr != 0)
+                ptx::mbar_arrive_cluster(tempty_cluster_addr + static_cast<uint32_t>(buf) * 8u);
+            else
+                ptx::mbar_arrive(&tempty_bar[buf]);
+        }
     }
     // shared memory must stay alive until the copy engine has drained this warp's last store
     if (p.tma_store && lane == 0) ptx::tma_store_wait_all<0>();

@@ -135,10 +135,14 @@ def test_gemm_search_space_obeys_constraints(shape):
         assert 2 <= c["stages"] <= 8
         assert c["store_mode"] in (1, 2)
         staging = 16 * 2048 if c["store_mode"] == 2 else 0
-        assert c["stages"] * (c["tile_m"] + c["tile_n"]) * 128 + 1024 + 512 + staging <= SMEM_LIMIT
+        rows_per_cta = 128 + c["tile_n"] // 2 if c["cta_pair"] == 2 else c["tile_m"] + c["tile_n"]
+        assert c["stages"] * rows_per_cta * 128 + 1024 + 512 + staging <= SMEM_LIMIT
+        if c["cta_pair"] == 2:
+            assert c["tile_m"] == 256 and c["split_k"] == 1 and c["tile_n"] % 128 == 0
         if c["store_mode"] == 2:
             assert c["split_k"] == 1
-        assert (c["tile_m"] // 128) * c["tile_n"] <= 512      # one tile's accumulators fit in TMEM
+        halves = 1 if c["cta_pair"] == 2 else c["tile_m"] // 128
+        assert halves * c["tile_n"] <= 512                     # one tile's accumulators fit in a CTA's TMEM
         per = -(-num_kb // c["split_k"])
         assert (c["split_k"] - 1) * per < num_kb               # no empty K slice
     if M * N <= 128 * 8192:

@@ -136,6 +136,33 @@ def test_umma_store_modes(cfgkw, store_mode):
         assert np.array_equal(C, C1)                             # same arithmetic, different way out
 
 
+@pytest.mark.parametrize("transA,transB", [(0, 1), (0, 0), (1, 1), (1, 0)])
+@pytest.mark.parametrize("cfgkw", [dict(tile_n=256), dict(tile_n=128, stages=3), dict(tile_n=256, store_mode=1, raster=2)])
+def test_umma_cta_pairs(cfgkw, transA, transB):
+    # a cluster of two CTAs per 256-row tile: each stages half of the operands, one thread issues MMAs over both
+    M, N, K = 1416, 1160, 392          # ragged last tile in M, N and K; more tiles than CTA pairs along the way
+    A, B = si.gemm_bf16_normal(M, N, K, seed=69, transA=transA, transB=transB)
+    st, C, ok = run_gemm(M, N, K, transA, transB, -1.0, "bf16", A, B, cfg=umma(cta_pair=2, **cfgkw))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert gemm_error(M, N, K, transA, transB, -1.0, "bf16", A, B, C) < TIGHT["bf16"]
+    assert tdx.tdx_check_device_status() == 0
+
+
+def test_umma_cta_pairs_many_tiles_exact_and_deterministic():
+    M, N, K = 256 * 40, 256 * 5, 192       # 200 pair tiles over 74 pairs: accumulator slots wrap around
+    A = si.small_integers(70, 0, (M, K), "bf16", -1, 1)
+    B = si.small_integers(70, 1, (N, K), "bf16", -1, 1)
+    st, C, ok = run_gemm(M, N, K, 0, 1, 1.0, "bf16", A, B, cfg=umma(cta_pair=2, tile_n=256))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    rows = structured_rows(M, extra=2, max_blocks=20)
+    assert np.array_equal(oracle.decode(C, "bf16")[rows], oracle.gemm(M, N, K, 0, 1, 1.0, "bf16", A, B, rows=rows))
+    st, C2, _ = run_gemm(M, N, K, 0, 1, 1.0, "bf16", A, B, cfg=umma(cta_pair=2, tile_n=256))
+    assert np.array_equal(C, C2)
+    # a pair needs 256-row tiles and has no split-K: refused, output untouched
+    st, _, untouched = run_gemm(M, N, K, 0, 1, 1.0, "bf16", A, B, cfg=umma(cta_pair=2, tile_m=128))
+    assert st == tdx.TDX_ERR_CONFIG and untouched
+
+
 @pytest.mark.parametrize("cfgkw", [dict(tile_m=128, tile_n=64, stages=3), dict(tile_m=256, tile_n=128, stages=2)])
 def test_umma_staggered_k_order(cfgkw):
     # each CTA starts its K loop at a different block: same products, rotated order
