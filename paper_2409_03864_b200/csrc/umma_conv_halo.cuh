@@ -145,6 +145,13 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         if (lane == 0) {
             const uint32_t idesc = ptx::make_idesc_bf16_f32(kHalfM, p.bn, 0, 0);
             const uint32_t a_sbo = static_cast<uint32_t>(p.hpitch) * 128u;     // one window row between 8-row groups
+            // descriptors are built once and advanced by additions (16-byte units): the issuing thread has only
+            // a few dozen cycles per MMA when the tile is narrow
+            const uint64_t halo_desc0 = ptx::make_smem_desc_sw128(ptx::smem_u32(a_ring), 16u, a_sbo);
+            const uint64_t b_desc0 = ptx::make_smem_desc_sw128(ptx::smem_u32(b_ring), 16u, 1024u);
+            const uint64_t a_stage_step = a_stage_bytes >> 4, b_stage_step = b_bytes >> 4;
+            const uint64_t half_step = static_cast<uint64_t>(p.halo_bytes) >> 4;
+            uint64_t halo_desc = halo_desc0, b_desc = b_desc0;
             int a_buf = 0, b_stage = 0, local = 0;
             uint32_t a_phase = 0, b_phase = 0;
             bool ok = true;
@@ -165,32 +172,29 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 ptx::tc_fence_after_sync();
                 for (int cc = 0; ok && cc < p.cchunks; ++cc) {
                     if (!wait_bounded(&afull_bar[a_buf], a_phase, abort_flag, p.status, kTimeoutMma)) { ok = false; break; }
-                    const uint32_t halo_addr = ptx::smem_u32(a_ring + static_cast<size_t>(a_buf) * a_stage_bytes);
+                    int r = 0, s = 0;                         // filter tap (r, s), advanced without divisions
+                    uint64_t row_desc = halo_desc;            // window row r, column 0 (one pixel = 128 B = 8 units)
                     for (int tap = 0; tap < taps; ++tap) {
                         if (!wait_bounded(&bfull_bar[b_stage], b_phase, abort_flag, p.status, kTimeoutMma)) { ok = false; break; }
                         ptx::tc_fence_after_sync();
-                        const int r = tap / p.S;
-                        const int s = tap - r * p.S;
-                        const uint32_t a_off = static_cast<uint32_t>(r * p.hpitch + s) * 128u;
-                        const uint32_t b_addr = ptx::smem_u32(b_ring + static_cast<size_t>(b_stage) * b_bytes);
+                        const uint64_t a_tap = row_desc + static_cast<uint64_t>(s) * 8u;
+                        const uint32_t first = (cc > 0 || tap > 0) ? 1u : 0u;
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
                             if (h < mh) {
 #pragma unroll
-                                for (int j = 0; j < kBK / kUmmaK; ++j) {
-                                    const uint64_t adesc = ptx::make_smem_desc_sw128(
-                                        halo_addr + h * p.halo_bytes + a_off + j * 32u, 16u, a_sbo);
-                                    const uint64_t bdesc = ptx::make_smem_desc_sw128(b_addr + j * 32u, 16u, 1024u);
-                                    ptx::umma_bf16(d_tmem[h], adesc, bdesc, idesc, (cc > 0 || tap > 0 || j > 0) ? 1u : 0u);
-                                }
+                                for (int j = 0; j < kBK / kUmmaK; ++j)
+                                    ptx::umma_bf16(d_tmem[h], a_tap + (h ? half_step : 0) + 2 * j, b_desc + 2 * j, idesc,
+                                                   j > 0 ? 1u : first);
                             }
                         }
                         ptx::umma_commit(&bempty_bar[b_stage]);
-                        if (++b_stage == p.stages) { b_stage = 0; b_phase ^= 1u; }
+                        if (++b_stage == p.stages) { b_stage = 0; b_phase ^= 1u; b_desc = b_desc0; } else { b_desc += b_stage_step; }
+                        if (++s == p.S) { s = 0; ++r; row_desc += static_cast<uint64_t>(p.hpitch) * 8u; }
                     }
                     if (!ok) break;
                     ptx::umma_commit(&aempty_bar[a_buf]);
-                    if (++a_buf == p.a_stages) { a_buf = 0; a_phase ^= 1u; }
+                    if (++a_buf == p.a_stages) { a_buf = 0; a_phase ^= 1u; halo_desc = halo_desc0; } else { halo_desc += a_stage_step; }
                 }
                 if (ok) {
                     ptx::umma_commit(&tfull_bar[slot[0]]);

@@ -447,6 +447,13 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             const uint32_t b_lbo = p.b_mn_major ? 8192u : 16u;
             const uint32_t a_kstep = p.a_mn_major ? 2048u : 32u;
             const uint32_t b_kstep = p.b_mn_major ? 2048u : 32u;
+            // The issuing thread must spend far fewer cycles per MMA than the MMA takes (128 at N = 256, 32 at
+            // N = 64), so the descriptors are built once and only advanced by additions in 16-byte units.
+            const uint64_t a_desc0 = ptx::make_smem_desc_sw128(ptx::smem_u32(smem), a_lbo, 1024u);
+            const uint64_t b_desc0 = ptx::make_smem_desc_sw128(ptx::smem_u32(smem) + a_bytes, b_lbo, 1024u);
+            const uint64_t stage_step = stage_bytes >> 4;
+            const uint64_t a_k16 = a_kstep >> 4, b_k16 = b_kstep >> 4;
+            uint64_t a_desc = a_desc0, b_desc = b_desc0;       // descriptors of the current stage
             int stage = 0;
             uint32_t phase = 0;
             int local = 0;
@@ -476,24 +483,25 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         break;
                     }
                     ptx::tc_fence_after_sync();
-                    const uint32_t a_addr = ptx::smem_u32(smem + static_cast<size_t>(stage) * stage_bytes);
-                    const uint32_t b_addr = a_addr + a_bytes;
+                    const uint32_t first = i > 0 ? 1u : 0u;
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         if (h < mh) {
 #pragma unroll
-                            for (int j = 0; j < kBK / kUmmaK; ++j) {
-                                const uint64_t adesc =
-                                    ptx::make_smem_desc_sw128(a_addr + h * kHalfABytes + j * a_kstep, a_lbo, 1024u);
-                                const uint64_t bdesc = ptx::make_smem_desc_sw128(b_addr + j * b_kstep, b_lbo, 1024u);
-                                ptx::umma_bf16(d_tmem[h], adesc, bdesc, idesc, (i > 0 || j > 0) ? 1u : 0u);
-                            }
+                            for (int j = 0; j < kBK / kUmmaK; ++j)
+                                ptx::umma_bf16(d_tmem[h], a_desc + (h * (kHalfABytes >> 4) + j * a_k16), b_desc + j * b_k16,
+                                               idesc, j > 0 ? 1u : first);
                         }
                     }
                     ptx::umma_commit(&empty_bar[stage]);
                     if (++stage == p.stages) {
                         stage = 0;
                         phase ^= 1u;
+                        a_desc = a_desc0;
+                        b_desc = b_desc0;
+                    } else {
+                        a_desc += stage_step;
+                        b_desc += stage_step;
                     }
                 }
                 if (ok) {
