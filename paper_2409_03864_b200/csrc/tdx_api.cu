@@ -270,7 +270,12 @@ int pair_max_stages(int tile_n, int smem_limit, int store_mode) {
     return std::min(s, tdx::kMaxStages);
 }
 
-int tmem_slots_for(int tile_m, int bn) { return (tile_m == 256 && bn <= 128) ? 4 : 2; }
+int tmem_slots_for(int tile_m, int bn) {
+    const int mh = tile_m / 128;
+    int s = std::min(tdx::kMaxSlots, 512 / bn);     // as many as TMEM holds: narrow tiles are short, and the
+    s -= s % mh;                                    // epilogue's latency then spans several tiles
+    return std::max(s, mh);
+}
 int tmem_cols_for(int tile_m, int bn) {
     int c = 32;
     while (c < tmem_slots_for(tile_m, bn) * bn) c *= 2;
@@ -646,6 +651,21 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     p.k_stagger = cfg.k_stagger;
     p.bn = cfg.tile_n;
     p.stages = cfg.stages;
+    if (halo && cfg.tile_n >= c.Cout) {
+        // small filters stay resident: all (chunk, tap) slices of the one column tile fit beside the halo ring,
+        // so they are loaded once per CTA and the main loop has no per-tap handshake
+        const int64_t slices = c.R * c.S * cchunks;
+        const int64_t need = static_cast<int64_t>(p.a_stages) * (cfg.tile_m / 128) * p.halo_bytes + slices * cfg.tile_n * 128 +
+                             staging_bytes_for(cfg.tile_m, cfg.store_mode) + 1024;
+        if (need <= ctx->smem_optin - kStaticSmemReserve) {
+            p.b_resident = 1;
+            p.stages = static_cast<int>(slices);
+            // spend what is left on more halo tiles in flight (their load latency is what a short tile waits for)
+            const int64_t per_stage = static_cast<int64_t>(cfg.tile_m / 128) * p.halo_bytes;
+            while (p.a_stages < tdx::kMaxAStages && need + (p.a_stages - kHaloAStages + 1) * per_stage <= ctx->smem_optin - kStaticSmemReserve)
+                ++p.a_stages;
+        }
+    }
     p.tmem_cols = tmem_cols_for(cfg.tile_m, cfg.tile_n);
     p.a_mn_major = 0;
     p.b_mn_major = 0;

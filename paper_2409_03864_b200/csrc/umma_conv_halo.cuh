@@ -18,7 +18,7 @@
 
 namespace tdx {
 
-constexpr int kMaxAStages = 3;
+constexpr int kMaxAStages = 4;
 
 // output patch of 128-row half `half` of tile `m_blk`: image n and top-left output pixel (p0, q0)
 __device__ __forceinline__ void halo_patch_origin(const UmmaParams& p, int m_blk, int half, int mh, int* n, int* p0,
@@ -62,7 +62,7 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             ptx::mbar_init(&afull_bar[s], 1);
             ptx::mbar_init(&aempty_bar[s], 1);
         }
-        for (int s = 0; s < p.stages; ++s) {
+        for (int s = 0; s < (p.b_resident ? 1 : p.stages); ++s) {
             ptx::mbar_init(&bfull_bar[s], 1);
             ptx::mbar_init(&bempty_bar[s], 1);
         }
@@ -113,6 +113,18 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                 ++a_issued;
             };
 
+            if (p.b_resident) {
+                // the whole filter once (slot = chunk * taps + tap), then only halo tiles
+                ptx::mbar_arrive_expect_tx(&bfull_bar[0], static_cast<uint32_t>(p.cchunks * taps) * b_bytes);
+                for (int cc = 0; cc < p.cchunks; ++cc)
+                    for (int tap = 0; tap < taps; ++tap)
+                        ptx::tma_load_3d(b_ring + static_cast<size_t>(cc * taps + tap) * b_bytes, &tmB, &bfull_bar[0],
+                                         cc * kBK, tap, 0);
+                while (ok && a_item < total_items) {
+                    if (!wait_bounded(&aempty_bar[a_buf], a_phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) ok = false;
+                    else issue_halo();
+                }
+            } else
             for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
                 const TileCoord t = decode_item(p, item);
                 for (int cc = 0; ok && cc < p.cchunks; ++cc, ++b_chunk) {
@@ -155,6 +167,7 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             int a_buf = 0, b_stage = 0, local = 0;
             uint32_t a_phase = 0, b_phase = 0;
             bool ok = true;
+            if (p.b_resident && !wait_bounded(&bfull_bar[0], 0, abort_flag, p.status, kTimeoutMma)) ok = false;
             for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++local) {
                 uint32_t d_tmem[2] = {0u, 0u};
                 int slot[2] = {0, 0};
@@ -174,8 +187,10 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     if (!wait_bounded(&afull_bar[a_buf], a_phase, abort_flag, p.status, kTimeoutMma)) { ok = false; break; }
                     int r = 0, s = 0;                         // filter tap (r, s), advanced without divisions
                     uint64_t row_desc = halo_desc;            // window row r, column 0 (one pixel = 128 B = 8 units)
+                    if (p.b_resident) b_desc = b_desc0 + static_cast<uint64_t>(cc * taps) * b_stage_step;
                     for (int tap = 0; tap < taps; ++tap) {
-                        if (!wait_bounded(&bfull_bar[b_stage], b_phase, abort_flag, p.status, kTimeoutMma)) { ok = false; break; }
+                        if (!p.b_resident &&
+                            !wait_bounded(&bfull_bar[b_stage], b_phase, abort_flag, p.status, kTimeoutMma)) { ok = false; break; }
                         ptx::tc_fence_after_sync();
                         const uint64_t a_tap = row_desc + static_cast<uint64_t>(s) * 8u;
                         const uint32_t first = (cc > 0 || tap > 0) ? 1u : 0u;
@@ -188,8 +203,12 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                                                    j > 0 ? 1u : first);
                             }
                         }
-                        ptx::umma_commit(&bempty_bar[b_stage]);
-                        if (++b_stage == p.stages) { b_stage = 0; b_phase ^= 1u; b_desc = b_desc0; } else { b_desc += b_stage_step; }
+                        if (p.b_resident) {
+                            b_desc += b_stage_step;
+                        } else {
+                            ptx::umma_commit(&bempty_bar[b_stage]);
+                            if (++b_stage == p.stages) { b_stage = 0; b_phase ^= 1u; b_desc = b_desc0; } else { b_desc += b_stage_step; }
+                        }
                         if (++s == p.S) { s = 0; ++r; row_desc += static_cast<uint64_t>(p.hpitch) * 8u; }
                     }
                     if (!ok) break;

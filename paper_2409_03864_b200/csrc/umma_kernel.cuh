@@ -34,7 +34,7 @@ constexpr int kHalfM = 128;       // rows of one MMA / one accumulator slot = TM
 constexpr int kBK = 64;           // K per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaK = 16;        // K of one tcgen05.mma for 16-bit inputs
 constexpr int kMaxStages = 8;
-constexpr int kMaxSlots = 4;
+constexpr int kMaxSlots = 8;
 constexpr int kHalfABytes = kHalfM * kBK * 2;          // 16 KiB: one 128-row half of the A slice
 constexpr long long kWaitLimitCycles = 4000000000LL;  // ~2 s at boost clock
 
@@ -68,6 +68,8 @@ struct UmmaParams {
     int hpitch, hrows;        // halo tile: (8 + S - 1) pixels wide, (16 + R - 1) pixels high
     int halo_bytes;           // hpitch * hrows * 128 rounded up to 1024
     int a_stages;             // halo tiles in flight per 128-row half
+    int b_resident;           // the whole filter (all chunks and taps, one column tile) stays in shared memory:
+                              // loaded once per CTA instead of once per tile, no per-tap handshake
     int* status;              // device status word
 };
 
