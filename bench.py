@@ -168,6 +168,23 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+def max_over_ranks(x, device):
+    """Slowest rank's figure (the job's time); a no-op without a process group.  Works with NCCL (cuda tensors)
+    and gloo (cpu tensors)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(x)
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(flops_per_step, steps, ms_slowest, world):
+    """Whole-job TFLOP/s of `world` independent replicas that each did `steps` steps; time = the slowest rank's."""
+    return world * flops_per_step * steps / (ms_slowest * 1e-3) / 1e12
+
+
 def oracle_sample(wl, host, target_seconds=12.0):
     """Times the CPU oracle on a row sample of the workload; returns (TFLOP/s, threads, description)."""
     import numpy as np
@@ -332,11 +349,9 @@ def run_tdx(args):
     tdx.check(tdx.tdx_check_device_status(stream))
 
     if distributed:
-        t = torch.tensor([ms_total], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+        ms_total = max_over_ranks(ms_total, "cuda")
         dist.barrier()
-    value = world * wl.flops * args.steps / (ms_total * 1e-3) / 1e12
+    value = replica_throughput(wl.flops, args.steps, ms_total, world)
 
     # end to end through the host-buffer entry point: H2D of the inputs, the kernels, D2H of the result, every step
     e2e_steps = max(3, min(args.steps, 20))
@@ -351,10 +366,8 @@ def run_tdx(args):
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     if distributed:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
-    e2e_value = world * wl.flops * e2e_steps / e2e_s / 1e12
+        e2e_s = max_over_ranks(e2e_s, "cuda")
+    e2e_value = replica_throughput(wl.flops, e2e_steps, e2e_s * 1e3, world)
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()

@@ -223,6 +223,15 @@ int tdx_check_device_status(void* stream);
 int tdx_gemm_splitk_static(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha,
                            const void* A, const void* B, void* C, int tile_n, int split_k, void* stream);
 
+/*
+ * Self-test of the failure path: launches a one-warp kernel that waits on a barrier nothing ever signals, with a
+ * wait limit of about `limit_us` microseconds (1 .. 100000).  The wait gives up, records its code in the device
+ * status word and the kernel returns normally -- nothing traps or hangs, the context stays usable.  The next
+ * tdx_check_device_status on that stream therefore reports TDX_ERR_TIMEOUT (once).  This is how the error model
+ * of the paper's Section 3 (a definite error is reported, not swallowed) is exercised without faulting a device.
+ */
+int tdx_selftest_bounded_wait(int limit_us, void* stream);
+
 /* Number of kernels this library has launched in this process (all threads). */
 int64_t tdx_kernel_launch_count(void);
 

@@ -85,6 +85,7 @@ def lib() -> ctypes.CDLL:
         L.tdx_tune_clear.argtypes = []
         L.tdx_gemm_splitk_static.argtypes = [i64, i64, i64, ci, ci, cf, vp, vp, vp, ci, ci, vp]
         L.tdx_check_device_status.argtypes = [vp]
+        L.tdx_selftest_bounded_wait.argtypes = [ci, vp]
         L.tdx_kernel_launch_count.argtypes = []
         L.tdx_kernel_launch_count.restype = i64
         L.tdx_last_error.restype = ctypes.c_char_p
@@ -107,7 +108,7 @@ EXPORTS = (
     "tdx_gemm", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_relu_ex",
     "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
     "tdx_enum_conv2d_configs", "tdx_default_gemm_config", "tdx_default_conv2d_config", "tdx_tune_save",
-    "tdx_tune_load", "tdx_tune_clear", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_kernel_launch_count", "tdx_last_error",
+    "tdx_tune_load", "tdx_tune_clear", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
     "tdx_version",
 )
 
@@ -267,6 +268,10 @@ def tdx_gemm_splitk_static(M, N, K, transA, transB, alpha, A, B, C, tile_n=0, sp
 
 def tdx_check_device_status(stream=None) -> int:
     return lib().tdx_check_device_status(_stream(stream))
+
+
+def tdx_selftest_bounded_wait(limit_us=200, stream=None) -> int:
+    return lib().tdx_selftest_bounded_wait(limit_us, _stream(stream))
 
 
 def tdx_kernel_launch_count() -> int:

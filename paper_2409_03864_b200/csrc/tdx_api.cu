@@ -1531,6 +1531,18 @@ int tdx_check_device_status(void* stream) {
     return TDX_OK;
 }
 
+int tdx_selftest_bounded_wait(int limit_us, void* stream) {
+    if (limit_us < 1 || limit_us > 100000) return fail(TDX_ERR_INVALID_ARG, "limit_us must be in [1, 100000]");
+    DeviceCtx* ctx;
+    int rc = get_ctx(&ctx);
+    if (rc) return rc;
+    const long long cycles = static_cast<long long>(limit_us) * 2000;   // ~2 GHz: exactness does not matter here
+    tdx::bounded_wait_selftest_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(ctx->status_ptr, cycles);
+    TDX_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return TDX_OK;
+}
+
 int64_t tdx_kernel_launch_count(void) { return g_launches.load(); }
 
 }  // extern "C"

@@ -73,8 +73,8 @@ struct UmmaParams {
     int* status;              // device status word
 };
 
-__device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, volatile int* s_abort, int* g_status,
-                                             int code) {
+__device__ __forceinline__ bool wait_bounded_for(uint64_t* bar, uint32_t parity, volatile int* s_abort, int* g_status,
+                                                 int code, long long limit_cycles) {
     if (ptx::mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
@@ -82,13 +82,32 @@ __device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, vol
         if (ptx::mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0u) {
             if (*s_abort) return false;
-            if (clock64() - t0 > kWaitLimitCycles) {
+            if (clock64() - t0 > limit_cycles) {
                 *s_abort = 1;
                 atomicCAS(g_status, 0, code);
                 return false;
             }
         }
     }
+}
+__device__ __forceinline__ bool wait_bounded(uint64_t* bar, uint32_t parity, volatile int* s_abort, int* g_status,
+                                             int code) {
+    return wait_bounded_for(bar, parity, s_abort, g_status, code, kWaitLimitCycles);
+}
+
+// Self-test of the bounded wait: one warp waits on a barrier that nothing ever signals, with a short limit; the wait
+// must give up, record `kTimeoutSelfTest` in the status word and let the kernel return normally.
+enum : int { kTimeoutSelfTest = 9 };
+__global__ void bounded_wait_selftest_kernel(int* status, long long limit_cycles) {
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int s_abort;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        s_abort = 0;
+        ptx::fence_barrier_init();
+    }
+    __syncthreads();
+    wait_bounded_for(&bar, 0, &s_abort, status, kTimeoutSelfTest, limit_cycles);
 }
 
 struct TileCoord {
