@@ -80,7 +80,9 @@ typedef struct {
                     /*     so that CTAs do not all fetch the same operand lines at the same moment       */
     int halo;       /* conv only: 1 = the input window is fetched again for every filter tap; 2 = it is   */
                     /*     loaded once per 64-channel chunk into shared memory and all taps read it there  */
-                    /*     (8 x 16 patches, stride 1, more than one tap); 0 = choose                      */
+                    /*     (8 x 16 patches, stride 1, more than one tap); 3 = as 2, but the 16-row patches */
+                    /*     are cut from the column formed by all images of the batch, H + pad rows apart, so */
+                    /*     that an image height that is no multiple of 16 wastes no rows; 0 = choose        */
 } tdx_config;
 
 /*

@@ -13,6 +13,22 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
+// One lane of a converged warp, chosen by the hardware.  Unlike a test of the lane index, this tells the compiler that
+// exactly one lane runs the branch, so descriptor operands stay in the uniform datapath: measured on B200, a
+// tcgen05.mma chain issued under `lane == 0` costs 143-153 cycles per instruction whatever its shape, under
+// elect.sync 127 cycles at N = 256 (the tensor pipe's own rate) and about 60 at N <= 128.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "elect.sync _|p, 0xffffffff;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");

@@ -253,6 +253,15 @@ int umma_max_stages(int tile_m, int tile_n, int smem_limit, int store_mode) {
 // when they fit so that the epilogue still overlaps the next tile's main loop.
 // Halo-reuse convolution: 8 x 16 output-pixel patches, input window kept in shared memory across the taps.
 constexpr int kHaloPatchW = 8, kHaloPatchH = 16, kHaloAStages = 2;
+// Stacked images: rows each image takes in the column of all images.  The rows between two images must read as
+// zero for both, i.e. be the bottom padding of one and the top padding of the next: H + pad rows per image
+// (never fewer than the P output rows).
+int64_t stacked_rows_per_image(const ConvProblem& c) { return std::max(c.P, c.H + c.pad); }
+// 128-row halves the halo kernel works on: 8 x 16 patches cut per image (halo 2) or from the stacked column (halo 3)
+int64_t halo_patches(const ConvProblem& c, int mode) {
+    const int64_t pw = ceil_div(c.Q, kHaloPatchW);
+    return mode == 3 ? pw * ceil_div(c.N * stacked_rows_per_image(c), kHaloPatchH) : pw * c.N * ceil_div(c.P, kHaloPatchH);
+}
 int halo_tile_bytes(int64_t R, int64_t S) {
     const int64_t b = (kHaloPatchW + S - 1) * (kHaloPatchH + R - 1) * 128;
     return static_cast<int>((b + 1023) / 1024 * 1024);
@@ -305,8 +314,9 @@ const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num
     if (c.tile_n < 32 || c.tile_n > 256 || c.tile_n % 32) return "tile_n must be a multiple of 32 in [32, 256]";
     if (b_mn_major && c.tile_n % 64) return "tile_n must be a multiple of 64 when B is read N-major";
     if (!conv && c.halo > 1) return "halo applies to the convolution only";
-    if (conv && c.halo != 1 && c.halo != 2) return "halo must be 1 (per-tap loads) or 2 (halo tile kept in shared memory)";
-    if (conv && c.halo == 2) {
+    if (conv && (c.halo < 1 || c.halo > 3))
+        return "halo must be 1 (per-tap loads), 2 (halo tile kept in shared memory) or 3 (the same over stacked images)";
+    if (conv && c.halo >= 2) {
         if (R * S < 2) return "halo reuse needs a filter with more than one tap";
         if (c.patch_w != kHaloPatchW || c.patch_h != kHaloPatchH) return "halo reuse works on 8 x 16 patches";
         if (kHaloPatchW + S - 1 > 256 || kHaloPatchH + R - 1 > 256) return "filter too large for a halo tile";
@@ -391,7 +401,8 @@ void default_umma_config(int64_t tiles_m, int64_t N, int64_t num_kb, bool b_mn_m
 
 // ------------------------------------------------------------------ launches
 int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
-                const UmmaParams& p, cudaStream_t st, bool halo = false) {
+                const UmmaParams& p, cudaStream_t st, bool halo = false, const CUtensorMap* ma_row = nullptr,
+                const CUtensorMap* mc_row = nullptr) {
     const long long items = static_cast<long long>(p.tiles_m) * p.tiles_n * p.split_k;
     const int grid = static_cast<int>(std::min<long long>(items, ctx->sm_count));
     size_t smem = static_cast<size_t>(p.stages) * ((p.bm + p.bn) * 128) + 1024 +
@@ -401,8 +412,8 @@ int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensor
                1024 + staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
     // producer warp, MMA warp, then 16 epilogue warps (staged epilogue) or 4 per 128-row half (direct)
     const int threads = p.tma_store ? 576 : (p.bm == 256 ? 320 : 192);
-    if (halo)
-        tdx::umma_conv_halo_kernel<<<grid, threads, smem, st>>>(ma, mb, mc, p);
+    if (halo)   // one more warp: the halo producer
+        tdx::umma_conv_halo_kernel<<<grid, threads + 32, smem, st>>>(ma, ma_row ? *ma_row : ma, mb, mc, mc_row ? *mc_row : mc, p);
     else if (conv)
         tdx::umma_contract_kernel<true><<<grid, threads, smem, st>>>(ma, mb, mc, p);
     else
@@ -629,7 +640,8 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     p.bm = cfg.tile_m;
     p.slots = tmem_slots_for(cfg.tile_m, cfg.tile_n);
     p.nb = cfg.tile_m / (p.bw * p.bh);
-    const bool halo = cfg.halo == 2;
+    const bool halo = cfg.halo >= 2;
+    const bool stacked = cfg.halo == 3;
     if (halo) {
         p.R = static_cast<int>(c.R);
         p.hpitch = static_cast<int>(kHaloPatchW + c.S - 1);
@@ -639,7 +651,13 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     }
     p.patches_w = static_cast<int>(ceil_div(c.Q, p.bw));
     p.patches_h = static_cast<int>(ceil_div(c.P, p.bh));
-    const int64_t total_patches = c.N * p.patches_w * p.patches_h;
+    int64_t total_patches = c.N * p.patches_w * p.patches_h;
+    if (stacked) {
+        p.Pv = static_cast<int>(stacked_rows_per_image(c));
+        p.H = static_cast<int>(c.H);
+        p.patches_h = static_cast<int>(ceil_div(c.N * p.Pv, p.bh));      // over the whole column of images
+        total_patches = static_cast<int64_t>(p.patches_w) * p.patches_h;
+    }
     p.M = static_cast<int>(c.N * c.P * c.Q);
     p.N = static_cast<int>(c.Cout);
     p.num_kb = static_cast<int>(c.R * c.S * cchunks);
@@ -683,7 +701,7 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     p.cchunks = cchunks;
     p.status = ctx->status_ptr;
 
-    CUtensorMap ma, mb;
+    CUtensorMap ma, ma_row, mb;
     {
         uint64_t dims[4] = {static_cast<uint64_t>(c.Cin), static_cast<uint64_t>(c.W), static_cast<uint64_t>(c.H),
                             static_cast<uint64_t>(c.N)};
@@ -692,6 +710,12 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
         uint32_t box[4] = {64, static_cast<uint32_t>(halo ? p.hpitch : p.bw), static_cast<uint32_t>(halo ? p.hrows : p.bh), 1};
         int rc = get_tensor_map(ctx, x, 4, dims, str, box, &ma);
         if (rc) return rc;
+        ma_row = ma;
+        if (stacked) {
+            box[2] = 1;              // windows that reach into the next image are copied one row at a time
+            rc = get_tensor_map(ctx, x, 4, dims, str, box, &ma_row);
+            if (rc) return rc;
+        }
     }
     {
         uint64_t dims[3] = {static_cast<uint64_t>(c.Cin), static_cast<uint64_t>(c.R * c.S),
@@ -701,8 +725,9 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
         int rc = get_tensor_map(ctx, w, 3, dims, str, box, &mb);
         if (rc) return rc;
     }
-    CUtensorMap mc = ma;
+    CUtensorMap mc = ma, mc_row = ma;
     p.tma_store = (cfg.store_mode == 2 && p.vec_store && p.bw * p.bh >= 32) ? 1 : 0;
+    if (halo) p.epi_warps = p.tma_store ? 16 : 4 * (cfg.tile_m / 128);
     if (p.tma_store) {
         p.sbx = std::min(p.bw, 32);
         p.sby = 32 / p.sbx;
@@ -713,8 +738,14 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
         uint32_t box[4] = {32, static_cast<uint32_t>(p.sbx), static_cast<uint32_t>(p.sby), 1};
         int rc = get_tensor_map(ctx, y, 4, dims, str, box, &mc, 64);
         if (rc) return rc;
+        mc_row = mc;
+        if (stacked) {
+            box[2] = 1;              // four pixel rows that cross the seam between two images leave one by one
+            rc = get_tensor_map(ctx, y, 4, dims, str, box, &mc_row, 64);
+            if (rc) return rc;
+        }
     }
-    return launch_umma(ctx, true, ma, mb, mc, p, st, halo);
+    return launch_umma(ctx, true, ma, mb, mc, p, st, halo, &ma_row, &mc_row);
 }
 
 void gemm_strides(const GemmProblem& g, long long* sa_i, long long* sa_k, long long* sb_k, long long* sb_j) {
@@ -902,14 +933,19 @@ int resolve_conv_config(const ConvProblem& cp, const tdx_config* user, int sm_co
             const int64_t best = ceil_div(cp.Q, bw) * bw * ceil_div(cp.P, bh) * bh;
             const int64_t mine = ceil_div(cp.Q, kHaloPatchW) * kHaloPatchW * ceil_div(cp.P, kHaloPatchH) * kHaloPatchH;
             const int tm = c.tile_m ? c.tile_m : 128, tn = c.tile_n ? c.tile_n : 64;
-            if (mine * 100 <= best * 120 && halo_max_stages(tm, tn, cp.R, cp.S, smem_limit, 2) >= 2) c.halo = 2;
+            if (halo_max_stages(tm, tn, cp.R, cp.S, smem_limit, 2) >= 2) {
+                // patches cut from the stacked column of images when that leaves fewer padded rows
+                if (halo_patches(cp, 3) < halo_patches(cp, 2)) c.halo = 3;
+                else if (mine * 100 <= best * 120) c.halo = 2;
+            }
         }
     }
-    if (c.halo == 2 && c.patch_w == 0 && c.patch_h == 0) { c.patch_w = kHaloPatchW; c.patch_h = kHaloPatchH; }
+    if (c.halo >= 2 && c.patch_w == 0 && c.patch_h == 0) { c.patch_w = kHaloPatchW; c.patch_h = kHaloPatchH; }
     if (c.patch_w == 0 && c.patch_h == 0) choose_patch(cp.P, cp.Q, &c.patch_w, &c.patch_h);
     if (!patch_ok(c.patch_w, c.patch_h)) return fail(TDX_ERR_CONFIG, "infeasible config: patch %dx%d", c.patch_w, c.patch_h);
     const int nb = 128 / (c.patch_w * c.patch_h);
-    const int64_t tiles_m = ceil_div(cp.N * ceil_div(cp.Q, c.patch_w) * ceil_div(cp.P, c.patch_h), nb);
+    const int64_t tiles_m = c.halo >= 2 ? halo_patches(cp, c.halo)
+                                        : ceil_div(cp.N * ceil_div(cp.Q, c.patch_w) * ceil_div(cp.P, c.patch_h), nb);
     const int64_t num_kb = cp.R * cp.S * ceil_div(cp.Cin, 64);
     tdx_config d;
     default_umma_config(tiles_m, cp.Cout, num_kb, false, sm_count, smem_limit, false, &d);
@@ -920,14 +956,14 @@ int resolve_conv_config(const ConvProblem& cp, const tdx_config* user, int sm_co
     if (c.split_k == 0) c.split_k = 1;
     if (c.store_mode == 0) {
         c.store_mode = (cp.Cout % 8 == 0 && c.patch_w * c.patch_h >= 32) ? 2 : 1;
-        if (c.store_mode == 2 && c.halo != 2 && c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, 2)) c.store_mode = 1;
+        if (c.store_mode == 2 && c.halo < 2 && c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, 2)) c.store_mode = 1;
     }
     if (c.stages == 0)
-        c.stages = c.halo == 2 ? std::max(2, halo_max_stages(c.tile_m, c.tile_n, cp.R, cp.S, smem_limit, c.store_mode))
+        c.stages = c.halo >= 2 ? std::max(2, halo_max_stages(c.tile_m, c.tile_n, cp.R, cp.S, smem_limit, c.store_mode))
                                : std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode));
     if (!user && !from_cache) c.raster = d.raster;
     const char* why = umma_config_reason(c, false, num_kb, smem_limit, true, cp.Cout, cp.R, cp.S);
-    if (why && halo_auto && c.halo == 2) {
+    if (why && halo_auto && c.halo >= 2) {
         // the automatic choice of halo reuse did not fit (large filter): fall back to per-tap loads
         tdx_config retry;
         std::memset(&retry, 0, sizeof retry);
@@ -1126,8 +1162,10 @@ int enum_conv(const ConvProblem& cp, int sm_count, int smem_limit, std::vector<t
     // halo-reuse candidates (8 x 16 patches)
     if (cp.R * cp.S > 1) {
         const int64_t num_kb = cp.R * cp.S * ceil_div(cp.Cin, 64);
+        for (int mode : {2, 3})
         for (int tm : {256, 128})
             for (int bn = 256; bn >= 32; bn -= 32) {
+                if (mode == 3 && halo_patches(cp, 3) >= halo_patches(cp, 2)) continue;   // stacking saves nothing
                 if (bn > 32 && bn - 32 >= cp.Cout) continue;
                 if (bn != 256 && bn != 128 && bn != 64 && bn != 32 && cp.Cout % bn) continue;
                 const int sm = cp.Cout % 8 == 0 ? 2 : 1;
@@ -1139,7 +1177,7 @@ int enum_conv(const ConvProblem& cp, int sm_count, int smem_limit, std::vector<t
                         std::memset(&c, 0, sizeof c);
                         c.kernel = TDX_KERNEL_UMMA;
                         c.tile_m = tm; c.tile_n = bn; c.tile_k = 64; c.stages = st; c.cta_pair = 1; c.split_k = 1;
-                        c.store_mode = sm; c.raster = raster; c.patch_w = kHaloPatchW; c.patch_h = kHaloPatchH; c.halo = 2;
+                        c.store_mode = sm; c.raster = raster; c.patch_w = kHaloPatchW; c.patch_h = kHaloPatchH; c.halo = mode;
                         if (umma_config_reason(c, false, num_kb, smem_limit, true, cp.Cout, cp.R, cp.S) == nullptr) v->push_back(c);
                     }
                 }

@@ -11,8 +11,13 @@
 // consistently what the copy engine wrote.
 //
 // Two rings: halo tiles (a_stages deep, one per channel chunk and 128-row half) and filter slices
-// (stages deep, one per (chunk, tap)).  Roles, accumulator slots, epilogue and bounded waits are those
-// of umma_contract_kernel.
+// (stages deep, one per (chunk, tap)), each filled by its own warp (the last warp and warp 0), so that a
+// halo tile that takes many copies never holds up the filter slices.  Accumulator slots, epilogue and
+// bounded waits are those of umma_contract_kernel.
+//
+// Stacked images (Pv > 0): the 16-row patches are cut from the column formed by all images, Pv = H + pad
+// rows per image, so an image height that is no multiple of 16 wastes no rows.  The Pv - P rows between
+// two images read as zero: they are the bottom padding of one image and the top padding of the next.
 #pragma once
 #include "umma_kernel.cuh"
 
@@ -24,6 +29,14 @@ constexpr int kMaxAStages = 4;
 __device__ __forceinline__ void halo_patch_origin(const UmmaParams& p, int m_blk, int half, int mh, int* n, int* p0,
                                                   int* q0) {
     const int patch = m_blk * mh + half;
+    if (p.Pv > 0) {
+        // stacked images: *p0 is the row in the column of all images, *n is not used
+        const int ph = patch / p.patches_w;
+        *n = 0;
+        *p0 = ph * p.bh;
+        *q0 = (patch - ph * p.patches_w) * p.bw;
+        return;
+    }
     const int ppi = p.patches_w * p.patches_h;
     *n = patch / ppi;
     const int rem = patch - *n * ppi;
@@ -32,9 +45,10 @@ __device__ __forceinline__ void halo_patch_origin(const UmmaParams& p, int m_blk
     *q0 = (rem - ph * p.patches_w) * p.bw;
 }
 
-__global__ void __launch_bounds__(576, 1)
-umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                      const __grid_constant__ CUtensorMap tmC, const UmmaParams p) {
+__global__ void __launch_bounds__(608, 1)
+umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA_row,
+                      const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmC,
+                      const __grid_constant__ CUtensorMap tmC_row, const UmmaParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t afull_bar[kMaxAStages];
     __shared__ __align__(8) uint64_t aempty_bar[kMaxAStages];
@@ -56,6 +70,7 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     uint8_t* staging = b_ring + static_cast<size_t>(p.stages) * b_bytes;
     volatile int* abort_flag = &s_abort;
     const int taps = p.R * p.S;
+    const int halo_warp = 2 + p.epi_warps;      // the last warp loads the halo tiles
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.a_stages; ++s) {
@@ -68,13 +83,17 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         }
         for (int b = 0; b < p.slots; ++b) {
             ptx::mbar_init(&tfull_bar[b], 1);
-            ptx::mbar_init(&tempty_bar[b], static_cast<uint32_t>(((blockDim.x >> 5) - 2) / mh));
+            ptx::mbar_init(&tempty_bar[b], static_cast<uint32_t>(p.epi_warps / mh));
         }
         s_abort = 0;
         ptx::fence_barrier_init();
         ptx::tma_prefetch_desc(&tmA);
         ptx::tma_prefetch_desc(&tmB);
-        if (p.tma_store) ptx::tma_prefetch_desc(&tmC);
+        if (p.Pv > 0) ptx::tma_prefetch_desc(&tmA_row);
+        if (p.tma_store) {
+            ptx::tma_prefetch_desc(&tmC);
+            if (p.Pv > 0) ptx::tma_prefetch_desc(&tmC_row);
+        }
     }
     if (warp == 1) {
         __syncwarp();
@@ -87,64 +106,88 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     const uint32_t tmem_base = s_tmem_base;
     const int total_items = p.tiles_m * p.tiles_n;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------ producer: two cursors, halo tiles ahead of slices
-        if (lane == 0) {
-            int a_item = blockIdx.x, a_cc = 0, a_buf = 0;     // next halo load to issue
-            uint32_t a_phase = 0;
-            long long a_issued = 0, b_chunk = 0;             // halo loads issued / channel chunks started by the slice cursor
-            int b_stage = 0;
-            uint32_t b_phase = 0;
-            bool ok = true;
+    if (warp == halo_warp) {
+        // ------------------------------------------------------------ halo producer: one tile per (item, channel chunk)
+        if (ptx::elect_one()) {
             const uint32_t halo_tx = static_cast<uint32_t>(mh * p.hpitch * p.hrows) * 128u;
-
-            auto issue_halo = [&]() {
-                const TileCoord t = decode_item(p, a_item);
-                uint64_t* bar = &afull_bar[a_buf];
-                ptx::mbar_arrive_expect_tx(bar, halo_tx);
-                for (int h = 0; h < mh; ++h) {
-                    int n, p0, q0;
-                    halo_patch_origin(p, t.m_blk, h, mh, &n, &p0, &q0);
-                    ptx::tma_load_4d(a_ring + static_cast<size_t>(a_buf) * a_stage_bytes + h * p.halo_bytes, &tmA, bar,
-                                     a_cc * kBK, q0 - p.pad, p0 - p.pad, n);
+            int a_buf = 0;
+            uint32_t a_phase = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
+                const TileCoord t = decode_item(p, item);
+                for (int cc = 0; cc < p.cchunks; ++cc) {
+                    if (!wait_bounded(&aempty_bar[a_buf], a_phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) {
+                        ok = false;
+                        break;
+                    }
+                    uint64_t* bar = &afull_bar[a_buf];
+                    ptx::mbar_arrive_expect_tx(bar, halo_tx);
+                    for (int h = 0; h < mh; ++h) {
+                        int n, p0, q0;
+                        halo_patch_origin(p, t.m_blk, h, mh, &n, &p0, &q0);
+                        uint8_t* dst = a_ring + static_cast<size_t>(a_buf) * a_stage_bytes + h * p.halo_bytes;
+                        if (p.Pv > 0) {
+                            // Row u of the stacked column is row u % Pv of image u / Pv when that is below H, and
+                            // zero otherwise.  A window that lies inside one image and the zero rows around it is
+                            // one box (rows outside [0, H) are zero-filled); a window that reaches into the next
+                            // image is copied row by row.
+                            const int u = p0 - p.pad;
+                            int img = u >= 0 ? u / p.Pv : 0;
+                            int row = u >= 0 ? u - img * p.Pv : u;       // negative: above the first image
+                            if (row >= p.H) {                            // starts in the zero rows below image img:
+                                row -= p.Pv;                             // the same rows lie above image img + 1
+                                ++img;
+                            }
+                            if (row + p.hrows <= p.Pv) {
+                                // img == Nimg happens past the last image: that coordinate is zero-filled too
+                                ptx::tma_load_4d(dst, &tmA, bar, cc * kBK, q0 - p.pad, row, img);
+                            } else {
+                                for (int j = 0; j < p.hrows; ++j) {
+                                    const bool real = row >= 0 && row < p.H && img < p.Nimg;
+                                    ptx::tma_load_4d(dst + j * p.hpitch * 128, &tmA_row, bar, cc * kBK, q0 - p.pad,
+                                                     real ? row : p.H, real ? img : 0);
+                                    if (++row == p.Pv) { row = 0; ++img; }
+                                }
+                            }
+                        } else {
+                            ptx::tma_load_4d(dst, &tmA, bar, cc * kBK, q0 - p.pad, p0 - p.pad, n);
+                        }
+                    }
+                    if (++a_buf == p.a_stages) { a_buf = 0; a_phase ^= 1u; }
                 }
-                if (++a_buf == p.a_stages) { a_buf = 0; a_phase ^= 1u; }
-                if (++a_cc == p.cchunks) { a_cc = 0; a_item += gridDim.x; }
-                ++a_issued;
-            };
-
+            }
+            if (!ok) {
+                for (int i = 0; i < 64; ++i) __nanosleep(2000);
+            }
+        }
+    } else if (warp == 0) {
+        // ------------------------------------------------------------ filter producer
+        if (ptx::elect_one()) {
+            bool ok = true;
             if (p.b_resident) {
-                // the whole filter once (slot = chunk * taps + tap), then only halo tiles
+                // the whole filter once (slot = chunk * taps + tap)
                 ptx::mbar_arrive_expect_tx(&bfull_bar[0], static_cast<uint32_t>(p.cchunks * taps) * b_bytes);
                 for (int cc = 0; cc < p.cchunks; ++cc)
                     for (int tap = 0; tap < taps; ++tap)
                         ptx::tma_load_3d(b_ring + static_cast<size_t>(cc * taps + tap) * b_bytes, &tmB, &bfull_bar[0],
                                          cc * kBK, tap, 0);
-                while (ok && a_item < total_items) {
-                    if (!wait_bounded(&aempty_bar[a_buf], a_phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) ok = false;
-                    else issue_halo();
-                }
-            } else
-            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
-                const TileCoord t = decode_item(p, item);
-                for (int cc = 0; ok && cc < p.cchunks; ++cc, ++b_chunk) {
-                    // the halo tile of this chunk must be on its way before its filter slices queue up behind it
-                    while (ok && a_issued <= b_chunk) {
-                        if (!wait_bounded(&aempty_bar[a_buf], a_phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) ok = false;
-                        else issue_halo();
-                    }
-                    for (int tap = 0; ok && tap < taps; ++tap) {
-                        // run ahead with halo tiles whenever a buffer is free
-                        if (a_item < total_items && ptx::mbar_try_wait(&aempty_bar[a_buf], a_phase ^ 1u)) issue_halo();
-                        if (!wait_bounded(&bempty_bar[b_stage], b_phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) {
-                            ok = false;
-                            break;
+            } else {
+                int b_stage = 0;
+                uint32_t b_phase = 0;
+                for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
+                    const TileCoord t = decode_item(p, item);
+                    for (int cc = 0; ok && cc < p.cchunks; ++cc) {
+                        for (int tap = 0; tap < taps; ++tap) {
+                            if (!wait_bounded(&bempty_bar[b_stage], b_phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) {
+                                ok = false;
+                                break;
+                            }
+                            uint64_t* bar = &bfull_bar[b_stage];
+                            ptx::mbar_arrive_expect_tx(bar, b_bytes);
+                            ptx::tma_load_3d(b_ring + static_cast<size_t>(b_stage) * b_bytes, &tmB, bar, cc * kBK, tap,
+                                             t.n_blk * p.bn);
+                            if (++b_stage == p.stages) { b_stage = 0; b_phase ^= 1u; }
                         }
-                        uint64_t* bar = &bfull_bar[b_stage];
-                        ptx::mbar_arrive_expect_tx(bar, b_bytes);
-                        ptx::tma_load_3d(b_ring + static_cast<size_t>(b_stage) * b_bytes, &tmB, bar, cc * kBK, tap,
-                                         t.n_blk * p.bn);
-                        if (++b_stage == p.stages) { b_stage = 0; b_phase ^= 1u; }
                     }
                 }
             }
@@ -154,7 +197,7 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        if (ptx::elect_one()) {
             const uint32_t idesc = ptx::make_idesc_bf16_f32(kHalfM, p.bn, 0, 0);
             const uint32_t a_sbo = static_cast<uint32_t>(p.hpitch) * 128u;     // one window row between 8-row groups
             // descriptors are built once and advanced by additions (16-byte units): the issuing thread has only
@@ -222,7 +265,8 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             }
         }
     } else {
-        epilogue_role<true>(p, &tmC, staging, tmem_base, tfull_bar, tempty_bar, abort_flag, mh, warp, lane, total_items);
+        epilogue_role<true>(p, &tmC, staging, tmem_base, tfull_bar, tempty_bar, abort_flag, mh, warp, lane, total_items,
+                            -1, 0, 1, 0, 0, &tmC_row);
     }
 
     ptx::tc_fence_before_sync();

@@ -70,6 +70,11 @@ struct UmmaParams {
     int a_stages;             // halo tiles in flight per 128-row half
     int b_resident;           // the whole filter (all chunks and taps, one column tile) stays in shared memory:
                               // loaded once per CTA instead of once per tile, no per-tap handshake
+    int epi_warps;            // epilogue warps (0: every warp from the third on)
+    int Pv, H;                // stacked images (Pv > 0): the images of the batch form one column of Nimg * Pv rows,
+                              // image n owning rows [n * Pv, n * Pv + P) and the Pv - P rows below it reading as
+                              // zero (they are the bottom padding of image n and the top padding of image n + 1);
+                              // 16-row patches are cut from that column, so they may straddle two images
     int* status;              // device status word
 };
 
@@ -138,7 +143,7 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                                               uint32_t tmem_base, uint64_t* tfull_bar, uint64_t* tempty_bar,
                                               volatile int* abort_flag, int mh, int warp, int lane, int total_items,
                                               int first_item = -1, int item_stride = 0, int m_mul = 1, int m_add = 0,
-                                              uint32_t tempty_cluster_addr = 0) {
+                                              uint32_t tempty_cluster_addr = 0, const CUtensorMap* tmC_row = nullptr) {
     // CTA pairs: the pair walks tiles of 256 rows, this CTA owns rows [128 * (2 m + rank), +128) of tile m, and the
     // accumulator-free signal goes to the leader CTA's barrier (tempty_cluster_addr, a shared::cluster address)
     if (first_item < 0) {
@@ -146,7 +151,7 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
         item_stride = gridDim.x;
     }
     const int ew = warp - 2;
-    const int nwarps_epi = (static_cast<int>(blockDim.x) >> 5) - 2;
+    const int nwarps_epi = p.epi_warps > 0 ? p.epi_warps : (static_cast<int>(blockDim.x) >> 5) - 2;
     const int ncgrp = nwarps_epi / (4 * mh);      // warps sharing one (half, quarter)
     const int half = (ew >> 2) % mh;              // which 128-row half of the tile this warp drains
     const int cgrp = (ew >> 2) / mh;              // which share of the columns
@@ -171,13 +176,22 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
             const int hl = within / p.bw;
             const int wl = within - hl * p.bw;
             const int patch = t.m_blk * p.nb + pl;
-            const int ppi = p.patches_w * p.patches_h;
-            const int n = patch / ppi;
-            const int rem = patch - n * ppi;
-            const int ph = rem / p.patches_w;
-            const int pw = rem - ph * p.patches_w;
-            const int pp = ph * p.bh + hl;
-            const int qq = pw * p.bw + wl;
+            int n, pp, qq;
+            if (p.Pv > 0) {
+                const int ph = patch / p.patches_w;
+                const int v = ph * p.bh + hl;            // row in the column of stacked images
+                n = v / p.Pv;
+                pp = v - n * p.Pv;
+                qq = (patch - ph * p.patches_w) * p.bw + wl;
+            } else {
+                const int ppi = p.patches_w * p.patches_h;
+                n = patch / ppi;
+                const int rem = patch - n * ppi;
+                const int ph = rem / p.patches_w;
+                const int pw = rem - ph * p.patches_w;
+                pp = ph * p.bh + hl;
+                qq = pw * p.bw + wl;
+            }
             valid = (n < p.Nimg) && (pp < p.P) && (qq < p.Q);
             grow = (static_cast<long long>(n) * p.P + pp) * p.Q + qq;
         } else {
@@ -191,7 +205,32 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
             const int wrow0 = half * kHalfM + quarter * 32;      // first tile row of this warp
             int sc1 = 0, sc2 = 0, sc3 = 0;                       // store coordinates above the column
             bool box_ok;
-            if (kConv) {
+            // stacked images: the warp's four pixel rows (8 pixels x 32 channels = 512 bytes of the staging block
+            // each) leave as one box when they lie in one image; where they cross the seam between two images,
+            // lanes 0..3 store one pixel row each
+            int nstore = 1;
+            const CUtensorMap* store_map = tmC;
+            if (kConv && p.Pv > 0) {
+                const int pl = wrow0 / kHalfM;
+                const int hl0 = (wrow0 - pl * kHalfM) / p.bw;
+                const int patch = t.m_blk * p.nb + pl;
+                const int ph = patch / p.patches_w;
+                const int v0 = ph * p.bh + hl0;
+                const int n0 = v0 / p.Pv;
+                sc1 = (patch - ph * p.patches_w) * p.bw;
+                if (v0 - n0 * p.Pv + 3 < p.P) {
+                    sc3 = n0;
+                    sc2 = v0 - n0 * p.Pv;
+                    box_ok = n0 < p.Nimg;
+                } else {
+                    const int v = v0 + (lane & 3);
+                    sc3 = v / p.Pv;
+                    sc2 = v - sc3 * p.Pv;
+                    box_ok = (sc3 < p.Nimg) && (sc2 < p.P);
+                    nstore = 4;
+                    store_map = tmC_row;
+                }
+            } else if (kConv) {
                 const int per_patch = p.bw * p.bh;
                 const int pl = wrow0 / per_patch;
                 const int within = wrow0 - pl * per_patch;
@@ -220,10 +259,14 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                        static_cast<uint32_t>(buf * p.bn + c0);
                 ptx::tmem_ld_32x32b_x32(taddr, r);
-                ptx::tmem_ld_wait();
                 const int col0 = t.n_blk * p.bn + c0;
+                // lane l fetches the bias of column col0 + l while the accumulator load is in flight; columns past N
+                // are clipped by the store, the index only has to stay in range
+                float bias_l = 0.0f;
+                if (p.bias != nullptr) bias_l = __ldg(p.bias + min(col0 + lane, p.N - 1));
+                ptx::tmem_ld_wait();
                 // the previous store of this warp must have finished reading the staging block
-                if (lane == 0) ptx::tma_store_wait_read<0>();
+                if (lane < nstore) ptx::tma_store_wait_read<0>();
                 __syncwarp();
                 if (plain) {
 #pragma unroll
@@ -238,19 +281,14 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                         *reinterpret_cast<uint4*>(my_row + ((g ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
                     }
                 } else {
-                    const int last = p.N - 1;    // columns past N are clipped by the store; keep the bias index in range
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         uint32_t pk[4];
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const int j = g * 8 + e * 2;
-                            float x0 = p.alpha * __uint_as_float(r[j]);
-                            float x1 = p.alpha * __uint_as_float(r[j + 1]);
-                            if (p.bias != nullptr) {
-                                x0 += __ldg(p.bias + min(col0 + j, last));
-                                x1 += __ldg(p.bias + min(col0 + j + 1, last));
-                            }
+                            float x0 = p.alpha * __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_l, j);
+                            float x1 = p.alpha * __uint_as_float(r[j + 1]) + __shfl_sync(0xffffffffu, bias_l, j + 1);
                             if (p.relu) {
                                 x0 = fmaxf(x0, 0.0f);
                                 x1 = fmaxf(x1, 0.0f);
@@ -263,9 +301,9 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                 }
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0 && box_ok && col0 < p.N) {
+                if (lane < nstore && box_ok && col0 < p.N) {
                     if (kConv)
-                        ptx::tma_store_4d(tmC, stage_buf, col0, sc1, sc2, sc3);
+                        ptx::tma_store_4d(store_map, stage_buf + lane * 512, col0, sc1, sc2, sc3);
                     else
                         ptx::tma_store_2d(tmC, stage_buf, col0, sc1);
                     ptx::tma_store_commit();
@@ -342,7 +380,7 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
         }
     }
     // shared memory must stay alive until the copy engine has drained this warp's last store
-    if (p.tma_store && lane == 0) ptx::tma_store_wait_all<0>();
+    if (p.tma_store && lane < 4) ptx::tma_store_wait_all<0>();
 }
 
 template <bool kConv>
@@ -396,7 +434,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
-        if (lane == 0) {
+        if (ptx::elect_one()) {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -459,7 +497,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        if (ptx::elect_one()) {
             const uint32_t idesc = ptx::make_idesc_bf16_f32(kHalfM, p.bn, p.a_mn_major, p.b_mn_major);
             // K-major: 8-row groups are 1024 B apart (SBO); K advances 32 B inside the swizzle row.
             // MN-major: 64-element groups along MN are one 64 x 64 box (8192 B) apart (LBO),

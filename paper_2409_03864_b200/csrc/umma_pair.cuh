@@ -73,7 +73,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer (one per CTA)
-        if (lane == 0) {
+        if (ptx::elect_one()) {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
@@ -114,7 +114,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
-        if (lane == 0 && rank == 0) {
+        if (rank == 0 && ptx::elect_one()) {
             const uint32_t idesc = ptx::make_idesc_bf16_f32(256, p.bn, p.a_mn_major, p.b_mn_major);
             const uint32_t a_lbo = p.a_mn_major ? 8192u : 16u;
             const uint32_t b_lbo = p.b_mn_major ? 8192u : 16u;

@@ -108,16 +108,21 @@ HALO_CASES = [
     (1, 24, 24, 64, 64, 3, 5, 0),         # no padding, non-square filter
     (1, 7, 7, 256, 256, 3, 3, 1),         # image smaller than a patch
     (1, 33, 17, 64, 72, 1, 3, 1),         # single filter row
+    (5, 9, 12, 64, 32, 3, 3, 1),          # stacked: 10 rows per image, patches straddle up to three images
+    (3, 12, 8, 64, 64, 3, 3, 2),          # padding wider than R - 1 - pad: more output rows than H + pad
+    (4, 20, 16, 64, 64, 5, 3, 0),         # no padding: the rows between images are R - 1 discarded outputs
 ]
 
 
 @pytest.mark.parametrize("case", HALO_CASES)
 @pytest.mark.parametrize("tile_m", [128, 256])
-def test_conv_halo_reuse_vs_oracle(case, tile_m):
-    # the input window of a patch is loaded once per channel chunk and every filter tap reads it from shared memory
+@pytest.mark.parametrize("halo", [2, 3])
+def test_conv_halo_reuse_vs_oracle(case, tile_m, halo):
+    # the input window of a patch is loaded once per channel chunk and every filter tap reads it from shared memory;
+    # halo 3 cuts the patches from the column of all images, so a patch may cover the seam between two images
     N, H, W, Cin, Cout, R, S, pad = case
     x, w, b = si.conv_bf16(N, H, W, Cin, Cout, R, S, seed=80)
-    st, y, ok = run_conv(N, H, W, Cin, Cout, R, S, pad, 1, "bf16", x, w, b, 1, cfg=umma(halo=2, tile_m=tile_m))
+    st, y, ok = run_conv(N, H, W, Cin, Cout, R, S, pad, 1, "bf16", x, w, b, 1, cfg=umma(halo=halo, tile_m=tile_m))
     assert st == 0 and ok, tdx.tdx_last_error()
     err = conv_error(N, H, W, Cin, Cout, R, S, pad, 1, "bf16", x, w, b, 1, y)
     assert err < TOL["bf16"] and err < TIGHT["bf16"], err
@@ -131,6 +136,9 @@ def test_conv_halo_reuse_equals_per_tap_loads_bitwise_for_one_channel_chunk():
     st, y2, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, cfg=umma(halo=2, tile_n=64, stages=2))
     assert st == 0 and ok, tdx.tdx_last_error()
     assert np.array_equal(y1, y2)
+    st, y3, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, cfg=umma(halo=3, tile_n=64, stages=2))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert np.array_equal(y1, y3)
     # a 1 x 1 filter has nothing to reuse: the halo kernel is refused, output untouched
     st, _, untouched = run_conv(N, H, W, Cin, Cout, 1, 1, 0, 1, "bf16", x, si.normal(82, 1, (Cout, 1, 1, Cin), "bf16"), b, 1,
                                 cfg=umma(halo=2))
