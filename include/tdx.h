@@ -83,6 +83,11 @@ typedef struct {
                     /*     (8 x 16 patches, stride 1, more than one tap); 3 = as 2, but the 16-row patches */
                     /*     are cut from the column formed by all images of the batch, H + pad rows apart, so */
                     /*     that an image height that is no multiple of 16 wastes no rows; 0 = choose        */
+    int fit;        /* GEMM, split_k = 1, tile_n >= 192: 2 = some row blocks are cut into narrower tiles    */
+                    /*     (multiples of 64 columns) so that all CTAs finish together when the uniform grid  */
+                    /*     would leave the last wave of CTAs partly idle; 1 = uniform grid; 0 = fitted when  */
+                    /*     the cost model predicts a gain of at least 3 %.  The first call for a shape       */
+                    /*     allocates and uploads a small tile table (make it before any stream capture).     */
 } tdx_config;
 
 /*
@@ -180,6 +185,18 @@ int tdx_enum_conv2d_configs(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_
 int tdx_default_gemm_config(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, tdx_config* out);
 int tdx_default_conv2d_config(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
                               int pad, int stride, int dtype, tdx_config* out);
+
+/*
+ * The tile plan `fit = 2` would use for a GEMM on `ctas` persistent CTAs (host only, no device needed).
+ * It is the counterpart of Case Study 5's divisibility constraints turned around: instead of asking
+ * that the tile divide the problem, some row blocks are cut into narrower tiles so that the tile
+ * count divides evenly over the CTAs.  table (may be NULL) receives up to cap_tiles triples
+ * (row block, first column, width), entry [round * n_ctas + cta]; width 0 = no tile.  n_rounds = 0
+ * means the uniform grid is kept.  model_cycles / model_cycles_uniform are the cost model's longest
+ * CTA for the plan and for the uniform grid.
+ */
+int tdx_gemm_tile_plan(int64_t M, int64_t N, int64_t K, int tile_m, int tile_n, int raster, int ctas, int* table,
+                       int cap_tiles, int* n_rounds, int* n_ctas, double* model_cycles, double* model_cycles_uniform);
 
 /* Persist / restore the tuning cache (a small JSON text file). */
 int tdx_tune_save(const char* json_path);

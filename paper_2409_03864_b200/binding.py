@@ -41,7 +41,7 @@ class TdxError(RuntimeError):
 class tdx_config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in
                 ("kernel", "tile_m", "tile_n", "tile_k", "stages", "cta_pair", "split_k", "store_mode", "raster",
-                 "patch_w", "patch_h", "k_stagger", "halo")]
+                 "patch_w", "patch_h", "k_stagger", "halo", "fit")]
 
     def as_dict(self) -> dict:
         return {n: int(getattr(self, n)) for n, _ in self._fields_}
@@ -83,6 +83,8 @@ def lib() -> ctypes.CDLL:
         L.tdx_tune_save.argtypes = [ctypes.c_char_p]
         L.tdx_tune_load.argtypes = [ctypes.c_char_p]
         L.tdx_tune_clear.argtypes = []
+        dp = ctypes.POINTER(ctypes.c_double)
+        L.tdx_gemm_tile_plan.argtypes = [i64, i64, i64, ci, ci, ci, ci, ip, ci, ip, ip, dp, dp]
         L.tdx_gemm_splitk_static.argtypes = [i64, i64, i64, ci, ci, cf, vp, vp, vp, ci, ci, vp]
         L.tdx_check_device_status.argtypes = [vp]
         L.tdx_selftest_bounded_wait.argtypes = [ci, vp]
@@ -108,7 +110,7 @@ EXPORTS = (
     "tdx_gemm", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_relu_ex",
     "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
     "tdx_enum_conv2d_configs", "tdx_default_gemm_config", "tdx_default_conv2d_config", "tdx_tune_save",
-    "tdx_tune_load", "tdx_tune_clear", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
+    "tdx_tune_load", "tdx_tune_clear", "tdx_gemm_tile_plan", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
     "tdx_version",
 )
 
@@ -252,6 +254,19 @@ def tdx_tune_load(path: str) -> int:
 
 def tdx_tune_clear() -> int:
     return lib().tdx_tune_clear()
+
+
+def tdx_gemm_tile_plan(M, N, K, tile_m=256, tile_n=256, raster=0, ctas=148, cap_tiles=1 << 16):
+    """-> (status, rounds, ctas_used, tiles, model_cycles, model_cycles_uniform); tiles[round][cta] =
+    (row block, first column, width), width 0 = no tile; rounds = 0 when the uniform grid is kept."""
+    table = (ctypes.c_int * (3 * cap_tiles))()
+    rounds, used = ctypes.c_int(0), ctypes.c_int(0)
+    fit, uni = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    st = lib().tdx_gemm_tile_plan(M, N, K, tile_m, tile_n, raster, ctas, table, cap_tiles, ctypes.byref(rounds),
+                                  ctypes.byref(used), ctypes.byref(fit), ctypes.byref(uni))
+    tiles = [[(table[3 * (r * used.value + c)], table[3 * (r * used.value + c) + 1], table[3 * (r * used.value + c) + 2])
+              for c in range(used.value)] for r in range(rounds.value)]
+    return st, rounds.value, used.value, tiles, fit.value, uni.value
 
 
 TDX_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024

@@ -6,12 +6,15 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cmath>
 #include <atomic>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
 #include <map>
+#include <functional>
 #include <mutex>
+#include <queue>
 #include <string>
 #include <vector>
 
@@ -198,12 +201,14 @@ void cfg_to_ints(const tdx_config& c, int* v) {
     v[0] = c.kernel; v[1] = c.tile_m; v[2] = c.tile_n; v[3] = c.tile_k; v[4] = c.stages; v[5] = c.cta_pair;
     v[6] = c.split_k; v[7] = c.store_mode; v[8] = c.raster; v[9] = c.patch_w; v[10] = c.patch_h; v[11] = c.k_stagger;
     v[12] = c.halo;
+    v[13] = c.fit;
 }
 void ints_to_cfg(const int* v, tdx_config* c) {
     c->kernel = v[0]; c->tile_m = v[1]; c->tile_n = v[2]; c->tile_k = v[3]; c->stages = v[4]; c->cta_pair = v[5];
     c->split_k = v[6]; c->store_mode = v[7]; c->raster = v[8]; c->patch_w = v[9]; c->patch_h = v[10];
     c->k_stagger = v[11];
     c->halo = v[12];
+    c->fit = v[13];
 }
 
 // ------------------------------------------------------------------ problem descriptions
@@ -333,6 +338,7 @@ const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num
         if ((c.split_k - 1) * per >= num_kb) return "split_k leaves an empty K slice";
     }
     if (c.raster < 0) return "raster must be >= 0";
+    if (c.fit < 0 || c.fit > 2) return "fit must be 0 (choose), 1 (uniform tiles) or 2 (tile widths fitted to the CTA count)";
     if (c.k_stagger != 0 && c.k_stagger != 1) return "k_stagger must be 0 or 1";
     return nullptr;
 }
@@ -399,12 +405,174 @@ void default_umma_config(int64_t tiles_m, int64_t N, int64_t num_kb, bool b_mn_m
     c->raster = 8;
 }
 
+
+// ------------------------------------------------------------------ tile plan fitted to the number of CTAs
+// A uniform grid of T tiles on G persistent CTAs takes ceil(T / G) tile times although it holds only T / G of
+// work per CTA (the 4096^3 GEMM: 256 tiles of 256 x 256 on 148 CTAs = 1.73 tile times of work done in 2).  The
+// plan keeps the tile height and cuts some row blocks into narrower tiles (widths w < tile_n, both multiples of
+// 64) so that every CTA ends at about the same time: tiles are dealt longest first, each to the CTA with the
+// least work so far.  The cost model is the measured instruction time of one MMA (N / 2 cycles, at least 60)
+// plus a fixed and a per-column epilogue cost.
+struct TilePlan {
+    std::vector<int4> table;   // [round * grid + cta] = (row block, first column, width, 0)
+    int rounds = 0;
+    int grid = 0;
+    double makespan = 0.0;     // model cycles
+    double uniform = 0.0;      // the same for the uniform grid
+};
+
+double tile_cost_cycles(int bm, int width, int64_t num_kb) {
+    const double mma = std::max(width / 2.0, 60.0);
+    return static_cast<double>(num_kb) * 4.0 * (bm / 128) * mma + 1500.0 + 13.0 * width;
+}
+
+// makespan of `na` tiles of cost ca and `nb` tiles of cost cb (ca >= cb > 0), dealt longest first on g CTAs, each
+// to the CTA with the least work so far (closed form of that greedy rule for two sizes)
+double lpt_two_sizes(int64_t na, double ca, int64_t nb, double cb, int g) {
+    const int64_t q = na / g, x = na % g;              // x CTAs hold q + 1 wide tiles, g - x hold q
+    const double low = ca * static_cast<double>(q), high = x > 0 ? low + ca : low;
+    if (nb <= 0) return high;
+    if (x == 0) return low + cb * static_cast<double>(ceil_div(nb, g));
+    // the g - x lighter CTAs take narrow tiles until they have caught up with the others
+    const int64_t catch_up = static_cast<int64_t>(std::ceil(ca / cb - 1e-9));
+    const int64_t lighter = g - x;
+    if (nb <= catch_up * lighter) return std::max(high, low + cb * static_cast<double>(ceil_div(nb, lighter)));
+    const double low2 = low + cb * static_cast<double>(catch_up);      // >= high, by less than cb
+    const int64_t rest = nb - catch_up * lighter;
+    const int64_t f = rest / g, rem = rest % g;
+    if (rem == 0) return low2 + cb * static_cast<double>(f);
+    if (rem <= x) return std::max(low2 + cb * static_cast<double>(f), high + cb * static_cast<double>(f + 1));
+    return low2 + cb * static_cast<double>(f + 1);
+}
+
+// Searches widths and how many row blocks take the narrower cut.  Returns false when nothing beats the uniform grid
+// by `min_gain` (relative).
+bool plan_fitted_tiles(int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int raster, int g, double min_gain,
+                       TilePlan* out) {
+    const int64_t tiles_m = ceil_div(M, bm);
+    const int64_t uniform_tiles = tiles_m * ceil_div(N, bn);
+    const double c_big = tile_cost_cycles(bm, bn, num_kb);
+    const double uniform = lpt_two_sizes(uniform_tiles, c_big, 0, 0.0, g);
+    double best = uniform;
+    int best_w = 0;
+    int64_t best_b = 0, best_b1 = 0, best_e = 0;
+    for (int w = bn - 64; w >= 128; w -= 64) {
+        const double c_small = tile_cost_cycles(bm, w, num_kb);
+        // option b of a row block: b tiles of width w at the high columns, a(b) tiles of width bn before them
+        auto bigs_for = [&](int64_t b) { return ceil_div(std::max<int64_t>(0, N - b * w), bn); };
+        // options that do not carry a tile more than needed
+        std::vector<int64_t> opts;
+        for (int64_t b = 0; b <= ceil_div(N, w); ++b)
+            if (b == 0 || bigs_for(b) * bn + b * w - N < w) opts.push_back(b);
+        for (size_t i = 0; i < opts.size(); ++i)
+        for (size_t j = i + 1; j < opts.size(); ++j) {
+            const int64_t b0 = opts[i], b1 = opts[j];
+            for (int64_t e = 0; e <= tiles_m; ++e) {                            // e row blocks take option b1
+                const int64_t na = (tiles_m - e) * bigs_for(b0) + e * bigs_for(b1);
+                const int64_t nb = (tiles_m - e) * b0 + e * b1;
+                const double m = lpt_two_sizes(na, c_big, nb, c_small, g);
+                if (m < best * (1.0 - 1e-9)) { best = m; best_w = w; best_b = b0; best_b1 = b1; best_e = e; }
+            }
+        }
+    }
+    out->uniform = uniform;
+    out->makespan = best;
+    if (best_w == 0 || best > uniform * (1.0 - min_gain)) return false;
+    // list the tiles: wide ones first, each group in the panel order of the uniform grid (row blocks fastest
+    // inside a panel of `raster` row blocks, then columns, then panels)
+    const int w = best_w;
+    auto bigs_for = [&](int64_t b) { return ceil_div(std::max<int64_t>(0, N - b * w), static_cast<int64_t>(bn)); };
+    struct T { int m, n0, width; };
+    std::vector<T> wide, narrow;
+    const int64_t panel = raster <= 0 ? tiles_m : std::min<int64_t>(raster, tiles_m);
+    for (int64_t m0 = 0; m0 < tiles_m; m0 += panel) {
+        const int64_t rows = std::min(panel, tiles_m - m0);
+        const int64_t max_cols = ceil_div(N, 64) + 1;
+        for (int64_t c = 0; c < max_cols; ++c)          // c-th tile of each row block of the panel
+            for (int64_t r = 0; r < rows; ++r) {
+                const int64_t m = m0 + r;
+                const int64_t b = (m >= tiles_m - best_e) ? best_b1 : best_b;
+                const int64_t a = bigs_for(b);
+                if (c < a) wide.push_back({static_cast<int>(m), static_cast<int>(c * bn), bn});
+                else if (c < a + b) narrow.push_back({static_cast<int>(m), static_cast<int>(a * bn + (c - a) * w), w});
+            }
+    }
+    const int64_t total = static_cast<int64_t>(wide.size() + narrow.size());
+    const int grid = static_cast<int>(std::min<int64_t>(total, g));
+    std::vector<std::vector<T>> per(grid);
+    std::vector<double> load(grid, 0.0);
+    const double c_small = tile_cost_cycles(bm, w, num_kb);
+    auto deal = [&](const std::vector<T>& v, double cost) {
+        for (const T& t : v) {
+            int who = 0;
+            for (int i = 1; i < grid; ++i) if (load[i] < load[who] - 1e-6) who = i;
+            per[who].push_back(t);
+            load[who] += cost;
+        }
+    };
+    deal(wide, c_big);
+    deal(narrow, c_small);
+    size_t rounds = 0;
+    for (auto& v : per) rounds = std::max(rounds, v.size());
+    out->grid = grid;
+    out->rounds = static_cast<int>(rounds);
+    out->table.assign(rounds * grid, make_int4(0, 0, 0, 0));
+    for (int i = 0; i < grid; ++i)
+        for (size_t k = 0; k < per[i].size(); ++k)
+            out->table[k * grid + i] = make_int4(per[i][k].m, per[i][k].n0, per[i][k].width, 0);
+    return true;
+}
+
+// Device copies of tile plans, one per (shape, tile, CTA count); never freed (a few KB each).
+struct PlanKey {
+    int64_t M, N, num_kb;
+    int bm, bn, raster, g, forced;
+    bool operator<(const PlanKey& o) const { return std::memcmp(this, &o, sizeof(PlanKey)) < 0; }
+};
+struct DevicePlan { int4* dev = nullptr; int rounds = 0, grid = 0; bool fitted = false; };
+std::map<PlanKey, DevicePlan> g_plans;
+
+// Looks the plan up (building and uploading it on first use; the upload is ordered on `st` before the kernel).
+int get_tile_plan(DeviceCtx* ctx, int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int raster, double min_gain,
+                  cudaStream_t st, DevicePlan* out) {
+    PlanKey key;
+    std::memset(&key, 0, sizeof key);
+    key.M = M; key.N = N; key.num_kb = num_kb; key.bm = bm; key.bn = bn; key.raster = raster; key.g = ctx->sm_count; key.forced = min_gain <= 0.0 ? 1 : 0;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        auto it = g_plans.find(key);
+        if (it != g_plans.end()) { *out = it->second; return TDX_OK; }
+    }
+    TilePlan plan;
+    DevicePlan d;
+    d.fitted = plan_fitted_tiles(M, N, num_kb, bm, bn, raster, ctx->sm_count, min_gain, &plan);
+    if (d.fitted) {
+        const size_t bytes = plan.table.size() * sizeof(int4);
+        void* dev = nullptr;
+        TDX_CUDA(cudaMalloc(&dev, bytes));
+        // the table is a std::vector about to go out of scope: copy synchronously (once per shape)
+        TDX_CUDA(cudaMemcpy(dev, plan.table.data(), bytes, cudaMemcpyHostToDevice));
+        d.dev = static_cast<int4*>(dev);
+        d.rounds = plan.rounds;
+        d.grid = plan.grid;
+    }
+    (void)st;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        g_plans[key] = d;
+    }
+    *out = d;
+    return TDX_OK;
+}
+
 // ------------------------------------------------------------------ launches
 int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
-                const UmmaParams& p, cudaStream_t st, bool halo = false, const CUtensorMap* ma_row = nullptr,
-                const CUtensorMap* mc_row = nullptr) {
-    const long long items = static_cast<long long>(p.tiles_m) * p.tiles_n * p.split_k;
-    const int grid = static_cast<int>(std::min<long long>(items, ctx->sm_count));
+                const UmmaParams& p_in, cudaStream_t st, bool halo = false, const CUtensorMap* ma_row = nullptr,
+                const CUtensorMap* mc_row = nullptr, int plan_grid = 0) {
+    const long long items = static_cast<long long>(p_in.tiles_m) * p_in.tiles_n * p_in.split_k;
+    UmmaParams p = p_in;
+    if (p.b_box == 0) p.b_box = p.bn;
+    const int grid = p.tiles != nullptr ? plan_grid : static_cast<int>(std::min<long long>(items, ctx->sm_count));
     size_t smem = static_cast<size_t>(p.stages) * ((p.bm + p.bn) * 128) + 1024 +
                   staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
     if (halo)
@@ -511,6 +679,19 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
     }
     if (rc) return rc;
+    // tile widths fitted to the number of CTAs (see plan_fitted_tiles): B then arrives in 64-row copies
+    int plan_grid = 0;
+    if (cfg.fit != 1 && cfg.split_k == 1 && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0) {
+        DevicePlan dp;
+        rc = get_tile_plan(ctx, g.M, g.N, num_kb, cfg.tile_m, cfg.tile_n, cfg.raster, cfg.fit == 2 ? 0.0 : 0.03, st, &dp);
+        if (rc) return rc;
+        if (dp.fitted) {
+            p.tiles = dp.dev;
+            p.rounds = dp.rounds;
+            p.b_box = 64;
+            plan_grid = dp.grid;
+        }
+    }
     if (p.b_mn_major) {
         uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.K)};
         uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
@@ -519,7 +700,7 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     } else {
         uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.N)};
         uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
-        uint32_t box[2] = {64, static_cast<uint32_t>(cfg.tile_n)};
+        uint32_t box[2] = {64, static_cast<uint32_t>(p.tiles ? 64 : cfg.tile_n)};
         rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
     }
     if (rc) return rc;
@@ -533,7 +714,7 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         rc = get_tensor_map(ctx, C, 2, dims, str, box, &mc, 64);
         if (rc) return rc;
     }
-    rc = launch_umma(ctx, false, ma, mb, mc, p, st);
+    rc = launch_umma(ctx, false, ma, mb, mc, p, st, false, nullptr, nullptr, plan_grid);
     if (rc) return rc;
     if (cfg.split_k > 1) {
         const long long MN = static_cast<long long>(g.M) * g.N;
@@ -1098,7 +1279,17 @@ void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int 
                                 c.split_k = sk; c.store_mode = sm; c.raster = raster; c.k_stagger = stagger;
                                 c.patch_w = patch_w; c.patch_h = patch_h;
                                 c.halo = conv ? 1 : 0;
-                                if (umma_config_reason(c, b_mn, num_kb, smem_limit, conv, N, 3, 3) == nullptr) out->push_back(c);
+                                c.fit = conv ? 0 : 1;
+                                if (umma_config_reason(c, b_mn, num_kb, smem_limit, conv, N, 3, 3) != nullptr) continue;
+                                out->push_back(c);
+                                if (!conv && sk == 1 && bn >= 192 && bn % 64 == 0 && stagger == 0) {
+                                    // the same tile with widths fitted to the CTA count, where that changes anything
+                                    TilePlan plan;
+                                    if (plan_fitted_tiles(tiles_m * 128, N, num_kb, tm, bn, raster, sm_count, 0.0, &plan)) {
+                                        c.fit = 2;
+                                        out->push_back(c);
+                                    }
+                                }
                             }
                 }
         }
@@ -1492,10 +1683,10 @@ int tdx_tune_save(const char* json_path) {
     fprintf(f, "{\"version\": 1, \"entries\": [\n");
     size_t i = 0;
     for (const auto& kv : g_tune) {
-        int v[13];
+        int v[14];
         cfg_to_ints(kv.second.cfg, v);
         fprintf(f, "  {\"key\": \"%s\", \"cfg\": [", kv.first.c_str());
-        for (int j = 0; j < 13; ++j) fprintf(f, "%d%s", v[j], j < 12 ? ", " : "");
+        for (int j = 0; j < 14; ++j) fprintf(f, "%d%s", v[j], j < 13 ? ", " : "");
         fprintf(f, "], \"us\": %.3f}%s\n", kv.second.us, ++i < g_tune.size() ? "," : "");
     }
     fprintf(f, "]}\n");
@@ -1521,11 +1712,11 @@ int tdx_tune_load(const char* json_path) {
         const size_t b1 = b0 == std::string::npos ? b0 : text.find(']', b0);
         if (b1 == std::string::npos) return fail(TDX_ERR_INVALID_ARG, "malformed tuning cache %s", json_path);
         const std::string key = text.substr(q0 + 1, q1 - q0 - 1);
-        int v[13] = {0};
+        int v[14] = {0};
         int n = 0;
         const char* s = text.c_str() + b0 + 1;
         const char* end = text.c_str() + b1;
-        while (s < end && n < 13) {
+        while (s < end && n < 14) {
             char* next;
             long val = strtol(s, &next, 10);
             if (next == s) break;
@@ -1533,7 +1724,7 @@ int tdx_tune_load(const char* json_path) {
             s = next;
             while (s < end && (*s == ',' || *s == ' ')) ++s;
         }
-        if (n < 11 || n > 13) return fail(TDX_ERR_INVALID_ARG, "malformed cfg list in %s", json_path);
+        if (n < 11 || n > 14) return fail(TDX_ERR_INVALID_ARG, "malformed cfg list in %s", json_path);
         TuneEntry e;
         ints_to_cfg(v, &e.cfg);
         e.us = 0.0f;
@@ -1546,6 +1737,26 @@ int tdx_tune_load(const char* json_path) {
     }
     std::lock_guard<std::mutex> lk(g_mu);
     for (auto& kv : loaded) g_tune[kv.first] = kv.second;
+    return TDX_OK;
+}
+
+int tdx_gemm_tile_plan(int64_t M, int64_t N, int64_t K, int tile_m, int tile_n, int raster, int ctas, int* table,
+                       int cap_tiles, int* n_rounds, int* n_ctas, double* model_cycles, double* model_cycles_uniform) {
+    if (M <= 0 || N <= 0 || K <= 0 || ctas <= 0 || (tile_m != 128 && tile_m != 256) || tile_n < 192 || tile_n > 256 ||
+        tile_n % 64 || raster < 0)
+        return fail(TDX_ERR_INVALID_ARG, "tdx_gemm_tile_plan: bad argument");
+    TilePlan plan;
+    const bool fitted = plan_fitted_tiles(M, N, ceil_div(K, 64), tile_m, tile_n, raster, ctas, 0.0, &plan);
+    if (model_cycles) *model_cycles = plan.makespan;
+    if (model_cycles_uniform) *model_cycles_uniform = plan.uniform;
+    if (n_rounds) *n_rounds = fitted ? plan.rounds : 0;
+    if (n_ctas) *n_ctas = fitted ? plan.grid : 0;
+    if (fitted && table)
+        for (size_t i = 0; i < plan.table.size() && static_cast<int>(i) < cap_tiles; ++i) {
+            table[3 * i] = plan.table[i].x;
+            table[3 * i + 1] = plan.table[i].y;
+            table[3 * i + 2] = plan.table[i].z;
+        }
     return TDX_OK;
 }
 

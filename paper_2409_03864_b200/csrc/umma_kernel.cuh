@@ -71,6 +71,13 @@ struct UmmaParams {
     int b_resident;           // the whole filter (all chunks and taps, one column tile) stays in shared memory:
                               // loaded once per CTA instead of once per tile, no per-tap handshake
     int epi_warps;            // epilogue warps (0: every warp from the third on)
+    // Tile table (GEMM, optional): instead of a uniform grid of bm x bn tiles, the output is cut into tiles of
+    // bm rows and individually chosen widths (multiples of b_box, at most bn), and the host has already dealt
+    // them to the CTAs: entry [round * gridDim.x + cta] = (row block, first column, width, 0); width 0 ends a
+    // CTA's list.  This is how a tile count that does not fill the last wave of CTAs is evened out.
+    const int4* tiles;
+    int rounds;
+    int b_box;                // rows of one B copy (K-major B); bn when there is no table
     int Pv, H;                // stacked images (Pv > 0): the images of the batch form one column of Nimg * Pv rows,
                               // image n owning rows [n * Pv, n * Pv + P) and the Pv - P rows below it reading as
                               // zero (they are the bottom padding of image n and the top padding of image n + 1);
@@ -117,6 +124,7 @@ __global__ void bounded_wait_selftest_kernel(int* status, long long limit_cycles
 
 struct TileCoord {
     int m_blk, n_blk, kb0, kb1, split;
+    int n0, bn;               // first output column and width of the tile
 };
 
 __device__ __forceinline__ TileCoord decode_item(const UmmaParams& p, int item) {
@@ -132,7 +140,32 @@ __device__ __forceinline__ TileCoord decode_item(const UmmaParams& p, int item) 
     t.m_blk = m_first + (rem - t.n_blk * w);
     t.kb0 = t.split * p.kb_per_split;
     t.kb1 = min(p.num_kb, t.kb0 + p.kb_per_split);
+    t.n0 = t.n_blk * p.bn;
+    t.bn = p.bn;
     return t;
+}
+
+// The `local`-th tile of this CTA: from the tile table when there is one, else item first_item + local * item_stride
+// of the uniform grid.  Returns false when the CTA has no more tiles.
+__device__ __forceinline__ bool get_tile(const UmmaParams& p, int local, int first_item, int item_stride, int total_items,
+                                         TileCoord* t) {
+    if (p.tiles != nullptr) {
+        if (local >= p.rounds) return false;
+        const int4 e = __ldg(p.tiles + static_cast<size_t>(local) * gridDim.x + blockIdx.x);
+        if (e.z == 0) return false;
+        t->m_blk = e.x;
+        t->n_blk = 0;
+        t->n0 = e.y;
+        t->bn = e.z;
+        t->kb0 = 0;
+        t->kb1 = p.num_kb;
+        t->split = 0;
+        return true;
+    }
+    const int item = first_item + local * item_stride;
+    if (item >= total_items) return false;
+    *t = decode_item(p, item);
+    return true;
 }
 
 // Epilogue role (all warps from the third on).  With the staged epilogue there are 16 of them (4 per TMEM
@@ -157,9 +190,8 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
     const int cgrp = (ew >> 2) / mh;              // which share of the columns
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
     const int row_in_tile = half * kHalfM + quarter * 32 + lane;
-    int local = 0;
-    for (int item = first_item; item < total_items; item += item_stride, ++local) {
-        TileCoord t = decode_item(p, item);
+    TileCoord t;
+    for (int local = 0; get_tile(p, local, first_item, item_stride, total_items, &t); ++local) {
         t.m_blk = t.m_blk * m_mul + m_add;
         const int sidx = local * mh + half;
         const int buf = sidx % p.slots;
@@ -254,12 +286,12 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
             uint8_t* my_row = stage_buf + lane * 64;
             const int sw = (lane >> 1) & 3;
             const bool plain = (p.bias == nullptr) && (p.relu == 0);
-            for (int c0 = cgrp * 32; c0 < p.bn; c0 += ncgrp * 32) {
+            for (int c0 = cgrp * 32; c0 < t.bn; c0 += ncgrp * 32) {
                 uint32_t r[32];
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                        static_cast<uint32_t>(buf * p.bn + c0);
                 ptx::tmem_ld_32x32b_x32(taddr, r);
-                const int col0 = t.n_blk * p.bn + c0;
+                const int col0 = t.n0 + c0;
                 // lane l fetches the bias of column col0 + l while the accumulator load is in flight; columns past N
                 // are clipped by the store, the index only has to stay in range
                 float bias_l = 0.0f;
@@ -311,13 +343,13 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                 __syncwarp();
             }
         } else
-        for (int c0 = 0; c0 < p.bn; c0 += 32) {
+        for (int c0 = 0; c0 < t.bn; c0 += 32) {
             uint32_t r[32];
             const uint32_t taddr =
                 tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * p.bn + c0);
             ptx::tmem_ld_32x32b_x32(taddr, r);
             ptx::tmem_ld_wait();
-            const int col0 = t.n_blk * p.bn + c0;
+            const int col0 = t.n0 + c0;
             if (valid && col0 < p.N) {
             if (p.split_k > 1) {
                 float* dst = p.partial + (static_cast<long long>(t.split) * p.M + grow) * p.N + col0;
@@ -438,9 +470,10 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
-                const TileCoord t = decode_item(p, item);
+            TileCoord t;
+            for (int local = 0; ok && get_tile(p, local, blockIdx.x, gridDim.x, total_items, &t); ++local) {
                 const int nkb = t.kb1 - t.kb0;
+                const uint32_t tile_tx = a_bytes + static_cast<uint32_t>(t.bn) * 128u;
                 int kb = t.kb0 + (p.k_stagger ? static_cast<int>((static_cast<long long>(blockIdx.x) * nkb) / gridDim.x) : 0);
                 for (int i = 0; i < nkb; ++i, kb = (kb + 1 == t.kb1) ? t.kb0 : kb + 1) {
                     if (!wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) {
@@ -448,7 +481,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         break;
                     }
                     uint64_t* bar = &full_bar[stage];
-                    ptx::mbar_arrive_expect_tx(bar, stage_bytes);
+                    ptx::mbar_arrive_expect_tx(bar, tile_tx);
                     uint8_t* a_dst = smem + static_cast<size_t>(stage) * stage_bytes;
                     uint8_t* b_dst = a_dst + a_bytes;
                     if (kConv) {
@@ -467,7 +500,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                             ptx::tma_load_4d(a_dst + i * patch_bytes, &tmA, bar, cc * kBK, pw * p.bw + s - p.pad,
                                              ph * p.bh + r - p.pad, n);
                         }
-                        ptx::tma_load_3d(b_dst, &tmB, bar, cc * kBK, tap, t.n_blk * p.bn);
+                        ptx::tma_load_3d(b_dst, &tmB, bar, cc * kBK, tap, t.n0);
                     } else {
                         if (p.a_mn_major) {
                             for (int i = 0; i < 2 * mh; ++i)
@@ -478,10 +511,11 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                                                  t.m_blk * p.bm + h * kHalfM);
                         }
                         if (p.b_mn_major) {
-                            for (int i = 0; i < p.bn / 64; ++i)
-                                ptx::tma_load_2d(b_dst + i * 8192, &tmB, bar, t.n_blk * p.bn + i * 64, kb * kBK);
+                            for (int i = 0; i < t.bn / 64; ++i)
+                                ptx::tma_load_2d(b_dst + i * 8192, &tmB, bar, t.n0 + i * 64, kb * kBK);
                         } else {
-                            ptx::tma_load_2d(b_dst, &tmB, bar, kb * kBK, t.n_blk * p.bn);
+                            for (int r0 = 0; r0 < t.bn; r0 += p.b_box)
+                                ptx::tma_load_2d(b_dst + r0 * 128, &tmB, bar, kb * kBK, t.n0 + r0);
                         }
                     }
                     if (++stage == p.stages) {
@@ -498,7 +532,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (ptx::elect_one()) {
-            const uint32_t idesc = ptx::make_idesc_bf16_f32(kHalfM, p.bn, p.a_mn_major, p.b_mn_major);
+            const uint32_t idesc0 = ptx::make_idesc_bf16_f32(kHalfM, p.bn, p.a_mn_major, p.b_mn_major);
             // K-major: 8-row groups are 1024 B apart (SBO); K advances 32 B inside the swizzle row.
             // MN-major: 64-element groups along MN are one 64 x 64 box (8192 B) apart (LBO),
             //           8-k groups are 1024 B apart (SBO); K advances 16 rows = 2048 B.
@@ -515,10 +549,11 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             uint64_t a_desc = a_desc0, b_desc = b_desc0;       // descriptors of the current stage
             int stage = 0;
             uint32_t phase = 0;
-            int local = 0;
             bool ok = true;
-            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++local) {
-                const TileCoord t = decode_item(p, item);
+            TileCoord t;
+            for (int local = 0; ok && get_tile(p, local, blockIdx.x, gridDim.x, total_items, &t); ++local) {
+                // N field of the instruction descriptor (bits 17..22) follows the tile's width
+                const uint32_t idesc = (idesc0 & ~(0x3Fu << 17)) | (static_cast<uint32_t>(t.bn >> 3) << 17);
                 // accumulator slots of this tile: use number u of slot s has barrier phase (u & 1)
                 uint32_t d_tmem[2] = {0u, 0u};
                 int slot[2] = {0, 0};

@@ -55,6 +55,8 @@ def tune_one(spec, iters):
 
 def brief(c):
     s = f"{'pair ' if c['cta_pair'] == 2 else ''}m{c['tile_m']} n{c['tile_n']} st{c['stages']} sk{c['split_k']} r{c['raster']} ks{c['k_stagger']} sm{c['store_mode']}"
+    if c.get("fit"):
+        s += f" fit{c['fit']}"
     if c["patch_w"]:
         s += f" p{c['patch_w']}x{c['patch_h']} h{c['halo']}"
     return s

@@ -184,6 +184,49 @@ def test_default_configs():
     assert st == tdx.TDX_OK and c.halo in (1, 2, 3) and c.stages >= 2
 
 
+@pytest.mark.parametrize("shape", [(4096, 4096, 4096), (4096, 4096, 512), (2048, 3072, 1024), (1000, 2000, 512),
+                                   (5000, 3000, 256), (256, 640, 64), (8192, 8192, 8192)])
+@pytest.mark.parametrize("tile", [(256, 256), (128, 256), (256, 192)])
+def test_fitted_tile_plan_covers_the_output_once_and_balances_the_ctas(shape, tile):
+    # host logic of fit = 2: every row block's columns are covered exactly once by tiles whose widths are multiples
+    # of 64 and at most tile_n; each CTA's list is dense; the model's longest CTA is never worse than the uniform grid
+    M, N, K = shape
+    tm, tn = tile
+    ctas = 148
+    st, rounds, used, tiles, fit, uni = tdx.tdx_gemm_tile_plan(M, N, K, tm, tn, 2, ctas)
+    assert st == tdx.TDX_OK
+    assert fit <= uni * (1 + 1e-12)
+    if rounds == 0:
+        assert fit == uni                       # uniform grid kept
+        return
+    assert 1 <= used <= ctas
+    cover = {}
+    for cta in range(used):
+        ended = False
+        for r in range(rounds):
+            m, n0, w = tiles[r][cta]
+            if w == 0:
+                ended = True
+                continue
+            assert not ended, "a CTA's tile list must not have holes"
+            assert w % 64 == 0 and 128 <= w <= tn and n0 % 64 == 0 and 0 <= m < -(-M // tm)
+            cover.setdefault(m, []).append((n0, w))
+    assert sorted(cover) == list(range(-(-M // tm)))
+    for m, segs in cover.items():
+        segs.sort()
+        pos = 0
+        for n0, w in segs:
+            assert n0 == pos, (m, segs)
+            pos += w
+        assert N <= pos < N + tn
+    per_cta = [sum(tiles[r][c][2] for r in range(rounds)) for c in range(used)]
+    assert max(per_cta) - min(per_cta) <= tn     # column-weighted load differs by at most one wide tile
+    if shape == (4096, 4096, 4096) and tile == (256, 256):
+        # 256 uniform tiles on 148 CTAs take two tile times; 148 wide + 144 tiles of 192 columns take 1.75
+        widths = sorted(t[2] for row in tiles for t in row if t[2])
+        assert widths.count(256) == 148 and widths.count(192) == 144 and fit < 0.9 * uni
+
+
 def test_tuning_cache_round_trip(tmp_path):
     path = tmp_path / "cache.json"
     path.write_text('{"version": 1, "entries": [\n  {"key": "gemm:640:640:640:0:1:1", '
@@ -194,7 +237,7 @@ def test_tuning_cache_round_trip(tmp_path):
     assert st == tdx.TDX_OK and (c.tile_n, c.stages, c.split_k, c.raster) == (64, 3, 2, 2)
     out = tmp_path / "out.json"
     assert tdx.tdx_tune_save(str(out)) == tdx.TDX_OK
-    assert "gemm:640:640:640:0:1:1" in out.read_text() and "[1, 128, 64, 64, 3, 1, 2, 1, 2, 0, 0, 0, 0]" in out.read_text()
+    assert "gemm:640:640:640:0:1:1" in out.read_text() and "[1, 128, 64, 64, 3, 1, 2, 1, 2, 0, 0, 0, 0, 0]" in out.read_text()
     assert tdx.tdx_tune_clear() == tdx.TDX_OK
     st, c = tdx.tdx_default_gemm_config(640, 640, 640, 0, 1, tdx.TDX_BF16)
     assert c.tile_n != 64 or c.split_k != 2

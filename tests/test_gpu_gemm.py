@@ -108,6 +108,35 @@ def test_umma_256_row_tiles(cfgkw, transA, transB):
     assert err < TIGHT["bf16"], err
 
 
+@pytest.mark.parametrize("transA,transB", [(0, 1), (0, 0), (1, 1), (1, 0)])
+@pytest.mark.parametrize("tile_m", [256, 128])
+def test_umma_tile_widths_fitted_to_the_cta_count(tile_m, transA, transB):
+    # fit = 2: 256- and 192-column tiles from a host-made table, B arriving in 64-row copies; ragged M, N and K tails
+    M, N, K = 3304, 2840, 200
+    A, B = si.gemm_bf16_normal(M, N, K, seed=64, transA=transA, transB=transB)
+    _, rounds, _, _, _, _ = tdx.tdx_gemm_tile_plan(M, N, K, tile_m, 256, 2, torch.cuda.get_device_properties(0).multi_processor_count)
+    assert rounds > 0, "this shape is meant to get a fitted plan"
+    st, C, ok = run_gemm(M, N, K, transA, transB, -1.0, "bf16", A, B, cfg=umma(tile_m=tile_m, tile_n=256, raster=2, fit=2))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    err = gemm_error(M, N, K, transA, transB, -1.0, "bf16", A, B, C)
+    assert err < TIGHT["bf16"], err
+    # same bits as the uniform grid: the reduction order inside an output element does not depend on the tile width
+    st, C1, ok = run_gemm(M, N, K, transA, transB, -1.0, "bf16", A, B, cfg=umma(tile_m=tile_m, tile_n=256, raster=2, fit=1))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert np.array_equal(C, C1)
+
+
+def test_umma_fitted_tiles_exact_integers_and_direct_stores():
+    M, N, K = 256 * 9, 64 * 37, 192
+    A = si.small_integers(65, 0, (M, K), "bf16", -1, 1)
+    B = si.small_integers(65, 1, (N, K), "bf16", -1, 1)
+    ref = oracle.gemm(M, N, K, 0, 1, 1.0, "bf16", A, B)
+    for sm in (1, 2):
+        st, C, ok = run_gemm(M, N, K, 0, 1, 1.0, "bf16", A, B, cfg=umma(tile_m=256, tile_n=256, fit=2, store_mode=sm))
+        assert st == 0 and ok, tdx.tdx_last_error()
+        assert np.array_equal(oracle.decode(C, "bf16"), ref), sm
+
+
 def test_umma_256_row_tiles_exact_integers_many_tiles_per_cta():
     # more tiles than SMs, so every CTA walks several tiles and the accumulator slots wrap around
     M, N, K = 256 * 20, 64 * 16, 128
