@@ -47,6 +47,9 @@ def _load():
         lib.oracle_gemm.argtypes = [i64, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_double,
                                     ctypes.c_int, p, p, p, i64, p]
         lib.oracle_gemm.restype = ctypes.c_int
+        lib.oracle_gemm_batched.argtypes = [i64, i64, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_double,
+                                            ctypes.c_double, ctypes.c_int, p, i64, p, i64, p, i64, p]
+        lib.oracle_gemm_batched.restype = ctypes.c_int
         lib.oracle_conv2d.argtypes = [i64] * 9 + [ctypes.c_int, p, p, p, ctypes.c_int, p, i64, p]
         lib.oracle_conv2d.restype = ctypes.c_int
         lib.oracle_conv_out_dim.argtypes = [i64] * 4
@@ -96,6 +99,40 @@ def gemm(M, N, K, transA, transB, alpha, dtype, A, B, rows=None) -> np.ndarray:
     return out
 
 
+def gemm_batched(batch, M, N, K, transA, transB, alpha, beta, dtype, A, B, C=None, strideA=None, strideB=None,
+                 strideC=None) -> np.ndarray:
+    """fp64 reference of C[b] = beta * C[b] + alpha * op(A[b]) . op(B[b]); returns batch x M x N doubles.
+
+    Strides are in elements and default to the dense ones (M*K, K*N, M*N); C is only read when beta != 0.
+    """
+    lib, dt = _load(), _DT[dtype]
+    sa = M * K if strideA is None else strideA
+    sb = K * N if strideB is None else strideB
+    sc = M * N if strideC is None else strideC
+    need = lambda stride, dense: (batch - 1) * stride + dense if batch > 0 else 0   # noqa: E731
+    want = np.float32 if dt == F32 else np.uint16
+    A = np.ascontiguousarray(A)
+    B = np.ascontiguousarray(B)
+    if A.dtype != want or B.dtype != want:
+        raise TypeError(f"expected {want.__name__} storage")
+    if A.size < need(sa, M * K) or B.size < need(sb, K * N):
+        raise ValueError("operand smaller than its strides imply")
+    cp = None
+    if beta != 0.0:
+        if C is None:
+            raise ValueError("beta != 0 needs C")
+        C = np.ascontiguousarray(C)
+        if C.dtype != want or C.size < need(sc, M * N):
+            raise ValueError("bad C")
+        cp = C.ctypes.data
+    out = np.empty((batch, M, N), dtype=np.float64)
+    rc = lib.oracle_gemm_batched(batch, M, N, K, int(transA), int(transB), float(alpha), float(beta), dt,
+                                 A.ctypes.data, sa, B.ctypes.data, sb, cp, sc, out.ctypes.data)
+    if rc:
+        raise RuntimeError(f"oracle_gemm_batched failed ({rc})")
+    return out
+
+
 def conv_out_dim(H, R, pad, stride) -> int:
     return int(_load().oracle_conv_out_dim(H, R, pad, stride))
 
@@ -133,4 +170,4 @@ def round_bf16(v: np.ndarray) -> np.ndarray:
     return out
 
 
-from .metric import (decode, gemm_row_scales, conv_row_scales, max_normalised_error)  # noqa: E402,F401
+from .metric import (decode, gemm_row_scales, gemm_batched_row_scales, conv_row_scales, max_normalised_error)  # noqa: E402,F401

@@ -5,6 +5,7 @@ A result C^ is compared with the fp64 reference C per output row i:
     err = max_i max_j |C^[i,j] - C[i,j]| / scale_i
 
 GEMM:  scale_i = |alpha| * ||Aop(i,:)||_2 * max_j ||Bop(:,j)||_2
+batched GEMM with accumulate: scale_(b,i) = the GEMM scale of batch b + |beta| * max_j |C_in[b,i,j]|
 conv:  scale_i = ||patch_i||_2 * max_k ||w_k||_2 + max_k |bias_k|
        (patch_i = the R*S*Cin input window of output pixel i, zero taps included;
         ReLU is 1-Lipschitz so the same bound carries through it)
@@ -33,6 +34,19 @@ def gemm_row_scales(M, N, K, transA, transB, alpha, dtype, A, B, rows=None) -> n
     bmax = b_norm.max() if b_norm.size else 0.0
     s = abs(float(alpha)) * a_norm * bmax
     return s if rows is None else s[np.asarray(rows, dtype=np.int64)]
+
+
+def gemm_batched_row_scales(batch, M, N, K, transA, transB, alpha, beta, dtype, A, B, C=None) -> np.ndarray:
+    """Scales of the batch * M output rows of a dense batched GEMM (row b*M + i), accumulate term included."""
+    a = decode(A, dtype).reshape((batch, K, M) if transA else (batch, M, K))
+    b = decode(B, dtype).reshape((batch, N, K) if transB else (batch, K, N))
+    a_norm = np.sqrt((a * a).sum(axis=1 if transA else 2))          # batch x M
+    b_norm = np.sqrt((b * b).sum(axis=2 if transB else 1))          # batch x N
+    bmax = b_norm.max(axis=1, keepdims=True) if N else np.zeros((batch, 1))
+    s = abs(float(alpha)) * a_norm * bmax
+    if beta != 0.0 and C is not None:
+        s = s + abs(float(beta)) * np.abs(decode(C, dtype).reshape(batch, M, N)).max(axis=2)
+    return s.reshape(-1)
 
 
 def conv_row_scales(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, rows=None) -> np.ndarray:

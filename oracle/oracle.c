@@ -6,7 +6,7 @@
  * What it computes is the plain definition, written out:
  *   - GEMM: the (batch-)matmul loop nest of the paper's Case Study 4 (the
  *     OpenMP tiling figure), without the batch loop and overwriting instead of
- *     accumulating, with the operand transposes that the `matmul_of_transpose`
+ *     accumulating (oracle_gemm), and with both (oracle_gemm_batched), with the operand transposes that the `matmul_of_transpose`
  *     pattern of Case Study 3 folds into the matmul expressed as index maps,
  *     and the negate of `negate_of_transpose` expressed as alpha = -1.
  *   - conv2d + bias + ReLU: cross-correlation over a zero-padded NHWC input
@@ -90,6 +90,41 @@ int oracle_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, double 
                     c[j] += a * load_elem(B, k * N + j, dtype);
             }
             for (int64_t j = 0; j < N; ++j) c[j] = alpha * c[j];
+        }
+    }
+    return 0;
+}
+
+/*
+ * The batch-matmul loop nest of the paper's Case Study 4 (the OpenMP tiling figure) as it is printed, with the
+ * accumulate:  C[b,i,j] += A[b,i,k] * B[b,k,j],  generalised by two scalars and the operand transposes:
+ *   C_ref[b,i,j] = beta * C_in[b,i,j] + alpha * sum_{k<K} Aop(b,i,k) * Bop(b,k,j)
+ *   Aop(b,i,k) = transA ? A[b*strideA + k*M + i] : A[b*strideA + i*K + k]
+ *   Bop(b,k,j) = transB ? B[b*strideB + j*K + k] : B[b*strideB + k*N + j]
+ *   C_in[b,i,j] = C[b*strideC + i*N + j]   (same storage type as A and B; not read when beta == 0)
+ * (alpha = beta = 1 is the paper's nest).  Strides are in elements.  out: batch x M x N doubles, dense.
+ */
+int oracle_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int transA, int transB,
+                        double alpha, double beta, int dtype,
+                        const void *A, int64_t strideA, const void *B, int64_t strideB,
+                        const void *C, int64_t strideC, double *out)
+{
+    if (batch < 0 || M < 0 || N < 0 || K < 0) return 1;
+    if (beta != 0.0 && C == NULL) return 2;
+#pragma omp parallel for collapse(2) schedule(dynamic, 1)
+    for (int64_t b = 0; b < batch; ++b) {
+        for (int64_t i = 0; i < M; ++i) {
+            for (int64_t j = 0; j < N; ++j) {
+                double acc = 0.0;
+                for (int64_t k = 0; k < K; ++k) {
+                    double a = load_elem(A, b * strideA + (transA ? k * M + i : i * K + k), dtype);
+                    double bb = load_elem(B, b * strideB + (transB ? j * K + k : k * N + j), dtype);
+                    acc += a * bb;
+                }
+                double r = alpha * acc;
+                if (beta != 0.0) r += beta * load_elem(C, b * strideC + i * N + j, dtype);
+                out[(b * M + i) * N + j] = r;
+            }
         }
     }
     return 0;

@@ -118,6 +118,67 @@ def test_gemm_empty_reduction_gives_zero():
     assert np.array_equal(out, np.zeros((3, 2)))
 
 
+# --------------------------------------------------------------------- batch-matmul with accumulate
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_gemm_batched_hand_computed_literals(dtype):
+    g = read_golden("gemm_batched_2x2x2x2.txt")
+    enc = f32 if dtype == "f32" else bf
+    A, B, Cin = enc(g["A"]), enc(g["B"]), enc(g["Cin"])
+    out = oracle.gemm_batched(2, 2, 2, 2, 0, 0, 1.0, 1.0, dtype, A, B, Cin)       # the paper's nest: C += A . B
+    assert np.array_equal(out.ravel(), np.array(g["C11"]))
+    out = oracle.gemm_batched(2, 2, 2, 2, 0, 0, 2.0, -1.0, dtype, A, B, Cin)
+    assert np.array_equal(out.ravel(), np.array(g["C2m1"]))
+
+
+@pytest.mark.parametrize("transA,transB", [(0, 0), (0, 1), (1, 0), (1, 1)])
+def test_gemm_batched_exact_integers_vs_library_einsum_with_gapped_strides(transA, transB):
+    # small integers: exact in fp64, so the oracle must equal numpy's batched product bit for bit; the batches are
+    # laid out with gaps (stride > dense size) filled with NaN, which a wrong stride or index map would pull in
+    rng = np.random.default_rng(5)
+    batch, M, N, K = 3, 5, 4, 7
+    A = rng.integers(-4, 5, (batch, M, K)).astype(np.float64)
+    B = rng.integers(-4, 5, (batch, K, N)).astype(np.float64)
+    C = rng.integers(-9, 10, (batch, M, N)).astype(np.float64)
+    sa, sb, sc = M * K + 3, K * N + 5, M * N + 2
+
+    def lay(x, stride, transposed):
+        buf = np.full(batch * stride, np.nan, dtype=np.float32)
+        for b in range(batch):
+            v = (x[b].T if transposed else x[b]).ravel()
+            buf[b * stride: b * stride + v.size] = v
+        return buf
+
+    out = oracle.gemm_batched(batch, M, N, K, transA, transB, 3.0, -2.0, "f32", lay(A, sa, transA), lay(B, sb, transB),
+                              lay(C, sc, False), strideA=sa, strideB=sb, strideC=sc)
+    assert np.array_equal(out, 3.0 * np.einsum("bik,bkj->bij", A, B) - 2.0 * C)
+
+
+def test_gemm_batched_closed_forms_and_special_cases():
+    batch, M, N, K = 4, 3, 5, 11
+    ones = lambda *sh: f32(np.ones(sh))                                    # noqa: E731
+    # all-ones operands and C: every entry = alpha K + beta
+    out = oracle.gemm_batched(batch, M, N, K, 0, 0, 0.5, 3.0, "f32", ones(batch, M, K), ones(batch, K, N), ones(batch, M, N))
+    assert np.array_equal(out, np.full((batch, M, N), 0.5 * K + 3.0))
+    # zero A: the result is beta C;  beta = 0: C is not read (NaNs in it do not matter, and it may be absent)
+    Cin = si.uniform(12, 2, (batch, M, N), "f32")
+    out = oracle.gemm_batched(batch, M, N, K, 0, 0, 1.0, -1.5, "f32", f32(np.zeros((batch, M, K))), ones(batch, K, N), Cin)
+    assert np.array_equal(out, -1.5 * Cin.astype(np.float64))
+    A, B = si.uniform(12, 0, (batch, M, K), "f32"), si.uniform(12, 1, (batch, K, N), "f32")
+    nan_c = f32(np.full((batch, M, N), np.nan))
+    out0 = oracle.gemm_batched(batch, M, N, K, 0, 0, 1.0, 0.0, "f32", A, B, nan_c)
+    assert np.array_equal(out0, oracle.gemm_batched(batch, M, N, K, 0, 0, 1.0, 0.0, "f32", A, B))
+    # each batch of the batched call is the single-matrix definition (pinned above) on that batch's operands
+    for b in range(batch):
+        assert np.array_equal(out0[b], oracle.gemm(M, N, K, 0, 0, 1.0, "f32", A[b], B[b]))
+    # accumulating twice from zero doubles the product (integers: exact)
+    Ai = f32(np.random.default_rng(6).integers(-3, 4, (batch, M, K)))
+    Bi = f32(np.random.default_rng(7).integers(-3, 4, (batch, K, N)))
+    once = oracle.gemm_batched(batch, M, N, K, 0, 0, 1.0, 1.0, "f32", Ai, Bi, f32(np.zeros((batch, M, N))))
+    twice = oracle.gemm_batched(batch, M, N, K, 0, 0, 1.0, 1.0, "f32", Ai, Bi, f32(once))
+    assert np.array_equal(twice, 2.0 * once)
+
+
 # --------------------------------------------------------------------- conv
 
 def test_conv_hand_computed_literals():
