@@ -60,6 +60,9 @@ WORKLOADS = {
                 label="gemm_bf16_8192x128x8192"),
     "c5e": dict(kind="gemm", dtype="bf16", M=4096, N=4096, K=512, tA=0, tB=0, alpha=1.0, seed=4, bound="tensor",
                 label="gemm_bf16_4096x4096x512"),
+    # the paper's own workload (Case Study 4): C[b,i,j] += A[b,i,k] * B[b,k,j], b < 6, i < 196, j < 256, k < 2305
+    "cs4": dict(kind="gemm_batched", dtype="f32", batch=6, M=196, N=256, K=2305, tA=0, tB=0, alpha=1.0, beta=1.0, seed=5,
+                bound="alu", label="batch_matmul_accumulate_f32_6x196x256x2305"),
 }
 
 
@@ -69,7 +72,15 @@ class Workload:
     def __init__(self, name):
         self.name, self.w = name, WORKLOADS[name]
         w = self.w
-        if w["kind"] == "gemm":
+        if w["kind"] == "gemm_batched":
+            self.el = 4 if w["dtype"] == "f32" else 2
+            self.flops = 2.0 * w["batch"] * w["M"] * w["N"] * w["K"]
+            self.in_bytes = w["batch"] * (w["M"] * w["K"] + w["K"] * w["N"] + w["M"] * w["N"]) * self.el   # A, B and C read
+            self.out_bytes = w["batch"] * w["M"] * w["N"] * self.el
+            self.rows = w["batch"]            # the oracle sample is taken in whole batches
+            self.unit = "batches"
+
+        elif w["kind"] == "gemm":
             self.el = 4 if w["dtype"] == "f32" else 2
             self.flops = 2.0 * w["M"] * w["N"] * w["K"]
             self.in_bytes = (w["M"] * w["K"] + w["K"] * w["N"]) * self.el
@@ -83,12 +94,18 @@ class Workload:
             self.flops = 2.0 * self.rows * w["Cout"] * w["R"] * w["S"] * w["Cin"]
             self.in_bytes = (w["N"] * w["H"] * w["W"] * w["Cin"] + w["Cout"] * w["R"] * w["S"] * w["Cin"]) * 2 + w["Cout"] * 4
             self.out_bytes = self.rows * w["Cout"] * 2
+        self.unit = getattr(self, "unit", "output rows (all columns)")
         self.algo_bytes = self.in_bytes + self.out_bytes       # each operand read once, the output written once
         self.dtype = w.get("dtype", "bf16")
 
     def host_inputs(self):
         import seeded_inputs as si
         w = self.w
+        if w["kind"] == "gemm_batched":
+            gen = si.uniform if w["dtype"] == "f32" else si.normal
+            return (gen(w["seed"], 0, (w["batch"], w["M"], w["K"]), w["dtype"]),
+                    gen(w["seed"], 1, (w["batch"], w["K"], w["N"]), w["dtype"]),
+                    gen(w["seed"], 2, (w["batch"], w["M"], w["N"]), w["dtype"]))
         if w["kind"] == "gemm":
             if w["dtype"] == "f32":
                 return si.gemm_f32_uniform(w["M"], w["N"], w["K"], seed=w["seed"])
@@ -101,6 +118,10 @@ class Workload:
     def oracle_rows(self, host, rows):
         import oracle
         w = self.w
+        if w["kind"] == "gemm_batched":      # rows = batch indices
+            import numpy as np
+            return np.stack([oracle.gemm_batched(1, w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], w["beta"], w["dtype"],
+                                                 host[0][b], host[1][b], host[2][b])[0] for b in rows])
         if w["kind"] == "gemm":
             return oracle.gemm(w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], w["dtype"], host[0], host[1], rows=rows)
         return oracle.conv2d(w["N"], w["H"], w["W"], w["Cin"], w["Cout"], w["R"], w["S"], w["pad"], w["stride"], "bf16",
@@ -202,7 +223,7 @@ def oracle_sample(wl, host, target_seconds=12.0):
     wl.oracle_rows(host, rows)
     t = time.perf_counter() - t0
     return (wl.flops_for_rows(n_rows) / t / 1e12, oracle.num_threads(),
-            f"{n_rows} of {wl.rows} output rows (all columns), {t:.1f} s")
+            f"{n_rows} of {wl.rows} {wl.unit}, {t:.1f} s")
 
 
 def run_reference(args):
@@ -230,7 +251,7 @@ def run_reference(args):
         wl.oracle_rows(host, rows)
     t = time.perf_counter() - t0
     value = wl.flops_for_rows(rows_per_step) * args.steps / t / 1e12
-    sample = f"each step = {rows_per_step} of {wl.rows} output rows (all columns) of the workload"
+    sample = f"each step = {rows_per_step} of {wl.rows} {wl.unit} of the workload"
     cfg = dict(wl.config_dict(), workload=wl.w["label"], sample=sample)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
@@ -284,7 +305,21 @@ def run_tdx(args):
     sets = [([h.cuda(non_blocking=True) for h in h_in], torch.empty_like(h_out, device="cuda")) for _ in range(n_sets)]
     stream = torch.cuda.current_stream()
     DT = tdx.TDX_F32 if wl.dtype == "f32" else tdx.TDX_BF16
-    if w["kind"] == "gemm":
+    if w["kind"] == "gemm_batched":
+        st_cfg, cfg = 1, None
+        # the step accumulates into C (beta = 1); each buffer set carries its own copy of C, and the output IS that buffer
+        sets = [(ins, ins[2]) for ins, _ in sets]
+
+        def launch(ins, out):
+            return tdx.tdx_gemm_batched(w["batch"], w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], w["beta"], DT,
+                                        ins[0], ins[1], out, stream=stream)
+
+        def launch_host():
+            h_out.copy_(h_in[2].reshape(-1))
+            return tdx.tdx_gemm_batched_host(w["batch"], w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], w["beta"], DT,
+                                             h_in[0], h_in[1], h_out, stream)
+        kernel_name = "sgemm_tiled_kernel / sgemm_small_kernel (fp32 CUDA cores)"
+    elif w["kind"] == "gemm":
         st_cfg, cfg = tdx.tdx_default_gemm_config(w["M"], w["N"], w["K"], w["tA"], w["tB"], DT)
 
         def launch(ins, out):

@@ -111,6 +111,22 @@ int tdx_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, float alph
              const void* A, const void* B, void* C, void* stream);
 
 /*
+ * Batch-matmul with accumulate: C[b] = beta * C[b] + alpha * op(A[b]) . op(B[b]),  b < batch.
+ *
+ * With alpha = beta = 1 this is the loop nest of the paper's Case Study 4 exactly as printed
+ * (C[b,i,j] += A[b,i,k] * B[b,k,j]; its workload is batch 6, M 196, N 256, K 2305).  Layouts per batch
+ * as for tdx_gemm; batch b of an operand starts strideX elements after batch b - 1 (strideA or strideB
+ * may be 0: the operand is shared by all batches; strideC >= M * N).  C is read only when beta != 0 and
+ * must not alias A or B.  fp32 runs on the CUDA cores (any shape); bf16 runs on the tensor cores when
+ * every batch's operands meet the 16-byte rules of tdx_gemm (contiguous dims and batch strides multiples
+ * of 8 elements, 16-byte aligned bases) and otherwise -- K = 2305 is such a case -- on the generic GPU
+ * kernel.  batch, M or N = 0: no-op.  K = 0: C = beta * C.  Errors as for tdx_gemm.
+ */
+int tdx_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, float beta,
+                     int dtype, const void* A, int64_t strideA, const void* B, int64_t strideB, void* C, int64_t strideC,
+                     void* stream);
+
+/*
  * Same as tdx_gemm with an explicit configuration and caller-owned split-K workspace.
  * cfg = NULL or cfg->split_k = 0: the library chooses split_k (tuning cache, else heuristic); then
  * `workspace` may be NULL and the library uses an internal, lazily grown buffer.  With an explicit
@@ -155,6 +171,9 @@ int tdx_conv2d_bias_relu_ex(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_
  */
 int tdx_gemm_host(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype,
                   const void* A_host, const void* B_host, void* C_host, void* stream);
+/* tdx_gemm_batched on dense host buffers (strides M*K, K*N, M*N); C_host is copied in only when beta != 0. */
+int tdx_gemm_batched_host(int64_t batch, int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha,
+                          float beta, int dtype, const void* A_host, const void* B_host, void* C_host, void* stream);
 int tdx_conv2d_bias_relu_host(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
                               int pad, int stride, int dtype, const void* x_host, const void* w_host,
                               const float* bias_host, int relu, void* y_host, void* stream);

@@ -69,6 +69,8 @@ def lib() -> ctypes.CDLL:
         conv_args = [i64] * 7 + [ci, ci, ci, vp, vp, vp, ci, vp, vp]
         L.tdx_gemm.argtypes = gemm_args
         L.tdx_gemm_ex.argtypes = gemm_args + [cfgp, vp, sz]
+        L.tdx_gemm_batched.argtypes = [i64, i64, i64, i64, ci, ci, cf, cf, ci, vp, i64, vp, i64, vp, i64, vp]
+        L.tdx_gemm_batched_host.argtypes = [i64, i64, i64, i64, ci, ci, cf, cf, ci, vp, vp, vp, vp]
         L.tdx_gemm_workspace_size.argtypes = [i64, i64, i64, ci, cfgp, ctypes.POINTER(sz)]
         L.tdx_conv2d_bias_relu.argtypes = conv_args
         L.tdx_conv2d_bias_relu_ex.argtypes = conv_args + [cfgp]
@@ -107,7 +109,7 @@ def lib() -> ctypes.CDLL:
 
 # every symbol include/tdx.h declares
 EXPORTS = (
-    "tdx_gemm", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_relu_ex",
+    "tdx_gemm", "tdx_gemm_batched", "tdx_gemm_batched_host", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_relu_ex",
     "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
     "tdx_enum_conv2d_configs", "tdx_default_gemm_config", "tdx_default_conv2d_config", "tdx_tune_save",
     "tdx_tune_load", "tdx_tune_clear", "tdx_gemm_tile_plan", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
@@ -161,6 +163,22 @@ def tdx_gemm_ex(M, N, K, transA, transB, alpha, dtype, A, B, C, stream=None, cfg
                 workspace_bytes=0) -> int:
     return lib().tdx_gemm_ex(M, N, K, transA, transB, alpha, dtype, _ptr(A), _ptr(B), _ptr(C), _stream(stream),
                              _cfg(cfg), _ptr(workspace), workspace_bytes)
+
+
+def tdx_gemm_batched(batch, M, N, K, transA, transB, alpha, beta, dtype, A, B, C, strideA=None, strideB=None,
+                     strideC=None, stream=None) -> int:
+    """C[b] = beta * C[b] + alpha * op(A[b]) . op(B[b]); strides in elements, dense by default."""
+    sa = M * K if strideA is None else strideA
+    sb = K * N if strideB is None else strideB
+    sc = M * N if strideC is None else strideC
+    return lib().tdx_gemm_batched(batch, M, N, K, transA, transB, alpha, beta, dtype, _ptr(A), sa, _ptr(B), sb, _ptr(C),
+                                  sc, _stream(stream))
+
+
+def tdx_gemm_batched_host(batch, M, N, K, transA, transB, alpha, beta, dtype, A, B, C, stream=None) -> int:
+    """A, B, C are dense host arrays (numpy, or pinned torch CPU tensors)."""
+    return lib().tdx_gemm_batched_host(batch, M, N, K, transA, transB, alpha, beta, dtype, _ptr(A), _ptr(B), _ptr(C),
+                                       _stream(stream))
 
 
 def tdx_gemm_workspace_size(M, N, K, dtype, cfg):

@@ -12,6 +12,8 @@ __device__ __forceinline__ float ld_as_float(const float* p, long long i) { retu
 __device__ __forceinline__ float ld_as_float(const __nv_bfloat16* p, long long i) {
     return __bfloat162float(p[i]);
 }
+__device__ __forceinline__ float as_float(float v) { return v; }
+__device__ __forceinline__ float as_float(__nv_bfloat16 v) { return __bfloat162float(v); }
 __device__ __forceinline__ void st_from_float(float* p, long long i, float v) { p[i] = v; }
 __device__ __forceinline__ void st_from_float(__nv_bfloat16* p, long long i, float v) {
     p[i] = __float2bfloat16_rn(v);
@@ -25,8 +27,13 @@ __device__ __forceinline__ void st_from_float(__nv_bfloat16* p, long long i, flo
 template <int BM, int BN, int BK, int TM, int TN>
 __global__ void __launch_bounds__((BM / TM) * (BN / TN))
 sgemm_tiled_kernel(int M, int N, int K, long long sa_i, long long sa_k, long long sb_k, long long sb_j, float alpha,
-                   const float* __restrict__ A, const float* __restrict__ B, float* __restrict__ C) {
+                   const float* __restrict__ A, const float* __restrict__ B, float* __restrict__ C, float beta = 0.0f,
+                   long long batch_a = 0, long long batch_b = 0, long long batch_c = 0) {
     constexpr int NT = (BM / TM) * (BN / TN);
+    // batch = blockIdx.z; C = beta * C + alpha * A . B (C is not read when beta == 0)
+    A += blockIdx.z * batch_a;
+    B += blockIdx.z * batch_b;
+    C += blockIdx.z * batch_c;
     __shared__ float As[BK][BM + 4];
     __shared__ float Bs[BK][BN + 4];
     const int tid = threadIdx.x;
@@ -75,7 +82,10 @@ sgemm_tiled_kernel(int M, int N, int K, long long sa_i, long long sa_k, long lon
 #pragma unroll
         for (int j = 0; j < TN; ++j) {
             const int gj = n0 + tx * TN + j;
-            if (gj < N) C[static_cast<long long>(gi) * N + gj] = alpha * acc[i][j];
+            if (gj < N) {
+                float* c = C + static_cast<long long>(gi) * N + gj;
+                *c = beta != 0.0f ? fmaf(beta, *c, alpha * acc[i][j]) : alpha * acc[i][j];
+            }
         }
     }
 }
@@ -97,8 +107,12 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 
 __global__ void __launch_bounds__(256)
 sgemm_small_kernel(int M, int N, int K, long long sa_i, long long sa_k, long long sb_k, long long sb_j, float alpha,
-                   const float* __restrict__ A, const float* __restrict__ B, float* __restrict__ C) {
+                   const float* __restrict__ A, const float* __restrict__ B, float* __restrict__ C, float beta = 0.0f,
+                   long long batch_a = 0, long long batch_b = 0, long long batch_c = 0) {
     constexpr int BM = 32, BN = 32, BK = 32, ST = 4, LD = BM + 2;
+    A += blockIdx.z * batch_a;
+    B += blockIdx.z * batch_b;
+    C += blockIdx.z * batch_c;
     __shared__ __align__(16) float As[ST][BK][LD];
     __shared__ __align__(16) float Bs[ST][BK][LD];
     const int tid = threadIdx.x;
@@ -157,7 +171,10 @@ sgemm_small_kernel(int M, int N, int K, long long sa_i, long long sa_k, long lon
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
             const int gj = n0 + tx * 2 + j;
-            if (gj < N) C[static_cast<long long>(gi) * N + gj] = alpha * acc[i][j];
+            if (gj < N) {
+                float* c = C + static_cast<long long>(gi) * N + gj;
+                *c = beta != 0.0f ? fmaf(beta, *c, alpha * acc[i][j]) : alpha * acc[i][j];
+            }
         }
     }
 }
@@ -241,15 +258,24 @@ sgemm_small_rowmajor_kernel(int M, int N, int K, float alpha, const float* __res
 template <typename TIn, typename TOut>
 __global__ void gemm_generic_kernel(long long M, long long N, long long K, long long sa_i, long long sa_k,
                                     long long sb_k, long long sb_j, float alpha, const TIn* __restrict__ A,
-                                    const TIn* __restrict__ B, TOut* __restrict__ C) {
-    const long long total = M * N;
+                                    const TIn* __restrict__ B, TOut* __restrict__ C, float beta = 0.0f,
+                                    long long batch = 1, long long batch_a = 0, long long batch_b = 0,
+                                    long long batch_c = 0) {
+    // batched: C[b] = beta * C[b] + alpha * A[b] . B[b]; C is not read when beta == 0
+    const long long per = M * N, total = per * batch;
     for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < total;
          e += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const long long i = e / N, j = e - i * N;
+        const long long b = e / per, r = e - b * per;
+        const long long i = r / N, j = r - i * N;
+        const TIn* a = A + b * batch_a;
+        const TIn* bb = B + b * batch_b;
         float acc = 0.0f;
         for (long long k = 0; k < K; ++k)
-            acc = fmaf(ld_as_float(A, i * sa_i + k * sa_k), ld_as_float(B, k * sb_k + j * sb_j), acc);
-        st_from_float(C, e, alpha * acc);
+            acc = fmaf(ld_as_float(a, i * sa_i + k * sa_k), ld_as_float(bb, k * sb_k + j * sb_j), acc);
+        TOut* c = C + b * batch_c;
+        float v = alpha * acc;
+        if (beta != 0.0f) v = fmaf(beta, as_float(c[r]), v);     // plain load: this thread overwrites it next
+        st_from_float(c, r, v);
     }
 }
 
@@ -294,7 +320,7 @@ __global__ void conv2d_generic_kernel(int Nimg, int H, int W, int Cin, int Cout,
 // ---------------------------------------------------------------------------
 __global__ void splitk_reduce_kernel(long long MN, int N, int split, const float* __restrict__ partial, float alpha,
                                      const float* __restrict__ bias, int relu, __nv_bfloat16* __restrict__ out,
-                                     int vec8) {
+                                     int vec8, float beta = 0.0f) {
     // launched with programmatic stream serialization: this grid may start while the GEMM drains; wait here
     // until the GEMM grid has completed and its partial sums are visible (a no-op for an ordinary launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -317,6 +343,10 @@ __global__ void splitk_reduce_kernel(long long MN, int N, int split, const float
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 float a = alpha * acc[2 * j], b = alpha * acc[2 * j + 1];
+                if (beta != 0.0f) {          // accumulate into what the output held
+                    a = fmaf(beta, __bfloat162float(out[e + 2 * j]), a);
+                    b = fmaf(beta, __bfloat162float(out[e + 2 * j + 1]), b);
+                }
                 if (bias != nullptr) { a += __ldg(bias + col + 2 * j); b += __ldg(bias + col + 2 * j + 1); }
                 if (relu) { a = fmaxf(a, 0.0f); b = fmaxf(b, 0.0f); }
                 __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -330,6 +360,7 @@ __global__ void splitk_reduce_kernel(long long MN, int N, int split, const float
             float acc = 0.0f;
             for (int s = 0; s < split; ++s) acc += __ldg(partial + s * MN + e);
             float v = alpha * acc;
+            if (beta != 0.0f) v = fmaf(beta, __bfloat162float(out[e]), v);
             if (bias != nullptr) v += __ldg(bias + e % N);
             if (relu) v = fmaxf(v, 0.0f);
             out[e] = __float2bfloat16_rn(v);

@@ -594,7 +594,7 @@ int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensor
 // The reduction is launched with programmatic stream serialization so that its launch latency hides behind
 // the tail of the GEMM kernel; it waits on the device for the GEMM grid to complete before reading partials.
 int launch_splitk_reduce(int grid, cudaStream_t st, long long MN, int N, int split, const float* partial, float alpha,
-                         __nv_bfloat16* out, int vec8) {
+                         __nv_bfloat16* out, int vec8, float beta = 0.0f) {
     cudaLaunchConfig_t lc;
     std::memset(&lc, 0, sizeof lc);
     lc.gridDim = dim3(static_cast<unsigned>(grid));
@@ -608,7 +608,7 @@ int launch_splitk_reduce(int grid, cudaStream_t st, long long MN, int N, int spl
     lc.numAttrs = 1;
     const float* bias = nullptr;
     int relu = 0;
-    TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::splitk_reduce_kernel, MN, N, split, partial, alpha, bias, relu, out, vec8));
+    TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::splitk_reduce_kernel, MN, N, split, partial, alpha, bias, relu, out, vec8, beta));
     g_launches.fetch_add(1);
     return TDX_OK;
 }
@@ -626,7 +626,7 @@ int ensure_ws(DeviceCtx* ctx, size_t bytes, void** out) {
 }
 
 int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
-                  const tdx_config& cfg, void* ws, size_t ws_bytes, bool internal_ws, cudaStream_t st) {
+                  const tdx_config& cfg, void* ws, size_t ws_bytes, bool internal_ws, cudaStream_t st, float beta = 0.0f) {
     const int64_t num_kb = ceil_div(g.K, 64);
     UmmaParams p;
     std::memset(&p, 0, sizeof p);
@@ -647,6 +647,7 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     p.a_mn_major = g.transA ? 1 : 0;   // A stored K x M: M contiguous
     p.b_mn_major = g.transB ? 0 : 1;   // B stored K x N: N contiguous
     p.alpha = alpha;
+    p.beta = beta;
     p.bias = nullptr;
     p.relu = 0;
     p.C = static_cast<__nv_bfloat16*>(C);
@@ -706,7 +707,8 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     if (rc) return rc;
 
     CUtensorMap mc = ma;   // unused unless the staged epilogue is on
-    p.tma_store = (cfg.store_mode == 2 && cfg.split_k == 1 && p.vec_store) ? 1 : 0;
+    // the accumulate term is read by the direct-store epilogue (and by the split-K reduction) only
+    p.tma_store = (cfg.store_mode == 2 && cfg.split_k == 1 && p.vec_store && beta == 0.0f) ? 1 : 0;
     if (p.tma_store) {
         uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.M)};
         uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
@@ -721,7 +723,7 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         const int vec8 = p.vec_store ? 1 : 0;
         const long long work = vec8 ? MN / 8 : MN;
         const int grid = static_cast<int>(std::min<long long>(ceil_div(work, 256), 148LL * 16));
-        rc = launch_splitk_reduce(std::max(grid, 1), st, MN, static_cast<int>(g.N), cfg.split_k, p.partial, alpha, p.C, vec8);
+        rc = launch_splitk_reduce(std::max(grid, 1), st, MN, static_cast<int>(g.N), cfg.split_k, p.partial, alpha, p.C, vec8, beta);
         if (rc) return rc;
     }
     return TDX_OK;
@@ -936,8 +938,14 @@ void gemm_strides(const GemmProblem& g, long long* sa_i, long long* sa_k, long l
     *sb_j = g.transB ? g.K : 1;
 }
 
+// batch count, batch strides in elements, and the accumulate factor of tdx_gemm_batched (one batch, beta = 0: tdx_gemm)
+struct BatchArgs {
+    int64_t batch = 1, stride_a = 0, stride_b = 0, stride_c = 0;
+    float beta = 0.0f;
+};
+
 int run_gemm_simt_f32(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
-                      cudaStream_t st) {
+                      cudaStream_t st, const BatchArgs& ba = BatchArgs()) {
     if (g.M >= (1LL << 31) || g.N >= (1LL << 31) || g.K >= (1LL << 31))
         return fail(TDX_ERR_UNSUPPORTED, "fp32 tiled GEMM needs dimensions below 2^31");
     long long sa_i, sa_k, sb_k, sb_j;
@@ -945,18 +953,23 @@ int run_gemm_simt_f32(DeviceCtx* ctx, const GemmProblem& g, float alpha, const v
     const float* a = static_cast<const float*>(A);
     const float* b = static_cast<const float*>(B);
     float* c = static_cast<float*>(C);
-    if (ceil_div(g.M, 64) * ceil_div(g.N, 64) >= ctx->sm_count) {
-        dim3 grid(static_cast<unsigned>(ceil_div(g.N, 64)), static_cast<unsigned>(ceil_div(g.M, 64)));
+    if (ba.batch > 65535) return fail(TDX_ERR_UNSUPPORTED, "fp32 batched GEMM takes at most 65535 batches");
+    const unsigned nz = static_cast<unsigned>(ba.batch);
+    const bool plain = ba.batch == 1 && ba.beta == 0.0f;
+    if (ceil_div(g.M, 64) * ceil_div(g.N, 64) * ba.batch >= ctx->sm_count) {
+        dim3 grid(static_cast<unsigned>(ceil_div(g.N, 64)), static_cast<unsigned>(ceil_div(g.M, 64)), nz);
         tdx::sgemm_tiled_kernel<64, 64, 16, 4, 4><<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k,
-                                                                       sb_j, alpha, a, b, c);
+                                                                       sb_j, alpha, a, b, c, ba.beta, ba.stride_a,
+                                                                       ba.stride_b, ba.stride_c);
     } else {
-        dim3 grid(static_cast<unsigned>(ceil_div(g.N, 32)), static_cast<unsigned>(ceil_div(g.M, 32)));
-        const bool rowmajor16 = !g.transA && !g.transB && g.K % 4 == 0 && g.N % 4 == 0 &&
+        dim3 grid(static_cast<unsigned>(ceil_div(g.N, 32)), static_cast<unsigned>(ceil_div(g.M, 32)), nz);
+        const bool rowmajor16 = plain && !g.transA && !g.transB && g.K % 4 == 0 && g.N % 4 == 0 &&
                                 reinterpret_cast<uintptr_t>(A) % 16 == 0 && reinterpret_cast<uintptr_t>(B) % 16 == 0;
         if (rowmajor16)
             tdx::sgemm_small_rowmajor_kernel<<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, alpha, a, b, c);
         else
-            tdx::sgemm_small_kernel<<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k, sb_j, alpha, a, b, c);
+            tdx::sgemm_small_kernel<<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k, sb_j, alpha, a, b,
+                                                          c, ba.beta, ba.stride_a, ba.stride_b, ba.stride_c);
     }
     TDX_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
@@ -964,19 +977,21 @@ int run_gemm_simt_f32(DeviceCtx* ctx, const GemmProblem& g, float alpha, const v
 }
 
 int run_gemm_generic(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
-                     cudaStream_t st) {
+                     cudaStream_t st, const BatchArgs& ba = BatchArgs()) {
     long long sa_i, sa_k, sb_k, sb_j;
     gemm_strides(g, &sa_i, &sa_k, &sb_k, &sb_j);
-    const long long total = g.M * g.N;
+    const long long total = g.M * g.N * ba.batch;
     const int grid = static_cast<int>(std::min<long long>(ceil_div(total, 256), static_cast<long long>(ctx->sm_count) * 32));
     if (g.dtype == TDX_F32)
         tdx::gemm_generic_kernel<float, float><<<grid, 256, 0, st>>>(g.M, g.N, g.K, sa_i, sa_k, sb_k, sb_j, alpha,
                                                                     static_cast<const float*>(A),
-                                                                    static_cast<const float*>(B), static_cast<float*>(C));
+                                                                    static_cast<const float*>(B), static_cast<float*>(C),
+                                                                    ba.beta, ba.batch, ba.stride_a, ba.stride_b, ba.stride_c);
     else
         tdx::gemm_generic_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
             g.M, g.N, g.K, sa_i, sa_k, sb_k, sb_j, alpha, static_cast<const __nv_bfloat16*>(A),
-            static_cast<const __nv_bfloat16*>(B), static_cast<__nv_bfloat16*>(C));
+            static_cast<const __nv_bfloat16*>(B), static_cast<__nv_bfloat16*>(C), ba.beta, ba.batch, ba.stride_a,
+            ba.stride_b, ba.stride_c);
     TDX_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     return TDX_OK;
@@ -1468,6 +1483,50 @@ int tdx_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, float alph
     return gemm_dispatch(M, N, K, transA, transB, alpha, dtype, A, B, C, stream, nullptr, nullptr, 0, true);
 }
 
+int tdx_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, float beta,
+                     int dtype, const void* A, int64_t strideA, const void* B, int64_t strideB, void* C, int64_t strideC,
+                     void* stream) {
+    int rc = validate_gemm(M, N, K, transA, transB, dtype, A, B, C, true);
+    if (rc) return rc;
+    if (batch < 0) return fail(TDX_ERR_INVALID_ARG, "negative batch count");
+    if (strideA < 0 || strideB < 0) return fail(TDX_ERR_INVALID_ARG, "negative batch stride");
+    if (batch > 1 && strideC < M * N) return fail(TDX_ERR_INVALID_ARG, "strideC < M * N: the outputs of two batches would overlap");
+    if (!(beta == beta) || !(alpha == alpha)) return fail(TDX_ERR_INVALID_ARG, "alpha or beta is NaN");
+    if (batch == 0 || M == 0 || N == 0) return TDX_OK;
+    if (batch >= (1LL << 31)) return fail(TDX_ERR_UNSUPPORTED, "batch count must be below 2^31");
+    DeviceCtx* ctx;
+    rc = get_ctx(&ctx);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    GemmProblem g{M, N, K, transA, transB, dtype};
+    BatchArgs ba;
+    ba.batch = batch; ba.stride_a = strideA; ba.stride_b = strideB; ba.stride_c = strideC; ba.beta = beta;
+    if (K == 0) {
+        // empty reduction: C = beta * C.  The generic kernel does exactly that (its k loop is empty).
+        return run_gemm_generic(ctx, g, alpha, C, C, C, st, ba);
+    }
+    if (dtype == TDX_F32) return run_gemm_simt_f32(ctx, g, alpha, A, B, C, st, ba);
+    // bf16: the tensor-core kernel, one launch per batch, when every batch's operands meet its layout rules
+    const bool aligned = gemm_umma_layout_ok(g) && reinterpret_cast<uintptr_t>(A) % 16 == 0 &&
+                         reinterpret_cast<uintptr_t>(B) % 16 == 0 && (strideA % 8 == 0) && (strideB % 8 == 0);
+    if (!aligned) return run_gemm_generic(ctx, g, alpha, A, B, C, st, ba);
+    tdx_config want;
+    std::memset(&want, 0, sizeof want);
+    if (beta != 0.0f) want.store_mode = 1;          // the accumulate term is read by the direct-store epilogue
+    tdx_config cfg;
+    rc = resolve_gemm_config(g, beta != 0.0f ? &want : nullptr, ctx->sm_count, ctx->smem_optin, &cfg);
+    if (rc) return rc;
+    if (cfg.kernel != TDX_KERNEL_UMMA || cfg.cta_pair == 2) return run_gemm_generic(ctx, g, alpha, A, B, C, st, ba);
+    for (int64_t b = 0; b < batch; ++b) {
+        const char* a = static_cast<const char*>(A) + b * strideA * 2;
+        const char* bb = static_cast<const char*>(B) + b * strideB * 2;
+        char* c = static_cast<char*>(C) + b * strideC * 2;
+        rc = run_gemm_umma(ctx, g, alpha, a, bb, c, cfg, nullptr, 0, true, st, beta);
+        if (rc) return rc;
+    }
+    return TDX_OK;
+}
+
 int tdx_gemm_ex(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype, const void* A,
                 const void* B, void* C, void* stream, const tdx_config* cfg, void* workspace, size_t workspace_bytes) {
     // the library's own workspace serves every split-K it chose itself
@@ -1515,6 +1574,33 @@ int tdx_gemm_host(int64_t M, int64_t N, int64_t K, int transA, int transB, float
     if (a_bytes) TDX_CUDA(cudaMemcpyAsync(dA, A_host, a_bytes, cudaMemcpyHostToDevice, st));
     if (b_bytes) TDX_CUDA(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, st));
     rc = gemm_dispatch(M, N, K, transA, transB, alpha, dtype, dA, dB, dC, stream, nullptr, nullptr, 0, true);
+    if (rc) return rc;
+    TDX_CUDA(cudaMemcpyAsync(C_host, dC, c_bytes, cudaMemcpyDeviceToHost, st));
+    TDX_CUDA(cudaStreamSynchronize(st));
+    return TDX_OK;
+}
+
+int tdx_gemm_batched_host(int64_t batch, int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, float beta,
+                          int dtype, const void* A_host, const void* B_host, void* C_host, void* stream) {
+    int rc = validate_gemm(M, N, K, transA, transB, dtype, A_host, B_host, C_host, true);
+    if (rc) return rc;
+    if (batch < 0) return fail(TDX_ERR_INVALID_ARG, "negative batch count");
+    if (batch == 0 || M == 0 || N == 0) return TDX_OK;
+    DeviceCtx* ctx;
+    rc = get_ctx(&ctx);
+    if (rc) return rc;
+    const size_t el = dtype == TDX_F32 ? 4 : 2;
+    const size_t a_bytes = static_cast<size_t>(batch) * M * K * el, b_bytes = static_cast<size_t>(batch) * K * N * el,
+                 c_bytes = static_cast<size_t>(batch) * M * N * el;
+    void *dA, *dB, *dC;
+    if ((rc = ensure_staging(ctx, 0, a_bytes, &dA))) return rc;
+    if ((rc = ensure_staging(ctx, 1, b_bytes, &dB))) return rc;
+    if ((rc = ensure_staging(ctx, 2, c_bytes, &dC))) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (a_bytes) TDX_CUDA(cudaMemcpyAsync(dA, A_host, a_bytes, cudaMemcpyHostToDevice, st));
+    if (b_bytes) TDX_CUDA(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, st));
+    if (beta != 0.0f) TDX_CUDA(cudaMemcpyAsync(dC, C_host, c_bytes, cudaMemcpyHostToDevice, st));
+    rc = tdx_gemm_batched(batch, M, N, K, transA, transB, alpha, beta, dtype, dA, M * K, dB, K * N, dC, M * N, stream);
     if (rc) return rc;
     TDX_CUDA(cudaMemcpyAsync(C_host, dC, c_bytes, cudaMemcpyDeviceToHost, st));
     TDX_CUDA(cudaStreamSynchronize(st));

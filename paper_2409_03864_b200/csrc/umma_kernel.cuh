@@ -50,6 +50,7 @@ struct UmmaParams {
     int slots;                        // accumulator slots of 128 x bn in TMEM (2 or 4)
     int a_mn_major, b_mn_major;
     float alpha;
+    float beta;               // GEMM with accumulate: out = alpha * acc + beta * (what C held); direct stores only
     const float* bias;        // [N] or nullptr
     int relu;
     __nv_bfloat16* C;         // bf16 output, row pitch ldc elements
@@ -372,6 +373,8 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     float x = p.alpha * __uint_as_float(r[j]);
+                    if (p.beta != 0.0f && col0 + j < p.N)
+                        x = fmaf(p.beta, __bfloat162float(p.C[grow * p.ldc + col0 + j]), x);
                     if (p.bias != nullptr && col0 + j < p.N) x += __ldg(p.bias + col0 + j);
                     if (p.relu) x = fmaxf(x, 0.0f);
                     v[j] = x;

@@ -73,6 +73,17 @@ def test_gemm_argument_validation_is_silenceable_and_precedes_cuda():
     assert tdx.tdx_gemm(**dict(base, N=0)) == tdx.TDX_OK
 
 
+def test_batched_gemm_argument_validation():
+    base = dict(batch=2, M=8, N=8, K=8, transA=0, transB=0, alpha=1.0, beta=1.0, dtype=tdx.TDX_F32, A=256, B=512, C=1024)
+    for b in [dict(batch=-1), dict(M=-1), dict(K=-2), dict(transB=3), dict(dtype=9), dict(A=None), dict(C=None),
+              dict(strideA=-8), dict(strideC=63), dict(alpha=float("nan")), dict(beta=float("nan"))]:
+        st = tdx.tdx_gemm_batched(**dict(base, **b))
+        assert st == tdx.TDX_ERR_INVALID_ARG, (b, st)
+    assert tdx.tdx_gemm_batched(**dict(base, C=1026)) == tdx.TDX_ERR_ALIGNMENT
+    assert tdx.tdx_gemm_batched(**dict(base, batch=0)) == tdx.TDX_OK
+    assert tdx.tdx_gemm_batched(**dict(base, N=0)) == tdx.TDX_OK
+
+
 def test_conv_argument_validation():
     base = dict(N=1, H=8, W=8, Cin=8, Cout=8, R=3, S=3, pad=1, stride=1, dtype=tdx.TDX_BF16, x=256, w=512, bias=None,
                 relu=1, y=1024)

@@ -1,0 +1,116 @@
+"""GPU parity of tdx_gemm_batched (batch-matmul with accumulate) against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2409_03864_b200 as tdx
+import seeded_inputs as si
+from gpu_util import TIGHT, TOL, to_dev
+
+pytestmark = pytest.mark.gpu
+
+DT = {"f32": tdx.TDX_F32, "bf16": tdx.TDX_BF16}
+
+
+def operands(batch, M, N, K, dtype, seed, transA=0, transB=0, integers=False):
+    gen = (lambda t, sh: si.small_integers(seed, t, sh, dtype, -2, 2)) if integers else \
+          (lambda t, sh: (si.uniform if dtype == "f32" else si.normal)(seed, t, sh, dtype))
+    A = gen(0, (batch, K, M) if transA else (batch, M, K))
+    B = gen(1, (batch, N, K) if transB else (batch, K, N))
+    C = gen(2, (batch, M, N))
+    return A, B, C
+
+
+def run(batch, M, N, K, tA, tB, alpha, beta, dtype, A, B, C):
+    dA, dB, dC = to_dev(A), to_dev(B), to_dev(C)
+    st = tdx.tdx_gemm_batched(batch, M, N, K, tA, tB, alpha, beta, DT[dtype], dA, dB, dC)
+    torch.cuda.synchronize()
+    out = dC.cpu().numpy()
+    return st, (out.view(np.uint16) if dtype == "bf16" else out).reshape(batch * M, N)
+
+
+def error(batch, M, N, K, tA, tB, alpha, beta, dtype, A, B, C, got):
+    ref = oracle.gemm_batched(batch, M, N, K, tA, tB, alpha, beta, dtype, A, B, C).reshape(batch * M, N)
+    sc = oracle.gemm_batched_row_scales(batch, M, N, K, tA, tB, alpha, beta, dtype, A, B, C)
+    return oracle.max_normalised_error(oracle.decode(got, dtype), ref, sc)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_the_papers_batch_matmul_workload(dtype):
+    # Case Study 4's loop nest as printed: 6 batches of 196 x 256 x 2305, C += A . B.  K = 2305 breaks every 16-byte
+    # rule, so bf16 runs on the generic GPU kernel; fp32 runs on the CUDA-core tiled kernel.
+    batch, M, N, K = 6, 196, 256, 2305
+    A, B, C = operands(batch, M, N, K, dtype, seed=90)
+    st, got = run(batch, M, N, K, 0, 0, 1.0, 1.0, dtype, A, B, C)
+    assert st == 0, tdx.tdx_last_error()
+    err = error(batch, M, N, K, 0, 0, 1.0, 1.0, dtype, A, B, C, got)
+    assert err < TOL[dtype] and err < TIGHT[dtype], err
+
+
+@pytest.mark.parametrize("tA,tB", [(0, 0), (0, 1), (1, 0), (1, 1)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_batched_exact_integers_all_layouts(dtype, tA, tB):
+    # small integers: every path must return the oracle's values exactly (sums stay far below 2^8 .. 2^24)
+    batch, M, N, K = 3, 136, 72, 40
+    A, B, C = operands(batch, M, N, K, dtype, seed=91, transA=tA, transB=tB, integers=True)
+    st, got = run(batch, M, N, K, tA, tB, 1.0, 1.0, dtype, A, B, C)
+    assert st == 0, tdx.tdx_last_error()
+    ref = oracle.gemm_batched(batch, M, N, K, tA, tB, 1.0, 1.0, dtype, A, B, C).reshape(batch * M, N)
+    assert np.array_equal(oracle.decode(got, dtype), ref)
+
+
+@pytest.mark.parametrize("shape", [(4, 384, 320, 448), (2, 128, 8192, 512), (5, 520, 264, 200)])
+@pytest.mark.parametrize("alpha,beta", [(1.0, 1.0), (-0.5, 2.0), (1.0, 0.0)])
+def test_batched_bf16_on_the_tensor_cores(shape, alpha, beta):
+    # aligned shapes: one tensor-core launch per batch; the accumulate term goes through the direct-store epilogue
+    # (or the split-K reduction for the skinny shape)
+    batch, M, N, K = shape
+    A, B, C = operands(batch, M, N, K, "bf16", seed=92, transB=1)
+    n0 = tdx.tdx_kernel_launch_count()
+    st, got = run(batch, M, N, K, 0, 1, alpha, beta, "bf16", A, B, C)
+    assert st == 0, tdx.tdx_last_error()
+    assert tdx.tdx_kernel_launch_count() - n0 >= batch
+    err = error(batch, M, N, K, 0, 1, alpha, beta, "bf16", A, B, C, got)
+    assert err < TIGHT["bf16"], err
+
+
+def test_batched_strides_shared_operand_and_gaps():
+    # strideB = 0 shares one B among the batches; strideA / strideC larger than dense leave gaps that must stay untouched
+    batch, M, N, K = 3, 70, 50, 33
+    A = si.uniform(93, 0, (batch, M * K + 7), "f32")
+    Bm = si.uniform(93, 1, (K, N), "f32")
+    C = si.uniform(93, 2, (batch, M * N + 5), "f32")
+    dA, dB, dC = to_dev(A), to_dev(Bm), to_dev(C)
+    st = tdx.tdx_gemm_batched(batch, M, N, K, 0, 0, 2.0, -1.0, tdx.TDX_F32, dA, dB, dC, strideA=M * K + 7, strideB=0,
+                              strideC=M * N + 5)
+    torch.cuda.synchronize()
+    assert st == 0, tdx.tdx_last_error()
+    got = dC.cpu().numpy()
+    ref = oracle.gemm_batched(batch, M, N, K, 0, 0, 2.0, -1.0, "f32", A, np.tile(Bm.ravel(), batch), C,
+                              strideA=M * K + 7, strideC=M * N + 5)
+    assert np.array_equal(got[:, M * N:], C[:, M * N:])                       # gaps untouched
+    sc = oracle.gemm_batched_row_scales(batch, M, N, K, 0, 0, 2.0, -1.0, "f32", A[:, :M * K], np.tile(Bm.ravel(), batch),
+                                        C[:, :M * N])
+    err = oracle.max_normalised_error(got[:, :M * N].reshape(batch * M, N).astype(np.float64), ref.reshape(batch * M, N), sc)
+    assert err < TIGHT["f32"], err
+
+
+def test_batched_edge_cases():
+    M, N, K = 16, 24, 8
+    A, B, C = operands(2, M, N, K, "f32", seed=94)
+    dA, dB, dC = to_dev(A), to_dev(B), to_dev(C)
+    # empty batch / empty output: no-op
+    assert tdx.tdx_gemm_batched(0, M, N, K, 0, 0, 1.0, 1.0, tdx.TDX_F32, dA, dB, dC) == 0
+    assert tdx.tdx_gemm_batched(2, 0, N, K, 0, 0, 1.0, 1.0, tdx.TDX_F32, dA, dB, dC) == 0
+    torch.cuda.synchronize()
+    assert np.array_equal(dC.cpu().numpy(), C)
+    # K = 0: C = beta * C
+    assert tdx.tdx_gemm_batched(2, M, N, 0, 0, 0, 1.0, 0.5, tdx.TDX_F32, dA, dB, dC) == 0
+    torch.cuda.synchronize()
+    assert np.array_equal(dC.cpu().numpy(), np.float32(0.5) * C)
+    # overlapping outputs and negative strides are refused before anything runs
+    assert tdx.tdx_gemm_batched(2, M, N, K, 0, 0, 1.0, 1.0, tdx.TDX_F32, dA, dB, dC, strideC=M * N - 1) == tdx.TDX_ERR_INVALID_ARG
+    assert tdx.tdx_gemm_batched(2, M, N, K, 0, 0, 1.0, 1.0, tdx.TDX_F32, dA, dB, dC, strideA=-1) == tdx.TDX_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert np.array_equal(dC.cpu().numpy(), np.float32(0.5) * C)
