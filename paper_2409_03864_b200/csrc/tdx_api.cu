@@ -421,9 +421,10 @@ struct TilePlan {
     double uniform = 0.0;      // the same for the uniform grid
 };
 
-double tile_cost_cycles(int bm, int width, int64_t num_kb) {
+// mmas_per_kb: MMAs one CTA's tensor core runs per 64-deep K block (4 per 128 rows it owns)
+double tile_cost_cycles(int mmas_per_kb, int width, int64_t num_kb) {
     const double mma = std::max(width / 2.0, 60.0);
-    return static_cast<double>(num_kb) * 4.0 * (bm / 128) * mma + 1500.0 + 13.0 * width;
+    return static_cast<double>(num_kb) * mmas_per_kb * mma + 1500.0 + 13.0 * width;
 }
 
 // makespan of `na` tiles of cost ca and `nb` tiles of cost cb (ca >= cb > 0), dealt longest first on g CTAs, each
@@ -447,17 +448,21 @@ double lpt_two_sizes(int64_t na, double ca, int64_t nb, double cb, int g) {
 
 // Searches widths and how many row blocks take the narrower cut.  Returns false when nothing beats the uniform grid
 // by `min_gain` (relative).
+// `g` workers (CTAs, or CTA pairs when pair is set: a pair's two tensor cores share a 256-row tile).
 bool plan_fitted_tiles(int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int raster, int g, double min_gain,
-                       TilePlan* out) {
+                       TilePlan* out, bool pair = false) {
     const int64_t tiles_m = ceil_div(M, bm);
     const int64_t uniform_tiles = tiles_m * ceil_div(N, bn);
-    const double c_big = tile_cost_cycles(bm, bn, num_kb);
+    const int mmas = pair ? 4 : 4 * (bm / 128);
+    const double c_big = tile_cost_cycles(mmas, bn, num_kb);
     const double uniform = lpt_two_sizes(uniform_tiles, c_big, 0, 0.0, g);
     double best = uniform;
     int best_w = 0;
     int64_t best_b = 0, best_b1 = 0, best_e = 0;
-    for (int w = bn - 64; w >= 128; w -= 64) {
-        const double c_small = tile_cost_cycles(bm, w, num_kb);
+    // pairs: each CTA loads half of a tile's columns, kept a multiple of 64 (one copy per 64 rows)
+    const int w_step = pair ? 128 : 64;
+    for (int w = bn - w_step; w >= 128; w -= w_step) {
+        const double c_small = tile_cost_cycles(mmas, w, num_kb);
         // option b of a row block: b tiles of width w at the high columns, a(b) tiles of width bn before them
         auto bigs_for = [&](int64_t b) { return ceil_div(std::max<int64_t>(0, N - b * w), bn); };
         // options that do not carry a tile more than needed
@@ -501,7 +506,7 @@ bool plan_fitted_tiles(int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int
     const int grid = static_cast<int>(std::min<int64_t>(total, g));
     std::vector<std::vector<T>> per(grid);
     std::vector<double> load(grid, 0.0);
-    const double c_small = tile_cost_cycles(bm, w, num_kb);
+    const double c_small = tile_cost_cycles(mmas, w, num_kb);
     auto deal = [&](const std::vector<T>& v, double cost) {
         for (const T& t : v) {
             int who = 0;
@@ -526,7 +531,7 @@ bool plan_fitted_tiles(int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int
 // Device copies of tile plans, one per (shape, tile, CTA count); never freed (a few KB each).
 struct PlanKey {
     int64_t M, N, num_kb;
-    int bm, bn, raster, g, forced;
+    int bm, bn, raster, g, forced, pair;
     bool operator<(const PlanKey& o) const { return std::memcmp(this, &o, sizeof(PlanKey)) < 0; }
 };
 struct DevicePlan { int4* dev = nullptr; int rounds = 0, grid = 0; bool fitted = false; };
@@ -534,10 +539,11 @@ std::map<PlanKey, DevicePlan> g_plans;
 
 // Looks the plan up (building and uploading it on first use; the upload is ordered on `st` before the kernel).
 int get_tile_plan(DeviceCtx* ctx, int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int raster, double min_gain,
-                  cudaStream_t st, DevicePlan* out) {
+                  cudaStream_t st, DevicePlan* out, bool pair = false) {
     PlanKey key;
     std::memset(&key, 0, sizeof key);
-    key.M = M; key.N = N; key.num_kb = num_kb; key.bm = bm; key.bn = bn; key.raster = raster; key.g = ctx->sm_count; key.forced = min_gain <= 0.0 ? 1 : 0;
+    key.M = M; key.N = N; key.num_kb = num_kb; key.bm = bm; key.bn = bn; key.raster = raster; key.g = pair ? ctx->sm_count / 2 : ctx->sm_count; key.forced = min_gain <= 0.0 ? 1 : 0;
+    key.pair = pair ? 1 : 0;
     {
         std::lock_guard<std::mutex> lk(g_mu);
         auto it = g_plans.find(key);
@@ -545,7 +551,7 @@ int get_tile_plan(DeviceCtx* ctx, int64_t M, int64_t N, int64_t num_kb, int bm, 
     }
     TilePlan plan;
     DevicePlan d;
-    d.fitted = plan_fitted_tiles(M, N, num_kb, bm, bn, raster, ctx->sm_count, min_gain, &plan);
+    d.fitted = plan_fitted_tiles(M, N, num_kb, bm, bn, raster, key.g, min_gain, &plan, pair);
     if (d.fitted) {
         const size_t bytes = plan.table.size() * sizeof(int4);
         void* dev = nullptr;
@@ -772,6 +778,21 @@ int run_gemm_pair(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
     }
     if (rc) return rc;
+    // tile widths fitted to the number of pairs; each CTA's half of a tile's B columns then arrives in 64-row copies
+    // (K-major B only: an N-major half would have to be a multiple of 64 columns)
+    p.b_box = cfg.tile_n / 2;
+    int plan_pairs = 0;
+    if (cfg.fit != 1 && !p.b_mn_major && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0) {
+        DevicePlan dp;
+        rc = get_tile_plan(ctx, g.M, g.N, num_kb, 256, cfg.tile_n, cfg.raster, cfg.fit == 2 ? 0.0 : 0.03, st, &dp, true);
+        if (rc) return rc;
+        if (dp.fitted) {
+            p.tiles = dp.dev;
+            p.rounds = dp.rounds;
+            p.b_box = 64;
+            plan_pairs = dp.grid;
+        }
+    }
     if (p.b_mn_major) {
         uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.K)};
         uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
@@ -780,7 +801,7 @@ int run_gemm_pair(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     } else {
         uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.N)};
         uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
-        uint32_t box[2] = {64, static_cast<uint32_t>(cfg.tile_n / 2)};
+        uint32_t box[2] = {64, static_cast<uint32_t>(p.b_box)};
         rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
     }
     if (rc) return rc;
@@ -793,7 +814,7 @@ int run_gemm_pair(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         if (rc) return rc;
     }
     const long long pair_tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
-    const int pairs = static_cast<int>(std::min<long long>(pair_tiles, ctx->sm_count / 2));
+    const int pairs = p.tiles ? plan_pairs : static_cast<int>(std::min<long long>(pair_tiles, ctx->sm_count / 2));
     cudaLaunchConfig_t lc;
     std::memset(&lc, 0, sizeof lc);
     lc.gridDim = dim3(static_cast<unsigned>(2 * pairs));
@@ -1350,8 +1371,16 @@ int enum_gemm(const GemmProblem& g, int sm_count, int smem_limit, std::vector<td
                 std::memset(&c, 0, sizeof c);
                 c.kernel = TDX_KERNEL_UMMA;
                 c.tile_m = 256; c.tile_n = bn; c.tile_k = 64; c.stages = stg; c.cta_pair = 2; c.split_k = 1;
-                c.store_mode = sm; c.raster = raster;
-                if (umma_config_reason(c, b_mn, ceil_div(g.K, 64), smem_limit, false, g.N) == nullptr) v->push_back(c);
+                c.store_mode = sm; c.raster = raster; c.fit = 1;
+                if (umma_config_reason(c, b_mn, ceil_div(g.K, 64), smem_limit, false, g.N) != nullptr) continue;
+                v->push_back(c);
+                if (!b_mn && bn >= 192 && bn % 64 == 0) {
+                    TilePlan plan;
+                    if (plan_fitted_tiles(g.M, g.N, ceil_div(g.K, 64), 256, bn, raster, sm_count / 2, 0.0, &plan, true)) {
+                        c.fit = 2;
+                        v->push_back(c);
+                    }
+                }
             }
     }
     return TDX_OK;

@@ -74,8 +74,9 @@ struct UmmaParams {
     int epi_warps;            // epilogue warps (0: every warp from the third on)
     // Tile table (GEMM, optional): instead of a uniform grid of bm x bn tiles, the output is cut into tiles of
     // bm rows and individually chosen widths (multiples of b_box, at most bn), and the host has already dealt
-    // them to the CTAs: entry [round * gridDim.x + cta] = (row block, first column, width, 0); width 0 ends a
-    // CTA's list.  This is how a tile count that does not fill the last wave of CTAs is evened out.
+    // them to the CTAs (CTA pairs for the pair kernel): entry [round * workers + worker] = (row block, first
+    // column, width, 0); width 0 ends a worker's list.  This is how a tile count that does not fill the last
+    // wave of CTAs is evened out.
     const int4* tiles;
     int rounds;
     int b_box;                // rows of one B copy (K-major B); bn when there is no table
@@ -146,13 +147,13 @@ __device__ __forceinline__ TileCoord decode_item(const UmmaParams& p, int item) 
     return t;
 }
 
-// The `local`-th tile of this CTA: from the tile table when there is one, else item first_item + local * item_stride
-// of the uniform grid.  Returns false when the CTA has no more tiles.
+// The `local`-th tile of worker `first_item` of `item_stride` workers (CTAs, or CTA pairs): from the tile table when
+// there is one, else item first_item + local * item_stride of the uniform grid.  Returns false when there is none.
 __device__ __forceinline__ bool get_tile(const UmmaParams& p, int local, int first_item, int item_stride, int total_items,
                                          TileCoord* t) {
     if (p.tiles != nullptr) {
         if (local >= p.rounds) return false;
-        const int4 e = __ldg(p.tiles + static_cast<size_t>(local) * gridDim.x + blockIdx.x);
+        const int4 e = __ldg(p.tiles + static_cast<size_t>(local) * item_stride + first_item);
         if (e.z == 0) return false;
         t->m_blk = e.x;
         t->n_blk = 0;

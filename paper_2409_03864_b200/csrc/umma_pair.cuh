@@ -77,16 +77,18 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int item = pair_id; ok && item < total_items; item += num_pairs) {
-                const TileCoord t = decode_item(p, item);
+            TileCoord t;
+            for (int local = 0; ok && get_tile(p, local, pair_id, num_pairs, total_items, &t); ++local) {
+                const int my_bn = t.bn / 2;                                            // this CTA's share of the tile's columns
                 const int row0 = t.m_blk * 256 + static_cast<int>(rank) * kHalfM;      // this CTA's rows of op(A)
-                const int col0 = t.n_blk * p.bn + static_cast<int>(rank) * half_bn;    // this CTA's columns of op(B)
+                const int col0 = t.n0 + static_cast<int>(rank) * my_bn;                // this CTA's columns of op(B)
+                const uint32_t pair_tx = 2u * (kHalfABytes + static_cast<uint32_t>(my_bn) * 128u);
                 for (int kb = 0; kb < p.num_kb; ++kb) {
                     if (!wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) {
                         ok = false;
                         break;
                     }
-                    if (rank == 0) ptx::mbar_arrive_expect_tx(&full_bar[stage], 2u * stage_bytes);
+                    if (rank == 0) ptx::mbar_arrive_expect_tx(&full_bar[stage], pair_tx);
                     const uint32_t bar = ptx::mapa_u32(ptx::smem_u32(&full_bar[stage]), 0);   // the leader's barrier
                     uint8_t* a_dst = smem + static_cast<size_t>(stage) * stage_bytes;
                     uint8_t* b_dst = a_dst + kHalfABytes;
@@ -97,10 +99,11 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         ptx::tma_load_2d_pair(a_dst, &tmA, bar, kb * kBK, row0);
                     }
                     if (p.b_mn_major) {
-                        for (int i = 0; i < half_bn / 64; ++i)
+                        for (int i = 0; i < my_bn / 64; ++i)
                             ptx::tma_load_2d_pair(b_dst + i * 8192, &tmB, bar, col0 + i * 64, kb * kBK);
                     } else {
-                        ptx::tma_load_2d_pair(b_dst, &tmB, bar, kb * kBK, col0);
+                        for (int r0 = 0; r0 < my_bn; r0 += p.b_box)
+                            ptx::tma_load_2d_pair(b_dst + r0 * 128, &tmB, bar, kb * kBK, col0 + r0);
                     }
                     if (++stage == p.stages) {
                         stage = 0;
@@ -115,7 +118,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer (leader CTA only)
         if (rank == 0 && ptx::elect_one()) {
-            const uint32_t idesc = ptx::make_idesc_bf16_f32(256, p.bn, p.a_mn_major, p.b_mn_major);
+            const uint32_t idesc0 = ptx::make_idesc_bf16_f32(256, p.bn, p.a_mn_major, p.b_mn_major);
             const uint32_t a_lbo = p.a_mn_major ? 8192u : 16u;
             const uint32_t b_lbo = p.b_mn_major ? 8192u : 16u;
             const uint32_t a_kstep = p.a_mn_major ? 2048u : 32u;
@@ -125,10 +128,13 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const uint64_t stage_step = stage_bytes >> 4;
             const uint64_t a_k16 = a_kstep >> 4, b_k16 = b_kstep >> 4;
             uint64_t a_desc = a_desc0, b_desc = b_desc0;
-            int stage = 0, local = 0;
+            int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int item = pair_id; ok && item < total_items; item += num_pairs, ++local) {
+            TileCoord t;
+            for (int local = 0; ok && get_tile(p, local, pair_id, num_pairs, total_items, &t); ++local) {
+                // N field of the instruction descriptor (bits 17..22) follows the tile's width
+                const uint32_t idesc = (idesc0 & ~(0x3Fu << 17)) | (static_cast<uint32_t>(t.bn >> 3) << 17);
                 const int slot = local % p.slots;
                 const uint32_t aphase = (local / p.slots) & 1;
                 if (!wait_bounded(&tempty_bar[slot], aphase ^ 1u, abort_flag, p.status, kTimeoutMma)) break;

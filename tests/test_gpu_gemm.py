@@ -126,6 +126,26 @@ def test_umma_tile_widths_fitted_to_the_cta_count(tile_m, transA, transB):
     assert np.array_equal(C, C1)
 
 
+def test_umma_cta_pairs_with_fitted_tile_widths():
+    # the tile table dealt to CTA pairs: each CTA loads its half of a tile's B columns in 32-row copies
+    M, N, K = 3304, 2840, 200
+    A, B = si.gemm_bf16_normal(M, N, K, seed=66, transA=0, transB=1)
+    st, C, ok = run_gemm(M, N, K, 0, 1, 1.0, "bf16", A, B, cfg=umma(cta_pair=2, tile_n=256, fit=2))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    err = gemm_error(M, N, K, 0, 1, 1.0, "bf16", A, B, C)
+    assert err < TIGHT["bf16"], err
+    st, C1, ok = run_gemm(M, N, K, 0, 1, 1.0, "bf16", A, B, cfg=umma(cta_pair=2, tile_n=256, fit=1))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert np.array_equal(C, C1)
+    # exact integers, many tiles per pair
+    M, N, K = 256 * 9, 64 * 37, 192
+    Ai = si.small_integers(67, 0, (M, K), "bf16", -1, 1)
+    Bi = si.small_integers(67, 1, (N, K), "bf16", -1, 1)
+    st, C, ok = run_gemm(M, N, K, 0, 1, 1.0, "bf16", Ai, Bi, cfg=umma(cta_pair=2, tile_n=256, fit=2))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert np.array_equal(oracle.decode(C, "bf16"), oracle.gemm(M, N, K, 0, 1, 1.0, "bf16", Ai, Bi))
+
+
 def test_umma_fitted_tiles_exact_integers_and_direct_stores():
     M, N, K = 256 * 9, 64 * 37, 192
     A = si.small_integers(65, 0, (M, K), "bf16", -1, 1)
