@@ -132,6 +132,7 @@ struct MapKey {
     uint64_t dims[4];
     uint64_t strides[3];
     uint32_t box[4];
+    uint32_t estride[4];
     int swizzle;
     bool operator<(const MapKey& o) const { return std::memcmp(this, &o, sizeof(MapKey)) < 0; }
 };
@@ -139,13 +140,13 @@ std::map<MapKey, CUtensorMap> g_maps;
 
 // bf16 tensor, 128-byte (or 64-byte) swizzle, zero fill outside the tensor.
 int get_tensor_map(DeviceCtx* ctx, const void* ptr, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                   const uint32_t* box, CUtensorMap* out, int swizzle_bytes = 128) {
+                   const uint32_t* box, CUtensorMap* out, int swizzle_bytes = 128, const uint32_t* elem_strides = nullptr) {
     MapKey key;
     std::memset(&key, 0, sizeof key);
     key.ptr = ptr;
     key.rank = rank;
     key.swizzle = swizzle_bytes;
-    for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+    for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; key.estride[i] = elem_strides ? elem_strides[i] : 1; }
     for (int i = 0; i + 1 < rank; ++i) key.strides[i] = strides_bytes[i];
     {
         std::lock_guard<std::mutex> lk(g_mu);
@@ -154,7 +155,7 @@ int get_tensor_map(DeviceCtx* ctx, const void* ptr, int rank, const uint64_t* di
     }
     cuuint64_t gdim[4], gstr[3];
     cuuint32_t gbox[4], estr[4];
-    for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; gbox[i] = box[i]; estr[i] = 1; }
+    for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; gbox[i] = box[i]; estr[i] = elem_strides ? elem_strides[i] : 1; }
     for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_bytes[i];
     CUtensorMap m;
     CUresult r = ctx->encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank),
@@ -238,7 +239,7 @@ bool gemm_umma_layout_ok(const GemmProblem& g) {
     return true;
 }
 bool conv_umma_layout_ok(const ConvProblem& c) {
-    if (c.dtype != TDX_BF16 || c.stride != 1) return false;
+    if (c.dtype != TDX_BF16 || c.stride > 8) return false;      // strided windows: per-tap loads with a traversal stride
     if (c.Cin % 8) return false;
     if (c.N * c.P * c.Q >= (1LL << 31) || c.H * c.W * c.Cin * 2 >= (1LL << 40)) return false;
     if (c.R * c.S >= (1LL << 15) || c.Cout >= (1LL << 31)) return false;
@@ -299,7 +300,7 @@ int tmem_cols_for(int tile_m, int bn) {
 // Static feasibility of a fully specified tensor-core configuration (the search-space constraints).
 // Returns 0 when feasible, else a short reason.
 const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num_kb, int smem_limit, bool conv,
-                               int64_t N, int64_t R = 1, int64_t S = 1) {
+                               int64_t N, int64_t R = 1, int64_t S = 1, int stride = 1) {
     if (c.tile_m != 128 && c.tile_m != 256) return "tile_m must be 128 or 256";
     if (c.tile_k != 64) return "tile_k must be 64";
     if (c.cta_pair != 1 && c.cta_pair != 2) return "cta_pair must be 1 or 2";
@@ -321,7 +322,10 @@ const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num
     if (!conv && c.halo > 1) return "halo applies to the convolution only";
     if (conv && (c.halo < 1 || c.halo > 3))
         return "halo must be 1 (per-tap loads), 2 (halo tile kept in shared memory) or 3 (the same over stacked images)";
+    if (conv && stride > 1 && (c.patch_w * stride > 256 || c.patch_h * stride > 256))
+        return "patch times stride exceeds the 256-element limit of a copy";
     if (conv && c.halo >= 2) {
+        if (stride != 1) return "halo reuse needs stride 1";
         if (R * S < 2) return "halo reuse needs a filter with more than one tap";
         if (c.patch_w != kHaloPatchW || c.patch_h != kHaloPatchH) return "halo reuse works on 8 x 16 patches";
         if (kHaloPatchW + S - 1 > 256 || kHaloPatchH + R - 1 > 256) return "filter too large for a halo tile";
@@ -348,11 +352,12 @@ bool patch_ok(int bw, int bh) {
     return bw >= 8 && bw <= 128 && bh >= 1 && a <= 128 && (a & (a - 1)) == 0 && (bw & (bw - 1)) == 0;
 }
 
-void choose_patch(int64_t P, int64_t Q, int* bw_out, int* bh_out) {
+// stride: a patch side times the stride must stay within the 256 elements one copy can span
+void choose_patch(int64_t P, int64_t Q, int* bw_out, int* bh_out, int stride = 1) {
     int64_t best_cost = -1;
     int best_bw = 8, best_bh = 1;
-    for (int bw = 8; bw <= 128; bw *= 2) {
-        for (int bh = 1; bw * bh <= 128; bh *= 2) {
+    for (int bw = 8; bw <= 128 && bw * stride <= 256; bw *= 2) {
+        for (int bh = 1; bw * bh <= 128 && bh * stride <= 256; bh *= 2) {
             const int64_t cost = ceil_div(Q, bw) * bw * ceil_div(P, bh) * bh;
             const bool better = best_cost < 0 || cost < best_cost ||
                                 (cost == best_cost && (bw * bh > best_bw * best_bh ||
@@ -903,6 +908,7 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     p.Nimg = static_cast<int>(c.N);
     p.S = static_cast<int>(c.S);
     p.pad = c.pad;
+    p.stride = c.stride;
     p.cchunks = cchunks;
     p.status = ctx->status_ptr;
 
@@ -913,7 +919,11 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
         uint64_t str[3] = {static_cast<uint64_t>(c.Cin) * 2, static_cast<uint64_t>(c.W * c.Cin) * 2,
                            static_cast<uint64_t>(c.H * c.W * c.Cin) * 2};
         uint32_t box[4] = {64, static_cast<uint32_t>(halo ? p.hpitch : p.bw), static_cast<uint32_t>(halo ? p.hrows : p.bh), 1};
-        int rc = get_tensor_map(ctx, x, 4, dims, str, box, &ma);
+        // strided convolution (per-tap loads only): the copy walks the image with the convolution's stride, so a
+        // box spanning bw * stride input pixels delivers exactly the bw pixels under one filter tap
+        uint32_t estr[4] = {1, static_cast<uint32_t>(c.stride), static_cast<uint32_t>(c.stride), 1};
+        if (c.stride > 1) { box[1] *= c.stride; box[2] *= c.stride; }
+        int rc = get_tensor_map(ctx, x, 4, dims, str, box, &ma, 128, c.stride > 1 ? estr : nullptr);
         if (rc) return rc;
         ma_row = ma;
         if (stacked) {
@@ -1140,12 +1150,12 @@ int resolve_conv_config(const ConvProblem& cp, const tdx_config* user, int sm_co
     }
     if (c.kernel == TDX_KERNEL_GENERIC) { *out = c; return TDX_OK; }
     if (cp.dtype != TDX_BF16) return fail(TDX_ERR_CONFIG, "the tensor-core kernel is bf16 only");
-    if (!layout_ok) return fail(TDX_ERR_ALIGNMENT, "tensor-core conv needs stride 1 and Cin %% 8 == 0");
+    if (!layout_ok) return fail(TDX_ERR_ALIGNMENT, "tensor-core conv needs stride <= 8 and Cin %% 8 == 0");
     const bool halo_auto = c.halo == 0 && !from_cache;
     if (c.halo == 0) {
         // halo reuse unless its fixed 8 x 16 patches waste much more of the image than the best free patch shape
         c.halo = 1;
-        if (cp.R * cp.S > 1 && c.patch_w == 0 && c.patch_h == 0) {
+        if (cp.stride == 1 && cp.R * cp.S > 1 && c.patch_w == 0 && c.patch_h == 0) {
             int bw, bh;
             choose_patch(cp.P, cp.Q, &bw, &bh);
             const int64_t best = ceil_div(cp.Q, bw) * bw * ceil_div(cp.P, bh) * bh;
@@ -1159,7 +1169,7 @@ int resolve_conv_config(const ConvProblem& cp, const tdx_config* user, int sm_co
         }
     }
     if (c.halo >= 2 && c.patch_w == 0 && c.patch_h == 0) { c.patch_w = kHaloPatchW; c.patch_h = kHaloPatchH; }
-    if (c.patch_w == 0 && c.patch_h == 0) choose_patch(cp.P, cp.Q, &c.patch_w, &c.patch_h);
+    if (c.patch_w == 0 && c.patch_h == 0) choose_patch(cp.P, cp.Q, &c.patch_w, &c.patch_h, cp.stride);
     if (!patch_ok(c.patch_w, c.patch_h)) return fail(TDX_ERR_CONFIG, "infeasible config: patch %dx%d", c.patch_w, c.patch_h);
     const int nb = 128 / (c.patch_w * c.patch_h);
     const int64_t tiles_m = c.halo >= 2 ? halo_patches(cp, c.halo)
@@ -1180,7 +1190,7 @@ int resolve_conv_config(const ConvProblem& cp, const tdx_config* user, int sm_co
         c.stages = c.halo >= 2 ? std::max(2, halo_max_stages(c.tile_m, c.tile_n, cp.R, cp.S, smem_limit, c.store_mode))
                                : std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode));
     if (!user && !from_cache) c.raster = d.raster;
-    const char* why = umma_config_reason(c, false, num_kb, smem_limit, true, cp.Cout, cp.R, cp.S);
+    const char* why = umma_config_reason(c, false, num_kb, smem_limit, true, cp.Cout, cp.R, cp.S, cp.stride);
     if (why && halo_auto && c.halo >= 2) {
         // the automatic choice of halo reuse did not fit (large filter): fall back to per-tap loads
         tdx_config retry;
@@ -1281,7 +1291,7 @@ int conv_dispatch(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, in
 
 // ------------------------------------------------------------------ search space
 void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int sm_count, int smem_limit, bool conv,
-                     int patch_w, int patch_h, std::vector<tdx_config>* out) {
+                     int patch_w, int patch_h, std::vector<tdx_config>* out, int stride = 1) {
     for (int tm : {256, 128}) {
         const int64_t tiles_m_t = ceil_div(tiles_m, tm / 128);
         for (int bn = 256; bn >= 32; bn -= 32) {
@@ -1317,7 +1327,7 @@ void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int 
                                 c.patch_w = patch_w; c.patch_h = patch_h;
                                 c.halo = conv ? 1 : 0;
                                 c.fit = conv ? 0 : 1;
-                                if (umma_config_reason(c, b_mn, num_kb, smem_limit, conv, N, 3, 3) != nullptr) continue;
+                                if (umma_config_reason(c, b_mn, num_kb, smem_limit, conv, N, 3, 3, stride) != nullptr) continue;
                                 out->push_back(c);
                                 if (!conv && sk == 1 && bn >= 192 && bn % 64 == 0 && stagger == 0) {
                                     // the same tile with widths fitted to the CTA count, where that changes anything
@@ -1396,7 +1406,7 @@ int enum_conv(const ConvProblem& cp, int sm_count, int smem_limit, std::vector<t
         return TDX_OK;
     }
     // halo-reuse candidates (8 x 16 patches)
-    if (cp.R * cp.S > 1) {
+    if (cp.R * cp.S > 1 && cp.stride == 1) {
         const int64_t num_kb = cp.R * cp.S * ceil_div(cp.Cin, 64);
         for (int mode : {2, 3})
         for (int tm : {256, 128})
@@ -1421,7 +1431,7 @@ int enum_conv(const ConvProblem& cp, int sm_count, int smem_limit, std::vector<t
     }
     // patch shapes: every shape whose padded area is within 15 % of the best one
     int bbw, bbh;
-    choose_patch(cp.P, cp.Q, &bbw, &bbh);
+    choose_patch(cp.P, cp.Q, &bbw, &bbh, cp.stride);
     const int64_t best_cost = ceil_div(cp.Q, bbw) * bbw * ceil_div(cp.P, bbh) * bbh;
     for (int bw = 8; bw <= 128; bw *= 2)
         for (int bh = 1; bw * bh <= 128; bh *= 2) {
@@ -1430,8 +1440,9 @@ int enum_conv(const ConvProblem& cp, int sm_count, int smem_limit, std::vector<t
             if (cost * 100 > best_cost * 115) continue;
             const int nb = 128 / (bw * bh);
             const int64_t tiles_m = ceil_div(cp.N * ceil_div(cp.Q, bw) * ceil_div(cp.P, bh), nb);
+            if (bw * cp.stride > 256 || bh * cp.stride > 256) continue;
             enum_umma_space(false, tiles_m, cp.Cout, cp.R * cp.S * ceil_div(cp.Cin, 64), sm_count, smem_limit, true, bw, bh,
-                            v);
+                            v, cp.stride);
         }
     return TDX_OK;
 }

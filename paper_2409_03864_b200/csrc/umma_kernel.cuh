@@ -63,6 +63,7 @@ struct UmmaParams {
     int bw, bh, nb;           // spatial patch (bw x bh output pixels), patches per tile = bm / (bw*bh)
     int patches_w, patches_h; // patches per image along Q and P
     int P, Q, Nimg, S, pad, cchunks;
+    int stride;               // convolution stride (per-tap loads; the tensor map carries the same traversal stride)
     // halo-reuse convolution (umma_conv_halo_kernel): the input window of an 8 x 16 pixel patch is loaded once
     // per channel chunk and shared by all filter taps
     int R;                    // filter rows (taps = R * S)
@@ -501,8 +502,8 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                             const int rem = patch - n * ppi;
                             const int ph = rem / p.patches_w;
                             const int pw = rem - ph * p.patches_w;
-                            ptx::tma_load_4d(a_dst + i * patch_bytes, &tmA, bar, cc * kBK, pw * p.bw + s - p.pad,
-                                             ph * p.bh + r - p.pad, n);
+                            ptx::tma_load_4d(a_dst + i * patch_bytes, &tmA, bar, cc * kBK, pw * p.bw * p.stride + s - p.pad,
+                                             ph * p.bh * p.stride + r - p.pad, n);
                         }
                         ptx::tma_load_3d(b_dst, &tmB, bar, cc * kBK, tap, t.n0);
                     } else {

@@ -172,7 +172,12 @@ def test_search_space_for_other_kernels():
     for c in cfgs:
         a = c["patch_w"] * c["patch_h"]
         assert c["patch_w"] >= 8 and a <= 128 and a & (a - 1) == 0 and c["split_k"] == 1
-    st, cfgs = tdx.tdx_enum_conv2d_configs(1, 8, 8, 8, 8, 3, 3, 1, 2, tdx.TDX_BF16)  # stride 2
+    st, cfgs = tdx.tdx_enum_conv2d_configs(8, 56, 56, 64, 128, 3, 3, 1, 2, tdx.TDX_BF16)  # stride 2: per-tap loads only
+    assert st == tdx.TDX_OK and cfgs and all(c["kernel"] == tdx.TDX_KERNEL_UMMA and c["halo"] == 1 for c in cfgs)
+    assert all(c["patch_w"] * 2 <= 256 and c["patch_h"] * 2 <= 256 for c in cfgs)
+    st, cfgs = tdx.tdx_enum_conv2d_configs(1, 8, 8, 8, 8, 3, 3, 1, 9, tdx.TDX_BF16)   # stride 9: beyond the copy's reach
+    assert [c["kernel"] for c in cfgs] == [tdx.TDX_KERNEL_GENERIC]
+    st, cfgs = tdx.tdx_enum_conv2d_configs(1, 8, 8, 7, 8, 3, 3, 1, 1, tdx.TDX_BF16)   # Cin pitch not 16-byte aligned
     assert [c["kernel"] for c in cfgs] == [tdx.TDX_KERNEL_GENERIC]
 
 

@@ -166,6 +166,49 @@ def test_conv_padding_equals_explicit_zero_padded_copy_bitwise():
     assert np.array_equal(y1, y2)
 
 
+STRIDED_CASES = [
+    # N, H,  W,  Cin, Cout, R, S, pad, stride
+    (2, 56, 56, 64, 128, 3, 3, 1, 2),        # a ResNet-style down-sampling 3 x 3
+    (3, 57, 41, 72, 40, 3, 3, 1, 2),         # odd sizes: ragged patches, channel tail
+    (2, 28, 28, 128, 256, 1, 1, 0, 2),       # strided 1 x 1 (projection shortcut)
+    (1, 40, 40, 64, 64, 5, 5, 2, 3),         # stride 3, 5 x 5
+    (2, 17, 23, 64, 32, 2, 4, 0, 2),         # no padding, even filter
+]
+
+
+@pytest.mark.parametrize("case", STRIDED_CASES)
+@pytest.mark.parametrize("tile_m", [128, 256])
+def test_conv_strided_on_the_tensor_cores(case, tile_m):
+    # per-tap loads whose copies walk the image with the convolution's stride
+    N, H, W, Cin, Cout, R, S, pad, stride = case
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, R, S, seed=83)
+    st, y, ok = run_conv(N, H, W, Cin, Cout, R, S, pad, stride, "bf16", x, w, b, 1, cfg=umma(tile_m=tile_m))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    err = conv_error(N, H, W, Cin, Cout, R, S, pad, stride, "bf16", x, w, b, 1, y)
+    assert err < TOL["bf16"] and err < TIGHT["bf16"], err
+    # the automatic choice takes the tensor-core path too
+    n0 = tdx.tdx_kernel_launch_count()
+    st, y0, ok = run_conv(N, H, W, Cin, Cout, R, S, pad, stride, "bf16", x, w, b, 1)
+    assert st == 0 and ok, tdx.tdx_last_error()
+    st_cfg, c = tdx.tdx_default_conv2d_config(N, H, W, Cin, Cout, R, S, pad, stride, tdx.TDX_BF16)
+    assert st_cfg == 0 and c.kernel == tdx.TDX_KERNEL_UMMA and c.halo == 1
+    assert conv_error(N, H, W, Cin, Cout, R, S, pad, stride, "bf16", x, w, b, 1, y0) < TIGHT["bf16"]
+
+
+def test_conv_strided_delta_filter_is_subsampled_shift():
+    # exact: a delta filter at tap (r0, s0) with stride 2 copies every second pixel of the shifted input
+    N, H, W, C = 2, 20, 24, 64
+    x = si.small_integers(84, 0, (N, H, W, C), "bf16", -8, 8)
+    wf = np.zeros((C, 3, 3, C), dtype=np.float32)
+    for k in range(C):
+        wf[k, 2, 0, k] = 1.0
+    w = si.f32_to_bf16_bits(wf)
+    st, y, ok = run_conv(N, H, W, C, C, 3, 3, 1, 2, "bf16", x, w, None, 0)
+    assert st == 0 and ok, tdx.tdx_last_error()
+    ref = oracle.conv2d(N, H, W, C, C, 3, 3, 1, 2, "bf16", x, w, None, 0)
+    assert np.array_equal(oracle.decode(y, "bf16"), ref)
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 @pytest.mark.parametrize("stride", [1, 2])
 def test_conv_generic_kernel(dtype, stride):
@@ -185,7 +228,9 @@ def test_conv_infeasible_config_leaves_output_untouched():
     x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=75)
     st, _, untouched = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, cfg=umma(patch_w=4, patch_h=4))
     assert st == tdx.TDX_ERR_CONFIG and untouched
-    st, _, untouched = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 2, "bf16", x, w, b, 1, cfg=umma())   # stride 2
+    st, _, untouched = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 2, "bf16", x, w, b, 1, cfg=umma(halo=2))   # halo reuse is stride 1 only
+    assert st == tdx.TDX_ERR_CONFIG and untouched
+    st, _, untouched = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 9, "bf16", x, w, b, 1, cfg=umma())   # stride 9
     assert st == tdx.TDX_ERR_ALIGNMENT and untouched
 
 
