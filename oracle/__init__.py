@@ -50,6 +50,8 @@ def _load():
         lib.oracle_gemm_batched.argtypes = [i64, i64, i64, i64, ctypes.c_int, ctypes.c_int, ctypes.c_double,
                                             ctypes.c_double, ctypes.c_int, p, i64, p, i64, p, i64, p]
         lib.oracle_gemm_batched.restype = ctypes.c_int
+        lib.oracle_add_zero_pad.argtypes = [i64] * 8 + [ctypes.c_int, p, p, p]
+        lib.oracle_add_zero_pad.restype = ctypes.c_int
         lib.oracle_conv2d.argtypes = [i64] * 9 + [ctypes.c_int, p, p, p, ctypes.c_int, p, i64, p]
         lib.oracle_conv2d.restype = ctypes.c_int
         lib.oracle_conv_out_dim.argtypes = [i64] * 4
@@ -130,6 +132,19 @@ def gemm_batched(batch, M, N, K, transA, transB, alpha, beta, dtype, A, B, C=Non
                                  A.ctypes.data, sa, B.ctypes.data, sb, cp, sc, out.ctypes.data)
     if rc:
         raise RuntimeError(f"oracle_gemm_batched failed ({rc})")
+    return out
+
+
+def add_zero_pad(N, H, W, C, top, bottom, left, right, dtype, x, y) -> np.ndarray:
+    """fp64 reference of zero_pad(x) + y; x is N x H x W x C, y is N x (H+top+bottom) x (W+left+right) x C."""
+    lib, dt = _load(), _DT[dtype]
+    Hp, Wp = H + top + bottom, W + left + right
+    x = _check(x, dt, N * H * W * C, "x")
+    y = _check(y, dt, N * Hp * Wp * C, "y")
+    out = np.empty((N, Hp, Wp, C), dtype=np.float64)
+    rc = lib.oracle_add_zero_pad(N, H, W, C, top, bottom, left, right, dt, x.ctypes.data, y.ctypes.data, out.ctypes.data)
+    if rc:
+        raise RuntimeError(f"oracle_add_zero_pad failed ({rc})")
     return out
 
 

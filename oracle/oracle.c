@@ -181,6 +181,31 @@ int oracle_conv2d(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, in
     return 0;
 }
 
+/*
+ * add(zero_pad(x), y): the expression that Case Study 3's `add_of_zero_pad` pattern rewrites, computed the
+ * unrewritten way -- the padded tensor is materialised (zeros outside the interior) and then added elementwise.
+ *   xp[n, h, w, c] = x[n, h - top, w - left, c]  if top <= h < top + H and left <= w < left + W, else 0
+ *   out[n, h, w, c] = xp[n, h, w, c] + y[n, h, w, c]      (h < H + top + bottom, w < W + left + right)
+ * x is N x H x W x C, y and out are N x Hp x Wp x C (NHWC, dense).  out: doubles.
+ */
+int oracle_add_zero_pad(int64_t N, int64_t H, int64_t W, int64_t C, int64_t top, int64_t bottom, int64_t left,
+                        int64_t right, int dtype, const void *x, const void *y, double *out)
+{
+    if (N < 0 || H < 0 || W < 0 || C < 0 || top < 0 || bottom < 0 || left < 0 || right < 0) return 1;
+    int64_t Hp = H + top + bottom, Wp = W + left + right;
+    int64_t total = N * Hp * Wp * C;
+    double *xp = (double *)calloc(total > 0 ? (size_t)total : 1, sizeof(double));   /* the padded copy */
+    if (!xp) return 2;
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t h = 0; h < H; ++h)
+            for (int64_t w = 0; w < W; ++w)
+                for (int64_t c = 0; c < C; ++c)
+                    xp[((n * Hp + h + top) * Wp + w + left) * C + c] = load_elem(x, ((n * H + h) * W + w) * C + c, dtype);
+    for (int64_t i = 0; i < total; ++i) out[i] = xp[i] + load_elem(y, i, dtype);
+    free(xp);
+    return 0;
+}
+
 /* double -> bf16 bit pattern, round to nearest, ties to even, in one rounding
  * (diagnostics only: distance in bf16 ulps between a result and the reference). */
 void oracle_round_bf16(const double *in, int64_t n, uint16_t *out)

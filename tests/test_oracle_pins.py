@@ -179,6 +179,34 @@ def test_gemm_batched_closed_forms_and_special_cases():
     assert np.array_equal(twice, 2.0 * once)
 
 
+# --------------------------------------------------------------------- add of zero pad
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_add_zero_pad_hand_computed_literals(dtype):
+    g = read_golden("add_zero_pad_2x2_into_4x3.txt")
+    enc = f32 if dtype == "f32" else bf
+    out = oracle.add_zero_pad(1, 2, 2, 1, 1, 1, 0, 1, dtype, enc(g["x"]), enc(g["y"]))
+    assert np.array_equal(out.ravel(), np.array(g["out"]))
+
+
+@pytest.mark.parametrize("pads", [(0, 0, 0, 0), (1, 1, 1, 1), (2, 0, 1, 3), (0, 3, 0, 0)])
+def test_add_zero_pad_vs_library_pad_and_closed_forms(pads):
+    top, bottom, left, right = pads
+    N, H, W, C = 2, 5, 4, 3
+    x = si.uniform(21, 0, (N, H, W, C), "f32")
+    y = si.uniform(21, 1, (N, H + top + bottom, W + left + right, C), "f32")
+    ref = np.pad(x.astype(np.float64), ((0, 0), (top, bottom), (left, right), (0, 0))) + y.astype(np.float64)
+    assert np.array_equal(oracle.add_zero_pad(N, H, W, C, top, bottom, left, right, "f32", x, y), ref)
+    # all ones: 2 in the interior, 1 on the padding ring; the ring of the result is y's ring untouched
+    one_x, one_y = f32(np.ones((N, H, W, C))), f32(np.ones(y.shape))
+    out = oracle.add_zero_pad(N, H, W, C, top, bottom, left, right, "f32", one_x, one_y)
+    interior = np.zeros(y.shape, dtype=bool)
+    interior[:, top:top + H, left:left + W, :] = True
+    assert np.array_equal(out, np.where(interior, 2.0, 1.0))
+    assert np.array_equal(oracle.add_zero_pad(N, H, W, C, top, bottom, left, right, "f32", x, y)[~interior],
+                          y.astype(np.float64)[~interior])
+
+
 # --------------------------------------------------------------------- conv
 
 def test_conv_hand_computed_literals():
