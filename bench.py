@@ -63,6 +63,9 @@ WORKLOADS = {
     # the paper's own workload (Case Study 4): C[b,i,j] += A[b,i,k] * B[b,k,j], b < 6, i < 196, j < 256, k < 2305
     "cs4": dict(kind="gemm_batched", dtype="f32", batch=6, M=196, N=256, K=2305, tA=0, tB=0, alpha=1.0, beta=1.0, seed=5,
                 bound="alu", label="batch_matmul_accumulate_f32_6x196x256x2305"),
+    # Case Study 3's add_of_zero_pad pattern as an op: y += zero_pad(x) in place, the activation shape of c4
+    "azp": dict(kind="add_zero_pad", dtype="bf16", N=32, H=56, W=56, C=256, pad=1, seed=6, bound="hbm",
+                label="add_of_zero_pad_bf16_32x56x56x256_pad1_in_place"),
 }
 
 
@@ -72,7 +75,18 @@ class Workload:
     def __init__(self, name):
         self.name, self.w = name, WORKLOADS[name]
         w = self.w
-        if w["kind"] == "gemm_batched":
+        if w["kind"] == "add_zero_pad":
+            self.el = 2
+            interior = w["N"] * w["H"] * w["W"] * w["C"]
+            self.padded = w["N"] * (w["H"] + 2 * w["pad"]) * (w["W"] + 2 * w["pad"]) * w["C"]
+            self.flops = float(interior)                       # one add per interior element
+            self.in_bytes = 2 * interior * self.el             # x and the interior of y; the ring is never read
+            self.out_bytes = interior * self.el
+            self.rows = w["N"]                                 # the oracle sample is taken in whole images
+            self.unit = "images"
+            self.h2d_bytes = (interior + self.padded) * self.el    # the host-buffer call moves x and the whole y
+            self.d2h_bytes = self.padded * self.el
+        elif w["kind"] == "gemm_batched":
             self.el = 4 if w["dtype"] == "f32" else 2
             self.flops = 2.0 * w["batch"] * w["M"] * w["N"] * w["K"]
             self.in_bytes = w["batch"] * (w["M"] * w["K"] + w["K"] * w["N"] + w["M"] * w["N"]) * self.el   # A, B and C read
@@ -101,6 +115,9 @@ class Workload:
     def host_inputs(self):
         import seeded_inputs as si
         w = self.w
+        if w["kind"] == "add_zero_pad":
+            return (si.normal(w["seed"], 0, (w["N"], w["H"], w["W"], w["C"]), "bf16"),
+                    si.normal(w["seed"], 1, (w["N"], w["H"] + 2 * w["pad"], w["W"] + 2 * w["pad"], w["C"]), "bf16"))
         if w["kind"] == "gemm_batched":
             gen = si.uniform if w["dtype"] == "f32" else si.normal
             return (gen(w["seed"], 0, (w["batch"], w["M"], w["K"]), w["dtype"]),
@@ -118,6 +135,11 @@ class Workload:
     def oracle_rows(self, host, rows):
         import oracle
         w = self.w
+        if w["kind"] == "add_zero_pad":      # rows = image indices
+            import numpy as np
+            p = w["pad"]
+            return np.stack([oracle.add_zero_pad(1, w["H"], w["W"], w["C"], p, p, p, p, "bf16", host[0][n], host[1][n])[0]
+                             for n in rows])
         if w["kind"] == "gemm_batched":      # rows = batch indices
             import numpy as np
             return np.stack([oracle.gemm_batched(1, w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], w["beta"], w["dtype"],
@@ -305,7 +327,20 @@ def run_tdx(args):
     sets = [([h.cuda(non_blocking=True) for h in h_in], torch.empty_like(h_out, device="cuda")) for _ in range(n_sets)]
     stream = torch.cuda.current_stream()
     DT = tdx.TDX_F32 if wl.dtype == "f32" else tdx.TDX_BF16
-    if w["kind"] == "gemm_batched":
+    if w["kind"] == "add_zero_pad":
+        st_cfg, cfg = 1, None
+        pd = w["pad"]
+        sets = [(ins, ins[1]) for ins, _ in sets]        # in place: the output is the set's own y
+
+        def launch(ins, out):
+            return tdx.tdx_add_zero_pad(w["N"], w["H"], w["W"], w["C"], pd, pd, pd, pd, DT, ins[0], out, out, stream)
+
+        h_y = h_in[1].clone().pin_memory()
+
+        def launch_host():
+            return tdx.tdx_add_zero_pad_host(w["N"], w["H"], w["W"], w["C"], pd, pd, pd, pd, DT, h_in[0], h_y, stream)
+        kernel_name = "add_zero_pad_kernel<bf16>"
+    elif w["kind"] == "gemm_batched":
         st_cfg, cfg = 1, None
         # the step accumulates into C (beta = 1); each buffer set carries its own copy of C, and the output IS that buffer
         sets = [(ins, ins[2]) for ins, _ in sets]
@@ -431,8 +466,8 @@ def run_tdx(args):
                            l2=f"rotating {n_sets} buffer sets ({n_sets * wl.algo_bytes / 1e6:.0f} MB) larger than L2",
                            tile_config=cfg.as_dict() if st_cfg == 0 else None),
             "clocks": clocks,
-            "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": int(wl.in_bytes),
-                    "d2h_bytes_per_step": int(wl.out_bytes), "steps": e2e_steps,
+            "e2e": {"value": e2e_value, "unit": "TFLOP/s", "h2d_bytes_per_step": int(getattr(wl, "h2d_bytes", wl.in_bytes)),
+                    "d2h_bytes_per_step": int(getattr(wl, "d2h_bytes", wl.out_bytes)), "steps": e2e_steps,
                     "api": "tdx_gemm_host / tdx_conv2d_bias_relu_host (pinned host buffers)"},
             "gpu_launches": int(launches),
             "roofline": roof,

@@ -127,6 +127,22 @@ int tdx_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int transA,
                      void* stream);
 
 /*
+ * out = zero_pad(x) + y, computed the way Case Study 3's add_of_zero_pad pattern rewrites it: the padded copy of x is
+ * never built and the elements that padding would produce (zeros) are never added.
+ *
+ *   x:        N x H x W x C  (NHWC, dense)
+ *   y, out:   N x (H + pad_top + pad_bottom) x (W + pad_left + pad_right) x C
+ *   out[n, h + pad_top, w + pad_left, c] = x[n, h, w, c] + y[n, h + pad_top, w + pad_left, c];  elsewhere out = y.
+ *
+ * out may be y itself (in place): then only the interior is read and written and the padding ring is not touched at
+ * all; otherwise out must not overlap x or y, and the ring is copied.  fp32: one fp32 add; bf16: the fp32 sum of the
+ * two values rounded once to bf16.  16-byte accesses when every interior row starts on a 16-byte boundary, scalar
+ * otherwise; any shape is accepted.  Empty tensors: no-op.  Errors: INVALID_ARG, ALIGNMENT (element alignment), CUDA.
+ */
+int tdx_add_zero_pad(int64_t N, int64_t H, int64_t W, int64_t C, int pad_top, int pad_bottom, int pad_left, int pad_right,
+                     int dtype, const void* x, const void* y, void* out, void* stream);
+
+/*
  * Same as tdx_gemm with an explicit configuration and caller-owned split-K workspace.
  * cfg = NULL or cfg->split_k = 0: the library chooses split_k (tuning cache, else heuristic); then
  * `workspace` may be NULL and the library uses an internal, lazily grown buffer.  With an explicit
@@ -171,6 +187,9 @@ int tdx_conv2d_bias_relu_ex(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_
  */
 int tdx_gemm_host(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype,
                   const void* A_host, const void* B_host, void* C_host, void* stream);
+/* tdx_add_zero_pad in place on host buffers: y_host = zero_pad(x_host) + y_host. */
+int tdx_add_zero_pad_host(int64_t N, int64_t H, int64_t W, int64_t C, int pad_top, int pad_bottom, int pad_left,
+                          int pad_right, int dtype, const void* x_host, void* y_host, void* stream);
 /* tdx_gemm_batched on dense host buffers (strides M*K, K*N, M*N); C_host is copied in only when beta != 0. */
 int tdx_gemm_batched_host(int64_t batch, int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha,
                           float beta, int dtype, const void* A_host, const void* B_host, void* C_host, void* stream);

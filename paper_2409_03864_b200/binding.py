@@ -71,6 +71,8 @@ def lib() -> ctypes.CDLL:
         L.tdx_gemm_ex.argtypes = gemm_args + [cfgp, vp, sz]
         L.tdx_gemm_batched.argtypes = [i64, i64, i64, i64, ci, ci, cf, cf, ci, vp, i64, vp, i64, vp, i64, vp]
         L.tdx_gemm_batched_host.argtypes = [i64, i64, i64, i64, ci, ci, cf, cf, ci, vp, vp, vp, vp]
+        L.tdx_add_zero_pad.argtypes = [i64, i64, i64, i64, ci, ci, ci, ci, ci, vp, vp, vp, vp]
+        L.tdx_add_zero_pad_host.argtypes = [i64, i64, i64, i64, ci, ci, ci, ci, ci, vp, vp, vp]
         L.tdx_gemm_workspace_size.argtypes = [i64, i64, i64, ci, cfgp, ctypes.POINTER(sz)]
         L.tdx_conv2d_bias_relu.argtypes = conv_args
         L.tdx_conv2d_bias_relu_ex.argtypes = conv_args + [cfgp]
@@ -109,7 +111,7 @@ def lib() -> ctypes.CDLL:
 
 # every symbol include/tdx.h declares
 EXPORTS = (
-    "tdx_gemm", "tdx_gemm_batched", "tdx_gemm_batched_host", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_relu_ex",
+    "tdx_gemm", "tdx_add_zero_pad", "tdx_add_zero_pad_host", "tdx_gemm_batched", "tdx_gemm_batched_host", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_relu_ex",
     "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
     "tdx_enum_conv2d_configs", "tdx_default_gemm_config", "tdx_default_conv2d_config", "tdx_tune_save",
     "tdx_tune_load", "tdx_tune_clear", "tdx_gemm_tile_plan", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
@@ -178,6 +180,18 @@ def tdx_gemm_batched(batch, M, N, K, transA, transB, alpha, beta, dtype, A, B, C
 def tdx_gemm_batched_host(batch, M, N, K, transA, transB, alpha, beta, dtype, A, B, C, stream=None) -> int:
     """A, B, C are dense host arrays (numpy, or pinned torch CPU tensors)."""
     return lib().tdx_gemm_batched_host(batch, M, N, K, transA, transB, alpha, beta, dtype, _ptr(A), _ptr(B), _ptr(C),
+                                       _stream(stream))
+
+
+def tdx_add_zero_pad(N, H, W, C, pad_top, pad_bottom, pad_left, pad_right, dtype, x, y, out, stream=None) -> int:
+    """out = zero_pad(x) + y without building the padded copy; out may be y (in place: the ring is untouched)."""
+    return lib().tdx_add_zero_pad(N, H, W, C, pad_top, pad_bottom, pad_left, pad_right, dtype, _ptr(x), _ptr(y), _ptr(out),
+                                  _stream(stream))
+
+
+def tdx_add_zero_pad_host(N, H, W, C, pad_top, pad_bottom, pad_left, pad_right, dtype, x, y, stream=None) -> int:
+    """In place on host arrays: y = zero_pad(x) + y."""
+    return lib().tdx_add_zero_pad_host(N, H, W, C, pad_top, pad_bottom, pad_left, pad_right, dtype, _ptr(x), _ptr(y),
                                        _stream(stream))
 
 

@@ -368,6 +368,57 @@ __global__ void splitk_reduce_kernel(long long MN, int N, int split, const float
     }
 }
 
+// ---------------------------------------------------------------------------
+// add(zero_pad(x), y) without the padded copy and without adding the zeros: out = y, plus x inside the interior.
+// x is N x H x W x C, y / out are N x Hp x Wp x C.  An interior row (n, h) is W * C contiguous elements in x and
+// in y.  In place (out == y) only the interior is read and written: the padding ring is never touched.  Out of
+// place the ring is copied.  `vec` = elements per 16-byte access when every row start is 16-byte aligned, else 1.
+// HBM-bound: 3 x interior bytes in place.
+// ---------------------------------------------------------------------------
+template <typename T>
+__device__ __forceinline__ void add_vec16(const T* __restrict__ a, const T* b, T* o) {
+    constexpr int V = 16 / sizeof(T);
+    const uint4 ua = __ldg(reinterpret_cast<const uint4*>(a));
+    const uint4 ub = *reinterpret_cast<const uint4*>(b);
+    const T* pa = reinterpret_cast<const T*>(&ua);
+    const T* pb = reinterpret_cast<const T*>(&ub);
+    uint4 uo;
+    T* po = reinterpret_cast<T*>(&uo);
+#pragma unroll
+    for (int i = 0; i < V; ++i) st_from_float(po, i, as_float(pa[i]) + as_float(pb[i]));
+    *reinterpret_cast<uint4*>(o) = uo;
+}
+
+template <typename T>
+__global__ void add_zero_pad_kernel(long long rows, long long H, long long row_elems, long long y_img_elems,
+                                    long long y_row_elems, long long y_first, int vec, const T* __restrict__ x,
+                                    const T* y, T* out) {
+    // row r = (n, h): x + r * row_elems  <->  y + n * y_img_elems + y_first + h * y_row_elems
+    const long long per_row = vec > 1 ? row_elems / vec : row_elems;
+    const long long total = rows * per_row;
+    for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < total;
+         e += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const long long r = e / per_row, i = (e - r * per_row) * (vec > 1 ? vec : 1);
+        const long long n = r / H, h = r - n * H;
+        const long long xo = r * row_elems + i;
+        const long long yo = n * y_img_elems + y_first + h * y_row_elems + i;
+        if (vec > 1) add_vec16<T>(x + xo, y + yo, out + yo);
+        else st_from_float(out, yo, as_float(x[xo]) + as_float(y[yo]));
+    }
+}
+
+// out-of-place only: copies the elements of y outside the interior (the padding ring) to out
+template <typename T>
+__global__ void copy_pad_ring_kernel(long long total, long long C, long long Hp, long long Wp, long long top, long long H,
+                                     long long left, long long W, const T* __restrict__ y, T* __restrict__ out) {
+    for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < total;
+         e += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const long long pix = e / C;
+        const long long w = pix % Wp, h = (pix / Wp) % Hp;
+        if (h < top || h >= top + H || w < left || w >= left + W) out[e] = y[e];
+    }
+}
+
 // Deterministic pseudo-random fill used only by the tuner's scratch operands.
 __global__ void fill_pattern_bf16_kernel(__nv_bfloat16* p, long long n, uint32_t seed) {
     for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < n;

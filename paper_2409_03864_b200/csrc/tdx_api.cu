@@ -1568,6 +1568,61 @@ int tdx_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int transA,
     return TDX_OK;
 }
 
+int tdx_add_zero_pad(int64_t N, int64_t H, int64_t W, int64_t C, int pad_top, int pad_bottom, int pad_left, int pad_right,
+                     int dtype, const void* x, const void* y, void* out, void* stream) {
+    if (N < 0 || H < 0 || W < 0 || C < 0) return fail(TDX_ERR_INVALID_ARG, "negative dimension");
+    if (pad_top < 0 || pad_bottom < 0 || pad_left < 0 || pad_right < 0) return fail(TDX_ERR_INVALID_ARG, "negative padding");
+    if (dtype != TDX_F32 && dtype != TDX_BF16) return fail(TDX_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    const int64_t Hp = H + pad_top + pad_bottom, Wp = W + pad_left + pad_right;
+    const int64_t total = N * Hp * Wp * C;
+    if (total == 0) return TDX_OK;
+    if (y == nullptr || out == nullptr) return fail(TDX_ERR_INVALID_ARG, "y or out is NULL");
+    const int64_t interior = N * H * W * C;
+    if (interior > 0 && x == nullptr) return fail(TDX_ERR_INVALID_ARG, "x is NULL");
+    const uintptr_t el = dtype == TDX_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(x) % el || reinterpret_cast<uintptr_t>(y) % el || reinterpret_cast<uintptr_t>(out) % el)
+        return fail(TDX_ERR_ALIGNMENT, "pointer not aligned to its element size");
+    DeviceCtx* ctx;
+    int rc = get_ctx(&ctx);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const long long row_elems = W * C, y_row = Wp * C, y_img = Hp * Wp * C, y_first = (pad_top * Wp + pad_left) * C;
+    const int per16 = static_cast<int>(16 / el);
+    // 16-byte accesses when every interior row starts on a 16-byte boundary in x, y and out
+    const bool vec_ok = row_elems % per16 == 0 && y_row % per16 == 0 && y_img % per16 == 0 && y_first % per16 == 0 &&
+                        reinterpret_cast<uintptr_t>(x) % 16 == 0 && reinterpret_cast<uintptr_t>(y) % 16 == 0 &&
+                        reinterpret_cast<uintptr_t>(out) % 16 == 0;
+    const int vec = vec_ok ? per16 : 1;
+    const int max_grid = ctx->sm_count * 16;
+    if (out != y) {
+        const int grid = static_cast<int>(std::min<long long>(ceil_div(total, 256), max_grid));
+        if (dtype == TDX_F32)
+            tdx::copy_pad_ring_kernel<float><<<grid, 256, 0, st>>>(total, C, Hp, Wp, pad_top, H, pad_left, W,
+                                                                   static_cast<const float*>(y), static_cast<float*>(out));
+        else
+            tdx::copy_pad_ring_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(total, C, Hp, Wp, pad_top, H, pad_left, W,
+                                                                           static_cast<const __nv_bfloat16*>(y),
+                                                                           static_cast<__nv_bfloat16*>(out));
+        TDX_CUDA(cudaGetLastError());
+        g_launches.fetch_add(1);
+    }
+    if (interior > 0) {
+        const long long work = interior / vec;
+        const int grid = static_cast<int>(std::min<long long>(ceil_div(work, 256), max_grid));
+        if (dtype == TDX_F32)
+            tdx::add_zero_pad_kernel<float><<<grid, 256, 0, st>>>(N * H, H, row_elems, y_img, y_row, y_first, vec,
+                                                                  static_cast<const float*>(x), static_cast<const float*>(y),
+                                                                  static_cast<float*>(out));
+        else
+            tdx::add_zero_pad_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
+                N * H, H, row_elems, y_img, y_row, y_first, vec, static_cast<const __nv_bfloat16*>(x),
+                static_cast<const __nv_bfloat16*>(y), static_cast<__nv_bfloat16*>(out));
+        TDX_CUDA(cudaGetLastError());
+        g_launches.fetch_add(1);
+    }
+    return TDX_OK;
+}
+
 int tdx_gemm_ex(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype, const void* A,
                 const void* B, void* C, void* stream, const tdx_config* cfg, void* workspace, size_t workspace_bytes) {
     // the library's own workspace serves every split-K it chose itself
@@ -1644,6 +1699,32 @@ int tdx_gemm_batched_host(int64_t batch, int64_t M, int64_t N, int64_t K, int tr
     rc = tdx_gemm_batched(batch, M, N, K, transA, transB, alpha, beta, dtype, dA, M * K, dB, K * N, dC, M * N, stream);
     if (rc) return rc;
     TDX_CUDA(cudaMemcpyAsync(C_host, dC, c_bytes, cudaMemcpyDeviceToHost, st));
+    TDX_CUDA(cudaStreamSynchronize(st));
+    return TDX_OK;
+}
+
+int tdx_add_zero_pad_host(int64_t N, int64_t H, int64_t W, int64_t C, int pad_top, int pad_bottom, int pad_left,
+                          int pad_right, int dtype, const void* x_host, void* y_host, void* stream) {
+    if (N < 0 || H < 0 || W < 0 || C < 0 || pad_top < 0 || pad_bottom < 0 || pad_left < 0 || pad_right < 0)
+        return fail(TDX_ERR_INVALID_ARG, "negative dimension or padding");
+    if (dtype != TDX_F32 && dtype != TDX_BF16) return fail(TDX_ERR_INVALID_ARG, "unknown dtype %d", dtype);
+    const size_t el = dtype == TDX_F32 ? 4 : 2;
+    const size_t x_bytes = static_cast<size_t>(N) * H * W * C * el;
+    const size_t y_bytes = static_cast<size_t>(N) * (H + pad_top + pad_bottom) * (W + pad_left + pad_right) * C * el;
+    if (y_bytes == 0) return TDX_OK;
+    if (y_host == nullptr || (x_bytes && x_host == nullptr)) return fail(TDX_ERR_INVALID_ARG, "NULL host pointer");
+    DeviceCtx* ctx;
+    int rc = get_ctx(&ctx);
+    if (rc) return rc;
+    void *dx, *dy;
+    if ((rc = ensure_staging(ctx, 0, x_bytes, &dx))) return rc;
+    if ((rc = ensure_staging(ctx, 1, y_bytes, &dy))) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (x_bytes) TDX_CUDA(cudaMemcpyAsync(dx, x_host, x_bytes, cudaMemcpyHostToDevice, st));
+    TDX_CUDA(cudaMemcpyAsync(dy, y_host, y_bytes, cudaMemcpyHostToDevice, st));
+    rc = tdx_add_zero_pad(N, H, W, C, pad_top, pad_bottom, pad_left, pad_right, dtype, dx, dy, dy, stream);
+    if (rc) return rc;
+    TDX_CUDA(cudaMemcpyAsync(y_host, dy, y_bytes, cudaMemcpyDeviceToHost, st));
     TDX_CUDA(cudaStreamSynchronize(st));
     return TDX_OK;
 }
