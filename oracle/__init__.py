@@ -54,6 +54,8 @@ def _load():
         lib.oracle_add_zero_pad.restype = ctypes.c_int
         lib.oracle_conv2d.argtypes = [i64] * 9 + [ctypes.c_int, p, p, p, ctypes.c_int, p, i64, p]
         lib.oracle_conv2d.restype = ctypes.c_int
+        lib.oracle_conv2d_residual.argtypes = [i64] * 9 + [ctypes.c_int, p, p, p, p, ctypes.c_int, p, i64, p]
+        lib.oracle_conv2d_residual.restype = ctypes.c_int
         lib.oracle_conv_out_dim.argtypes = [i64] * 4
         lib.oracle_conv_out_dim.restype = i64
         lib.oracle_round_bf16.argtypes = [p, i64, p]
@@ -152,8 +154,9 @@ def conv_out_dim(H, R, pad, stride) -> int:
     return int(_load().oracle_conv_out_dim(H, R, pad, stride))
 
 
-def conv2d(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, relu, rows=None) -> np.ndarray:
-    """fp64 reference of y = relu?(conv(x, w) + bias); returns (rows or N*P*Q) x Cout."""
+def conv2d(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, relu, rows=None, residual=None) -> np.ndarray:
+    """fp64 reference of y = relu?(conv(x, w) + bias [+ residual]); returns (rows or N*P*Q) x Cout.
+    residual, if given, is N*P*Q x Cout in the storage type of x."""
     lib, dt = _load(), _DT[dtype]
     x = _check(x, dt, N * H * W * Cin, "x")
     w = _check(w, dt, Cout * R * S * Cin, "w")
@@ -170,8 +173,13 @@ def conv2d(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, relu, rows=
             raise ValueError("row index out of range")
         nr, rp = rows_arr.size, rows_arr.ctypes.data
     out = np.empty((nr, Cout), dtype=np.float64)
-    rc = lib.oracle_conv2d(N, H, W, Cin, Cout, R, S, pad, stride, dt, x.ctypes.data, w.ctypes.data,
-                           bp, int(relu), rp, nr, out.ctypes.data)
+    if residual is not None:
+        residual = _check(residual, dt, N * P * Q * Cout, "residual")
+        rc = lib.oracle_conv2d_residual(N, H, W, Cin, Cout, R, S, pad, stride, dt, x.ctypes.data, w.ctypes.data,
+                                        bp, residual.ctypes.data, int(relu), rp, nr, out.ctypes.data)
+    else:
+        rc = lib.oracle_conv2d(N, H, W, Cin, Cout, R, S, pad, stride, dt, x.ctypes.data, w.ctypes.data,
+                               bp, int(relu), rp, nr, out.ctypes.data)
     if rc:
         raise RuntimeError(f"oracle_conv2d failed ({rc})")
     return out

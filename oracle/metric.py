@@ -49,7 +49,7 @@ def gemm_batched_row_scales(batch, M, N, K, transA, transB, alpha, beta, dtype, 
     return s.reshape(-1)
 
 
-def conv_row_scales(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, rows=None) -> np.ndarray:
+def conv_row_scales(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, rows=None, residual=None) -> np.ndarray:
     xe = decode(x, dtype).reshape(N, H, W, Cin)
     energy = (xe * xe).sum(axis=3)                                   # per input pixel
     ep = np.zeros((N, H + 2 * pad, W + 2 * pad))
@@ -64,6 +64,8 @@ def conv_row_scales(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, ro
     wmax = np.sqrt((wd * wd).sum(axis=1)).max()
     bmax = 0.0 if bias is None else float(np.abs(np.asarray(bias, dtype=np.float64)).max())
     sc = (np.sqrt(acc) * wmax + bmax).reshape(-1)
+    if residual is not None:                                          # + max_k |residual[row, k]|
+        sc = sc + np.abs(decode(residual, dtype).reshape(-1, Cout)).max(axis=1)
     return sc if rows is None else sc[np.asarray(rows, dtype=np.int64)]
 
 

@@ -146,10 +146,36 @@ int64_t oracle_conv_out_dim(int64_t H, int64_t R, int64_t pad, int64_t stride)
  * added last, so it is independent of the reduction.
  * rows == NULL: all N*P*Q rows; else the listed rows.  out: nrows_eff x Cout.
  */
+static int conv2d_impl(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
+                       int64_t pad, int64_t stride, int dtype, const void *x, const void *w,
+                       const float *bias, const void *residual, int relu,
+                       const int64_t *rows, int64_t nrows, double *out);
+
 int oracle_conv2d(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
                   int64_t pad, int64_t stride, int dtype, const void *x, const void *w,
                   const float *bias, int relu,
                   const int64_t *rows, int64_t nrows, double *out)
+{
+    return conv2d_impl(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, NULL, relu, rows, nrows, out);
+}
+
+/*
+ * The same with a residual term (the shortcut of a ResNet block, the network the paper's workload comes from):
+ *   y_ref[row, k] = relu?( conv(x, w)[row, k] + bias[k] + residual[row, k] )
+ * residual is N*P*Q x Cout in the storage type of x; it joins the sum after the bias and before the ReLU.
+ */
+int oracle_conv2d_residual(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
+                           int64_t pad, int64_t stride, int dtype, const void *x, const void *w,
+                           const float *bias, const void *residual, int relu,
+                           const int64_t *rows, int64_t nrows, double *out)
+{
+    return conv2d_impl(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, residual, relu, rows, nrows, out);
+}
+
+static int conv2d_impl(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
+                       int64_t pad, int64_t stride, int dtype, const void *x, const void *w,
+                       const float *bias, const void *residual, int relu,
+                       const int64_t *rows, int64_t nrows, double *out)
 {
     int64_t P = oracle_conv_out_dim(H, R, pad, stride);
     int64_t Q = oracle_conv_out_dim(W, S, pad, stride);
@@ -174,6 +200,7 @@ int oracle_conv2d(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, in
                 }
             }
             if (bias) acc += (double)bias[k];
+            if (residual) acc += load_elem(residual, row * Cout + k, dtype);
             if (relu && acc < 0.0) acc = 0.0;
             out[rr * Cout + k] = acc;
         }

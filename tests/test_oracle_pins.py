@@ -306,6 +306,29 @@ def test_conv_bias_relu():
     assert np.allclose(lin - nob, b.astype(np.float64)[None, :], rtol=0, atol=1e-12)
 
 
+def test_conv_residual_joins_before_the_relu():
+    N, H, W, Cin, Cout = 2, 5, 6, 3, 4
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=19)
+    xf, wf = si.bf16_bits_to_f32(x), si.bf16_bits_to_f32(w)
+    res = si.uniform(19, 3, (N * H * W, Cout), "f32", scale=2.0)
+    pre = oracle.conv2d(N, H, W, Cin, Cout, 3, 3, 1, 1, "f32", xf, wf, b, 0)
+    # without ReLU the residual is a plain elementwise addend; with it, the ReLU sees the sum (not relu(conv) + residual)
+    assert np.array_equal(oracle.conv2d(N, H, W, Cin, Cout, 3, 3, 1, 1, "f32", xf, wf, b, 0, residual=res),
+                          pre + res.astype(np.float64))
+    out = oracle.conv2d(N, H, W, Cin, Cout, 3, 3, 1, 1, "f32", xf, wf, b, 1, residual=res)
+    assert np.array_equal(out, np.maximum(pre + res.astype(np.float64), 0.0)) and (out >= 0).all()
+    assert not np.array_equal(out, np.maximum(pre, 0.0) + res.astype(np.float64))
+    # zero weights and bias: y = relu(residual); a zero residual changes nothing
+    z = np.zeros_like(wf)
+    assert np.array_equal(oracle.conv2d(N, H, W, Cin, Cout, 3, 3, 1, 1, "f32", xf, z, None, 1, residual=res),
+                          np.maximum(res.astype(np.float64), 0.0))
+    assert np.array_equal(oracle.conv2d(N, H, W, Cin, Cout, 3, 3, 1, 1, "f32", xf, wf, b, 1, residual=np.zeros_like(res)),
+                          oracle.conv2d(N, H, W, Cin, Cout, 3, 3, 1, 1, "f32", xf, wf, b, 1))
+    # row subsets index the residual by output row
+    rows = np.array([0, 7, 31, N * H * W - 1])
+    assert np.array_equal(oracle.conv2d(N, H, W, Cin, Cout, 3, 3, 1, 1, "f32", xf, wf, b, 1, rows=rows, residual=res), out[rows])
+
+
 def test_conv_linear_in_input_without_bias_and_relu():
     N, H, W, Cin, Cout = 1, 5, 5, 2, 2
     x1 = si.small_integers(37, 0, (N, H, W, Cin), "f32")
