@@ -175,6 +175,16 @@ int tdx_conv2d_bias_relu(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t C
                          int pad, int stride, int dtype, const void* x, const void* w, const float* bias,
                          int relu, void* y, void* stream);
 
+/*
+ * The same with a residual term: y = relu?( conv(x, w) + bias + residual ), the closing step of a ResNet block
+ * (the network the paper's workload is a layer of).  residual is N x P x Q x Cout in the type of y (NULL: none); it
+ * joins the fp32 sum after the bias and before the ReLU, fused into the epilogue.  It must not overlap y.
+ * cfg: NULL = choose, else as for tdx_conv2d_bias_relu_ex.
+ */
+int tdx_conv2d_bias_add_relu(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
+                             int pad, int stride, int dtype, const void* x, const void* w, const float* bias,
+                             const void* residual, int relu, void* y, void* stream, const tdx_config* cfg);
+
 /* As above with an explicit configuration (split_k must be 1).  Infeasible cfg -> CONFIG, y untouched. */
 int tdx_conv2d_bias_relu_ex(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
                             int pad, int stride, int dtype, const void* x, const void* w, const float* bias,

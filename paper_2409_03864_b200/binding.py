@@ -76,6 +76,7 @@ def lib() -> ctypes.CDLL:
         L.tdx_gemm_workspace_size.argtypes = [i64, i64, i64, ci, cfgp, ctypes.POINTER(sz)]
         L.tdx_conv2d_bias_relu.argtypes = conv_args
         L.tdx_conv2d_bias_relu_ex.argtypes = conv_args + [cfgp]
+        L.tdx_conv2d_bias_add_relu.argtypes = [i64] * 7 + [ci, ci, ci, vp, vp, vp, vp, ci, vp, vp, cfgp]
         L.tdx_gemm_host.argtypes = gemm_args
         L.tdx_conv2d_bias_relu_host.argtypes = conv_args
         L.tdx_tune_gemm.argtypes = [i64, i64, i64, ci, ci, ci, ci, cfgp, fp, cfgp, fp, ci, ip, vp]
@@ -111,7 +112,7 @@ def lib() -> ctypes.CDLL:
 
 # every symbol include/tdx.h declares
 EXPORTS = (
-    "tdx_gemm", "tdx_add_zero_pad", "tdx_add_zero_pad_host", "tdx_gemm_batched", "tdx_gemm_batched_host", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_relu_ex",
+    "tdx_gemm", "tdx_add_zero_pad", "tdx_add_zero_pad_host", "tdx_gemm_batched", "tdx_gemm_batched_host", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_add_relu", "tdx_conv2d_bias_relu_ex",
     "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
     "tdx_enum_conv2d_configs", "tdx_default_gemm_config", "tdx_default_conv2d_config", "tdx_tune_save",
     "tdx_tune_load", "tdx_tune_clear", "tdx_gemm_tile_plan", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
@@ -205,6 +206,13 @@ def tdx_gemm_workspace_size(M, N, K, dtype, cfg):
 def tdx_conv2d_bias_relu(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, relu, y, stream=None) -> int:
     return lib().tdx_conv2d_bias_relu(N, H, W, Cin, Cout, R, S, pad, stride, dtype, _ptr(x), _ptr(w), _ptr(bias),
                                       relu, _ptr(y), _stream(stream))
+
+
+def tdx_conv2d_bias_add_relu(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, residual, relu, y, stream=None,
+                             cfg=None) -> int:
+    """y = relu?(conv(x, w) + bias + residual); residual is N*P*Q x Cout in the type of y, or None."""
+    return lib().tdx_conv2d_bias_add_relu(N, H, W, Cin, Cout, R, S, pad, stride, dtype, _ptr(x), _ptr(w), _ptr(bias),
+                                          _ptr(residual), relu, _ptr(y), _stream(stream), _cfg(cfg))
 
 
 def tdx_conv2d_bias_relu_ex(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, relu, y, stream=None,

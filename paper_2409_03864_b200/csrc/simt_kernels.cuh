@@ -286,7 +286,8 @@ __global__ void gemm_generic_kernel(long long M, long long N, long long K, long 
 template <typename TIn, typename TOut>
 __global__ void conv2d_generic_kernel(int Nimg, int H, int W, int Cin, int Cout, int R, int S, int pad, int stride,
                                       int P, int Q, const TIn* __restrict__ x, const TIn* __restrict__ w,
-                                      const float* __restrict__ bias, int relu, TOut* __restrict__ y) {
+                                      const float* __restrict__ bias, int relu, TOut* __restrict__ y,
+                                      const TOut* __restrict__ residual = nullptr) {
     const long long total = static_cast<long long>(Nimg) * P * Q * Cout;
     for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < total;
          e += static_cast<long long>(gridDim.x) * blockDim.x) {
@@ -309,6 +310,7 @@ __global__ void conv2d_generic_kernel(int Nimg, int H, int W, int Cin, int Cout,
             }
         }
         if (bias != nullptr) acc += __ldg(bias + k);
+        if (residual != nullptr) acc += as_float(residual[e]);
         if (relu) acc = fmaxf(acc, 0.0f);
         st_from_float(y, e, acc);
     }

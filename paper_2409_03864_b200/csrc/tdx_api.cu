@@ -841,7 +841,7 @@ int run_gemm_pair(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
 }
 
 int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const void* w, const float* bias, int relu,
-                  void* y, const tdx_config& cfg, cudaStream_t st) {
+                  void* y, const tdx_config& cfg, cudaStream_t st, const void* residual = nullptr) {
     const int cchunks = static_cast<int>(ceil_div(c.Cin, 64));
     UmmaParams p;
     std::memset(&p, 0, sizeof p);
@@ -899,6 +899,7 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     p.b_mn_major = 0;
     p.alpha = 1.0f;
     p.bias = bias;
+    p.residual = static_cast<const __nv_bfloat16*>(residual);
     p.relu = relu;
     p.C = static_cast<__nv_bfloat16*>(y);
     p.ldc = c.Cout;
@@ -942,6 +943,8 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     }
     CUtensorMap mc = ma, mc_row = ma;
     p.tma_store = (cfg.store_mode == 2 && p.vec_store && p.bw * p.bh >= 32) ? 1 : 0;
+    // the staged epilogue reads the residual 16 bytes at a time
+    if (reinterpret_cast<uintptr_t>(residual) % 16) p.tma_store = 0;
     if (halo) p.epi_warps = p.tma_store ? 16 : 4 * (cfg.tile_m / 128);
     if (p.tma_store) {
         p.sbx = std::min(p.bw, 32);
@@ -1030,7 +1033,7 @@ int run_gemm_generic(DeviceCtx* ctx, const GemmProblem& g, float alpha, const vo
 }
 
 int run_conv_generic(DeviceCtx* ctx, const ConvProblem& c, const void* x, const void* w, const float* bias, int relu,
-                     void* y, cudaStream_t st) {
+                     void* y, cudaStream_t st, const void* residual = nullptr) {
     if (c.N >= (1LL << 31) || c.H >= (1LL << 31) || c.W >= (1LL << 31) || c.Cin >= (1LL << 31) ||
         c.Cout >= (1LL << 31) || c.R >= (1LL << 31) || c.S >= (1LL << 31))
         return fail(TDX_ERR_UNSUPPORTED, "conv dimensions must be below 2^31");
@@ -1039,12 +1042,13 @@ int run_conv_generic(DeviceCtx* ctx, const ConvProblem& c, const void* x, const 
     if (c.dtype == TDX_F32)
         tdx::conv2d_generic_kernel<float, float><<<grid, 256, 0, st>>>(
             (int)c.N, (int)c.H, (int)c.W, (int)c.Cin, (int)c.Cout, (int)c.R, (int)c.S, c.pad, c.stride, (int)c.P,
-            (int)c.Q, static_cast<const float*>(x), static_cast<const float*>(w), bias, relu, static_cast<float*>(y));
+            (int)c.Q, static_cast<const float*>(x), static_cast<const float*>(w), bias, relu, static_cast<float*>(y),
+            static_cast<const float*>(residual));
     else
         tdx::conv2d_generic_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
             (int)c.N, (int)c.H, (int)c.W, (int)c.Cin, (int)c.Cout, (int)c.R, (int)c.S, c.pad, c.stride, (int)c.P,
             (int)c.Q, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w), bias, relu,
-            static_cast<__nv_bfloat16*>(y));
+            static_cast<__nv_bfloat16*>(y), static_cast<const __nv_bfloat16*>(residual));
     TDX_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     return TDX_OK;
@@ -1262,10 +1266,12 @@ int gemm_dispatch(int64_t M, int64_t N, int64_t K, int transA, int transB, float
 
 int conv_dispatch(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad, int stride,
                   int dtype, const void* x, const void* w, const float* bias, int relu, void* y, void* stream,
-                  const tdx_config* cfg) {
+                  const tdx_config* cfg, const void* residual = nullptr) {
     ConvProblem cp;
     int rc = validate_conv(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, y, relu, true, &cp);
     if (rc) return rc;
+    if (reinterpret_cast<uintptr_t>(residual) % (dtype == TDX_F32 ? 4 : 2))
+        return fail(TDX_ERR_ALIGNMENT, "residual not aligned to its element size");
     if (N == 0 || Cout == 0 || cp.P == 0 || cp.Q == 0) return TDX_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int sm_count, smem_limit;
@@ -1281,12 +1287,12 @@ int conv_dispatch(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, in
     tdx_config c;
     rc = resolve_conv_config(cp, cfg, ctx->sm_count, ctx->smem_optin, &c);
     if (rc) return rc;
-    if (c.kernel == TDX_KERNEL_GENERIC) return run_conv_generic(ctx, cp, x, w, bias, relu, y, st);
+    if (c.kernel == TDX_KERNEL_GENERIC) return run_conv_generic(ctx, cp, x, w, bias, relu, y, st, residual);
     if (reinterpret_cast<uintptr_t>(x) % 16 || reinterpret_cast<uintptr_t>(w) % 16) {
         if (cfg && cfg->kernel == TDX_KERNEL_UMMA) return fail(TDX_ERR_ALIGNMENT, "tensor-core path needs 16-byte aligned x and w");
-        return run_conv_generic(ctx, cp, x, w, bias, relu, y, st);
+        return run_conv_generic(ctx, cp, x, w, bias, relu, y, st, residual);
     }
-    return run_conv_umma(ctx, cp, x, w, bias, relu, y, c, st);
+    return run_conv_umma(ctx, cp, x, w, bias, relu, y, c, st, residual);
 }
 
 // ------------------------------------------------------------------ search space
@@ -1643,6 +1649,12 @@ int tdx_conv2d_bias_relu(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t C
                          int stride, int dtype, const void* x, const void* w, const float* bias, int relu, void* y,
                          void* stream) {
     return conv_dispatch(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, relu, y, stream, nullptr);
+}
+
+int tdx_conv2d_bias_add_relu(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
+                             int stride, int dtype, const void* x, const void* w, const float* bias, const void* residual,
+                             int relu, void* y, void* stream, const tdx_config* cfg) {
+    return conv_dispatch(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, relu, y, stream, cfg, residual);
 }
 
 int tdx_conv2d_bias_relu_ex(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,

@@ -52,6 +52,7 @@ struct UmmaParams {
     float alpha;
     float beta;               // GEMM with accumulate: out = alpha * acc + beta * (what C held); direct stores only
     const float* bias;        // [N] or nullptr
+    const __nv_bfloat16* residual;   // convolution: [M][N] added after the bias and before the ReLU, or nullptr
     int relu;
     __nv_bfloat16* C;         // bf16 output, row pitch ldc elements
     long long ldc;
@@ -288,7 +289,7 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
             // 64-byte swizzle of the staging block: 16-byte slot c of row `lane` lives at slot c ^ ((lane / 2) % 4)
             uint8_t* my_row = stage_buf + lane * 64;
             const int sw = (lane >> 1) & 3;
-            const bool plain = (p.bias == nullptr) && (p.relu == 0);
+            const bool plain = (p.bias == nullptr) && (p.relu == 0) && (p.residual == nullptr);
             for (int c0 = cgrp * 32; c0 < t.bn; c0 += ncgrp * 32) {
                 uint32_t r[32];
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
@@ -300,6 +301,26 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                 float bias_l = 0.0f;
                 if (p.bias != nullptr) bias_l = __ldg(p.bias + min(col0 + lane, p.N - 1));
                 ptx::tmem_ld_wait();
+                if (kConv && p.residual != nullptr) {
+                    // residual term (convolution only, where alpha is 1): this thread's 32 values of its output row
+                    // (64 bytes; the staged epilogue implies N % 8 == 0) join the accumulators before bias and ReLU
+                    if (valid) {
+                        const uint4* rp = reinterpret_cast<const uint4*>(p.residual + grow * p.ldc + col0);
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            if (col0 + g * 8 < p.N) {
+                                const uint4 v = __ldg(rp + g);
+                                const uint32_t rw[4] = {v.x, v.y, v.z, v.w};      // two bf16 values each
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const int j = g * 8 + e * 2;
+                                    r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(rw[e] << 16));
+                                    r[j + 1] = __float_as_uint(__uint_as_float(r[j + 1]) + __uint_as_float(rw[e] & 0xFFFF0000u));
+                                }
+                            }
+                        }
+                    }
+                }
                 // the previous store of this warp must have finished reading the staging block
                 if (lane < nstore) ptx::tma_store_wait_read<0>();
                 __syncwarp();
@@ -378,6 +399,7 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                     if (p.beta != 0.0f && col0 + j < p.N)
                         x = fmaf(p.beta, __bfloat162float(p.C[grow * p.ldc + col0 + j]), x);
                     if (p.bias != nullptr && col0 + j < p.N) x += __ldg(p.bias + col0 + j);
+                    if (p.residual != nullptr && col0 + j < p.N) x += __bfloat162float(p.residual[grow * p.ldc + col0 + j]);
                     if (p.relu) x = fmaxf(x, 0.0f);
                     v[j] = x;
                 }

@@ -6,7 +6,7 @@ import torch
 import oracle
 import paper_2409_03864_b200 as tdx
 import seeded_inputs as si
-from gpu_util import TIGHT, TOL, conv_error, run_conv, structured_rows
+from gpu_util import TIGHT, TOL, GuardedOut, conv_error, run_conv, structured_rows, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -274,3 +274,39 @@ def test_full_size_conv_56x56x256():
     assert err < TOL["bf16"] and err < TIGHT["bf16"], err
     assert (oracle.decode(y[::53], "bf16") >= 0).all()
     assert tdx.tdx_check_device_status() == 0
+
+
+RESIDUAL_CASES = [
+    # N, H,  W,  Cin, Cout, R, S, pad, stride, cfg
+    (2, 56, 56, 64, 64, 3, 3, 1, 1, None),                          # automatic: halo reuse over stacked images
+    (3, 20, 36, 72, 40, 3, 3, 1, 1, dict(halo=2, tile_m=256)),      # ragged patches, channel tail
+    (2, 28, 28, 128, 256, 1, 1, 0, 1, None),                        # 1 x 1: per-tap kernel
+    (2, 30, 30, 64, 128, 3, 3, 1, 2, None),                         # strided
+    (2, 16, 24, 64, 64, 3, 3, 1, 1, dict(store_mode=1)),            # direct-store epilogue
+    (1, 9, 11, 5, 7, 3, 3, 1, 1, None),                             # generic kernel (Cin % 8 != 0)
+]
+
+
+@pytest.mark.parametrize("case", RESIDUAL_CASES)
+@pytest.mark.parametrize("relu", [0, 1])
+def test_conv_with_residual_term_vs_oracle(case, relu):
+    N, H, W, Cin, Cout, R, S, pad, stride, cfgkw = case
+    P, Q = oracle.conv_out_dim(H, R, pad, stride), oracle.conv_out_dim(W, S, pad, stride)
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, R, S, seed=85)
+    res = si.normal(85, 3, (N * P * Q, Cout), "bf16", sigma=2.0)
+    dx, dw, db, dres = to_dev(x), to_dev(w), to_dev(b), to_dev(res)
+    out = GuardedOut(N * P * Q * Cout, "bf16")
+    st = tdx.tdx_conv2d_bias_add_relu(N, H, W, Cin, Cout, R, S, pad, stride, tdx.TDX_BF16, dx, dw, db, dres, relu, out.ptr,
+                                      cfg=None if cfgkw is None else umma(**cfgkw))
+    torch.cuda.synchronize()
+    assert st == 0 and out.guards_intact(), tdx.tdx_last_error()
+    got = oracle.decode(out.payload().reshape(N * P * Q, Cout), "bf16")
+    ref = oracle.conv2d(N, H, W, Cin, Cout, R, S, pad, stride, "bf16", x, w, b, relu, residual=res)
+    sc = oracle.conv_row_scales(N, H, W, Cin, Cout, R, S, pad, stride, "bf16", x, w, b, residual=res)
+    err = oracle.max_normalised_error(got, ref, sc)
+    assert err < TIGHT["bf16"], err
+    if relu:
+        assert (got >= 0).all()
+    # the residual really entered: the result differs from the plain convolution
+    st, y_plain, _ = run_conv(N, H, W, Cin, Cout, R, S, pad, stride, "bf16", x, w, b, relu)
+    assert st == 0 and not np.array_equal(oracle.decode(y_plain, "bf16"), got)
