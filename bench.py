@@ -353,7 +353,7 @@ def run_tdx(args):
             h_out.copy_(h_in[2].reshape(-1))
             return tdx.tdx_gemm_batched_host(w["batch"], w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], w["beta"], DT,
                                              h_in[0], h_in[1], h_out, stream)
-        kernel_name = "sgemm_tiled_kernel / sgemm_small_kernel (fp32 CUDA cores)"
+        kernel_name = "sgemm_small_kernel (fp32 CUDA cores, batch in grid.z)"
     elif w["kind"] == "gemm":
         st_cfg, cfg = tdx.tdx_default_gemm_config(w["M"], w["N"], w["K"], w["tA"], w["tB"], DT)
 
@@ -363,7 +363,7 @@ def run_tdx(args):
         def launch_host():
             return tdx.tdx_gemm_host(w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], DT, h_in[0], h_in[1], h_out,
                                      stream)
-        kernel_name = "sgemm_tiled_kernel" if wl.dtype == "f32" else "umma_contract_kernel<false>"
+        kernel_name = "sgemm_small_rowmajor_kernel" if wl.dtype == "f32" else "umma_contract_kernel<false>"
     else:
         cargs = (w["N"], w["H"], w["W"], w["Cin"], w["Cout"], w["R"], w["S"], w["pad"], w["stride"], DT)
         st_cfg, cfg = tdx.tdx_default_conv2d_config(*cargs)

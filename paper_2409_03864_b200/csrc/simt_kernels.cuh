@@ -20,81 +20,11 @@ __device__ __forceinline__ void st_from_float(__nv_bfloat16* p, long long i, flo
 }
 
 // ---------------------------------------------------------------------------
-// fp32 tiled GEMM: C = alpha * op(A) op(B), element (i,k) of op(A) at A[i*sa_i + k*sa_k],
-// element (k,j) of op(B) at B[k*sb_k + j*sb_j].  Each thread owns a TM x TN register tile;
-// the reduction runs k = 0..K-1 in order with fp32 FMAs.
-// ---------------------------------------------------------------------------
-template <int BM, int BN, int BK, int TM, int TN>
-__global__ void __launch_bounds__((BM / TM) * (BN / TN))
-sgemm_tiled_kernel(int M, int N, int K, long long sa_i, long long sa_k, long long sb_k, long long sb_j, float alpha,
-                   const float* __restrict__ A, const float* __restrict__ B, float* __restrict__ C, float beta = 0.0f,
-                   long long batch_a = 0, long long batch_b = 0, long long batch_c = 0) {
-    constexpr int NT = (BM / TM) * (BN / TN);
-    // batch = blockIdx.z; C = beta * C + alpha * A . B (C is not read when beta == 0)
-    A += blockIdx.z * batch_a;
-    B += blockIdx.z * batch_b;
-    C += blockIdx.z * batch_c;
-    __shared__ float As[BK][BM + 4];
-    __shared__ float Bs[BK][BN + 4];
-    const int tid = threadIdx.x;
-    const int tx = tid % (BN / TN);
-    const int ty = tid / (BN / TN);
-    const int m0 = blockIdx.y * BM;
-    const int n0 = blockIdx.x * BN;
-    float acc[TM][TN];
-#pragma unroll
-    for (int i = 0; i < TM; ++i)
-#pragma unroll
-        for (int j = 0; j < TN; ++j) acc[i][j] = 0.0f;
-
-    for (int k0 = 0; k0 < K; k0 += BK) {
-        for (int idx = tid; idx < BM * BK; idx += NT) {
-            int i, k;
-            if (sa_k == 1) { i = idx / BK; k = idx % BK; } else { i = idx % BM; k = idx / BM; }
-            const int gi = m0 + i, gk = k0 + k;
-            As[k][i] = (gi < M && gk < K) ? __ldg(A + gi * sa_i + gk * sa_k) : 0.0f;
-        }
-        for (int idx = tid; idx < BN * BK; idx += NT) {
-            int j, k;
-            if (sb_j == 1) { k = idx / BN; j = idx % BN; } else { j = idx / BK; k = idx % BK; }
-            const int gj = n0 + j, gk = k0 + k;
-            Bs[k][j] = (gj < N && gk < K) ? __ldg(B + gk * sb_k + gj * sb_j) : 0.0f;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int k = 0; k < BK; ++k) {
-            float a[TM], b[TN];
-#pragma unroll
-            for (int i = 0; i < TM; ++i) a[i] = As[k][ty * TM + i];
-#pragma unroll
-            for (int j = 0; j < TN; ++j) b[j] = Bs[k][tx * TN + j];
-#pragma unroll
-            for (int i = 0; i < TM; ++i)
-#pragma unroll
-                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
-        }
-        __syncthreads();
-    }
-#pragma unroll
-    for (int i = 0; i < TM; ++i) {
-        const int gi = m0 + ty * TM + i;
-        if (gi >= M) continue;
-#pragma unroll
-        for (int j = 0; j < TN; ++j) {
-            const int gj = n0 + tx * TN + j;
-            if (gj < N) {
-                float* c = C + static_cast<long long>(gi) * N + gj;
-                *c = beta != 0.0f ? fmaf(beta, *c, alpha * acc[i][j]) : alpha * acc[i][j];
-            }
-        }
-    }
-}
-
-// ---------------------------------------------------------------------------
-// fp32 GEMM for small problems: 32 x 32 tiles, 2 x 2 outputs per thread, and a 4-stage cp.async ring so
-// that the global-load latency of K-tile t+3 hides behind the FMAs of tile t (a small problem has too few
-// CTAs per SM to hide it any other way).  Same index maps and the same k-ascending fp32 FMA order as
-// sgemm_tiled_kernel.
+// fp32 GEMM, C = beta * C + alpha * op(A) op(B): element (i,k) of op(A) at A[i*sa_i + k*sa_k], element (k,j) of
+// op(B) at B[k*sb_k + j*sb_j]; the reduction runs k = 0..K-1 in order with fp32 FMAs; batch = blockIdx.z.
+// For small problems: 32 x 32 tiles, 2 x 2 outputs per thread, and a 4-stage cp.async ring so that the
+// global-load latency of K-tile t+3 hides behind the FMAs of tile t (a small problem has too few CTAs per SM
+// to hide it any other way).
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ void cp_async_f32(float* smem_dst, const float* gmem_src, bool valid) {
     const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
@@ -171,6 +101,94 @@ sgemm_small_kernel(int M, int N, int K, long long sa_i, long long sa_k, long lon
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
             const int gj = n0 + tx * 2 + j;
+            if (gj < N) {
+                float* c = C + static_cast<long long>(gi) * N + gj;
+                *c = beta != 0.0f ? fmaf(beta, *c, alpha * acc[i][j]) : alpha * acc[i][j];
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// The same ring with larger tiles: BM x BN per CTA, TM x TN outputs per thread, ST stages of BK.  A TM x TN register
+// tile needs (TM + TN) shared-memory reads for TM * TN FMAs (4 x 4: 2 FMAs per read, where the 2 x 2 tile of the
+// small kernel has 1), so this is the kernel for problems that offer at least one 64 x 64 tile per SM.
+// Same index maps, batch / beta handling and k-ascending fp32 FMA order as above.
+// ---------------------------------------------------------------------------
+template <int BM, int BN, int BK, int TM, int TN, int ST>
+__global__ void __launch_bounds__((BM / TM) * (BN / TN))
+sgemm_ring_kernel(int M, int N, int K, long long sa_i, long long sa_k, long long sb_k, long long sb_j, float alpha,
+                  const float* __restrict__ A, const float* __restrict__ B, float* __restrict__ C, float beta,
+                  long long batch_a, long long batch_b, long long batch_c) {
+    constexpr int NT = (BM / TM) * (BN / TN);
+    static_assert(TM == 4 && TN == 4, "register tile is read with one 16-byte load per operand");
+    static_assert((BM * BK) % NT == 0 && (BN * BK) % NT == 0, "whole number of copies per thread");
+    A += blockIdx.z * batch_a;
+    B += blockIdx.z * batch_b;
+    C += blockIdx.z * batch_c;
+    __shared__ __align__(16) float As[ST][BK][BM + 4];
+    __shared__ __align__(16) float Bs[ST][BK][BN + 4];
+    const int tid = threadIdx.x;
+    const int tx = tid % (BN / TN), ty = tid / (BN / TN);
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int ktiles = (K + BK - 1) / BK;
+
+    auto load_tile = [&](int kt, int st) {
+        const int k0 = kt * BK;
+#pragma unroll
+        for (int e = 0; e < (BM * BK) / NT; ++e) {
+            const int idx = tid + e * NT;
+            int i, k;
+            if (sa_k == 1) { i = idx / BK; k = idx % BK; } else { i = idx % BM; k = idx / BM; }
+            const int gi = m0 + i, gk = k0 + k;
+            const bool ok = gi < M && gk < K;
+            cp_async_f32(&As[st][k][i], A + (ok ? gi * sa_i + gk * sa_k : 0), ok);
+        }
+#pragma unroll
+        for (int e = 0; e < (BN * BK) / NT; ++e) {
+            const int idx = tid + e * NT;
+            int j, k;
+            if (sb_j == 1) { k = idx / BN; j = idx % BN; } else { j = idx / BK; k = idx % BK; }
+            const int gj = n0 + j, gk = k0 + k;
+            const bool ok = gj < N && gk < K;
+            cp_async_f32(&Bs[st][k][j], B + (ok ? gk * sb_k + gj * sb_j : 0), ok);
+        }
+    };
+
+    for (int s = 0; s < ST - 1; ++s) {
+        if (s < ktiles) load_tile(s, s);
+        cp_async_commit();
+    }
+    float acc[TM][TN];
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) acc[i][j] = 0.0f;
+    for (int kt = 0; kt < ktiles; ++kt) {
+        cp_async_wait<ST - 2>();
+        __syncthreads();                               // tile kt has landed; everyone is done with tile kt-1
+        if (kt + ST - 1 < ktiles) load_tile(kt + ST - 1, (kt + ST - 1) % ST);
+        cp_async_commit();
+        const int st = kt % ST;
+#pragma unroll
+        for (int k = 0; k < BK; ++k) {
+            const float4 a4 = *reinterpret_cast<const float4*>(&As[st][k][ty * TM]);
+            const float4 b4 = *reinterpret_cast<const float4*>(&Bs[st][k][tx * TN]);
+            const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
+#pragma unroll
+            for (int i = 0; i < TM; ++i)
+#pragma unroll
+                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+    }
+    cp_async_wait<0>();
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+        const int gi = m0 + ty * TM + i;
+        if (gi >= M) continue;
+#pragma unroll
+        for (int j = 0; j < TN; ++j) {
+            const int gj = n0 + tx * TN + j;
             if (gj < N) {
                 float* c = C + static_cast<long long>(gi) * N + gj;
                 *c = beta != 0.0f ? fmaf(beta, *c, alpha * acc[i][j]) : alpha * acc[i][j];

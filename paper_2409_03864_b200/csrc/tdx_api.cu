@@ -10,6 +10,7 @@
 #include <atomic>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <functional>
@@ -991,11 +992,13 @@ int run_gemm_simt_f32(DeviceCtx* ctx, const GemmProblem& g, float alpha, const v
     if (ba.batch > 65535) return fail(TDX_ERR_UNSUPPORTED, "fp32 batched GEMM takes at most 65535 batches");
     const unsigned nz = static_cast<unsigned>(ba.batch);
     const bool plain = ba.batch == 1 && ba.beta == 0.0f;
-    if (ceil_div(g.M, 64) * ceil_div(g.N, 64) * ba.batch >= ctx->sm_count) {
+    const int64_t tiles64 = ceil_div(g.M, 64) * ceil_div(g.N, 64) * ba.batch;
+    if (tiles64 >= ctx->sm_count) {
+        // 64 x 64 tiles (4 x 4 outputs per thread) once there is one per SM; smaller problems take 32 x 32 tiles
         dim3 grid(static_cast<unsigned>(ceil_div(g.N, 64)), static_cast<unsigned>(ceil_div(g.M, 64)), nz);
-        tdx::sgemm_tiled_kernel<64, 64, 16, 4, 4><<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k,
-                                                                       sb_j, alpha, a, b, c, ba.beta, ba.stride_a,
-                                                                       ba.stride_b, ba.stride_c);
+        tdx::sgemm_ring_kernel<64, 64, 16, 4, 4, 4><<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k,
+                                                                         sb_j, alpha, a, b, c, ba.beta, ba.stride_a,
+                                                                         ba.stride_b, ba.stride_c);
     } else {
         dim3 grid(static_cast<unsigned>(ceil_div(g.N, 32)), static_cast<unsigned>(ceil_div(g.M, 32)), nz);
         const bool rowmajor16 = plain && !g.transA && !g.transB && g.K % 4 == 0 && g.N % 4 == 0 &&
