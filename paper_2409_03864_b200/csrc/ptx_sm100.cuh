@@ -29,6 +29,15 @@ __device__ __forceinline__ bool elect_one() {
     return pred != 0;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// A grid launched with programmatic stream serialization may start while its predecessor in the stream still runs:
+// everything before grid_dependency_wait() (barrier and tensor-memory set-up) then overlaps the predecessor's tail;
+// the wait returns once the predecessor has completed and its memory is visible, so no global memory may be touched
+// before it.  launch_dependents() lets the successor of THIS grid start in the same way.  Both are no-ops for an
+// ordinary launch.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");

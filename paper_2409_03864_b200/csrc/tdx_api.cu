@@ -592,12 +592,25 @@ int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensor
                1024 + staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
     // producer warp, MMA warp, then 16 epilogue warps (staged epilogue) or 4 per 128-row half (direct)
     const int threads = p.tma_store ? 576 : (p.bm == 256 ? 320 : 192);
-    if (halo)   // one more warp: the halo producer
-        tdx::umma_conv_halo_kernel<<<grid, threads + 32, smem, st>>>(ma, ma_row ? *ma_row : ma, mb, mc, mc_row ? *mc_row : mc, p);
+    // programmatic stream serialization: the grid may be scheduled while the previous kernel of the stream drains; its
+    // set-up then overlaps that tail, and it waits on the device for the predecessor before touching global memory
+    cudaLaunchConfig_t lc;
+    std::memset(&lc, 0, sizeof lc);
+    lc.gridDim = dim3(static_cast<unsigned>(grid));
+    lc.blockDim = dim3(static_cast<unsigned>(halo ? threads + 32 : threads));   // halo: one more warp, the halo producer
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    if (halo)
+        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_conv_halo_kernel, ma, ma_row ? *ma_row : ma, mb, mc, mc_row ? *mc_row : mc, p));
     else if (conv)
-        tdx::umma_contract_kernel<true><<<grid, threads, smem, st>>>(ma, mb, mc, p);
+        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_contract_kernel<true>, ma, mb, mc, p));
     else
-        tdx::umma_contract_kernel<false><<<grid, threads, smem, st>>>(ma, mb, mc, p);
+        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_contract_kernel<false>, ma, mb, mc, p));
     TDX_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     return TDX_OK;

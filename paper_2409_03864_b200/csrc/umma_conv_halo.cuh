@@ -105,6 +105,8 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = s_tmem_base;
     const int total_items = p.tiles_m * p.tiles_n;
+    ptx::grid_launch_dependents();     // see umma_contract_kernel
+    ptx::grid_dependency_wait();
 
     if (warp == halo_warp) {
         // ------------------------------------------------------------ halo producer: one tile per (item, channel chunk)

@@ -488,8 +488,10 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = s_tmem_base;
     const int total_items = p.tiles_m * p.tiles_n * p.split_k;
-    // split-K: let the reduction kernel's CTAs get scheduled while this grid still runs (they wait for its end)
-    if (p.split_k > 1) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // the next grid in the stream (the split-K reduction, or the next call's kernel) may be scheduled as SMs free up and
+    // run its set-up; this grid touches global memory only after its own predecessor has completed
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer
