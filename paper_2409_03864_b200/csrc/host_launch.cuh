@@ -1,0 +1,500 @@
+// Kernel launches: parameter blocks, tensor maps and grids of the tensor-core, CUDA-core and generic kernels.
+#pragma once
+#include "host_plan.cuh"
+
+namespace {
+
+// ------------------------------------------------------------------ launches
+int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
+                const UmmaParams& p_in, cudaStream_t st, bool halo = false, const CUtensorMap* ma_row = nullptr,
+                const CUtensorMap* mc_row = nullptr, int plan_grid = 0) {
+    const long long items = static_cast<long long>(p_in.tiles_m) * p_in.tiles_n * p_in.split_k;
+    UmmaParams p = p_in;
+    if (p.b_box == 0) p.b_box = p.bn;
+    const int grid = p.tiles != nullptr ? plan_grid : static_cast<int>(std::min<long long>(items, ctx->sm_count));
+    size_t smem = static_cast<size_t>(p.stages) * ((p.bm + p.bn) * 128) + 1024 +
+                  staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
+    if (halo)
+        smem = static_cast<size_t>(p.a_stages) * (p.bm / 128) * p.halo_bytes + static_cast<size_t>(p.stages) * p.bn * 128 +
+               1024 + staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
+    // producer warp, MMA warp, then 16 epilogue warps (staged epilogue) or 4 per 128-row half (direct)
+    const int threads = p.tma_store ? 576 : (p.bm == 256 ? 320 : 192);
+    // programmatic stream serialization: the grid may be scheduled while the previous kernel of the stream drains; its
+    // set-up then overlaps that tail, and it waits on the device for the predecessor before touching global memory
+    cudaLaunchConfig_t lc;
+    std::memset(&lc, 0, sizeof lc);
+    lc.gridDim = dim3(static_cast<unsigned>(grid));
+    lc.blockDim = dim3(static_cast<unsigned>(halo ? threads + 32 : threads));   // halo: one more warp, the halo producer
+    lc.dynamicSmemBytes = smem;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    if (halo)
+        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_conv_halo_kernel, ma, ma_row ? *ma_row : ma, mb, mc, mc_row ? *mc_row : mc, p));
+    else if (conv)
+        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_contract_kernel<true>, ma, mb, mc, p));
+    else
+        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_contract_kernel<false>, ma, mb, mc, p));
+    TDX_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return TDX_OK;
+}
+
+// The reduction is launched with programmatic stream serialization so that its launch latency hides behind
+// the tail of the GEMM kernel; it waits on the device for the GEMM grid to complete before reading partials.
+int launch_splitk_reduce(int grid, cudaStream_t st, long long MN, int N, int split, const float* partial, float alpha,
+                         __nv_bfloat16* out, int vec8, float beta = 0.0f) {
+    cudaLaunchConfig_t lc;
+    std::memset(&lc, 0, sizeof lc);
+    lc.gridDim = dim3(static_cast<unsigned>(grid));
+    lc.blockDim = dim3(256);
+    lc.dynamicSmemBytes = 0;
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    const float* bias = nullptr;
+    int relu = 0;
+    TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::splitk_reduce_kernel, MN, N, split, partial, alpha, bias, relu, out, vec8, beta));
+    g_launches.fetch_add(1);
+    return TDX_OK;
+}
+
+int ensure_ws(DeviceCtx* ctx, size_t bytes, void** out) {
+    if (ctx->ws_bytes < bytes) {
+        if (ctx->ws) TDX_CUDA(cudaFree(ctx->ws));
+        ctx->ws = nullptr;
+        ctx->ws_bytes = 0;
+        TDX_CUDA(cudaMalloc(&ctx->ws, bytes));
+        ctx->ws_bytes = bytes;
+    }
+    *out = ctx->ws;
+    return TDX_OK;
+}
+
+int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
+                  const tdx_config& cfg, void* ws, size_t ws_bytes, bool internal_ws, cudaStream_t st, float beta = 0.0f) {
+    const int64_t num_kb = ceil_div(g.K, 64);
+    UmmaParams p;
+    std::memset(&p, 0, sizeof p);
+    p.M = static_cast<int>(g.M);
+    p.N = static_cast<int>(g.N);
+    p.num_kb = static_cast<int>(num_kb);
+    p.bm = cfg.tile_m;
+    p.slots = tmem_slots_for(cfg.tile_m, cfg.tile_n);
+    p.tiles_m = static_cast<int>(ceil_div(g.M, cfg.tile_m));
+    p.tiles_n = static_cast<int>(ceil_div(g.N, cfg.tile_n));
+    p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
+    p.split_k = cfg.split_k;
+    p.kb_per_split = static_cast<int>(ceil_div(num_kb, cfg.split_k));
+    p.k_stagger = cfg.k_stagger;
+    p.bn = cfg.tile_n;
+    p.stages = cfg.stages;
+    p.tmem_cols = tmem_cols_for(cfg.tile_m, cfg.tile_n);
+    p.a_mn_major = g.transA ? 1 : 0;   // A stored K x M: M contiguous
+    p.b_mn_major = g.transB ? 0 : 1;   // B stored K x N: N contiguous
+    p.alpha = alpha;
+    p.beta = beta;
+    p.bias = nullptr;
+    p.relu = 0;
+    p.C = static_cast<__nv_bfloat16*>(C);
+    p.ldc = g.N;
+    p.status = ctx->status_ptr;
+    p.vec_store = (g.N % 8 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+
+    if (cfg.split_k > 1) {
+        const size_t need = static_cast<size_t>(cfg.split_k) * g.M * g.N * sizeof(float);
+        if (internal_ws) {
+            int rc = ensure_ws(ctx, need, &ws);
+            if (rc) return rc;
+        } else if (ws == nullptr || ws_bytes < need || reinterpret_cast<uintptr_t>(ws) % 256) {
+            return fail(TDX_ERR_WORKSPACE, "split_k=%d needs %zu bytes of 256-byte aligned workspace", cfg.split_k, need);
+        }
+        p.partial = static_cast<float*>(ws);
+    }
+
+    CUtensorMap ma, mb;
+    int rc;
+    if (p.a_mn_major) {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.M), static_cast<uint64_t>(g.K)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.M) * 2};
+        uint32_t box[2] = {64, 64};
+        rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
+    } else {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.M)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
+        uint32_t box[2] = {64, 128};
+        rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
+    }
+    if (rc) return rc;
+    // tile widths fitted to the number of CTAs (see plan_fitted_tiles): B then arrives in 64-row copies
+    int plan_grid = 0;
+    if (cfg.fit != 1 && cfg.split_k == 1 && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0) {
+        DevicePlan dp;
+        rc = get_tile_plan(ctx, g.M, g.N, num_kb, cfg.tile_m, cfg.tile_n, cfg.raster, cfg.fit == 2 ? 0.0 : 0.03, st, &dp);
+        if (rc) return rc;
+        if (dp.fitted) {
+            p.tiles = dp.dev;
+            p.rounds = dp.rounds;
+            p.b_box = 64;
+            plan_grid = dp.grid;
+        }
+    }
+    if (p.b_mn_major) {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.K)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
+        uint32_t box[2] = {64, 64};
+        rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
+    } else {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.N)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
+        uint32_t box[2] = {64, static_cast<uint32_t>(p.tiles ? 64 : cfg.tile_n)};
+        rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
+    }
+    if (rc) return rc;
+
+    CUtensorMap mc = ma;   // unused unless the staged epilogue is on
+    // the accumulate term is read by the direct-store epilogue (and by the split-K reduction) only
+    p.tma_store = (cfg.store_mode == 2 && cfg.split_k == 1 && p.vec_store && beta == 0.0f) ? 1 : 0;
+    if (p.tma_store) {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.M)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
+        uint32_t box[2] = {32, 32};
+        rc = get_tensor_map(ctx, C, 2, dims, str, box, &mc, 64);
+        if (rc) return rc;
+    }
+    rc = launch_umma(ctx, false, ma, mb, mc, p, st, false, nullptr, nullptr, plan_grid);
+    if (rc) return rc;
+    if (cfg.split_k > 1) {
+        const long long MN = static_cast<long long>(g.M) * g.N;
+        const int vec8 = p.vec_store ? 1 : 0;
+        const long long work = vec8 ? MN / 8 : MN;
+        const int grid = static_cast<int>(std::min<long long>(ceil_div(work, 256), 148LL * 16));
+        rc = launch_splitk_reduce(std::max(grid, 1), st, MN, static_cast<int>(g.N), cfg.split_k, p.partial, alpha, p.C, vec8, beta);
+        if (rc) return rc;
+    }
+    return TDX_OK;
+}
+
+// GEMM on CTA pairs: 256 x tile_n per pair, each CTA loads its 128 rows of A and tile_n / 2 columns of B.
+int run_gemm_pair(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
+                  const tdx_config& cfg, cudaStream_t st) {
+    const int64_t num_kb = ceil_div(g.K, 64);
+    UmmaParams p;
+    std::memset(&p, 0, sizeof p);
+    p.M = static_cast<int>(g.M);
+    p.N = static_cast<int>(g.N);
+    p.num_kb = static_cast<int>(num_kb);
+    p.bm = 128;                                      // what one CTA of the pair owns (epilogue geometry)
+    p.slots = 2 * cfg.tile_n <= 256 ? 4 : 2;
+    p.tiles_m = static_cast<int>(ceil_div(g.M, 256));
+    p.tiles_n = static_cast<int>(ceil_div(g.N, cfg.tile_n));
+    p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
+    p.split_k = 1;
+    p.kb_per_split = p.num_kb;
+    p.bn = cfg.tile_n;
+    p.stages = cfg.stages;
+    p.tmem_cols = 32;
+    while (p.tmem_cols < p.slots * cfg.tile_n) p.tmem_cols *= 2;
+    p.a_mn_major = g.transA ? 1 : 0;
+    p.b_mn_major = g.transB ? 0 : 1;
+    p.alpha = alpha;
+    p.C = static_cast<__nv_bfloat16*>(C);
+    p.ldc = g.N;
+    p.status = ctx->status_ptr;
+    p.vec_store = (g.N % 8 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+    p.tma_store = (cfg.store_mode == 2 && p.vec_store) ? 1 : 0;
+
+    CUtensorMap ma, mb, mc;
+    int rc;
+    if (p.a_mn_major) {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.M), static_cast<uint64_t>(g.K)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.M) * 2};
+        uint32_t box[2] = {64, 64};
+        rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
+    } else {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.M)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
+        uint32_t box[2] = {64, 128};
+        rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
+    }
+    if (rc) return rc;
+    // tile widths fitted to the number of pairs; each CTA's half of a tile's B columns then arrives in 64-row copies
+    // (K-major B only: an N-major half would have to be a multiple of 64 columns)
+    p.b_box = cfg.tile_n / 2;
+    int plan_pairs = 0;
+    // only on request: a 256 x 128 x 16 pair MMA measured 115 cycles, not 64, so narrow tiles gain nothing here
+    if (cfg.fit == 2 && !p.b_mn_major && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0) {
+        DevicePlan dp;
+        rc = get_tile_plan(ctx, g.M, g.N, num_kb, 256, cfg.tile_n, cfg.raster, 0.0, st, &dp, true);
+        if (rc) return rc;
+        if (dp.fitted) {
+            p.tiles = dp.dev;
+            p.rounds = dp.rounds;
+            p.b_box = 64;
+            plan_pairs = dp.grid;
+        }
+    }
+    if (p.b_mn_major) {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.K)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
+        uint32_t box[2] = {64, 64};
+        rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
+    } else {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.N)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
+        uint32_t box[2] = {64, static_cast<uint32_t>(p.b_box)};
+        rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
+    }
+    if (rc) return rc;
+    mc = ma;
+    if (p.tma_store) {
+        uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.M)};
+        uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
+        uint32_t box[2] = {32, 32};
+        rc = get_tensor_map(ctx, C, 2, dims, str, box, &mc, 64);
+        if (rc) return rc;
+    }
+    const long long pair_tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
+    const int pairs = p.tiles ? plan_pairs : static_cast<int>(std::min<long long>(pair_tiles, ctx->sm_count / 2));
+    cudaLaunchConfig_t lc;
+    std::memset(&lc, 0, sizeof lc);
+    lc.gridDim = dim3(static_cast<unsigned>(2 * pairs));
+    lc.blockDim = dim3(p.tma_store ? 576 : 192);
+    lc.dynamicSmemBytes = static_cast<size_t>(p.stages) * ((128 + p.bn / 2) * 128) + 1024 +
+                          staging_bytes_for(128, p.tma_store ? 2 : 1);
+    lc.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    lc.attrs = attr;
+    lc.numAttrs = 1;
+    TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_pair_kernel, ma, mb, mc, p));
+    g_launches.fetch_add(1);
+    return TDX_OK;
+}
+
+int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const void* w, const float* bias, int relu,
+                  void* y, const tdx_config& cfg, cudaStream_t st, const void* residual = nullptr) {
+    const int cchunks = static_cast<int>(ceil_div(c.Cin, 64));
+    UmmaParams p;
+    std::memset(&p, 0, sizeof p);
+    p.bw = cfg.patch_w;
+    p.bh = cfg.patch_h;
+    p.bm = cfg.tile_m;
+    p.slots = tmem_slots_for(cfg.tile_m, cfg.tile_n);
+    p.nb = cfg.tile_m / (p.bw * p.bh);
+    const bool halo = cfg.halo >= 2;
+    const bool stacked = cfg.halo == 3;
+    if (halo) {
+        p.R = static_cast<int>(c.R);
+        p.hpitch = static_cast<int>(kHaloPatchW + c.S - 1);
+        p.hrows = static_cast<int>(kHaloPatchH + c.R - 1);
+        p.halo_bytes = halo_tile_bytes(c.R, c.S);
+        p.a_stages = kHaloAStages;
+    }
+    p.patches_w = static_cast<int>(ceil_div(c.Q, p.bw));
+    p.patches_h = static_cast<int>(ceil_div(c.P, p.bh));
+    int64_t total_patches = c.N * p.patches_w * p.patches_h;
+    if (stacked) {
+        p.Pv = static_cast<int>(stacked_rows_per_image(c));
+        p.H = static_cast<int>(c.H);
+        p.patches_h = static_cast<int>(ceil_div(c.N * p.Pv, p.bh));      // over the whole column of images
+        total_patches = static_cast<int64_t>(p.patches_w) * p.patches_h;
+    }
+    p.M = static_cast<int>(c.N * c.P * c.Q);
+    p.N = static_cast<int>(c.Cout);
+    p.num_kb = static_cast<int>(c.R * c.S * cchunks);
+    p.tiles_m = static_cast<int>(ceil_div(total_patches, p.nb));
+    p.tiles_n = static_cast<int>(ceil_div(c.Cout, cfg.tile_n));
+    p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
+    p.split_k = 1;
+    p.kb_per_split = p.num_kb;
+    p.k_stagger = cfg.k_stagger;
+    p.bn = cfg.tile_n;
+    p.stages = cfg.stages;
+    if (halo && cfg.tile_n >= c.Cout) {
+        // small filters stay resident: all (chunk, tap) slices of the one column tile fit beside the halo ring,
+        // so they are loaded once per CTA and the main loop has no per-tap handshake
+        const int64_t slices = c.R * c.S * cchunks;
+        const int64_t need = static_cast<int64_t>(p.a_stages) * (cfg.tile_m / 128) * p.halo_bytes + slices * cfg.tile_n * 128 +
+                             staging_bytes_for(cfg.tile_m, cfg.store_mode) + 1024;
+        if (need <= ctx->smem_optin - kStaticSmemReserve) {
+            p.b_resident = 1;
+            p.stages = static_cast<int>(slices);
+            // spend what is left on more halo tiles in flight (their load latency is what a short tile waits for)
+            const int64_t per_stage = static_cast<int64_t>(cfg.tile_m / 128) * p.halo_bytes;
+            while (p.a_stages < tdx::kMaxAStages && need + (p.a_stages - kHaloAStages + 1) * per_stage <= ctx->smem_optin - kStaticSmemReserve)
+                ++p.a_stages;
+        }
+    }
+    p.tmem_cols = tmem_cols_for(cfg.tile_m, cfg.tile_n);
+    p.a_mn_major = 0;
+    p.b_mn_major = 0;
+    p.alpha = 1.0f;
+    p.bias = bias;
+    p.residual = static_cast<const __nv_bfloat16*>(residual);
+    p.relu = relu;
+    p.C = static_cast<__nv_bfloat16*>(y);
+    p.ldc = c.Cout;
+    p.vec_store = (c.Cout % 8 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
+    p.P = static_cast<int>(c.P);
+    p.Q = static_cast<int>(c.Q);
+    p.Nimg = static_cast<int>(c.N);
+    p.S = static_cast<int>(c.S);
+    p.pad = c.pad;
+    p.stride = c.stride;
+    p.cchunks = cchunks;
+    p.status = ctx->status_ptr;
+
+    CUtensorMap ma, ma_row, mb;
+    {
+        uint64_t dims[4] = {static_cast<uint64_t>(c.Cin), static_cast<uint64_t>(c.W), static_cast<uint64_t>(c.H),
+                            static_cast<uint64_t>(c.N)};
+        uint64_t str[3] = {static_cast<uint64_t>(c.Cin) * 2, static_cast<uint64_t>(c.W * c.Cin) * 2,
+                           static_cast<uint64_t>(c.H * c.W * c.Cin) * 2};
+        uint32_t box[4] = {64, static_cast<uint32_t>(halo ? p.hpitch : p.bw), static_cast<uint32_t>(halo ? p.hrows : p.bh), 1};
+        // strided convolution (per-tap loads only): the copy walks the image with the convolution's stride, so a
+        // box spanning bw * stride input pixels delivers exactly the bw pixels under one filter tap
+        uint32_t estr[4] = {1, static_cast<uint32_t>(c.stride), static_cast<uint32_t>(c.stride), 1};
+        if (c.stride > 1) { box[1] *= c.stride; box[2] *= c.stride; }
+        int rc = get_tensor_map(ctx, x, 4, dims, str, box, &ma, 128, c.stride > 1 ? estr : nullptr);
+        if (rc) return rc;
+        ma_row = ma;
+        if (stacked) {
+            box[2] = 1;              // windows that reach into the next image are copied one row at a time
+            rc = get_tensor_map(ctx, x, 4, dims, str, box, &ma_row);
+            if (rc) return rc;
+        }
+    }
+    {
+        uint64_t dims[3] = {static_cast<uint64_t>(c.Cin), static_cast<uint64_t>(c.R * c.S),
+                            static_cast<uint64_t>(c.Cout)};
+        uint64_t str[2] = {static_cast<uint64_t>(c.Cin) * 2, static_cast<uint64_t>(c.R * c.S * c.Cin) * 2};
+        uint32_t box[3] = {64, 1, static_cast<uint32_t>(cfg.tile_n)};
+        int rc = get_tensor_map(ctx, w, 3, dims, str, box, &mb);
+        if (rc) return rc;
+    }
+    CUtensorMap mc = ma, mc_row = ma;
+    p.tma_store = (cfg.store_mode == 2 && p.vec_store && p.bw * p.bh >= 32) ? 1 : 0;
+    // the staged epilogue reads the residual 16 bytes at a time
+    if (reinterpret_cast<uintptr_t>(residual) % 16) p.tma_store = 0;
+    if (halo) p.epi_warps = p.tma_store ? 16 : 4 * (cfg.tile_m / 128);
+    if (p.tma_store) {
+        p.sbx = std::min(p.bw, 32);
+        p.sby = 32 / p.sbx;
+        uint64_t dims[4] = {static_cast<uint64_t>(c.Cout), static_cast<uint64_t>(c.Q), static_cast<uint64_t>(c.P),
+                            static_cast<uint64_t>(c.N)};
+        uint64_t str[3] = {static_cast<uint64_t>(c.Cout) * 2, static_cast<uint64_t>(c.Q * c.Cout) * 2,
+                           static_cast<uint64_t>(c.P * c.Q * c.Cout) * 2};
+        uint32_t box[4] = {32, static_cast<uint32_t>(p.sbx), static_cast<uint32_t>(p.sby), 1};
+        int rc = get_tensor_map(ctx, y, 4, dims, str, box, &mc, 64);
+        if (rc) return rc;
+        mc_row = mc;
+        if (stacked) {
+            box[2] = 1;              // four pixel rows that cross the seam between two images leave one by one
+            rc = get_tensor_map(ctx, y, 4, dims, str, box, &mc_row, 64);
+            if (rc) return rc;
+        }
+    }
+    return launch_umma(ctx, true, ma, mb, mc, p, st, halo, &ma_row, &mc_row);
+}
+
+void gemm_strides(const GemmProblem& g, long long* sa_i, long long* sa_k, long long* sb_k, long long* sb_j) {
+    *sa_i = g.transA ? 1 : g.K;
+    *sa_k = g.transA ? g.M : 1;
+    *sb_k = g.transB ? 1 : g.N;
+    *sb_j = g.transB ? g.K : 1;
+}
+
+// batch count, batch strides in elements, and the accumulate factor of tdx_gemm_batched (one batch, beta = 0: tdx_gemm)
+struct BatchArgs {
+    int64_t batch = 1, stride_a = 0, stride_b = 0, stride_c = 0;
+    float beta = 0.0f;
+};
+
+int run_gemm_simt_f32(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
+                      cudaStream_t st, const BatchArgs& ba = BatchArgs()) {
+    if (g.M >= (1LL << 31) || g.N >= (1LL << 31) || g.K >= (1LL << 31))
+        return fail(TDX_ERR_UNSUPPORTED, "fp32 tiled GEMM needs dimensions below 2^31");
+    long long sa_i, sa_k, sb_k, sb_j;
+    gemm_strides(g, &sa_i, &sa_k, &sb_k, &sb_j);
+    const float* a = static_cast<const float*>(A);
+    const float* b = static_cast<const float*>(B);
+    float* c = static_cast<float*>(C);
+    if (ba.batch > 65535) return fail(TDX_ERR_UNSUPPORTED, "fp32 batched GEMM takes at most 65535 batches");
+    const unsigned nz = static_cast<unsigned>(ba.batch);
+    const bool plain = ba.batch == 1 && ba.beta == 0.0f;
+    const int64_t tiles64 = ceil_div(g.M, 64) * ceil_div(g.N, 64) * ba.batch;
+    if (tiles64 >= ctx->sm_count) {
+        // 64 x 64 tiles (4 x 4 outputs per thread) once there is one per SM; smaller problems take 32 x 32 tiles
+        dim3 grid(static_cast<unsigned>(ceil_div(g.N, 64)), static_cast<unsigned>(ceil_div(g.M, 64)), nz);
+        tdx::sgemm_ring_kernel<64, 64, 16, 4, 4, 4><<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k,
+                                                                         sb_j, alpha, a, b, c, ba.beta, ba.stride_a,
+                                                                         ba.stride_b, ba.stride_c);
+    } else {
+        dim3 grid(static_cast<unsigned>(ceil_div(g.N, 32)), static_cast<unsigned>(ceil_div(g.M, 32)), nz);
+        const bool rowmajor16 = plain && !g.transA && !g.transB && g.K % 4 == 0 && g.N % 4 == 0 &&
+                                reinterpret_cast<uintptr_t>(A) % 16 == 0 && reinterpret_cast<uintptr_t>(B) % 16 == 0;
+        if (rowmajor16)
+            tdx::sgemm_small_rowmajor_kernel<<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, alpha, a, b, c);
+        else
+            tdx::sgemm_small_kernel<<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k, sb_j, alpha, a, b,
+                                                          c, ba.beta, ba.stride_a, ba.stride_b, ba.stride_c);
+    }
+    TDX_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return TDX_OK;
+}
+
+int run_gemm_generic(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
+                     cudaStream_t st, const BatchArgs& ba = BatchArgs()) {
+    long long sa_i, sa_k, sb_k, sb_j;
+    gemm_strides(g, &sa_i, &sa_k, &sb_k, &sb_j);
+    const long long total = g.M * g.N * ba.batch;
+    const int grid = static_cast<int>(std::min<long long>(ceil_div(total, 256), static_cast<long long>(ctx->sm_count) * 32));
+    if (g.dtype == TDX_F32)
+        tdx::gemm_generic_kernel<float, float><<<grid, 256, 0, st>>>(g.M, g.N, g.K, sa_i, sa_k, sb_k, sb_j, alpha,
+                                                                    static_cast<const float*>(A),
+                                                                    static_cast<const float*>(B), static_cast<float*>(C),
+                                                                    ba.beta, ba.batch, ba.stride_a, ba.stride_b, ba.stride_c);
+    else
+        tdx::gemm_generic_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
+            g.M, g.N, g.K, sa_i, sa_k, sb_k, sb_j, alpha, static_cast<const __nv_bfloat16*>(A),
+            static_cast<const __nv_bfloat16*>(B), static_cast<__nv_bfloat16*>(C), ba.beta, ba.batch, ba.stride_a,
+            ba.stride_b, ba.stride_c);
+    TDX_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return TDX_OK;
+}
+
+int run_conv_generic(DeviceCtx* ctx, const ConvProblem& c, const void* x, const void* w, const float* bias, int relu,
+                     void* y, cudaStream_t st, const void* residual = nullptr) {
+    if (c.N >= (1LL << 31) || c.H >= (1LL << 31) || c.W >= (1LL << 31) || c.Cin >= (1LL << 31) ||
+        c.Cout >= (1LL << 31) || c.R >= (1LL << 31) || c.S >= (1LL << 31))
+        return fail(TDX_ERR_UNSUPPORTED, "conv dimensions must be below 2^31");
+    const long long total = c.N * c.P * c.Q * c.Cout;
+    const int grid = static_cast<int>(std::min<long long>(ceil_div(total, 256), static_cast<long long>(ctx->sm_count) * 32));
+    if (c.dtype == TDX_F32)
+        tdx::conv2d_generic_kernel<float, float><<<grid, 256, 0, st>>>(
+            (int)c.N, (int)c.H, (int)c.W, (int)c.Cin, (int)c.Cout, (int)c.R, (int)c.S, c.pad, c.stride, (int)c.P,
+            (int)c.Q, static_cast<const float*>(x), static_cast<const float*>(w), bias, relu, static_cast<float*>(y),
+            static_cast<const float*>(residual));
+    else
+        tdx::conv2d_generic_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
+            (int)c.N, (int)c.H, (int)c.W, (int)c.Cin, (int)c.Cout, (int)c.R, (int)c.S, c.pad, c.stride, (int)c.P,
+            (int)c.Q, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w), bias, relu,
+            static_cast<__nv_bfloat16*>(y), static_cast<const __nv_bfloat16*>(residual));
+    TDX_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    return TDX_OK;
+}
+
+}  // namespace

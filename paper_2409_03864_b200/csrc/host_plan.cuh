@@ -1,0 +1,172 @@
+// Tile plan fitted to the number of CTAs: cost model, longest-first dealing, device copies of the tables.
+#pragma once
+#include "host_config.cuh"
+
+namespace {
+
+// ------------------------------------------------------------------ tile plan fitted to the number of CTAs
+// A uniform grid of T tiles on G persistent CTAs takes ceil(T / G) tile times although it holds only T / G of
+// work per CTA (the 4096^3 GEMM: 256 tiles of 256 x 256 on 148 CTAs = 1.73 tile times of work done in 2).  The
+// plan keeps the tile height and cuts some row blocks into narrower tiles (widths w < tile_n, both multiples of
+// 64) so that every CTA ends at about the same time: tiles are dealt longest first, each to the CTA with the
+// least work so far.  The cost model is the measured instruction time of one MMA (N / 2 cycles, at least 60)
+// plus a fixed and a per-column epilogue cost.
+struct TilePlan {
+    std::vector<int4> table;   // [round * grid + cta] = (row block, first column, width, 0)
+    int rounds = 0;
+    int grid = 0;
+    double makespan = 0.0;     // model cycles
+    double uniform = 0.0;      // the same for the uniform grid
+};
+
+// mmas_per_kb: MMAs one CTA's tensor core runs per 64-deep K block (4 per 128 rows it owns)
+double tile_cost_cycles(int mmas_per_kb, int width, int64_t num_kb) {
+    const double mma = std::max(width / 2.0, 60.0);
+    return static_cast<double>(num_kb) * mmas_per_kb * mma + 1500.0 + 13.0 * width;
+}
+
+// makespan of `na` tiles of cost ca and `nb` tiles of cost cb (ca >= cb > 0), dealt longest first on g CTAs, each
+// to the CTA with the least work so far (closed form of that greedy rule for two sizes)
+double lpt_two_sizes(int64_t na, double ca, int64_t nb, double cb, int g) {
+    const int64_t q = na / g, x = na % g;              // x CTAs hold q + 1 wide tiles, g - x hold q
+    const double low = ca * static_cast<double>(q), high = x > 0 ? low + ca : low;
+    if (nb <= 0) return high;
+    if (x == 0) return low + cb * static_cast<double>(ceil_div(nb, g));
+    // the g - x lighter CTAs take narrow tiles until they have caught up with the others
+    const int64_t catch_up = static_cast<int64_t>(std::ceil(ca / cb - 1e-9));
+    const int64_t lighter = g - x;
+    if (nb <= catch_up * lighter) return std::max(high, low + cb * static_cast<double>(ceil_div(nb, lighter)));
+    const double low2 = low + cb * static_cast<double>(catch_up);      // >= high, by less than cb
+    const int64_t rest = nb - catch_up * lighter;
+    const int64_t f = rest / g, rem = rest % g;
+    if (rem == 0) return low2 + cb * static_cast<double>(f);
+    if (rem <= x) return std::max(low2 + cb * static_cast<double>(f), high + cb * static_cast<double>(f + 1));
+    return low2 + cb * static_cast<double>(f + 1);
+}
+
+// Searches widths and how many row blocks take the narrower cut.  Returns false when nothing beats the uniform grid
+// by `min_gain` (relative).
+// `g` workers (CTAs, or CTA pairs when pair is set: a pair's two tensor cores share a 256-row tile).
+bool plan_fitted_tiles(int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int raster, int g, double min_gain,
+                       TilePlan* out, bool pair = false) {
+    const int64_t tiles_m = ceil_div(M, bm);
+    const int64_t uniform_tiles = tiles_m * ceil_div(N, bn);
+    const int mmas = pair ? 4 : 4 * (bm / 128);
+    const double c_big = tile_cost_cycles(mmas, bn, num_kb);
+    const double uniform = lpt_two_sizes(uniform_tiles, c_big, 0, 0.0, g);
+    double best = uniform;
+    int best_w = 0;
+    int64_t best_b = 0, best_b1 = 0, best_e = 0;
+    // pairs: each CTA loads half of a tile's columns, kept a multiple of 64 (one copy per 64 rows)
+    const int w_step = pair ? 128 : 64;
+    for (int w = bn - w_step; w >= 128; w -= w_step) {
+        const double c_small = tile_cost_cycles(mmas, w, num_kb);
+        // option b of a row block: b tiles of width w at the high columns, a(b) tiles of width bn before them
+        auto bigs_for = [&](int64_t b) { return ceil_div(std::max<int64_t>(0, N - b * w), bn); };
+        // options that do not carry a tile more than needed
+        std::vector<int64_t> opts;
+        for (int64_t b = 0; b <= ceil_div(N, w); ++b)
+            if (b == 0 || bigs_for(b) * bn + b * w - N < w) opts.push_back(b);
+        for (size_t i = 0; i < opts.size(); ++i)
+        for (size_t j = i + 1; j < opts.size(); ++j) {
+            const int64_t b0 = opts[i], b1 = opts[j];
+            for (int64_t e = 0; e <= tiles_m; ++e) {                            // e row blocks take option b1
+                const int64_t na = (tiles_m - e) * bigs_for(b0) + e * bigs_for(b1);
+                const int64_t nb = (tiles_m - e) * b0 + e * b1;
+                const double m = lpt_two_sizes(na, c_big, nb, c_small, g);
+                if (m < best * (1.0 - 1e-9)) { best = m; best_w = w; best_b = b0; best_b1 = b1; best_e = e; }
+            }
+        }
+    }
+    out->uniform = uniform;
+    out->makespan = best;
+    if (best_w == 0 || best > uniform * (1.0 - min_gain)) return false;
+    // list the tiles: wide ones first, each group in the panel order of the uniform grid (row blocks fastest
+    // inside a panel of `raster` row blocks, then columns, then panels)
+    const int w = best_w;
+    auto bigs_for = [&](int64_t b) { return ceil_div(std::max<int64_t>(0, N - b * w), static_cast<int64_t>(bn)); };
+    struct T { int m, n0, width; };
+    std::vector<T> wide, narrow;
+    const int64_t panel = raster <= 0 ? tiles_m : std::min<int64_t>(raster, tiles_m);
+    for (int64_t m0 = 0; m0 < tiles_m; m0 += panel) {
+        const int64_t rows = std::min(panel, tiles_m - m0);
+        const int64_t max_cols = ceil_div(N, 64) + 1;
+        for (int64_t c = 0; c < max_cols; ++c)          // c-th tile of each row block of the panel
+            for (int64_t r = 0; r < rows; ++r) {
+                const int64_t m = m0 + r;
+                const int64_t b = (m >= tiles_m - best_e) ? best_b1 : best_b;
+                const int64_t a = bigs_for(b);
+                if (c < a) wide.push_back({static_cast<int>(m), static_cast<int>(c * bn), bn});
+                else if (c < a + b) narrow.push_back({static_cast<int>(m), static_cast<int>(a * bn + (c - a) * w), w});
+            }
+    }
+    const int64_t total = static_cast<int64_t>(wide.size() + narrow.size());
+    const int grid = static_cast<int>(std::min<int64_t>(total, g));
+    std::vector<std::vector<T>> per(grid);
+    std::vector<double> load(grid, 0.0);
+    const double c_small = tile_cost_cycles(mmas, w, num_kb);
+    auto deal = [&](const std::vector<T>& v, double cost) {
+        for (const T& t : v) {
+            int who = 0;
+            for (int i = 1; i < grid; ++i) if (load[i] < load[who] - 1e-6) who = i;
+            per[who].push_back(t);
+            load[who] += cost;
+        }
+    };
+    deal(wide, c_big);
+    deal(narrow, c_small);
+    size_t rounds = 0;
+    for (auto& v : per) rounds = std::max(rounds, v.size());
+    out->grid = grid;
+    out->rounds = static_cast<int>(rounds);
+    out->table.assign(rounds * grid, make_int4(0, 0, 0, 0));
+    for (int i = 0; i < grid; ++i)
+        for (size_t k = 0; k < per[i].size(); ++k)
+            out->table[k * grid + i] = make_int4(per[i][k].m, per[i][k].n0, per[i][k].width, 0);
+    return true;
+}
+
+// Device copies of tile plans, one per (shape, tile, CTA count); never freed (a few KB each).
+struct PlanKey {
+    int64_t M, N, num_kb;
+    int bm, bn, raster, g, forced, pair;
+    bool operator<(const PlanKey& o) const { return std::memcmp(this, &o, sizeof(PlanKey)) < 0; }
+};
+struct DevicePlan { int4* dev = nullptr; int rounds = 0, grid = 0; bool fitted = false; };
+std::map<PlanKey, DevicePlan> g_plans;
+
+// Looks the plan up (building and uploading it on first use; the upload is ordered on `st` before the kernel).
+int get_tile_plan(DeviceCtx* ctx, int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int raster, double min_gain,
+                  cudaStream_t st, DevicePlan* out, bool pair = false) {
+    PlanKey key;
+    std::memset(&key, 0, sizeof key);
+    key.M = M; key.N = N; key.num_kb = num_kb; key.bm = bm; key.bn = bn; key.raster = raster; key.g = pair ? ctx->sm_count / 2 : ctx->sm_count; key.forced = min_gain <= 0.0 ? 1 : 0;
+    key.pair = pair ? 1 : 0;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        auto it = g_plans.find(key);
+        if (it != g_plans.end()) { *out = it->second; return TDX_OK; }
+    }
+    TilePlan plan;
+    DevicePlan d;
+    d.fitted = plan_fitted_tiles(M, N, num_kb, bm, bn, raster, key.g, min_gain, &plan, pair);
+    if (d.fitted) {
+        const size_t bytes = plan.table.size() * sizeof(int4);
+        void* dev = nullptr;
+        TDX_CUDA(cudaMalloc(&dev, bytes));
+        // the table is a std::vector about to go out of scope: copy synchronously (once per shape)
+        TDX_CUDA(cudaMemcpy(dev, plan.table.data(), bytes, cudaMemcpyHostToDevice));
+        d.dev = static_cast<int4*>(dev);
+        d.rounds = plan.rounds;
+        d.grid = plan.grid;
+    }
+    (void)st;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        g_plans[key] = d;
+    }
+    *out = d;
+    return TDX_OK;
+}
+
+}  // namespace

@@ -1,1075 +1,10 @@
-// C-ABI of the tdx library: argument validation, kernel choice, TMA descriptor cache,
-// launches, the tile-configuration search and its cache.  See include/tdx.h for the contract.
-#include "tdx.h"
-
-#include <cuda.h>
-#include <cuda_runtime.h>
-
-#include <algorithm>
-#include <cmath>
-#include <atomic>
-#include <cstdarg>
-#include <cstdio>
-#include <cstdlib>
-#include <cstring>
-#include <map>
-#include <functional>
-#include <mutex>
-#include <queue>
-#include <string>
-#include <vector>
-
-#include "simt_kernels.cuh"
-#include "umma_conv_halo.cuh"
-#include "umma_kernel.cuh"
-#include "umma_pair.cuh"
+// C-ABI of the tdx library: argument validation, kernel choice, the tile-configuration search and its cache, and the
+// extern "C" entry points.  See include/tdx.h for the contract.  The pieces it builds on are headers of this one
+// translation unit: host_state.cuh (context, caches), host_config.cuh (configuration rules), host_plan.cuh (fitted
+// tile plans), host_launch.cuh (launches).
+#include "host_launch.cuh"
 
 namespace {
-
-using tdx::UmmaParams;
-
-// ------------------------------------------------------------------ errors
-thread_local std::string g_err;
-
-int fail(int status, const char* fmt, ...) {
-    char buf[512];
-    va_list ap;
-    va_start(ap, fmt);
-    vsnprintf(buf, sizeof buf, fmt, ap);
-    va_end(ap);
-    g_err = buf;
-    return status;
-}
-
-#define TDX_CUDA(expr)                                                                                   \
-    do {                                                                                                 \
-        cudaError_t e_ = (expr);                                                                         \
-        if (e_ != cudaSuccess) return fail(TDX_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_)); \
-    } while (0)
-
-std::atomic<int64_t> g_launches{0};
-
-__device__ int g_device_status_word = 0;
-
-// ------------------------------------------------------------------ per-device state
-constexpr int kSmemLimitDefault = 232448;  // 227 KiB opt-in limit of sm_100
-constexpr int kStaticSmemReserve = 512;    // barriers and flags declared statically in the kernel
-constexpr int kDefaultSmCount = 148;
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-struct DeviceCtx {
-    int dev = -1;
-    int sm_count = kDefaultSmCount;
-    int smem_optin = kSmemLimitDefault;
-    int* status_ptr = nullptr;
-    EncodeTiledFn encode = nullptr;
-    void* ws = nullptr;          // internal split-K workspace
-    size_t ws_bytes = 0;
-    void* staging[4] = {nullptr, nullptr, nullptr, nullptr};  // host-variant device copies
-    size_t staging_bytes[4] = {0, 0, 0, 0};
-};
-
-std::mutex g_mu;
-std::map<int, DeviceCtx> g_ctx;
-
-int get_ctx(DeviceCtx** out) {
-    int dev = -1;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) {
-        cudaGetLastError();
-        return fail(TDX_ERR_NO_DEVICE, "no CUDA device: %s", cudaGetErrorString(e));
-    }
-    std::lock_guard<std::mutex> lk(g_mu);
-    auto it = g_ctx.find(dev);
-    if (it != g_ctx.end()) {
-        *out = &it->second;
-        return TDX_OK;
-    }
-    cudaDeviceProp prop;
-    e = cudaGetDeviceProperties(&prop, dev);
-    if (e != cudaSuccess) {
-        cudaGetLastError();
-        return fail(TDX_ERR_NO_DEVICE, "cudaGetDeviceProperties: %s", cudaGetErrorString(e));
-    }
-    if (prop.major != 10) return fail(TDX_ERR_NO_DEVICE, "device %d is sm_%d%d, this library is built for sm_100a", dev, prop.major, prop.minor);
-    DeviceCtx c;
-    c.dev = dev;
-    c.sm_count = prop.multiProcessorCount;
-    c.smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
-    void* sym = nullptr;
-    e = cudaGetSymbolAddress(&sym, g_device_status_word);
-    if (e != cudaSuccess) return fail(TDX_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
-    c.status_ptr = static_cast<int*>(sym);
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    e = cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres);
-    if (e != cudaSuccess || fn == nullptr || qres != cudaDriverEntryPointSuccess)
-        return fail(TDX_ERR_NO_DEVICE, "driver does not export cuTensorMapEncodeTiled");
-    c.encode = reinterpret_cast<EncodeTiledFn>(fn);
-    e = cudaFuncSetAttribute(tdx::umma_contract_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             c.smem_optin - kStaticSmemReserve);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(tdx::umma_contract_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 c.smem_optin - kStaticSmemReserve);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(tdx::umma_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 c.smem_optin - kStaticSmemReserve);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(tdx::umma_conv_halo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 c.smem_optin - kStaticSmemReserve);
-    if (e != cudaSuccess) return fail(TDX_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
-    auto ins = g_ctx.emplace(dev, c);
-    *out = &ins.first->second;
-    return TDX_OK;
-}
-
-// ------------------------------------------------------------------ TMA descriptor cache
-struct MapKey {
-    const void* ptr;
-    int rank;
-    uint64_t dims[4];
-    uint64_t strides[3];
-    uint32_t box[4];
-    uint32_t estride[4];
-    int swizzle;
-    bool operator<(const MapKey& o) const { return std::memcmp(this, &o, sizeof(MapKey)) < 0; }
-};
-std::map<MapKey, CUtensorMap> g_maps;
-
-// bf16 tensor, 128-byte (or 64-byte) swizzle, zero fill outside the tensor.
-int get_tensor_map(DeviceCtx* ctx, const void* ptr, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                   const uint32_t* box, CUtensorMap* out, int swizzle_bytes = 128, const uint32_t* elem_strides = nullptr) {
-    MapKey key;
-    std::memset(&key, 0, sizeof key);
-    key.ptr = ptr;
-    key.rank = rank;
-    key.swizzle = swizzle_bytes;
-    for (int i = 0; i < rank; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; key.estride[i] = elem_strides ? elem_strides[i] : 1; }
-    for (int i = 0; i + 1 < rank; ++i) key.strides[i] = strides_bytes[i];
-    {
-        std::lock_guard<std::mutex> lk(g_mu);
-        auto it = g_maps.find(key);
-        if (it != g_maps.end()) { *out = it->second; return TDX_OK; }
-    }
-    cuuint64_t gdim[4], gstr[3];
-    cuuint32_t gbox[4], estr[4];
-    for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; gbox[i] = box[i]; estr[i] = elem_strides ? elem_strides[i] : 1; }
-    for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_bytes[i];
-    CUtensorMap m;
-    CUresult r = ctx->encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, static_cast<cuuint32_t>(rank),
-                             const_cast<void*>(ptr), gdim, gstr, gbox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                             swizzle_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
-                             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (r != CUDA_SUCCESS)
-        return fail(TDX_ERR_CUDA, "cuTensorMapEncodeTiled failed (%d) rank %d dims %llu %llu box %u %u", (int)r, rank,
-                    (unsigned long long)dims[0], (unsigned long long)(rank > 1 ? dims[1] : 0), box[0],
-                    rank > 1 ? box[1] : 0);
-    {
-        std::lock_guard<std::mutex> lk(g_mu);
-        if (g_maps.size() > 4096) g_maps.clear();
-        g_maps[key] = m;
-    }
-    *out = m;
-    return TDX_OK;
-}
-
-// ------------------------------------------------------------------ tuning cache
-struct TuneEntry { tdx_config cfg; float us; };
-std::map<std::string, TuneEntry> g_tune;
-
-std::string gemm_key(int64_t M, int64_t N, int64_t K, int tA, int tB, int dtype) {
-    char b[160];
-    snprintf(b, sizeof b, "gemm:%lld:%lld:%lld:%d:%d:%d", (long long)M, (long long)N, (long long)K, tA, tB, dtype);
-    return b;
-}
-std::string conv_key(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
-                     int stride, int dtype) {
-    char b[200];
-    snprintf(b, sizeof b, "conv:%lld:%lld:%lld:%lld:%lld:%lld:%lld:%d:%d:%d", (long long)N, (long long)H, (long long)W,
-             (long long)Cin, (long long)Cout, (long long)R, (long long)S, pad, stride, dtype);
-    return b;
-}
-bool tune_lookup(const std::string& key, tdx_config* out) {
-    std::lock_guard<std::mutex> lk(g_mu);
-    auto it = g_tune.find(key);
-    if (it == g_tune.end()) return false;
-    *out = it->second.cfg;
-    return true;
-}
-void cfg_to_ints(const tdx_config& c, int* v) {
-    v[0] = c.kernel; v[1] = c.tile_m; v[2] = c.tile_n; v[3] = c.tile_k; v[4] = c.stages; v[5] = c.cta_pair;
-    v[6] = c.split_k; v[7] = c.store_mode; v[8] = c.raster; v[9] = c.patch_w; v[10] = c.patch_h; v[11] = c.k_stagger;
-    v[12] = c.halo;
-    v[13] = c.fit;
-}
-void ints_to_cfg(const int* v, tdx_config* c) {
-    c->kernel = v[0]; c->tile_m = v[1]; c->tile_n = v[2]; c->tile_k = v[3]; c->stages = v[4]; c->cta_pair = v[5];
-    c->split_k = v[6]; c->store_mode = v[7]; c->raster = v[8]; c->patch_w = v[9]; c->patch_h = v[10];
-    c->k_stagger = v[11];
-    c->halo = v[12];
-    c->fit = v[13];
-}
-
-// ------------------------------------------------------------------ problem descriptions
-struct GemmProblem {
-    int64_t M, N, K;
-    int transA, transB, dtype;
-};
-struct ConvProblem {
-    int64_t N, H, W, Cin, Cout, R, S;
-    int pad, stride, dtype;
-    int64_t P, Q;
-};
-
-int64_t conv_out_dim(int64_t H, int64_t R, int64_t pad, int64_t stride) {
-    const int64_t span = H + 2 * pad - R;
-    return span < 0 ? 0 : span / stride + 1;
-}
-inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
-
-// Layout rules of the tensor-core GEMM path: every TMA row pitch must be a multiple of 16 bytes.
-bool gemm_umma_layout_ok(const GemmProblem& g) {
-    if (g.dtype != TDX_BF16) return false;
-    if (g.M >= (1LL << 31) || g.N >= (1LL << 31) || g.K >= (1LL << 31)) return false;
-    if (g.transA ? (g.M % 8) : (g.K % 8)) return false;
-    if (g.transB ? (g.K % 8) : (g.N % 8)) return false;
-    if (ceil_div(g.M, 128) * ceil_div(g.N, 32) * 64 >= (1LL << 31)) return false;
-    return true;
-}
-bool conv_umma_layout_ok(const ConvProblem& c) {
-    if (c.dtype != TDX_BF16 || c.stride > 8) return false;      // strided windows: per-tap loads with a traversal stride
-    if (c.Cin % 8) return false;
-    if (c.N * c.P * c.Q >= (1LL << 31) || c.H * c.W * c.Cin * 2 >= (1LL << 40)) return false;
-    if (c.R * c.S >= (1LL << 15) || c.Cout >= (1LL << 31)) return false;
-    return true;
-}
-
-// Shared memory the staged (TMA-store) epilogue needs: one 32 x 32 bf16 block for each of its 16 warps.
-int staging_bytes_for(int /*tile_m*/, int store_mode) { return store_mode == 2 ? 16 * 2048 : 0; }
-
-int umma_max_stages(int tile_m, int tile_n, int smem_limit, int store_mode) {
-    const int stage = (tile_m + tile_n) * 128;
-    int s = (smem_limit - kStaticSmemReserve - 1024 - staging_bytes_for(tile_m, store_mode)) / stage;
-    return std::min(s, tdx::kMaxStages);
-}
-
-// Accumulator slots (128 x tile_n each) kept in TMEM: a 256-row tile uses two per tile, and gets four
-// when they fit so that the epilogue still overlaps the next tile's main loop.
-// Halo-reuse convolution: 8 x 16 output-pixel patches, input window kept in shared memory across the taps.
-constexpr int kHaloPatchW = 8, kHaloPatchH = 16, kHaloAStages = 2;
-// Stacked images: rows each image takes in the column of all images.  The rows between two images must read as
-// zero for both, i.e. be the bottom padding of one and the top padding of the next: H + pad rows per image
-// (never fewer than the P output rows).
-int64_t stacked_rows_per_image(const ConvProblem& c) { return std::max(c.P, c.H + c.pad); }
-// 128-row halves the halo kernel works on: 8 x 16 patches cut per image (halo 2) or from the stacked column (halo 3)
-int64_t halo_patches(const ConvProblem& c, int mode) {
-    const int64_t pw = ceil_div(c.Q, kHaloPatchW);
-    return mode == 3 ? pw * ceil_div(c.N * stacked_rows_per_image(c), kHaloPatchH) : pw * c.N * ceil_div(c.P, kHaloPatchH);
-}
-int halo_tile_bytes(int64_t R, int64_t S) {
-    const int64_t b = (kHaloPatchW + S - 1) * (kHaloPatchH + R - 1) * 128;
-    return static_cast<int>((b + 1023) / 1024 * 1024);
-}
-int halo_max_stages(int tile_m, int tile_n, int64_t R, int64_t S, int smem_limit, int store_mode) {
-    const int a = kHaloAStages * (tile_m / 128) * halo_tile_bytes(R, S);
-    const int left = smem_limit - kStaticSmemReserve - 1024 - staging_bytes_for(tile_m, store_mode) - a;
-    return left <= 0 ? 0 : std::min(left / (tile_n * 128), tdx::kMaxStages);
-}
-
-// CTA pair (256 x tile_n per pair): each CTA stages its 128 rows of A and tile_n / 2 columns of B
-int pair_max_stages(int tile_n, int smem_limit, int store_mode) {
-    const int stage = (128 + tile_n / 2) * 128;
-    const int s = (smem_limit - kStaticSmemReserve - 1024 - staging_bytes_for(128, store_mode)) / stage;
-    return std::min(s, tdx::kMaxStages);
-}
-
-int tmem_slots_for(int tile_m, int bn) {
-    const int mh = tile_m / 128;
-    int s = std::min(tdx::kMaxSlots, 512 / bn);     // as many as TMEM holds: narrow tiles are short, and the
-    s -= s % mh;                                    // epilogue's latency then spans several tiles
-    return std::max(s, mh);
-}
-int tmem_cols_for(int tile_m, int bn) {
-    int c = 32;
-    while (c < tmem_slots_for(tile_m, bn) * bn) c *= 2;
-    return c;
-}
-
-// Static feasibility of a fully specified tensor-core configuration (the search-space constraints).
-// Returns 0 when feasible, else a short reason.
-const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num_kb, int smem_limit, bool conv,
-                               int64_t N, int64_t R = 1, int64_t S = 1, int stride = 1) {
-    if (c.tile_m != 128 && c.tile_m != 256) return "tile_m must be 128 or 256";
-    if (c.tile_k != 64) return "tile_k must be 64";
-    if (c.cta_pair != 1 && c.cta_pair != 2) return "cta_pair must be 1 or 2";
-    if (c.cta_pair == 2) {
-        if (conv) return "CTA pairs are implemented for the GEMM only";
-        if (c.tile_m != 256) return "a CTA pair works on 256-row tiles";
-        if (c.split_k != 1) return "CTA pairs have no split-K";
-        if (b_mn_major && c.tile_n % 128) return "tile_n must be a multiple of 128 for a CTA pair when B is read N-major";
-        if (c.k_stagger) return "CTA pairs have no k_stagger";
-    }
-    if (c.store_mode != 1 && c.store_mode != 2) return "store_mode must be 1 (direct) or 2 (TMA store)";
-    if (c.store_mode == 2) {
-        if (N % 8) return "the TMA-store epilogue needs an output row pitch that is a multiple of 16 bytes";
-        if (c.split_k > 1) return "split-K writes fp32 partials directly: use store_mode 1";
-        if (conv && c.patch_w * c.patch_h < 32) return "the TMA-store epilogue needs patches of at least 32 pixels";
-    }
-    if (c.tile_n < 32 || c.tile_n > 256 || c.tile_n % 32) return "tile_n must be a multiple of 32 in [32, 256]";
-    if (b_mn_major && c.tile_n % 64) return "tile_n must be a multiple of 64 when B is read N-major";
-    if (!conv && c.halo > 1) return "halo applies to the convolution only";
-    if (conv && (c.halo < 1 || c.halo > 3))
-        return "halo must be 1 (per-tap loads), 2 (halo tile kept in shared memory) or 3 (the same over stacked images)";
-    if (conv && stride > 1 && (c.patch_w * stride > 256 || c.patch_h * stride > 256))
-        return "patch times stride exceeds the 256-element limit of a copy";
-    if (conv && c.halo >= 2) {
-        if (stride != 1) return "halo reuse needs stride 1";
-        if (R * S < 2) return "halo reuse needs a filter with more than one tap";
-        if (c.patch_w != kHaloPatchW || c.patch_h != kHaloPatchH) return "halo reuse works on 8 x 16 patches";
-        if (kHaloPatchW + S - 1 > 256 || kHaloPatchH + R - 1 > 256) return "filter too large for a halo tile";
-        if (c.stages < 2 || c.stages > halo_max_stages(c.tile_m, c.tile_n, R, S, smem_limit, c.store_mode))
-            return "stages outside the shared-memory budget";
-    } else if (c.cta_pair == 2) {
-        if (c.stages < 2 || c.stages > pair_max_stages(c.tile_n, smem_limit, c.store_mode)) return "stages outside the shared-memory budget";
-    } else
-    if (c.stages < 2 || c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode)) return "stages outside the shared-memory budget";
-    if (c.split_k < 1) return "split_k must be >= 1";
-    if (conv && c.split_k != 1) return "conv has no split-K";
-    if (c.split_k > 1) {
-        const int64_t per = ceil_div(num_kb, c.split_k);
-        if ((c.split_k - 1) * per >= num_kb) return "split_k leaves an empty K slice";
-    }
-    if (c.raster < 0) return "raster must be >= 0";
-    if (c.fit < 0 || c.fit > 2) return "fit must be 0 (choose), 1 (uniform tiles) or 2 (tile widths fitted to the CTA count)";
-    if (c.k_stagger != 0 && c.k_stagger != 1) return "k_stagger must be 0 or 1";
-    return nullptr;
-}
-
-bool patch_ok(int bw, int bh) {
-    const int a = bw * bh;
-    return bw >= 8 && bw <= 128 && bh >= 1 && a <= 128 && (a & (a - 1)) == 0 && (bw & (bw - 1)) == 0;
-}
-
-// stride: a patch side times the stride must stay within the 256 elements one copy can span
-void choose_patch(int64_t P, int64_t Q, int* bw_out, int* bh_out, int stride = 1) {
-    int64_t best_cost = -1;
-    int best_bw = 8, best_bh = 1;
-    for (int bw = 8; bw <= 128 && bw * stride <= 256; bw *= 2) {
-        for (int bh = 1; bw * bh <= 128 && bh * stride <= 256; bh *= 2) {
-            const int64_t cost = ceil_div(Q, bw) * bw * ceil_div(P, bh) * bh;
-            const bool better = best_cost < 0 || cost < best_cost ||
-                                (cost == best_cost && (bw * bh > best_bw * best_bh ||
-                                                       (bw * bh == best_bw * best_bh && bw > best_bw)));
-            if (better) { best_cost = cost; best_bw = bw; best_bh = bh; }
-        }
-    }
-    *bw_out = best_bw;
-    *bh_out = best_bh;
-}
-
-// Heuristic default (used when neither the caller nor the tuning cache gives a configuration).
-void default_umma_config(int64_t tiles_m, int64_t N, int64_t num_kb, bool b_mn_major, int sm_count, int smem_limit,
-                         bool allow_split, tdx_config* c) {
-    std::memset(c, 0, sizeof *c);
-    c->kernel = TDX_KERNEL_UMMA;
-    c->tile_m = 128;
-    c->tile_k = 64;
-    c->cta_pair = 1;
-    c->store_mode = 1;
-    c->split_k = 1;
-    const int min_bn = b_mn_major ? 64 : 32;
-    int bn = 0, tm = 128;
-    const int64_t n_cap = ceil_div(N, min_bn) * min_bn;   // narrowest tile that covers N at once
-    // widest tile that still gives every SM at least one tile; 256-row tiles first (fewest L2 bytes per flop)
-    for (int cand_m : {256, 128}) {
-        if (bn) break;
-        for (int cand : {256, 128, 64, 32}) {
-            if (cand < min_bn) continue;
-            if (cand_m == 256 && cand < 128) continue;
-            if (cand > n_cap && cand / 2 >= n_cap) continue;  // a narrower tile covers N just as well
-            if (ceil_div(tiles_m, cand_m / 128) * ceil_div(N, cand) >= sm_count) { bn = cand; tm = cand_m; break; }
-        }
-    }
-    if (bn == 0) {
-        bn = N > 64 ? 128 : (N > 32 ? 64 : min_bn);
-        const int64_t tiles = tiles_m * ceil_div(N, bn);
-        if (allow_split && tiles < sm_count) {
-            int64_t s = std::min<int64_t>(ceil_div(sm_count, tiles), std::max<int64_t>(1, num_kb / 4));
-            s = std::min<int64_t>(s, 32);
-            while (s > 1 && (s - 1) * ceil_div(num_kb, s) >= num_kb) --s;
-            c->split_k = static_cast<int>(std::max<int64_t>(1, s));
-        }
-    }
-    c->tile_m = tm;
-    c->tile_n = bn;
-    // staged epilogue whenever the layout allows it (whole-line writes instead of 16-byte pieces)
-    if (c->split_k == 1 && N % 8 == 0) c->store_mode = 2;
-    c->stages = std::max(2, umma_max_stages(tm, bn, smem_limit, c->store_mode));
-    c->raster = 8;
-}
-
-
-// ------------------------------------------------------------------ tile plan fitted to the number of CTAs
-// A uniform grid of T tiles on G persistent CTAs takes ceil(T / G) tile times although it holds only T / G of
-// work per CTA (the 4096^3 GEMM: 256 tiles of 256 x 256 on 148 CTAs = 1.73 tile times of work done in 2).  The
-// plan keeps the tile height and cuts some row blocks into narrower tiles (widths w < tile_n, both multiples of
-// 64) so that every CTA ends at about the same time: tiles are dealt longest first, each to the CTA with the
-// least work so far.  The cost model is the measured instruction time of one MMA (N / 2 cycles, at least 60)
-// plus a fixed and a per-column epilogue cost.
-struct TilePlan {
-    std::vector<int4> table;   // [round * grid + cta] = (row block, first column, width, 0)
-    int rounds = 0;
-    int grid = 0;
-    double makespan = 0.0;     // model cycles
-    double uniform = 0.0;      // the same for the uniform grid
-};
-
-// mmas_per_kb: MMAs one CTA's tensor core runs per 64-deep K block (4 per 128 rows it owns)
-double tile_cost_cycles(int mmas_per_kb, int width, int64_t num_kb) {
-    const double mma = std::max(width / 2.0, 60.0);
-    return static_cast<double>(num_kb) * mmas_per_kb * mma + 1500.0 + 13.0 * width;
-}
-
-// makespan of `na` tiles of cost ca and `nb` tiles of cost cb (ca >= cb > 0), dealt longest first on g CTAs, each
-// to the CTA with the least work so far (closed form of that greedy rule for two sizes)
-double lpt_two_sizes(int64_t na, double ca, int64_t nb, double cb, int g) {
-    const int64_t q = na / g, x = na % g;              // x CTAs hold q + 1 wide tiles, g - x hold q
-    const double low = ca * static_cast<double>(q), high = x > 0 ? low + ca : low;
-    if (nb <= 0) return high;
-    if (x == 0) return low + cb * static_cast<double>(ceil_div(nb, g));
-    // the g - x lighter CTAs take narrow tiles until they have caught up with the others
-    const int64_t catch_up = static_cast<int64_t>(std::ceil(ca / cb - 1e-9));
-    const int64_t lighter = g - x;
-    if (nb <= catch_up * lighter) return std::max(high, low + cb * static_cast<double>(ceil_div(nb, lighter)));
-    const double low2 = low + cb * static_cast<double>(catch_up);      // >= high, by less than cb
-    const int64_t rest = nb - catch_up * lighter;
-    const int64_t f = rest / g, rem = rest % g;
-    if (rem == 0) return low2 + cb * static_cast<double>(f);
-    if (rem <= x) return std::max(low2 + cb * static_cast<double>(f), high + cb * static_cast<double>(f + 1));
-    return low2 + cb * static_cast<double>(f + 1);
-}
-
-// Searches widths and how many row blocks take the narrower cut.  Returns false when nothing beats the uniform grid
-// by `min_gain` (relative).
-// `g` workers (CTAs, or CTA pairs when pair is set: a pair's two tensor cores share a 256-row tile).
-bool plan_fitted_tiles(int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int raster, int g, double min_gain,
-                       TilePlan* out, bool pair = false) {
-    const int64_t tiles_m = ceil_div(M, bm);
-    const int64_t uniform_tiles = tiles_m * ceil_div(N, bn);
-    const int mmas = pair ? 4 : 4 * (bm / 128);
-    const double c_big = tile_cost_cycles(mmas, bn, num_kb);
-    const double uniform = lpt_two_sizes(uniform_tiles, c_big, 0, 0.0, g);
-    double best = uniform;
-    int best_w = 0;
-    int64_t best_b = 0, best_b1 = 0, best_e = 0;
-    // pairs: each CTA loads half of a tile's columns, kept a multiple of 64 (one copy per 64 rows)
-    const int w_step = pair ? 128 : 64;
-    for (int w = bn - w_step; w >= 128; w -= w_step) {
-        const double c_small = tile_cost_cycles(mmas, w, num_kb);
-        // option b of a row block: b tiles of width w at the high columns, a(b) tiles of width bn before them
-        auto bigs_for = [&](int64_t b) { return ceil_div(std::max<int64_t>(0, N - b * w), bn); };
-        // options that do not carry a tile more than needed
-        std::vector<int64_t> opts;
-        for (int64_t b = 0; b <= ceil_div(N, w); ++b)
-            if (b == 0 || bigs_for(b) * bn + b * w - N < w) opts.push_back(b);
-        for (size_t i = 0; i < opts.size(); ++i)
-        for (size_t j = i + 1; j < opts.size(); ++j) {
-            const int64_t b0 = opts[i], b1 = opts[j];
-            for (int64_t e = 0; e <= tiles_m; ++e) {                            // e row blocks take option b1
-                const int64_t na = (tiles_m - e) * bigs_for(b0) + e * bigs_for(b1);
-                const int64_t nb = (tiles_m - e) * b0 + e * b1;
-                const double m = lpt_two_sizes(na, c_big, nb, c_small, g);
-                if (m < best * (1.0 - 1e-9)) { best = m; best_w = w; best_b = b0; best_b1 = b1; best_e = e; }
-            }
-        }
-    }
-    out->uniform = uniform;
-    out->makespan = best;
-    if (best_w == 0 || best > uniform * (1.0 - min_gain)) return false;
-    // list the tiles: wide ones first, each group in the panel order of the uniform grid (row blocks fastest
-    // inside a panel of `raster` row blocks, then columns, then panels)
-    const int w = best_w;
-    auto bigs_for = [&](int64_t b) { return ceil_div(std::max<int64_t>(0, N - b * w), static_cast<int64_t>(bn)); };
-    struct T { int m, n0, width; };
-    std::vector<T> wide, narrow;
-    const int64_t panel = raster <= 0 ? tiles_m : std::min<int64_t>(raster, tiles_m);
-    for (int64_t m0 = 0; m0 < tiles_m; m0 += panel) {
-        const int64_t rows = std::min(panel, tiles_m - m0);
-        const int64_t max_cols = ceil_div(N, 64) + 1;
-        for (int64_t c = 0; c < max_cols; ++c)          // c-th tile of each row block of the panel
-            for (int64_t r = 0; r < rows; ++r) {
-                const int64_t m = m0 + r;
-                const int64_t b = (m >= tiles_m - best_e) ? best_b1 : best_b;
-                const int64_t a = bigs_for(b);
-                if (c < a) wide.push_back({static_cast<int>(m), static_cast<int>(c * bn), bn});
-                else if (c < a + b) narrow.push_back({static_cast<int>(m), static_cast<int>(a * bn + (c - a) * w), w});
-            }
-    }
-    const int64_t total = static_cast<int64_t>(wide.size() + narrow.size());
-    const int grid = static_cast<int>(std::min<int64_t>(total, g));
-    std::vector<std::vector<T>> per(grid);
-    std::vector<double> load(grid, 0.0);
-    const double c_small = tile_cost_cycles(mmas, w, num_kb);
-    auto deal = [&](const std::vector<T>& v, double cost) {
-        for (const T& t : v) {
-            int who = 0;
-            for (int i = 1; i < grid; ++i) if (load[i] < load[who] - 1e-6) who = i;
-            per[who].push_back(t);
-            load[who] += cost;
-        }
-    };
-    deal(wide, c_big);
-    deal(narrow, c_small);
-    size_t rounds = 0;
-    for (auto& v : per) rounds = std::max(rounds, v.size());
-    out->grid = grid;
-    out->rounds = static_cast<int>(rounds);
-    out->table.assign(rounds * grid, make_int4(0, 0, 0, 0));
-    for (int i = 0; i < grid; ++i)
-        for (size_t k = 0; k < per[i].size(); ++k)
-            out->table[k * grid + i] = make_int4(per[i][k].m, per[i][k].n0, per[i][k].width, 0);
-    return true;
-}
-
-// Device copies of tile plans, one per (shape, tile, CTA count); never freed (a few KB each).
-struct PlanKey {
-    int64_t M, N, num_kb;
-    int bm, bn, raster, g, forced, pair;
-    bool operator<(const PlanKey& o) const { return std::memcmp(this, &o, sizeof(PlanKey)) < 0; }
-};
-struct DevicePlan { int4* dev = nullptr; int rounds = 0, grid = 0; bool fitted = false; };
-std::map<PlanKey, DevicePlan> g_plans;
-
-// Looks the plan up (building and uploading it on first use; the upload is ordered on `st` before the kernel).
-int get_tile_plan(DeviceCtx* ctx, int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int raster, double min_gain,
-                  cudaStream_t st, DevicePlan* out, bool pair = false) {
-    PlanKey key;
-    std::memset(&key, 0, sizeof key);
-    key.M = M; key.N = N; key.num_kb = num_kb; key.bm = bm; key.bn = bn; key.raster = raster; key.g = pair ? ctx->sm_count / 2 : ctx->sm_count; key.forced = min_gain <= 0.0 ? 1 : 0;
-    key.pair = pair ? 1 : 0;
-    {
-        std::lock_guard<std::mutex> lk(g_mu);
-        auto it = g_plans.find(key);
-        if (it != g_plans.end()) { *out = it->second; return TDX_OK; }
-    }
-    TilePlan plan;
-    DevicePlan d;
-    d.fitted = plan_fitted_tiles(M, N, num_kb, bm, bn, raster, key.g, min_gain, &plan, pair);
-    if (d.fitted) {
-        const size_t bytes = plan.table.size() * sizeof(int4);
-        void* dev = nullptr;
-        TDX_CUDA(cudaMalloc(&dev, bytes));
-        // the table is a std::vector about to go out of scope: copy synchronously (once per shape)
-        TDX_CUDA(cudaMemcpy(dev, plan.table.data(), bytes, cudaMemcpyHostToDevice));
-        d.dev = static_cast<int4*>(dev);
-        d.rounds = plan.rounds;
-        d.grid = plan.grid;
-    }
-    (void)st;
-    {
-        std::lock_guard<std::mutex> lk(g_mu);
-        g_plans[key] = d;
-    }
-    *out = d;
-    return TDX_OK;
-}
-
-// ------------------------------------------------------------------ launches
-int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
-                const UmmaParams& p_in, cudaStream_t st, bool halo = false, const CUtensorMap* ma_row = nullptr,
-                const CUtensorMap* mc_row = nullptr, int plan_grid = 0) {
-    const long long items = static_cast<long long>(p_in.tiles_m) * p_in.tiles_n * p_in.split_k;
-    UmmaParams p = p_in;
-    if (p.b_box == 0) p.b_box = p.bn;
-    const int grid = p.tiles != nullptr ? plan_grid : static_cast<int>(std::min<long long>(items, ctx->sm_count));
-    size_t smem = static_cast<size_t>(p.stages) * ((p.bm + p.bn) * 128) + 1024 +
-                  staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
-    if (halo)
-        smem = static_cast<size_t>(p.a_stages) * (p.bm / 128) * p.halo_bytes + static_cast<size_t>(p.stages) * p.bn * 128 +
-               1024 + staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
-    // producer warp, MMA warp, then 16 epilogue warps (staged epilogue) or 4 per 128-row half (direct)
-    const int threads = p.tma_store ? 576 : (p.bm == 256 ? 320 : 192);
-    // programmatic stream serialization: the grid may be scheduled while the previous kernel of the stream drains; its
-    // set-up then overlaps that tail, and it waits on the device for the predecessor before touching global memory
-    cudaLaunchConfig_t lc;
-    std::memset(&lc, 0, sizeof lc);
-    lc.gridDim = dim3(static_cast<unsigned>(grid));
-    lc.blockDim = dim3(static_cast<unsigned>(halo ? threads + 32 : threads));   // halo: one more warp, the halo producer
-    lc.dynamicSmemBytes = smem;
-    lc.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    lc.attrs = attr;
-    lc.numAttrs = 1;
-    if (halo)
-        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_conv_halo_kernel, ma, ma_row ? *ma_row : ma, mb, mc, mc_row ? *mc_row : mc, p));
-    else if (conv)
-        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_contract_kernel<true>, ma, mb, mc, p));
-    else
-        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_contract_kernel<false>, ma, mb, mc, p));
-    TDX_CUDA(cudaGetLastError());
-    g_launches.fetch_add(1);
-    return TDX_OK;
-}
-
-// The reduction is launched with programmatic stream serialization so that its launch latency hides behind
-// the tail of the GEMM kernel; it waits on the device for the GEMM grid to complete before reading partials.
-int launch_splitk_reduce(int grid, cudaStream_t st, long long MN, int N, int split, const float* partial, float alpha,
-                         __nv_bfloat16* out, int vec8, float beta = 0.0f) {
-    cudaLaunchConfig_t lc;
-    std::memset(&lc, 0, sizeof lc);
-    lc.gridDim = dim3(static_cast<unsigned>(grid));
-    lc.blockDim = dim3(256);
-    lc.dynamicSmemBytes = 0;
-    lc.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    lc.attrs = attr;
-    lc.numAttrs = 1;
-    const float* bias = nullptr;
-    int relu = 0;
-    TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::splitk_reduce_kernel, MN, N, split, partial, alpha, bias, relu, out, vec8, beta));
-    g_launches.fetch_add(1);
-    return TDX_OK;
-}
-
-int ensure_ws(DeviceCtx* ctx, size_t bytes, void** out) {
-    if (ctx->ws_bytes < bytes) {
-        if (ctx->ws) TDX_CUDA(cudaFree(ctx->ws));
-        ctx->ws = nullptr;
-        ctx->ws_bytes = 0;
-        TDX_CUDA(cudaMalloc(&ctx->ws, bytes));
-        ctx->ws_bytes = bytes;
-    }
-    *out = ctx->ws;
-    return TDX_OK;
-}
-
-int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
-                  const tdx_config& cfg, void* ws, size_t ws_bytes, bool internal_ws, cudaStream_t st, float beta = 0.0f) {
-    const int64_t num_kb = ceil_div(g.K, 64);
-    UmmaParams p;
-    std::memset(&p, 0, sizeof p);
-    p.M = static_cast<int>(g.M);
-    p.N = static_cast<int>(g.N);
-    p.num_kb = static_cast<int>(num_kb);
-    p.bm = cfg.tile_m;
-    p.slots = tmem_slots_for(cfg.tile_m, cfg.tile_n);
-    p.tiles_m = static_cast<int>(ceil_div(g.M, cfg.tile_m));
-    p.tiles_n = static_cast<int>(ceil_div(g.N, cfg.tile_n));
-    p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
-    p.split_k = cfg.split_k;
-    p.kb_per_split = static_cast<int>(ceil_div(num_kb, cfg.split_k));
-    p.k_stagger = cfg.k_stagger;
-    p.bn = cfg.tile_n;
-    p.stages = cfg.stages;
-    p.tmem_cols = tmem_cols_for(cfg.tile_m, cfg.tile_n);
-    p.a_mn_major = g.transA ? 1 : 0;   // A stored K x M: M contiguous
-    p.b_mn_major = g.transB ? 0 : 1;   // B stored K x N: N contiguous
-    p.alpha = alpha;
-    p.beta = beta;
-    p.bias = nullptr;
-    p.relu = 0;
-    p.C = static_cast<__nv_bfloat16*>(C);
-    p.ldc = g.N;
-    p.status = ctx->status_ptr;
-    p.vec_store = (g.N % 8 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
-
-    if (cfg.split_k > 1) {
-        const size_t need = static_cast<size_t>(cfg.split_k) * g.M * g.N * sizeof(float);
-        if (internal_ws) {
-            int rc = ensure_ws(ctx, need, &ws);
-            if (rc) return rc;
-        } else if (ws == nullptr || ws_bytes < need || reinterpret_cast<uintptr_t>(ws) % 256) {
-            return fail(TDX_ERR_WORKSPACE, "split_k=%d needs %zu bytes of 256-byte aligned workspace", cfg.split_k, need);
-        }
-        p.partial = static_cast<float*>(ws);
-    }
-
-    CUtensorMap ma, mb;
-    int rc;
-    if (p.a_mn_major) {
-        uint64_t dims[2] = {static_cast<uint64_t>(g.M), static_cast<uint64_t>(g.K)};
-        uint64_t str[1] = {static_cast<uint64_t>(g.M) * 2};
-        uint32_t box[2] = {64, 64};
-        rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
-    } else {
-        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.M)};
-        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
-        uint32_t box[2] = {64, 128};
-        rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
-    }
-    if (rc) return rc;
-    // tile widths fitted to the number of CTAs (see plan_fitted_tiles): B then arrives in 64-row copies
-    int plan_grid = 0;
-    if (cfg.fit != 1 && cfg.split_k == 1 && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0) {
-        DevicePlan dp;
-        rc = get_tile_plan(ctx, g.M, g.N, num_kb, cfg.tile_m, cfg.tile_n, cfg.raster, cfg.fit == 2 ? 0.0 : 0.03, st, &dp);
-        if (rc) return rc;
-        if (dp.fitted) {
-            p.tiles = dp.dev;
-            p.rounds = dp.rounds;
-            p.b_box = 64;
-            plan_grid = dp.grid;
-        }
-    }
-    if (p.b_mn_major) {
-        uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.K)};
-        uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
-        uint32_t box[2] = {64, 64};
-        rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
-    } else {
-        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.N)};
-        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
-        uint32_t box[2] = {64, static_cast<uint32_t>(p.tiles ? 64 : cfg.tile_n)};
-        rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
-    }
-    if (rc) return rc;
-
-    CUtensorMap mc = ma;   // unused unless the staged epilogue is on
-    // the accumulate term is read by the direct-store epilogue (and by the split-K reduction) only
-    p.tma_store = (cfg.store_mode == 2 && cfg.split_k == 1 && p.vec_store && beta == 0.0f) ? 1 : 0;
-    if (p.tma_store) {
-        uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.M)};
-        uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
-        uint32_t box[2] = {32, 32};
-        rc = get_tensor_map(ctx, C, 2, dims, str, box, &mc, 64);
-        if (rc) return rc;
-    }
-    rc = launch_umma(ctx, false, ma, mb, mc, p, st, false, nullptr, nullptr, plan_grid);
-    if (rc) return rc;
-    if (cfg.split_k > 1) {
-        const long long MN = static_cast<long long>(g.M) * g.N;
-        const int vec8 = p.vec_store ? 1 : 0;
-        const long long work = vec8 ? MN / 8 : MN;
-        const int grid = static_cast<int>(std::min<long long>(ceil_div(work, 256), 148LL * 16));
-        rc = launch_splitk_reduce(std::max(grid, 1), st, MN, static_cast<int>(g.N), cfg.split_k, p.partial, alpha, p.C, vec8, beta);
-        if (rc) return rc;
-    }
-    return TDX_OK;
-}
-
-// GEMM on CTA pairs: 256 x tile_n per pair, each CTA loads its 128 rows of A and tile_n / 2 columns of B.
-int run_gemm_pair(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
-                  const tdx_config& cfg, cudaStream_t st) {
-    const int64_t num_kb = ceil_div(g.K, 64);
-    UmmaParams p;
-    std::memset(&p, 0, sizeof p);
-    p.M = static_cast<int>(g.M);
-    p.N = static_cast<int>(g.N);
-    p.num_kb = static_cast<int>(num_kb);
-    p.bm = 128;                                      // what one CTA of the pair owns (epilogue geometry)
-    p.slots = 2 * cfg.tile_n <= 256 ? 4 : 2;
-    p.tiles_m = static_cast<int>(ceil_div(g.M, 256));
-    p.tiles_n = static_cast<int>(ceil_div(g.N, cfg.tile_n));
-    p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
-    p.split_k = 1;
-    p.kb_per_split = p.num_kb;
-    p.bn = cfg.tile_n;
-    p.stages = cfg.stages;
-    p.tmem_cols = 32;
-    while (p.tmem_cols < p.slots * cfg.tile_n) p.tmem_cols *= 2;
-    p.a_mn_major = g.transA ? 1 : 0;
-    p.b_mn_major = g.transB ? 0 : 1;
-    p.alpha = alpha;
-    p.C = static_cast<__nv_bfloat16*>(C);
-    p.ldc = g.N;
-    p.status = ctx->status_ptr;
-    p.vec_store = (g.N % 8 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
-    p.tma_store = (cfg.store_mode == 2 && p.vec_store) ? 1 : 0;
-
-    CUtensorMap ma, mb, mc;
-    int rc;
-    if (p.a_mn_major) {
-        uint64_t dims[2] = {static_cast<uint64_t>(g.M), static_cast<uint64_t>(g.K)};
-        uint64_t str[1] = {static_cast<uint64_t>(g.M) * 2};
-        uint32_t box[2] = {64, 64};
-        rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
-    } else {
-        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.M)};
-        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
-        uint32_t box[2] = {64, 128};
-        rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
-    }
-    if (rc) return rc;
-    // tile widths fitted to the number of pairs; each CTA's half of a tile's B columns then arrives in 64-row copies
-    // (K-major B only: an N-major half would have to be a multiple of 64 columns)
-    p.b_box = cfg.tile_n / 2;
-    int plan_pairs = 0;
-    // only on request: a 256 x 128 x 16 pair MMA measured 115 cycles, not 64, so narrow tiles gain nothing here
-    if (cfg.fit == 2 && !p.b_mn_major && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0) {
-        DevicePlan dp;
-        rc = get_tile_plan(ctx, g.M, g.N, num_kb, 256, cfg.tile_n, cfg.raster, 0.0, st, &dp, true);
-        if (rc) return rc;
-        if (dp.fitted) {
-            p.tiles = dp.dev;
-            p.rounds = dp.rounds;
-            p.b_box = 64;
-            plan_pairs = dp.grid;
-        }
-    }
-    if (p.b_mn_major) {
-        uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.K)};
-        uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
-        uint32_t box[2] = {64, 64};
-        rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
-    } else {
-        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.N)};
-        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
-        uint32_t box[2] = {64, static_cast<uint32_t>(p.b_box)};
-        rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
-    }
-    if (rc) return rc;
-    mc = ma;
-    if (p.tma_store) {
-        uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.M)};
-        uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
-        uint32_t box[2] = {32, 32};
-        rc = get_tensor_map(ctx, C, 2, dims, str, box, &mc, 64);
-        if (rc) return rc;
-    }
-    const long long pair_tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
-    const int pairs = p.tiles ? plan_pairs : static_cast<int>(std::min<long long>(pair_tiles, ctx->sm_count / 2));
-    cudaLaunchConfig_t lc;
-    std::memset(&lc, 0, sizeof lc);
-    lc.gridDim = dim3(static_cast<unsigned>(2 * pairs));
-    lc.blockDim = dim3(p.tma_store ? 576 : 192);
-    lc.dynamicSmemBytes = static_cast<size_t>(p.stages) * ((128 + p.bn / 2) * 128) + 1024 +
-                          staging_bytes_for(128, p.tma_store ? 2 : 1);
-    lc.stream = st;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
-    lc.attrs = attr;
-    lc.numAttrs = 1;
-    TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_pair_kernel, ma, mb, mc, p));
-    g_launches.fetch_add(1);
-    return TDX_OK;
-}
-
-int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const void* w, const float* bias, int relu,
-                  void* y, const tdx_config& cfg, cudaStream_t st, const void* residual = nullptr) {
-    const int cchunks = static_cast<int>(ceil_div(c.Cin, 64));
-    UmmaParams p;
-    std::memset(&p, 0, sizeof p);
-    p.bw = cfg.patch_w;
-    p.bh = cfg.patch_h;
-    p.bm = cfg.tile_m;
-    p.slots = tmem_slots_for(cfg.tile_m, cfg.tile_n);
-    p.nb = cfg.tile_m / (p.bw * p.bh);
-    const bool halo = cfg.halo >= 2;
-    const bool stacked = cfg.halo == 3;
-    if (halo) {
-        p.R = static_cast<int>(c.R);
-        p.hpitch = static_cast<int>(kHaloPatchW + c.S - 1);
-        p.hrows = static_cast<int>(kHaloPatchH + c.R - 1);
-        p.halo_bytes = halo_tile_bytes(c.R, c.S);
-        p.a_stages = kHaloAStages;
-    }
-    p.patches_w = static_cast<int>(ceil_div(c.Q, p.bw));
-    p.patches_h = static_cast<int>(ceil_div(c.P, p.bh));
-    int64_t total_patches = c.N * p.patches_w * p.patches_h;
-    if (stacked) {
-        p.Pv = static_cast<int>(stacked_rows_per_image(c));
-        p.H = static_cast<int>(c.H);
-        p.patches_h = static_cast<int>(ceil_div(c.N * p.Pv, p.bh));      // over the whole column of images
-        total_patches = static_cast<int64_t>(p.patches_w) * p.patches_h;
-    }
-    p.M = static_cast<int>(c.N * c.P * c.Q);
-    p.N = static_cast<int>(c.Cout);
-    p.num_kb = static_cast<int>(c.R * c.S * cchunks);
-    p.tiles_m = static_cast<int>(ceil_div(total_patches, p.nb));
-    p.tiles_n = static_cast<int>(ceil_div(c.Cout, cfg.tile_n));
-    p.panel = cfg.raster == 0 ? p.tiles_m : std::min(cfg.raster, p.tiles_m);
-    p.split_k = 1;
-    p.kb_per_split = p.num_kb;
-    p.k_stagger = cfg.k_stagger;
-    p.bn = cfg.tile_n;
-    p.stages = cfg.stages;
-    if (halo && cfg.tile_n >= c.Cout) {
-        // small filters stay resident: all (chunk, tap) slices of the one column tile fit beside the halo ring,
-        // so they are loaded once per CTA and the main loop has no per-tap handshake
-        const int64_t slices = c.R * c.S * cchunks;
-        const int64_t need = static_cast<int64_t>(p.a_stages) * (cfg.tile_m / 128) * p.halo_bytes + slices * cfg.tile_n * 128 +
-                             staging_bytes_for(cfg.tile_m, cfg.store_mode) + 1024;
-        if (need <= ctx->smem_optin - kStaticSmemReserve) {
-            p.b_resident = 1;
-            p.stages = static_cast<int>(slices);
-            // spend what is left on more halo tiles in flight (their load latency is what a short tile waits for)
-            const int64_t per_stage = static_cast<int64_t>(cfg.tile_m / 128) * p.halo_bytes;
-            while (p.a_stages < tdx::kMaxAStages && need + (p.a_stages - kHaloAStages + 1) * per_stage <= ctx->smem_optin - kStaticSmemReserve)
-                ++p.a_stages;
-        }
-    }
-    p.tmem_cols = tmem_cols_for(cfg.tile_m, cfg.tile_n);
-    p.a_mn_major = 0;
-    p.b_mn_major = 0;
-    p.alpha = 1.0f;
-    p.bias = bias;
-    p.residual = static_cast<const __nv_bfloat16*>(residual);
-    p.relu = relu;
-    p.C = static_cast<__nv_bfloat16*>(y);
-    p.ldc = c.Cout;
-    p.vec_store = (c.Cout % 8 == 0) && (reinterpret_cast<uintptr_t>(y) % 16 == 0);
-    p.P = static_cast<int>(c.P);
-    p.Q = static_cast<int>(c.Q);
-    p.Nimg = static_cast<int>(c.N);
-    p.S = static_cast<int>(c.S);
-    p.pad = c.pad;
-    p.stride = c.stride;
-    p.cchunks = cchunks;
-    p.status = ctx->status_ptr;
-
-    CUtensorMap ma, ma_row, mb;
-    {
-        uint64_t dims[4] = {static_cast<uint64_t>(c.Cin), static_cast<uint64_t>(c.W), static_cast<uint64_t>(c.H),
-                            static_cast<uint64_t>(c.N)};
-        uint64_t str[3] = {static_cast<uint64_t>(c.Cin) * 2, static_cast<uint64_t>(c.W * c.Cin) * 2,
-                           static_cast<uint64_t>(c.H * c.W * c.Cin) * 2};
-        uint32_t box[4] = {64, static_cast<uint32_t>(halo ? p.hpitch : p.bw), static_cast<uint32_t>(halo ? p.hrows : p.bh), 1};
-        // strided convolution (per-tap loads only): the copy walks the image with the convolution's stride, so a
-        // box spanning bw * stride input pixels delivers exactly the bw pixels under one filter tap
-        uint32_t estr[4] = {1, static_cast<uint32_t>(c.stride), static_cast<uint32_t>(c.stride), 1};
-        if (c.stride > 1) { box[1] *= c.stride; box[2] *= c.stride; }
-        int rc = get_tensor_map(ctx, x, 4, dims, str, box, &ma, 128, c.stride > 1 ? estr : nullptr);
-        if (rc) return rc;
-        ma_row = ma;
-        if (stacked) {
-            box[2] = 1;              // windows that reach into the next image are copied one row at a time
-            rc = get_tensor_map(ctx, x, 4, dims, str, box, &ma_row);
-            if (rc) return rc;
-        }
-    }
-    {
-        uint64_t dims[3] = {static_cast<uint64_t>(c.Cin), static_cast<uint64_t>(c.R * c.S),
-                            static_cast<uint64_t>(c.Cout)};
-        uint64_t str[2] = {static_cast<uint64_t>(c.Cin) * 2, static_cast<uint64_t>(c.R * c.S * c.Cin) * 2};
-        uint32_t box[3] = {64, 1, static_cast<uint32_t>(cfg.tile_n)};
-        int rc = get_tensor_map(ctx, w, 3, dims, str, box, &mb);
-        if (rc) return rc;
-    }
-    CUtensorMap mc = ma, mc_row = ma;
-    p.tma_store = (cfg.store_mode == 2 && p.vec_store && p.bw * p.bh >= 32) ? 1 : 0;
-    // the staged epilogue reads the residual 16 bytes at a time
-    if (reinterpret_cast<uintptr_t>(residual) % 16) p.tma_store = 0;
-    if (halo) p.epi_warps = p.tma_store ? 16 : 4 * (cfg.tile_m / 128);
-    if (p.tma_store) {
-        p.sbx = std::min(p.bw, 32);
-        p.sby = 32 / p.sbx;
-        uint64_t dims[4] = {static_cast<uint64_t>(c.Cout), static_cast<uint64_t>(c.Q), static_cast<uint64_t>(c.P),
-                            static_cast<uint64_t>(c.N)};
-        uint64_t str[3] = {static_cast<uint64_t>(c.Cout) * 2, static_cast<uint64_t>(c.Q * c.Cout) * 2,
-                           static_cast<uint64_t>(c.P * c.Q * c.Cout) * 2};
-        uint32_t box[4] = {32, static_cast<uint32_t>(p.sbx), static_cast<uint32_t>(p.sby), 1};
-        int rc = get_tensor_map(ctx, y, 4, dims, str, box, &mc, 64);
-        if (rc) return rc;
-        mc_row = mc;
-        if (stacked) {
-            box[2] = 1;              // four pixel rows that cross the seam between two images leave one by one
-            rc = get_tensor_map(ctx, y, 4, dims, str, box, &mc_row, 64);
-            if (rc) return rc;
-        }
-    }
-    return launch_umma(ctx, true, ma, mb, mc, p, st, halo, &ma_row, &mc_row);
-}
-
-void gemm_strides(const GemmProblem& g, long long* sa_i, long long* sa_k, long long* sb_k, long long* sb_j) {
-    *sa_i = g.transA ? 1 : g.K;
-    *sa_k = g.transA ? g.M : 1;
-    *sb_k = g.transB ? 1 : g.N;
-    *sb_j = g.transB ? g.K : 1;
-}
-
-// batch count, batch strides in elements, and the accumulate factor of tdx_gemm_batched (one batch, beta = 0: tdx_gemm)
-struct BatchArgs {
-    int64_t batch = 1, stride_a = 0, stride_b = 0, stride_c = 0;
-    float beta = 0.0f;
-};
-
-int run_gemm_simt_f32(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
-                      cudaStream_t st, const BatchArgs& ba = BatchArgs()) {
-    if (g.M >= (1LL << 31) || g.N >= (1LL << 31) || g.K >= (1LL << 31))
-        return fail(TDX_ERR_UNSUPPORTED, "fp32 tiled GEMM needs dimensions below 2^31");
-    long long sa_i, sa_k, sb_k, sb_j;
-    gemm_strides(g, &sa_i, &sa_k, &sb_k, &sb_j);
-    const float* a = static_cast<const float*>(A);
-    const float* b = static_cast<const float*>(B);
-    float* c = static_cast<float*>(C);
-    if (ba.batch > 65535) return fail(TDX_ERR_UNSUPPORTED, "fp32 batched GEMM takes at most 65535 batches");
-    const unsigned nz = static_cast<unsigned>(ba.batch);
-    const bool plain = ba.batch == 1 && ba.beta == 0.0f;
-    const int64_t tiles64 = ceil_div(g.M, 64) * ceil_div(g.N, 64) * ba.batch;
-    if (tiles64 >= ctx->sm_count) {
-        // 64 x 64 tiles (4 x 4 outputs per thread) once there is one per SM; smaller problems take 32 x 32 tiles
-        dim3 grid(static_cast<unsigned>(ceil_div(g.N, 64)), static_cast<unsigned>(ceil_div(g.M, 64)), nz);
-        tdx::sgemm_ring_kernel<64, 64, 16, 4, 4, 4><<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k,
-                                                                         sb_j, alpha, a, b, c, ba.beta, ba.stride_a,
-                                                                         ba.stride_b, ba.stride_c);
-    } else {
-        dim3 grid(static_cast<unsigned>(ceil_div(g.N, 32)), static_cast<unsigned>(ceil_div(g.M, 32)), nz);
-        const bool rowmajor16 = plain && !g.transA && !g.transB && g.K % 4 == 0 && g.N % 4 == 0 &&
-                                reinterpret_cast<uintptr_t>(A) % 16 == 0 && reinterpret_cast<uintptr_t>(B) % 16 == 0;
-        if (rowmajor16)
-            tdx::sgemm_small_rowmajor_kernel<<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, alpha, a, b, c);
-        else
-            tdx::sgemm_small_kernel<<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k, sb_j, alpha, a, b,
-                                                          c, ba.beta, ba.stride_a, ba.stride_b, ba.stride_c);
-    }
-    TDX_CUDA(cudaGetLastError());
-    g_launches.fetch_add(1);
-    return TDX_OK;
-}
-
-int run_gemm_generic(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
-                     cudaStream_t st, const BatchArgs& ba = BatchArgs()) {
-    long long sa_i, sa_k, sb_k, sb_j;
-    gemm_strides(g, &sa_i, &sa_k, &sb_k, &sb_j);
-    const long long total = g.M * g.N * ba.batch;
-    const int grid = static_cast<int>(std::min<long long>(ceil_div(total, 256), static_cast<long long>(ctx->sm_count) * 32));
-    if (g.dtype == TDX_F32)
-        tdx::gemm_generic_kernel<float, float><<<grid, 256, 0, st>>>(g.M, g.N, g.K, sa_i, sa_k, sb_k, sb_j, alpha,
-                                                                    static_cast<const float*>(A),
-                                                                    static_cast<const float*>(B), static_cast<float*>(C),
-                                                                    ba.beta, ba.batch, ba.stride_a, ba.stride_b, ba.stride_c);
-    else
-        tdx::gemm_generic_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
-            g.M, g.N, g.K, sa_i, sa_k, sb_k, sb_j, alpha, static_cast<const __nv_bfloat16*>(A),
-            static_cast<const __nv_bfloat16*>(B), static_cast<__nv_bfloat16*>(C), ba.beta, ba.batch, ba.stride_a,
-            ba.stride_b, ba.stride_c);
-    TDX_CUDA(cudaGetLastError());
-    g_launches.fetch_add(1);
-    return TDX_OK;
-}
-
-int run_conv_generic(DeviceCtx* ctx, const ConvProblem& c, const void* x, const void* w, const float* bias, int relu,
-                     void* y, cudaStream_t st, const void* residual = nullptr) {
-    if (c.N >= (1LL << 31) || c.H >= (1LL << 31) || c.W >= (1LL << 31) || c.Cin >= (1LL << 31) ||
-        c.Cout >= (1LL << 31) || c.R >= (1LL << 31) || c.S >= (1LL << 31))
-        return fail(TDX_ERR_UNSUPPORTED, "conv dimensions must be below 2^31");
-    const long long total = c.N * c.P * c.Q * c.Cout;
-    const int grid = static_cast<int>(std::min<long long>(ceil_div(total, 256), static_cast<long long>(ctx->sm_count) * 32));
-    if (c.dtype == TDX_F32)
-        tdx::conv2d_generic_kernel<float, float><<<grid, 256, 0, st>>>(
-            (int)c.N, (int)c.H, (int)c.W, (int)c.Cin, (int)c.Cout, (int)c.R, (int)c.S, c.pad, c.stride, (int)c.P,
-            (int)c.Q, static_cast<const float*>(x), static_cast<const float*>(w), bias, relu, static_cast<float*>(y),
-            static_cast<const float*>(residual));
-    else
-        tdx::conv2d_generic_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
-            (int)c.N, (int)c.H, (int)c.W, (int)c.Cin, (int)c.Cout, (int)c.R, (int)c.S, c.pad, c.stride, (int)c.P,
-            (int)c.Q, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w), bias, relu,
-            static_cast<__nv_bfloat16*>(y), static_cast<const __nv_bfloat16*>(residual));
-    TDX_CUDA(cudaGetLastError());
-    g_launches.fetch_add(1);
-    return TDX_OK;
-}
-
 // ------------------------------------------------------------------ validation
 int validate_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const void* A, const void* B,
                   const void* C, bool need_ptrs) {
