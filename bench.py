@@ -62,7 +62,7 @@ WORKLOADS = {
                 label="gemm_bf16_4096x4096x512"),
     # the paper's own workload (Case Study 4): C[b,i,j] += A[b,i,k] * B[b,k,j], b < 6, i < 196, j < 256, k < 2305
     "cs4": dict(kind="gemm_batched", dtype="f32", batch=6, M=196, N=256, K=2305, tA=0, tB=0, alpha=1.0, beta=1.0, seed=5,
-                bound="alu", label="batch_matmul_accumulate_f32_6x196x256x2305"),
+                bound="tensor", label="batch_matmul_accumulate_f32_6x196x256x2305"),
     # Case Study 3's add_of_zero_pad pattern as an op: y += zero_pad(x) in place, the activation shape of c4
     "azp": dict(kind="add_zero_pad", dtype="bf16", N=32, H=56, W=56, C=256, pad=1, seed=6, bound="hbm",
                 label="add_of_zero_pad_bf16_32x56x56x256_pad1_in_place"),
@@ -354,7 +354,7 @@ def run_tdx(args):
             h_out.copy_(h_in[2].reshape(-1))
             return tdx.tdx_gemm_batched_host(w["batch"], w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], w["beta"], DT,
                                              h_in[0], h_in[1], h_out, stream)
-        kernel_name = "sgemm_small_kernel (fp32 CUDA cores, batch in grid.z)"
+        kernel_name = "umma_contract_kernel<false> on bf16 pieces (+ split_f32_bf16x3_kernel, splitk_reduce_f32_kernel)"
     elif w["kind"] == "gemm":
         st_cfg, cfg = tdx.tdx_default_gemm_config(w["M"], w["N"], w["K"], w["tA"], w["tB"], DT)
 

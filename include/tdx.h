@@ -51,7 +51,8 @@ typedef enum {
 
 typedef enum {
     TDX_KERNEL_AUTO = 0,
-    TDX_KERNEL_UMMA = 1,    /* tcgen05 tensor-core pipeline (bf16 only, needs 16-byte aligned pitches) */
+    TDX_KERNEL_UMMA = 1,    /* tcgen05 tensor-core pipeline (bf16: needs 16-byte aligned pitches; fp32 GEMM: */
+                            /* through three bf16 pieces per operand, any shape)                        */
     TDX_KERNEL_SIMT = 2,    /* tiled fp32 CUDA-core GEMM (fp32 GEMM only)                              */
     TDX_KERNEL_GENERIC = 3  /* one thread per output; any dtype, shape and alignment                   */
 } tdx_kernel;
@@ -103,6 +104,11 @@ typedef struct {
  *   transB = 0: B stored K x N;  transB = 1: B stored N x K.
  *   dtype: TDX_F32 (all fp32) or TDX_BF16 (bf16 in, fp32 accumulate, bf16 out, one rounding of alpha*acc).
  *   M or N = 0: no-op.  K = 0: C is zero-filled.
+ *   fp32: small problems run fp32 FMAs on the CUDA cores; from about 2^28 multiply-adds on (or with kernel =
+ *   TDX_KERNEL_UMMA in an explicit config) each operand is cut into three bf16 pieces that together hold all 24
+ *   significand bits, and the tensor cores accumulate the six piece products that matter in fp32 -- same 1e-5
+ *   bound, several times faster.  That path keeps its pieces in device scratch owned by the library, grown on
+ *   demand by cudaMalloc (make the first call for a size before any stream capture).
  * Errors: INVALID_ARG (negative size, flag not 0/1, NULL pointer with non-empty problem, unknown dtype,
  *         non-finite alpha is allowed), CUDA.  Shapes that miss the tensor-core path's alignment rules
  *         are served by the generic GPU kernel, not rejected.  There is no CPU fallback.

@@ -77,9 +77,18 @@ int ensure_ws(DeviceCtx* ctx, size_t bytes, void** out) {
     return TDX_OK;
 }
 
+// fp32 GEMM from bf16 pieces: the operands handed to run_gemm_umma hold three pieces of `seg_kb` K blocks side by side
+// (cols = 3 * 64 * seg_kb columns), g.K spans the six piece pairs, and C is fp32.
+struct PieceInfo {
+    int seg_kb = 0;
+    int64_t cols = 0;
+};
+
 int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
-                  const tdx_config& cfg, void* ws, size_t ws_bytes, bool internal_ws, cudaStream_t st, float beta = 0.0f) {
+                  const tdx_config& cfg, void* ws, size_t ws_bytes, bool internal_ws, cudaStream_t st, float beta = 0.0f,
+                  const PieceInfo* pieces = nullptr) {
     const int64_t num_kb = ceil_div(g.K, 64);
+    const int64_t k_cols = pieces ? pieces->cols : g.K;        // columns the K-major operands really have
     UmmaParams p;
     std::memset(&p, 0, sizeof p);
     p.M = static_cast<int>(g.M);
@@ -106,6 +115,16 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     p.ldc = g.N;
     p.status = ctx->status_ptr;
     p.vec_store = (g.N % 8 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+    if (pieces) {
+        if (p.a_mn_major || p.b_mn_major) return fail(TDX_ERR_CONFIG, "the fp32 GEMM from bf16 pieces runs K-major operands");
+        // smallest terms first, the hi * hi products last: (hi, lo) (lo, hi) (mid, mid) (hi, mid) (mid, hi) (hi, hi)
+        const int a_seg[6] = {0, 2, 1, 0, 1, 0}, b_seg[6] = {2, 0, 1, 1, 0, 0};
+        for (int i = 0; i < 6; ++i) { p.a_seg[i] = a_seg[i]; p.b_seg[i] = b_seg[i]; }
+        p.seg_kb = pieces->seg_kb;
+        p.Cf = static_cast<float*>(C);
+        p.C = nullptr;
+        p.vec_store = (g.N % 4 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+    }
 
     if (cfg.split_k > 1) {
         const size_t need = static_cast<size_t>(cfg.split_k) * g.M * g.N * sizeof(float);
@@ -126,8 +145,8 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         uint32_t box[2] = {64, 64};
         rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
     } else {
-        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.M)};
-        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
+        uint64_t dims[2] = {static_cast<uint64_t>(k_cols), static_cast<uint64_t>(g.M)};
+        uint64_t str[1] = {static_cast<uint64_t>(k_cols) * 2};
         uint32_t box[2] = {64, 128};
         rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
     }
@@ -151,8 +170,8 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         uint32_t box[2] = {64, 64};
         rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
     } else {
-        uint64_t dims[2] = {static_cast<uint64_t>(g.K), static_cast<uint64_t>(g.N)};
-        uint64_t str[1] = {static_cast<uint64_t>(g.K) * 2};
+        uint64_t dims[2] = {static_cast<uint64_t>(k_cols), static_cast<uint64_t>(g.N)};
+        uint64_t str[1] = {static_cast<uint64_t>(k_cols) * 2};
         uint32_t box[2] = {64, static_cast<uint32_t>(p.tiles ? 64 : cfg.tile_n)};
         rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
     }
@@ -160,7 +179,7 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
 
     CUtensorMap mc = ma;   // unused unless the staged epilogue is on
     // the accumulate term is read by the direct-store epilogue (and by the split-K reduction) only
-    p.tma_store = (cfg.store_mode == 2 && cfg.split_k == 1 && p.vec_store && beta == 0.0f) ? 1 : 0;
+    p.tma_store = (cfg.store_mode == 2 && cfg.split_k == 1 && p.vec_store && beta == 0.0f && !pieces) ? 1 : 0;
     if (p.tma_store) {
         uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.M)};
         uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
@@ -170,6 +189,26 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     }
     rc = launch_umma(ctx, false, ma, mb, mc, p, st, false, nullptr, nullptr, plan_grid);
     if (rc) return rc;
+    if (cfg.split_k > 1 && pieces) {
+        // fp32 result: partial sums (fp32, dense) -> alpha * sum + beta * C
+        const long long MN = static_cast<long long>(g.M) * g.N;
+        const int vec4 = (MN % 4 == 0 && reinterpret_cast<uintptr_t>(C) % 16 == 0) ? 1 : 0;
+        const int grid = static_cast<int>(std::min<long long>(ceil_div(vec4 ? MN / 4 : MN, 256), 148LL * 16));
+        cudaLaunchConfig_t lc;
+        std::memset(&lc, 0, sizeof lc);
+        lc.gridDim = dim3(static_cast<unsigned>(std::max(grid, 1)));
+        lc.blockDim = dim3(256);
+        lc.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = attr;
+        lc.numAttrs = 1;
+        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::splitk_reduce_f32_kernel, MN, cfg.split_k, static_cast<const float*>(p.partial), alpha,
+                                    beta, static_cast<float*>(C), vec4));
+        g_launches.fetch_add(1);
+        return TDX_OK;
+    }
     if (cfg.split_k > 1) {
         const long long MN = static_cast<long long>(g.M) * g.N;
         const int vec8 = p.vec_store ? 1 : 0;
@@ -451,6 +490,99 @@ int run_gemm_simt_f32(DeviceCtx* ctx, const GemmProblem& g, float alpha, const v
     }
     TDX_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
+    return TDX_OK;
+}
+
+// fp32 GEMM on the tensor cores.  Each fp32 operand is cut into three bf16 pieces (hi + mid + lo = the value, all 24
+// significand bits), written K-major whatever the operand's own layout, and the tensor-core kernel accumulates the six
+// piece pairs that matter ((mid, lo), (lo, mid) and (lo, lo) are below 2^-24 of the product) in fp32 -- six times
+// the MMA work of a bf16 GEMM, still several times faster than fp32 FMAs.  Scratch for the pieces is grown on demand.
+int ensure_pieces(DeviceCtx* ctx, int slot, size_t bytes, void** out) {
+    if (ctx->pieces_bytes[slot] < bytes) {
+        if (ctx->pieces[slot]) TDX_CUDA(cudaFree(ctx->pieces[slot]));
+        ctx->pieces[slot] = nullptr;
+        ctx->pieces_bytes[slot] = 0;
+        TDX_CUDA(cudaMalloc(&ctx->pieces[slot], bytes));
+        ctx->pieces_bytes[slot] = bytes;
+    }
+    *out = ctx->pieces[slot];
+    return TDX_OK;
+}
+
+int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_count, int smem_limit, tdx_config* out);
+
+constexpr size_t kPiecesMaxBytes = size_t(3) << 30;     // per operand; larger problems go batch by batch, or to the CUDA cores
+
+bool gemm_f32_pieces_fit(const GemmProblem& g) {
+    if (g.M >= (1LL << 31) || g.N >= (1LL << 31) || g.K >= (1LL << 28)) return false;
+    const int64_t Kp = ceil_div(g.K, 64) * 64;
+    return static_cast<size_t>(std::max(g.M, g.N)) * 3 * Kp * 2 <= kPiecesMaxBytes;
+}
+
+// The automatic choice for fp32: the pieces cost two extra kernels and six times the MMA work, which pays once the
+// problem has about 2^28 multiply-adds (measured: 512^3 is still faster on the CUDA cores, 1024^3 and the paper's
+// 6 x 196 x 256 x 2305 batch are not; the 256^3 configuration is launch-bound either way).
+bool prefer_f32_pieces(const GemmProblem& g, int64_t batch) {
+    if (!gemm_f32_pieces_fit(g) || g.M < 64 || g.N < 64 || g.K < 64) return false;
+    return static_cast<double>(batch) * g.M * g.N * g.K >= 268435456.0;
+}
+
+int run_gemm_f32_pieces(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
+                        cudaStream_t st, const BatchArgs& ba, const tdx_config* user_cfg) {
+    if (!gemm_f32_pieces_fit(g)) return fail(TDX_ERR_UNSUPPORTED, "problem too large for the fp32 tensor-core path");
+    const int64_t Kp = ceil_div(g.K, 64) * 64;
+    const size_t a_one = static_cast<size_t>(g.M) * 3 * Kp * 2, b_one = static_cast<size_t>(g.N) * 3 * Kp * 2;
+    // all batches at once when the pieces fit the budget, else one batch at a time; a shared operand (stride 0) once
+    const bool a_shared = ba.batch > 1 && ba.stride_a == 0, b_shared = ba.batch > 1 && ba.stride_b == 0;
+    int64_t chunk = ba.batch;
+    while (chunk > 1 && (a_one * (a_shared ? 1 : chunk) > kPiecesMaxBytes || b_one * (b_shared ? 1 : chunk) > kPiecesMaxBytes))
+        chunk = (chunk + 1) / 2;
+    if (chunk > 65535) chunk = 65535;
+    void *pa, *pb;
+    int rc;
+    if ((rc = ensure_pieces(ctx, 0, a_one * (a_shared ? 1 : chunk), &pa))) return rc;
+    if ((rc = ensure_pieces(ctx, 1, b_one * (b_shared ? 1 : chunk), &pb))) return rc;
+    // the tensor-core problem: K-major A'' (M x 3Kp) and B'' (N x 3Kp), six piece pairs of Kp each
+    GemmProblem gg{g.M, g.N, 6 * Kp, 0, 1, TDX_BF16};
+    tdx_config want;
+    std::memset(&want, 0, sizeof want);
+    if (user_cfg) want = *user_cfg;
+    want.kernel = TDX_KERNEL_UMMA;
+    want.store_mode = 1;
+    want.cta_pair = 1;          // split_k: the caller's, else chosen like for any GEMM with few tiles and a long reduction
+    tdx_config cfg;
+    rc = resolve_gemm_config(gg, &want, ctx->sm_count, ctx->smem_optin, &cfg);
+    if (rc) return rc;
+    long long sa_i, sa_k, sb_k, sb_j;
+    gemm_strides(g, &sa_i, &sa_k, &sb_k, &sb_j);
+    PieceInfo pi;
+    pi.seg_kb = static_cast<int>(Kp / 64);
+    pi.cols = 3 * Kp;
+    const float* a = static_cast<const float*>(A);
+    const float* b = static_cast<const float*>(B);
+    float* c = static_cast<float*>(C);
+    auto split = [&](const float* src, int rows, long long s_row, long long s_k, long long bstride, int64_t nb, void* dst) -> int {
+        dim3 grid(static_cast<unsigned>(ceil_div(Kp, 32)), static_cast<unsigned>(ceil_div(rows, 32)), static_cast<unsigned>(nb));
+        if (grid.y > 65535) return fail(TDX_ERR_UNSUPPORTED, "operand too tall for the piece kernel");
+        tdx::split_f32_bf16x3_kernel<<<grid, 256, 0, st>>>(rows, static_cast<int>(g.K), static_cast<int>(Kp), s_row, s_k, bstride,
+                                                           src, static_cast<__nv_bfloat16*>(dst));
+        TDX_CUDA(cudaGetLastError());
+        g_launches.fetch_add(1);
+        return TDX_OK;
+    };
+    for (int64_t b0 = 0; b0 < ba.batch; b0 += chunk) {
+        const int64_t nb = std::min(chunk, ba.batch - b0);
+        if (!a_shared || b0 == 0)
+            if ((rc = split(a + (a_shared ? 0 : b0 * ba.stride_a), static_cast<int>(g.M), sa_i, sa_k, ba.stride_a, a_shared ? 1 : nb, pa))) return rc;
+        if (!b_shared || b0 == 0)     // B'' rows are the columns j of op(B): element (j, k) at B[k * sb_k + j * sb_j]
+            if ((rc = split(b + (b_shared ? 0 : b0 * ba.stride_b), static_cast<int>(g.N), sb_j, sb_k, ba.stride_b, b_shared ? 1 : nb, pb))) return rc;
+        for (int64_t i = 0; i < nb; ++i) {
+            const char* ai = static_cast<const char*>(pa) + (a_shared ? 0 : i * a_one);
+            const char* bi = static_cast<const char*>(pb) + (b_shared ? 0 : i * b_one);
+            rc = run_gemm_umma(ctx, gg, alpha, ai, bi, c + (b0 + i) * ba.stride_c, cfg, nullptr, 0, true, st, ba.beta, &pi);
+            if (rc) return rc;
+        }
+    }
     return TDX_OK;
 }
 

@@ -71,6 +71,8 @@ struct DeviceCtx {
     size_t ws_bytes = 0;
     void* staging[4] = {nullptr, nullptr, nullptr, nullptr};  // host-variant device copies
     size_t staging_bytes[4] = {0, 0, 0, 0};
+    void* pieces[2] = {nullptr, nullptr};                     // bf16 pieces of fp32 operands (A, B)
+    size_t pieces_bytes[2] = {0, 0};
 };
 
 std::mutex g_mu;

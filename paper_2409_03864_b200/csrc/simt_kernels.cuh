@@ -439,6 +439,82 @@ __global__ void copy_pad_ring_kernel(long long total, long long C, long long Hp,
     }
 }
 
+// The same reduction with an fp32 result: out = alpha * sum_s partial[s] + beta * out (the fp32 GEMM from bf16 pieces).
+__global__ void splitk_reduce_f32_kernel(long long MN, int split, const float* __restrict__ partial, float alpha, float beta,
+                                         float* out, int vec4) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (vec4) {
+        const long long groups = MN / 4;
+        for (long long g = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; g < groups;
+             g += static_cast<long long>(gridDim.x) * blockDim.x) {
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int s = 0; s < split; ++s) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(partial + s * MN) + g);
+                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            }
+            float4 r = make_float4(alpha * acc.x, alpha * acc.y, alpha * acc.z, alpha * acc.w);
+            float4* o = reinterpret_cast<float4*>(out) + g;
+            if (beta != 0.0f) {
+                const float4 old = *o;
+                r.x = fmaf(beta, old.x, r.x); r.y = fmaf(beta, old.y, r.y); r.z = fmaf(beta, old.z, r.z); r.w = fmaf(beta, old.w, r.w);
+            }
+            *o = r;
+        }
+    } else {
+        for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < MN;
+             e += static_cast<long long>(gridDim.x) * blockDim.x) {
+            float acc = 0.0f;
+            for (int s = 0; s < split; ++s) acc += __ldg(partial + s * MN + e);
+            const float v = alpha * acc;
+            out[e] = beta != 0.0f ? fmaf(beta, out[e], v) : v;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// fp32 -> three bf16 pieces, for the fp32 GEMM on the tensor cores: x = hi + mid + lo with hi = bf16(x),
+// mid = bf16(x - hi), lo = bf16(x - hi - mid); both differences are exact in fp32 and the three pieces carry all
+// 24 significand bits.  Source: `rows` x K logical matrix, element (i, k) at src[b * batch_stride + i * s_row + k * s_k]
+// (either stride may be 1).  Destination, per batch: rows x (3 * Kp) bf16, row-major, piece p of element (i, k) at
+// column p * Kp + k; columns K..Kp-1 of every piece are zero (Kp is K rounded up to the K block of the MMA pipeline).
+// 32 x 32 tiles through shared memory, so that reads and writes are both coalesced whichever stride is 1.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+split_f32_bf16x3_kernel(int rows, int K, int Kp, long long s_row, long long s_k, long long batch_stride,
+                        const float* __restrict__ src, __nv_bfloat16* __restrict__ dst) {
+    __shared__ float tile[32][33];
+    const int k0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    const float* s = src + blockIdx.z * batch_stride;
+    __nv_bfloat16* d = dst + static_cast<long long>(blockIdx.z) * rows * 3 * Kp;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;        // 32 x 8 threads
+    if (s_k == 1) {
+        for (int j = ty; j < 32; j += 8) {
+            const int r = r0 + j, k = k0 + tx;
+            tile[j][tx] = (r < rows && k < K) ? __ldg(s + r * s_row + k) : 0.0f;
+        }
+    } else {       // rows are the contiguous dimension of the source: read along them, transpose in shared memory
+        for (int j = ty; j < 32; j += 8) {
+            const int k = k0 + j, r = r0 + tx;
+            tile[tx][j] = (r < rows && k < K) ? __ldg(s + r * s_row + k * s_k) : 0.0f;
+        }
+    }
+    __syncthreads();
+    for (int j = ty; j < 32; j += 8) {
+        const int r = r0 + j, k = k0 + tx;
+        if (r < rows && k < Kp) {
+            const float x = tile[j][tx];
+            const __nv_bfloat16 hi = __float2bfloat16_rn(x);
+            const float r1 = x - __bfloat162float(hi);
+            const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+            const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+            __nv_bfloat16* o = d + static_cast<long long>(r) * 3 * Kp + k;
+            o[0] = hi;
+            o[Kp] = mid;
+            o[2 * Kp] = lo;
+        }
+    }
+}
+
 // Deterministic pseudo-random fill used only by the tuner's scratch operands.
 __global__ void fill_pattern_bf16_kernel(__nv_bfloat16* p, long long n, uint32_t seed) {
     for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < n;

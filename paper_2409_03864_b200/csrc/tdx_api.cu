@@ -54,7 +54,9 @@ int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_cou
             tdx_config cached;
             if (tune_lookup(gemm_key(g.M, g.N, g.K, g.transA, g.transB, g.dtype), &cached)) { c = cached; from_cache = true; }
         }
-        if (!from_cache) c.kernel = g.dtype == TDX_F32 ? TDX_KERNEL_SIMT : (layout_ok ? TDX_KERNEL_UMMA : TDX_KERNEL_GENERIC);
+        if (!from_cache)
+            c.kernel = g.dtype == TDX_F32 ? (prefer_f32_pieces(g, 1) ? TDX_KERNEL_UMMA : TDX_KERNEL_SIMT)
+                                          : (layout_ok ? TDX_KERNEL_UMMA : TDX_KERNEL_GENERIC);
     }
     if (c.kernel == TDX_KERNEL_SIMT) {
         if (g.dtype != TDX_F32) return fail(TDX_ERR_CONFIG, "the tiled SIMT kernel is fp32 only");
@@ -63,6 +65,14 @@ int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_cou
     }
     if (c.kernel == TDX_KERNEL_GENERIC) { *out = c; return TDX_OK; }
     // tensor-core path
+    if (g.dtype == TDX_F32) {
+        // fp32 on the tensor cores = bf16 pieces; the tile fields are resolved against the piece problem at launch
+        if (!gemm_f32_pieces_fit(g)) return fail(TDX_ERR_CONFIG, "problem too large for the fp32 tensor-core path");
+        if (c.cta_pair == 2 || c.store_mode == 2)
+            return fail(TDX_ERR_CONFIG, "the fp32 tensor-core path takes no CTA pairs or staged stores");
+        *out = c;
+        return TDX_OK;
+    }
     if (g.dtype != TDX_BF16) return fail(TDX_ERR_CONFIG, "the tensor-core kernel is bf16 only");
     if (!layout_ok) return fail(TDX_ERR_ALIGNMENT, "tensor-core path needs 16-byte aligned row pitches (contiguous dims %% 8 == 0)");
     const int64_t num_kb = ceil_div(g.K, 64);
@@ -205,6 +215,7 @@ int gemm_dispatch(int64_t M, int64_t N, int64_t K, int transA, int transB, float
         case TDX_KERNEL_SIMT: return run_gemm_simt_f32(ctx, g, alpha, A, B, C, st);
         case TDX_KERNEL_GENERIC: return run_gemm_generic(ctx, g, alpha, A, B, C, st);
         default:
+            if (dtype == TDX_F32) return run_gemm_f32_pieces(ctx, g, alpha, A, B, C, st, BatchArgs(), cfg);
             if (reinterpret_cast<uintptr_t>(A) % 16 || reinterpret_cast<uintptr_t>(B) % 16) {
                 if (cfg && cfg->kernel == TDX_KERNEL_UMMA)
                     return fail(TDX_ERR_ALIGNMENT, "tensor-core path needs 16-byte aligned A and B");
@@ -503,7 +514,10 @@ int tdx_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int transA,
         // empty reduction: C = beta * C.  The generic kernel does exactly that (its k loop is empty).
         return run_gemm_generic(ctx, g, alpha, C, C, C, st, ba);
     }
-    if (dtype == TDX_F32) return run_gemm_simt_f32(ctx, g, alpha, A, B, C, st, ba);
+    if (dtype == TDX_F32) {
+        if (prefer_f32_pieces(g, batch)) return run_gemm_f32_pieces(ctx, g, alpha, A, B, C, st, ba, nullptr);
+        return run_gemm_simt_f32(ctx, g, alpha, A, B, C, st, ba);
+    }
     // bf16: the tensor-core kernel, one launch per batch, when every batch's operands meet its layout rules
     const bool aligned = gemm_umma_layout_ok(g) && reinterpret_cast<uintptr_t>(A) % 16 == 0 &&
                          reinterpret_cast<uintptr_t>(B) % 16 == 0 && (strideA % 8 == 0) && (strideB % 8 == 0);

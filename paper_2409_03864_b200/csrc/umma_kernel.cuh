@@ -79,6 +79,12 @@ struct UmmaParams {
     // them to the CTAs (CTA pairs for the pair kernel): entry [round * workers + worker] = (row block, first
     // column, width, 0); width 0 ends a worker's list.  This is how a tile count that does not fill the last
     // wave of CTAs is evened out.
+    // fp32 GEMM from bf16 pieces (seg_kb > 0): the operands hold three pieces side by side (seg_kb K blocks each) and the
+    // reduction walks six piece pairs: K block kb reads piece a_seg[kb / seg_kb] of A and b_seg[kb / seg_kb] of B.
+    // The result is written as fp32 to Cf (direct stores).
+    int seg_kb;
+    int a_seg[6], b_seg[6];
+    float* Cf;
     const int4* tiles;
     int rounds;
     int b_box;                // rows of one B copy (K-major B); bn when there is no table
@@ -391,6 +397,31 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                     for (int j = 0; j < 32; ++j)
                         if (col0 + j < p.N) dst[j] = __uint_as_float(r[j]);
                 }
+            } else if (!kConv && p.Cf != nullptr) {
+                // fp32 output (the fp32 GEMM from bf16 pieces): out = alpha * acc + beta * (what Cf held)
+                float* dst = p.Cf + grow * p.ldc + col0;
+                if (p.vec_store) {
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) {
+                        if (col0 + g * 4 < p.N) {
+                            float4 v = make_float4(p.alpha * __uint_as_float(r[g * 4]), p.alpha * __uint_as_float(r[g * 4 + 1]),
+                                                   p.alpha * __uint_as_float(r[g * 4 + 2]), p.alpha * __uint_as_float(r[g * 4 + 3]));
+                            if (p.beta != 0.0f) {
+                                const float4 o = *reinterpret_cast<const float4*>(dst + g * 4);
+                                v.x = fmaf(p.beta, o.x, v.x); v.y = fmaf(p.beta, o.y, v.y);
+                                v.z = fmaf(p.beta, o.z, v.z); v.w = fmaf(p.beta, o.w, v.w);
+                            }
+                            *reinterpret_cast<float4*>(dst + g * 4) = v;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (col0 + j < p.N) {
+                            const float x = p.alpha * __uint_as_float(r[j]);
+                            dst[j] = p.beta != 0.0f ? fmaf(p.beta, dst[j], x) : x;
+                        }
+                }
             } else {
                 float v[32];
 #pragma unroll
@@ -531,20 +562,26 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                         }
                         ptx::tma_load_3d(b_dst, &tmB, bar, cc * kBK, tap, t.n0);
                     } else {
+                        int ka = kb, kbb = kb;                  // K block of A and of B
+                        if (p.seg_kb > 0) {
+                            const int sg = kb / p.seg_kb, r = kb - sg * p.seg_kb;
+                            ka = p.a_seg[sg] * p.seg_kb + r;
+                            kbb = p.b_seg[sg] * p.seg_kb + r;
+                        }
                         if (p.a_mn_major) {
                             for (int i = 0; i < 2 * mh; ++i)
-                                ptx::tma_load_2d(a_dst + i * 8192, &tmA, bar, t.m_blk * p.bm + i * 64, kb * kBK);
+                                ptx::tma_load_2d(a_dst + i * 8192, &tmA, bar, t.m_blk * p.bm + i * 64, ka * kBK);
                         } else {
                             for (int h = 0; h < mh; ++h)
-                                ptx::tma_load_2d(a_dst + h * kHalfABytes, &tmA, bar, kb * kBK,
+                                ptx::tma_load_2d(a_dst + h * kHalfABytes, &tmA, bar, ka * kBK,
                                                  t.m_blk * p.bm + h * kHalfM);
                         }
                         if (p.b_mn_major) {
                             for (int i = 0; i < t.bn / 64; ++i)
-                                ptx::tma_load_2d(b_dst + i * 8192, &tmB, bar, t.n0 + i * 64, kb * kBK);
+                                ptx::tma_load_2d(b_dst + i * 8192, &tmB, bar, t.n0 + i * 64, kbb * kBK);
                         } else {
                             for (int r0 = 0; r0 < t.bn; r0 += p.b_box)
-                                ptx::tma_load_2d(b_dst + r0 * 128, &tmB, bar, kb * kBK, t.n0 + r0);
+                                ptx::tma_load_2d(b_dst + r0 * 128, &tmB, bar, kbb * kBK, t.n0 + r0);
                         }
                     }
                     if (++stage == p.stages) {

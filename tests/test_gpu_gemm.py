@@ -375,3 +375,57 @@ def test_sweep_shape_8192_cubed():
     err = gemm_error(M, N, K, 0, 0, 1.0, "bf16", A, B, C, rows=rows)
     assert err < TOL["bf16"] and err < TIGHT["bf16"], err
     assert tdx.tdx_check_device_status() == 0
+
+
+# ------------------------------------------------------------------ fp32 on the tensor cores (three bf16 pieces per operand)
+
+@pytest.mark.parametrize("transA,transB", [(0, 0), (0, 1), (1, 0), (1, 1)])
+@pytest.mark.parametrize("shape", [(200, 136, 300), (520, 264, 70), (64, 64, 64)])
+def test_fp32_gemm_from_bf16_pieces_all_layouts(shape, transA, transB):
+    # explicit request (kernel = UMMA with fp32 data): ragged M, N and K; K not a multiple of the 64-deep K block
+    M, N, K = shape
+    A = si.uniform(68, 0, (K, M) if transA else (M, K), "f32")
+    B = si.uniform(68, 1, (N, K) if transB else (K, N), "f32")
+    st, C, ok = run_gemm(M, N, K, transA, transB, -1.5, "f32", A, B, cfg=umma())
+    assert st == 0 and ok, tdx.tdx_last_error()
+    err = gemm_error(M, N, K, transA, transB, -1.5, "f32", A, B, C)
+    assert err < TOL["f32"] and err < TIGHT["f32"], err
+
+
+def test_fp32_gemm_from_bf16_pieces_keeps_all_24_bits():
+    # operands whose low significand bits matter: x = 1 + u * 2^-20 -- a two-piece split would lose them.  Compare with the
+    # CUDA-core kernel's error on the same problem: the tensor-core path must be in the same class.
+    M, N, K = 256, 192, 512
+    A = (1.0 + si.uniform(69, 0, (M, K), "f32").astype(np.float64) * 2.0 ** -20).astype(np.float32)
+    B = (1.0 + si.uniform(69, 1, (K, N), "f32").astype(np.float64) * 2.0 ** -20).astype(np.float32)
+    st, C, ok = run_gemm(M, N, K, 0, 0, 1.0, "f32", A, B, cfg=umma())
+    assert st == 0 and ok, tdx.tdx_last_error()
+    ref = oracle.gemm(M, N, K, 0, 0, 1.0, "f32", A, B)
+    rel = np.abs(C.astype(np.float64) - ref).max() / np.abs(ref).max()
+    assert rel < 4e-7, rel                       # a few fp32 ulps of the result; two pieces would give ~1e-5
+    st, Cs, ok = run_gemm(M, N, K, 0, 0, 1.0, "f32", A, B, cfg=tdx.tdx_config(kernel=tdx.TDX_KERNEL_SIMT))
+    assert st == 0 and ok
+    rel_simt = np.abs(Cs.astype(np.float64) - ref).max() / np.abs(ref).max()
+    assert rel < 8 * max(rel_simt, 6e-8), (rel, rel_simt)
+
+
+def test_fp32_gemm_large_takes_the_tensor_cores_automatically():
+    M = N = K = 1024
+    A, B = si.gemm_f32_uniform(M, N, K, seed=70)
+    st, c = tdx.tdx_default_gemm_config(M, N, K, 0, 0, tdx.TDX_F32)
+    assert st == 0 and c.kernel == tdx.TDX_KERNEL_UMMA
+    st, c1 = tdx.tdx_default_gemm_config(256, 256, 256, 0, 0, tdx.TDX_F32)
+    assert st == 0 and c1.kernel == tdx.TDX_KERNEL_SIMT      # the small configuration stays on the CUDA cores
+    n0 = tdx.tdx_kernel_launch_count()
+    st, C, ok = run_gemm(M, N, K, 0, 0, 1.0, "f32", A, B)
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert tdx.tdx_kernel_launch_count() - n0 == 3            # two piece kernels and the GEMM
+    rows = structured_rows(M, max_blocks=4)
+    err = gemm_error(M, N, K, 0, 0, 1.0, "f32", A, B, C, rows=rows)
+    assert err < TIGHT["f32"], err
+    # integer operands: exact
+    Ai = si.small_integers(71, 0, (M, K), "f32", -8, 8)
+    Bi = si.small_integers(71, 1, (K, N), "f32", -8, 8)
+    st, Ci, ok = run_gemm(M, N, K, 0, 0, 1.0, "f32", Ai, Bi)
+    assert st == 0 and ok
+    assert np.array_equal(Ci[rows].astype(np.float64), oracle.gemm(M, N, K, 0, 0, 1.0, "f32", Ai, Bi, rows=rows))
