@@ -235,6 +235,20 @@ int tdx_enum_gemm_configs(int64_t M, int64_t N, int64_t K, int transA, int trans
 int tdx_enum_conv2d_configs(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
                             int pad, int stride, int dtype, tdx_config* out, int cap, int* n);
 
+/*
+ * Guided search: the candidates of tdx_tune_gemm are ranked by a host-side cost model (MMA time by tile width, L2
+ * ingest, epilogue overlap, wave count or fitted plan, split-K traffic, HBM floor) and only the `budget` best-ranked
+ * ones, plus the heuristic default, are timed on the device -- the model-guided counterpart of Case Study 5's
+ * search under constraints.  n_candidates (may be NULL) receives the size of the full search space.  bf16 GEMM;
+ * other problems are searched exhaustively.  tdx_model_gemm_us evaluates the model for one configuration on
+ * `ctas` SMs (host only).
+ */
+int tdx_tune_gemm_guided(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, int iters, int budget,
+                         tdx_config* best, float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried,
+                         int* n_candidates, void* stream);
+int tdx_model_gemm_us(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const tdx_config* cfg, int ctas,
+                      double* us);
+
 /* The configuration the automatic choice would use right now (tuning cache, else heuristic). */
 int tdx_default_gemm_config(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, tdx_config* out);
 int tdx_default_conv2d_config(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,

@@ -80,6 +80,8 @@ def lib() -> ctypes.CDLL:
         L.tdx_gemm_host.argtypes = gemm_args
         L.tdx_conv2d_bias_relu_host.argtypes = conv_args
         L.tdx_tune_gemm.argtypes = [i64, i64, i64, ci, ci, ci, ci, cfgp, fp, cfgp, fp, ci, ip, vp]
+        L.tdx_tune_gemm_guided.argtypes = [i64, i64, i64, ci, ci, ci, ci, ci, cfgp, fp, cfgp, fp, ci, ip, ip, vp]
+        L.tdx_model_gemm_us.argtypes = [i64, i64, i64, ci, ci, ci, cfgp, ci, ctypes.POINTER(ctypes.c_double)]
         L.tdx_tune_conv2d.argtypes = [i64] * 7 + [ci, ci, ci, ci, cfgp, fp, cfgp, fp, ci, ip, vp]
         L.tdx_enum_gemm_configs.argtypes = [i64, i64, i64, ci, ci, ci, cfgp, ci, ip]
         L.tdx_enum_conv2d_configs.argtypes = [i64] * 7 + [ci, ci, ci, cfgp, ci, ip]
@@ -113,7 +115,7 @@ def lib() -> ctypes.CDLL:
 # every symbol include/tdx.h declares
 EXPORTS = (
     "tdx_gemm", "tdx_add_zero_pad", "tdx_add_zero_pad_host", "tdx_gemm_batched", "tdx_gemm_batched_host", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_add_relu", "tdx_conv2d_bias_relu_ex",
-    "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
+    "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_gemm_guided", "tdx_model_gemm_us", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
     "tdx_enum_conv2d_configs", "tdx_default_gemm_config", "tdx_default_conv2d_config", "tdx_tune_save",
     "tdx_tune_load", "tdx_tune_clear", "tdx_gemm_tile_plan", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
     "tdx_version",
@@ -247,6 +249,22 @@ def tdx_tune_gemm(M, N, K, transA, transB, dtype, iters=20, stream=None, cap=512
     L = lib()
     return _tune(lambda b, bu, t, tu, c, n: L.tdx_tune_gemm(M, N, K, transA, transB, dtype, iters, b, bu, t, tu, c, n,
                                                             _stream(stream)), cap)
+
+
+def tdx_tune_gemm_guided(M, N, K, transA, transB, dtype, budget, iters=20, stream=None, cap=512):
+    """Returns (status, best tdx_config, best microseconds, [(config dict, microseconds), ...], size of the full space)."""
+    L = lib()
+    n_cand = ctypes.c_int(0)
+    st, best, us, tried = _tune(lambda b, bu, t, tu, c, n: L.tdx_tune_gemm_guided(
+        M, N, K, transA, transB, dtype, iters, budget, b, bu, t, tu, c, n, ctypes.byref(n_cand), _stream(stream)), cap)
+    return st, best, us, tried, int(n_cand.value)
+
+
+def tdx_model_gemm_us(M, N, K, transA, transB, dtype, cfg, ctas=148):
+    """Returns (status, predicted microseconds) of the cost model that ranks the guided search (host only)."""
+    us = ctypes.c_double(0.0)
+    st = lib().tdx_model_gemm_us(M, N, K, transA, transB, dtype, _cfg(cfg), ctas, ctypes.byref(us))
+    return st, float(us.value)
 
 
 def tdx_tune_conv2d(N, H, W, Cin, Cout, R, S, pad, stride, dtype, iters=20, stream=None, cap=512):

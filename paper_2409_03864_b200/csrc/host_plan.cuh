@@ -169,4 +169,43 @@ int get_tile_plan(DeviceCtx* ctx, int64_t M, int64_t N, int64_t num_kb, int bm, 
     return TDX_OK;
 }
 
+// ------------------------------------------------------------------ cost model of a GEMM configuration
+// Predicted device time (microseconds) of a fully specified tensor-core configuration; it ranks the candidates of
+// the guided search, so only its ordering matters.  Pieces, all from measurements on B200: an MMA of N columns takes
+// max(N / 2, 60) cycles; one SM ingests about 70 bytes per cycle from L2; start-up to the first MMA 5500 cycles; the
+// staged epilogue about 600 cycles per 32 x 32 block and warp (16 warps), the direct one twice that; an epilogue
+// overlaps the next main loop only when TMEM holds more accumulator slots than a tile uses; split-K adds the fp32
+// partial traffic and a reduction launch; nothing beats streaming the operands once from HBM.
+double model_gemm_us(const GemmProblem& g, const tdx_config& c, int sm_count) {
+    const double clk_mhz = 1600.0;
+    const int64_t num_kb = ceil_div(g.K, 64);
+    const bool pair = c.cta_pair == 2;
+    const int workers = pair ? sm_count / 2 : sm_count;
+    const int tm = pair ? 256 : c.tile_m, bn = c.tile_n, split = std::max(1, c.split_k);
+    const int64_t kb = ceil_div(num_kb, split);
+    const int64_t tiles = ceil_div(g.M, tm) * ceil_div(g.N, bn) * split;
+    const int halves = pair ? 1 : tm / 128;                                 // 128-row halves one CTA computes
+    const double mma = 4.0 * halves * std::max(bn / 2.0, 60.0);
+    const double l2 = (pair ? (128.0 + bn / 2.0) : (tm + static_cast<double>(bn))) * 128.0 / 70.0;
+    const double main_loop = static_cast<double>(kb) * std::max(mma, l2);
+    const double blocks = halves * 4.0 * (bn / 32.0);                       // 32 x 32 output blocks per CTA and tile
+    double epi = (c.store_mode == 2 ? 600.0 * std::ceil(blocks / 16.0) : 1200.0 * std::ceil(blocks / (4.0 * halves)));
+    if (split > 1) epi *= 1.5;                                              // fp32 partials: twice the bytes
+    const int slots = pair ? (2 * bn <= 256 ? 4 : 2) : tmem_slots_for(tm, bn);
+    const bool overlapped = slots > halves;
+    double rounds = std::ceil(static_cast<double>(tiles) / workers);
+    double cycles;
+    TilePlan plan;
+    if (c.fit == 2 && split == 1 && !pair && plan_fitted_tiles(g.M, g.N, num_kb, tm, bn, c.raster, sm_count, 0.0, &plan)) {
+        cycles = 5500.0 + plan.makespan;                                    // the plan's own figure includes the epilogues
+    } else {
+        const double per_tile = overlapped ? std::max(main_loop, epi) : main_loop + epi;
+        cycles = 5500.0 + rounds * per_tile + (overlapped ? epi : 0.0) + (pair ? 4000.0 : 0.0);
+    }
+    double us = cycles / clk_mhz;
+    if (split > 1) us += 3.0 + (static_cast<double>(split) * g.M * g.N * 4.0 * 2.0 + g.M * g.N * 2.0) / 4.0e6;
+    const double hbm_us = (static_cast<double>(g.M) * g.K + static_cast<double>(g.K) * g.N + static_cast<double>(g.M) * g.N) * 2.0 / 5.0e6;
+    return std::max(us, hbm_us);
+}
+
 }  // namespace

@@ -4,6 +4,8 @@
 // tile plans), host_launch.cuh (launches).
 #include "host_launch.cuh"
 
+#include <tuple>
+
 namespace {
 // ------------------------------------------------------------------ validation
 int validate_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const void* A, const void* B,
@@ -785,8 +787,11 @@ int tdx_default_conv2d_config(int64_t N, int64_t H, int64_t W, int64_t Cin, int6
     return resolve_conv_config(cp, nullptr, sm_count, smem_limit, out);
 }
 
-int tdx_tune_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, int iters, tdx_config* best,
-                  float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried, void* stream) {
+// budget <= 0: every statically feasible candidate is timed; budget > 0: the candidates are ranked by the cost model and
+// only the `budget` best-ranked ones (plus the heuristic default) are timed
+static int tune_gemm_impl(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, int iters, int budget,
+                          tdx_config* best, float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried,
+                          int* n_candidates, void* stream) {
     int rc = validate_gemm(M, N, K, transA, transB, dtype, nullptr, nullptr, nullptr, false);
     if (rc) return rc;
     if (best == nullptr || iters < 1 || cap < 0) return fail(TDX_ERR_INVALID_ARG, "best is NULL, iters < 1 or cap < 0");
@@ -797,6 +802,34 @@ int tdx_tune_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, int d
     GemmProblem g{M, N, K, transA, transB, dtype};
     std::vector<tdx_config> cands;
     enum_gemm(g, ctx->sm_count, ctx->smem_optin, &cands);
+    if (n_candidates) *n_candidates = static_cast<int>(cands.size());
+    if (budget > 0 && static_cast<int>(cands.size()) > budget && dtype == TDX_BF16 && cands[0].kernel == TDX_KERNEL_UMMA) {
+        std::vector<std::pair<double, size_t>> ranked;
+        for (size_t i = 0; i < cands.size(); ++i) ranked.push_back({model_gemm_us(g, cands[i], ctx->sm_count), i});
+        std::stable_sort(ranked.begin(), ranked.end());
+        // The model knows tile shape, split, store mode, pairs and fitting, not pipeline depth, raster or K stagger:
+        // half of the budget goes to the best-ranked DISTINCT shapes (first variant of each), the rest to further
+        // variants in rank order.
+        auto shape_of = [](const tdx_config& c) {
+            return std::make_tuple(c.tile_m, c.tile_n, c.split_k, c.store_mode, c.cta_pair, c.fit);
+        };
+        std::vector<char> taken(cands.size(), 0);
+        std::vector<tdx_config> keep;
+        std::vector<decltype(shape_of(cands[0]))> seen;
+        for (size_t r = 0; r < ranked.size() && static_cast<int>(keep.size()) < (budget + 1) / 2; ++r) {
+            const tdx_config& c = cands[ranked[r].second];
+            if (std::find(seen.begin(), seen.end(), shape_of(c)) != seen.end()) continue;
+            seen.push_back(shape_of(c));
+            keep.push_back(c);
+            taken[ranked[r].second] = 1;
+        }
+        for (size_t r = 0; r < ranked.size() && static_cast<int>(keep.size()) < budget; ++r)
+            if (!taken[ranked[r].second]) keep.push_back(cands[ranked[r].second]);
+        tdx_config d;
+        if (resolve_gemm_config(g, nullptr, ctx->sm_count, ctx->smem_optin, &d) == TDX_OK && d.kernel == TDX_KERNEL_UMMA)
+            keep.push_back(d);                                  // what an untuned call would use: never do worse than that
+        cands.swap(keep);
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t el = dtype == TDX_F32 ? 4 : 2;
     ScratchGuard guard;
@@ -820,6 +853,34 @@ int tdx_tune_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, int d
         std::lock_guard<std::mutex> lk(g_mu);
         g_tune[gemm_key(M, N, K, transA, transB, dtype)] = TuneEntry{*best, best_us ? *best_us : 0.0f};
     }
+    return TDX_OK;
+}
+
+int tdx_tune_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, int iters, tdx_config* best,
+                  float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried, void* stream) {
+    return tune_gemm_impl(M, N, K, transA, transB, dtype, iters, 0, best, best_us, tried, tried_us, cap, n_tried, nullptr, stream);
+}
+
+int tdx_tune_gemm_guided(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, int iters, int budget,
+                         tdx_config* best, float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried,
+                         int* n_candidates, void* stream) {
+    if (budget < 1) return fail(TDX_ERR_INVALID_ARG, "budget must be >= 1");
+    return tune_gemm_impl(M, N, K, transA, transB, dtype, iters, budget, best, best_us, tried, tried_us, cap, n_tried,
+                          n_candidates, stream);
+}
+
+int tdx_model_gemm_us(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const tdx_config* cfg, int ctas,
+                      double* us) {
+    int rc = validate_gemm(M, N, K, transA, transB, dtype, nullptr, nullptr, nullptr, false);
+    if (rc) return rc;
+    if (cfg == nullptr || us == nullptr || ctas < 2 || M == 0 || N == 0 || K == 0)
+        return fail(TDX_ERR_INVALID_ARG, "cfg or us is NULL, ctas < 2, or empty problem");
+    GemmProblem g{M, N, K, transA, transB, dtype};
+    tdx_config c;
+    rc = resolve_gemm_config(g, cfg, ctas, kSmemLimitDefault, &c);
+    if (rc) return rc;
+    if (c.kernel != TDX_KERNEL_UMMA || dtype != TDX_BF16) return fail(TDX_ERR_UNSUPPORTED, "the cost model covers the bf16 tensor-core kernel");
+    *us = model_gemm_us(g, c, ctas);
     return TDX_OK;
 }
 

@@ -43,10 +43,12 @@ def flops(spec):
     return 2.0 * N * P * Q * Cout * R * S * Cin
 
 
-def tune_one(spec, iters):
+def tune_one(spec, iters, budget=0):
     f = spec.split(":")
     v = [int(x) for x in f[1:]]
     if f[0] == "gemm":
+        if budget > 0:      # model-guided: time only the candidates the cost model ranks best
+            return tdx.tdx_tune_gemm_guided(*v, tdx.TDX_BF16, budget, iters=iters, cap=8192)[:4]
         return tdx.tdx_tune_gemm(*v, tdx.TDX_BF16, iters=iters, cap=8192)
     if f[0] == "conv":
         return tdx.tdx_tune_conv2d(*v, tdx.TDX_BF16, iters=iters, cap=8192)
@@ -67,12 +69,14 @@ def main(argv=None):
     ap.add_argument("workloads", nargs="*")
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--top", type=int, default=5)
+    ap.add_argument("--budget", type=int, default=0,
+                    help="GEMM: time only this many candidates, chosen by the cost model (0 = all)")
     ap.add_argument("--out", default=None, help="save the tuning cache (JSON) here")
     ap.add_argument("--json", default=None, help="also write every candidate's time to this file")
     args = ap.parse_args(argv)
     report = {}
     for spec in expand(args.workloads):
-        st, best, best_us, tried = tune_one(spec, args.iters)
+        st, best, best_us, tried = tune_one(spec, args.iters, args.budget)
         if st != tdx.TDX_OK:
             print(f"{spec}: status {st}: {tdx.tdx_last_error()}")
             continue

@@ -1,0 +1,46 @@
+"""The model-guided tile-configuration search against the exhaustive one (GPU), and the cost model's ordering (host)."""
+import pytest
+
+import paper_2409_03864_b200 as tdx
+
+
+def umma(**kw):
+    return tdx.tdx_config(kernel=tdx.TDX_KERNEL_UMMA, **kw)
+
+
+def test_cost_model_orders_known_cases():
+    # host only: orderings that the measurements behind the model established
+    def us(M, N, K, tB, **kw):
+        st, v = tdx.tdx_model_gemm_us(M, N, K, 0, tB, tdx.TDX_BF16, umma(**kw))
+        assert st == tdx.TDX_OK, tdx.tdx_last_error()
+        return v
+    big = (4096, 4096, 4096, 1)
+    assert us(*big, tile_m=256, tile_n=256, fit=2) < us(*big, tile_m=256, tile_n=256, fit=1)     # the fitted plan fills the last wave
+    assert us(*big, tile_m=256, tile_n=256, fit=1) < us(*big, tile_m=128, tile_n=256, fit=1)     # L2 ingest bounds 128-row tiles
+    assert us(*big, tile_m=128, tile_n=256, fit=1) < us(*big, tile_m=128, tile_n=64)             # narrow MMAs run at half rate
+    skinny = (128, 8192, 8192, 0)
+    assert us(*skinny, tile_m=128, tile_n=128, split_k=2, store_mode=1) < us(*skinny, tile_m=128, tile_n=128, split_k=1)
+    assert us(*skinny, tile_m=128, tile_n=128, split_k=2, store_mode=1) < us(*skinny, tile_m=128, tile_n=128, split_k=16, store_mode=1)
+    # never below the time to stream the operands once
+    assert us(*skinny, tile_m=128, tile_n=128, split_k=2, store_mode=1) >= (128 * 8192 + 8192 * 8192 + 128 * 8192) * 2 / 5.0e6
+    st, _ = tdx.tdx_model_gemm_us(256, 256, 256, 0, 0, tdx.TDX_F32, umma())
+    assert st == tdx.TDX_ERR_UNSUPPORTED
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("shape", [(1024, 1024, 1024, 0), (2048, 2048, 1024, 1), (128, 4096, 4096, 0)])
+def test_guided_search_finds_a_configuration_close_to_the_exhaustive_best(shape):
+    M, N, K, tB = shape
+    budget = 16
+    st, best_all, us_all, tried_all = tdx.tdx_tune_gemm(M, N, K, 0, tB, tdx.TDX_BF16, iters=10, cap=8192)
+    assert st == 0, tdx.tdx_last_error()
+    st, best, us, tried, n_space = tdx.tdx_tune_gemm_guided(M, N, K, 0, tB, tdx.TDX_BF16, budget, iters=10, cap=8192)
+    assert st == 0, tdx.tdx_last_error()
+    assert n_space == len(tried_all) and n_space > 4 * budget         # the model really pruned something
+    assert 1 <= len(tried) <= budget + 1                              # the budget, plus the heuristic default
+    # within 15 % of the exhaustive winner (timing noise between the two searches is a few per cent)
+    assert us <= 1.15 * us_all, (best.as_dict(), us, best_all.as_dict(), us_all)
+    # the winner is stored like the exhaustive one and is what the next call uses
+    st, c = tdx.tdx_default_gemm_config(M, N, K, 0, tB, tdx.TDX_BF16)
+    assert st == 0 and c.as_dict() == best.as_dict()
+    assert tdx.tdx_tune_clear() == 0
