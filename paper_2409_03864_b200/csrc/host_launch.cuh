@@ -8,7 +8,7 @@ namespace {
 int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensorMap& mb, const CUtensorMap& mc,
                 const UmmaParams& p_in, cudaStream_t st, bool halo = false, const CUtensorMap* ma_row = nullptr,
                 const CUtensorMap* mc_row = nullptr, int plan_grid = 0) {
-    const long long items = static_cast<long long>(p_in.tiles_m) * p_in.tiles_n * p_in.split_k;
+    const long long items = static_cast<long long>(p_in.tiles_m) * p_in.tiles_n * p_in.split_k * (p_in.batch > 1 ? p_in.batch : 1);
     UmmaParams p = p_in;
     if (p.b_box == 0) p.b_box = p.bn;
     const int grid = p.tiles != nullptr ? plan_grid : static_cast<int>(std::min<long long>(items, ctx->sm_count));
@@ -82,6 +82,8 @@ int ensure_ws(DeviceCtx* ctx, size_t bytes, void** out) {
 struct PieceInfo {
     int seg_kb = 0;
     int64_t cols = 0;
+    int64_t batch = 1;        // > 1: all batches in one launch (operands dense per batch, C batch_c elements apart)
+    int64_t batch_c = 0;
 };
 
 int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
@@ -123,11 +125,18 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         p.seg_kb = pieces->seg_kb;
         p.Cf = static_cast<float*>(C);
         p.C = nullptr;
-        p.vec_store = (g.N % 4 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+        p.vec_store = (g.N % 4 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0) && (pieces->batch_c % 4 == 0);
+        if (pieces->batch > 1) {
+            if (static_cast<long long>(pieces->batch) * p.tiles_m * p.tiles_n * cfg.split_k >= (1LL << 31))
+                return fail(TDX_ERR_UNSUPPORTED, "too many batched tiles for one launch");
+            p.batch = static_cast<int>(pieces->batch);
+            p.batch_c = pieces->batch_c;
+        }
     }
+    const int64_t nbatch = pieces ? pieces->batch : 1;
 
     if (cfg.split_k > 1) {
-        const size_t need = static_cast<size_t>(cfg.split_k) * g.M * g.N * sizeof(float);
+        const size_t need = static_cast<size_t>(cfg.split_k) * g.M * g.N * sizeof(float) * nbatch;
         if (internal_ws) {
             int rc = ensure_ws(ctx, need, &ws);
             if (rc) return rc;
@@ -144,6 +153,11 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         uint64_t str[1] = {static_cast<uint64_t>(g.M) * 2};
         uint32_t box[2] = {64, 64};
         rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
+    } else if (nbatch > 1) {
+        uint64_t dims[3] = {static_cast<uint64_t>(k_cols), static_cast<uint64_t>(g.M), static_cast<uint64_t>(nbatch)};
+        uint64_t str[2] = {static_cast<uint64_t>(k_cols) * 2, static_cast<uint64_t>(k_cols) * 2 * g.M};
+        uint32_t box[3] = {64, 128, 1};
+        rc = get_tensor_map(ctx, A, 3, dims, str, box, &ma);
     } else {
         uint64_t dims[2] = {static_cast<uint64_t>(k_cols), static_cast<uint64_t>(g.M)};
         uint64_t str[1] = {static_cast<uint64_t>(k_cols) * 2};
@@ -153,7 +167,7 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     if (rc) return rc;
     // tile widths fitted to the number of CTAs (see plan_fitted_tiles): B then arrives in 64-row copies
     int plan_grid = 0;
-    if (cfg.fit != 1 && cfg.split_k == 1 && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0) {
+    if (cfg.fit != 1 && cfg.split_k == 1 && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0 && nbatch == 1) {
         DevicePlan dp;
         rc = get_tile_plan(ctx, g.M, g.N, num_kb, cfg.tile_m, cfg.tile_n, cfg.raster, cfg.fit == 2 ? 0.0 : 0.03, st, &dp);
         if (rc) return rc;
@@ -169,6 +183,11 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
         uint32_t box[2] = {64, 64};
         rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
+    } else if (nbatch > 1) {
+        uint64_t dims[3] = {static_cast<uint64_t>(k_cols), static_cast<uint64_t>(g.N), static_cast<uint64_t>(nbatch)};
+        uint64_t str[2] = {static_cast<uint64_t>(k_cols) * 2, static_cast<uint64_t>(k_cols) * 2 * g.N};
+        uint32_t box[3] = {64, static_cast<uint32_t>(cfg.tile_n), 1};
+        rc = get_tensor_map(ctx, B, 3, dims, str, box, &mb);
     } else {
         uint64_t dims[2] = {static_cast<uint64_t>(k_cols), static_cast<uint64_t>(g.N)};
         uint64_t str[1] = {static_cast<uint64_t>(k_cols) * 2};
@@ -192,8 +211,8 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     if (cfg.split_k > 1 && pieces) {
         // fp32 result: partial sums (fp32, dense) -> alpha * sum + beta * C
         const long long MN = static_cast<long long>(g.M) * g.N;
-        const int vec4 = (MN % 4 == 0 && reinterpret_cast<uintptr_t>(C) % 16 == 0) ? 1 : 0;
-        const int grid = static_cast<int>(std::min<long long>(ceil_div(vec4 ? MN / 4 : MN, 256), 148LL * 16));
+        const int vec4 = (MN % 4 == 0 && reinterpret_cast<uintptr_t>(C) % 16 == 0 && pieces->batch_c % 4 == 0) ? 1 : 0;
+        const int grid = static_cast<int>(std::min<long long>(ceil_div((vec4 ? MN / 4 : MN) * nbatch, 256), 148LL * 16));
         cudaLaunchConfig_t lc;
         std::memset(&lc, 0, sizeof lc);
         lc.gridDim = dim3(static_cast<unsigned>(std::max(grid, 1)));
@@ -205,7 +224,7 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         lc.attrs = attr;
         lc.numAttrs = 1;
         TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::splitk_reduce_f32_kernel, MN, cfg.split_k, static_cast<const float*>(p.partial), alpha,
-                                    beta, static_cast<float*>(C), vec4));
+                                    beta, static_cast<float*>(C), vec4, static_cast<int>(nbatch), static_cast<long long>(pieces->batch_c)));
         g_launches.fetch_add(1);
         return TDX_OK;
     }
@@ -576,6 +595,23 @@ int run_gemm_f32_pieces(DeviceCtx* ctx, const GemmProblem& g, float alpha, const
             if ((rc = split(a + (a_shared ? 0 : b0 * ba.stride_a), static_cast<int>(g.M), sa_i, sa_k, ba.stride_a, a_shared ? 1 : nb, pa))) return rc;
         if (!b_shared || b0 == 0)     // B'' rows are the columns j of op(B): element (j, k) at B[k * sb_k + j * sb_j]
             if ((rc = split(b + (b_shared ? 0 : b0 * ba.stride_b), static_cast<int>(g.N), sb_j, sb_k, ba.stride_b, b_shared ? 1 : nb, pb))) return rc;
+        if (nb > 1 && !a_shared && !b_shared) {
+            // all batches of the chunk in one launch: 3-D operands, items over batch x tiles x splits
+            PieceInfo pb_info = pi;
+            pb_info.batch = nb;
+            pb_info.batch_c = ba.stride_c;
+            tdx_config bc = cfg;
+            if (!user_cfg || user_cfg->split_k == 0) {
+                // the batches already multiply the tiles: split K only as far as it takes to give every SM an item
+                const int64_t tiles = nb * ceil_div(g.M, cfg.tile_m) * ceil_div(g.N, cfg.tile_n);
+                int64_t sk = std::max<int64_t>(1, std::min<int64_t>({32, ctx->sm_count / std::max<int64_t>(1, tiles), gg.K / 64 / 4}));
+                while (sk > 1 && (sk - 1) * ceil_div(gg.K / 64, sk) >= gg.K / 64) --sk;
+                bc.split_k = static_cast<int>(sk);
+            }
+            rc = run_gemm_umma(ctx, gg, alpha, pa, pb, c + b0 * ba.stride_c, bc, nullptr, 0, true, st, ba.beta, &pb_info);
+            if (rc) return rc;
+            continue;
+        }
         for (int64_t i = 0; i < nb; ++i) {
             const char* ai = static_cast<const char*>(pa) + (a_shared ? 0 : i * a_one);
             const char* bi = static_cast<const char*>(pb) + (b_shared ? 0 : i * b_one);

@@ -440,20 +440,23 @@ __global__ void copy_pad_ring_kernel(long long total, long long C, long long Hp,
 }
 
 // The same reduction with an fp32 result: out = alpha * sum_s partial[s] + beta * out (the fp32 GEMM from bf16 pieces).
+// Batched: partial is [batch][split][MN], batch b of out starts batch_c elements after batch b - 1.
 __global__ void splitk_reduce_f32_kernel(long long MN, int split, const float* __restrict__ partial, float alpha, float beta,
-                                         float* out, int vec4) {
+                                         float* out, int vec4, int batch = 1, long long batch_c = 0) {
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (vec4) {
-        const long long groups = MN / 4;
-        for (long long g = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; g < groups;
-             g += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const long long per = MN / 4, groups = per * batch;
+        for (long long gg = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; gg < groups;
+             gg += static_cast<long long>(gridDim.x) * blockDim.x) {
+            const long long b = gg / per, g = gg - b * per;
+            const float* pb = partial + b * split * MN;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int s = 0; s < split; ++s) {
-                const float4 v = __ldg(reinterpret_cast<const float4*>(partial + s * MN) + g);
+                const float4 v = __ldg(reinterpret_cast<const float4*>(pb + s * MN) + g);
                 acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
             }
             float4 r = make_float4(alpha * acc.x, alpha * acc.y, alpha * acc.z, alpha * acc.w);
-            float4* o = reinterpret_cast<float4*>(out) + g;
+            float4* o = reinterpret_cast<float4*>(out + b * batch_c) + g;
             if (beta != 0.0f) {
                 const float4 old = *o;
                 r.x = fmaf(beta, old.x, r.x); r.y = fmaf(beta, old.y, r.y); r.z = fmaf(beta, old.z, r.z); r.w = fmaf(beta, old.w, r.w);
@@ -461,12 +464,14 @@ __global__ void splitk_reduce_f32_kernel(long long MN, int split, const float* _
             *o = r;
         }
     } else {
-        for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < MN;
-             e += static_cast<long long>(gridDim.x) * blockDim.x) {
+        for (long long ee = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; ee < MN * batch;
+             ee += static_cast<long long>(gridDim.x) * blockDim.x) {
+            const long long b = ee / MN, e = ee - b * MN;
             float acc = 0.0f;
-            for (int s = 0; s < split; ++s) acc += __ldg(partial + s * MN + e);
+            for (int s = 0; s < split; ++s) acc += __ldg(partial + (b * split + s) * MN + e);
             const float v = alpha * acc;
-            out[e] = beta != 0.0f ? fmaf(beta, out[e], v) : v;
+            float* o = out + b * batch_c + e;
+            *o = beta != 0.0f ? fmaf(beta, *o, v) : v;
         }
     }
 }

@@ -85,6 +85,11 @@ struct UmmaParams {
     int seg_kb;
     int a_seg[6], b_seg[6];
     float* Cf;
+    // batched (pieces path only, batch > 1): the operands are 3-D tensors (K, rows, batch), the items run over
+    // batch x tiles x splits, C of batch b starts batch_c elements after that of b - 1, and the split-K partials
+    // are laid out [batch][split][M][N]
+    int batch;
+    long long batch_c;
     const int4* tiles;
     int rounds;
     int b_box;                // rows of one B copy (K-major B); bn when there is no table
@@ -134,11 +139,18 @@ __global__ void bounded_wait_selftest_kernel(int* status, long long limit_cycles
 
 struct TileCoord {
     int m_blk, n_blk, kb0, kb1, split;
+    int batch;                // batch index (0 unless the launch is batched)
     int n0, bn;               // first output column and width of the tile
 };
 
 __device__ __forceinline__ TileCoord decode_item(const UmmaParams& p, int item) {
     TileCoord t;
+    t.batch = 0;
+    if (p.batch > 1) {
+        const int per_batch = p.tiles_m * p.tiles_n * p.split_k;
+        t.batch = item / per_batch;
+        item -= t.batch * per_batch;
+    }
     const int tile = item / p.split_k;
     t.split = item - tile * p.split_k;
     const int per_panel = p.panel * p.tiles_n;
@@ -163,6 +175,7 @@ __device__ __forceinline__ bool get_tile(const UmmaParams& p, int local, int fir
         if (local >= p.rounds) return false;
         const int4 e = __ldg(p.tiles + static_cast<size_t>(local) * item_stride + first_item);
         if (e.z == 0) return false;
+        t->batch = 0;
         t->m_blk = e.x;
         t->n_blk = 0;
         t->n0 = e.y;
@@ -382,7 +395,7 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
             const int col0 = t.n0 + c0;
             if (valid && col0 < p.N) {
             if (p.split_k > 1) {
-                float* dst = p.partial + (static_cast<long long>(t.split) * p.M + grow) * p.N + col0;
+                float* dst = p.partial + ((static_cast<long long>(t.batch) * p.split_k + t.split) * p.M + grow) * p.N + col0;
                 if (p.vec_store) {
 #pragma unroll
                     for (int g = 0; g < 8; ++g) {
@@ -399,7 +412,7 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                 }
             } else if (!kConv && p.Cf != nullptr) {
                 // fp32 output (the fp32 GEMM from bf16 pieces): out = alpha * acc + beta * (what Cf held)
-                float* dst = p.Cf + grow * p.ldc + col0;
+                float* dst = p.Cf + t.batch * p.batch_c + grow * p.ldc + col0;
                 if (p.vec_store) {
 #pragma unroll
                     for (int g = 0; g < 8; ++g) {
@@ -518,7 +531,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = s_tmem_base;
-    const int total_items = p.tiles_m * p.tiles_n * p.split_k;
+    const int total_items = p.tiles_m * p.tiles_n * p.split_k * (p.batch > 1 ? p.batch : 1);
     // the next grid in the stream (the split-K reduction, or the next call's kernel) may be scheduled as SMs free up and
     // run its set-up; this grid touches global memory only after its own predecessor has completed
     ptx::grid_launch_dependents();
@@ -568,20 +581,28 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                             ka = p.a_seg[sg] * p.seg_kb + r;
                             kbb = p.b_seg[sg] * p.seg_kb + r;
                         }
-                        if (p.a_mn_major) {
-                            for (int i = 0; i < 2 * mh; ++i)
-                                ptx::tma_load_2d(a_dst + i * 8192, &tmA, bar, t.m_blk * p.bm + i * 64, ka * kBK);
-                        } else {
+                        if (p.batch > 1) {
+                            // batched: K-major 3-D operands; rows past M or N of a batch are zero-filled, not the next batch's
                             for (int h = 0; h < mh; ++h)
-                                ptx::tma_load_2d(a_dst + h * kHalfABytes, &tmA, bar, ka * kBK,
-                                                 t.m_blk * p.bm + h * kHalfM);
-                        }
-                        if (p.b_mn_major) {
-                            for (int i = 0; i < t.bn / 64; ++i)
-                                ptx::tma_load_2d(b_dst + i * 8192, &tmB, bar, t.n0 + i * 64, kbb * kBK);
-                        } else {
+                                ptx::tma_load_3d(a_dst + h * kHalfABytes, &tmA, bar, ka * kBK, t.m_blk * p.bm + h * kHalfM, t.batch);
                             for (int r0 = 0; r0 < t.bn; r0 += p.b_box)
-                                ptx::tma_load_2d(b_dst + r0 * 128, &tmB, bar, kbb * kBK, t.n0 + r0);
+                                ptx::tma_load_3d(b_dst + r0 * 128, &tmB, bar, kbb * kBK, t.n0 + r0, t.batch);
+                        } else {
+                            if (p.a_mn_major) {
+                                for (int i = 0; i < 2 * mh; ++i)
+                                    ptx::tma_load_2d(a_dst + i * 8192, &tmA, bar, t.m_blk * p.bm + i * 64, ka * kBK);
+                            } else {
+                                for (int h = 0; h < mh; ++h)
+                                    ptx::tma_load_2d(a_dst + h * kHalfABytes, &tmA, bar, ka * kBK,
+                                                     t.m_blk * p.bm + h * kHalfM);
+                            }
+                            if (p.b_mn_major) {
+                                for (int i = 0; i < t.bn / 64; ++i)
+                                    ptx::tma_load_2d(b_dst + i * 8192, &tmB, bar, t.n0 + i * 64, kbb * kBK);
+                            } else {
+                                for (int r0 = 0; r0 < t.bn; r0 += p.b_box)
+                                    ptx::tma_load_2d(b_dst + r0 * 128, &tmB, bar, kbb * kBK, t.n0 + r0);
+                            }
                         }
                     }
                     if (++stage == p.stages) {
