@@ -19,6 +19,11 @@
  *    tdx_check_device_status.
  *  - All matrices are dense row-major; bf16 values are the upper 16 bits of the fp32 pattern.
  *  - tdx_last_error() returns a thread-local, library-owned description of the last failure.
+ *  - Library-owned device scratch (split-K partial sums of the non-_ex calls, the bf16 pieces of the fp32
+ *    tensor-core path, staging buffers of the *_host calls, tile tables) is per device, grown on demand with
+ *    cudaMalloc and reused from call to call in stream order: calls that use it must all be issued on ONE stream per
+ *    device, and from one host thread at a time.  Calls that use none (bf16 GEMM / convolution without split-K, or
+ *    with a caller workspace through the _ex entry points) have no such restriction; the caches behind them are locked.
  */
 #ifndef TDX_H_
 #define TDX_H_
@@ -45,7 +50,7 @@ typedef enum {
 } tdx_status;
 
 typedef enum {
-    TDX_F32 = 0, /* A, B, C fp32; fp32 FMA on CUDA cores                     */
+    TDX_F32 = 0, /* A, B, C fp32; fp32 FMAs on CUDA cores, or bf16 pieces on tensor cores */
     TDX_BF16 = 1 /* A, B bf16; fp32 accumulate (tensor cores); C bf16        */
 } tdx_dtype;
 
