@@ -219,6 +219,18 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
         const int sidx = local * mh + half;
         const int buf = sidx % p.slots;
         const uint32_t aphase = (sidx / p.slots) & 1;
+        // Staged epilogue: lane l fetches the bias of column (step's first column + l) for each of this warp's (at most
+        // four) 32-column steps NOW, so that the loads complete while the warp waits for the accumulators -- fetched
+        // inside the step, their L2 latency was paid four times per tile (conv 56x56x256: epilogue 3.8 us vs 2.5 for
+        // the same tile without bias).  Columns past N are clipped by the store; the index only has to stay in range.
+        float bias_pre0 = 0.0f, bias_pre1 = 0.0f, bias_pre2 = 0.0f, bias_pre3 = 0.0f;
+        if (p.bias != nullptr && p.tma_store && p.split_k == 1) {
+            const int c_first = t.n0 + cgrp * 32 + lane, c_step = ncgrp * 32, last = p.N - 1;
+            bias_pre0 = __ldg(p.bias + min(c_first, last));
+            bias_pre1 = __ldg(p.bias + min(c_first + c_step, last));
+            bias_pre2 = __ldg(p.bias + min(c_first + 2 * c_step, last));
+            bias_pre3 = __ldg(p.bias + min(c_first + 3 * c_step, last));
+        }
         if (!wait_bounded(&tfull_bar[buf], aphase, abort_flag, p.status, kTimeoutEpilogue)) break;
         ptx::tc_fence_after_sync();
 
@@ -309,16 +321,17 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
             uint8_t* my_row = stage_buf + lane * 64;
             const int sw = (lane >> 1) & 3;
             const bool plain = (p.bias == nullptr) && (p.relu == 0) && (p.residual == nullptr);
-            for (int c0 = cgrp * 32; c0 < t.bn; c0 += ncgrp * 32) {
+            int step = 0;
+            for (int c0 = cgrp * 32; c0 < t.bn; c0 += ncgrp * 32, ++step) {
                 uint32_t r[32];
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                        static_cast<uint32_t>(buf * p.bn + c0);
                 ptx::tmem_ld_32x32b_x32(taddr, r);
                 const int col0 = t.n0 + c0;
-                // lane l fetches the bias of column col0 + l while the accumulator load is in flight; columns past N
-                // are clipped by the store, the index only has to stay in range
-                float bias_l = 0.0f;
-                if (p.bias != nullptr) bias_l = __ldg(p.bias + min(col0 + lane, p.N - 1));
+                // the bias of column col0 + lane: prefetched above for the first four steps of a warp (all there are
+                // with 16 epilogue warps and tiles of up to 256 columns)
+                float bias_l = step == 0 ? bias_pre0 : step == 1 ? bias_pre1 : step == 2 ? bias_pre2 : bias_pre3;
+                if (step > 3 && p.bias != nullptr) bias_l = __ldg(p.bias + min(col0 + lane, p.N - 1));
                 ptx::tmem_ld_wait();
                 if (kConv && p.residual != nullptr) {
                     // residual term (convolution only, where alpha is 1): this thread's 32 values of its output row
