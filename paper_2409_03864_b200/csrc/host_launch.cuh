@@ -412,6 +412,21 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     p.cchunks = cchunks;
     p.status = ctx->status_ptr;
 
+    // tile widths fitted to the CTA count, as for the GEMM (halo kernel, streamed filter): the filter slices then
+    // arrive in 64-row copies
+    int plan_grid = 0;
+    if (halo && !p.b_resident && cfg.fit != 1 && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0) {
+        DevicePlan dp;
+        int rcp = get_tile_plan(ctx, static_cast<int64_t>(p.tiles_m) * cfg.tile_m, c.Cout, p.num_kb, cfg.tile_m, cfg.tile_n,
+                                cfg.raster, cfg.fit == 2 ? 0.0 : 0.03, st, &dp);
+        if (rcp) return rcp;
+        if (dp.fitted) {
+            p.tiles = dp.dev;
+            p.rounds = dp.rounds;
+            p.b_box = 64;
+            plan_grid = dp.grid;
+        }
+    }
     CUtensorMap ma, ma_row, mb;
     {
         uint64_t dims[4] = {static_cast<uint64_t>(c.Cin), static_cast<uint64_t>(c.W), static_cast<uint64_t>(c.H),
@@ -436,7 +451,7 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
         uint64_t dims[3] = {static_cast<uint64_t>(c.Cin), static_cast<uint64_t>(c.R * c.S),
                             static_cast<uint64_t>(c.Cout)};
         uint64_t str[2] = {static_cast<uint64_t>(c.Cin) * 2, static_cast<uint64_t>(c.R * c.S * c.Cin) * 2};
-        uint32_t box[3] = {64, 1, static_cast<uint32_t>(cfg.tile_n)};
+        uint32_t box[3] = {64, 1, static_cast<uint32_t>(p.tiles ? 64 : cfg.tile_n)};
         int rc = get_tensor_map(ctx, w, 3, dims, str, box, &mb);
         if (rc) return rc;
     }
@@ -462,7 +477,7 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
             if (rc) return rc;
         }
     }
-    return launch_umma(ctx, true, ma, mb, mc, p, st, halo, &ma_row, &mc_row);
+    return launch_umma(ctx, true, ma, mb, mc, p, st, halo, &ma_row, &mc_row, plan_grid);
 }
 
 void gemm_strides(const GemmProblem& g, long long* sa_i, long long* sa_k, long long* sb_k, long long* sb_j) {

@@ -394,7 +394,18 @@ int enum_conv(const ConvProblem& cp, int sm_count, int smem_limit, std::vector<t
                         c.kernel = TDX_KERNEL_UMMA;
                         c.tile_m = tm; c.tile_n = bn; c.tile_k = 64; c.stages = st; c.cta_pair = 1; c.split_k = 1;
                         c.store_mode = sm; c.raster = raster; c.patch_w = kHaloPatchW; c.patch_h = kHaloPatchH; c.halo = mode;
-                        if (umma_config_reason(c, false, num_kb, smem_limit, true, cp.Cout, cp.R, cp.S) == nullptr) v->push_back(c);
+                        c.fit = 1;
+                        if (umma_config_reason(c, false, num_kb, smem_limit, true, cp.Cout, cp.R, cp.S) != nullptr) continue;
+                        v->push_back(c);
+                        if (bn >= 192 && bn % 64 == 0 && bn < cp.Cout + 64) {
+                            // the same tile with widths fitted to the CTA count, where that changes anything
+                            TilePlan plan;
+                            const int64_t rows = ceil_div(halo_patches(cp, mode), tm / 128) * tm;
+                            if (plan_fitted_tiles(rows, cp.Cout, num_kb, tm, bn, raster, sm_count, 0.0, &plan)) {
+                                c.fit = 2;
+                                v->push_back(c);
+                            }
+                        }
                     }
                 }
             }

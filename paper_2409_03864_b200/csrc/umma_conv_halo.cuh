@@ -115,8 +115,8 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             int a_buf = 0;
             uint32_t a_phase = 0;
             bool ok = true;
-            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
-                const TileCoord t = decode_item(p, item);
+            TileCoord t;
+            for (int local = 0; ok && get_tile(p, local, blockIdx.x, gridDim.x, total_items, &t); ++local) {
                 for (int cc = 0; cc < p.cchunks; ++cc) {
                     if (!wait_bounded(&aempty_bar[a_buf], a_phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) {
                         ok = false;
@@ -176,8 +176,9 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             } else {
                 int b_stage = 0;
                 uint32_t b_phase = 0;
-                for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x) {
-                    const TileCoord t = decode_item(p, item);
+                TileCoord t;
+                for (int local = 0; ok && get_tile(p, local, blockIdx.x, gridDim.x, total_items, &t); ++local) {
+                    const uint32_t slice_tx = static_cast<uint32_t>(t.bn) * 128u;     // the tile's width (fitted plans vary it)
                     for (int cc = 0; ok && cc < p.cchunks; ++cc) {
                         for (int tap = 0; tap < taps; ++tap) {
                             if (!wait_bounded(&bempty_bar[b_stage], b_phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) {
@@ -185,9 +186,10 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                                 break;
                             }
                             uint64_t* bar = &bfull_bar[b_stage];
-                            ptx::mbar_arrive_expect_tx(bar, b_bytes);
-                            ptx::tma_load_3d(b_ring + static_cast<size_t>(b_stage) * b_bytes, &tmB, bar, cc * kBK, tap,
-                                             t.n_blk * p.bn);
+                            ptx::mbar_arrive_expect_tx(bar, slice_tx);
+                            for (int r0 = 0; r0 < t.bn; r0 += p.b_box)
+                                ptx::tma_load_3d(b_ring + static_cast<size_t>(b_stage) * b_bytes + r0 * 128, &tmB, bar, cc * kBK,
+                                                 tap, t.n0 + r0);
                             if (++b_stage == p.stages) { b_stage = 0; b_phase ^= 1u; }
                         }
                     }
@@ -200,7 +202,7 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issuer
         if (ptx::elect_one()) {
-            const uint32_t idesc = ptx::make_idesc_bf16_f32(kHalfM, p.bn, 0, 0);
+            const uint32_t idesc0 = ptx::make_idesc_bf16_f32(kHalfM, p.bn, 0, 0);
             const uint32_t a_sbo = static_cast<uint32_t>(p.hpitch) * 128u;     // one window row between 8-row groups
             // descriptors are built once and advanced by additions (16-byte units): the issuing thread has only
             // a few dozen cycles per MMA when the tile is narrow
@@ -213,7 +215,10 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             uint32_t a_phase = 0, b_phase = 0;
             bool ok = true;
             if (p.b_resident && !wait_bounded(&bfull_bar[0], 0, abort_flag, p.status, kTimeoutMma)) ok = false;
-            for (int item = blockIdx.x; ok && item < total_items; item += gridDim.x, ++local) {
+            TileCoord t;
+            for (; ok && get_tile(p, local, blockIdx.x, gridDim.x, total_items, &t); ++local) {
+                // N field of the instruction descriptor (bits 17..22) follows the tile's width
+                const uint32_t idesc = (idesc0 & ~(0x3Fu << 17)) | (static_cast<uint32_t>(t.bn >> 3) << 17);
                 uint32_t d_tmem[2] = {0u, 0u};
                 int slot[2] = {0, 0};
 #pragma unroll

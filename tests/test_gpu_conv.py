@@ -310,3 +310,18 @@ def test_conv_with_residual_term_vs_oracle(case, relu):
     # the residual really entered: the result differs from the plain convolution
     st, y_plain, _ = run_conv(N, H, W, Cin, Cout, R, S, pad, stride, "bf16", x, w, b, relu)
     assert st == 0 and not np.array_equal(oracle.decode(y_plain, "bf16"), got)
+
+
+@pytest.mark.parametrize("tile_m", [128, 256])
+def test_conv_halo_with_tile_widths_fitted_to_the_cta_count(tile_m):
+    # fit = 2 on the halo kernel: some row blocks are cut into two 128-column tiles; filter slices arrive in 64-row copies
+    N, H, W, Cin, Cout = 8, 56, 56, 64, 256
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=86)
+    st, y, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, cfg=umma(halo=3, tile_m=tile_m, tile_n=256, fit=2))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    rows = structured_rows(N * H * W, max_blocks=24)
+    err = conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y, rows=rows)
+    assert err < TIGHT["bf16"], err
+    st, y1, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, cfg=umma(halo=3, tile_m=tile_m, tile_n=256, fit=1))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert np.array_equal(y, y1)          # the reduction order inside an output does not depend on the tile width
