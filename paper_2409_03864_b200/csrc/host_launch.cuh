@@ -516,11 +516,24 @@ int run_gemm_simt_f32(DeviceCtx* ctx, const GemmProblem& g, float alpha, const v
         dim3 grid(static_cast<unsigned>(ceil_div(g.N, 32)), static_cast<unsigned>(ceil_div(g.M, 32)), nz);
         const bool rowmajor16 = plain && !g.transA && !g.transB && g.K % 4 == 0 && g.N % 4 == 0 &&
                                 reinterpret_cast<uintptr_t>(A) % 16 == 0 && reinterpret_cast<uintptr_t>(B) % 16 == 0;
+        // small problems are launch-bound: programmatic stream serialization lets a call's launch overlap the
+        // previous kernel's tail (the kernels wait on the device before touching memory)
+        cudaLaunchConfig_t lc;
+        std::memset(&lc, 0, sizeof lc);
+        lc.gridDim = grid;
+        lc.blockDim = dim3(256);
+        lc.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = attr;
+        lc.numAttrs = 1;
         if (rowmajor16)
-            tdx::sgemm_small_rowmajor_kernel<<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, alpha, a, b, c);
+            TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::sgemm_small_rowmajor_kernel, (int)g.M, (int)g.N, (int)g.K, alpha, a, b, c));
         else
-            tdx::sgemm_small_kernel<<<grid, 256, 0, st>>>((int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k, sb_j, alpha, a, b,
-                                                          c, ba.beta, ba.stride_a, ba.stride_b, ba.stride_c);
+            TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::sgemm_small_kernel, (int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k, sb_j, alpha,
+                                        a, b, c, ba.beta, static_cast<long long>(ba.stride_a), static_cast<long long>(ba.stride_b),
+                                        static_cast<long long>(ba.stride_c)));
     }
     TDX_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);

@@ -40,6 +40,8 @@ sgemm_small_kernel(int M, int N, int K, long long sa_i, long long sa_k, long lon
                    const float* __restrict__ A, const float* __restrict__ B, float* __restrict__ C, float beta = 0.0f,
                    long long batch_a = 0, long long batch_b = 0, long long batch_c = 0) {
     constexpr int BM = 32, BN = 32, BK = 32, ST = 4, LD = BM + 2;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     // see sgemm_small_rowmajor_kernel
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     A += blockIdx.z * batch_a;
     B += blockIdx.z * batch_b;
     C += blockIdx.z * batch_c;
@@ -209,6 +211,10 @@ __global__ void __launch_bounds__(256)
 sgemm_small_rowmajor_kernel(int M, int N, int K, float alpha, const float* __restrict__ A, const float* __restrict__ B,
                             float* __restrict__ C) {
     constexpr int BM = 32, BN = 32, BK = 32, ST = 4, LDA = BK + 4, LDB = BN + 4;
+    // launched with programmatic stream serialization: let the next kernel of the stream be scheduled, and touch
+    // global memory only once the previous one has completed (no-ops for an ordinary launch)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     __shared__ __align__(16) float As[ST][BM][LDA];   // [m][k]
     __shared__ __align__(16) float Bs[ST][BK][LDB];   // [k][n]
     const int tid = threadIdx.x;
