@@ -154,6 +154,15 @@ int tdx_add_zero_pad(int64_t N, int64_t H, int64_t W, int64_t C, int pad_top, in
                      int dtype, const void* x, const void* y, void* out, void* stream);
 
 /*
+ * tdx_gemm with bf16 operands and an fp32 result: C[M x N] (fp32) = alpha * op(A) . op(B), A and B bf16 as for
+ * tdx_gemm.  The fp32 accumulator is written as it is (times alpha), without the rounding to bf16 -- for results that
+ * feed a reduction or a loss, or that are accumulated further.  Same kernels and layout rules as the bf16 GEMM
+ * (tensor cores when the 16-byte rules hold, the generic GPU kernel otherwise); C needs 4-byte alignment.
+ */
+int tdx_gemm_f32out(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, const void* A, const void* B,
+                    void* C, void* stream);
+
+/*
  * Same as tdx_gemm with an explicit configuration and caller-owned split-K workspace.
  * cfg = NULL or cfg->split_k = 0: the library chooses split_k (tuning cache, else heuristic); then
  * `workspace` may be NULL and the library uses an internal, lazily grown buffer.  With an explicit

@@ -73,6 +73,7 @@ def lib() -> ctypes.CDLL:
         L.tdx_gemm_batched_host.argtypes = [i64, i64, i64, i64, ci, ci, cf, cf, ci, vp, vp, vp, vp]
         L.tdx_add_zero_pad.argtypes = [i64, i64, i64, i64, ci, ci, ci, ci, ci, vp, vp, vp, vp]
         L.tdx_add_zero_pad_host.argtypes = [i64, i64, i64, i64, ci, ci, ci, ci, ci, vp, vp, vp]
+        L.tdx_gemm_f32out.argtypes = [i64, i64, i64, ci, ci, cf, vp, vp, vp, vp]
         L.tdx_gemm_workspace_size.argtypes = [i64, i64, i64, ci, cfgp, ctypes.POINTER(sz)]
         L.tdx_conv2d_bias_relu.argtypes = conv_args
         L.tdx_conv2d_bias_relu_ex.argtypes = conv_args + [cfgp]
@@ -114,7 +115,7 @@ def lib() -> ctypes.CDLL:
 
 # every symbol include/tdx.h declares
 EXPORTS = (
-    "tdx_gemm", "tdx_add_zero_pad", "tdx_add_zero_pad_host", "tdx_gemm_batched", "tdx_gemm_batched_host", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_add_relu", "tdx_conv2d_bias_relu_ex",
+    "tdx_gemm", "tdx_gemm_f32out", "tdx_add_zero_pad", "tdx_add_zero_pad_host", "tdx_gemm_batched", "tdx_gemm_batched_host", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_add_relu", "tdx_conv2d_bias_relu_ex",
     "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_gemm_guided", "tdx_model_gemm_us", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
     "tdx_enum_conv2d_configs", "tdx_default_gemm_config", "tdx_default_conv2d_config", "tdx_tune_save",
     "tdx_tune_load", "tdx_tune_clear", "tdx_gemm_tile_plan", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
@@ -196,6 +197,11 @@ def tdx_add_zero_pad_host(N, H, W, C, pad_top, pad_bottom, pad_left, pad_right, 
     """In place on host arrays: y = zero_pad(x) + y."""
     return lib().tdx_add_zero_pad_host(N, H, W, C, pad_top, pad_bottom, pad_left, pad_right, dtype, _ptr(x), _ptr(y),
                                        _stream(stream))
+
+
+def tdx_gemm_f32out(M, N, K, transA, transB, alpha, A, B, C, stream=None) -> int:
+    """bf16 A and B, fp32 C = alpha * op(A) . op(B) (the accumulator without the rounding to bf16)."""
+    return lib().tdx_gemm_f32out(M, N, K, transA, transB, alpha, _ptr(A), _ptr(B), _ptr(C), _stream(stream))
 
 
 def tdx_gemm_workspace_size(M, N, K, dtype, cfg):

@@ -88,7 +88,8 @@ struct PieceInfo {
 
 int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
                   const tdx_config& cfg, void* ws, size_t ws_bytes, bool internal_ws, cudaStream_t st, float beta = 0.0f,
-                  const PieceInfo* pieces = nullptr) {
+                  const PieceInfo* pieces = nullptr, bool c_f32 = false) {
+    // c_f32: bf16 operands, fp32 result (C points to floats); pieces imply it
     const int64_t num_kb = ceil_div(g.K, 64);
     const int64_t k_cols = pieces ? pieces->cols : g.K;        // columns the K-major operands really have
     UmmaParams p;
@@ -134,6 +135,13 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         }
     }
     const int64_t nbatch = pieces ? pieces->batch : 1;
+    const long long out_batch_c = pieces ? static_cast<long long>(pieces->batch_c) : 0;
+    if (c_f32 && !pieces) {
+        p.Cf = static_cast<float*>(C);
+        p.C = nullptr;
+        p.vec_store = (g.N % 4 == 0) && (reinterpret_cast<uintptr_t>(C) % 16 == 0);
+    }
+    const bool f32_result = pieces != nullptr || c_f32;
 
     if (cfg.split_k > 1) {
         const size_t need = static_cast<size_t>(cfg.split_k) * g.M * g.N * sizeof(float) * nbatch;
@@ -198,7 +206,7 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
 
     CUtensorMap mc = ma;   // unused unless the staged epilogue is on
     // the accumulate term is read by the direct-store epilogue (and by the split-K reduction) only
-    p.tma_store = (cfg.store_mode == 2 && cfg.split_k == 1 && p.vec_store && beta == 0.0f && !pieces) ? 1 : 0;
+    p.tma_store = (cfg.store_mode == 2 && cfg.split_k == 1 && p.vec_store && beta == 0.0f && !f32_result) ? 1 : 0;
     if (p.tma_store) {
         uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.M)};
         uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
@@ -208,10 +216,10 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     }
     rc = launch_umma(ctx, false, ma, mb, mc, p, st, false, nullptr, nullptr, plan_grid);
     if (rc) return rc;
-    if (cfg.split_k > 1 && pieces) {
+    if (cfg.split_k > 1 && f32_result) {
         // fp32 result: partial sums (fp32, dense) -> alpha * sum + beta * C
         const long long MN = static_cast<long long>(g.M) * g.N;
-        const int vec4 = (MN % 4 == 0 && reinterpret_cast<uintptr_t>(C) % 16 == 0 && pieces->batch_c % 4 == 0) ? 1 : 0;
+        const int vec4 = (MN % 4 == 0 && reinterpret_cast<uintptr_t>(C) % 16 == 0 && out_batch_c % 4 == 0) ? 1 : 0;
         const int grid = static_cast<int>(std::min<long long>(ceil_div((vec4 ? MN / 4 : MN) * nbatch, 256), 148LL * 16));
         cudaLaunchConfig_t lc;
         std::memset(&lc, 0, sizeof lc);
@@ -224,7 +232,7 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         lc.attrs = attr;
         lc.numAttrs = 1;
         TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::splitk_reduce_f32_kernel, MN, cfg.split_k, static_cast<const float*>(p.partial), alpha,
-                                    beta, static_cast<float*>(C), vec4, static_cast<int>(nbatch), static_cast<long long>(pieces->batch_c)));
+                                    beta, static_cast<float*>(C), vec4, static_cast<int>(nbatch), out_batch_c));
         g_launches.fetch_add(1);
         return TDX_OK;
     }
@@ -651,12 +659,16 @@ int run_gemm_f32_pieces(DeviceCtx* ctx, const GemmProblem& g, float alpha, const
 }
 
 int run_gemm_generic(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
-                     cudaStream_t st, const BatchArgs& ba = BatchArgs()) {
+                     cudaStream_t st, const BatchArgs& ba = BatchArgs(), bool c_f32 = false) {
     long long sa_i, sa_k, sb_k, sb_j;
     gemm_strides(g, &sa_i, &sa_k, &sb_k, &sb_j);
     const long long total = g.M * g.N * ba.batch;
     const int grid = static_cast<int>(std::min<long long>(ceil_div(total, 256), static_cast<long long>(ctx->sm_count) * 32));
-    if (g.dtype == TDX_F32)
+    if (g.dtype == TDX_BF16 && c_f32)      // bf16 operands, fp32 result
+        tdx::gemm_generic_kernel<__nv_bfloat16, float><<<grid, 256, 0, st>>>(
+            g.M, g.N, g.K, sa_i, sa_k, sb_k, sb_j, alpha, static_cast<const __nv_bfloat16*>(A),
+            static_cast<const __nv_bfloat16*>(B), static_cast<float*>(C), ba.beta, ba.batch, ba.stride_a, ba.stride_b, ba.stride_c);
+    else if (g.dtype == TDX_F32)
         tdx::gemm_generic_kernel<float, float><<<grid, 256, 0, st>>>(g.M, g.N, g.K, sa_i, sa_k, sb_k, sb_j, alpha,
                                                                     static_cast<const float*>(A),
                                                                     static_cast<const float*>(B), static_cast<float*>(C),

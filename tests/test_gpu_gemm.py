@@ -429,3 +429,33 @@ def test_fp32_gemm_large_takes_the_tensor_cores_automatically():
     st, Ci, ok = run_gemm(M, N, K, 0, 0, 1.0, "f32", Ai, Bi)
     assert st == 0 and ok
     assert np.array_equal(Ci[rows].astype(np.float64), oracle.gemm(M, N, K, 0, 0, 1.0, "f32", Ai, Bi, rows=rows))
+
+
+# ------------------------------------------------------------------ bf16 operands, fp32 result
+
+@pytest.mark.parametrize("transA,transB", [(0, 1), (0, 0), (1, 0)])
+@pytest.mark.parametrize("shape", [(384, 320, 448), (130, 72, 1032), (128, 4096, 2048), (37, 53, 71)])
+def test_bf16_gemm_with_fp32_result(shape, transA, transB):
+    # the accumulator leaves as fp32: errors are those of fp32 accumulation, far below the bf16 rounding of tdx_gemm;
+    # (128, 4096, 2048) takes split-K and the fp32 reduction, (37, 53, 71) the generic kernel (no 16-byte pitches)
+    M, N, K = shape
+    A, B = si.gemm_bf16_normal(M, N, K, seed=72, transA=transA, transB=transB)
+    out = GuardedOut(M * N, "f32")
+    st = tdx.tdx_gemm_f32out(M, N, K, transA, transB, -2.0, to_dev(A), to_dev(B), out.ptr)
+    torch.cuda.synchronize()
+    assert st == 0 and out.guards_intact(), tdx.tdx_last_error()
+    err = oracle.max_normalised_error(out.payload().reshape(M, N).astype(np.float64),
+                                      oracle.gemm(M, N, K, transA, transB, -2.0, "bf16", A, B),
+                                      oracle.gemm_row_scales(M, N, K, transA, transB, -2.0, "bf16", A, B))
+    assert err < TIGHT["f32"], err
+
+
+def test_bf16_gemm_with_fp32_result_exact_integers():
+    M, N, K = 520, 264, 320
+    A = si.small_integers(73, 0, (M, K), "bf16", -8, 8)
+    B = si.small_integers(73, 1, (N, K), "bf16", -8, 8)
+    out = GuardedOut(M * N, "f32")
+    assert tdx.tdx_gemm_f32out(M, N, K, 0, 1, 1.0, to_dev(A), to_dev(B), out.ptr) == 0
+    torch.cuda.synchronize()
+    assert out.guards_intact()
+    assert np.array_equal(out.payload().reshape(M, N).astype(np.float64), oracle.gemm(M, N, K, 0, 1, 1.0, "bf16", A, B))
