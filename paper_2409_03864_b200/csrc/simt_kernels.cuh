@@ -358,6 +358,8 @@ __global__ void splitk_reduce_kernel(long long MN, int N, int split, const float
             float acc[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
+            // unrolled so that the loads of four splits are in flight together (the adds keep their order)
+#pragma unroll 4
             for (int s = 0; s < split; ++s) {
                 const float4* src = reinterpret_cast<const float4*>(partial + s * MN + e);
                 const float4 v0 = __ldg(src), v1 = __ldg(src + 1);
@@ -457,6 +459,11 @@ __global__ void splitk_reduce_f32_kernel(long long MN, int split, const float* _
             const long long b = gg / per, g = gg - b * per;
             const float* pb = partial + b * split * MN;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            // the accumulate term is fetched before the partial sums are needed, and the loads of several splits
+            // are in flight together (the adds keep their order)
+            float4 old = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (beta != 0.0f) old = *(reinterpret_cast<const float4*>(out + b * batch_c) + g);
+#pragma unroll 8
             for (int s = 0; s < split; ++s) {
                 const float4 v = __ldg(reinterpret_cast<const float4*>(pb + s * MN) + g);
                 acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
@@ -464,7 +471,6 @@ __global__ void splitk_reduce_f32_kernel(long long MN, int split, const float* _
             float4 r = make_float4(alpha * acc.x, alpha * acc.y, alpha * acc.z, alpha * acc.w);
             float4* o = reinterpret_cast<float4*>(out + b * batch_c) + g;
             if (beta != 0.0f) {
-                const float4 old = *o;
                 r.x = fmaf(beta, old.x, r.x); r.y = fmaf(beta, old.y, r.y); r.z = fmaf(beta, old.z, r.z); r.w = fmaf(beta, old.w, r.w);
             }
             *o = r;
