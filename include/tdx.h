@@ -214,6 +214,12 @@ int tdx_conv2d_bias_relu_ex(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_
  * Host-buffer variants: A, B, C (x, w, bias, y) are HOST pointers (pinned memory gives the best
  * copy rate).  The call copies the inputs to device staging buffers owned by the library, runs the
  * same kernels as above, copies the result back and returns after the stream has drained.
+ * Large problems move in chunks (tdx_gemm_host with transA == 0: row blocks of A and C;
+ * tdx_conv2d_bias_relu_host: groups of images): chunk i goes up on a copy stream owned by the
+ * library while chunk i - 1 is computed on `stream` and chunk i - 2 comes down on a second copy
+ * stream, ordered by events, so the two directions of the bus and the kernels overlap.  Each
+ * output element is computed as in one call over the whole problem.  The host buffers must stay
+ * valid and unmodified until the call returns (it returns only when all three streams are idle).
  */
 int tdx_gemm_host(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype,
                   const void* A_host, const void* B_host, void* C_host, void* stream);

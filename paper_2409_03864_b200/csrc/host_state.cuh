@@ -73,6 +73,10 @@ struct DeviceCtx {
     size_t staging_bytes[4] = {0, 0, 0, 0};
     void* pieces[2] = {nullptr, nullptr};                     // bf16 pieces of fp32 operands (A, B)
     size_t pieces_bytes[2] = {0, 0};
+    // host-buffer entry points: copies in and out run on their own streams, chunk by chunk, around the kernels
+    static constexpr int kHostChunks = 8;
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_done = nullptr, ev_in[kHostChunks] = {}, ev_out[kHostChunks] = {};
 };
 
 std::mutex g_mu;

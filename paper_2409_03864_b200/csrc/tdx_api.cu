@@ -495,6 +495,40 @@ int ensure_staging(DeviceCtx* ctx, int slot, size_t bytes, void** out) {
     return TDX_OK;
 }
 
+// Streams and events of the chunked host-buffer path, created on first use.
+int ensure_host_pipe(DeviceCtx* ctx) {
+    if (ctx->h2d != nullptr) return TDX_OK;
+    cudaStream_t a = nullptr, b = nullptr;
+    TDX_CUDA(cudaStreamCreateWithFlags(&a, cudaStreamNonBlocking));
+    TDX_CUDA(cudaStreamCreateWithFlags(&b, cudaStreamNonBlocking));
+    TDX_CUDA(cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming));
+    TDX_CUDA(cudaEventCreateWithFlags(&ctx->ev_done, cudaEventDisableTiming));
+    for (int i = 0; i < DeviceCtx::kHostChunks; ++i) {
+        TDX_CUDA(cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming));
+        TDX_CUDA(cudaEventCreateWithFlags(&ctx->ev_out[i], cudaEventDisableTiming));
+    }
+    ctx->d2h = b;
+    ctx->h2d = a;
+    return TDX_OK;
+}
+
+// How many chunks the host-buffer path cuts `units` (rows, images) into: one per 8 MiB that crosses the bus, at most
+// kHostChunks, each of at least `min_units`.
+int host_chunk_count(int64_t units, int64_t min_units, size_t bus_bytes) {
+    int64_t c = static_cast<int64_t>(bus_bytes >> 23);
+    c = std::min<int64_t>(c, DeviceCtx::kHostChunks);
+    c = std::min<int64_t>(c, units / std::max<int64_t>(min_units, 1));
+    return static_cast<int>(std::max<int64_t>(c, 1));
+}
+
+// Leave the helper streams idle before an error return (their copies touch the caller's host buffers).
+int drain_host_pipe(DeviceCtx* ctx, cudaStream_t st, int rc) {
+    cudaStreamSynchronize(ctx->h2d);
+    cudaStreamSynchronize(st);
+    cudaStreamSynchronize(ctx->d2h);
+    return rc;
+}
+
 }  // namespace
 
 // ====================================================================== C ABI
@@ -685,6 +719,43 @@ int tdx_gemm_host(int64_t M, int64_t N, int64_t K, int transA, int transB, float
     if ((rc = ensure_staging(ctx, 1, b_bytes, &dB))) return rc;
     if ((rc = ensure_staging(ctx, 2, c_bytes, &dC))) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // Row-major A: the rows are cut into chunks; chunk i's rows of A go up on one stream while chunk i - 1 is
+    // multiplied on the caller's stream and chunk i - 2's rows of C come down on a third, so the two directions of
+    // the bus and the kernels overlap.  Every row of C is computed exactly as in one call over all rows.
+    const int chunks = (transA == 0 && K > 0) ? host_chunk_count(M, 512, a_bytes + c_bytes) : 1;
+    if (chunks > 1) {
+        if ((rc = ensure_host_pipe(ctx))) return rc;
+        const int64_t rows_per = ceil_div(ceil_div(M, chunks), 256) * 256;
+        TDX_CUDA(cudaEventRecord(ctx->ev_start, st));
+        TDX_CUDA(cudaStreamWaitEvent(ctx->h2d, ctx->ev_start, 0));
+        TDX_CUDA(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, ctx->h2d));
+        int used = 0;
+        for (int i = 0; i < chunks; ++i) {
+            const int64_t r0 = i * rows_per, rows = std::min(rows_per, M - r0);
+            if (rows <= 0) break;
+            const size_t off = static_cast<size_t>(r0) * K * el;
+            TDX_CUDA(cudaMemcpyAsync(static_cast<char*>(dA) + off, static_cast<const char*>(A_host) + off,
+                                     static_cast<size_t>(rows) * K * el, cudaMemcpyHostToDevice, ctx->h2d));
+            TDX_CUDA(cudaEventRecord(ctx->ev_in[i], ctx->h2d));
+            used = i + 1;
+        }
+        for (int i = 0; i < used; ++i) {
+            const int64_t r0 = i * rows_per, rows = std::min(rows_per, M - r0);
+            const size_t a_off = static_cast<size_t>(r0) * K * el, c_off = static_cast<size_t>(r0) * N * el;
+            TDX_CUDA(cudaStreamWaitEvent(st, ctx->ev_in[i], 0));
+            rc = gemm_dispatch(rows, N, K, transA, transB, alpha, dtype, static_cast<char*>(dA) + a_off, dB,
+                               static_cast<char*>(dC) + c_off, stream, nullptr, nullptr, 0, true);
+            if (rc) return drain_host_pipe(ctx, st, rc);
+            TDX_CUDA(cudaEventRecord(ctx->ev_out[i], st));
+            TDX_CUDA(cudaStreamWaitEvent(ctx->d2h, ctx->ev_out[i], 0));
+            TDX_CUDA(cudaMemcpyAsync(static_cast<char*>(C_host) + c_off, static_cast<char*>(dC) + c_off,
+                                     static_cast<size_t>(rows) * N * el, cudaMemcpyDeviceToHost, ctx->d2h));
+        }
+        TDX_CUDA(cudaEventRecord(ctx->ev_done, ctx->d2h));
+        TDX_CUDA(cudaStreamWaitEvent(st, ctx->ev_done, 0));
+        TDX_CUDA(cudaStreamSynchronize(st));
+        return TDX_OK;
+    }
     if (a_bytes) TDX_CUDA(cudaMemcpyAsync(dA, A_host, a_bytes, cudaMemcpyHostToDevice, st));
     if (b_bytes) TDX_CUDA(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, st));
     rc = gemm_dispatch(M, N, K, transA, transB, alpha, dtype, dA, dB, dC, stream, nullptr, nullptr, 0, true);
@@ -765,12 +836,46 @@ int tdx_conv2d_bias_relu_host(int64_t N, int64_t H, int64_t W, int64_t Cin, int6
     if ((rc = ensure_staging(ctx, 1, w_bytes, &dw))) return rc;
     if ((rc = ensure_staging(ctx, 2, y_bytes, &dy))) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (bias_host && (rc = ensure_staging(ctx, 3, b_bytes, &db))) return rc;
+    // The batch is cut into groups of images that go up, are convolved and come down on three streams (see
+    // tdx_gemm_host); an image's output does not depend on which other images share its launch.
+    const int chunks = (x_bytes > 0 && w_bytes > 0) ? host_chunk_count(N, 1, x_bytes + y_bytes) : 1;
+    if (chunks > 1) {
+        if ((rc = ensure_host_pipe(ctx))) return rc;
+        const int64_t per = ceil_div(N, chunks);
+        const size_t x_img = static_cast<size_t>(H) * W * Cin * el, y_img = static_cast<size_t>(cp.P) * cp.Q * Cout * el;
+        TDX_CUDA(cudaEventRecord(ctx->ev_start, st));
+        TDX_CUDA(cudaStreamWaitEvent(ctx->h2d, ctx->ev_start, 0));
+        TDX_CUDA(cudaMemcpyAsync(dw, w_host, w_bytes, cudaMemcpyHostToDevice, ctx->h2d));
+        if (bias_host) TDX_CUDA(cudaMemcpyAsync(db, bias_host, b_bytes, cudaMemcpyHostToDevice, ctx->h2d));
+        int used = 0;
+        for (int i = 0; i < chunks; ++i) {
+            const int64_t n0 = i * per, imgs = std::min(per, N - n0);
+            if (imgs <= 0) break;
+            TDX_CUDA(cudaMemcpyAsync(static_cast<char*>(dx) + n0 * x_img, static_cast<const char*>(x_host) + n0 * x_img,
+                                     imgs * x_img, cudaMemcpyHostToDevice, ctx->h2d));
+            TDX_CUDA(cudaEventRecord(ctx->ev_in[i], ctx->h2d));
+            used = i + 1;
+        }
+        for (int i = 0; i < used; ++i) {
+            const int64_t n0 = i * per, imgs = std::min(per, N - n0);
+            TDX_CUDA(cudaStreamWaitEvent(st, ctx->ev_in[i], 0));
+            rc = conv_dispatch(imgs, H, W, Cin, Cout, R, S, pad, stride, dtype, static_cast<char*>(dx) + n0 * x_img, dw,
+                               static_cast<const float*>(db), relu, static_cast<char*>(dy) + n0 * y_img, stream, nullptr);
+            if (rc) return drain_host_pipe(ctx, st, rc);
+            TDX_CUDA(cudaEventRecord(ctx->ev_out[i], st));
+            TDX_CUDA(cudaStreamWaitEvent(ctx->d2h, ctx->ev_out[i], 0));
+            TDX_CUDA(cudaMemcpyAsync(static_cast<char*>(y_host) + n0 * y_img, static_cast<char*>(dy) + n0 * y_img, imgs * y_img,
+                                     cudaMemcpyDeviceToHost, ctx->d2h));
+        }
+        TDX_CUDA(cudaEventRecord(ctx->ev_done, ctx->d2h));
+        TDX_CUDA(cudaStreamWaitEvent(st, ctx->ev_done, 0));
+        TDX_CUDA(cudaStreamSynchronize(st));
+        return TDX_OK;
+    }
     if (x_bytes) TDX_CUDA(cudaMemcpyAsync(dx, x_host, x_bytes, cudaMemcpyHostToDevice, st));
     TDX_CUDA(cudaMemcpyAsync(dw, w_host, w_bytes, cudaMemcpyHostToDevice, st));
-    if (bias_host) {
-        if ((rc = ensure_staging(ctx, 3, b_bytes, &db))) return rc;
-        TDX_CUDA(cudaMemcpyAsync(db, bias_host, b_bytes, cudaMemcpyHostToDevice, st));
-    }
+    if (bias_host) TDX_CUDA(cudaMemcpyAsync(db, bias_host, b_bytes, cudaMemcpyHostToDevice, st));
     rc = conv_dispatch(N, H, W, Cin, Cout, R, S, pad, stride, dtype, dx, dw, static_cast<const float*>(db), relu, dy,
                        stream, nullptr);
     if (rc) return rc;

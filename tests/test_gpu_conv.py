@@ -243,6 +243,16 @@ def test_conv_host_buffer_entry_point():
     assert conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y) < TIGHT["bf16"]
 
 
+def test_conv_host_buffer_entry_point_in_chunks():
+    # 5 images of 96 x 96 x 128: enough bytes for two groups of images (3 + 2) on the three-stream path
+    N, H, W, Cin, Cout = 5, 96, 96, 128, 128
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=77)
+    y = np.zeros((N * H * W, Cout), dtype=np.uint16)
+    st = tdx.tdx_conv2d_bias_relu_host(N, H, W, Cin, Cout, 3, 3, 1, 1, tdx.TDX_BF16, x, w, b, 1, y)
+    assert st == 0, tdx.tdx_last_error()
+    assert conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y) < TIGHT["bf16"]
+
+
 # ------------------------------------------------------------------ full-size workloads
 
 def test_full_size_conv_128x128x64():

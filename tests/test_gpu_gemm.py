@@ -338,6 +338,24 @@ def test_host_buffer_entry_point():
     assert gemm_error(M, N, K, 0, 1, -1.0, "bf16", A, B, C) < TIGHT["bf16"]
 
 
+@pytest.mark.parametrize("shape", [(2304, 1024, 4096, 1), (4100, 512, 4096, 0)])
+def test_host_buffer_entry_point_in_chunks(shape):
+    # large enough for the rows to go up, be multiplied and come down chunk by chunk on three streams (two chunks of
+    # 1280 + 1024 rows; four of 1280, 1280, 1280 and 260); called twice, the second call on the warm streams
+    M, N, K, tB = shape
+    A, B = si.gemm_bf16_normal(M, N, K, seed=62, transB=tB)
+    ref = None
+    for rep in range(2):
+        C = np.zeros((M, N), dtype=np.uint16)
+        st = tdx.tdx_gemm_host(M, N, K, 0, tB, -1.0, tdx.TDX_BF16, A, B, C)
+        assert st == 0, tdx.tdx_last_error()
+        if ref is None:
+            assert gemm_error(M, N, K, 0, tB, -1.0, "bf16", A, B, C) < TIGHT["bf16"]
+            ref = C
+        else:
+            assert np.array_equal(C, ref)
+
+
 # ------------------------------------------------------------------ full-size workloads (sampled rows)
 
 def test_full_size_negated_gemm_with_transposed_right_operand():
