@@ -523,7 +523,8 @@ int run_gemm_simt_f32(DeviceCtx* ctx, const GemmProblem& g, float alpha, const v
     } else {
         dim3 grid(static_cast<unsigned>(ceil_div(g.N, 32)), static_cast<unsigned>(ceil_div(g.M, 32)), nz);
         const bool rowmajor16 = plain && !g.transA && !g.transB && g.K % 4 == 0 && g.N % 4 == 0 &&
-                                reinterpret_cast<uintptr_t>(A) % 16 == 0 && reinterpret_cast<uintptr_t>(B) % 16 == 0;
+                                reinterpret_cast<uintptr_t>(A) % 16 == 0 && reinterpret_cast<uintptr_t>(B) % 16 == 0 &&
+                                reinterpret_cast<uintptr_t>(C) % 16 == 0;
         // small problems are launch-bound: programmatic stream serialization lets a call's launch overlap the
         // previous kernel's tail (the kernels wait on the device before touching memory)
         cudaLaunchConfig_t lc;
@@ -536,9 +537,10 @@ int run_gemm_simt_f32(DeviceCtx* ctx, const GemmProblem& g, float alpha, const v
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         lc.attrs = attr;
         lc.numAttrs = 1;
-        if (rowmajor16)
+        if (rowmajor16) {
+            lc.dynamicSmemBytes = tdx::kSmallRowmajorSmem;
             TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::sgemm_small_rowmajor_kernel, (int)g.M, (int)g.N, (int)g.K, alpha, a, b, c));
-        else
+        } else
             TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::sgemm_small_kernel, (int)g.M, (int)g.N, (int)g.K, sa_i, sa_k, sb_k, sb_j, alpha,
                                         a, b, c, ba.beta, static_cast<long long>(ba.stride_a), static_cast<long long>(ba.stride_b),
                                         static_cast<long long>(ba.stride_c)));

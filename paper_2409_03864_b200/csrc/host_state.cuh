@@ -127,6 +127,9 @@ int get_ctx(DeviceCtx** out) {
     if (e == cudaSuccess)
         e = cudaFuncSetAttribute(tdx::umma_conv_halo_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  c.smem_optin - kStaticSmemReserve);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(tdx::sgemm_small_rowmajor_kernel,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, tdx::kSmallRowmajorSmem);
     if (e != cudaSuccess) return fail(TDX_ERR_CUDA, "cudaFuncSetAttribute: %s", cudaGetErrorString(e));
     auto ins = g_ctx.emplace(dev, c);
     *out = &ins.first->second;

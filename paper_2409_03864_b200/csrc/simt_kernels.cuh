@@ -207,33 +207,52 @@ __device__ __forceinline__ void cp_async_16(float* smem_dst, const float* gmem_s
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(gmem_src), "r"(src_bytes) : "memory");
 }
 
+// What bounds a small problem on this kernel is not global memory but the shared-memory latency of the inner loop:
+// with 2 x 2 outputs per thread every four FMAs wait for a shared-memory read, and a 32 x 32 tile offers only two
+// warps per scheduler to hide it (256^3: 41 % issue utilisation, 9.7 k cycles per CTA).  So here the CTA's four groups
+// of 64 threads each take one quarter of every 128-deep K tile, a thread owns 4 x 4 outputs (eight 16-byte reads per
+// 64 FMAs), and the four partial tiles are added in a fixed order (group 0 + 1 + 2 + 3) through shared memory at the
+// end: the result is deterministic, each group's chain runs k ascending.  Two K tiles of 128 are in flight ahead of the
+// FMAs (three stages), which covers K <= 256 before the first FMA.
+constexpr int kSmallBK = 128, kSmallStages = 3;
+constexpr int kSmallLDA = kSmallBK + 4, kSmallLDB = 32 + 4;
+constexpr int kSmallStageFloats = 32 * kSmallLDA + kSmallBK * kSmallLDB;
+constexpr int kSmallRowmajorSmem = kSmallStages * kSmallStageFloats * 4;
+
 __global__ void __launch_bounds__(256)
 sgemm_small_rowmajor_kernel(int M, int N, int K, float alpha, const float* __restrict__ A, const float* __restrict__ B,
                             float* __restrict__ C) {
-    constexpr int BM = 32, BN = 32, BK = 32, ST = 4, LDA = BK + 4, LDB = BN + 4;
+    constexpr int BM = 32, BN = 32, BK = kSmallBK, ST = kSmallStages, LDA = kSmallLDA, LDB = kSmallLDB;
     // launched with programmatic stream serialization: let the next kernel of the stream be scheduled, and touch
     // global memory only once the previous one has completed (no-ops for an ordinary launch)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    __shared__ __align__(16) float As[ST][BM][LDA];   // [m][k]
-    __shared__ __align__(16) float Bs[ST][BK][LDB];   // [k][n]
+    extern __shared__ __align__(16) float ring[];
     const int tid = threadIdx.x;
-    const int tx = tid & 15, ty = tid >> 4;
+    const int grp = tid >> 6;                         // which quarter of each K tile
+    const int tx = tid & 7, ty = (tid & 63) >> 3;     // 8 x 8 threads per group; rows ty + 8 i, columns 4 tx + j
     const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
     const int ktiles = (K + BK - 1) / BK;
-    const int lr = tid >> 3, lc = (tid & 7) * 4;     // 32 rows x 8 groups of 4 floats: one 16-byte copy per thread and operand
 
     auto load_tile = [&](int kt, int st) {
         const int k0 = kt * BK;
-        {
-            const int gi = m0 + lr, gk = k0 + lc;
-            const bool ok = gi < M && gk < K;            // K % 4 == 0: a group is all in or all out
-            cp_async_16(&As[st][lr][lc], A + (ok ? static_cast<long long>(gi) * K + gk : 0), ok);
-        }
-        {
-            const int gk = k0 + lr, gj = n0 + lc;
-            const bool ok = gk < K && gj < N;
-            cp_async_16(&Bs[st][lr][lc], B + (ok ? static_cast<long long>(gk) * N + gj : 0), ok);
+        float* as = ring + st * kSmallStageFloats;    // [m][k], 32 x 128
+        float* bs = as + BM * LDA;                    // [k][n], 128 x 32
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int idx = tid + e * 256;
+            {
+                const int row = idx >> 5, c4 = (idx & 31) * 4;
+                const int gi = m0 + row, gk = k0 + c4;
+                const bool ok = gi < M && gk < K;            // K % 4 == 0: a group is all in or all out
+                cp_async_16(as + row * LDA + c4, A + (ok ? static_cast<long long>(gi) * K + gk : 0), ok);
+            }
+            {
+                const int row = idx >> 3, c4 = (idx & 7) * 4;
+                const int gk = k0 + row, gj = n0 + c4;
+                const bool ok = gk < K && gj < N;
+                cp_async_16(bs + row * LDB + c4, B + (ok ? static_cast<long long>(gk) * N + gj : 0), ok);
+            }
         }
     };
 
@@ -241,38 +260,60 @@ sgemm_small_rowmajor_kernel(int M, int N, int K, float alpha, const float* __res
         if (s < ktiles) load_tile(s, s);
         cp_async_commit();
     }
-    float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
     for (int kt = 0; kt < ktiles; ++kt) {
         cp_async_wait<ST - 2>();
         __syncthreads();
         if (kt + ST - 1 < ktiles) load_tile(kt + ST - 1, (kt + ST - 1) % ST);
         cp_async_commit();
-        const int st = kt % ST;
+        const float* as = ring + (kt % ST) * kSmallStageFloats + ty * LDA + grp * 32;
+        const float* bs = ring + (kt % ST) * kSmallStageFloats + BM * LDA + grp * 32 * LDB + tx * 4;
 #pragma unroll
-        for (int k4 = 0; k4 < BK; k4 += 4) {
-            const float4 a0 = *reinterpret_cast<const float4*>(&As[st][ty * 2][k4]);
-            const float4 a1 = *reinterpret_cast<const float4*>(&As[st][ty * 2 + 1][k4]);
-            const float av0[4] = {a0.x, a0.y, a0.z, a0.w}, av1[4] = {a1.x, a1.y, a1.z, a1.w};
+        for (int k4 = 0; k4 < 32; k4 += 4) {
+            float a[4][4];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const float2 b = *reinterpret_cast<const float2*>(&Bs[st][k4 + k][tx * 2]);
-                acc[0][0] = fmaf(av0[k], b.x, acc[0][0]);
-                acc[0][1] = fmaf(av0[k], b.y, acc[0][1]);
-                acc[1][0] = fmaf(av1[k], b.x, acc[1][0]);
-                acc[1][1] = fmaf(av1[k], b.y, acc[1][1]);
+            for (int i = 0; i < 4; ++i) {
+                const float4 v = *reinterpret_cast<const float4*>(as + i * 8 * LDA + k4);
+                a[i][0] = v.x; a[i][1] = v.y; a[i][2] = v.z; a[i][3] = v.w;
+            }
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) {
+                const float4 b = *reinterpret_cast<const float4*>(bs + (k4 + kk) * LDB);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    acc[i][0] = fmaf(a[i][kk], b.x, acc[i][0]);
+                    acc[i][1] = fmaf(a[i][kk], b.y, acc[i][1]);
+                    acc[i][2] = fmaf(a[i][kk], b.z, acc[i][2]);
+                    acc[i][3] = fmaf(a[i][kk], b.w, acc[i][3]);
+                }
             }
         }
     }
     cp_async_wait<0>();
+    __syncthreads();                                   // every group is done with the ring: reuse it for the partial tiles
+    constexpr int LDR = BN + 4;
+    float* red = ring;                                 // [group][row][column]
 #pragma unroll
-    for (int i = 0; i < 2; ++i) {
-        const int gi = m0 + ty * 2 + i;
-        if (gi >= M) continue;
+    for (int i = 0; i < 4; ++i)
+        *reinterpret_cast<float4*>(red + (grp * BM + ty + 8 * i) * LDR + tx * 4) =
+            make_float4(acc[i][0], acc[i][1], acc[i][2], acc[i][3]);
+    __syncthreads();
+    {
+        const int row = tid >> 3, c4 = (tid & 7) * 4;   // 32 rows x 8 groups of 4 columns: one per thread
+        float4 s = *reinterpret_cast<const float4*>(red + row * LDR + c4);
 #pragma unroll
-        for (int j = 0; j < 2; ++j) {
-            const int gj = n0 + tx * 2 + j;
-            if (gj < N) C[static_cast<long long>(gi) * N + gj] = alpha * acc[i][j];
+        for (int g = 1; g < 4; ++g) {
+            const float4 v = *reinterpret_cast<const float4*>(red + (g * BM + row) * LDR + c4);
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
         }
+        const int gi = m0 + row, gj = n0 + c4;
+        if (gi < M && gj < N)                            // N % 4 == 0 and C 16-byte aligned: a group is all in or all out
+            *reinterpret_cast<float4*>(C + static_cast<long long>(gi) * N + gj) =
+                make_float4(alpha * s.x, alpha * s.y, alpha * s.z, alpha * s.w);
     }
 }
 
