@@ -358,8 +358,10 @@ def run_tdx(args):
     elif w["kind"] == "gemm":
         st_cfg, cfg = tdx.tdx_default_gemm_config(w["M"], w["N"], w["K"], w["tA"], w["tB"], DT)
 
+        c_gemm = tdx.lib().tdx_gemm              # the C entry point itself: integers in, status out
+
         def launch(ins, out):
-            return tdx.tdx_gemm(w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], DT, ins[0], ins[1], out, raw_stream)
+            return c_gemm(w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], DT, ins[0], ins[1], out, raw_stream)
 
         def launch_host():
             return tdx.tdx_gemm_host(w["M"], w["N"], w["K"], w["tA"], w["tB"], w["alpha"], DT, h_in[0], h_in[1], h_out,

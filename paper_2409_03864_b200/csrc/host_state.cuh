@@ -202,12 +202,28 @@ std::string conv_key(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout,
              (long long)Cin, (long long)Cout, (long long)R, (long long)S, pad, stride, dtype);
     return b;
 }
+// every change of the cache bumps the epoch, which invalidates the per-thread memo of the last GEMM query below
+std::atomic<unsigned long long> g_tune_epoch{1};
 bool tune_lookup(const std::string& key, tdx_config* out) {
     std::lock_guard<std::mutex> lk(g_mu);
     auto it = g_tune.find(key);
     if (it == g_tune.end()) return false;
     *out = it->second.cfg;
     return true;
+}
+// A stream of calls on one shape asks the same question every time: remember the last answer per thread instead of
+// formatting the key and searching the map again (about half a microsecond of a launch-bound call).
+bool tune_lookup_gemm(int64_t M, int64_t N, int64_t K, int tA, int tB, int dtype, tdx_config* out) {
+    struct Memo { unsigned long long epoch = 0; int64_t M = 0, N = 0, K = 0; int tA = 0, tB = 0, dtype = 0; bool found = false; tdx_config cfg; };
+    static thread_local Memo memo;
+    const unsigned long long epoch = g_tune_epoch.load(std::memory_order_acquire);
+    if (memo.epoch != epoch || memo.M != M || memo.N != N || memo.K != K || memo.tA != tA || memo.tB != tB ||
+        memo.dtype != dtype) {
+        memo.found = tune_lookup(gemm_key(M, N, K, tA, tB, dtype), &memo.cfg);
+        memo.epoch = epoch; memo.M = M; memo.N = N; memo.K = K; memo.tA = tA; memo.tB = tB; memo.dtype = dtype;
+    }
+    if (memo.found) *out = memo.cfg;
+    return memo.found;
 }
 void cfg_to_ints(const tdx_config& c, int* v) {
     v[0] = c.kernel; v[1] = c.tile_m; v[2] = c.tile_n; v[3] = c.tile_k; v[4] = c.stages; v[5] = c.cta_pair;

@@ -54,7 +54,7 @@ int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_cou
     if (c.kernel == TDX_KERNEL_AUTO) {
         if (!user) {
             tdx_config cached;
-            if (tune_lookup(gemm_key(g.M, g.N, g.K, g.transA, g.transB, g.dtype), &cached)) { c = cached; from_cache = true; }
+            if (tune_lookup_gemm(g.M, g.N, g.K, g.transA, g.transB, g.dtype, &cached)) { c = cached; from_cache = true; }
         }
         if (!from_cache)
             c.kernel = g.dtype == TDX_F32 ? (prefer_f32_pieces(g, 1) ? TDX_KERNEL_UMMA : TDX_KERNEL_SIMT)
@@ -199,11 +199,11 @@ int gemm_dispatch(int64_t M, int64_t N, int64_t K, int transA, int transB, float
         TDX_CUDA(cudaMemsetAsync(C, 0, static_cast<size_t>(M) * N * (dtype == TDX_F32 ? 4 : 2), st));
         return TDX_OK;
     }
-    int sm_count, smem_limit;
-    device_limits(&sm_count, &smem_limit);
     // configuration errors are reported before anything touches the device
-    tdx_config pre;
     if (cfg) {
+        int sm_count, smem_limit;
+        device_limits(&sm_count, &smem_limit);
+        tdx_config pre;
         rc = resolve_gemm_config(g, cfg, sm_count, smem_limit, &pre);
         if (rc) return rc;
     }
@@ -1012,6 +1012,7 @@ static int tune_gemm_impl(int64_t M, int64_t N, int64_t K, int transA, int trans
     {
         std::lock_guard<std::mutex> lk(g_mu);
         g_tune[gemm_key(M, N, K, transA, transB, dtype)] = TuneEntry{*best, best_us ? *best_us : 0.0f};
+        g_tune_epoch.fetch_add(1, std::memory_order_release);
     }
     return TDX_OK;
 }
@@ -1084,6 +1085,7 @@ int tdx_tune_conv2d(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, 
     {
         std::lock_guard<std::mutex> lk(g_mu);
         g_tune[conv_key(N, H, W, Cin, Cout, R, S, pad, stride, dtype)] = TuneEntry{*best, best_us ? *best_us : 0.0f};
+        g_tune_epoch.fetch_add(1, std::memory_order_release);
     }
     return TDX_OK;
 }
@@ -1150,6 +1152,7 @@ int tdx_tune_load(const char* json_path) {
     }
     std::lock_guard<std::mutex> lk(g_mu);
     for (auto& kv : loaded) g_tune[kv.first] = kv.second;
+    g_tune_epoch.fetch_add(1, std::memory_order_release);
     return TDX_OK;
 }
 
@@ -1176,6 +1179,7 @@ int tdx_gemm_tile_plan(int64_t M, int64_t N, int64_t K, int tile_m, int tile_n, 
 int tdx_tune_clear(void) {
     std::lock_guard<std::mutex> lk(g_mu);
     g_tune.clear();
+    g_tune_epoch.fetch_add(1, std::memory_order_release);
     return TDX_OK;
 }
 
