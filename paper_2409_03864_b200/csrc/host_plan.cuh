@@ -19,10 +19,15 @@ struct TilePlan {
     double uniform = 0.0;      // the same for the uniform grid
 };
 
-// mmas_per_kb: MMAs one CTA's tensor core runs per 64-deep K block (4 per 128 rows it owns)
-double tile_cost_cycles(int mmas_per_kb, int width, int64_t num_kb) {
+// mmas_per_kb: MMAs one CTA's tensor core runs per 64-deep K block (4 per 128 rows it owns); b_rows: rows of B the
+// CTA loads per K block (the tile's width, half of it in a CTA pair).  A K block costs the MMAs or the time the SM
+// needs to take its operand slices in from L2 (about 70 bytes per cycle), whichever is longer: narrow tiles under
+// 128 rows of A are bound by the latter (128 x 128: 32 KB per 256 MMA cycles).
+double tile_cost_cycles(int mmas_per_kb, int width, int64_t num_kb, int b_rows = -1) {
     const double mma = std::max(width / 2.0, 60.0);
-    return static_cast<double>(num_kb) * mmas_per_kb * mma + 1500.0 + 13.0 * width;
+    if (b_rows < 0) b_rows = width;
+    const double ingest = (32.0 * mmas_per_kb + b_rows) * 128.0 / 70.0;
+    return static_cast<double>(num_kb) * std::max(mmas_per_kb * mma, ingest) + 1500.0 + 13.0 * width;
 }
 
 // makespan of `na` tiles of cost ca and `nb` tiles of cost cb (ca >= cb > 0), dealt longest first on g CTAs, each
@@ -52,7 +57,7 @@ bool plan_fitted_tiles(int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int
     const int64_t tiles_m = ceil_div(M, bm);
     const int64_t uniform_tiles = tiles_m * ceil_div(N, bn);
     const int mmas = pair ? 4 : 4 * (bm / 128);
-    const double c_big = tile_cost_cycles(mmas, bn, num_kb);
+    const double c_big = tile_cost_cycles(mmas, bn, num_kb, pair ? bn / 2 : bn);
     const double uniform = lpt_two_sizes(uniform_tiles, c_big, 0, 0.0, g);
     double best = uniform;
     int best_w = 0;
@@ -60,7 +65,7 @@ bool plan_fitted_tiles(int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int
     // pairs: each CTA loads half of a tile's columns, kept a multiple of 64 (one copy per 64 rows)
     const int w_step = pair ? 128 : 64;
     for (int w = bn - w_step; w >= 128; w -= w_step) {
-        const double c_small = tile_cost_cycles(mmas, w, num_kb);
+        const double c_small = tile_cost_cycles(mmas, w, num_kb, pair ? w / 2 : w);
         // option b of a row block: b tiles of width w at the high columns, a(b) tiles of width bn before them
         auto bigs_for = [&](int64_t b) { return ceil_div(std::max<int64_t>(0, N - b * w), bn); };
         // options that do not carry a tile more than needed
@@ -104,7 +109,7 @@ bool plan_fitted_tiles(int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int
     const int grid = static_cast<int>(std::min<int64_t>(total, g));
     std::vector<std::vector<T>> per(grid);
     std::vector<double> load(grid, 0.0);
-    const double c_small = tile_cost_cycles(mmas, w, num_kb);
+    const double c_small = tile_cost_cycles(mmas, w, num_kb, pair ? w / 2 : w);
     auto deal = [&](const std::vector<T>& v, double cost) {
         for (const T& t : v) {
             int who = 0;
@@ -186,7 +191,9 @@ double model_gemm_us(const GemmProblem& g, const tdx_config& c, int sm_count) {
     const int64_t tiles = ceil_div(g.M, tm) * ceil_div(g.N, bn) * split;
     const int halves = pair ? 1 : tm / 128;                                 // 128-row halves one CTA computes
     const double mma = 4.0 * halves * std::max(bn / 2.0, 60.0);
-    const double l2 = (pair ? (128.0 + bn / 2.0) : (tm + static_cast<double>(bn))) * 128.0 / 70.0;
+    // operand slices of tiles narrower than 128 columns arrive at about 46 bytes per cycle (measured: 128 x 64 tiles,
+    // 533 cycles per 24 KB K block), wider ones at about 70
+    const double l2 = (pair ? (128.0 + bn / 2.0) : (tm + static_cast<double>(bn))) * 128.0 / (bn < 128 ? 46.0 : 70.0);
     const double main_loop = static_cast<double>(kb) * std::max(mma, l2);
     const double blocks = halves * 4.0 * (bn / 32.0);                       // 32 x 32 output blocks per CTA and tile
     double epi = (c.store_mode == 2 ? 600.0 * std::ceil(blocks / 16.0) : 1200.0 * std::ceil(blocks / (4.0 * halves)));
@@ -203,7 +210,9 @@ double model_gemm_us(const GemmProblem& g, const tdx_config& c, int sm_count) {
         cycles = 5500.0 + rounds * per_tile + (overlapped ? epi : 0.0) + (pair ? 4000.0 : 0.0);
     }
     double us = cycles / clk_mhz;
-    if (split > 1) us += 3.0 + (static_cast<double>(split) * g.M * g.N * 4.0 * 2.0 + g.M * g.N * 2.0) / 4.0e6;
+    // split-K: the reduction kernel's launch hides behind the GEMM's tail and the partial sums are still in L2 when it
+    // reads them (128 x 8192 x 8192 in three splits: about 4 us on top of the GEMM kernel)
+    if (split > 1) us += 2.0 + (static_cast<double>(split) * g.M * g.N * 4.0 * 2.0 + g.M * g.N * 2.0) / 8.0e6;
     const double hbm_us = (static_cast<double>(g.M) * g.K + static_cast<double>(g.K) * g.N + static_cast<double>(g.M) * g.N) * 2.0 / 5.0e6;
     return std::max(us, hbm_us);
 }
