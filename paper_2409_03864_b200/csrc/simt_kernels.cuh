@@ -463,6 +463,9 @@ __global__ void add_zero_pad_kernel(long long rows, long long H, long long row_e
                                     long long y_row_elems, long long y_first, int vec, const T* __restrict__ x,
                                     const T* y, T* out) {
     // row r = (n, h): x + r * row_elems  <->  y + n * y_img_elems + y_first + h * y_row_elems
+    // launched with programmatic stream serialization (see sgemm_small_rowmajor_kernel)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const long long per_row = vec > 1 ? row_elems / vec : row_elems;
     const long long total = rows * per_row;
     for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < total;

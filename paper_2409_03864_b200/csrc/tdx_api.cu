@@ -698,14 +698,25 @@ int tdx_add_zero_pad(int64_t N, int64_t H, int64_t W, int64_t C, int pad_top, in
     if (interior > 0) {
         const long long work = interior / vec;
         const int grid = static_cast<int>(std::min<long long>(ceil_div(work, 256), max_grid));
+        // programmatic stream serialization: in a stream of calls the launch overlaps the previous kernel's tail
+        cudaLaunchConfig_t lc;
+        std::memset(&lc, 0, sizeof lc);
+        lc.gridDim = dim3(static_cast<unsigned>(grid));
+        lc.blockDim = dim3(256);
+        lc.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = attr;
+        lc.numAttrs = 1;
+        const long long rows = N * H, Hll = H;
         if (dtype == TDX_F32)
-            tdx::add_zero_pad_kernel<float><<<grid, 256, 0, st>>>(N * H, H, row_elems, y_img, y_row, y_first, vec,
-                                                                  static_cast<const float*>(x), static_cast<const float*>(y),
-                                                                  static_cast<float*>(out));
+            TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::add_zero_pad_kernel<float>, rows, Hll, row_elems, y_img, y_row, y_first, vec,
+                                        static_cast<const float*>(x), static_cast<const float*>(y), static_cast<float*>(out)));
         else
-            tdx::add_zero_pad_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
-                N * H, H, row_elems, y_img, y_row, y_first, vec, static_cast<const __nv_bfloat16*>(x),
-                static_cast<const __nv_bfloat16*>(y), static_cast<__nv_bfloat16*>(out));
+            TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::add_zero_pad_kernel<__nv_bfloat16>, rows, Hll, row_elems, y_img, y_row,
+                                        y_first, vec, static_cast<const __nv_bfloat16*>(x),
+                                        static_cast<const __nv_bfloat16*>(y), static_cast<__nv_bfloat16*>(out)));
         TDX_CUDA(cudaGetLastError());
         g_launches.fetch_add(1);
     }
