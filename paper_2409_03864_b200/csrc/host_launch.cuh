@@ -621,8 +621,18 @@ int run_gemm_f32_pieces(DeviceCtx* ctx, const GemmProblem& g, float alpha, const
     auto split = [&](const float* src, int rows, long long s_row, long long s_k, long long bstride, int64_t nb, void* dst) -> int {
         dim3 grid(static_cast<unsigned>(ceil_div(Kp, 32)), static_cast<unsigned>(ceil_div(rows, 32)), static_cast<unsigned>(nb));
         if (grid.y > 65535) return fail(TDX_ERR_UNSUPPORTED, "operand too tall for the piece kernel");
-        tdx::split_f32_bf16x3_kernel<<<grid, 256, 0, st>>>(rows, static_cast<int>(g.K), static_cast<int>(Kp), s_row, s_k, bstride,
-                                                           src, static_cast<__nv_bfloat16*>(dst));
+        cudaLaunchConfig_t lc;
+        std::memset(&lc, 0, sizeof lc);
+        lc.gridDim = grid;
+        lc.blockDim = dim3(256);
+        lc.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = attr;
+        lc.numAttrs = 1;
+        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::split_f32_bf16x3_kernel, rows, static_cast<int>(g.K), static_cast<int>(Kp), s_row,
+                                    s_k, bstride, src, static_cast<__nv_bfloat16*>(dst)));
         TDX_CUDA(cudaGetLastError());
         g_launches.fetch_add(1);
         return TDX_OK;

@@ -544,6 +544,10 @@ __global__ void __launch_bounds__(256)
 split_f32_bf16x3_kernel(int rows, int K, int Kp, long long s_row, long long s_k, long long batch_stride,
                         const float* __restrict__ src, __nv_bfloat16* __restrict__ dst) {
     __shared__ float tile[32][33];
+    // launched with programmatic stream serialization (see sgemm_small_rowmajor_kernel): the piece buffers are shared
+    // by successive calls, and the wait orders this kernel after everything the stream held before it
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int k0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
     const float* s = src + blockIdx.z * batch_stride;
     __nv_bfloat16* d = dst + static_cast<long long>(blockIdx.z) * rows * 3 * Kp;
