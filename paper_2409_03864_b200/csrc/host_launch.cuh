@@ -619,7 +619,7 @@ int run_gemm_f32_pieces(DeviceCtx* ctx, const GemmProblem& g, float alpha, const
     const float* b = static_cast<const float*>(B);
     float* c = static_cast<float*>(C);
     auto split = [&](const float* src, int rows, long long s_row, long long s_k, long long bstride, int64_t nb, void* dst) -> int {
-        dim3 grid(static_cast<unsigned>(ceil_div(Kp, 32)), static_cast<unsigned>(ceil_div(rows, 32)), static_cast<unsigned>(nb));
+        dim3 grid(static_cast<unsigned>(ceil_div(Kp, 64)), static_cast<unsigned>(ceil_div(rows, 32)), static_cast<unsigned>(nb));
         if (grid.y > 65535) return fail(TDX_ERR_UNSUPPORTED, "operand too tall for the piece kernel");
         cudaLaunchConfig_t lc;
         std::memset(&lc, 0, sizeof lc);

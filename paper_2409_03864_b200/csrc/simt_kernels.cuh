@@ -538,44 +538,55 @@ __global__ void splitk_reduce_f32_kernel(long long MN, int split, const float* _
 // 24 significand bits.  Source: `rows` x K logical matrix, element (i, k) at src[b * batch_stride + i * s_row + k * s_k]
 // (either stride may be 1).  Destination, per batch: rows x (3 * Kp) bf16, row-major, piece p of element (i, k) at
 // column p * Kp + k; columns K..Kp-1 of every piece are zero (Kp is K rounded up to the K block of the MMA pipeline).
-// 32 x 32 tiles through shared memory, so that reads and writes are both coalesced whichever stride is 1.
+// Tiles of 32 rows x 64 columns through shared memory, so that reads and writes are both coalesced whichever stride
+// is 1; a thread issues its eight loads back to back and writes pairs of pieces (4-byte stores, whole 128-byte lines
+// per warp).
 // ---------------------------------------------------------------------------
 __global__ void __launch_bounds__(256)
 split_f32_bf16x3_kernel(int rows, int K, int Kp, long long s_row, long long s_k, long long batch_stride,
                         const float* __restrict__ src, __nv_bfloat16* __restrict__ dst) {
-    __shared__ float tile[32][33];
+    __shared__ float tile[32][65];
     // launched with programmatic stream serialization (see sgemm_small_rowmajor_kernel): the piece buffers are shared
     // by successive calls, and the wait orders this kernel after everything the stream held before it
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    const int k0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    const int k0 = blockIdx.x * 64, r0 = blockIdx.y * 32;
     const float* s = src + blockIdx.z * batch_stride;
     __nv_bfloat16* d = dst + static_cast<long long>(blockIdx.z) * rows * 3 * Kp;
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;        // 32 x 8 threads
     if (s_k == 1) {
-        for (int j = ty; j < 32; j += 8) {
-            const int r = r0 + j, k = k0 + tx;
-            tile[j][tx] = (r < rows && k < K) ? __ldg(s + r * s_row + k) : 0.0f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int jj = ty + 8 * j, r = r0 + jj;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int k = k0 + tx + 32 * h;
+                tile[jj][tx + 32 * h] = (r < rows && k < K) ? __ldg(s + r * s_row + k) : 0.0f;
+            }
         }
     } else {       // rows are the contiguous dimension of the source: read along them, transpose in shared memory
-        for (int j = ty; j < 32; j += 8) {
-            const int k = k0 + j, r = r0 + tx;
-            tile[tx][j] = (r < rows && k < K) ? __ldg(s + r * s_row + k * s_k) : 0.0f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int kk = ty + 8 * j, k = k0 + kk, r = r0 + tx;
+            tile[tx][kk] = (r < rows && k < K) ? __ldg(s + r * s_row + k * s_k) : 0.0f;
         }
     }
     __syncthreads();
-    for (int j = ty; j < 32; j += 8) {
-        const int r = r0 + j, k = k0 + tx;
-        if (r < rows && k < Kp) {
-            const float x = tile[j][tx];
-            const __nv_bfloat16 hi = __float2bfloat16_rn(x);
-            const float r1 = x - __bfloat162float(hi);
-            const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
-            const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+    const int k = k0 + 2 * tx;                                     // Kp is a multiple of 64: a pair is all in or all out
+    if (k < Kp) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int jj = ty + 8 * j, r = r0 + jj;
+            if (r >= rows) continue;
+            const float x0 = tile[jj][2 * tx], x1 = tile[jj][2 * tx + 1];
+            const __nv_bfloat162 hi = __floats2bfloat162_rn(x0, x1);
+            const float r0x = x0 - __low2float(hi), r1x = x1 - __high2float(hi);
+            const __nv_bfloat162 mid = __floats2bfloat162_rn(r0x, r1x);
+            const __nv_bfloat162 lo = __floats2bfloat162_rn(r0x - __low2float(mid), r1x - __high2float(mid));
             __nv_bfloat16* o = d + static_cast<long long>(r) * 3 * Kp + k;
-            o[0] = hi;
-            o[Kp] = mid;
-            o[2 * Kp] = lo;
+            *reinterpret_cast<__nv_bfloat162*>(o) = hi;
+            *reinterpret_cast<__nv_bfloat162*>(o + Kp) = mid;
+            *reinterpret_cast<__nv_bfloat162*>(o + 2 * Kp) = lo;
         }
     }
 }
