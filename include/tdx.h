@@ -256,6 +256,17 @@ int tdx_enum_conv2d_configs(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_
                             int pad, int stride, int dtype, tdx_config* out, int cap, int* n);
 
 /*
+ * Search on first use (the paper's autotuner integration, Case Study 5, applied lazily).  budget = 0 (the default)
+ * switches it off; budget > 0: the first tdx_gemm / tdx_gemm_host call on a bf16 shape that the tuning cache does
+ * not know runs the guided search with that budget on scratch operands of the shape (see tdx_tune_gemm_guided:
+ * it allocates device memory, launches and synchronises `stream`; typically well under a second) and caches the
+ * winner; budget < 0: the same with every candidate timed.  Calls with an explicit configuration, calls inside a
+ * stream capture and shapes off the tensor-core path are never searched.  A search that fails does not fail the
+ * call.  Process-wide; returns TDX_OK.
+ */
+int tdx_set_autotune(int budget);
+
+/*
  * Guided search: the candidates of tdx_tune_gemm are ranked by a host-side cost model (MMA time by tile width, L2
  * ingest, epilogue overlap, wave count or fitted plan, split-K traffic, HBM floor) and only the `budget` best-ranked
  * ones, plus the heuristic default, are timed on the device -- the model-guided counterpart of Case Study 5's

@@ -91,6 +91,7 @@ def lib() -> ctypes.CDLL:
         L.tdx_tune_save.argtypes = [ctypes.c_char_p]
         L.tdx_tune_load.argtypes = [ctypes.c_char_p]
         L.tdx_tune_clear.argtypes = []
+        L.tdx_set_autotune.argtypes = [ci]
         dp = ctypes.POINTER(ctypes.c_double)
         L.tdx_gemm_tile_plan.argtypes = [i64, i64, i64, ci, ci, ci, ci, ip, ci, ip, ip, dp, dp]
         L.tdx_gemm_splitk_static.argtypes = [i64, i64, i64, ci, ci, cf, vp, vp, vp, ci, ci, vp]
@@ -118,7 +119,7 @@ EXPORTS = (
     "tdx_gemm", "tdx_gemm_f32out", "tdx_add_zero_pad", "tdx_add_zero_pad_host", "tdx_gemm_batched", "tdx_gemm_batched_host", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_add_relu", "tdx_conv2d_bias_relu_ex",
     "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_gemm_guided", "tdx_model_gemm_us", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
     "tdx_enum_conv2d_configs", "tdx_default_gemm_config", "tdx_default_conv2d_config", "tdx_tune_save",
-    "tdx_tune_load", "tdx_tune_clear", "tdx_gemm_tile_plan", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
+    "tdx_tune_load", "tdx_tune_clear", "tdx_set_autotune", "tdx_gemm_tile_plan", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
     "tdx_version",
 )
 
@@ -264,6 +265,11 @@ def tdx_tune_gemm_guided(M, N, K, transA, transB, dtype, budget, iters=20, strea
     st, best, us, tried = _tune(lambda b, bu, t, tu, c, n: L.tdx_tune_gemm_guided(
         M, N, K, transA, transB, dtype, iters, budget, b, bu, t, tu, c, n, ctypes.byref(n_cand), _stream(stream)), cap)
     return st, best, us, tried, int(n_cand.value)
+
+
+def tdx_set_autotune(budget: int) -> int:
+    """Search on first use: 0 off (default), > 0 guided search with that budget, < 0 exhaustive."""
+    return lib().tdx_set_autotune(int(budget))
 
 
 def tdx_model_gemm_us(M, N, K, transA, transB, dtype, cfg, ctas=148):

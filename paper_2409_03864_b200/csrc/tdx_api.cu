@@ -7,6 +7,13 @@
 #include <array>
 #include <tuple>
 
+// defined with the tuning entry points below; the dispatcher calls it for the search on first use
+extern "C" {
+static int tune_gemm_impl(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, int iters, int budget,
+                          tdx_config* best, float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried,
+                          int* n_candidates, void* stream);
+}
+
 namespace {
 // ------------------------------------------------------------------ validation
 int validate_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const void* A, const void* B,
@@ -227,6 +234,8 @@ void device_limits(int* sm_count, int* smem_limit) {
     }
 }
 
+// Search on first use (tdx_set_autotune): 0 = off, > 0 = the guided search with that budget, < 0 = every candidate.
+std::atomic<int> g_autotune_budget{0};
 int gemm_dispatch(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype, const void* A,
                   const void* B, void* C, void* stream, const tdx_config* cfg, void* ws, size_t ws_bytes,
                   bool internal_ws) {
@@ -235,6 +244,21 @@ int gemm_dispatch(int64_t M, int64_t N, int64_t K, int transA, int transB, float
     if (M == 0 || N == 0) return TDX_OK;
     GemmProblem g{M, N, K, transA, transB, dtype};
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int autotune = g_autotune_budget.load(std::memory_order_relaxed);
+    if (autotune != 0 && cfg == nullptr && K > 0 && dtype == TDX_BF16 && gemm_umma_layout_ok(g)) {
+        // a shape the tuning cache does not know yet is searched now, on scratch operands of its size, and the winner
+        // cached; a failed search is not an error of this call (the model-ranked choice below serves it)
+        tdx_config known;
+        cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+        if (!tune_lookup_gemm(M, N, K, transA, transB, dtype, &known) &&
+            cudaStreamIsCapturing(st, &capturing) == cudaSuccess && capturing == cudaStreamCaptureStatusNone) {
+            tdx_config best;
+            float best_us = 0.0f;
+            int n_tried = 0;
+            (void)::tune_gemm_impl(M, N, K, transA, transB, dtype, 10, autotune < 0 ? 0 : autotune, &best, &best_us, nullptr,
+                                 nullptr, 0, &n_tried, nullptr, stream);
+        }
+    }
     if (K == 0) {
         DeviceCtx* ctx0;
         rc = get_ctx(&ctx0);
@@ -1082,6 +1106,11 @@ int tdx_tune_gemm_guided(int64_t M, int64_t N, int64_t K, int transA, int transB
     if (budget < 1) return fail(TDX_ERR_INVALID_ARG, "budget must be >= 1");
     return tune_gemm_impl(M, N, K, transA, transB, dtype, iters, budget, best, best_us, tried, tried_us, cap, n_tried,
                           n_candidates, stream);
+}
+
+int tdx_set_autotune(int budget) {
+    g_autotune_budget.store(budget, std::memory_order_relaxed);
+    return TDX_OK;
 }
 
 int tdx_model_gemm_us(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const tdx_config* cfg, int ctas,

@@ -44,3 +44,29 @@ def test_guided_search_finds_a_configuration_close_to_the_exhaustive_best(shape)
     st, c = tdx.tdx_default_gemm_config(M, N, K, 0, tB, tdx.TDX_BF16)
     assert st == 0 and c.as_dict() == best.as_dict()
     assert tdx.tdx_tune_clear() == 0
+
+
+@pytest.mark.gpu
+def test_search_on_first_use_caches_the_winner_and_keeps_parity(tmp_path):
+    # tdx_set_autotune(budget): the first automatic call on an unknown bf16 shape runs the guided search and caches its
+    # winner; the result of that call and of the next one (served from the cache) match the oracle
+    import json
+    import numpy as np
+    import seeded_inputs as si
+    from gpu_util import TIGHT, gemm_error, run_gemm
+    M, N, K = 1152, 896, 640
+    key = f"gemm:{M}:{N}:{K}:0:1:{tdx.TDX_BF16}"
+    path = tmp_path / "cache.json"
+    assert tdx.tdx_tune_save(str(path)) == 0
+    assert key not in path.read_text()
+    A, B = si.gemm_bf16_normal(M, N, K, seed=95, transB=1)
+    assert tdx.tdx_set_autotune(6) == 0
+    try:
+        for _ in range(2):
+            st, C, ok = run_gemm(M, N, K, 0, 1, 1.0, "bf16", A, B)
+            assert st == 0 and ok, tdx.tdx_last_error()
+            assert gemm_error(M, N, K, 0, 1, 1.0, "bf16", A, B, C) < TIGHT["bf16"]
+    finally:
+        assert tdx.tdx_set_autotune(0) == 0
+    assert tdx.tdx_tune_save(str(path)) == 0
+    assert key in path.read_text()
