@@ -567,6 +567,7 @@ int ensure_pieces(DeviceCtx* ctx, int slot, size_t bytes, void** out) {
 }
 
 int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_count, int smem_limit, tdx_config* out);
+bool model_pick_direct_store(const GemmProblem& g, int sm_count, int smem_limit, tdx_config* out);
 
 constexpr size_t kPiecesMaxBytes = size_t(3) << 30;     // per operand; larger problems go batch by batch, or to the CUDA cores
 
@@ -607,6 +608,16 @@ int run_gemm_f32_pieces(DeviceCtx* ctx, const GemmProblem& g, float alpha, const
     want.kernel = TDX_KERNEL_UMMA;
     want.store_mode = 1;
     want.cta_pair = 1;          // split_k: the caller's, else chosen like for any GEMM with few tiles and a long reduction
+    if (ba.batch == 1 && want.tile_m == 0 && want.tile_n == 0 && want.split_k == 0 && want.stages == 0) {
+        // no tile given: the cost model's first choice among the direct-store candidates of the piece problem
+        tdx_config ranked;
+        if (model_pick_direct_store(gg, ctx->sm_count, ctx->smem_optin, &ranked)) {
+            want.tile_m = ranked.tile_m;
+            want.tile_n = ranked.tile_n;
+            want.split_k = ranked.split_k;
+            want.raster = ranked.raster;
+        }
+    }
     tdx_config cfg;
     rc = resolve_gemm_config(gg, &want, ctx->sm_count, ctx->smem_optin, &cfg);
     if (rc) return rc;

@@ -88,6 +88,35 @@ bool model_default_gemm(const GemmProblem& g, int sm_count, int smem_limit, tdx_
     return memo.found;
 }
 
+// The same ranking for a launch that stores directly from registers (the fp32 result of the bf16-piece GEMM): every
+// tile shape and split of the search space, judged as a direct-store, uniform-grid configuration.  Kept per shape.
+bool model_pick_direct_store(const GemmProblem& g, int sm_count, int smem_limit, tdx_config* out) {
+    typedef std::array<int64_t, 5> Key;
+    const Key key = {g.M, g.N, g.K, sm_count, smem_limit};
+    static std::mutex mu;
+    static std::map<Key, std::pair<bool, tdx_config>> cache;
+    std::lock_guard<std::mutex> lk(mu);
+    auto it = cache.find(key);
+    if (it == cache.end()) {
+        std::vector<tdx_config> cands;
+        enum_gemm(g, sm_count, smem_limit, &cands);
+        std::pair<bool, tdx_config> pick;
+        pick.first = false;
+        std::memset(&pick.second, 0, sizeof pick.second);
+        double best_us = 0.0;
+        for (tdx_config c : cands) {
+            if (c.cta_pair == 2 || c.k_stagger != 0) continue;
+            c.store_mode = 1;
+            c.fit = 1;
+            const double us = model_gemm_us(g, c, sm_count);
+            if (!pick.first || us < best_us) { pick.first = true; pick.second = c; best_us = us; }
+        }
+        it = cache.emplace(key, pick).first;
+    }
+    if (it->second.first) *out = it->second.second;
+    return it->second.first;
+}
+
 // Fill the zero fields of a (possibly partial) GEMM config and check it.  smem_limit / sm_count come from the
 // device when there is one, else from the sm_100 defaults, so the search space can be listed without a GPU.
 int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_count, int smem_limit, tdx_config* out) {
