@@ -91,8 +91,8 @@ bool model_default_gemm(const GemmProblem& g, int sm_count, int smem_limit, tdx_
 // The same ranking for a launch that stores directly from registers (the fp32 result of the bf16-piece GEMM): every
 // tile shape and split of the search space, judged as a direct-store, uniform-grid configuration.  Kept per shape.
 bool model_pick_direct_store(const GemmProblem& g, int sm_count, int smem_limit, tdx_config* out) {
-    typedef std::array<int64_t, 5> Key;
-    const Key key = {g.M, g.N, g.K, sm_count, smem_limit};
+    typedef std::array<int64_t, 7> Key;
+    const Key key = {g.M, g.N, g.K, g.transA, g.transB, sm_count, smem_limit};
     static std::mutex mu;
     static std::map<Key, std::pair<bool, tdx_config>> cache;
     std::lock_guard<std::mutex> lk(mu);
@@ -657,6 +657,13 @@ int tdx_gemm_f32out(int64_t M, int64_t N, int64_t K, int transA, int transB, flo
     want.kernel = TDX_KERNEL_UMMA;
     want.store_mode = 1;         // fp32 results leave through the direct-store epilogue (or the fp32 split-K reduction)
     want.cta_pair = 1;
+    tdx_config ranked;           // tile shape and K split: the cost model's first choice among the direct-store candidates
+    if (model_pick_direct_store(g, ctx->sm_count, ctx->smem_optin, &ranked)) {
+        want.tile_m = ranked.tile_m;
+        want.tile_n = ranked.tile_n;
+        want.split_k = ranked.split_k;
+        want.raster = ranked.raster;
+    }
     tdx_config cfg;
     rc = resolve_gemm_config(g, &want, ctx->sm_count, ctx->smem_optin, &cfg);
     if (rc) return rc;
