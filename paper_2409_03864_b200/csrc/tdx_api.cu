@@ -702,7 +702,17 @@ int tdx_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int transA,
     if (!aligned) return run_gemm_generic(ctx, g, alpha, A, B, C, st, ba);
     tdx_config want;
     std::memset(&want, 0, sizeof want);
-    if (beta != 0.0f) want.store_mode = 1;          // the accumulate term is read by the direct-store epilogue
+    if (beta != 0.0f) {
+        want.store_mode = 1;                        // the accumulate term is read by the direct-store epilogue
+        want.kernel = TDX_KERNEL_UMMA;
+        tdx_config ranked;                          // tile shape and K split: the cost model's direct-store choice
+        if (model_pick_direct_store(g, ctx->sm_count, ctx->smem_optin, &ranked)) {
+            want.tile_m = ranked.tile_m;
+            want.tile_n = ranked.tile_n;
+            want.split_k = ranked.split_k;
+            want.raster = ranked.raster;
+        }
+    }
     tdx_config cfg;
     rc = resolve_gemm_config(g, beta != 0.0f ? &want : nullptr, ctx->sm_count, ctx->smem_optin, &cfg);
     if (rc) return rc;
