@@ -164,7 +164,7 @@ int tdx_gemm_f32out(int64_t M, int64_t N, int64_t K, int transA, int transB, flo
 
 /*
  * Same as tdx_gemm with an explicit configuration and caller-owned split-K workspace.
- * cfg = NULL or cfg->split_k = 0: the library chooses split_k (tuning cache, else heuristic); then
+ * cfg = NULL or cfg->split_k = 0: the library chooses split_k (tuning cache, else the cost model's first-ranked candidate); then
  * `workspace` may be NULL and the library uses an internal, lazily grown buffer.  With an explicit
  * cfg->split_k > 1 the caller must pass at least tdx_gemm_workspace_size bytes (256-byte aligned)
  * -> else WORKSPACE.
@@ -269,7 +269,7 @@ int tdx_set_autotune(int budget);
 /*
  * Guided search: the candidates of tdx_tune_gemm are ranked by a host-side cost model (MMA time by tile width, L2
  * ingest, epilogue overlap, wave count or fitted plan, split-K traffic, HBM floor) and only the `budget` best-ranked
- * ones, plus the heuristic default, are timed on the device -- the model-guided counterpart of Case Study 5's
+ * ones, plus the automatic choice, are timed on the device -- the model-guided counterpart of Case Study 5's
  * search under constraints.  n_candidates (may be NULL) receives the size of the full search space.  bf16 GEMM;
  * other problems are searched exhaustively.  tdx_model_gemm_us evaluates the model for one configuration on
  * `ctas` SMs (host only).
@@ -280,7 +280,8 @@ int tdx_tune_gemm_guided(int64_t M, int64_t N, int64_t K, int transA, int transB
 int tdx_model_gemm_us(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const tdx_config* cfg, int ctas,
                       double* us);
 
-/* The configuration the automatic choice would use right now (tuning cache, else heuristic). */
+/* The configuration the automatic choice would use right now: the tuning cache's entry, else (bf16 GEMM on the
+ * tensor-core path) the candidate of the search space that the cost model ranks first, else a size heuristic. */
 int tdx_default_gemm_config(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, tdx_config* out);
 int tdx_default_conv2d_config(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S,
                               int pad, int stride, int dtype, tdx_config* out);

@@ -107,7 +107,7 @@ def lib() -> ctypes.CDLL:
                 fn.restype = ci
         _lib = L
         # Tuned tile configurations measured on B200 ship next to the library; TDX_TUNE_CACHE names another
-        # file, or "0" for none.  A missing or unreadable file only means the heuristic defaults are used.
+        # file, or "0" for none.  A missing or unreadable file only means the library's automatic choice is used.
         cache = os.environ.get("TDX_TUNE_CACHE", str(_LIB_PATH.parent / "tuned_b200.json"))
         if cache != "0" and os.path.exists(cache):
             L.tdx_tune_load(cache.encode())

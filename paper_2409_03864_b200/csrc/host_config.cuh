@@ -162,7 +162,8 @@ void choose_patch(int64_t P, int64_t Q, int* bw_out, int* bh_out, int stride = 1
     *bh_out = best_bh;
 }
 
-// Heuristic default (used when neither the caller nor the tuning cache gives a configuration).
+// Size heuristic: fills the fields a partial configuration leaves open, and is the automatic choice where the cost
+// model does not apply (convolutions, layouts off the tensor-core path).
 void default_umma_config(int64_t tiles_m, int64_t N, int64_t num_kb, bool b_mn_major, int sm_count, int smem_limit,
                          bool allow_split, tdx_config* c) {
     std::memset(c, 0, sizeof *c);

@@ -1066,7 +1066,7 @@ int tune_operand_sets(size_t bytes_per_set) {
 }
 
 // budget <= 0: every statically feasible candidate is timed; budget > 0: the candidates are ranked by the cost model and
-// only the `budget` best-ranked ones (plus the heuristic default) are timed
+// only the `budget` best-ranked ones (plus the automatic choice) are timed
 static int tune_gemm_impl(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, int iters, int budget,
                           tdx_config* best, float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried,
                           int* n_candidates, void* stream) {
