@@ -629,9 +629,16 @@ int run_gemm_f32_pieces(DeviceCtx* ctx, const GemmProblem& g, float alpha, const
     const float* a = static_cast<const float*>(A);
     const float* b = static_cast<const float*>(B);
     float* c = static_cast<float*>(C);
-    auto split = [&](const float* src, int rows, long long s_row, long long s_k, long long bstride, int64_t nb, void* dst) -> int {
-        dim3 grid(static_cast<unsigned>(ceil_div(Kp, 64)), static_cast<unsigned>(ceil_div(rows, 32)), static_cast<unsigned>(nb));
-        if (grid.y > 65535) return fail(TDX_ERR_UNSUPPORTED, "operand too tall for the piece kernel");
+    // one launch splits both operands (nb_b == 0: only the first)
+    auto split = [&](const float* src_a, int rows_a, long long s_row_a, long long s_k_a, long long bstride_a, int64_t nb_a, void* dst_a,
+                     const float* src_b, int rows_b, long long s_row_b, long long s_k_b, long long bstride_b, int64_t nb_b,
+                     void* dst_b) -> int {
+        const int rows_max = nb_b > 0 ? std::max(rows_a, rows_b) : rows_a;
+        dim3 grid(static_cast<unsigned>(ceil_div(Kp, 64)), static_cast<unsigned>(ceil_div(rows_max, 32)),
+                  static_cast<unsigned>(nb_a + nb_b));
+        if (grid.y > 65535 || nb_a + nb_b > 65535) return fail(TDX_ERR_UNSUPPORTED, "operand too tall for the piece kernel");
+        tdx::SplitOperand o0{rows_a, s_row_a, s_k_a, bstride_a, src_a, static_cast<__nv_bfloat16*>(dst_a)};
+        tdx::SplitOperand o1{rows_b, s_row_b, s_k_b, bstride_b, src_b, static_cast<__nv_bfloat16*>(dst_b)};
         cudaLaunchConfig_t lc;
         std::memset(&lc, 0, sizeof lc);
         lc.gridDim = grid;
@@ -642,18 +649,27 @@ int run_gemm_f32_pieces(DeviceCtx* ctx, const GemmProblem& g, float alpha, const
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         lc.attrs = attr;
         lc.numAttrs = 1;
-        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::split_f32_bf16x3_kernel, rows, static_cast<int>(g.K), static_cast<int>(Kp), s_row,
-                                    s_k, bstride, src, static_cast<__nv_bfloat16*>(dst)));
+        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::split_f32_bf16x3_kernel, static_cast<int>(g.K), static_cast<int>(Kp),
+                                    static_cast<int>(nb_a), o0, o1));
         TDX_CUDA(cudaGetLastError());
         g_launches.fetch_add(1);
         return TDX_OK;
     };
     for (int64_t b0 = 0; b0 < ba.batch; b0 += chunk) {
         const int64_t nb = std::min(chunk, ba.batch - b0);
-        if (!a_shared || b0 == 0)
-            if ((rc = split(a + (a_shared ? 0 : b0 * ba.stride_a), static_cast<int>(g.M), sa_i, sa_k, ba.stride_a, a_shared ? 1 : nb, pa))) return rc;
-        if (!b_shared || b0 == 0)     // B'' rows are the columns j of op(B): element (j, k) at B[k * sb_k + j * sb_j]
-            if ((rc = split(b + (b_shared ? 0 : b0 * ba.stride_b), static_cast<int>(g.N), sb_j, sb_k, ba.stride_b, b_shared ? 1 : nb, pb))) return rc;
+        // B'' rows are the columns j of op(B): element (j, k) at B[k * sb_k + j * sb_j]
+        const bool do_a = !a_shared || b0 == 0, do_b = !b_shared || b0 == 0;
+        const float* src_a = a + (a_shared ? 0 : b0 * ba.stride_a);
+        const float* src_b = b + (b_shared ? 0 : b0 * ba.stride_b);
+        const int64_t nb_a = a_shared ? 1 : nb, nb_b = b_shared ? 1 : nb;
+        if (do_a && do_b) {
+            if ((rc = split(src_a, static_cast<int>(g.M), sa_i, sa_k, ba.stride_a, nb_a, pa,
+                            src_b, static_cast<int>(g.N), sb_j, sb_k, ba.stride_b, nb_b, pb))) return rc;
+        } else if (do_a) {
+            if ((rc = split(src_a, static_cast<int>(g.M), sa_i, sa_k, ba.stride_a, nb_a, pa, nullptr, 0, 0, 0, 0, 0, nullptr))) return rc;
+        } else if (do_b) {
+            if ((rc = split(src_b, static_cast<int>(g.N), sb_j, sb_k, ba.stride_b, nb_b, pb, nullptr, 0, 0, 0, 0, 0, nullptr))) return rc;
+        }
         if (nb > 1 && !a_shared && !b_shared) {
             // all batches of the chunk in one launch: 3-D operands, items over batch x tiles x splits
             PieceInfo pb_info = pi;

@@ -542,17 +542,30 @@ __global__ void splitk_reduce_f32_kernel(long long MN, int split, const float* _
 // is 1; a thread issues its eight loads back to back and writes pairs of pieces (4-byte stores, whole 128-byte lines
 // per warp).
 // ---------------------------------------------------------------------------
+// One launch may split two operands (A and B of a GEMM): blockIdx.z below `nb0` works on the first, the rest on the
+// second; an operand with fewer 32-row blocks than the grid has lets the surplus CTAs leave at once.
+struct SplitOperand {
+    int rows;
+    long long s_row, s_k, batch_stride;
+    const float* src;
+    __nv_bfloat16* dst;
+};
 __global__ void __launch_bounds__(256)
-split_f32_bf16x3_kernel(int rows, int K, int Kp, long long s_row, long long s_k, long long batch_stride,
-                        const float* __restrict__ src, __nv_bfloat16* __restrict__ dst) {
+split_f32_bf16x3_kernel(int K, int Kp, int nb0, SplitOperand op0, SplitOperand op1) {
     __shared__ float tile[32][65];
+    const bool second = static_cast<int>(blockIdx.z) >= nb0;
+    const SplitOperand& op = second ? op1 : op0;
+    const int rows = op.rows;
+    const long long s_row = op.s_row, s_k = op.s_k;
+    const int bz = static_cast<int>(blockIdx.z) - (second ? nb0 : 0);
     // launched with programmatic stream serialization (see sgemm_small_rowmajor_kernel): the piece buffers are shared
     // by successive calls, and the wait orders this kernel after everything the stream held before it
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const int k0 = blockIdx.x * 64, r0 = blockIdx.y * 32;
-    const float* s = src + blockIdx.z * batch_stride;
-    __nv_bfloat16* d = dst + static_cast<long long>(blockIdx.z) * rows * 3 * Kp;
+    if (r0 >= rows) return;                           // CTA-uniform: before any barrier
+    const float* s = op.src + bz * op.batch_stride;
+    __nv_bfloat16* d = op.dst + static_cast<long long>(bz) * rows * 3 * Kp;
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;        // 32 x 8 threads
     if (s_k == 1) {
 #pragma unroll
