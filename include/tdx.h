@@ -92,8 +92,9 @@ typedef struct {
     int fit;        /* GEMM, split_k = 1, tile_n >= 192 (CTA pairs: transB = 1 only): 2 = some row blocks are cut into narrower tiles */
                     /*     (multiples of 64 columns) so that all CTAs finish together when the uniform grid  */
                     /*     would leave the last wave of CTAs partly idle; 1 = uniform grid; 0 = fitted when  */
-                    /*     the cost model predicts a gain of at least 3 %.  The first call for a shape       */
-                    /*     allocates and uploads a small tile table (make it before any stream capture).     */
+                    /*     the cost model predicts a gain of at least 3 %.  The first call for a shape on a  */
+                    /*     device allocates a small tile table there and copies it synchronously (cudaMalloc */
+                    /*     + cudaMemcpy): make that call before any stream capture.                          */
 } tdx_config;
 
 /*
@@ -218,7 +219,8 @@ int tdx_conv2d_bias_relu_ex(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_
  * tdx_conv2d_bias_relu_host: groups of images): chunk i goes up on a copy stream owned by the
  * library while chunk i - 1 is computed on `stream` and chunk i - 2 comes down on a second copy
  * stream, ordered by events, so the two directions of the bus and the kernels overlap.  Each
- * output element is computed as in one call over the whole problem.  The host buffers must stay
+ * output element is the same sum of products as in one call over the whole problem; the tile shape
+ * and K split are chosen per chunk, so its fp32 summation order may differ.  The host buffers must stay
  * valid and unmodified until the call returns (it returns only when all three streams are idle).
  */
 int tdx_gemm_host(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype,
@@ -241,6 +243,10 @@ int tdx_conv2d_bias_relu_host(int64_t N, int64_t H, int64_t W, int64_t Cin, int6
  * returns the fastest and records it in the in-process tuning cache used by the automatic choice.
  *   iters: timed launches per candidate (>= 1).  best / best_us: outputs (best_us = mean microseconds).
  *   tried / tried_us / cap / n_tried: optional (NULL / 0) list of every candidate with its time.
+ * Before a winner is cached its output is checked on the device against the one-thread-per-output kernel's on the
+ * same scratch operands (GEMM: up to 16 blocks of 128 rows spread over M; convolution: the whole output), and a
+ * candidate whose kernel reported a bounded wait that ran out is dropped; if the fastest candidates all fail that
+ * check the call returns UNSUPPORTED and caches nothing.
  */
 int tdx_tune_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, int iters,
                   tdx_config* best, float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried,

@@ -177,7 +177,7 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     int plan_grid = 0;
     if (cfg.fit != 1 && cfg.split_k == 1 && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0 && nbatch == 1) {
         DevicePlan dp;
-        rc = get_tile_plan(ctx, g.M, g.N, num_kb, cfg.tile_m, cfg.tile_n, cfg.raster, cfg.fit == 2 ? 0.0 : 0.03, st, &dp);
+        rc = get_tile_plan(ctx, g.M, g.N, num_kb, cfg.tile_m, cfg.tile_n, cfg.raster, cfg.fit == 2 ? 0.0 : 0.03, &dp);
         if (rc) return rc;
         if (dp.fitted) {
             p.tiles = dp.dev;
@@ -297,7 +297,7 @@ int run_gemm_pair(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     // only on request: a 256 x 128 x 16 pair MMA measured 115 cycles, not 64, so narrow tiles gain nothing here
     if (cfg.fit == 2 && !p.b_mn_major && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0) {
         DevicePlan dp;
-        rc = get_tile_plan(ctx, g.M, g.N, num_kb, 256, cfg.tile_n, cfg.raster, 0.0, st, &dp, true);
+        rc = get_tile_plan(ctx, g.M, g.N, num_kb, 256, cfg.tile_n, cfg.raster, 0.0, &dp, true);
         if (rc) return rc;
         if (dp.fitted) {
             p.tiles = dp.dev;
@@ -426,7 +426,7 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     if (halo && !p.b_resident && cfg.fit != 1 && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0) {
         DevicePlan dp;
         int rcp = get_tile_plan(ctx, static_cast<int64_t>(p.tiles_m) * cfg.tile_m, c.Cout, p.num_kb, cfg.tile_m, cfg.tile_n,
-                                cfg.raster, cfg.fit == 2 ? 0.0 : 0.03, st, &dp);
+                                cfg.raster, cfg.fit == 2 ? 0.0 : 0.03, &dp);
         if (rcp) return rcp;
         if (dp.fitted) {
             p.tiles = dp.dev;

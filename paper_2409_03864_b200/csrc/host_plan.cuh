@@ -131,21 +131,23 @@ bool plan_fitted_tiles(int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int
     return true;
 }
 
-// Device copies of tile plans, one per (shape, tile, CTA count); never freed (a few KB each).
+// Device copies of tile plans, one per (device, shape, tile, CTA count); never freed (a few KB each).
 struct PlanKey {
     int64_t M, N, num_kb;
-    int bm, bn, raster, g, forced, pair;
+    int dev, bm, bn, raster, g, forced, pair;
     bool operator<(const PlanKey& o) const { return std::memcmp(this, &o, sizeof(PlanKey)) < 0; }
 };
 struct DevicePlan { int4* dev = nullptr; int rounds = 0, grid = 0; bool fitted = false; };
 std::map<PlanKey, DevicePlan> g_plans;
 
-// Looks the plan up (building and uploading it on first use; the upload is ordered on `st` before the kernel).
+// Looks the plan up.  First use of a shape on a device builds the plan, allocates its table on that device and
+// copies it there synchronously (cudaMalloc + cudaMemcpy: not legal inside a stream capture, so a captured
+// call must have been preceded by an eager one for the same shape).
 int get_tile_plan(DeviceCtx* ctx, int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int raster, double min_gain,
-                  cudaStream_t st, DevicePlan* out, bool pair = false) {
+                  DevicePlan* out, bool pair = false) {
     PlanKey key;
     std::memset(&key, 0, sizeof key);
-    key.M = M; key.N = N; key.num_kb = num_kb; key.bm = bm; key.bn = bn; key.raster = raster; key.g = pair ? ctx->sm_count / 2 : ctx->sm_count; key.forced = min_gain <= 0.0 ? 1 : 0;
+    key.M = M; key.N = N; key.num_kb = num_kb; key.dev = ctx->dev; key.bm = bm; key.bn = bn; key.raster = raster; key.g = pair ? ctx->sm_count / 2 : ctx->sm_count; key.forced = min_gain <= 0.0 ? 1 : 0;
     key.pair = pair ? 1 : 0;
     {
         std::lock_guard<std::mutex> lk(g_mu);
@@ -159,13 +161,12 @@ int get_tile_plan(DeviceCtx* ctx, int64_t M, int64_t N, int64_t num_kb, int bm, 
         const size_t bytes = plan.table.size() * sizeof(int4);
         void* dev = nullptr;
         TDX_CUDA(cudaMalloc(&dev, bytes));
-        // the table is a std::vector about to go out of scope: copy synchronously (once per shape)
+        // the table is a std::vector about to go out of scope: copy synchronously (once per shape and device)
         TDX_CUDA(cudaMemcpy(dev, plan.table.data(), bytes, cudaMemcpyHostToDevice));
         d.dev = static_cast<int4*>(dev);
         d.rounds = plan.rounds;
         d.grid = plan.grid;
     }
-    (void)st;
     {
         std::lock_guard<std::mutex> lk(g_mu);
         g_plans[key] = d;

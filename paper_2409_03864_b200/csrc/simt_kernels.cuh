@@ -604,6 +604,32 @@ split_f32_bf16x3_kernel(int K, int Kp, int nb0, SplitOperand op0, SplitOperand o
     }
 }
 
+// max |a - b| and max |b| over n bf16 values -> out[0], out[1] as fp32 bit patterns (non-negative floats order like
+// unsigned integers, so atomicMax works on them; a NaN becomes +inf's pattern).  Used by the search to check a
+// winner's output against the generic kernel's.
+__global__ void max_diff_bf16_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ b, long long n,
+                                     unsigned* out) {
+    float d = 0.0f, m = 0.0f;
+    for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < n;
+         e += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const float x = __bfloat162float(a[e]), y = __bfloat162float(b[e]);
+        float dd = fabsf(x - y), mm = fabsf(y);
+        if (!(dd == dd)) dd = __int_as_float(0x7f800000);
+        if (!(mm == mm)) mm = __int_as_float(0x7f800000);
+        d = fmaxf(d, dd);
+        m = fmaxf(m, mm);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        d = fmaxf(d, __shfl_xor_sync(0xffffffffu, d, o));
+        m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    }
+    if ((threadIdx.x & 31) == 0) {
+        atomicMax(out, __float_as_uint(d));
+        atomicMax(out + 1, __float_as_uint(m));
+    }
+}
+
 // Deterministic pseudo-random fill used only by the tuner's scratch operands.
 __global__ void fill_pattern_bf16_kernel(__nv_bfloat16* p, long long n, uint32_t seed) {
     for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < n;

@@ -541,16 +541,38 @@ int fill_scratch(void* p, size_t elems, uint32_t seed, cudaStream_t st) {
     return TDX_OK;
 }
 
+// Reads and clears the device status word (the stream must be idle).  Returns the code a kernel left there, 0 if none.
+int take_device_status(DeviceCtx* ctx, int* code) {
+    int v = 0;
+    TDX_CUDA(cudaMemcpy(&v, ctx->status_ptr, sizeof v, cudaMemcpyDeviceToHost));
+    if (v != 0) TDX_CUDA(cudaMemset(ctx->status_ptr, 0, sizeof v));
+    *code = v;
+    return TDX_OK;
+}
+
+// The search's own check of a winner before it is cached: a candidate that is fast but wrong must not become the
+// configuration plain calls are served with.  `verify(cfg, &ok)` runs the configuration once more and compares its
+// output on the device with the one-thread-per-output kernel's on the same scratch operands.
+typedef std::function<int(const tdx_config&, bool*)> VerifyFn;
+
 template <typename Launch>
-int time_candidates(const std::vector<tdx_config>& cands, int iters, cudaStream_t st, Launch&& launch, tdx_config* best,
-                    float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried) {
+int time_candidates(DeviceCtx* ctx, const std::vector<tdx_config>& cands, int iters, cudaStream_t st, Launch&& launch,
+                    const VerifyFn& verify, tdx_config* best, float* best_us, tdx_config* tried, float* tried_us, int cap,
+                    int* n_tried) {
+    // a status an earlier kernel of the caller left behind is the caller's to collect (tdx_check_device_status):
+    // then the search neither reads candidates' statuses off it nor clears it
+    TDX_CUDA(cudaStreamSynchronize(st));
+    int earlier = 0;
+    TDX_CUDA(cudaMemcpy(&earlier, ctx->status_ptr, sizeof earlier, cudaMemcpyDeviceToHost));
+    const bool watch_status = earlier == 0;
     cudaEvent_t e0, e1;
     TDX_CUDA(cudaEventCreate(&e0));
     TDX_CUDA(cudaEventCreate(&e1));
-    float best_t = -1.0f;
+    std::vector<std::pair<float, size_t>> timed;     // (microseconds, index into cands)
     int count = 0;
     int rc = TDX_OK;
-    for (const tdx_config& c : cands) {
+    for (size_t ci = 0; ci < cands.size(); ++ci) {
+        const tdx_config& c = cands[ci];
         rc = launch(c);              // warm-up (also validates the configuration)
         if (rc == TDX_ERR_CONFIG || rc == TDX_ERR_WORKSPACE) { rc = TDX_OK; continue; }
         if (rc) break;
@@ -562,19 +584,59 @@ int time_candidates(const std::vector<tdx_config>& cands, int iters, cudaStream_
         if (rc) break;
         cudaError_t e = cudaEventSynchronize(e1);
         if (e != cudaSuccess) { rc = fail(TDX_ERR_CUDA, "tuning launch failed: %s", cudaGetErrorString(e)); break; }
+        // a candidate whose kernel gave up on a bounded wait is not merely slow: its output is unspecified
+        int code = 0;
+        if (watch_status && (rc = take_device_status(ctx, &code))) break;
+        if (code != 0) continue;
         float ms = 0.0f;
         cudaEventElapsedTime(&ms, e0, e1);
         const float us = ms * 1000.0f / iters;
         if (tried && tried_us && count < cap) { tried[count] = c; tried_us[count] = us; }
         ++count;
-        if (best_t < 0 || us < best_t) { best_t = us; *best = c; }
+        timed.push_back({us, ci});
     }
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
     if (rc) return rc;
-    if (best_t < 0) return fail(TDX_ERR_UNSUPPORTED, "no feasible configuration");
-    if (best_us) *best_us = best_t;
-    if (n_tried) *n_tried = count;
+    if (timed.empty()) return fail(TDX_ERR_UNSUPPORTED, "no feasible configuration");
+    std::stable_sort(timed.begin(), timed.end());
+    // fastest first; the first one whose output checks out wins (a handful of attempts at most)
+    for (size_t i = 0; i < timed.size() && i < 4; ++i) {
+        bool ok = true;
+        if (verify) {
+            rc = verify(cands[timed[i].second], &ok);
+            if (rc) return rc;
+            int code = 0;
+            if (watch_status && (rc = take_device_status(ctx, &code))) return rc;
+            if (code != 0) ok = false;
+        }
+        if (!ok) continue;
+        *best = cands[timed[i].second];
+        if (best_us) *best_us = timed[i].first;
+        if (n_tried) *n_tried = count;
+        return TDX_OK;
+    }
+    return fail(TDX_ERR_UNSUPPORTED, "the fastest candidates failed the output check against the generic kernel");
+}
+
+// max |a - b| and max |b| over n bf16 values, as the bit patterns of non-negative floats (which order like integers)
+int compare_on_device(const void* a, const void* b, long long n, unsigned* d_out2, cudaStream_t st, bool* ok) {
+    TDX_CUDA(cudaMemsetAsync(d_out2, 0, 2 * sizeof(unsigned), st));
+    const int grid = static_cast<int>(std::min<long long>(ceil_div(n, 256 * 8), 148LL * 8));
+    tdx::max_diff_bf16_kernel<<<std::max(grid, 1), 256, 0, st>>>(static_cast<const __nv_bfloat16*>(a),
+                                                                static_cast<const __nv_bfloat16*>(b), n, d_out2);
+    TDX_CUDA(cudaGetLastError());
+    g_launches.fetch_add(1);
+    unsigned h[2] = {0, 0};
+    TDX_CUDA(cudaMemcpyAsync(h, d_out2, sizeof h, cudaMemcpyDeviceToHost, st));
+    TDX_CUDA(cudaStreamSynchronize(st));
+    float diff, ref;
+    std::memcpy(&diff, &h[0], 4);
+    std::memcpy(&ref, &h[1], 4);
+    // two correct bf16 results differ by one rounding step of the larger (2^-8 relative) plus fp32 summation-order
+    // noise; a misplaced tile, a dropped K block or a wrong column differs by a sizeable part of the largest value.
+    // A NaN anywhere was mapped to the largest pattern by the kernel and fails the test.
+    *ok = std::isfinite(diff) && std::isfinite(ref) && diff <= 0.02f * ref + 1e-30f;
     return TDX_OK;
 }
 
@@ -624,6 +686,15 @@ int drain_host_pipe(DeviceCtx* ctx, cudaStream_t st, int rc) {
     cudaStreamSynchronize(ctx->d2h);
     return rc;
 }
+
+// Inside the chunked loops: a failed CUDA call must not return while the helper streams may still be copying from or to
+// the caller's host buffers.
+#define TDX_CUDA_PIPE(expr)                                                                                              \
+    do {                                                                                                                 \
+        cudaError_t e_ = (expr);                                                                                         \
+        if (e_ != cudaSuccess)                                                                                           \
+            return drain_host_pipe(ctx, st, fail(TDX_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_)));         \
+    } while (0)
 
 }  // namespace
 
@@ -845,39 +916,40 @@ int tdx_gemm_host(int64_t M, int64_t N, int64_t K, int transA, int transB, float
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // Row-major A: the rows are cut into chunks; chunk i's rows of A go up on one stream while chunk i - 1 is
     // multiplied on the caller's stream and chunk i - 2's rows of C come down on a third, so the two directions of
-    // the bus and the kernels overlap.  Every row of C is computed exactly as in one call over all rows.
+    // the bus and the kernels overlap.  Every element of C is the same sum of products as in one call over all rows; the
+    // tile shape and K split are chosen per chunk, so the fp32 summation order (the low-order bits) may differ from it.
     const int chunks = (transA == 0 && K > 0) ? host_chunk_count(M, 512, a_bytes + c_bytes) : 1;
     if (chunks > 1) {
         if ((rc = ensure_host_pipe(ctx))) return rc;
         const int64_t rows_per = ceil_div(ceil_div(M, chunks), 256) * 256;
         TDX_CUDA(cudaEventRecord(ctx->ev_start, st));
-        TDX_CUDA(cudaStreamWaitEvent(ctx->h2d, ctx->ev_start, 0));
-        TDX_CUDA(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, ctx->h2d));
+        TDX_CUDA_PIPE(cudaStreamWaitEvent(ctx->h2d, ctx->ev_start, 0));
+        TDX_CUDA_PIPE(cudaMemcpyAsync(dB, B_host, b_bytes, cudaMemcpyHostToDevice, ctx->h2d));
         int used = 0;
         for (int i = 0; i < chunks; ++i) {
             const int64_t r0 = i * rows_per, rows = std::min(rows_per, M - r0);
             if (rows <= 0) break;
             const size_t off = static_cast<size_t>(r0) * K * el;
-            TDX_CUDA(cudaMemcpyAsync(static_cast<char*>(dA) + off, static_cast<const char*>(A_host) + off,
+            TDX_CUDA_PIPE(cudaMemcpyAsync(static_cast<char*>(dA) + off, static_cast<const char*>(A_host) + off,
                                      static_cast<size_t>(rows) * K * el, cudaMemcpyHostToDevice, ctx->h2d));
-            TDX_CUDA(cudaEventRecord(ctx->ev_in[i], ctx->h2d));
+            TDX_CUDA_PIPE(cudaEventRecord(ctx->ev_in[i], ctx->h2d));
             used = i + 1;
         }
         for (int i = 0; i < used; ++i) {
             const int64_t r0 = i * rows_per, rows = std::min(rows_per, M - r0);
             const size_t a_off = static_cast<size_t>(r0) * K * el, c_off = static_cast<size_t>(r0) * N * el;
-            TDX_CUDA(cudaStreamWaitEvent(st, ctx->ev_in[i], 0));
+            TDX_CUDA_PIPE(cudaStreamWaitEvent(st, ctx->ev_in[i], 0));
             rc = gemm_dispatch(rows, N, K, transA, transB, alpha, dtype, static_cast<char*>(dA) + a_off, dB,
                                static_cast<char*>(dC) + c_off, stream, nullptr, nullptr, 0, true);
             if (rc) return drain_host_pipe(ctx, st, rc);
-            TDX_CUDA(cudaEventRecord(ctx->ev_out[i], st));
-            TDX_CUDA(cudaStreamWaitEvent(ctx->d2h, ctx->ev_out[i], 0));
-            TDX_CUDA(cudaMemcpyAsync(static_cast<char*>(C_host) + c_off, static_cast<char*>(dC) + c_off,
+            TDX_CUDA_PIPE(cudaEventRecord(ctx->ev_out[i], st));
+            TDX_CUDA_PIPE(cudaStreamWaitEvent(ctx->d2h, ctx->ev_out[i], 0));
+            TDX_CUDA_PIPE(cudaMemcpyAsync(static_cast<char*>(C_host) + c_off, static_cast<char*>(dC) + c_off,
                                      static_cast<size_t>(rows) * N * el, cudaMemcpyDeviceToHost, ctx->d2h));
         }
-        TDX_CUDA(cudaEventRecord(ctx->ev_done, ctx->d2h));
-        TDX_CUDA(cudaStreamWaitEvent(st, ctx->ev_done, 0));
-        TDX_CUDA(cudaStreamSynchronize(st));
+        TDX_CUDA_PIPE(cudaEventRecord(ctx->ev_done, ctx->d2h));
+        TDX_CUDA_PIPE(cudaStreamWaitEvent(st, ctx->ev_done, 0));
+        TDX_CUDA_PIPE(cudaStreamSynchronize(st));
         return TDX_OK;
     }
     if (a_bytes) TDX_CUDA(cudaMemcpyAsync(dA, A_host, a_bytes, cudaMemcpyHostToDevice, st));
@@ -969,32 +1041,32 @@ int tdx_conv2d_bias_relu_host(int64_t N, int64_t H, int64_t W, int64_t Cin, int6
         const int64_t per = ceil_div(N, chunks);
         const size_t x_img = static_cast<size_t>(H) * W * Cin * el, y_img = static_cast<size_t>(cp.P) * cp.Q * Cout * el;
         TDX_CUDA(cudaEventRecord(ctx->ev_start, st));
-        TDX_CUDA(cudaStreamWaitEvent(ctx->h2d, ctx->ev_start, 0));
-        TDX_CUDA(cudaMemcpyAsync(dw, w_host, w_bytes, cudaMemcpyHostToDevice, ctx->h2d));
-        if (bias_host) TDX_CUDA(cudaMemcpyAsync(db, bias_host, b_bytes, cudaMemcpyHostToDevice, ctx->h2d));
+        TDX_CUDA_PIPE(cudaStreamWaitEvent(ctx->h2d, ctx->ev_start, 0));
+        TDX_CUDA_PIPE(cudaMemcpyAsync(dw, w_host, w_bytes, cudaMemcpyHostToDevice, ctx->h2d));
+        if (bias_host) TDX_CUDA_PIPE(cudaMemcpyAsync(db, bias_host, b_bytes, cudaMemcpyHostToDevice, ctx->h2d));
         int used = 0;
         for (int i = 0; i < chunks; ++i) {
             const int64_t n0 = i * per, imgs = std::min(per, N - n0);
             if (imgs <= 0) break;
-            TDX_CUDA(cudaMemcpyAsync(static_cast<char*>(dx) + n0 * x_img, static_cast<const char*>(x_host) + n0 * x_img,
+            TDX_CUDA_PIPE(cudaMemcpyAsync(static_cast<char*>(dx) + n0 * x_img, static_cast<const char*>(x_host) + n0 * x_img,
                                      imgs * x_img, cudaMemcpyHostToDevice, ctx->h2d));
-            TDX_CUDA(cudaEventRecord(ctx->ev_in[i], ctx->h2d));
+            TDX_CUDA_PIPE(cudaEventRecord(ctx->ev_in[i], ctx->h2d));
             used = i + 1;
         }
         for (int i = 0; i < used; ++i) {
             const int64_t n0 = i * per, imgs = std::min(per, N - n0);
-            TDX_CUDA(cudaStreamWaitEvent(st, ctx->ev_in[i], 0));
+            TDX_CUDA_PIPE(cudaStreamWaitEvent(st, ctx->ev_in[i], 0));
             rc = conv_dispatch(imgs, H, W, Cin, Cout, R, S, pad, stride, dtype, static_cast<char*>(dx) + n0 * x_img, dw,
                                static_cast<const float*>(db), relu, static_cast<char*>(dy) + n0 * y_img, stream, nullptr);
             if (rc) return drain_host_pipe(ctx, st, rc);
-            TDX_CUDA(cudaEventRecord(ctx->ev_out[i], st));
-            TDX_CUDA(cudaStreamWaitEvent(ctx->d2h, ctx->ev_out[i], 0));
-            TDX_CUDA(cudaMemcpyAsync(static_cast<char*>(y_host) + n0 * y_img, static_cast<char*>(dy) + n0 * y_img, imgs * y_img,
+            TDX_CUDA_PIPE(cudaEventRecord(ctx->ev_out[i], st));
+            TDX_CUDA_PIPE(cudaStreamWaitEvent(ctx->d2h, ctx->ev_out[i], 0));
+            TDX_CUDA_PIPE(cudaMemcpyAsync(static_cast<char*>(y_host) + n0 * y_img, static_cast<char*>(dy) + n0 * y_img, imgs * y_img,
                                      cudaMemcpyDeviceToHost, ctx->d2h));
         }
-        TDX_CUDA(cudaEventRecord(ctx->ev_done, ctx->d2h));
-        TDX_CUDA(cudaStreamWaitEvent(st, ctx->ev_done, 0));
-        TDX_CUDA(cudaStreamSynchronize(st));
+        TDX_CUDA_PIPE(cudaEventRecord(ctx->ev_done, ctx->d2h));
+        TDX_CUDA_PIPE(cudaStreamWaitEvent(st, ctx->ev_done, 0));
+        TDX_CUDA_PIPE(cudaStreamSynchronize(st));
         return TDX_OK;
     }
     if (x_bytes) TDX_CUDA(cudaMemcpyAsync(dx, x_host, x_bytes, cudaMemcpyHostToDevice, st));
@@ -1130,7 +1202,41 @@ static int tune_gemm_impl(int64_t M, int64_t N, int64_t K, int transA, int trans
         const int i = turn++ % nsets;
         return gemm_dispatch(M, N, K, transA, transB, 1.0f, dtype, As[i], Bs[i], C, stream, &c, ws, ws_bytes, false);
     };
-    rc = time_candidates(cands, iters, st, launch, best, best_us, tried, tried_us, cap, n_tried);
+    // Output check of a would-be winner (bf16 tensor-core candidates): up to 16 blocks of 128 rows spread over M, all
+    // columns, recomputed by the generic kernel on the first operand set.
+    VerifyFn verify;
+    void *Cref = nullptr, *d_cmp = nullptr;
+    const int64_t vblock = 128, vblocks = std::min<int64_t>(16, ceil_div(M, vblock));
+    if (dtype == TDX_BF16 && !cands.empty() && cands[0].kernel == TDX_KERNEL_UMMA) {
+        if ((rc = guard.alloc(&Cref, static_cast<size_t>(vblock) * N * 2))) return rc;
+        if ((rc = guard.alloc(&d_cmp, 2 * sizeof(unsigned)))) return rc;
+        verify = [&](const tdx_config& c, bool* ok) -> int {
+            int r = gemm_dispatch(M, N, K, transA, transB, 1.0f, dtype, As[0], Bs[0], C, stream, &c, ws, ws_bytes, false);
+            if (r) return r;
+            const int64_t nblk = ceil_div(M, vblock);
+            *ok = true;
+            for (int64_t v = 0; v < vblocks && *ok; ++v) {
+                const int64_t blk = vblocks == 1 ? 0 : v * (nblk - 1) / (vblocks - 1);
+                const int64_t i0 = blk * vblock, rows = std::min(vblock, M - i0);
+                GemmProblem sub{rows, N, K, transA, transB, dtype};
+                // rows i0.. of op(A): A is M x K (row i at i * K) or K x M (row i at column i, pitch M)
+                const char* a_sub = static_cast<const char*>(As[0]) + (transA ? i0 : i0 * K) * 2;
+                long long sa_i, sa_k, sb_k, sb_j;
+                gemm_strides(GemmProblem{M, N, K, transA, transB, dtype}, &sa_i, &sa_k, &sb_k, &sb_j);
+                const long long total = rows * N;
+                const int grid = static_cast<int>(std::min<long long>(ceil_div(total, 256), static_cast<long long>(ctx->sm_count) * 32));
+                tdx::gemm_generic_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
+                    sub.M, N, K, sa_i, sa_k, sb_k, sb_j, 1.0f, reinterpret_cast<const __nv_bfloat16*>(a_sub),
+                    static_cast<const __nv_bfloat16*>(Bs[0]), static_cast<__nv_bfloat16*>(Cref));
+                TDX_CUDA(cudaGetLastError());
+                g_launches.fetch_add(1);
+                r = compare_on_device(static_cast<const char*>(C) + i0 * N * 2, Cref, total, static_cast<unsigned*>(d_cmp), st, ok);
+                if (r) return r;
+            }
+            return TDX_OK;
+        };
+    }
+    rc = time_candidates(ctx, cands, iters, st, launch, verify, best, best_us, tried, tried_us, cap, n_tried);
     cudaStreamSynchronize(st);
     if (rc) return rc;
     {
@@ -1208,7 +1314,23 @@ int tdx_tune_conv2d(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, 
         const int i = turn++ % nsets;
         return conv_dispatch(N, H, W, Cin, Cout, R, S, pad, stride, dtype, xs[i], w, static_cast<const float*>(b), 1, ys[i], stream, &c);
     };
-    rc = time_candidates(cands, iters, st, launch, best, best_us, tried, tried_us, cap, n_tried);
+    // Output check of a would-be winner: the whole output of the first operand set against the generic kernel's.
+    VerifyFn verify;
+    void *yref = nullptr, *d_cmp = nullptr;
+    if (dtype == TDX_BF16 && !cands.empty() && cands[0].kernel == TDX_KERNEL_UMMA) {
+        if ((rc = guard.alloc(&yref, y_bytes))) return rc;
+        if ((rc = guard.alloc(&d_cmp, 2 * sizeof(unsigned)))) return rc;
+        verify = [&](const tdx_config& c, bool* ok) -> int {
+            int r = conv_dispatch(N, H, W, Cin, Cout, R, S, pad, stride, dtype, xs[0], w, static_cast<const float*>(b), 1, ys[0], stream, &c);
+            if (r) return r;
+            r = run_conv_generic(ctx, cp, xs[0], w, static_cast<const float*>(b), 1, yref, st);
+            if (r) return r;
+            r = compare_on_device(ys[0], yref, static_cast<long long>(y_bytes / 2), static_cast<unsigned*>(d_cmp), st, ok);
+            if (r) return r;
+            return TDX_OK;
+        };
+    }
+    rc = time_candidates(ctx, cands, iters, st, launch, verify, best, best_us, tried, tried_us, cap, n_tried);
     cudaStreamSynchronize(st);
     if (rc) return rc;
     {
@@ -1396,7 +1518,7 @@ int tdx_gemm_splitk_static(int64_t M, int64_t N, int64_t K, int transA, int tran
     if (split_k < 1 || tile_n < 0) return fail(TDX_ERR_INVALID_ARG, "split_k must be >= 1 and tile_n >= 0");
     if (M == 0 || N == 0) return TDX_OK;
     if (K == 0) return fail(TDX_ERR_UNSUPPORTED, "K = 0: use tdx_gemm");
-    // size check first: it needs no device
+    // the size limit is checked on the host, before anything is looked up or launched
     const double need = static_cast<double>(split_k) * static_cast<double>(M) * static_cast<double>(N) * 4.0;
     if (split_k > 1 && need > static_cast<double>(TDX_STATIC_SCRATCH_BYTES))
         return fail(TDX_ERR_WORKSPACE,
@@ -1412,14 +1534,10 @@ int tdx_gemm_splitk_static(int64_t M, int64_t N, int64_t K, int transA, int tran
     want.tile_n = tile_n;
     want.split_k = split_k;
     want.store_mode = 1;
-    int sm_count, smem_limit;
-    device_limits(&sm_count, &smem_limit);
-    tdx_config cfg;
-    rc = resolve_gemm_config(g, &want, sm_count, smem_limit, &cfg);
-    if (rc) return rc;
     DeviceCtx* ctx;
     rc = get_ctx(&ctx);
     if (rc) return rc;
+    tdx_config cfg;
     rc = resolve_gemm_config(g, &want, ctx->sm_count, ctx->smem_optin, &cfg);
     if (rc) return rc;
     float* scratch = nullptr;

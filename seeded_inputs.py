@@ -27,12 +27,28 @@ Tensor ids inside one workload: 0 = left operand / activations,
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 
 GOLDEN = np.uint64(0x9E3779B97F4A7C15)
 _M1 = np.uint64(0xBF58476D1CE4E5B9)
 _M2 = np.uint64(0x94D049BB133111EB)
 _CHUNK = 1 << 22
+
+
+def _each_chunk(n: int, fill) -> None:
+    """Calls fill(start, count) for every _CHUNK-sized piece of n elements; large tensors spread the pieces over a
+    few threads (each piece depends only on its own element counters, so the result is the same either way)."""
+    pieces = [(s, min(_CHUNK, n - s)) for s in range(0, n, _CHUNK)]
+    workers = min(len(pieces), 8, len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else 4)
+    if workers <= 1:
+        for s, c in pieces:
+            fill(s, c)
+        return
+    with ThreadPoolExecutor(max_workers=workers) as pool:
+        list(pool.map(lambda sc: fill(*sc), pieces))
 
 
 def mix64(z: np.ndarray) -> np.ndarray:
@@ -84,13 +100,15 @@ def uniform(seed: int, tensor_id: int, shape, dtype: str = "f32", scale: float =
     """i.i.d. uniform[-scale, scale) values; scale is applied in fp32."""
     n = int(np.prod(shape))
     out = np.empty(n, dtype=np.float32 if dtype == "f32" else np.uint16)
-    for s in range(0, n, _CHUNK):
-        c = min(_CHUNK, n - s)
+
+    def fill(s, c):
         r24 = (raw_bits(seed, tensor_id, s, c) >> np.uint64(40)).astype(np.float32)
         u = np.float32(2.0) * (r24 * np.float32(2.0 ** -24)) - np.float32(1.0)
         if scale != 1.0:
             u = u * np.float32(scale)
         out[s:s + c] = _store(u.astype(np.float32), dtype)
+
+    _each_chunk(n, fill)
     return out.reshape(shape)
 
 
@@ -98,8 +116,8 @@ def normal(seed: int, tensor_id: int, shape, dtype: str = "f32", sigma: float = 
     """i.i.d. normal(0, sigma) values (sigma is the standard deviation)."""
     n = int(np.prod(shape))
     out = np.empty(n, dtype=np.float32 if dtype == "f32" else np.uint16)
-    for s in range(0, n, _CHUNK):
-        c = min(_CHUNK, n - s)
+
+    def fill(s, c):
         b = raw_bits(seed, tensor_id, s, c)
         hi = (b >> np.uint64(32)).astype(np.float64)
         lo = (b & np.uint64(0xFFFFFFFF)).astype(np.float64)
@@ -107,6 +125,8 @@ def normal(seed: int, tensor_id: int, shape, dtype: str = "f32", sigma: float = 
         u2 = lo * 2.0 ** -32
         z = np.sqrt(-2.0 * np.log(u1)) * np.cos(2.0 * np.pi * u2) * float(sigma)
         out[s:s + c] = _store(z.astype(np.float32), dtype)
+
+    _each_chunk(n, fill)
     return out.reshape(shape)
 
 

@@ -268,20 +268,18 @@ def test_full_size_conv_128x128x64():
 
 
 def test_full_size_conv_56x56x256():
-    # N=32, H=W=56, Cin=Cout=256, seed 3 -- rows sampled from every part of the image batch
+    # N=32, H=W=56, Cin=Cout=256, seed 3 -- every output element (5.9e10 multiply-adds for the oracle), in the
+    # configuration the benchmark times (the automatic choice)
     N, H, W, Cin, Cout = 32, 56, 56, 256, 256
     x, w, b = si.conv_bf16(N, H, W, Cin, Cout, 3, 3, seed=3)
     st, y, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1)
     assert st == 0 and ok, tdx.tdx_last_error()
     M = N * H * W
-    rows = structured_rows(M, extra=2, max_blocks=24)
-    # image corners and edges of the first and last image
-    for n in (0, N - 1):
-        for p, q in [(0, 0), (0, W - 1), (H - 1, 0), (H - 1, W - 1), (0, 7), (8, 0), (27, 55)]:
-            rows = np.append(rows, (n * H + p) * W + q)
-    rows = np.unique(rows)
-    err = conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y, rows=rows)
-    assert err < TOL["bf16"] and err < TIGHT["bf16"], err
+    worst = 0.0
+    for r0 in range(0, M, 12544):                  # four images at a time bounds the fp64 reference's memory
+        rows = np.arange(r0, min(M, r0 + 12544), dtype=np.int64)
+        worst = max(worst, conv_error(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, y, rows=rows))
+    assert worst < TOL["bf16"] and worst < TIGHT["bf16"], worst
     assert (oracle.decode(y[::53], "bf16") >= 0).all()
     assert tdx.tdx_check_device_status() == 0
 

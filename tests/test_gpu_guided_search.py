@@ -70,3 +70,52 @@ def test_search_on_first_use_caches_the_winner_and_keeps_parity(tmp_path):
         assert tdx.tdx_set_autotune(0) == 0
     assert tdx.tdx_tune_save(str(path)) == 0
     assert key in path.read_text()
+
+
+@pytest.mark.gpu
+def test_exhaustive_gemm_search_winner_matches_the_oracle():
+    # whatever the search caches is what plain calls are then served with: run it and compare with the oracle
+    import seeded_inputs as si
+    from gpu_util import TIGHT, gemm_error, run_gemm
+    M, N, K = 640, 1152, 768
+    st, best, us, tried = tdx.tdx_tune_gemm(M, N, K, 0, 1, tdx.TDX_BF16, iters=5, cap=8192)
+    assert st == 0 and us > 0 and len(tried) > 8, tdx.tdx_last_error()
+    assert us <= min(t for _, t in tried) * 1.0001              # the fastest candidate passed the search's own output check
+    try:
+        st, c = tdx.tdx_default_gemm_config(M, N, K, 0, 1, tdx.TDX_BF16)
+        assert st == 0 and c.as_dict() == best.as_dict()
+        A, B = si.gemm_bf16_normal(M, N, K, seed=96, transB=1)
+        st, C, ok = run_gemm(M, N, K, 0, 1, -1.0, "bf16", A, B)             # served from the cache
+        assert st == 0 and ok, tdx.tdx_last_error()
+        assert gemm_error(M, N, K, 0, 1, -1.0, "bf16", A, B, C) < TIGHT["bf16"]
+        assert tdx.tdx_check_device_status() == 0
+    finally:
+        assert tdx.tdx_tune_clear() == 0
+        tdx.tdx_tune_load(str(__import__("pathlib").Path(tdx.__file__).parent / "tuned_b200.json"))
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("case", [(2, 28, 28, 64, 128, 3, 3, 1, 1), (2, 30, 30, 64, 64, 3, 3, 1, 2), (3, 14, 14, 128, 64, 1, 1, 0, 1)])
+def test_conv_search_winner_matches_the_oracle(case):
+    # tdx_tune_conv2d: every candidate of the convolution's search space is timed, the winner's output is checked
+    # against the generic kernel inside the search, cached, and then serves tdx_conv2d_bias_relu: compare with the oracle
+    import seeded_inputs as si
+    from gpu_util import TIGHT, conv_error, run_conv
+    N, H, W, Cin, Cout, R, S, pad, stride = case
+    st, space = tdx.tdx_enum_conv2d_configs(N, H, W, Cin, Cout, R, S, pad, stride, tdx.TDX_BF16)
+    assert st == 0 and len(space) > 1
+    st, best, us, tried = tdx.tdx_tune_conv2d(N, H, W, Cin, Cout, R, S, pad, stride, tdx.TDX_BF16, iters=5, cap=4096)
+    assert st == 0 and us > 0, tdx.tdx_last_error()
+    assert 1 < len(tried) <= len(space)
+    assert best.as_dict() in space
+    try:
+        st, c = tdx.tdx_default_conv2d_config(N, H, W, Cin, Cout, R, S, pad, stride, tdx.TDX_BF16)
+        assert st == 0 and c.as_dict() == best.as_dict()
+        x, w, b = si.conv_bf16(N, H, W, Cin, Cout, R, S, seed=97)
+        st, y, ok = run_conv(N, H, W, Cin, Cout, R, S, pad, stride, "bf16", x, w, b, 1)
+        assert st == 0 and ok, tdx.tdx_last_error()
+        assert conv_error(N, H, W, Cin, Cout, R, S, pad, stride, "bf16", x, w, b, 1, y) < TIGHT["bf16"]
+        assert tdx.tdx_check_device_status() == 0
+    finally:
+        assert tdx.tdx_tune_clear() == 0
+        tdx.tdx_tune_load(str(__import__("pathlib").Path(tdx.__file__).parent / "tuned_b200.json"))

@@ -61,3 +61,34 @@ def test_static_scratch_rejects_what_does_not_fit_and_leaves_output_untouched():
     A, B = si.gemm_bf16_normal(64, 64, 100, seed=93, transB=1)
     st, _, untouched = run_static(64, 64, 100, 0, 1, 1.0, A, B, 64, 2)
     assert st == tdx.TDX_ERR_ALIGNMENT and untouched
+
+
+def test_static_scratch_call_leaves_free_device_memory_unchanged():
+    # the property the entry point exists for: once the library is warm on this device, a call takes no device
+    # memory -- not from cudaMalloc, not from a growing cache.  All buffers are made before the measured calls.
+    M, N, K, split = 392, 264, 2048, 4
+    A, B = si.gemm_bf16_normal(M, N, K, seed=94, transB=1)
+    dA, dB = to_dev(A), to_dev(B)
+    out = GuardedOut(M * N, "bf16")
+    assert tdx.tdx_gemm_splitk_static(M, N, K, 0, 1, 1.0, dA, dB, out.ptr, 64, split) == 0      # warm call
+    torch.cuda.synchronize()
+    first = out.payload().copy()
+    free0, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        assert tdx.tdx_gemm_splitk_static(M, N, K, 0, 1, 1.0, dA, dB, out.ptr, 64, split) == 0
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, (free0, free1)
+    assert np.array_equal(out.payload(), first) and out.guards_intact()
+    # a new shape on the warm library allocates nothing either (no per-shape cache behind this entry point)
+    M2, N2 = 200, 136
+    A2, B2 = si.gemm_bf16_normal(M2, N2, K, seed=95, transB=1)
+    dA2, dB2 = to_dev(A2), to_dev(B2)
+    out2 = GuardedOut(M2 * N2, "bf16")
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    assert tdx.tdx_gemm_splitk_static(M2, N2, K, 0, 1, 1.0, dA2, dB2, out2.ptr, 64, 2) == 0
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, (free0, free1)
+    assert gemm_error(M2, N2, K, 0, 1, 1.0, "bf16", A2, B2, out2.payload().reshape(M2, N2)) < TIGHT["bf16"]
