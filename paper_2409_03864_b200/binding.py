@@ -285,7 +285,7 @@ def tdx_tune_conv2d(N, H, W, Cin, Cout, R, S, pad, stride, dtype, iters=20, stre
                                                               bu, t, tu, c, n, _stream(stream)), cap)
 
 
-def _enum(call, cap=1024):
+def _enum(call, cap=8192):
     out = (tdx_config * cap)()
     n = ctypes.c_int(0)
     st = call(out, cap, ctypes.byref(n))
