@@ -335,13 +335,15 @@ int run_gemm_pair(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     lc.dynamicSmemBytes = static_cast<size_t>(p.stages) * ((128 + p.bn / 2) * 128) + 1024 +
                           staging_bytes_for(128, p.tma_store ? 2 : 1);
     lc.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;      // as for the single-CTA kernel
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
-    lc.numAttrs = 1;
+    lc.numAttrs = 2;
     TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_pair_kernel, ma, mb, mc, p));
     g_launches.fetch_add(1);
     return TDX_OK;

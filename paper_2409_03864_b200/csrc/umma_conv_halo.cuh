@@ -45,6 +45,44 @@ __device__ __forceinline__ void halo_patch_origin(const UmmaParams& p, int m_blk
     *q0 = (rem - ph * p.patches_w) * p.bw;
 }
 
+// The input windows of channel chunk `cc` for the 128-row halves of tile `m_blk`, loaded into one halo stage.
+__device__ __forceinline__ void issue_halo_windows(const UmmaParams& p, const CUtensorMap* tmA, const CUtensorMap* tmA_row,
+                                                   int m_blk, int cc, int mh, uint8_t* stage_dst, uint64_t* bar) {
+    auto ld4 = [&](uint8_t* dst, const CUtensorMap* m, int c0, int c1, int c2, int c3) {
+        ptx::tma_load_4d(dst, m, bar, c0, c1, c2, c3);
+    };
+    for (int h = 0; h < mh; ++h) {
+        int n, p0, q0;
+        halo_patch_origin(p, m_blk, h, mh, &n, &p0, &q0);
+        uint8_t* dst = stage_dst + h * p.halo_bytes;
+        if (p.Pv > 0) {
+            // Row u of the stacked column is row u % Pv of image u / Pv when that is below H, and
+            // zero otherwise.  A window that lies inside one image and the zero rows around it is
+            // one box (rows outside [0, H) are zero-filled); a window that reaches into the next
+            // image is copied row by row.
+            const int u = p0 - p.pad;
+            int img = u >= 0 ? u / p.Pv : 0;
+            int row = u >= 0 ? u - img * p.Pv : u;       // negative: above the first image
+            if (row >= p.H) {                            // starts in the zero rows below image img:
+                row -= p.Pv;                             // the same rows lie above image img + 1
+                ++img;
+            }
+            if (row + p.hrows <= p.Pv) {
+                // img == Nimg happens past the last image: that coordinate is zero-filled too
+                ld4(dst, tmA, cc * kBK, q0 - p.pad, row, img);
+            } else {
+                for (int j = 0; j < p.hrows; ++j) {
+                    const bool real = row >= 0 && row < p.H && img < p.Nimg;
+                    ld4(dst + j * p.hpitch * 128, tmA_row, cc * kBK, q0 - p.pad, real ? row : p.H, real ? img : 0);
+                    if (++row == p.Pv) { row = 0; ++img; }
+                }
+            }
+        } else {
+            ld4(dst, tmA, cc * kBK, q0 - p.pad, p0 - p.pad, n);
+        }
+    }
+}
+
 __global__ void __launch_bounds__(608, 1)
 umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmA_row,
                       const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmC,
@@ -100,11 +138,14 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         ptx::tmem_alloc(&s_tmem_base, static_cast<uint32_t>(p.tmem_cols));
         ptx::tmem_relinquish();
     }
+    // before the dependency wait (see umma_contract_kernel): every role works out its first tile
+    const int total_items = p.tiles_m * p.tiles_n;
+    TileCoord t_first;
+    const bool have_first = get_tile(p, 0, blockIdx.x, gridDim.x, total_items, &t_first);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = s_tmem_base;
-    const int total_items = p.tiles_m * p.tiles_n;
     ptx::grid_launch_dependents();     // see umma_contract_kernel
     ptx::grid_dependency_wait();
 
@@ -115,8 +156,9 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             int a_buf = 0;
             uint32_t a_phase = 0;
             bool ok = true;
-            TileCoord t;
-            for (int local = 0; ok && get_tile(p, local, blockIdx.x, gridDim.x, total_items, &t); ++local) {
+            TileCoord t = t_first;
+            bool have = have_first;
+            for (int local = 0; ok && have; have = get_tile(p, ++local, blockIdx.x, gridDim.x, total_items, &t)) {
                 for (int cc = 0; cc < p.cchunks; ++cc) {
                     if (!wait_bounded(&aempty_bar[a_buf], a_phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) {
                         ok = false;
@@ -124,37 +166,7 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
                     }
                     uint64_t* bar = &afull_bar[a_buf];
                     ptx::mbar_arrive_expect_tx(bar, halo_tx);
-                    for (int h = 0; h < mh; ++h) {
-                        int n, p0, q0;
-                        halo_patch_origin(p, t.m_blk, h, mh, &n, &p0, &q0);
-                        uint8_t* dst = a_ring + static_cast<size_t>(a_buf) * a_stage_bytes + h * p.halo_bytes;
-                        if (p.Pv > 0) {
-                            // Row u of the stacked column is row u % Pv of image u / Pv when that is below H, and
-                            // zero otherwise.  A window that lies inside one image and the zero rows around it is
-                            // one box (rows outside [0, H) are zero-filled); a window that reaches into the next
-                            // image is copied row by row.
-                            const int u = p0 - p.pad;
-                            int img = u >= 0 ? u / p.Pv : 0;
-                            int row = u >= 0 ? u - img * p.Pv : u;       // negative: above the first image
-                            if (row >= p.H) {                            // starts in the zero rows below image img:
-                                row -= p.Pv;                             // the same rows lie above image img + 1
-                                ++img;
-                            }
-                            if (row + p.hrows <= p.Pv) {
-                                // img == Nimg happens past the last image: that coordinate is zero-filled too
-                                ptx::tma_load_4d(dst, &tmA, bar, cc * kBK, q0 - p.pad, row, img);
-                            } else {
-                                for (int j = 0; j < p.hrows; ++j) {
-                                    const bool real = row >= 0 && row < p.H && img < p.Nimg;
-                                    ptx::tma_load_4d(dst + j * p.hpitch * 128, &tmA_row, bar, cc * kBK, q0 - p.pad,
-                                                     real ? row : p.H, real ? img : 0);
-                                    if (++row == p.Pv) { row = 0; ++img; }
-                                }
-                            }
-                        } else {
-                            ptx::tma_load_4d(dst, &tmA, bar, cc * kBK, q0 - p.pad, p0 - p.pad, n);
-                        }
-                    }
+                    issue_halo_windows(p, &tmA, &tmA_row, t.m_blk, cc, mh, a_ring + static_cast<size_t>(a_buf) * a_stage_bytes, bar);
                     if (++a_buf == p.a_stages) { a_buf = 0; a_phase ^= 1u; }
                 }
             }
@@ -176,8 +188,9 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             } else {
                 int b_stage = 0;
                 uint32_t b_phase = 0;
-                TileCoord t;
-                for (int local = 0; ok && get_tile(p, local, blockIdx.x, gridDim.x, total_items, &t); ++local) {
+                TileCoord t = t_first;
+                bool have = have_first;
+                for (int local = 0; ok && have; have = get_tile(p, ++local, blockIdx.x, gridDim.x, total_items, &t)) {
                     const uint32_t slice_tx = static_cast<uint32_t>(t.bn) * 128u;     // the tile's width (fitted plans vary it)
                     for (int cc = 0; ok && cc < p.cchunks; ++cc) {
                         for (int tap = 0; tap < taps; ++tap) {
@@ -215,8 +228,9 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
             uint32_t a_phase = 0, b_phase = 0;
             bool ok = true;
             if (p.b_resident && !wait_bounded(&bfull_bar[0], 0, abort_flag, p.status, kTimeoutMma)) ok = false;
-            TileCoord t;
-            for (; ok && get_tile(p, local, blockIdx.x, gridDim.x, total_items, &t); ++local) {
+            TileCoord t = t_first;
+            bool have = have_first;
+            for (; ok && have; have = get_tile(p, ++local, blockIdx.x, gridDim.x, total_items, &t)) {
                 // N field of the instruction descriptor (bits 17..22) follows the tile's width
                 const uint32_t idesc = (idesc0 & ~(0x3Fu << 17)) | (static_cast<uint32_t>(t.bn >> 3) << 17);
                 uint32_t d_tmem[2] = {0u, 0u};
@@ -273,7 +287,7 @@ umma_conv_halo_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_cons
         }
     } else {
         epilogue_role<true>(p, &tmC, staging, tmem_base, tfull_bar, tempty_bar, abort_flag, mh, warp, lane, total_items,
-                            -1, 0, 1, 0, 0, &tmC_row);
+                            -1, 0, 1, 0, 0, &tmC_row, &t_first, have_first);
     }
 
     ptx::tc_fence_before_sync();

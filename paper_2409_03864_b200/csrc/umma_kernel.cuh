@@ -167,6 +167,12 @@ __device__ __forceinline__ TileCoord decode_item(const UmmaParams& p, int item) 
     return t;
 }
 
+// K block a CTA starts a tile's reduction with (k_stagger: CTAs start at different blocks; same terms, rotated order)
+__device__ __forceinline__ int first_kblock(const UmmaParams& p, const TileCoord& t) {
+    const int nkb = t.kb1 - t.kb0;
+    return t.kb0 + (p.k_stagger ? static_cast<int>((static_cast<long long>(blockIdx.x) * nkb) / gridDim.x) : 0);
+}
+
 // The `local`-th tile of worker `first_item` of `item_stride` workers (CTAs, or CTA pairs): from the tile table when
 // there is one, else item first_item + local * item_stride of the uniform grid.  Returns false when there is none.
 __device__ __forceinline__ bool get_tile(const UmmaParams& p, int local, int first_item, int item_stride, int total_items,
@@ -191,6 +197,57 @@ __device__ __forceinline__ bool get_tile(const UmmaParams& p, int local, int fir
     return true;
 }
 
+// The copies of K block `kb` of tile `t` into one pipeline stage: op(A) rows and op(B) columns of that block.
+template <bool kConv>
+__device__ __forceinline__ void issue_kblock(const UmmaParams& p, const CUtensorMap* tmA, const CUtensorMap* tmB,
+                                             const TileCoord& t, int kb, int mh, uint8_t* a_dst, uint8_t* b_dst, uint64_t* bar) {
+    auto ld2 = [&](uint8_t* dst, const CUtensorMap* m, int c0, int c1) { ptx::tma_load_2d(dst, m, bar, c0, c1); };
+    auto ld3 = [&](uint8_t* dst, const CUtensorMap* m, int c0, int c1, int c2) { ptx::tma_load_3d(dst, m, bar, c0, c1, c2); };
+    auto ld4 = [&](uint8_t* dst, const CUtensorMap* m, int c0, int c1, int c2, int c3) {
+        ptx::tma_load_4d(dst, m, bar, c0, c1, c2, c3);
+    };
+    if (kConv) {
+        const int tap = kb / p.cchunks;
+        const int cc = kb - tap * p.cchunks;
+        const int r = tap / p.S;
+        const int s = tap - r * p.S;
+        const int ppi = p.patches_w * p.patches_h;
+        const uint32_t patch_bytes = static_cast<uint32_t>(p.bw * p.bh) * 128u;
+        for (int i = 0; i < p.nb; ++i) {
+            const int patch = t.m_blk * p.nb + i;
+            const int n = patch / ppi;
+            const int rem = patch - n * ppi;
+            const int ph = rem / p.patches_w;
+            const int pw = rem - ph * p.patches_w;
+            ld4(a_dst + i * patch_bytes, tmA, cc * kBK, pw * p.bw * p.stride + s - p.pad, ph * p.bh * p.stride + r - p.pad, n);
+        }
+        ld3(b_dst, tmB, cc * kBK, tap, t.n0);
+        return;
+    }
+    int ka = kb, kbb = kb;                  // K block of A and of B
+    if (p.seg_kb > 0) {
+        const int sg = kb / p.seg_kb, r = kb - sg * p.seg_kb;
+        ka = p.a_seg[sg] * p.seg_kb + r;
+        kbb = p.b_seg[sg] * p.seg_kb + r;
+    }
+    if (p.batch > 1) {
+        // batched: K-major 3-D operands; rows past M or N of a batch are zero-filled, not the next batch's
+        for (int h = 0; h < mh; ++h) ld3(a_dst + h * kHalfABytes, tmA, ka * kBK, t.m_blk * p.bm + h * kHalfM, t.batch);
+        for (int r0 = 0; r0 < t.bn; r0 += p.b_box) ld3(b_dst + r0 * 128, tmB, kbb * kBK, t.n0 + r0, t.batch);
+        return;
+    }
+    if (p.a_mn_major) {
+        for (int i = 0; i < 2 * mh; ++i) ld2(a_dst + i * 8192, tmA, t.m_blk * p.bm + i * 64, ka * kBK);
+    } else {
+        for (int h = 0; h < mh; ++h) ld2(a_dst + h * kHalfABytes, tmA, ka * kBK, t.m_blk * p.bm + h * kHalfM);
+    }
+    if (p.b_mn_major) {
+        for (int i = 0; i < t.bn / 64; ++i) ld2(b_dst + i * 8192, tmB, t.n0 + i * 64, kbb * kBK);
+    } else {
+        for (int r0 = 0; r0 < t.bn; r0 += p.b_box) ld2(b_dst + r0 * 128, tmB, kbb * kBK, t.n0 + r0);
+    }
+}
+
 // Epilogue role (all warps from the third on).  With the staged epilogue there are 16 of them (4 per TMEM
 // lane quarter) and the warps of a quarter take the 32-column steps round robin; the direct epilogue has one
 // warp per quarter and 128-row half.
@@ -199,7 +256,8 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                                               uint32_t tmem_base, uint64_t* tfull_bar, uint64_t* tempty_bar,
                                               volatile int* abort_flag, int mh, int warp, int lane, int total_items,
                                               int first_item = -1, int item_stride = 0, int m_mul = 1, int m_add = 0,
-                                              uint32_t tempty_cluster_addr = 0, const CUtensorMap* tmC_row = nullptr) {
+                                              uint32_t tempty_cluster_addr = 0, const CUtensorMap* tmC_row = nullptr,
+                                              const TileCoord* t_first = nullptr, bool have_first = false) {
     // CTA pairs: the pair walks tiles of 256 rows, this CTA owns rows [128 * (2 m + rank), +128) of tile m, and the
     // accumulator-free signal goes to the leader CTA's barrier (tempty_cluster_addr, a shared::cluster address)
     if (first_item < 0) {
@@ -213,8 +271,11 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
     const int cgrp = (ew >> 2) / mh;              // which share of the columns
     const int quarter = warp & 3;                 // TMEM lane quarter this warp may read
     const int row_in_tile = half * kHalfM + quarter * 32 + lane;
+    // the caller may have worked out the first tile already (before the grid-dependency wait)
     TileCoord t;
-    for (int local = 0; get_tile(p, local, first_item, item_stride, total_items, &t); ++local) {
+    bool have = have_first;
+    if (t_first != nullptr) t = *t_first; else have = get_tile(p, 0, first_item, item_stride, total_items, &t);
+    for (int local = 0; have; have = get_tile(p, ++local, first_item, item_stride, total_items, &t)) {
         t.m_blk = t.m_blk * m_mul + m_add;
         const int sidx = local * mh + half;
         const int buf = sidx % p.slots;
@@ -540,13 +601,20 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         ptx::tmem_alloc(&s_tmem_base, static_cast<uint32_t>(p.tmem_cols));
         ptx::tmem_relinquish();
     }
+    // What does not depend on the previous grid's results happens BEFORE the dependency wait below, in the microsecond
+    // or so between this CTA's start and the predecessor's completion: every role works out its first tile (the tile
+    // table was written by the host long before any launch that reads it).  Asking for the first K blocks to be brought
+    // into L2 here as well was measured and dropped: the loads after the wait did land 1-2 us sooner, but the wait itself
+    // returned later by more than that (1024^3: 11.5 vs 10.2 us per step).
+    const int total_items = p.tiles_m * p.tiles_n * p.split_k * (p.batch > 1 ? p.batch : 1);
+    TileCoord t_first;
+    const bool have_first = get_tile(p, 0, blockIdx.x, gridDim.x, total_items, &t_first);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = s_tmem_base;
-    const int total_items = p.tiles_m * p.tiles_n * p.split_k * (p.batch > 1 ? p.batch : 1);
     // the next grid in the stream (the split-K reduction, or the next call's kernel) may be scheduled as SMs free up and
-    // run its set-up; this grid touches global memory only after its own predecessor has completed
+    // run its set-up; this grid reads and writes global data only after its own predecessor has completed
     ptx::grid_launch_dependents();
     ptx::grid_dependency_wait();
 
@@ -556,11 +624,12 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            TileCoord t;
-            for (int local = 0; ok && get_tile(p, local, blockIdx.x, gridDim.x, total_items, &t); ++local) {
+            TileCoord t = t_first;
+            bool have = have_first;
+            for (int local = 0; ok && have; have = get_tile(p, ++local, blockIdx.x, gridDim.x, total_items, &t)) {
                 const int nkb = t.kb1 - t.kb0;
                 const uint32_t tile_tx = a_bytes + static_cast<uint32_t>(t.bn) * 128u;
-                int kb = t.kb0 + (p.k_stagger ? static_cast<int>((static_cast<long long>(blockIdx.x) * nkb) / gridDim.x) : 0);
+                int kb = first_kblock(p, t);
                 for (int i = 0; i < nkb; ++i, kb = (kb + 1 == t.kb1) ? t.kb0 : kb + 1) {
                     if (!wait_bounded(&empty_bar[stage], phase ^ 1u, abort_flag, p.status, kTimeoutProducer)) {
                         ok = false;
@@ -569,55 +638,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                     uint64_t* bar = &full_bar[stage];
                     ptx::mbar_arrive_expect_tx(bar, tile_tx);
                     uint8_t* a_dst = smem + static_cast<size_t>(stage) * stage_bytes;
-                    uint8_t* b_dst = a_dst + a_bytes;
-                    if (kConv) {
-                        const int tap = kb / p.cchunks;
-                        const int cc = kb - tap * p.cchunks;
-                        const int r = tap / p.S;
-                        const int s = tap - r * p.S;
-                        const int ppi = p.patches_w * p.patches_h;
-                        const uint32_t patch_bytes = static_cast<uint32_t>(p.bw * p.bh) * 128u;
-                        for (int i = 0; i < p.nb; ++i) {
-                            const int patch = t.m_blk * p.nb + i;
-                            const int n = patch / ppi;
-                            const int rem = patch - n * ppi;
-                            const int ph = rem / p.patches_w;
-                            const int pw = rem - ph * p.patches_w;
-                            ptx::tma_load_4d(a_dst + i * patch_bytes, &tmA, bar, cc * kBK, pw * p.bw * p.stride + s - p.pad,
-                                             ph * p.bh * p.stride + r - p.pad, n);
-                        }
-                        ptx::tma_load_3d(b_dst, &tmB, bar, cc * kBK, tap, t.n0);
-                    } else {
-                        int ka = kb, kbb = kb;                  // K block of A and of B
-                        if (p.seg_kb > 0) {
-                            const int sg = kb / p.seg_kb, r = kb - sg * p.seg_kb;
-                            ka = p.a_seg[sg] * p.seg_kb + r;
-                            kbb = p.b_seg[sg] * p.seg_kb + r;
-                        }
-                        if (p.batch > 1) {
-                            // batched: K-major 3-D operands; rows past M or N of a batch are zero-filled, not the next batch's
-                            for (int h = 0; h < mh; ++h)
-                                ptx::tma_load_3d(a_dst + h * kHalfABytes, &tmA, bar, ka * kBK, t.m_blk * p.bm + h * kHalfM, t.batch);
-                            for (int r0 = 0; r0 < t.bn; r0 += p.b_box)
-                                ptx::tma_load_3d(b_dst + r0 * 128, &tmB, bar, kbb * kBK, t.n0 + r0, t.batch);
-                        } else {
-                            if (p.a_mn_major) {
-                                for (int i = 0; i < 2 * mh; ++i)
-                                    ptx::tma_load_2d(a_dst + i * 8192, &tmA, bar, t.m_blk * p.bm + i * 64, ka * kBK);
-                            } else {
-                                for (int h = 0; h < mh; ++h)
-                                    ptx::tma_load_2d(a_dst + h * kHalfABytes, &tmA, bar, ka * kBK,
-                                                     t.m_blk * p.bm + h * kHalfM);
-                            }
-                            if (p.b_mn_major) {
-                                for (int i = 0; i < t.bn / 64; ++i)
-                                    ptx::tma_load_2d(b_dst + i * 8192, &tmB, bar, t.n0 + i * 64, kbb * kBK);
-                            } else {
-                                for (int r0 = 0; r0 < t.bn; r0 += p.b_box)
-                                    ptx::tma_load_2d(b_dst + r0 * 128, &tmB, bar, kbb * kBK, t.n0 + r0);
-                            }
-                        }
-                    }
+                    issue_kblock<kConv>(p, &tmA, &tmB, t, kb, mh, a_dst, a_dst + a_bytes, bar);
                     if (++stage == p.stages) {
                         stage = 0;
                         phase ^= 1u;
@@ -650,8 +671,9 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            TileCoord t;
-            for (int local = 0; ok && get_tile(p, local, blockIdx.x, gridDim.x, total_items, &t); ++local) {
+            TileCoord t = t_first;
+            bool have = have_first;
+            for (int local = 0; ok && have; have = get_tile(p, ++local, blockIdx.x, gridDim.x, total_items, &t)) {
                 // N field of the instruction descriptor (bits 17..22) follows the tile's width
                 const uint32_t idesc = (idesc0 & ~(0x3Fu << 17)) | (static_cast<uint32_t>(t.bn >> 3) << 17);
                 // accumulator slots of this tile: use number u of slot s has barrier phase (u & 1)
@@ -706,7 +728,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         }
     } else {
         epilogue_role<kConv>(p, &tmC, smem + static_cast<size_t>(p.stages) * stage_bytes, tmem_base, tfull_bar,
-                             tempty_bar, abort_flag, mh, warp, lane, total_items);
+                             tempty_bar, abort_flag, mh, warp, lane, total_items, -1, 0, 1, 0, 0, nullptr, &t_first, have_first);
     }
 
     ptx::tc_fence_before_sync();

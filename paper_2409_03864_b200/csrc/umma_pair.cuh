@@ -64,12 +64,17 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         ptx::tmem_alloc_pair(&s_tmem_base, static_cast<uint32_t>(p.tmem_cols));
         ptx::tmem_relinquish_pair();
     }
+    // before the dependency wait (see umma_contract_kernel): the pair's first tile
+    const int total_items = p.tiles_m * p.tiles_n;     // tiles of 256 rows
+    TileCoord t_first;
+    const bool have_first = get_tile(p, 0, pair_id, num_pairs, total_items, &t_first);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::cluster_sync_all();          // barriers of both CTAs are initialised before anyone signals across
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = s_tmem_base;
-    const int total_items = p.tiles_m * p.tiles_n;     // tiles of 256 rows
+    ptx::grid_launch_dependents();
+    ptx::grid_dependency_wait();
 
     if (warp == 0) {
         // ------------------------------------------------------------ producer (one per CTA)
@@ -77,8 +82,9 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            TileCoord t;
-            for (int local = 0; ok && get_tile(p, local, pair_id, num_pairs, total_items, &t); ++local) {
+            TileCoord t = t_first;
+            bool have = have_first;
+            for (int local = 0; ok && have; have = get_tile(p, ++local, pair_id, num_pairs, total_items, &t)) {
                 const int my_bn = t.bn / 2;                                            // this CTA's share of the tile's columns
                 const int row0 = t.m_blk * 256 + static_cast<int>(rank) * kHalfM;      // this CTA's rows of op(A)
                 const int col0 = t.n0 + static_cast<int>(rank) * my_bn;                // this CTA's columns of op(B)
@@ -131,8 +137,9 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            TileCoord t;
-            for (int local = 0; ok && get_tile(p, local, pair_id, num_pairs, total_items, &t); ++local) {
+            TileCoord t = t_first;
+            bool have = have_first;
+            for (int local = 0; ok && have; have = get_tile(p, ++local, pair_id, num_pairs, total_items, &t)) {
                 // N field of the instruction descriptor (bits 17..22) follows the tile's width
                 const uint32_t idesc = (idesc0 & ~(0x3Fu << 17)) | (static_cast<uint32_t>(t.bn >> 3) << 17);
                 const int slot = local % p.slots;
@@ -169,7 +176,7 @@ umma_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         const uint32_t leader_tempty = ptx::mapa_u32(ptx::smem_u32(&tempty_bar[0]), 0);
         epilogue_role<false>(p, &tmC, smem + static_cast<size_t>(p.stages) * stage_bytes, tmem_base, tfull_bar, tempty_bar,
                              abort_flag, 1, warp, lane, total_items, pair_id, num_pairs, 2, static_cast<int>(rank),
-                             leader_tempty);
+                             leader_tempty, nullptr, &t_first, have_first);
     }
 
     // neither CTA may free tensor memory or leave while the other can still touch its memory
