@@ -116,8 +116,12 @@ typedef struct {
  *   bound, several times faster.  That path keeps its pieces in device scratch owned by the library, grown on
  *   demand by cudaMalloc (make the first call for a size before any stream capture).
  * Errors: INVALID_ARG (negative size, flag not 0/1, NULL pointer with non-empty problem, unknown dtype,
- *         non-finite alpha is allowed), CUDA.  Shapes that miss the tensor-core path's alignment rules
- *         are served by the generic GPU kernel, not rejected.  There is no CPU fallback.
+ *         non-finite alpha is allowed), CUDA.  bf16 shapes that miss the tensor-core path's alignment rules
+ *         (a row pitch that is no multiple of 16 bytes, a misaligned base) are not rejected: from 2^21
+ *         multiply-adds on, the operands are first copied K-major with K padded to a multiple of 64 into device
+ *         scratch owned by the library (one more launch; grown by cudaMalloc, so make the first call for a size
+ *         before any stream capture) and the tensor cores run on the copies -- the padding adds exact zeros;
+ *         smaller ones run on the generic GPU kernel.  There is no CPU fallback.
  */
 int tdx_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype,
              const void* A, const void* B, void* C, void* stream);
@@ -129,10 +133,16 @@ int tdx_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, float alph
  * (C[b,i,j] += A[b,i,k] * B[b,k,j]; its workload is batch 6, M 196, N 256, K 2305).  Layouts per batch
  * as for tdx_gemm; batch b of an operand starts strideX elements after batch b - 1 (strideA or strideB
  * may be 0: the operand is shared by all batches; strideC >= M * N).  C is read only when beta != 0 and
- * must not alias A or B.  fp32 runs on the CUDA cores (any shape); bf16 runs on the tensor cores when
- * every batch's operands meet the 16-byte rules of tdx_gemm (contiguous dims and batch strides multiples
- * of 8 elements, 16-byte aligned bases) and otherwise -- K = 2305 is such a case -- on the generic GPU
- * kernel.  batch, M or N = 0: no-op.  K = 0: C = beta * C.  Errors as for tdx_gemm.
+ * must not alias A or B.  fp32: CUDA cores, or bf16 pieces on the tensor cores from about 2^28 multiply-adds.
+ * bf16: ONE tensor-core launch over all batches (3-D tensor maps: contiguous dimension, the other one, batch;
+ * rows past M or N of a batch read as zero, never as the next batch), straight from the caller's buffers when
+ * every batch's operands meet the 16-byte rules of tdx_gemm (contiguous dims and batch strides multiples of 8
+ * elements, 16-byte aligned bases), and otherwise -- K = 2305 is such a case: the paper's treatment of sizes that
+ * do not divide is to split and peel, here the remainder is padded with zeros instead -- from K-major copies with
+ * K padded to a multiple of 64, made by one more launch into scratch owned by the library.  A K split chosen so
+ * that every SM has an item is reduced in a fixed order by one launch for all batches, which also applies beta.
+ * Problems under 2^21 multiply-adds in an unaddressable layout run on the generic GPU kernel.
+ * batch, M or N = 0: no-op.  K = 0: C = beta * C.  Errors as for tdx_gemm.
  */
 int tdx_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, float beta,
                      int dtype, const void* A, int64_t strideA, const void* B, int64_t strideB, void* C, int64_t strideC,

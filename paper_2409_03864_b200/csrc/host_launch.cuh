@@ -46,7 +46,7 @@ int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensor
 // The reduction is launched with programmatic stream serialization so that its launch latency hides behind
 // the tail of the GEMM kernel; it waits on the device for the GEMM grid to complete before reading partials.
 int launch_splitk_reduce(int grid, cudaStream_t st, long long MN, int N, int split, const float* partial, float alpha,
-                         __nv_bfloat16* out, int vec8, float beta = 0.0f) {
+                         __nv_bfloat16* out, int vec8, float beta = 0.0f, int batch = 1, long long batch_c = 0) {
     cudaLaunchConfig_t lc;
     std::memset(&lc, 0, sizeof lc);
     lc.gridDim = dim3(static_cast<unsigned>(grid));
@@ -60,7 +60,8 @@ int launch_splitk_reduce(int grid, cudaStream_t st, long long MN, int N, int spl
     lc.numAttrs = 1;
     const float* bias = nullptr;
     int relu = 0;
-    TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::splitk_reduce_kernel, MN, N, split, partial, alpha, bias, relu, out, vec8, beta));
+    TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::splitk_reduce_kernel, MN, N, split, partial, alpha, bias, relu, out, vec8, beta, batch,
+                                batch_c));
     g_launches.fetch_add(1);
     return TDX_OK;
 }
@@ -77,21 +78,28 @@ int ensure_ws(DeviceCtx* ctx, size_t bytes, void** out) {
     return TDX_OK;
 }
 
-// fp32 GEMM from bf16 pieces: the operands handed to run_gemm_umma hold three pieces of `seg_kb` K blocks side by side
-// (cols = 3 * 64 * seg_kb columns), g.K spans the six piece pairs, and C is fp32.
+// Operand forms beyond the plain GEMM that run_gemm_umma takes.
+//  - fp32 GEMM from bf16 pieces (seg_kb > 0): the operands hold three pieces of `seg_kb` K blocks side by side
+//    (cols = 3 * 64 * seg_kb columns), g.K spans the six piece pairs, and C is fp32.
+//  - batched (batch > 1): all batches in one launch; batch b of A / B / C starts batch_a / batch_b / batch_c elements
+//    after batch b - 1 (batch_a or batch_b = 0: one matrix shared by all batches).
+//  - cols > 0: K-major operands whose rows really have `cols` columns (K padded up to the K block).
 struct PieceInfo {
     int seg_kb = 0;
     int64_t cols = 0;
-    int64_t batch = 1;        // > 1: all batches in one launch (operands dense per batch, C batch_c elements apart)
+    int64_t batch = 1;
+    int64_t batch_a = -1, batch_b = -1;   // -1: dense (rows * cols)
     int64_t batch_c = 0;
 };
 
 int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
                   const tdx_config& cfg, void* ws, size_t ws_bytes, bool internal_ws, cudaStream_t st, float beta = 0.0f,
                   const PieceInfo* pieces = nullptr, bool c_f32 = false) {
-    // c_f32: bf16 operands, fp32 result (C points to floats); pieces imply it
+    // c_f32: bf16 operands, fp32 result (C points to floats); bf16 pieces imply it
+    const PieceInfo* form = pieces;                            // any of the forms above
+    if (pieces && pieces->seg_kb == 0) pieces = nullptr;       // from here on `pieces` means the fp32 piece form only
     const int64_t num_kb = ceil_div(g.K, 64);
-    const int64_t k_cols = pieces ? pieces->cols : g.K;        // columns the K-major operands really have
+    const int64_t k_cols = (form && form->cols > 0) ? form->cols : g.K;      // columns the K-major operands really have
     UmmaParams p;
     std::memset(&p, 0, sizeof p);
     p.M = static_cast<int>(g.M);
@@ -134,8 +142,25 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
             p.batch_c = pieces->batch_c;
         }
     }
-    const int64_t nbatch = pieces ? pieces->batch : 1;
-    const long long out_batch_c = pieces ? static_cast<long long>(pieces->batch_c) : 0;
+    const int64_t nbatch = form ? form->batch : 1;
+    const long long out_batch_c = form ? static_cast<long long>(form->batch_c) : 0;
+    if (!pieces && nbatch > 1) {
+        if (static_cast<long long>(nbatch) * p.tiles_m * p.tiles_n * cfg.split_k >= (1LL << 31))
+            return fail(TDX_ERR_UNSUPPORTED, "too many batched tiles for one launch");
+        p.batch = static_cast<int>(nbatch);
+        p.batch_c = out_batch_c;
+        if (!c_f32) p.vec_store = p.vec_store && (out_batch_c % 8 == 0);
+    }
+    // batch strides of the operands (elements); a shared operand is a tensor with a single batch
+    const int64_t a_rows_stored = g.transA ? g.K : g.M, a_cols_stored = g.transA ? g.M : k_cols;
+    const int64_t b_rows_stored = g.transB ? g.N : g.K, b_cols_stored = g.transB ? k_cols : g.N;
+    const int64_t a_bstride = (form && form->batch_a >= 0) ? form->batch_a : a_rows_stored * a_cols_stored;
+    const int64_t b_bstride = (form && form->batch_b >= 0) ? form->batch_b : b_rows_stored * b_cols_stored;
+    p.a_shared = (nbatch > 1 && a_bstride == 0) ? 1 : 0;
+    p.b_shared = (nbatch > 1 && b_bstride == 0) ? 1 : 0;
+    const uint64_t a_nb = p.a_shared ? 1 : static_cast<uint64_t>(nbatch), b_nb = p.b_shared ? 1 : static_cast<uint64_t>(nbatch);
+    const uint64_t a_bbytes = static_cast<uint64_t>(p.a_shared ? a_rows_stored * a_cols_stored : a_bstride) * 2;
+    const uint64_t b_bbytes = static_cast<uint64_t>(p.b_shared ? b_rows_stored * b_cols_stored : b_bstride) * 2;
     if (c_f32 && !pieces) {
         p.Cf = static_cast<float*>(C);
         p.C = nullptr;
@@ -156,14 +181,19 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
 
     CUtensorMap ma, mb;
     int rc;
-    if (p.a_mn_major) {
+    if (p.a_mn_major && nbatch > 1) {
+        uint64_t dims[3] = {static_cast<uint64_t>(g.M), static_cast<uint64_t>(g.K), a_nb};
+        uint64_t str[2] = {static_cast<uint64_t>(g.M) * 2, a_bbytes};
+        uint32_t box[3] = {64, 64, 1};
+        rc = get_tensor_map(ctx, A, 3, dims, str, box, &ma);
+    } else if (p.a_mn_major) {
         uint64_t dims[2] = {static_cast<uint64_t>(g.M), static_cast<uint64_t>(g.K)};
         uint64_t str[1] = {static_cast<uint64_t>(g.M) * 2};
         uint32_t box[2] = {64, 64};
         rc = get_tensor_map(ctx, A, 2, dims, str, box, &ma);
     } else if (nbatch > 1) {
-        uint64_t dims[3] = {static_cast<uint64_t>(k_cols), static_cast<uint64_t>(g.M), static_cast<uint64_t>(nbatch)};
-        uint64_t str[2] = {static_cast<uint64_t>(k_cols) * 2, static_cast<uint64_t>(k_cols) * 2 * g.M};
+        uint64_t dims[3] = {static_cast<uint64_t>(k_cols), static_cast<uint64_t>(g.M), a_nb};
+        uint64_t str[2] = {static_cast<uint64_t>(k_cols) * 2, a_bbytes};
         uint32_t box[3] = {64, 128, 1};
         rc = get_tensor_map(ctx, A, 3, dims, str, box, &ma);
     } else {
@@ -186,14 +216,19 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
             plan_grid = dp.grid;
         }
     }
-    if (p.b_mn_major) {
+    if (p.b_mn_major && nbatch > 1) {
+        uint64_t dims[3] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.K), b_nb};
+        uint64_t str[2] = {static_cast<uint64_t>(g.N) * 2, b_bbytes};
+        uint32_t box[3] = {64, 64, 1};
+        rc = get_tensor_map(ctx, B, 3, dims, str, box, &mb);
+    } else if (p.b_mn_major) {
         uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.K)};
         uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
         uint32_t box[2] = {64, 64};
         rc = get_tensor_map(ctx, B, 2, dims, str, box, &mb);
     } else if (nbatch > 1) {
-        uint64_t dims[3] = {static_cast<uint64_t>(k_cols), static_cast<uint64_t>(g.N), static_cast<uint64_t>(nbatch)};
-        uint64_t str[2] = {static_cast<uint64_t>(k_cols) * 2, static_cast<uint64_t>(k_cols) * 2 * g.N};
+        uint64_t dims[3] = {static_cast<uint64_t>(k_cols), static_cast<uint64_t>(g.N), b_nb};
+        uint64_t str[2] = {static_cast<uint64_t>(k_cols) * 2, b_bbytes};
         uint32_t box[3] = {64, static_cast<uint32_t>(cfg.tile_n), 1};
         rc = get_tensor_map(ctx, B, 3, dims, str, box, &mb);
     } else {
@@ -206,7 +241,7 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
 
     CUtensorMap mc = ma;   // unused unless the staged epilogue is on
     // the accumulate term is read by the direct-store epilogue (and by the split-K reduction) only
-    p.tma_store = (cfg.store_mode == 2 && cfg.split_k == 1 && p.vec_store && beta == 0.0f && !f32_result) ? 1 : 0;
+    p.tma_store = (cfg.store_mode == 2 && cfg.split_k == 1 && p.vec_store && beta == 0.0f && !f32_result && nbatch == 1) ? 1 : 0;
     if (p.tma_store) {
         uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.M)};
         uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
@@ -238,10 +273,11 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     }
     if (cfg.split_k > 1) {
         const long long MN = static_cast<long long>(g.M) * g.N;
-        const int vec8 = p.vec_store ? 1 : 0;
-        const long long work = vec8 ? MN / 8 : MN;
+        const int vec8 = (p.vec_store && MN % 8 == 0) ? 1 : 0;
+        const long long work = (vec8 ? MN / 8 : MN) * nbatch;
         const int grid = static_cast<int>(std::min<long long>(ceil_div(work, 256), 148LL * 16));
-        rc = launch_splitk_reduce(std::max(grid, 1), st, MN, static_cast<int>(g.N), cfg.split_k, p.partial, alpha, p.C, vec8, beta);
+        rc = launch_splitk_reduce(std::max(grid, 1), st, MN, static_cast<int>(g.N), cfg.split_k, p.partial, alpha, p.C, vec8, beta,
+                                  static_cast<int>(nbatch), out_batch_c);
         if (rc) return rc;
     }
     return TDX_OK;
@@ -697,6 +733,89 @@ int run_gemm_f32_pieces(DeviceCtx* ctx, const GemmProblem& g, float alpha, const
         }
     }
     return TDX_OK;
+}
+
+// Batched bf16 GEMM with accumulate on the tensor cores, all batches in one launch.
+//   direct: every batch's operands meet the copy engine's layout rules as they are -> 3-D tensor maps over the
+//           caller's buffers (contiguous dimension, the other one, batch), whatever the transposes.
+//   else:   both operands are first copied K-major with K padded to a multiple of 64 (pad_k_bf16_kernel, one launch for
+//           both; zeros add nothing to the sums), which removes every alignment rule -- the paper's K = 2305 qualifies --
+//           exactly as the fp32 piece path does.
+// Tile shape from the cost model's direct-store ranking of one batch's problem; K split only as far as it takes to give
+// every SM an item, reduced in a fixed order by one launch for all batches (it also applies beta).
+int run_gemm_batched_bf16(DeviceCtx* ctx, const GemmProblem& g, float alpha, float beta, const void* A, int64_t strideA,
+                          const void* B, int64_t strideB, void* C, int64_t strideC, int64_t batch, bool direct,
+                          cudaStream_t st) {
+    GemmProblem gg = g;
+    const void *pa = A, *pb = B;
+    PieceInfo form;
+    form.batch = batch;
+    form.batch_c = strideC;
+    const bool a_shared = batch > 1 && strideA == 0, b_shared = batch > 1 && strideB == 0;
+    if (direct) {
+        form.batch_a = strideA;
+        form.batch_b = strideB;
+    } else {
+        const int64_t Kp = ceil_div(g.K, 64) * 64;
+        const int64_t nb_a = a_shared ? 1 : batch, nb_b = b_shared ? 1 : batch;
+        const size_t a_bytes = static_cast<size_t>(g.M) * Kp * 2 * nb_a, b_bytes = static_cast<size_t>(g.N) * Kp * 2 * nb_b;
+        if (a_bytes > kPiecesMaxBytes || b_bytes > kPiecesMaxBytes || nb_a + nb_b > 65535 || ceil_div(std::max(g.M, g.N), 32) > 65535)
+            return TDX_ERR_UNSUPPORTED;            // the caller falls back to the generic kernel
+        void *da, *db;
+        int rc;
+        if ((rc = ensure_pieces(ctx, 0, a_bytes, &da))) return rc;
+        if ((rc = ensure_pieces(ctx, 1, b_bytes, &db))) return rc;
+        long long sa_i, sa_k, sb_k, sb_j;
+        gemm_strides(g, &sa_i, &sa_k, &sb_k, &sb_j);
+        tdx::PadOperand o0{static_cast<int>(g.M), sa_i, sa_k, strideA, static_cast<const __nv_bfloat16*>(A), static_cast<__nv_bfloat16*>(da)};
+        // rows of the copy of B are the columns j of op(B): element (j, k) at B[k * sb_k + j * sb_j]
+        tdx::PadOperand o1{static_cast<int>(g.N), sb_j, sb_k, strideB, static_cast<const __nv_bfloat16*>(B), static_cast<__nv_bfloat16*>(db)};
+        cudaLaunchConfig_t lc;
+        std::memset(&lc, 0, sizeof lc);
+        lc.gridDim = dim3(static_cast<unsigned>(Kp / 64), static_cast<unsigned>(ceil_div(std::max(g.M, g.N), 32)),
+                          static_cast<unsigned>(nb_a + nb_b));
+        lc.blockDim = dim3(256);
+        lc.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = attr;
+        lc.numAttrs = 1;
+        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::pad_k_bf16_kernel, static_cast<int>(g.K), static_cast<int>(Kp), static_cast<int>(nb_a), o0, o1));
+        TDX_CUDA(cudaGetLastError());
+        g_launches.fetch_add(1);
+        gg = GemmProblem{g.M, g.N, Kp, 0, 1, TDX_BF16};
+        pa = da;
+        pb = db;
+        form.cols = Kp;
+        form.batch_a = a_shared ? 0 : g.M * Kp;
+        form.batch_b = b_shared ? 0 : g.N * Kp;
+    }
+    tdx_config want;
+    std::memset(&want, 0, sizeof want);
+    want.kernel = TDX_KERNEL_UMMA;
+    want.store_mode = 1;          // direct stores: they carry the batch offset and the accumulate term
+    want.cta_pair = 1;
+    want.fit = 1;
+    tdx_config ranked;
+    if (model_pick_direct_store(gg, ctx->sm_count, ctx->smem_optin, &ranked)) {
+        want.tile_m = ranked.tile_m;
+        want.tile_n = ranked.tile_n;
+        want.raster = ranked.raster;
+        want.split_k = ranked.split_k;
+    }
+    tdx_config cfg;
+    int rc = resolve_gemm_config(gg, &want, ctx->sm_count, ctx->smem_optin, &cfg);
+    if (rc) return rc;
+    if (batch > 1) {
+        // the batches already multiply the tiles: split K only as far as it takes to give every SM an item
+        const int64_t num_kb = ceil_div(gg.K, 64);
+        const int64_t tiles = batch * ceil_div(g.M, cfg.tile_m) * ceil_div(g.N, cfg.tile_n);
+        int64_t sk = std::max<int64_t>(1, std::min<int64_t>({32, ctx->sm_count / std::max<int64_t>(1, tiles), num_kb / 4}));
+        while (sk > 1 && (sk - 1) * ceil_div(num_kb, sk) >= num_kb) --sk;
+        cfg.split_k = static_cast<int>(sk);
+    }
+    return run_gemm_umma(ctx, gg, alpha, pa, pb, C, cfg, nullptr, 0, true, st, beta, &form);
 }
 
 int run_gemm_generic(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,

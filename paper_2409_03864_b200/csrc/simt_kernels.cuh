@@ -385,12 +385,58 @@ __global__ void conv2d_generic_kernel(int Nimg, int H, int W, int Cin, int Cout,
 // Split-K reduction: out[i,j] = epilogue( sum_{s = 0..split-1, ascending} partial[s][i][j] ).
 // The order is fixed, so results do not depend on scheduling.
 // ---------------------------------------------------------------------------
+// Batched (batch > 1): partial is [batch][split][MN] and batch b of out starts batch_c elements after batch b - 1.
 __global__ void splitk_reduce_kernel(long long MN, int N, int split, const float* __restrict__ partial, float alpha,
                                      const float* __restrict__ bias, int relu, __nv_bfloat16* __restrict__ out,
-                                     int vec8, float beta = 0.0f) {
+                                     int vec8, float beta = 0.0f, int batch = 1, long long batch_c = 0) {
     // launched with programmatic stream serialization: this grid may start while the GEMM drains; wait here
     // until the GEMM grid has completed and its partial sums are visible (a no-op for an ordinary launch)
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (batch > 1) {
+        // one element (or one group of eight) per thread and pass, batches included; same fixed order of the splits
+        const long long per = vec8 ? MN / 8 : MN, total = per * batch;
+        for (long long gg = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; gg < total;
+             gg += static_cast<long long>(gridDim.x) * blockDim.x) {
+            const long long b = gg / per, g = gg - b * per;
+            const float* pb = partial + b * split * MN;
+            __nv_bfloat16* ob = out + b * batch_c;
+            if (vec8) {
+                const long long e = g * 8;
+                float acc[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
+                uint4 old = make_uint4(0u, 0u, 0u, 0u);
+                if (beta != 0.0f) old = *reinterpret_cast<const uint4*>(ob + e);
+#pragma unroll 4
+                for (int s = 0; s < split; ++s) {
+                    const float4* src = reinterpret_cast<const float4*>(pb + s * MN + e);
+                    const float4 v0 = __ldg(src), v1 = __ldg(src + 1);
+                    acc[0] += v0.x; acc[1] += v0.y; acc[2] += v0.z; acc[3] += v0.w;
+                    acc[4] += v1.x; acc[5] += v1.y; acc[6] += v1.z; acc[7] += v1.w;
+                }
+                const uint32_t ow[4] = {old.x, old.y, old.z, old.w};
+                uint32_t pk[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    float a = alpha * acc[2 * j], c = alpha * acc[2 * j + 1];
+                    if (beta != 0.0f) {
+                        a = fmaf(beta, __uint_as_float(ow[j] << 16), a);
+                        c = fmaf(beta, __uint_as_float(ow[j] & 0xFFFF0000u), c);
+                    }
+                    __nv_bfloat162 h = __floats2bfloat162_rn(a, c);
+                    pk[j] = *reinterpret_cast<uint32_t*>(&h);
+                }
+                *reinterpret_cast<uint4*>(ob + e) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+            } else {
+                float acc = 0.0f;
+                for (int s = 0; s < split; ++s) acc += __ldg(pb + s * MN + g);
+                float v = alpha * acc;
+                if (beta != 0.0f) v = fmaf(beta, __bfloat162float(ob[g]), v);
+                ob[g] = __float2bfloat16_rn(v);
+            }
+        }
+        return;
+    }
     if (vec8) {
         const long long groups = MN / 8;
         for (long long g = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; g < groups;
@@ -600,6 +646,70 @@ split_f32_bf16x3_kernel(int K, int Kp, int nb0, SplitOperand op0, SplitOperand o
             *reinterpret_cast<__nv_bfloat162*>(o) = hi;
             *reinterpret_cast<__nv_bfloat162*>(o + Kp) = mid;
             *reinterpret_cast<__nv_bfloat162*>(o + 2 * Kp) = lo;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// bf16 operand -> K-major copy with K padded to the MMA pipeline's K block: for operands whose layout the copy
+// engine cannot address (a row pitch that is no multiple of 16 bytes -- K = 2305 is the paper's own example -- or a
+// misaligned base).  Source: `rows` x K logical matrix, element (i, k) at src[b * batch_stride + i * s_row + k * s_k]
+// (either stride may be 1).  Destination, per batch: rows x Kp bf16, row-major, columns K..Kp-1 zero.  The padding
+// adds exact zeros to every sum, so the result is that of the unpadded reduction.  Same tiling as the fp32 piece
+// kernel below: 32 rows x 64 columns through shared memory, both operands of a GEMM in one launch.
+// ---------------------------------------------------------------------------
+struct PadOperand {
+    int rows;
+    long long s_row, s_k, batch_stride;
+    const __nv_bfloat16* src;
+    __nv_bfloat16* dst;
+};
+__global__ void __launch_bounds__(256)
+pad_k_bf16_kernel(int K, int Kp, int nb0, PadOperand op0, PadOperand op1) {
+    __shared__ __nv_bfloat16 tile[32][66];
+    const bool second = static_cast<int>(blockIdx.z) >= nb0;
+    const PadOperand& op = second ? op1 : op0;
+    const int rows = op.rows;
+    const long long s_row = op.s_row, s_k = op.s_k;
+    const int bz = static_cast<int>(blockIdx.z) - (second ? nb0 : 0);
+    // launched with programmatic stream serialization: the scratch copies are shared by successive calls, and the
+    // wait orders this kernel after everything the stream held before it
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int k0 = blockIdx.x * 64, r0 = blockIdx.y * 32;
+    if (r0 >= rows) return;                           // CTA-uniform: before any barrier
+    const __nv_bfloat16* s = op.src + bz * op.batch_stride;
+    __nv_bfloat16* d = op.dst + static_cast<long long>(bz) * rows * Kp;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;        // 32 x 8 threads
+    const __nv_bfloat16 zero = __float2bfloat16_rn(0.0f);
+    if (s_k == 1) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int jj = ty + 8 * j, r = r0 + jj;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int k = k0 + tx + 32 * h;
+                tile[jj][tx + 32 * h] = (r < rows && k < K) ? s[r * s_row + k] : zero;
+            }
+        }
+    } else {       // rows are the contiguous dimension of the source: read along them, transpose in shared memory
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int kk = ty + 8 * j, k = k0 + kk, r = r0 + tx;
+            tile[tx][kk] = (r < rows && k < K) ? s[r * s_row + k * s_k] : zero;
+        }
+    }
+    __syncthreads();
+    const int k = k0 + 2 * tx;                                     // Kp is a multiple of 64: a pair is all in or all out
+    if (k < Kp) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int jj = ty + 8 * j, r = r0 + jj;
+            if (r >= rows) continue;
+            __nv_bfloat162 v;
+            v.x = tile[jj][2 * tx];
+            v.y = tile[jj][2 * tx + 1];
+            *reinterpret_cast<__nv_bfloat162*>(d + static_cast<long long>(r) * Kp + k) = v;
         }
     }
 }

@@ -309,15 +309,26 @@ int gemm_dispatch(int64_t M, int64_t N, int64_t K, int transA, int transB, float
     tdx_config c;
     rc = resolve_gemm_config(g, cfg, ctx->sm_count, ctx->smem_optin, &c);
     if (rc) return rc;
+    // bf16 operands in a layout the copy engine cannot address (odd pitch, misaligned base): unless the caller asked
+    // for a kernel, problems of 2^21 multiply-adds and more are repacked K-major with K padded and run on the tensor
+    // cores (see run_gemm_batched_bf16); smaller ones stay on the generic kernel
+    auto unaligned_bf16 = [&]() -> int {
+        if (cfg == nullptr && dtype == TDX_BF16 && static_cast<double>(M) * N * K >= 2097152.0 && M < (1LL << 31) &&
+            N < (1LL << 31) && K < (1LL << 31)) {
+            const int r = run_gemm_batched_bf16(ctx, g, alpha, 0.0f, A, 0, B, 0, C, M * N, 1, false, st);
+            if (r != TDX_ERR_UNSUPPORTED) return r;
+        }
+        return run_gemm_generic(ctx, g, alpha, A, B, C, st);
+    };
     switch (c.kernel) {
         case TDX_KERNEL_SIMT: return run_gemm_simt_f32(ctx, g, alpha, A, B, C, st);
-        case TDX_KERNEL_GENERIC: return run_gemm_generic(ctx, g, alpha, A, B, C, st);
+        case TDX_KERNEL_GENERIC: return unaligned_bf16();
         default:
             if (dtype == TDX_F32) return run_gemm_f32_pieces(ctx, g, alpha, A, B, C, st, BatchArgs(), cfg);
             if (reinterpret_cast<uintptr_t>(A) % 16 || reinterpret_cast<uintptr_t>(B) % 16) {
                 if (cfg && cfg->kernel == TDX_KERNEL_UMMA)
                     return fail(TDX_ERR_ALIGNMENT, "tensor-core path needs 16-byte aligned A and B");
-                return run_gemm_generic(ctx, g, alpha, A, B, C, st);
+                return unaligned_bf16();
             }
             if (c.cta_pair == 2) return run_gemm_pair(ctx, g, alpha, A, B, C, c, st);
             return run_gemm_umma(ctx, g, alpha, A, B, C, c, ws, ws_bytes, internal_ws, st);
@@ -767,35 +778,39 @@ int tdx_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int transA,
         if (prefer_f32_pieces(g, batch)) return run_gemm_f32_pieces(ctx, g, alpha, A, B, C, st, ba, nullptr);
         return run_gemm_simt_f32(ctx, g, alpha, A, B, C, st, ba);
     }
-    // bf16: the tensor-core kernel, one launch per batch, when every batch's operands meet its layout rules
-    const bool aligned = gemm_umma_layout_ok(g) && reinterpret_cast<uintptr_t>(A) % 16 == 0 &&
-                         reinterpret_cast<uintptr_t>(B) % 16 == 0 && (strideA % 8 == 0) && (strideB % 8 == 0);
-    if (!aligned) return run_gemm_generic(ctx, g, alpha, A, B, C, st, ba);
-    tdx_config want;
-    std::memset(&want, 0, sizeof want);
-    if (beta != 0.0f) {
-        want.store_mode = 1;                        // the accumulate term is read by the direct-store epilogue
-        want.kernel = TDX_KERNEL_UMMA;
-        tdx_config ranked;                          // tile shape and K split: the cost model's direct-store choice
-        if (model_pick_direct_store(g, ctx->sm_count, ctx->smem_optin, &ranked)) {
-            want.tile_m = ranked.tile_m;
-            want.tile_n = ranked.tile_n;
-            want.split_k = ranked.split_k;
-            want.raster = ranked.raster;
+    // bf16: the tensor cores, all batches in one launch.  Operands whose layout the copy engine can address are read
+    // where they are; any others are first copied K-major with K padded (one more launch).  Tiny or oversized problems
+    // stay on the generic kernel.
+    const bool dims_ok = M < (1LL << 31) && N < (1LL << 31) && K < (1LL << 31) && strideA < (1LL << 38) && strideB < (1LL << 38) &&
+                         strideC < (1LL << 40);
+    const bool direct = gemm_umma_layout_ok(g) && reinterpret_cast<uintptr_t>(A) % 16 == 0 &&
+                        reinterpret_cast<uintptr_t>(B) % 16 == 0 && (strideA % 8 == 0) && (strideB % 8 == 0);
+    const bool worth_it = static_cast<double>(batch) * M * N * K >= 2097152.0;     // below 2^21 multiply-adds a launch is all there is
+    if (!dims_ok || (!direct && !worth_it)) return run_gemm_generic(ctx, g, alpha, A, B, C, st, ba);
+    if (batch == 1 && direct) {
+        // one batch in the tensor-core layout: the plain GEMM path (staged stores when there is no accumulate term)
+        tdx_config want;
+        std::memset(&want, 0, sizeof want);
+        if (beta != 0.0f) {
+            want.store_mode = 1;                        // the accumulate term is read by the direct-store epilogue
+            want.kernel = TDX_KERNEL_UMMA;
+            tdx_config ranked;                          // tile shape and K split: the cost model's direct-store choice
+            if (model_pick_direct_store(g, ctx->sm_count, ctx->smem_optin, &ranked)) {
+                want.tile_m = ranked.tile_m;
+                want.tile_n = ranked.tile_n;
+                want.split_k = ranked.split_k;
+                want.raster = ranked.raster;
+            }
         }
-    }
-    tdx_config cfg;
-    rc = resolve_gemm_config(g, beta != 0.0f ? &want : nullptr, ctx->sm_count, ctx->smem_optin, &cfg);
-    if (rc) return rc;
-    if (cfg.kernel != TDX_KERNEL_UMMA || cfg.cta_pair == 2) return run_gemm_generic(ctx, g, alpha, A, B, C, st, ba);
-    for (int64_t b = 0; b < batch; ++b) {
-        const char* a = static_cast<const char*>(A) + b * strideA * 2;
-        const char* bb = static_cast<const char*>(B) + b * strideB * 2;
-        char* c = static_cast<char*>(C) + b * strideC * 2;
-        rc = run_gemm_umma(ctx, g, alpha, a, bb, c, cfg, nullptr, 0, true, st, beta);
+        tdx_config cfg;
+        rc = resolve_gemm_config(g, beta != 0.0f ? &want : nullptr, ctx->sm_count, ctx->smem_optin, &cfg);
         if (rc) return rc;
+        if (cfg.kernel != TDX_KERNEL_UMMA || cfg.cta_pair == 2) return run_gemm_generic(ctx, g, alpha, A, B, C, st, ba);
+        return run_gemm_umma(ctx, g, alpha, A, B, C, cfg, nullptr, 0, true, st, beta);
     }
-    return TDX_OK;
+    rc = run_gemm_batched_bf16(ctx, g, alpha, beta, A, strideA, B, strideB, C, strideC, batch, direct, st);
+    if (rc == TDX_ERR_UNSUPPORTED) return run_gemm_generic(ctx, g, alpha, A, B, C, st, ba);
+    return rc;
 }
 
 int tdx_add_zero_pad(int64_t N, int64_t H, int64_t W, int64_t C, int pad_top, int pad_bottom, int pad_left, int pad_right,

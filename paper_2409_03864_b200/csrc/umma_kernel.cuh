@@ -90,6 +90,7 @@ struct UmmaParams {
     // are laid out [batch][split][M][N]
     int batch;
     long long batch_c;
+    int a_shared, b_shared;   // batched: the operand is one matrix shared by all batches (its tensor has one batch)
     const int4* tiles;
     int rounds;
     int b_box;                // rows of one B copy (K-major B); bn when there is no table
@@ -231,9 +232,19 @@ __device__ __forceinline__ void issue_kblock(const UmmaParams& p, const CUtensor
         kbb = p.b_seg[sg] * p.seg_kb + r;
     }
     if (p.batch > 1) {
-        // batched: K-major 3-D operands; rows past M or N of a batch are zero-filled, not the next batch's
-        for (int h = 0; h < mh; ++h) ld3(a_dst + h * kHalfABytes, tmA, ka * kBK, t.m_blk * p.bm + h * kHalfM, t.batch);
-        for (int r0 = 0; r0 < t.bn; r0 += p.b_box) ld3(b_dst + r0 * 128, tmB, kbb * kBK, t.n0 + r0, t.batch);
+        // batched: 3-D operands (contiguous dimension, the other one, batch); rows past M or N of a batch are
+        // zero-filled, never the next batch's
+        const int ba = p.a_shared ? 0 : t.batch, bb = p.b_shared ? 0 : t.batch;
+        if (p.a_mn_major) {
+            for (int i = 0; i < 2 * mh; ++i) ld3(a_dst + i * 8192, tmA, t.m_blk * p.bm + i * 64, ka * kBK, ba);
+        } else {
+            for (int h = 0; h < mh; ++h) ld3(a_dst + h * kHalfABytes, tmA, ka * kBK, t.m_blk * p.bm + h * kHalfM, ba);
+        }
+        if (p.b_mn_major) {
+            for (int i = 0; i < t.bn / 64; ++i) ld3(b_dst + i * 8192, tmB, t.n0 + i * 64, kbb * kBK, bb);
+        } else {
+            for (int r0 = 0; r0 < t.bn; r0 += p.b_box) ld3(b_dst + r0 * 128, tmB, kbb * kBK, t.n0 + r0, bb);
+        }
         return;
     }
     if (p.a_mn_major) {
@@ -511,17 +522,17 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                 }
             } else {
                 float v[32];
+                __nv_bfloat16* const c_row = p.C + t.batch * p.batch_c + grow * p.ldc + col0;
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     float x = p.alpha * __uint_as_float(r[j]);
-                    if (p.beta != 0.0f && col0 + j < p.N)
-                        x = fmaf(p.beta, __bfloat162float(p.C[grow * p.ldc + col0 + j]), x);
+                    if (p.beta != 0.0f && col0 + j < p.N) x = fmaf(p.beta, __bfloat162float(c_row[j]), x);
                     if (p.bias != nullptr && col0 + j < p.N) x += __ldg(p.bias + col0 + j);
                     if (p.residual != nullptr && col0 + j < p.N) x += __bfloat162float(p.residual[grow * p.ldc + col0 + j]);
                     if (p.relu) x = fmaxf(x, 0.0f);
                     v[j] = x;
                 }
-                __nv_bfloat16* dst = p.C + grow * p.ldc + col0;
+                __nv_bfloat16* dst = c_row;
                 if (p.vec_store) {
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
