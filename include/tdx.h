@@ -95,6 +95,12 @@ typedef struct {
                     /*     the cost model predicts a gain of at least 3 %.  The first call for a shape on a  */
                     /*     device allocates a small tile table there and copies it synchronously (cudaMalloc */
                     /*     + cudaMemcpy): make that call before any stream capture.                          */
+                    /*     3 = (GEMM, few tiles and a long reduction; split_k = 1, store_mode = 1, tile_n a      */
+                    /*     multiple of 64) the tiles x K blocks units are dealt evenly to ALL CTAs instead of a  */
+                    /*     uniform K split, whose item count rarely fills the SMs; a tile cut by a CTA boundary   */
+                    /*     is completed from fp32 partial tiles in ascending K order by a reduction launch.       */
+                    /*     Needs the workspace tdx_gemm_workspace_size reports (the library's own when none is   */
+                    /*     passed); same first-call table upload as 2.                                           */
 } tdx_config;
 
 /*
@@ -313,6 +319,17 @@ int tdx_default_conv2d_config(int64_t N, int64_t H, int64_t W, int64_t Cin, int6
  */
 int tdx_gemm_tile_plan(int64_t M, int64_t N, int64_t K, int tile_m, int tile_n, int raster, int ctas, int* table,
                        int cap_tiles, int* n_rounds, int* n_ctas, double* model_cycles, double* model_cycles_uniform);
+
+/*
+ * The plan `fit = 3` would use on `ctas` persistent CTAs (host only): the tiles x K blocks units of the problem, tile
+ * after tile, cut into `ctas` nearly equal runs, so that every SM streams its share of the operands of a problem with
+ * few tiles and a long reduction (Case Study 5 tiles the reduction loop too; here the cut points follow the machine,
+ * not a divisor of K).  table (may be NULL) receives up to cap_entries groups of six ints, entry [round * n_ctas + cta]
+ * = (row block, first column, width, first K block, end K block, partial slot); width 0 = no entry.  max_slots is the
+ * largest number of pieces any tile is cut into, i.e. the workspace holds max_slots * M * N floats.
+ */
+int tdx_gemm_k_balanced_plan(int64_t M, int64_t N, int64_t K, int tile_m, int tile_n, int ctas, int* table, int cap_entries,
+                             int* n_rounds, int* n_ctas, int* max_slots);
 
 /* Persist / restore the tuning cache (a small JSON text file). */
 int tdx_tune_save(const char* json_path);

@@ -94,6 +94,7 @@ def lib() -> ctypes.CDLL:
         L.tdx_set_autotune.argtypes = [ci]
         dp = ctypes.POINTER(ctypes.c_double)
         L.tdx_gemm_tile_plan.argtypes = [i64, i64, i64, ci, ci, ci, ci, ip, ci, ip, ip, dp, dp]
+        L.tdx_gemm_k_balanced_plan.argtypes = [i64, i64, i64, ci, ci, ci, ip, ci, ip, ip, ip]
         L.tdx_gemm_splitk_static.argtypes = [i64, i64, i64, ci, ci, cf, vp, vp, vp, ci, ci, vp]
         L.tdx_check_device_status.argtypes = [vp]
         L.tdx_selftest_bounded_wait.argtypes = [ci, vp]
@@ -119,7 +120,7 @@ EXPORTS = (
     "tdx_gemm", "tdx_gemm_f32out", "tdx_add_zero_pad", "tdx_add_zero_pad_host", "tdx_gemm_batched", "tdx_gemm_batched_host", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_add_relu", "tdx_conv2d_bias_relu_ex",
     "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_gemm_guided", "tdx_model_gemm_us", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
     "tdx_enum_conv2d_configs", "tdx_default_gemm_config", "tdx_default_conv2d_config", "tdx_tune_save",
-    "tdx_tune_load", "tdx_tune_clear", "tdx_set_autotune", "tdx_gemm_tile_plan", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
+    "tdx_tune_load", "tdx_tune_clear", "tdx_set_autotune", "tdx_gemm_tile_plan", "tdx_gemm_k_balanced_plan", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
     "tdx_version",
 )
 
@@ -337,6 +338,17 @@ def tdx_gemm_tile_plan(M, N, K, tile_m=256, tile_n=256, raster=0, ctas=148, cap_
     tiles = [[(table[3 * (r * used.value + c)], table[3 * (r * used.value + c) + 1], table[3 * (r * used.value + c) + 2])
               for c in range(used.value)] for r in range(rounds.value)]
     return st, rounds.value, used.value, tiles, fit.value, uni.value
+
+
+def tdx_gemm_k_balanced_plan(M, N, K, tile_m=128, tile_n=128, ctas=148, cap_entries=1 << 14):
+    """-> (status, rounds, ctas_used, entries, max_slots); entries[round][cta] = (row block, first column, width,
+    first K block, end K block, partial slot), width 0 = no entry."""
+    table = (ctypes.c_int * (6 * cap_entries))()
+    rounds, used, slots = ctypes.c_int(0), ctypes.c_int(0), ctypes.c_int(0)
+    st = lib().tdx_gemm_k_balanced_plan(M, N, K, tile_m, tile_n, ctas, table, cap_entries, ctypes.byref(rounds), ctypes.byref(used),
+                                        ctypes.byref(slots))
+    ent = [[tuple(table[6 * (r * used.value + c) + i] for i in range(6)) for c in range(used.value)] for r in range(rounds.value)]
+    return st, rounds.value, used.value, ent, slots.value
 
 
 TDX_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024

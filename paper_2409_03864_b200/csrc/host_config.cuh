@@ -135,7 +135,15 @@ const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num
         if ((c.split_k - 1) * per >= num_kb) return "split_k leaves an empty K slice";
     }
     if (c.raster < 0) return "raster must be >= 0";
-    if (c.fit < 0 || c.fit > 2) return "fit must be 0 (choose), 1 (uniform tiles) or 2 (tile widths fitted to the CTA count)";
+    if (c.fit < 0 || c.fit > 3)
+        return "fit must be 0 (choose), 1 (uniform tiles), 2 (tile widths fitted to the CTA count) or 3 (K blocks dealt evenly to all CTAs)";
+    if (c.fit == 3) {
+        if (conv || c.cta_pair == 2) return "the K-balanced plan is implemented for the single-CTA GEMM only";
+        if (c.split_k != 1) return "the K-balanced plan replaces split_k: leave it at 1";
+        if (c.store_mode != 1) return "the K-balanced plan writes fp32 partial tiles: use store_mode 1";
+        if (num_kb > 4095) return "reduction too long for the K-balanced plan";
+        if (c.tile_n % 64) return "the K-balanced plan loads B in 64-row copies: tile_n must be a multiple of 64";
+    }
     if (c.k_stagger != 0 && c.k_stagger != 1) return "k_stagger must be 0 or 1";
     return nullptr;
 }

@@ -168,6 +168,28 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     }
     const bool f32_result = pieces != nullptr || c_f32;
 
+    // K-balanced plan: the tiles x K blocks units dealt evenly to all CTAs; partial tiles in up to max_seg slots
+    DevicePlan kplan;
+    const bool k_balanced = cfg.fit == 3 && !f32_result && nbatch == 1 && beta == 0.0f;
+    if (cfg.fit == 3 && !k_balanced) return fail(TDX_ERR_CONFIG, "the K-balanced plan serves the plain bf16 GEMM only");
+    if (k_balanced) {
+        int rcp = get_k_balanced_plan(ctx, g.M, g.N, num_kb, cfg.tile_m, cfg.tile_n, &kplan);
+        if (rcp) return rcp;
+        if (!kplan.fitted) return fail(TDX_ERR_CONFIG, "no K-balanced plan for this shape");
+        const size_t need = static_cast<size_t>(kplan.max_seg) * g.M * g.N * sizeof(float);
+        if (internal_ws) {
+            int rcw = ensure_ws(ctx, need, &ws);
+            if (rcw) return rcw;
+        } else if (ws == nullptr || ws_bytes < need || reinterpret_cast<uintptr_t>(ws) % 256) {
+            return fail(TDX_ERR_WORKSPACE, "the K-balanced plan needs %zu bytes of 256-byte aligned workspace", need);
+        }
+        p.partial = static_cast<float*>(ws);
+        p.split_k = kplan.max_seg > 1 ? kplan.max_seg : 2;      // > 1: the epilogue writes partial tiles to their slots
+        p.kb_per_split = p.num_kb;
+        p.tiles = kplan.dev;
+        p.rounds = kplan.rounds;
+        p.b_box = 64;
+    }
     if (cfg.split_k > 1) {
         const size_t need = static_cast<size_t>(cfg.split_k) * g.M * g.N * sizeof(float) * nbatch;
         if (internal_ws) {
@@ -205,7 +227,7 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
     if (rc) return rc;
     // tile widths fitted to the number of CTAs (see plan_fitted_tiles): B then arrives in 64-row copies
     int plan_grid = 0;
-    if (cfg.fit != 1 && cfg.split_k == 1 && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0 && nbatch == 1) {
+    if (cfg.fit != 1 && cfg.fit != 3 && cfg.split_k == 1 && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0 && nbatch == 1) {
         DevicePlan dp;
         rc = get_tile_plan(ctx, g.M, g.N, num_kb, cfg.tile_m, cfg.tile_n, cfg.raster, cfg.fit == 2 ? 0.0 : 0.03, &dp);
         if (rc) return rc;
@@ -249,8 +271,28 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         rc = get_tensor_map(ctx, C, 2, dims, str, box, &mc, 64);
         if (rc) return rc;
     }
+    if (k_balanced) plan_grid = kplan.grid;
     rc = launch_umma(ctx, false, ma, mb, mc, p, st, false, nullptr, nullptr, plan_grid);
     if (rc) return rc;
+    if (k_balanced) {
+        const long long MN = static_cast<long long>(g.M) * g.N;
+        const int vec8 = (p.vec_store && cfg.tile_n % 8 == 0) ? 1 : 0;
+        const long long work = vec8 ? MN / 8 : MN;
+        cudaLaunchConfig_t lc;
+        std::memset(&lc, 0, sizeof lc);
+        lc.gridDim = dim3(static_cast<unsigned>(std::max<long long>(1, std::min<long long>(ceil_div(work, 256), 148LL * 16))));
+        lc.blockDim = dim3(256);
+        lc.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = attr;
+        lc.numAttrs = 1;
+        TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::splitk_reduce_var_kernel, MN, static_cast<int>(g.N), cfg.tile_m, cfg.tile_n, kplan.tiles_n,
+                                    kplan.nseg, static_cast<const float*>(p.partial), alpha, p.C, vec8, 0.0f));
+        g_launches.fetch_add(1);
+        return TDX_OK;
+    }
     if (cfg.split_k > 1 && f32_result) {
         // fp32 result: partial sums (fp32, dense) -> alpha * sum + beta * C
         const long long MN = static_cast<long long>(g.M) * g.N;

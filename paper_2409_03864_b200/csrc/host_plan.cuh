@@ -131,13 +131,69 @@ bool plan_fitted_tiles(int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int
     return true;
 }
 
+// K-balanced plan (fit = 3), for problems with few tiles and a long reduction (the HBM-bound skinny shapes): the
+// tiles x K blocks units, tile after tile, are cut into g nearly equal runs, one per CTA, so that every SM streams its
+// share of the operands -- a uniform K split leaves SMs idle whenever tiles x splits is no multiple of the SM count
+// (128 x 8192 x 8192: 43 tiles x 3 splits = 129 items on 148 SMs).  A run that crosses a tile boundary becomes two
+// entries; a boundary that would leave a piece shorter than `min_len` K blocks snaps to the tile boundary (a partial
+// tile costs its fp32 store and reload whatever its length).  Every piece writes an fp32 partial tile to its slot
+// (ascending K within the tile); nseg[tile] slots are summed by splitk_reduce_var_kernel.
+struct KBalancedPlan {
+    std::vector<int4> table;   // [round * grid + cta] = (row block, first column, width, kb0 | kb1 << 12 | slot << 24)
+    std::vector<int> nseg;     // per tile (row block * tiles_n + column tile)
+    int rounds = 0, grid = 0, max_seg = 0, tiles_n = 0;
+};
+bool plan_k_balanced(int64_t M, int64_t N, int64_t num_kb, int bm, int bn, int g, KBalancedPlan* out, int min_len = 4) {
+    const int64_t tiles_m = ceil_div(M, bm), tiles_n = ceil_div(N, bn), T = tiles_m * tiles_n, U = T * num_kb;
+    if (num_kb < 1 || num_kb > 4095 || T < 1 || g < 1 || T > (1 << 20)) return false;
+    const int64_t G = std::max<int64_t>(1, std::min<int64_t>(g, U / std::max(1, min_len)));      // no run shorter than min_len
+    std::vector<int64_t> cut(G + 1);
+    for (int64_t c = 0; c <= G; ++c) {
+        int64_t b = (c * U + G / 2) / G;                           // even share, rounded
+        const int64_t r = b % num_kb;
+        if (c > 0 && c < G && r != 0) {                            // keep pieces at least min_len long
+            if (r < min_len) b -= r;
+            else if (num_kb - r < min_len) b += num_kb - r;
+        }
+        cut[c] = b;
+    }
+    std::vector<std::vector<int4>> per(G);
+    out->nseg.assign(T, 0);
+    for (int64_t c = 0; c < G; ++c) {
+        int64_t u = cut[c];
+        while (u < cut[c + 1]) {
+            const int64_t tile = u / num_kb, kb0 = u % num_kb, kb1 = std::min<int64_t>(num_kb, kb0 + (cut[c + 1] - u));
+            const int slot = out->nseg[tile]++;
+            if (slot > 127) return false;
+            const int64_t m_blk = tile / tiles_n, n_blk = tile % tiles_n;
+            const int width = static_cast<int>(std::min<int64_t>(bn, ceil_div(N - n_blk * bn, 64) * 64));
+            per[c].push_back(make_int4(static_cast<int>(m_blk), static_cast<int>(n_blk * bn), width,
+                                       static_cast<int>(kb0 | (kb1 << 12) | (static_cast<int64_t>(slot) << 24))));
+            u += kb1 - kb0;
+        }
+    }
+    size_t rounds = 0;
+    for (auto& v : per) rounds = std::max(rounds, v.size());
+    out->grid = static_cast<int>(G);
+    out->rounds = static_cast<int>(rounds);
+    out->tiles_n = static_cast<int>(tiles_n);
+    out->max_seg = *std::max_element(out->nseg.begin(), out->nseg.end());
+    out->table.assign(rounds * G, make_int4(0, 0, 0, 0));
+    for (int64_t c = 0; c < G; ++c)
+        for (size_t k = 0; k < per[c].size(); ++k) out->table[k * G + c] = per[c][k];
+    return true;
+}
+
 // Device copies of tile plans, one per (device, shape, tile, CTA count); never freed (a few KB each).
 struct PlanKey {
     int64_t M, N, num_kb;
     int dev, bm, bn, raster, g, forced, pair;
     bool operator<(const PlanKey& o) const { return std::memcmp(this, &o, sizeof(PlanKey)) < 0; }
 };
-struct DevicePlan { int4* dev = nullptr; int rounds = 0, grid = 0; bool fitted = false; };
+struct DevicePlan {
+    int4* dev = nullptr; int rounds = 0, grid = 0; bool fitted = false;
+    const int* nseg = nullptr; int max_seg = 0, tiles_n = 0;      // K-balanced plans only (nseg follows the table on the device)
+};
 std::map<PlanKey, DevicePlan> g_plans;
 
 // Looks the plan up.  First use of a shape on a device builds the plan, allocates its table on that device and
@@ -166,6 +222,41 @@ int get_tile_plan(DeviceCtx* ctx, int64_t M, int64_t N, int64_t num_kb, int bm, 
         d.dev = static_cast<int4*>(dev);
         d.rounds = plan.rounds;
         d.grid = plan.grid;
+    }
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        g_plans[key] = d;
+    }
+    *out = d;
+    return TDX_OK;
+}
+
+// The K-balanced plan of a shape on this device (built, uploaded and cached like the fitted tile plans).
+int get_k_balanced_plan(DeviceCtx* ctx, int64_t M, int64_t N, int64_t num_kb, int bm, int bn, DevicePlan* out) {
+    PlanKey key;
+    std::memset(&key, 0, sizeof key);
+    key.M = M; key.N = N; key.num_kb = num_kb; key.dev = ctx->dev; key.bm = bm; key.bn = bn; key.g = ctx->sm_count;
+    key.forced = 3;                                           // plan kind
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        auto it = g_plans.find(key);
+        if (it != g_plans.end()) { *out = it->second; return TDX_OK; }
+    }
+    KBalancedPlan plan;
+    DevicePlan d;
+    d.fitted = plan_k_balanced(M, N, num_kb, bm, bn, ctx->sm_count, &plan);
+    if (d.fitted) {
+        const size_t tbytes = plan.table.size() * sizeof(int4), nbytes = plan.nseg.size() * sizeof(int);
+        void* dev = nullptr;
+        TDX_CUDA(cudaMalloc(&dev, tbytes + nbytes));
+        TDX_CUDA(cudaMemcpy(dev, plan.table.data(), tbytes, cudaMemcpyHostToDevice));
+        TDX_CUDA(cudaMemcpy(static_cast<char*>(dev) + tbytes, plan.nseg.data(), nbytes, cudaMemcpyHostToDevice));
+        d.dev = static_cast<int4*>(dev);
+        d.nseg = reinterpret_cast<const int*>(static_cast<char*>(dev) + tbytes);
+        d.rounds = plan.rounds;
+        d.grid = plan.grid;
+        d.max_seg = plan.max_seg;
+        d.tiles_n = plan.tiles_n;
     }
     {
         std::lock_guard<std::mutex> lk(g_mu);
@@ -210,7 +301,23 @@ double model_gemm_us(const GemmProblem& g, const tdx_config& c, int sm_count) {
         const double per_tile = overlapped ? std::max(main_loop, epi) : main_loop + epi;
         cycles = 5500.0 + rounds * per_tile + (overlapped ? epi : 0.0) + (pair ? 4000.0 : 0.0);
     }
+    int kbal_slots = 0;
+    if (c.fit == 3 && !pair) {
+        // K-balanced: every CTA walks its even share of the tiles x K blocks units; a CTA's run touches one or two
+        // tiles, each of which costs it a partial-tile epilogue
+        KBalancedPlan kp;
+        if (plan_k_balanced(g.M, g.N, num_kb, tm, bn, sm_count, &kp)) {
+            const double units = static_cast<double>(ceil_div(g.M, tm) * ceil_div(g.N, bn)) * num_kb / kp.grid;
+            cycles = 5500.0 + units * std::max(mma, l2) + kp.rounds * 1.5 * 1200.0 * std::ceil(blocks / (4.0 * halves));
+            kbal_slots = kp.max_seg;
+        }
+    }
     double us = cycles / clk_mhz;
+    if (kbal_slots > 0) {
+        const double tiles_out = static_cast<double>(ceil_div(g.M, tm) * ceil_div(g.N, bn));
+        const double avg_seg = (tiles_out + sm_count) / tiles_out;      // each CTA boundary adds one piece
+        us += 2.0 + (avg_seg * g.M * g.N * 4.0 * 2.0 + g.M * g.N * 2.0) / 8.0e6;
+    }
     // split-K: the reduction kernel's launch hides behind the GEMM's tail and the partial sums are still in L2 when it
     // reads them (128 x 8192 x 8192 in three splits: about 4 us on top of the GEMM kernel)
     if (split > 1) us += 2.0 + (static_cast<double>(split) * g.M * g.N * 4.0 * 2.0 + g.M * g.N * 2.0) / 8.0e6;

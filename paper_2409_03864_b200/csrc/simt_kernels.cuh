@@ -483,6 +483,53 @@ __global__ void splitk_reduce_kernel(long long MN, int N, int split, const float
     }
 }
 
+// The same reduction for the K-balanced plan, where the number of partial tiles differs from tile to tile:
+// nseg[row block * tiles_n + column tile] slots hold that tile's partial sums (slot s at partial + s * MN), added in
+// ascending slot order = ascending K.  Tiles are bm rows x bn columns (bn a multiple of 8).
+__global__ void splitk_reduce_var_kernel(long long MN, int N, int bm, int bn, int tiles_n, const int* __restrict__ nseg,
+                                         const float* __restrict__ partial, float alpha, __nv_bfloat16* __restrict__ out,
+                                         int vec8, float beta) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const long long per = vec8 ? MN / 8 : MN;
+    for (long long g = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; g < per;
+         g += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const long long e = vec8 ? g * 8 : g;
+        const long long row = e / N;
+        const int col = static_cast<int>(e - row * N);
+        const int split = __ldg(nseg + (row / bm) * tiles_n + col / bn);
+        if (vec8) {
+            float acc[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
+#pragma unroll 4
+            for (int s = 0; s < split; ++s) {
+                const float4* src = reinterpret_cast<const float4*>(partial + s * MN + e);
+                const float4 v0 = __ldg(src), v1 = __ldg(src + 1);
+                acc[0] += v0.x; acc[1] += v0.y; acc[2] += v0.z; acc[3] += v0.w;
+                acc[4] += v1.x; acc[5] += v1.y; acc[6] += v1.z; acc[7] += v1.w;
+            }
+            uint32_t pk[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float a = alpha * acc[2 * j], b = alpha * acc[2 * j + 1];
+                if (beta != 0.0f) {
+                    a = fmaf(beta, __bfloat162float(out[e + 2 * j]), a);
+                    b = fmaf(beta, __bfloat162float(out[e + 2 * j + 1]), b);
+                }
+                __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+                pk[j] = *reinterpret_cast<uint32_t*>(&h);
+            }
+            *reinterpret_cast<uint4*>(out + e) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+        } else {
+            float acc = 0.0f;
+            for (int s = 0; s < split; ++s) acc += __ldg(partial + s * MN + e);
+            float v = alpha * acc;
+            if (beta != 0.0f) v = fmaf(beta, __bfloat162float(out[e]), v);
+            out[e] = __float2bfloat16_rn(v);
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------
 // add(zero_pad(x), y) without the padded copy and without adding the zeros: out = y, plus x inside the interior.
 // x is N x H x W x C, y / out are N x Hp x Wp x C.  An interior row (n, h) is W * C contiguous elements in x and

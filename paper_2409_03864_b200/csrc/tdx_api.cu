@@ -76,7 +76,7 @@ bool model_default_gemm(const GemmProblem& g, int sm_count, int smem_limit, tdx_
             pick.first = false;
             std::memset(&pick.second, 0, sizeof pick.second);
             for (const tdx_config& c : cands) {
-                if (c.cta_pair == 2) continue;
+                if (c.cta_pair == 2 || c.fit == 3) continue;      // chosen by measurement only (tuning cache, search)
                 const double us = model_gemm_us(g, c, sm_count);
                 if (!pick.first || us < best_us) { pick.first = true; pick.second = c; best_us = us; }
             }
@@ -105,7 +105,7 @@ bool model_pick_direct_store(const GemmProblem& g, int sm_count, int smem_limit,
         std::memset(&pick.second, 0, sizeof pick.second);
         double best_us = 0.0;
         for (tdx_config c : cands) {
-            if (c.cta_pair == 2 || c.k_stagger != 0) continue;
+            if (c.cta_pair == 2 || c.k_stagger != 0 || c.fit == 3) continue;
             c.store_mode = 1;
             c.fit = 1;
             const double us = model_gemm_us(g, c, sm_count);
@@ -166,7 +166,7 @@ int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_cou
     if (c.tile_n == 0) c.tile_n = d.tile_n;
     if (c.split_k == 0) c.split_k = (user && user->cta_pair == 2) ? 1 : (user && user->tile_n != 0 && user->tile_n != d.tile_n) ? 1 : d.split_k;
     if (c.store_mode == 0) {
-        c.store_mode = (c.split_k == 1 && g.N % 8 == 0) ? 2 : 1;
+        c.store_mode = (c.split_k == 1 && g.N % 8 == 0 && c.fit != 3) ? 2 : 1;
         if (c.store_mode == 2 && c.cta_pair != 2 && c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, 2)) c.store_mode = 1;
     }
     if (c.stages == 0)
@@ -416,6 +416,20 @@ void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int 
                                 }
                             }
                 }
+            // K blocks dealt evenly to all CTAs, for problems with few tiles and a long reduction
+            if (!conv && bn % 64 == 0 && bn >= 128 && tiles < 2LL * sm_count && tiles * num_kb >= 4LL * sm_count && num_kb <= 4095) {
+                const int max_st = umma_max_stages(tm, bn, smem_limit, 1);
+                for (int st : {max_st, max_st - 2}) {
+                    if (st < 3) continue;
+                    tdx_config c;
+                    std::memset(&c, 0, sizeof c);
+                    c.kernel = TDX_KERNEL_UMMA;
+                    c.tile_m = tm; c.tile_n = bn; c.tile_k = 64; c.stages = st; c.cta_pair = 1;
+                    c.split_k = 1; c.store_mode = 1; c.raster = 0; c.fit = 3;
+                    if (umma_config_reason(c, b_mn, num_kb, smem_limit, conv, N) != nullptr) continue;
+                    out->push_back(c);
+                }
+            }
         }
     }
 }
@@ -882,7 +896,7 @@ int tdx_add_zero_pad(int64_t N, int64_t H, int64_t W, int64_t C, int pad_top, in
 int tdx_gemm_ex(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype, const void* A,
                 const void* B, void* C, void* stream, const tdx_config* cfg, void* workspace, size_t workspace_bytes) {
     // the library's own workspace serves every split-K it chose itself
-    const bool internal = (workspace == nullptr) && (cfg == nullptr || cfg->split_k == 0);
+    const bool internal = (workspace == nullptr) && (cfg == nullptr || cfg->split_k == 0 || cfg->fit == 3);
     return gemm_dispatch(M, N, K, transA, transB, alpha, dtype, A, B, C, stream, cfg, workspace, workspace_bytes, internal);
 }
 
@@ -892,6 +906,15 @@ int tdx_gemm_workspace_size(int64_t M, int64_t N, int64_t K, int dtype, const td
     if (dtype != TDX_F32 && dtype != TDX_BF16) return fail(TDX_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     const int split = cfg ? std::max(cfg->split_k, 1) : 1;
     *bytes = split > 1 ? static_cast<size_t>(split) * M * N * sizeof(float) : 0;
+    if (cfg && cfg->fit == 3 && M > 0 && N > 0 && K > 0) {
+        // K-balanced plan: as many slots as the most finely cut tile has pieces (depends on the SM count)
+        int sm_count, smem_limit;
+        device_limits(&sm_count, &smem_limit);
+        KBalancedPlan plan;
+        const int tm = cfg->tile_m ? cfg->tile_m : 128, tn = cfg->tile_n ? cfg->tile_n : 128;
+        if (!plan_k_balanced(M, N, ceil_div(K, 64), tm, tn, sm_count, &plan)) return fail(TDX_ERR_CONFIG, "no K-balanced plan for this shape");
+        *bytes = static_cast<size_t>(plan.max_seg) * M * N * sizeof(float);
+    }
     return TDX_OK;
 }
 
@@ -1438,6 +1461,28 @@ int tdx_gemm_tile_plan(int64_t M, int64_t N, int64_t K, int tile_m, int tile_n, 
             table[3 * i] = plan.table[i].x;
             table[3 * i + 1] = plan.table[i].y;
             table[3 * i + 2] = plan.table[i].z;
+        }
+    return TDX_OK;
+}
+
+int tdx_gemm_k_balanced_plan(int64_t M, int64_t N, int64_t K, int tile_m, int tile_n, int ctas, int* table, int cap_entries,
+                             int* n_rounds, int* n_ctas, int* max_slots) {
+    if (M <= 0 || N <= 0 || K <= 0 || ctas <= 0 || (tile_m != 128 && tile_m != 256) || tile_n < 64 || tile_n > 256 || tile_n % 64)
+        return fail(TDX_ERR_INVALID_ARG, "tdx_gemm_k_balanced_plan: bad argument");
+    KBalancedPlan plan;
+    if (!plan_k_balanced(M, N, ceil_div(K, 64), tile_m, tile_n, ctas, &plan)) return fail(TDX_ERR_CONFIG, "no K-balanced plan for this shape");
+    if (n_rounds) *n_rounds = plan.rounds;
+    if (n_ctas) *n_ctas = plan.grid;
+    if (max_slots) *max_slots = plan.max_seg;
+    if (table)
+        for (size_t i = 0; i < plan.table.size() && static_cast<int>(i) < cap_entries; ++i) {
+            const int4 e = plan.table[i];
+            table[6 * i] = e.x;
+            table[6 * i + 1] = e.y;
+            table[6 * i + 2] = e.z;
+            table[6 * i + 3] = e.w & 0xFFF;
+            table[6 * i + 4] = (e.w >> 12) & 0xFFF;
+            table[6 * i + 5] = (e.w >> 24) & 0x7F;
         }
     return TDX_OK;
 }

@@ -77,8 +77,11 @@ struct UmmaParams {
     // Tile table (GEMM, optional): instead of a uniform grid of bm x bn tiles, the output is cut into tiles of
     // bm rows and individually chosen widths (multiples of b_box, at most bn), and the host has already dealt
     // them to the CTAs (CTA pairs for the pair kernel): entry [round * workers + worker] = (row block, first
-    // column, width, 0); width 0 ends a worker's list.  This is how a tile count that does not fill the last
-    // wave of CTAs is evened out.
+    // column, width, w); width 0 ends a worker's list.  This is how a tile count that does not fill the last
+    // wave of CTAs is evened out.  w = 0: the whole reduction of the tile; otherwise (K-balanced plan, few tiles and
+    // a long reduction) K blocks [w & 0xFFF, (w >> 12) & 0xFFF) of it, whose fp32 partial tile goes to slot
+    // (w >> 24) & 0x7F of the split-K workspace: the (tile, K block) units are dealt evenly to ALL CTAs, a tile cut
+    // by a CTA boundary is completed by the reduction kernel in ascending slot order.
     // fp32 GEMM from bf16 pieces (seg_kb > 0): the operands hold three pieces side by side (seg_kb K blocks each) and the
     // reduction walks six piece pairs: K block kb reads piece a_seg[kb / seg_kb] of A and b_seg[kb / seg_kb] of B.
     // The result is written as fp32 to Cf (direct stores).
@@ -190,6 +193,11 @@ __device__ __forceinline__ bool get_tile(const UmmaParams& p, int local, int fir
         t->kb0 = 0;
         t->kb1 = p.num_kb;
         t->split = 0;
+        if (e.w != 0) {          // K-balanced plan: this entry is K blocks [kb0, kb1) of the tile, partial sums to slot `split`
+            t->kb0 = e.w & 0xFFF;
+            t->kb1 = (e.w >> 12) & 0xFFF;
+            t->split = (e.w >> 24) & 0x7F;
+        }
         return true;
     }
     const int item = first_item + local * item_stride;

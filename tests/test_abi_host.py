@@ -261,3 +261,58 @@ def test_tuning_cache_round_trip(tmp_path):
     bad = tmp_path / "bad.json"
     bad.write_text('{"entries": [{"key": "gemm:1:1:1:0:0:1", "cfg": [1, 2, 3]}]}')
     assert tdx.tdx_tune_load(str(bad)) == tdx.TDX_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("shape", [(128, 8192, 8192, 128, 192), (8192, 128, 8192, 128, 128), (128, 8192, 8192, 128, 256),
+                                   (300, 1000, 4100, 128, 128), (128, 128, 64 * 9, 128, 128), (512, 512, 64 * 3, 256, 256)])
+@pytest.mark.parametrize("ctas", [148, 132, 7])
+def test_k_balanced_plan_covers_every_unit_once_and_evenly(shape, ctas):
+    # host only: the tiles x K blocks units are dealt to the CTAs in nearly equal runs; every unit exactly once;
+    # a tile's pieces carry slots in ascending K order; no piece shorter than the snapping length unless it is a whole tile
+    M, N, K, tm, tn = shape
+    st, rounds, used, ent, slots = tdx.tdx_gemm_k_balanced_plan(M, N, K, tm, tn, ctas)
+    assert st == tdx.TDX_OK, tdx.tdx_last_error()
+    num_kb = -(-K // 64)
+    tiles_m, tiles_n = -(-M // tm), -(-N // tn)
+    units = tiles_m * tiles_n * num_kb
+    assert 1 <= used <= min(ctas, max(1, units // 4)) and rounds >= 1
+    seen = {}
+    loads = []
+    for c in range(used):
+        load = 0
+        for r in range(rounds):
+            m, n0, w, kb0, kb1, slot = ent[r][c]
+            if w == 0:
+                continue
+            assert 0 <= m < tiles_m and n0 % tn == 0 and n0 < N and w % 64 == 0 and 0 < w <= tn and n0 + w >= min(N, n0 + tn)
+            assert 0 <= kb0 < kb1 <= num_kb
+            assert (kb1 - kb0 >= 4) or (kb0 == 0 and kb1 == num_kb) or num_kb < 8, (kb0, kb1)
+            seen.setdefault((m, n0), []).append((slot, kb0, kb1))
+            load += kb1 - kb0
+        loads.append(load)
+    assert len(seen) == tiles_m * tiles_n
+    for pieces in seen.values():
+        pieces.sort()
+        assert [s for s, _, _ in pieces] == list(range(len(pieces)))          # slots 0, 1, 2, ...
+        assert pieces[0][1] == 0 and pieces[-1][2] == num_kb
+        assert all(a[2] == b[1] for a, b in zip(pieces, pieces[1:]))          # contiguous, ascending K
+        assert len(pieces) <= slots
+    assert sum(loads) == units
+    share = units / used
+    assert max(loads) <= share + 5 and min(loads) >= share - 5                # even up to the snapping length
+
+
+def test_k_balanced_config_constraints_and_workspace_size():
+    M, N, K = 128, 8192, 8192
+    ok = tdx.tdx_config(kernel=tdx.TDX_KERNEL_UMMA, tile_m=128, tile_n=192, fit=3, split_k=1, store_mode=1)
+    st, need = tdx.tdx_gemm_workspace_size(M, N, K, tdx.TDX_BF16, ok)
+    _, _, _, _, slots = tdx.tdx_gemm_k_balanced_plan(M, N, K, 128, 192, 148)
+    assert st == 0 and need == slots * M * N * 4 and 2 <= slots <= 6
+    base = dict(M=M, N=N, K=K, transA=0, transB=0, alpha=1.0, dtype=tdx.TDX_BF16, A=256, B=512, C=1024)
+    for kw in [dict(split_k=2), dict(store_mode=2), dict(tile_n=96), dict(cta_pair=2, tile_m=256, tile_n=256)]:
+        cfg = tdx.tdx_config(kernel=tdx.TDX_KERNEL_UMMA, fit=3, **kw)
+        assert tdx.tdx_gemm_ex(**base, cfg=cfg) == tdx.TDX_ERR_CONFIG, kw
+    st, cfgs = tdx.tdx_enum_gemm_configs(M, N, K, 0, 0, tdx.TDX_BF16)
+    assert st == 0 and any(c["fit"] == 3 for c in cfgs)
+    st, cfgs = tdx.tdx_enum_gemm_configs(8192, 8192, 8192, 0, 0, tdx.TDX_BF16)
+    assert st == 0 and not any(c["fit"] == 3 for c in cfgs)                   # many tiles: nothing to balance

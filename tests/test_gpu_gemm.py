@@ -521,3 +521,45 @@ def test_bf16_gemm_with_odd_pitches_takes_the_tensor_cores_through_a_padded_copy
         assert tdx.tdx_gemm(M, N, K, transA, transB, -1.0, tdx.TDX_BF16, dA.data_ptr() + 2, dB.data_ptr() + 2, out.ptr) == 0
         torch.cuda.synchronize()
         assert out.guards_intact() and np.array_equal(out.payload().reshape(M, N), C)
+
+
+# ------------------------------------------------------------------ K blocks dealt evenly to all CTAs (fit = 3)
+
+@pytest.mark.parametrize("transA,transB", [(0, 0), (0, 1), (1, 0), (1, 1)])
+@pytest.mark.parametrize("case", [(128, 2048, 4096, 128, 192), (136, 1000, 4100 - 4, 128, 128), (520, 128, 8192, 128, 128),
+                                  (256, 768, 2048, 256, 256), (128, 128, 576, 128, 128)])
+def test_k_balanced_plan_matches_the_oracle(case, transA, transB):
+    # few tiles, long reduction: every CTA gets an even run of (tile, K block) units; tiles cut by a CTA boundary are
+    # completed from fp32 partial tiles in ascending K order.  Ragged M, N and K tails; all operand layouts.
+    M, N, K, tm, tn = case
+    A, B = si.gemm_bf16_normal(M, N, K, seed=75, transA=transA, transB=transB)
+    cfg = umma(tile_m=tm, tile_n=tn, fit=3, split_k=1, store_mode=1)
+    st, C, ok = run_gemm(M, N, K, transA, transB, -1.0, "bf16", A, B, cfg=cfg)       # the library's own workspace
+    assert st == 0 and ok, tdx.tdx_last_error()
+    err = gemm_error(M, N, K, transA, transB, -1.0, "bf16", A, B, C)
+    assert err < TIGHT["bf16"], err
+    # caller's workspace of the reported size: same bits (fixed reduction order); too small a one is refused
+    st, need = tdx.tdx_gemm_workspace_size(M, N, K, tdx.TDX_BF16, cfg)
+    assert st == 0 and need >= M * N * 4
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    st, C2, ok = run_gemm(M, N, K, transA, transB, -1.0, "bf16", A, B, cfg=cfg, workspace=ws)
+    assert st == 0 and ok and np.array_equal(C, C2)
+    st, _, untouched = run_gemm(M, N, K, transA, transB, -1.0, "bf16", A, B, cfg=cfg, workspace=ws[:need - 256])
+    assert st == tdx.TDX_ERR_WORKSPACE and untouched
+    assert tdx.tdx_check_device_status() == 0
+
+
+def test_k_balanced_plan_exact_integers():
+    M, N, K = 128, 1536, 192            # 12 tiles x 3 K blocks on 148 CTAs: pieces of one and two K blocks... snapped to whole tiles
+    A = si.small_integers(76, 0, (M, K), "bf16", -1, 1)
+    B = si.small_integers(76, 1, (K, N), "bf16", -1, 1)
+    st, C, ok = run_gemm(M, N, K, 0, 0, 1.0, "bf16", A, B, cfg=umma(tile_m=128, tile_n=128, fit=3, split_k=1, store_mode=1))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert np.array_equal(oracle.decode(C, "bf16"), oracle.gemm(M, N, K, 0, 0, 1.0, "bf16", A, B))
+    M, N, K = 128, 640, 64 * 40         # 5 tiles x 40 K blocks: every tile cut into many pieces
+    A = si.small_integers(77, 0, (M, K), "bf16", -1, 1)
+    B = si.small_integers(77, 1, (N, K), "bf16", -1, 1)
+    # sums of up to 2560 terms are not exact in bf16, so compare after the same single rounding
+    st, C, ok = run_gemm(M, N, K, 0, 1, 1.0, "bf16", A, B, cfg=umma(tile_m=128, tile_n=128, fit=3, split_k=1, store_mode=1))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert np.array_equal(C, oracle.round_bf16(oracle.gemm(M, N, K, 0, 1, 1.0, "bf16", A, B)))
