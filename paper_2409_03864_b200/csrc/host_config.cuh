@@ -42,6 +42,15 @@ bool conv_umma_layout_ok(const ConvProblem& c) {
 // Shared memory the staged (TMA-store) epilogue needs: one 32 x 32 bf16 block for each of its 16 warps.
 int staging_bytes_for(int /*tile_m*/, int store_mode) { return store_mode == 2 ? 16 * 2048 : 0; }
 
+// Shared memory for fp32 partial tiles that leave through the copy engine (split-K, K-balanced plan): two 32 x 32 fp32
+// blocks for each of the four epilogue warps per 128-row half.  Optional: a configuration whose stages leave no room for
+// it stores its partial tiles straight from registers.
+int partial_staging_bytes(int tile_m) { return (tile_m / 128) * 4 * 2 * 4096; }
+int umma_max_stages_partial(int tile_m, int tile_n, int smem_limit) {
+    const int stage = (tile_m + tile_n) * 128;
+    return std::min((smem_limit - kStaticSmemReserve - 1024 - partial_staging_bytes(tile_m)) / stage, tdx::kMaxStages);
+}
+
 int umma_max_stages(int tile_m, int tile_n, int smem_limit, int store_mode) {
     const int stage = (tile_m + tile_n) * 128;
     int s = (smem_limit - kStaticSmemReserve - 1024 - staging_bytes_for(tile_m, store_mode)) / stage;

@@ -13,7 +13,7 @@ int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensor
     if (p.b_box == 0) p.b_box = p.bn;
     const int grid = p.tiles != nullptr ? plan_grid : static_cast<int>(std::min<long long>(items, ctx->sm_count));
     size_t smem = static_cast<size_t>(p.stages) * ((p.bm + p.bn) * 128) + 1024 +
-                  staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
+                  staging_bytes_for(p.bm, p.tma_store ? 2 : 1) + (p.partial_tma ? partial_staging_bytes(p.bm) : 0);
     if (halo)
         smem = static_cast<size_t>(p.a_stages) * (p.bm / 128) * p.halo_bytes + static_cast<size_t>(p.stages) * p.bn * 128 +
                1024 + staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
@@ -272,6 +272,21 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         if (rc) return rc;
     }
     if (k_balanced) plan_grid = kplan.grid;
+    if (p.partial != nullptr && p.split_k > 1) {
+        // fp32 partial tiles leave through shared memory and the copy engine (whole 128-byte lines) when the workspace
+        // rows allow it and the pipeline leaves room for the staging blocks; else straight from registers
+        const size_t room = static_cast<size_t>(ctx->smem_optin - kStaticSmemReserve);
+        const size_t want = static_cast<size_t>(p.stages) * ((p.bm + p.bn) * 128) + 1024 + partial_staging_bytes(p.bm);
+        if (g.N % 4 == 0 && reinterpret_cast<uintptr_t>(p.partial) % 16 == 0 && want <= room) {
+            const uint64_t slots = static_cast<uint64_t>(p.split_k) * static_cast<uint64_t>(nbatch);
+            uint64_t dims[3] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.M), slots};
+            uint64_t str[2] = {static_cast<uint64_t>(g.N) * 4, static_cast<uint64_t>(g.N) * 4 * static_cast<uint64_t>(g.M)};
+            uint32_t box[3] = {32, 32, 1};
+            rc = get_tensor_map(ctx, p.partial, 3, dims, str, box, &mc, 128, nullptr, true);
+            if (rc) return rc;
+            p.partial_tma = 1;
+        }
+    }
     rc = launch_umma(ctx, false, ma, mb, mc, p, st, false, nullptr, nullptr, plan_grid);
     if (rc) return rc;
     if (k_balanced) {

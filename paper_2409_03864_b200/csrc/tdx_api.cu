@@ -169,9 +169,13 @@ int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_cou
         c.store_mode = (c.split_k == 1 && g.N % 8 == 0 && c.fit != 3) ? 2 : 1;
         if (c.store_mode == 2 && c.cta_pair != 2 && c.stages > umma_max_stages(c.tile_m, c.tile_n, smem_limit, 2)) c.store_mode = 1;
     }
-    if (c.stages == 0)
+    if (c.stages == 0) {
         c.stages = c.cta_pair == 2 ? std::max(2, pair_max_stages(c.tile_n, smem_limit, c.store_mode))
                                    : std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode));
+        // partial tiles (split-K, K-balanced plan): leave room for their staging blocks when that still leaves a pipeline
+        if (c.cta_pair != 2 && (c.split_k > 1 || c.fit == 3) && umma_max_stages_partial(c.tile_m, c.tile_n, smem_limit) >= 3)
+            c.stages = std::min(c.stages, umma_max_stages_partial(c.tile_m, c.tile_n, smem_limit));
+    }
     if (!user && !from_cache) c.raster = d.raster;
     const char* why = umma_config_reason(c, b_mn, num_kb, smem_limit, false, g.N);
     if (why) return fail(TDX_ERR_CONFIG, "infeasible config: %s", why);
@@ -392,6 +396,10 @@ void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int 
                     std::vector<int> stage_opts;
                     stage_opts.push_back(max_st);
                     if (max_st - 2 >= 3) stage_opts.push_back(max_st - 2);
+                    // split-K: also the deepest pipeline that leaves room for staging the partial tiles
+                    const int staged_st = umma_max_stages_partial(tm, bn, smem_limit);
+                    if (sk > 1 && staged_st >= 3 && std::find(stage_opts.begin(), stage_opts.end(), staged_st) == stage_opts.end())
+                        stage_opts.push_back(staged_st);
                     for (int st : stage_opts)
                         for (int raster : {0, 8, 2, 4, 16})
                             for (int stagger : {0, 1}) {
@@ -418,9 +426,10 @@ void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int 
                 }
             // K blocks dealt evenly to all CTAs, for problems with few tiles and a long reduction
             if (!conv && bn % 64 == 0 && bn >= 128 && tiles < 2LL * sm_count && tiles * num_kb >= 4LL * sm_count && num_kb <= 4095) {
-                const int max_st = umma_max_stages(tm, bn, smem_limit, 1);
-                for (int st : {max_st, max_st - 2}) {
-                    if (st < 3) continue;
+                const int max_st = umma_max_stages(tm, bn, smem_limit, 1), staged_st = umma_max_stages_partial(tm, bn, smem_limit);
+                for (int pass = 0; pass < 2; ++pass) {
+                    const int st = pass == 0 ? max_st : staged_st;
+                    if (st < 3 || (pass == 1 && staged_st == max_st)) continue;
                     tdx_config c;
                     std::memset(&c, 0, sizeof c);
                     c.kernel = TDX_KERNEL_UMMA;

@@ -59,6 +59,8 @@ struct UmmaParams {
     float* partial;           // split-K: [split][M][N] fp32
     int vec_store;            // rows of C / partial are 16-byte aligned and N % 8 == 0
     int tma_store;            // final output leaves through shared memory + TMA store (needs bn % 64 == 0)
+    int partial_tma;          // split-K: fp32 partial tiles leave through shared memory + TMA store (tmC then maps the
+                              // workspace as (N, M, batch * split) floats; two 32 x 32 fp32 blocks per epilogue warp)
     int sbx, sby;             // conv TMA-store box: sbx x sby output pixels (sbx * sby = 32)
     // convolution geometry (kConv only)
     int bw, bh, nb;           // spatial patch (bw x bh output pixels), patches per tile = bm / (bw*bh)
@@ -486,6 +488,30 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
             ptx::tmem_ld_32x32b_x32(taddr, r);
             ptx::tmem_ld_wait();
             const int col0 = t.n0 + c0;
+            if (p.split_k > 1 && p.partial_tma) {
+                // fp32 partial tile through shared memory: the thread writes its row's 32 values (128 bytes, 16-byte
+                // chunk c at chunk c ^ (row % 8): the 128-byte swizzle of the copy engine) and the copy engine stores
+                // the 32 x 32 block as whole 128-byte lines, clipped at the matrix edge; stores straight from registers
+                // reach the same lines in 16-byte pieces, eight instructions per line.  Two blocks per warp take turns, so
+                // a block is rewritten only after the store issued two steps earlier has read it.
+                const int estep = c0 >> 5;
+                uint8_t* blk = staging_base + ((warp - 2) * 2 + (estep & 1)) * 4096;
+                if (lane == 0) ptx::tma_store_wait_read<1>();
+                __syncwarp();
+                uint8_t* my_row = blk + lane * 128;
+#pragma unroll
+                for (int g = 0; g < 8; ++g)
+                    *reinterpret_cast<uint4*>(my_row + ((g ^ (lane & 7)) << 4)) = make_uint4(r[g * 4], r[g * 4 + 1], r[g * 4 + 2], r[g * 4 + 3]);
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                const int row0 = t.m_blk * p.bm + half * kHalfM + quarter * 32;
+                if (lane == 0 && row0 < p.M && col0 < p.N) {
+                    ptx::tma_store_3d(tmC, blk, col0, row0, t.batch * p.split_k + t.split);
+                    ptx::tma_store_commit();
+                }
+                __syncwarp();
+                continue;
+            }
             if (valid && col0 < p.N) {
             if (p.split_k > 1) {
                 float* dst = p.partial + ((static_cast<long long>(t.batch) * p.split_k + t.split) * p.M + grow) * p.N + col0;
@@ -576,7 +602,7 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
         }
     }
     // shared memory must stay alive until the copy engine has drained this warp's last store
-    if (p.tma_store && lane < 4) ptx::tma_store_wait_all<0>();
+    if ((p.tma_store || p.partial_tma) && lane < 4) ptx::tma_store_wait_all<0>();
 }
 
 template <bool kConv>
