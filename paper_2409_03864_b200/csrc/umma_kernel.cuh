@@ -403,12 +403,14 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
             uint8_t* my_row = stage_buf + lane * 64;
             const int sw = (lane >> 1) & 3;
             const bool plain = (p.bias == nullptr) && (p.relu == 0) && (p.residual == nullptr);
+            // Per 32-column step: the accumulators are converted into registers first; then the NEXT step's accumulators
+            // are requested from tensor memory, so that their latency passes while this step waits for its staging
+            // block (the copy engine may still be reading the previous store), writes it, and hands it to the copy engine.
             int step = 0;
+            uint32_t r[32];
+            const uint32_t trow = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * p.bn);
+            if (cgrp * 32 < t.bn) ptx::tmem_ld_32x32b_x32(trow + static_cast<uint32_t>(cgrp * 32), r);
             for (int c0 = cgrp * 32; c0 < t.bn; c0 += ncgrp * 32, ++step) {
-                uint32_t r[32];
-                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
-                                       static_cast<uint32_t>(buf * p.bn + c0);
-                ptx::tmem_ld_32x32b_x32(taddr, r);
                 const int col0 = t.n0 + c0;
                 // the bias of column col0 + lane: prefetched above for the first four steps of a warp (all there are
                 // with 16 epilogue warps and tiles of up to 256 columns)
@@ -435,40 +437,35 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                         }
                     }
                 }
-                // the previous store of this warp must have finished reading the staging block
-                if (lane < nstore) ptx::tma_store_wait_read<0>();
-                __syncwarp();
+                uint32_t pk[16];                                   // the step's 32 outputs as bf16 pairs
                 if (plain) {
 #pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        uint32_t pk[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(p.alpha * __uint_as_float(r[g * 8 + e * 2]),
-                                                                      p.alpha * __uint_as_float(r[g * 8 + e * 2 + 1]));
-                            pk[e] = *reinterpret_cast<uint32_t*>(&h2);
-                        }
-                        *reinterpret_cast<uint4*>(my_row + ((g ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    for (int e = 0; e < 16; ++e) {
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(p.alpha * __uint_as_float(r[2 * e]), p.alpha * __uint_as_float(r[2 * e + 1]));
+                        pk[e] = *reinterpret_cast<uint32_t*>(&h2);
                     }
                 } else {
 #pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        uint32_t pk[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const int j = g * 8 + e * 2;
-                            float x0 = p.alpha * __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_l, j);
-                            float x1 = p.alpha * __uint_as_float(r[j + 1]) + __shfl_sync(0xffffffffu, bias_l, j + 1);
-                            if (p.relu) {
-                                x0 = fmaxf(x0, 0.0f);
-                                x1 = fmaxf(x1, 0.0f);
-                            }
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
-                            pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+                    for (int e = 0; e < 16; ++e) {
+                        const int j = 2 * e;
+                        float x0 = p.alpha * __uint_as_float(r[j]) + __shfl_sync(0xffffffffu, bias_l, j);
+                        float x1 = p.alpha * __uint_as_float(r[j + 1]) + __shfl_sync(0xffffffffu, bias_l, j + 1);
+                        if (p.relu) {
+                            x0 = fmaxf(x0, 0.0f);
+                            x1 = fmaxf(x1, 0.0f);
                         }
-                        *reinterpret_cast<uint4*>(my_row + ((g ^ sw) << 4)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(x0, x1);
+                        pk[e] = *reinterpret_cast<uint32_t*>(&h2);
                     }
                 }
+                // r is free again: request the next step's accumulators now
+                if (c0 + ncgrp * 32 < t.bn) ptx::tmem_ld_32x32b_x32(trow + static_cast<uint32_t>(c0 + ncgrp * 32), r);
+                // the previous store of this warp must have finished reading the staging block
+                if (lane < nstore) ptx::tma_store_wait_read<0>();
+                __syncwarp();
+#pragma unroll
+                for (int g = 0; g < 4; ++g)
+                    *reinterpret_cast<uint4*>(my_row + ((g ^ sw) << 4)) = make_uint4(pk[4 * g], pk[4 * g + 1], pk[4 * g + 2], pk[4 * g + 3]);
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane < nstore && box_ok && col0 < p.N) {
