@@ -292,8 +292,9 @@ int tdx_set_autotune(int budget);
  * Guided search: the candidates of tdx_tune_gemm are ranked by a host-side cost model (MMA time by tile width, L2
  * ingest, epilogue overlap, wave count or fitted plan, split-K traffic, HBM floor) and only the `budget` best-ranked
  * ones, plus the automatic choice, are timed on the device -- the model-guided counterpart of Case Study 5's
- * search under constraints.  n_candidates (may be NULL) receives the size of the full search space.  bf16 GEMM;
- * other problems are searched exhaustively.  tdx_model_gemm_us evaluates the model for one configuration on
+ * search under constraints.  n_candidates (may be NULL) receives the size of the full search space.  The cached winners
+ * of other shapes with the same operand layouts are tried as well (up to four), so what earlier searches found carries
+ * over to a new shape.  bf16 GEMM; other problems are searched exhaustively.  tdx_model_gemm_us evaluates the model for one configuration on
  * `ctas` SMs (host only).
  */
 int tdx_tune_gemm_guided(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, int iters, int budget,
@@ -301,6 +302,45 @@ int tdx_tune_gemm_guided(int64_t M, int64_t N, int64_t K, int transA, int transB
                          int* n_candidates, void* stream);
 int tdx_model_gemm_us(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const tdx_config* cfg, int ctas,
                       double* us);
+
+/*
+ * The same for the convolution: the candidates of tdx_tune_conv2d are ranked by a host-side cost model of the two
+ * convolution kernels (wasted patch rows, input-window bytes per filter tap or per channel chunk, resident filter,
+ * strided windows, epilogue overlap, wave count) and only `budget` of them, plus the automatic choice, are timed;
+ * winner checked and cached as by tdx_tune_conv2d.  tdx_model_conv2d_us evaluates the model (host only).
+ */
+int tdx_tune_conv2d_guided(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
+                           int stride, int dtype, int iters, int budget, tdx_config* best, float* best_us, tdx_config* tried,
+                           float* tried_us, int cap, int* n_tried, int* n_candidates, void* stream);
+int tdx_model_conv2d_us(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad, int stride,
+                        int dtype, const tdx_config* cfg, int ctas, double* us);
+
+/*
+ * A search space stated by the caller, the way Case Study 5 hands its tuner a list of tuning parameters with ranges
+ * and constraints (tile sizes that must divide their dimension; vectorisation only under a divisibility condition):
+ *
+ *   "tile_m in {128, 256}; tile_n in 64..256 step 64; split_k in {1, 2, 4};
+ *    require M % tile_m == 0; require N % tile_n == 0;
+ *    store_mode == 2 only if N % 8 == 0 && split_k == 1"
+ *
+ * Statements are separated by ';'.  `<param> in {a, b, ...}` or `<param> in lo..hi [step s]` gives a parameter its
+ * range (parameters: tile_m tile_n tile_k stages cta_pair split_k store_mode raster k_stagger fit; one not mentioned
+ * stays "choose for me").  `require <expr>` keeps a candidate only if the expression holds; `<param> == <value> only
+ * if <expr>` lets that value through only under the condition.  Expressions are integer expressions over the
+ * parameters, the problem (M N K transA transB num_kb = ceil(K / 64)) and literals, with + - * / % == != < <= > >= && ||
+ * ! and parentheses.  The cross product of the ranges is filtered by the stated rules, each survivor is completed
+ * by the library's rules and checked against the hardware's own constraints (shared memory, tensor memory, layout).
+ *
+ * tdx_enum_gemm_space lists the survivors (host only; n_product = size of the cross product, n_after_rules = how many
+ * pass the stated rules).  tdx_tune_gemm_space searches them -- all of them (budget = 0) or the `budget` the cost model
+ * ranks best -- checks the winner's output and caches it like tdx_tune_gemm.  bf16 GEMM with 16-byte aligned pitches.
+ * Errors: INVALID_ARG (syntax, unknown name, NULL), UNSUPPORTED (nothing feasible is left; other dtypes / layouts).
+ */
+int tdx_enum_gemm_space(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const char* space, tdx_config* out,
+                        int cap, int* n, int64_t* n_product, int64_t* n_after_rules);
+int tdx_tune_gemm_space(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const char* space, int iters,
+                        int budget, tdx_config* best, float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried,
+                        int* n_candidates, void* stream);
 
 /* The configuration the automatic choice would use right now: the tuning cache's entry, else (bf16 GEMM on the
  * tensor-core path) the candidate of the search space that the cost model ranks first, else a size heuristic. */

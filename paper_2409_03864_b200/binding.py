@@ -94,6 +94,10 @@ def lib() -> ctypes.CDLL:
         L.tdx_set_autotune.argtypes = [ci]
         dp = ctypes.POINTER(ctypes.c_double)
         L.tdx_gemm_tile_plan.argtypes = [i64, i64, i64, ci, ci, ci, ci, ip, ci, ip, ip, dp, dp]
+        L.tdx_tune_conv2d_guided.argtypes = [i64] * 7 + [ci, ci, ci, ci, ci, cfgp, fp, cfgp, fp, ci, ip, ip, vp]
+        L.tdx_model_conv2d_us.argtypes = [i64] * 7 + [ci, ci, ci, cfgp, ci, ctypes.POINTER(ctypes.c_double)]
+        L.tdx_enum_gemm_space.argtypes = [i64, i64, i64, ci, ci, ci, ctypes.c_char_p, cfgp, ci, ip, ctypes.POINTER(i64), ctypes.POINTER(i64)]
+        L.tdx_tune_gemm_space.argtypes = [i64, i64, i64, ci, ci, ci, ctypes.c_char_p, ci, ci, cfgp, fp, cfgp, fp, ci, ip, ip, vp]
         L.tdx_gemm_k_balanced_plan.argtypes = [i64, i64, i64, ci, ci, ci, ip, ci, ip, ip, ip]
         L.tdx_gemm_splitk_static.argtypes = [i64, i64, i64, ci, ci, cf, vp, vp, vp, ci, ci, vp]
         L.tdx_check_device_status.argtypes = [vp]
@@ -120,7 +124,7 @@ EXPORTS = (
     "tdx_gemm", "tdx_gemm_f32out", "tdx_add_zero_pad", "tdx_add_zero_pad_host", "tdx_gemm_batched", "tdx_gemm_batched_host", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_add_relu", "tdx_conv2d_bias_relu_ex",
     "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_gemm_guided", "tdx_model_gemm_us", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
     "tdx_enum_conv2d_configs", "tdx_default_gemm_config", "tdx_default_conv2d_config", "tdx_tune_save",
-    "tdx_tune_load", "tdx_tune_clear", "tdx_set_autotune", "tdx_gemm_tile_plan", "tdx_gemm_k_balanced_plan", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
+    "tdx_tune_load", "tdx_tune_clear", "tdx_set_autotune", "tdx_gemm_tile_plan", "tdx_gemm_k_balanced_plan", "tdx_enum_gemm_space", "tdx_tune_gemm_space", "tdx_tune_conv2d_guided", "tdx_model_conv2d_us", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
     "tdx_version",
 )
 
@@ -286,6 +290,22 @@ def tdx_tune_conv2d(N, H, W, Cin, Cout, R, S, pad, stride, dtype, iters=20, stre
                                                               bu, t, tu, c, n, _stream(stream)), cap)
 
 
+def tdx_tune_conv2d_guided(N, H, W, Cin, Cout, R, S, pad, stride, dtype, budget, iters=20, stream=None, cap=512):
+    """Returns (status, best tdx_config, best microseconds, [(config dict, microseconds), ...], size of the full space)."""
+    L = lib()
+    n_cand = ctypes.c_int(0)
+    st, best, us, tried = _tune(lambda b, bu, t, tu, c, n: L.tdx_tune_conv2d_guided(
+        N, H, W, Cin, Cout, R, S, pad, stride, dtype, iters, budget, b, bu, t, tu, c, n, ctypes.byref(n_cand), _stream(stream)), cap)
+    return st, best, us, tried, int(n_cand.value)
+
+
+def tdx_model_conv2d_us(N, H, W, Cin, Cout, R, S, pad, stride, dtype, cfg, ctas=148):
+    """Returns (status, predicted microseconds) of the convolution cost model (host only)."""
+    us = ctypes.c_double(0.0)
+    st = lib().tdx_model_conv2d_us(N, H, W, Cin, Cout, R, S, pad, stride, dtype, _cfg(cfg), ctas, ctypes.byref(us))
+    return st, float(us.value)
+
+
 def _enum(call, cap=8192):
     out = (tdx_config * cap)()
     n = ctypes.c_int(0)
@@ -302,6 +322,24 @@ def tdx_enum_gemm_configs(M, N, K, transA, transB, dtype):
 def tdx_enum_conv2d_configs(N, H, W, Cin, Cout, R, S, pad, stride, dtype):
     L = lib()
     return _enum(lambda o, c, n: L.tdx_enum_conv2d_configs(N, H, W, Cin, Cout, R, S, pad, stride, dtype, o, c, n))
+
+
+def tdx_enum_gemm_space(M, N, K, transA, transB, dtype, space: str, cap=8192):
+    """Returns (status, [config dict, ...], size of the cross product, how many pass the stated rules)."""
+    out = (tdx_config * cap)()
+    n, prod, kept = ctypes.c_int(0), ctypes.c_int64(0), ctypes.c_int64(0)
+    st = lib().tdx_enum_gemm_space(M, N, K, transA, transB, dtype, space.encode(), out, cap, ctypes.byref(n), ctypes.byref(prod),
+                                   ctypes.byref(kept))
+    return st, [out[i].as_dict() for i in range(min(cap, int(n.value)))], int(prod.value), int(kept.value)
+
+
+def tdx_tune_gemm_space(M, N, K, transA, transB, dtype, space: str, budget=0, iters=20, stream=None, cap=512):
+    """Searches the stated space; returns (status, best, best microseconds, [(config dict, microseconds), ...], candidates)."""
+    L = lib()
+    n_cand = ctypes.c_int(0)
+    st, best, us, tried = _tune(lambda b, bu, t, tu, c, n: L.tdx_tune_gemm_space(
+        M, N, K, transA, transB, dtype, space.encode(), iters, budget, b, bu, t, tu, c, n, ctypes.byref(n_cand), _stream(stream)), cap)
+    return st, best, us, tried, int(n_cand.value)
 
 
 def tdx_default_gemm_config(M, N, K, transA, transB, dtype):

@@ -325,4 +325,42 @@ double model_gemm_us(const GemmProblem& g, const tdx_config& c, int sm_count) {
     return std::max(us, hbm_us);
 }
 
+// The same kind of model for a convolution configuration (ranks the candidates of the guided convolution search).
+// What differs from the GEMM: the rows of a tile are patches of output pixels (rows past the image edge are wasted
+// work), the A operand of a K block is an input window -- fetched once per filter tap (per-tap kernel; a strided
+// window drags in the pixels between its taps) or once per channel chunk for all taps (halo kernel) -- and a filter
+// that fits shared memory is loaded once per CTA.
+double model_conv_us(const ConvProblem& cp, const tdx_config& c, int sm_count, int smem_limit) {
+    const double clk_mhz = 1600.0;
+    const int64_t cchunks = ceil_div(cp.Cin, 64), taps = cp.R * cp.S, num_kb = taps * cchunks;
+    const int tm = c.tile_m, bn = c.tile_n, halves = tm / 128;
+    int64_t halves_total;
+    if (c.halo >= 2) halves_total = halo_patches(cp, c.halo);
+    else {
+        const int per = std::max(1, c.patch_w * c.patch_h);
+        halves_total = ceil_div(cp.N * ceil_div(cp.Q, c.patch_w) * ceil_div(cp.P, c.patch_h), std::max(1, 128 / per));
+    }
+    const int64_t tiles = ceil_div(halves_total, halves) * ceil_div(cp.Cout, bn);
+    const double mma = 4.0 * halves * std::max(bn / 2.0, 60.0);
+    double bytes_per_kb;
+    if (c.halo >= 2) {
+        const bool resident = bn >= cp.Cout && static_cast<int64_t>(kHaloAStages) * halves * halo_tile_bytes(cp.R, cp.S) + num_kb * bn * 128 +
+                                                    staging_bytes_for(tm, c.store_mode) + 1024 <= smem_limit - kStaticSmemReserve;
+        bytes_per_kb = static_cast<double>(halves) * halo_tile_bytes(cp.R, cp.S) / taps + (resident ? 0.0 : bn * 128.0);
+    } else {
+        bytes_per_kb = tm * 128.0 * cp.stride + bn * 128.0;
+    }
+    const double l2 = bytes_per_kb / (bn < 128 ? 46.0 : 70.0);
+    const double main_loop = static_cast<double>(num_kb) * std::max(mma, l2);
+    const double blocks = halves * 4.0 * (bn / 32.0);
+    const double epi = c.store_mode == 2 ? 600.0 * std::ceil(blocks / 16.0) : 1200.0 * std::ceil(blocks / (4.0 * halves));
+    const bool overlapped = tmem_slots_for(tm, bn) > halves;
+    const double rounds = std::ceil(static_cast<double>(tiles) / sm_count);
+    const double per_tile = overlapped ? std::max(main_loop, epi) : main_loop + epi;
+    const double cycles = 5500.0 + rounds * per_tile + (overlapped ? epi : 0.0);
+    const double hbm_us = (static_cast<double>(cp.N) * cp.H * cp.W * cp.Cin + static_cast<double>(cp.Cout) * taps * cp.Cin +
+                           static_cast<double>(cp.N) * cp.P * cp.Q * cp.Cout) * 2.0 / 5.0e6;
+    return std::max(cycles / clk_mhz, hbm_us);
+}
+
 }  // namespace

@@ -3,6 +3,7 @@
 // translation unit: host_state.cuh (context, caches), host_config.cuh (configuration rules), host_plan.cuh (fitted
 // tile plans), host_launch.cuh (launches).
 #include "host_launch.cuh"
+#include "host_space.cuh"
 
 #include <array>
 #include <tuple>
@@ -11,7 +12,7 @@
 extern "C" {
 static int tune_gemm_impl(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, int iters, int budget,
                           tdx_config* best, float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried,
-                          int* n_candidates, void* stream);
+                          int* n_candidates, void* stream, const void* given_candidates = nullptr);
 }
 
 namespace {
@@ -1186,9 +1187,10 @@ int tune_operand_sets(size_t bytes_per_set) {
 
 // budget <= 0: every statically feasible candidate is timed; budget > 0: the candidates are ranked by the cost model and
 // only the `budget` best-ranked ones (plus the automatic choice) are timed
+// given_candidates: a std::vector<tdx_config> to search instead of the library's own space (tdx_tune_gemm_space)
 static int tune_gemm_impl(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, int iters, int budget,
                           tdx_config* best, float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried,
-                          int* n_candidates, void* stream) {
+                          int* n_candidates, void* stream, const void* given_candidates) {
     int rc = validate_gemm(M, N, K, transA, transB, dtype, nullptr, nullptr, nullptr, false);
     if (rc) return rc;
     if (best == nullptr || iters < 1 || cap < 0) return fail(TDX_ERR_INVALID_ARG, "best is NULL, iters < 1 or cap < 0");
@@ -1198,7 +1200,9 @@ static int tune_gemm_impl(int64_t M, int64_t N, int64_t K, int transA, int trans
     if (rc) return rc;
     GemmProblem g{M, N, K, transA, transB, dtype};
     std::vector<tdx_config> cands;
-    enum_gemm(g, ctx->sm_count, ctx->smem_optin, &cands);
+    if (given_candidates) cands = *static_cast<const std::vector<tdx_config>*>(given_candidates);
+    else enum_gemm(g, ctx->sm_count, ctx->smem_optin, &cands);
+    if (cands.empty()) return fail(TDX_ERR_UNSUPPORTED, "the search space holds no feasible configuration");
     if (n_candidates) *n_candidates = static_cast<int>(cands.size());
     if (budget > 0 && static_cast<int>(cands.size()) > budget && dtype == TDX_BF16 && cands[0].kernel == TDX_KERNEL_UMMA) {
         std::vector<std::pair<double, size_t>> ranked;
@@ -1223,8 +1227,35 @@ static int tune_gemm_impl(int64_t M, int64_t N, int64_t K, int transA, int trans
         for (size_t r = 0; r < ranked.size() && static_cast<int>(keep.size()) < budget; ++r)
             if (!taken[ranked[r].second]) keep.push_back(cands[ranked[r].second]);
         tdx_config d;
-        if (resolve_gemm_config(g, nullptr, ctx->sm_count, ctx->smem_optin, &d) == TDX_OK && d.kernel == TDX_KERNEL_UMMA)
+        if (!given_candidates && resolve_gemm_config(g, nullptr, ctx->sm_count, ctx->smem_optin, &d) == TDX_OK && d.kernel == TDX_KERNEL_UMMA)
             keep.push_back(d);                                  // what an untuned call would use: never do worse than that
+        if (!given_candidates) {
+            // What earlier searches found carries over: the cached winners of other GEMM shapes with the same operand
+            // layouts are tried here too, tile shape and split as they are, where they are feasible for this problem.
+            std::vector<tdx_config> known;
+            {
+                std::lock_guard<std::mutex> lk(g_mu);
+                char suffix[32];
+                snprintf(suffix, sizeof suffix, ":%d:%d:%d", transA, transB, dtype);
+                const std::string mine = gemm_key(M, N, K, transA, transB, dtype);
+                for (const auto& kv : g_tune) {
+                    if (kv.first.compare(0, 5, "gemm:") != 0 || kv.first == mine) continue;
+                    if (kv.first.size() < std::strlen(suffix) || kv.first.compare(kv.first.size() - std::strlen(suffix), std::string::npos, suffix) != 0) continue;
+                    known.push_back(kv.second.cfg);
+                }
+            }
+            int added = 0;
+            for (tdx_config k : known) {
+                if (added >= 4 || k.kernel != TDX_KERNEL_UMMA) continue;
+                k.stages = 0;                                   // the depth follows the shared-memory budget
+                tdx_config full;
+                if (resolve_gemm_config(g, &k, ctx->sm_count, ctx->smem_optin, &full) != TDX_OK) continue;
+                bool dup = false;
+                for (const auto& o : keep)
+                    if (std::memcmp(&o, &full, sizeof full) == 0) { dup = true; break; }
+                if (!dup) { keep.push_back(full); ++added; }
+            }
+        }
         cands.swap(keep);
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1307,6 +1338,54 @@ int tdx_tune_gemm_guided(int64_t M, int64_t N, int64_t K, int transA, int transB
                           n_candidates, stream);
 }
 
+// ---- a search space stated by the caller (Case Study 5's tuning-parameter listing: ranges and constraints)
+static int build_gemm_space(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const char* space,
+                            std::vector<tdx_config>* cands, long long* n_product, long long* n_after_rules) {
+    int rc = validate_gemm(M, N, K, transA, transB, dtype, nullptr, nullptr, nullptr, false);
+    if (rc) return rc;
+    if (space == nullptr) return fail(TDX_ERR_INVALID_ARG, "space is NULL");
+    if (M == 0 || N == 0 || K == 0) return fail(TDX_ERR_INVALID_ARG, "empty problem");
+    GemmProblem g{M, N, K, transA, transB, dtype};
+    if (dtype != TDX_BF16 || !gemm_umma_layout_ok(g))
+        return fail(TDX_ERR_UNSUPPORTED, "a stated search space applies to the bf16 tensor-core GEMM (16-byte aligned pitches)");
+    SearchSpace sp;
+    std::string err;
+    if (!parse_search_space(space, &sp, &err)) return fail(TDX_ERR_INVALID_ARG, "search space: %s", err.c_str());
+    int sm_count, smem_limit;
+    device_limits(&sm_count, &smem_limit);
+    auto resolve = [&](const tdx_config& partial, tdx_config* full) {
+        return resolve_gemm_config(g, &partial, sm_count, smem_limit, full) == TDX_OK && full->kernel == TDX_KERNEL_UMMA;
+    };
+    if (!enumerate_search_space(sp, g, resolve, cands, n_product, n_after_rules, &err))
+        return fail(TDX_ERR_INVALID_ARG, "search space: %s", err.c_str());
+    return TDX_OK;
+}
+
+int tdx_enum_gemm_space(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const char* space, tdx_config* out,
+                        int cap, int* n, int64_t* n_product, int64_t* n_after_rules) {
+    if (cap < 0 || (cap > 0 && out == nullptr)) return fail(TDX_ERR_INVALID_ARG, "bad output list");
+    std::vector<tdx_config> v;
+    long long prod = 0, kept = 0;
+    int rc = build_gemm_space(M, N, K, transA, transB, dtype, space, &v, &prod, &kept);
+    if (rc) return rc;
+    if (n_product) *n_product = prod;
+    if (n_after_rules) *n_after_rules = kept;
+    return write_configs(v, out, cap, n);
+}
+
+int tdx_tune_gemm_space(int64_t M, int64_t N, int64_t K, int transA, int transB, int dtype, const char* space, int iters,
+                        int budget, tdx_config* best, float* best_us, tdx_config* tried, float* tried_us, int cap, int* n_tried,
+                        int* n_candidates, void* stream) {
+    if (budget < 0) return fail(TDX_ERR_INVALID_ARG, "budget must be >= 0");
+    std::vector<tdx_config> v;
+    long long prod = 0, kept = 0;
+    int rc = build_gemm_space(M, N, K, transA, transB, dtype, space, &v, &prod, &kept);
+    if (rc) return rc;
+    if (v.empty()) return fail(TDX_ERR_UNSUPPORTED, "the stated constraints leave no feasible configuration (%lld of %lld pass the rules)", kept, prod);
+    return tune_gemm_impl(M, N, K, transA, transB, dtype, iters, budget, best, best_us, tried, tried_us, cap, n_tried, n_candidates,
+                          stream, &v);
+}
+
 int tdx_set_autotune(int budget) {
     g_autotune_budget.store(budget, std::memory_order_relaxed);
     return TDX_OK;
@@ -1327,9 +1406,45 @@ int tdx_model_gemm_us(int64_t M, int64_t N, int64_t K, int transA, int transB, i
     return TDX_OK;
 }
 
+static int tune_conv_impl(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
+                          int stride, int dtype, int iters, int budget, tdx_config* best, float* best_us, tdx_config* tried,
+                          float* tried_us, int cap, int* n_tried, int* n_candidates, void* stream);
+
 int tdx_tune_conv2d(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
                     int stride, int dtype, int iters, tdx_config* best, float* best_us, tdx_config* tried,
                     float* tried_us, int cap, int* n_tried, void* stream) {
+    return tune_conv_impl(N, H, W, Cin, Cout, R, S, pad, stride, dtype, iters, 0, best, best_us, tried, tried_us, cap, n_tried,
+                          nullptr, stream);
+}
+
+int tdx_tune_conv2d_guided(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
+                           int stride, int dtype, int iters, int budget, tdx_config* best, float* best_us, tdx_config* tried,
+                           float* tried_us, int cap, int* n_tried, int* n_candidates, void* stream) {
+    if (budget < 1) return fail(TDX_ERR_INVALID_ARG, "budget must be >= 1");
+    return tune_conv_impl(N, H, W, Cin, Cout, R, S, pad, stride, dtype, iters, budget, best, best_us, tried, tried_us, cap, n_tried,
+                          n_candidates, stream);
+}
+
+int tdx_model_conv2d_us(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad, int stride,
+                        int dtype, const tdx_config* cfg, int ctas, double* us) {
+    ConvProblem cp;
+    int rc = validate_conv(N, H, W, Cin, Cout, R, S, pad, stride, dtype, nullptr, nullptr, nullptr, 0, false, &cp);
+    if (rc) return rc;
+    if (cfg == nullptr || us == nullptr || ctas < 2 || N == 0 || Cout == 0 || cp.P == 0 || cp.Q == 0)
+        return fail(TDX_ERR_INVALID_ARG, "cfg or us is NULL, ctas < 2, or empty problem");
+    tdx_config c;
+    rc = resolve_conv_config(cp, cfg, ctas, kSmemLimitDefault, &c);
+    if (rc) return rc;
+    if (c.kernel != TDX_KERNEL_UMMA) return fail(TDX_ERR_UNSUPPORTED, "the cost model covers the tensor-core kernels");
+    *us = model_conv_us(cp, c, ctas, kSmemLimitDefault);
+    return TDX_OK;
+}
+
+// budget <= 0: every candidate is timed; budget > 0: the candidates are ranked by model_conv_us and only the best-ranked
+// ones (half of the budget on distinct kernel / tile / patch shapes, the rest on their variants) plus the automatic choice
+static int tune_conv_impl(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
+                          int stride, int dtype, int iters, int budget, tdx_config* best, float* best_us, tdx_config* tried,
+                          float* tried_us, int cap, int* n_tried, int* n_candidates, void* stream) {
     ConvProblem cp;
     int rc = validate_conv(N, H, W, Cin, Cout, R, S, pad, stride, dtype, nullptr, nullptr, nullptr, 0, false, &cp);
     if (rc) return rc;
@@ -1340,6 +1455,30 @@ int tdx_tune_conv2d(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, 
     if (rc) return rc;
     std::vector<tdx_config> cands;
     enum_conv(cp, ctx->sm_count, ctx->smem_optin, &cands);
+    if (n_candidates) *n_candidates = static_cast<int>(cands.size());
+    if (budget > 0 && static_cast<int>(cands.size()) > budget && dtype == TDX_BF16 && cands[0].kernel == TDX_KERNEL_UMMA) {
+        std::vector<std::pair<double, size_t>> ranked;
+        for (size_t i = 0; i < cands.size(); ++i) ranked.push_back({model_conv_us(cp, cands[i], ctx->sm_count, ctx->smem_optin), i});
+        std::stable_sort(ranked.begin(), ranked.end());
+        auto shape_of = [](const tdx_config& c) {
+            return std::make_tuple(c.halo, c.tile_m, c.tile_n, c.patch_w, c.patch_h, c.store_mode, c.fit);
+        };
+        std::vector<char> taken(cands.size(), 0);
+        std::vector<tdx_config> keep;
+        std::vector<decltype(shape_of(cands[0]))> seen;
+        for (size_t r = 0; r < ranked.size() && static_cast<int>(keep.size()) < (budget + 1) / 2; ++r) {
+            const tdx_config& c = cands[ranked[r].second];
+            if (std::find(seen.begin(), seen.end(), shape_of(c)) != seen.end()) continue;
+            seen.push_back(shape_of(c));
+            keep.push_back(c);
+            taken[ranked[r].second] = 1;
+        }
+        for (size_t r = 0; r < ranked.size() && static_cast<int>(keep.size()) < budget; ++r)
+            if (!taken[ranked[r].second]) keep.push_back(cands[ranked[r].second]);
+        tdx_config d;
+        if (resolve_conv_config(cp, nullptr, ctx->sm_count, ctx->smem_optin, &d) == TDX_OK && d.kernel == TDX_KERNEL_UMMA) keep.push_back(d);
+        cands.swap(keep);
+    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t el = dtype == TDX_F32 ? 4 : 2;
     ScratchGuard guard;
