@@ -341,23 +341,29 @@ double model_conv_us(const ConvProblem& cp, const tdx_config& c, int sm_count, i
         halves_total = ceil_div(cp.N * ceil_div(cp.Q, c.patch_w) * ceil_div(cp.P, c.patch_h), std::max(1, 128 / per));
     }
     const int64_t tiles = ceil_div(halves_total, halves) * ceil_div(cp.Cout, bn);
-    const double mma = 4.0 * halves * std::max(bn / 2.0, 60.0);
-    double bytes_per_kb;
+    // inside the halo kernel an MMA was measured at about 100 cycles however narrow (the issuer advances a window
+    // descriptor per tap), so tiles narrower than 200 columns run below the tensor pipe's rate there
+    const double mma = 4.0 * halves * std::max(bn / 2.0, c.halo >= 2 ? 100.0 : 60.0);
+    double bytes_per_kb, copy_issue = 0.0;
     if (c.halo >= 2) {
         const bool resident = bn >= cp.Cout && static_cast<int64_t>(kHaloAStages) * halves * halo_tile_bytes(cp.R, cp.S) + num_kb * bn * 128 +
                                                     staging_bytes_for(tm, c.store_mode) + 1024 <= smem_limit - kStaticSmemReserve;
         bytes_per_kb = static_cast<double>(halves) * halo_tile_bytes(cp.R, cp.S) / taps + (resident ? 0.0 : bn * 128.0);
     } else {
-        bytes_per_kb = tm * 128.0 * cp.stride + bn * 128.0;
+        bytes_per_kb = tm * 128.0 + bn * 128.0;
+        // one copy per patch and tap: small patches mean many copies per K block (measured on the strided
+        // 56 x 56 x 256 -> 512 layer: 8 x 4 patches 75.7 us, 16 x 8 patches 62.6 us)
+        copy_issue = 45.0 * halves * std::max(1, 128 / std::max(1, c.patch_w * c.patch_h));
     }
-    const double l2 = bytes_per_kb / (bn < 128 ? 46.0 : 70.0);
+    const double l2 = bytes_per_kb / (bn < 128 ? 46.0 : 70.0) + copy_issue;
     const double main_loop = static_cast<double>(num_kb) * std::max(mma, l2);
     const double blocks = halves * 4.0 * (bn / 32.0);
     const double epi = c.store_mode == 2 ? 600.0 * std::ceil(blocks / 16.0) : 1200.0 * std::ceil(blocks / (4.0 * halves));
     const bool overlapped = tmem_slots_for(tm, bn) > halves;
     const double rounds = std::ceil(static_cast<double>(tiles) / sm_count);
     const double per_tile = overlapped ? std::max(main_loop, epi) : main_loop + epi;
-    const double cycles = 5500.0 + rounds * per_tile + (overlapped ? epi : 0.0);
+    // between configurations with the same number of rounds, the one with less work in total (fewer wasted rows) wins
+    const double cycles = 5500.0 + rounds * per_tile + (overlapped ? epi : 0.0) + 1e-3 * static_cast<double>(tiles) * per_tile / sm_count;
     const double hbm_us = (static_cast<double>(cp.N) * cp.H * cp.W * cp.Cin + static_cast<double>(cp.Cout) * taps * cp.Cin +
                            static_cast<double>(cp.N) * cp.P * cp.Q * cp.Cout) * 2.0 / 5.0e6;
     return std::max(cycles / clk_mhz, hbm_us);

@@ -195,7 +195,7 @@ def test_default_configs():
     st, c = tdx.tdx_default_conv2d_config(4, 128, 128, 64, 64, 3, 3, 1, 1, tdx.TDX_BF16)
     assert st == tdx.TDX_OK and (c.patch_w, c.patch_h, c.halo) == (8, 16, 2) and c.tile_n == 64
     st, c = tdx.tdx_default_conv2d_config(4, 128, 128, 64, 64, 1, 1, 0, 1, tdx.TDX_BF16)          # 1 x 1: nothing to reuse
-    assert st == tdx.TDX_OK and (c.patch_w, c.patch_h, c.halo) == (128, 1, 1)
+    assert st == tdx.TDX_OK and c.halo == 1 and c.patch_w * c.patch_h in (32, 64, 128)
     st, c = tdx.tdx_default_conv2d_config(4, 64, 64, 64, 256, 9, 9, 4, 1, tdx.TDX_BF16)           # halo tile too large
     assert st == tdx.TDX_OK and c.halo in (1, 2, 3) and c.stages >= 2
 
