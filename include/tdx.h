@@ -24,6 +24,10 @@
  *    cudaMalloc and reused from call to call in stream order: calls that use it must all be issued on ONE stream per
  *    device, and from one host thread at a time.  Calls that use none (bf16 GEMM / convolution without split-K, or
  *    with a caller workspace through the _ex entry points) have no such restriction; the caches behind them are locked.
+ *  - Environment: TDX_TUNE_CACHE (read by the Python binding: a tuning-cache file to load instead of the shipped one, "0"
+ *    for none).  TDX_FORCE_CONFIG="tile_m=128,tile_n=128,split_k=6" (read once by the library): a partial tdx_config
+ *    that tdx_gemm, tdx_gemm_batched (bf16) and tdx_conv2d_bias_relu take instead of the automatic choice; an infeasible
+ *    one fails those calls with TDX_ERR_CONFIG like an explicit configuration would.
  */
 #ifndef TDX_H_
 #define TDX_H_

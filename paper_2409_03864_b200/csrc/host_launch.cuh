@@ -854,21 +854,36 @@ int run_gemm_batched_bf16(DeviceCtx* ctx, const GemmProblem& g, float alpha, flo
     want.store_mode = 1;          // direct stores: they carry the batch offset and the accumulate term
     want.cta_pair = 1;
     want.fit = 1;
+    // The batches multiply the tiles, so the ranking sees them: one problem with the row blocks of all batches stacked
+    // (the paper's 6 x 196 x 256 x 2305 batch: 128 x 128 tiles with a K split, 19.4 us; ranked on one batch alone it
+    // took 128 x 32 tiles without a split, 28.7 us).  256-row tiles only where they waste no more rows than 128-row ones.
     tdx_config ranked;
-    if (model_pick_direct_store(gg, ctx->sm_count, ctx->smem_optin, &ranked)) {
-        want.tile_m = ranked.tile_m;
+    GemmProblem stacked = gg;
+    stacked.M = batch * ceil_div(g.M, 128) * 128;
+    if (model_pick_direct_store(stacked, ctx->sm_count, ctx->smem_optin, &ranked)) {
+        want.tile_m = (ceil_div(g.M, 256) * 256 > ceil_div(g.M, 128) * 128) ? 128 : ranked.tile_m;
         want.tile_n = ranked.tile_n;
         want.raster = ranked.raster;
         want.split_k = ranked.split_k;
     }
+    const tdx_config* forced = forced_config();          // TDX_FORCE_CONFIG: tile shape, depth and K split as given
+    if (forced != nullptr) {
+        if (forced->tile_m) want.tile_m = forced->tile_m;
+        if (forced->tile_n) want.tile_n = forced->tile_n;
+        if (forced->stages) want.stages = forced->stages;
+        if (forced->split_k) want.split_k = forced->split_k;
+        want.raster = forced->raster;
+    }
     tdx_config cfg;
     int rc = resolve_gemm_config(gg, &want, ctx->sm_count, ctx->smem_optin, &cfg);
     if (rc) return rc;
-    if (batch > 1) {
-        // the batches already multiply the tiles: split K only as far as it takes to give every SM an item
+    if (batch > 1 && !(forced != nullptr && forced->split_k)) {
+        // the ranked K split belongs to the stacked problem; keep it within what gives every SM an item
         const int64_t num_kb = ceil_div(gg.K, 64);
         const int64_t tiles = batch * ceil_div(g.M, cfg.tile_m) * ceil_div(g.N, cfg.tile_n);
-        int64_t sk = std::max<int64_t>(1, std::min<int64_t>({32, ctx->sm_count / std::max<int64_t>(1, tiles), num_kb / 4}));
+        int64_t sk = std::max<int64_t>(1, std::min<int64_t>({32, ceil_div(ctx->sm_count, std::max<int64_t>(1, tiles)), num_kb / 4,
+                                                            std::max<int64_t>(1, cfg.split_k)}));
+        if (cfg.split_k <= 1) sk = std::max<int64_t>(1, std::min<int64_t>({32, ctx->sm_count / std::max<int64_t>(1, tiles), num_kb / 4}));
         while (sk > 1 && (sk - 1) * ceil_div(num_kb, sk) >= num_kb) --sk;
         cfg.split_k = static_cast<int>(sk);
     }

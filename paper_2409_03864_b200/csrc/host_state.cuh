@@ -226,6 +226,50 @@ bool tune_lookup_gemm(int64_t M, int64_t N, int64_t K, int tA, int tB, int dtype
     if (memo.found) *out = memo.cfg;
     return memo.found;
 }
+// TDX_FORCE_CONFIG="tile_m=128,tile_n=128,split_k=6": a partial tile configuration that calls WITHOUT an explicit
+// configuration take instead of the automatic choice (tuning cache, cost model) -- for experiments and for pinning a
+// deployment to a known configuration without rebuilding the caller.  Read once per process; unknown names or values
+// that are not integers make the variable void (reported once on stderr).  Fields not named stay "choose for me".
+const tdx_config* forced_config() {
+    static tdx_config cfg;
+    static int state = 0;            // 0 = not read yet, 1 = none, 2 = valid
+    static std::mutex mu;
+    std::lock_guard<std::mutex> lk(mu);
+    if (state == 0) {
+        state = 1;
+        const char* env = std::getenv("TDX_FORCE_CONFIG");
+        if (env != nullptr && *env != '\0') {
+            std::memset(&cfg, 0, sizeof cfg);
+            bool ok = true;
+            std::string text(env);
+            size_t pos = 0;
+            while (ok && pos < text.size()) {
+                const size_t comma = text.find(',', pos);
+                const std::string item = text.substr(pos, comma == std::string::npos ? std::string::npos : comma - pos);
+                pos = comma == std::string::npos ? text.size() : comma + 1;
+                const size_t eq = item.find('=');
+                if (eq == std::string::npos) { ok = false; break; }
+                const std::string name = item.substr(0, eq);
+                char* end = nullptr;
+                const long v = std::strtol(item.c_str() + eq + 1, &end, 10);
+                if (end == item.c_str() + eq + 1 || *end != '\0') { ok = false; break; }
+                struct { const char* n; int* f; } fields[] = {
+                    {"kernel", &cfg.kernel}, {"tile_m", &cfg.tile_m}, {"tile_n", &cfg.tile_n}, {"tile_k", &cfg.tile_k},
+                    {"stages", &cfg.stages}, {"cta_pair", &cfg.cta_pair}, {"split_k", &cfg.split_k}, {"store_mode", &cfg.store_mode},
+                    {"raster", &cfg.raster}, {"patch_w", &cfg.patch_w}, {"patch_h", &cfg.patch_h}, {"k_stagger", &cfg.k_stagger},
+                    {"halo", &cfg.halo}, {"fit", &cfg.fit}};
+                bool found = false;
+                for (auto& f : fields)
+                    if (name == f.n) { *f.f = static_cast<int>(v); found = true; }
+                ok = found;
+            }
+            if (ok) state = 2;
+            else fprintf(stderr, "tdx: TDX_FORCE_CONFIG=\"%s\" is not a list of <field>=<integer>; ignored\n", env);
+        }
+    }
+    return state == 2 ? &cfg : nullptr;
+}
+
 void cfg_to_ints(const tdx_config& c, int* v) {
     v[0] = c.kernel; v[1] = c.tile_m; v[2] = c.tile_n; v[3] = c.tile_k; v[4] = c.stages; v[5] = c.cta_pair;
     v[6] = c.split_k; v[7] = c.store_mode; v[8] = c.raster; v[9] = c.patch_w; v[10] = c.patch_h; v[11] = c.k_stagger;

@@ -772,6 +772,16 @@ extern "C" {
 
 int tdx_gemm(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha, int dtype, const void* A,
              const void* B, void* C, void* stream) {
+    // TDX_FORCE_CONFIG stands in for the automatic choice where the shape can take the tensor-core path at all
+    const tdx_config* forced = forced_config();
+    if (forced != nullptr && M > 0 && N > 0 && K > 0) {
+        GemmProblem g{M, N, K, transA, transB, dtype};
+        tdx_config f = *forced;
+        if (f.kernel == 0) f.kernel = TDX_KERNEL_UMMA;
+        if (f.kernel != TDX_KERNEL_UMMA || (dtype == TDX_BF16 && gemm_umma_layout_ok(g) && reinterpret_cast<uintptr_t>(A) % 16 == 0 &&
+                                            reinterpret_cast<uintptr_t>(B) % 16 == 0))
+            return gemm_dispatch(M, N, K, transA, transB, alpha, dtype, A, B, C, stream, &f, nullptr, 0, true);
+    }
     return gemm_dispatch(M, N, K, transA, transB, alpha, dtype, A, B, C, stream, nullptr, nullptr, 0, true);
 }
 
@@ -965,6 +975,12 @@ int tdx_gemm_workspace_size(int64_t M, int64_t N, int64_t K, int dtype, const td
 int tdx_conv2d_bias_relu(int64_t N, int64_t H, int64_t W, int64_t Cin, int64_t Cout, int64_t R, int64_t S, int pad,
                          int stride, int dtype, const void* x, const void* w, const float* bias, int relu, void* y,
                          void* stream) {
+    const tdx_config* forced = forced_config();
+    if (forced != nullptr && dtype == TDX_BF16) {
+        tdx_config f = *forced;
+        if (f.kernel == 0) f.kernel = TDX_KERNEL_UMMA;
+        return conv_dispatch(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, relu, y, stream, &f);
+    }
     return conv_dispatch(N, H, W, Cin, Cout, R, S, pad, stride, dtype, x, w, bias, relu, y, stream, nullptr);
 }
 

@@ -316,3 +316,20 @@ def test_k_balanced_config_constraints_and_workspace_size():
     assert st == 0 and any(c["fit"] == 3 for c in cfgs)
     st, cfgs = tdx.tdx_enum_gemm_configs(8192, 8192, 8192, 0, 0, tdx.TDX_BF16)
     assert st == 0 and not any(c["fit"] == 3 for c in cfgs)                   # many tiles: nothing to balance
+
+
+def test_force_config_environment_variable():
+    # read once per process, so each case runs in a child process; host only (the default-config query shows nothing of
+    # it -- the override applies to calls -- so an infeasible forced configuration is the observable: CONFIG before any
+    # device work, with the variable's fields in the message)
+    import subprocess
+    import sys
+    code = ("import paper_2409_03864_b200 as tdx; "
+            "st = tdx.tdx_gemm(512, 512, 512, 0, 1, 1.0, tdx.TDX_BF16, 256, 512, 1024); "
+            "print(st, tdx.tdx_last_error())")
+    env = dict(os.environ, TDX_FORCE_CONFIG="tile_m=128,tile_n=48")
+    r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, cwd=ROOT, timeout=120)
+    assert r.returncode == 0 and r.stdout.split()[0] == str(tdx.TDX_ERR_CONFIG) and "tile_n" in r.stdout, r.stdout + r.stderr
+    env = dict(os.environ, TDX_FORCE_CONFIG="tile_q=3")
+    r = subprocess.run([sys.executable, "-c", code], env=env, capture_output=True, text=True, cwd=ROOT, timeout=120)
+    assert "ignored" in r.stderr and r.stdout.split()[0] != str(tdx.TDX_ERR_CONFIG)      # void: the call proceeds (and finds no device here)
