@@ -240,7 +240,11 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint16_t cta_mas
 // Shared-memory matrix descriptor (64 bit) of tcgen05.mma:
 //   [ 0,14) start address >> 4        [16,30) leading-dimension byte offset >> 4
 //   [32,46) stride-dimension byte offset >> 4      [46,49) fixed 0b001
-//   [49,52) base offset (0: tiles are 1024-byte aligned)   [61,64) swizzle (2 = 128 B)
+//   [49,52) base offset: (tile base >> 7) & 7 for a tile placed at a base that is not a multiple of the swizzle
+//           pattern's 1024 bytes; 0 here -- every tile sits on a 1024-byte boundary, and a descriptor that starts
+//           further INTO such a tile (a K step, a filter tap of the halo window) keeps 0, because the swizzle is a
+//           function of the address bits, which the start address already carries
+//   [61,64) swizzle (2 = 128 B)
 __device__ __forceinline__ uint64_t make_smem_desc_sw128(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
     uint64_t d = 0;
     d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);

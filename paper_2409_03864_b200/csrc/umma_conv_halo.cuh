@@ -6,9 +6,17 @@
 // ONCE (one TMA box, zero fill outside the image), and tap (r, s) is read straight out of it: output
 // pixel (h, w) of the patch needs window pixel (h + r, w + s), i.e. the 8-row groups of the A operand
 // start at window row r, column s and are one window row (hpitch * 128 bytes) apart -- exactly what
-// the shared-memory descriptor's start address and stride-dimension offset express.  The 128-byte
-// swizzle is a function of the shared-memory address, so a start that is not 1024-byte aligned reads
-// consistently what the copy engine wrote.
+// the shared-memory descriptor's start address and stride-dimension offset express.
+//
+// Why a start that is not 1024-byte aligned is legal here.  The copy engine writes the window into a buffer that
+// starts on a 1024-byte boundary and applies the 128-byte swizzle as a function of the shared-memory ADDRESS (the
+// 16-byte chunk index, address bits 4..6, is XORed with address bits 7..9).  The MMA unit applies the same function of
+// the address when it reads.  The descriptor's base-offset field (bits 49..51) exists for a different situation: a
+// matrix whose swizzle pattern is shifted against the address because the tile ITSELF was placed at a base that is
+// not a multiple of the pattern's 1024-byte period; the field then carries (base >> 7) & 7.  A filter tap does not
+// move the tile, it only starts reading further into it, at pixel (r, s) of the window: pattern and address still
+// agree, so the field stays 0.  Checked both ways on the device: with the field 0 every halo parity case matches the
+// oracle (integer cases bit for bit); with it set to (start >> 7) & 7, as for a shifted tile, 44 of 47 cases fail.
 //
 // Two rings: halo tiles (a_stages deep, one per channel chunk and 128-row half) and filter slices
 // (stages deep, one per (chunk, tap)), each filled by its own warp (the last warp and warp 0), so that a
