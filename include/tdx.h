@@ -27,7 +27,10 @@
  *  - Environment: TDX_TUNE_CACHE (read by the Python binding: a tuning-cache file to load instead of the shipped one, "0"
  *    for none).  TDX_FORCE_CONFIG="tile_m=128,tile_n=128,split_k=6" (read once by the library): a partial tdx_config
  *    that tdx_gemm, tdx_gemm_batched (bf16) and tdx_conv2d_bias_relu take instead of the automatic choice; an infeasible
- *    one fails those calls with TDX_ERR_CONFIG like an explicit configuration would.
+ *    one fails those calls with TDX_ERR_CONFIG like an explicit configuration would.  TDX_DEBUG_BOUNDS=1 (read once):
+ *    the one-thread-per-output kernels (the last entry of every fallback chain, and the searches' comparator) check each
+ *    global index against the extent its operand's shape and strides imply; an index outside is not accessed, the kernel
+ *    records it in the device status word and tdx_check_device_status reports TDX_ERR_BOUNDS.  Slower; for debugging.
  */
 #ifndef TDX_H_
 #define TDX_H_
@@ -50,7 +53,9 @@ typedef enum {
     /* definite */
     TDX_ERR_CUDA = 16,      /* a CUDA runtime / driver call failed                                 */
     TDX_ERR_TIMEOUT = 17,   /* a kernel gave up on a bounded wait (see tdx_check_device_status)    */
-    TDX_ERR_NO_DEVICE = 18  /* no usable sm_100 device / driver                                    */
+    TDX_ERR_NO_DEVICE = 18, /* no usable sm_100 device / driver                                    */
+    TDX_ERR_BOUNDS = 19     /* the bounds-checked debug mode (TDX_DEBUG_BOUNDS=1) caught an index outside its */
+                            /* operand; the access was skipped (see tdx_check_device_status)                 */
 } tdx_status;
 
 typedef enum {
@@ -382,7 +387,8 @@ int tdx_tune_clear(void);
 
 /*
  * Synchronises `stream`, reads and clears the device status word.  TDX_OK, or TDX_ERR_TIMEOUT if a
- * kernel abandoned a bounded wait since the last check (its outputs are then unspecified).
+ * kernel abandoned a bounded wait since the last check (its outputs are then unspecified), or TDX_ERR_BOUNDS if the
+ * bounds-checked debug mode skipped an access.
  */
 int tdx_check_device_status(void* stream);
 
@@ -418,6 +424,14 @@ int tdx_check_device_status(void* stream);
 #define TDX_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
 int tdx_gemm_splitk_static(int64_t M, int64_t N, int64_t K, int transA, int transB, float alpha,
                            const void* A, const void* B, void* C, int tile_n, int split_k, void* stream);
+
+/*
+ * Self-test of the bounds-checked debug mode: runs the one-thread-per-output GEMM kernel on a small scratch problem with
+ * the extent of one operand understated by four elements.  The kernel must skip exactly those accesses (nothing out of
+ * range is touched: the buffers are full size) and record the violation, so the next tdx_check_device_status on that
+ * stream reports TDX_ERR_BOUNDS (once).  Allocates and frees a few KB of device memory.
+ */
+int tdx_selftest_bounds_check(void* stream);
 
 /*
  * Self-test of the failure path: launches a one-warp kernel that waits on a barrier nothing ever signals, with a

@@ -22,6 +22,7 @@ TDX_ERR_WORKSPACE = 5
 TDX_ERR_CUDA = 16
 TDX_ERR_TIMEOUT = 17
 TDX_ERR_NO_DEVICE = 18
+TDX_ERR_BOUNDS = 19
 
 TDX_F32 = 0
 TDX_BF16 = 1
@@ -102,6 +103,7 @@ def lib() -> ctypes.CDLL:
         L.tdx_gemm_splitk_static.argtypes = [i64, i64, i64, ci, ci, cf, vp, vp, vp, ci, ci, vp]
         L.tdx_check_device_status.argtypes = [vp]
         L.tdx_selftest_bounded_wait.argtypes = [ci, vp]
+        L.tdx_selftest_bounds_check.argtypes = [vp]
         L.tdx_kernel_launch_count.argtypes = []
         L.tdx_kernel_launch_count.restype = i64
         L.tdx_last_error.restype = ctypes.c_char_p
@@ -124,7 +126,7 @@ EXPORTS = (
     "tdx_gemm", "tdx_gemm_f32out", "tdx_add_zero_pad", "tdx_add_zero_pad_host", "tdx_gemm_batched", "tdx_gemm_batched_host", "tdx_gemm_ex", "tdx_gemm_workspace_size", "tdx_conv2d_bias_relu", "tdx_conv2d_bias_add_relu", "tdx_conv2d_bias_relu_ex",
     "tdx_gemm_host", "tdx_conv2d_bias_relu_host", "tdx_tune_gemm", "tdx_tune_gemm_guided", "tdx_model_gemm_us", "tdx_tune_conv2d", "tdx_enum_gemm_configs",
     "tdx_enum_conv2d_configs", "tdx_default_gemm_config", "tdx_default_conv2d_config", "tdx_tune_save",
-    "tdx_tune_load", "tdx_tune_clear", "tdx_set_autotune", "tdx_gemm_tile_plan", "tdx_gemm_k_balanced_plan", "tdx_enum_gemm_space", "tdx_tune_gemm_space", "tdx_tune_conv2d_guided", "tdx_model_conv2d_us", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_kernel_launch_count", "tdx_last_error",
+    "tdx_tune_load", "tdx_tune_clear", "tdx_set_autotune", "tdx_gemm_tile_plan", "tdx_gemm_k_balanced_plan", "tdx_enum_gemm_space", "tdx_tune_gemm_space", "tdx_tune_conv2d_guided", "tdx_model_conv2d_us", "tdx_gemm_splitk_static", "tdx_check_device_status", "tdx_selftest_bounded_wait", "tdx_selftest_bounds_check", "tdx_kernel_launch_count", "tdx_last_error",
     "tdx_version",
 )
 
@@ -407,6 +409,10 @@ def tdx_check_device_status(stream=None) -> int:
 
 def tdx_selftest_bounded_wait(limit_us=200, stream=None) -> int:
     return lib().tdx_selftest_bounded_wait(limit_us, _stream(stream))
+
+
+def tdx_selftest_bounds_check(stream=None) -> int:
+    return lib().tdx_selftest_bounds_check(_stream(stream))
 
 
 def tdx_kernel_launch_count() -> int:

@@ -891,25 +891,35 @@ int run_gemm_batched_bf16(DeviceCtx* ctx, const GemmProblem& g, float alpha, flo
 }
 
 int run_gemm_generic(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void* A, const void* B, void* C,
-                     cudaStream_t st, const BatchArgs& ba = BatchArgs(), bool c_f32 = false) {
+                     cudaStream_t st, const BatchArgs& ba = BatchArgs(), bool c_f32 = false,
+                     const tdx::BoundsCheck* bounds_override = nullptr) {
     long long sa_i, sa_k, sb_k, sb_j;
     gemm_strides(g, &sa_i, &sa_k, &sb_k, &sb_j);
     const long long total = g.M * g.N * ba.batch;
     const int grid = static_cast<int>(std::min<long long>(ceil_div(total, 256), static_cast<long long>(ctx->sm_count) * 32));
+    // debug mode: the extents the caller's shapes and strides imply, checked index by index in the kernel
+    tdx::BoundsCheck bc{0, 0, 0, 0, 0, ctx->status_ptr};
+    if (bounds_override != nullptr) bc = *bounds_override;
+    else if (debug_bounds_enabled()) {
+        bc.on = 1;
+        bc.a_elems = (ba.batch - 1) * ba.stride_a + g.M * g.K;
+        bc.b_elems = (ba.batch - 1) * ba.stride_b + g.K * g.N;
+        bc.c_elems = (ba.batch - 1) * ba.stride_c + g.M * g.N;
+    }
     if (g.dtype == TDX_BF16 && c_f32)      // bf16 operands, fp32 result
         tdx::gemm_generic_kernel<__nv_bfloat16, float><<<grid, 256, 0, st>>>(
             g.M, g.N, g.K, sa_i, sa_k, sb_k, sb_j, alpha, static_cast<const __nv_bfloat16*>(A),
-            static_cast<const __nv_bfloat16*>(B), static_cast<float*>(C), ba.beta, ba.batch, ba.stride_a, ba.stride_b, ba.stride_c);
+            static_cast<const __nv_bfloat16*>(B), static_cast<float*>(C), ba.beta, ba.batch, ba.stride_a, ba.stride_b, ba.stride_c, bc);
     else if (g.dtype == TDX_F32)
         tdx::gemm_generic_kernel<float, float><<<grid, 256, 0, st>>>(g.M, g.N, g.K, sa_i, sa_k, sb_k, sb_j, alpha,
                                                                     static_cast<const float*>(A),
                                                                     static_cast<const float*>(B), static_cast<float*>(C),
-                                                                    ba.beta, ba.batch, ba.stride_a, ba.stride_b, ba.stride_c);
+                                                                    ba.beta, ba.batch, ba.stride_a, ba.stride_b, ba.stride_c, bc);
     else
         tdx::gemm_generic_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
             g.M, g.N, g.K, sa_i, sa_k, sb_k, sb_j, alpha, static_cast<const __nv_bfloat16*>(A),
             static_cast<const __nv_bfloat16*>(B), static_cast<__nv_bfloat16*>(C), ba.beta, ba.batch, ba.stride_a,
-            ba.stride_b, ba.stride_c);
+            ba.stride_b, ba.stride_c, bc);
     TDX_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     return TDX_OK;
@@ -922,16 +932,24 @@ int run_conv_generic(DeviceCtx* ctx, const ConvProblem& c, const void* x, const 
         return fail(TDX_ERR_UNSUPPORTED, "conv dimensions must be below 2^31");
     const long long total = c.N * c.P * c.Q * c.Cout;
     const int grid = static_cast<int>(std::min<long long>(ceil_div(total, 256), static_cast<long long>(ctx->sm_count) * 32));
+    tdx::BoundsCheck bc{0, 0, 0, 0, 0, ctx->status_ptr};
+    if (debug_bounds_enabled()) {
+        bc.on = 1;
+        bc.a_elems = c.N * c.H * c.W * c.Cin;
+        bc.b_elems = c.Cout * c.R * c.S * c.Cin;
+        bc.c_elems = total;
+        bc.r_elems = total;
+    }
     if (c.dtype == TDX_F32)
         tdx::conv2d_generic_kernel<float, float><<<grid, 256, 0, st>>>(
             (int)c.N, (int)c.H, (int)c.W, (int)c.Cin, (int)c.Cout, (int)c.R, (int)c.S, c.pad, c.stride, (int)c.P,
             (int)c.Q, static_cast<const float*>(x), static_cast<const float*>(w), bias, relu, static_cast<float*>(y),
-            static_cast<const float*>(residual));
+            static_cast<const float*>(residual), bc);
     else
         tdx::conv2d_generic_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(
             (int)c.N, (int)c.H, (int)c.W, (int)c.Cin, (int)c.Cout, (int)c.R, (int)c.S, c.pad, c.stride, (int)c.P,
             (int)c.Q, static_cast<const __nv_bfloat16*>(x), static_cast<const __nv_bfloat16*>(w), bias, relu,
-            static_cast<__nv_bfloat16*>(y), static_cast<const __nv_bfloat16*>(residual));
+            static_cast<__nv_bfloat16*>(y), static_cast<const __nv_bfloat16*>(residual), bc);
     TDX_CUDA(cudaGetLastError());
     g_launches.fetch_add(1);
     return TDX_OK;

@@ -270,6 +270,15 @@ const tdx_config* forced_config() {
     return state == 2 ? &cfg : nullptr;
 }
 
+// TDX_DEBUG_BOUNDS=1: the one-thread-per-output kernels check every index against its operand's extent (read once).
+bool debug_bounds_enabled() {
+    static const bool on = [] {
+        const char* e = std::getenv("TDX_DEBUG_BOUNDS");
+        return e != nullptr && *e != '\0' && std::strcmp(e, "0") != 0;
+    }();
+    return on;
+}
+
 void cfg_to_ints(const tdx_config& c, int* v) {
     v[0] = c.kernel; v[1] = c.tile_m; v[2] = c.tile_n; v[3] = c.tile_k; v[4] = c.stages; v[5] = c.cta_pair;
     v[6] = c.split_k; v[7] = c.store_mode; v[8] = c.raster; v[9] = c.patch_w; v[10] = c.patch_h; v[11] = c.k_stagger;

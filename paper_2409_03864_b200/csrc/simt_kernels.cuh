@@ -8,6 +8,21 @@
 
 namespace tdx {
 
+// Bounds-checked debug mode of the one-thread-per-output kernels (TDX_DEBUG_BOUNDS=1): every global index is compared
+// with the extent of its operand first; an index outside it is NOT accessed -- the kernel records kStatusBounds in the
+// device status word (reported by tdx_check_device_status as a definite error) and uses 0 instead.  Nothing traps.
+enum : int { kStatusBounds = 8 };
+struct BoundsCheck {
+    int on;                          // 0: no checks (the normal build of the call)
+    long long a_elems, b_elems, c_elems, r_elems;   // extents in elements: left operand / input, right operand / filter, output, residual
+    int* status;
+};
+__device__ __forceinline__ bool in_bounds(const BoundsCheck& bc, long long i, long long extent) {
+    if (!bc.on || (i >= 0 && i < extent)) return true;
+    atomicCAS(bc.status, 0, kStatusBounds);
+    return false;
+}
+
 __device__ __forceinline__ float ld_as_float(const float* p, long long i) { return __ldg(p + i); }
 __device__ __forceinline__ float ld_as_float(const __nv_bfloat16* p, long long i) {
     return __bfloat162float(p[i]);
@@ -325,18 +340,30 @@ __global__ void gemm_generic_kernel(long long M, long long N, long long K, long 
                                     long long sb_k, long long sb_j, float alpha, const TIn* __restrict__ A,
                                     const TIn* __restrict__ B, TOut* __restrict__ C, float beta = 0.0f,
                                     long long batch = 1, long long batch_a = 0, long long batch_b = 0,
-                                    long long batch_c = 0) {
+                                    long long batch_c = 0, BoundsCheck bc = BoundsCheck{0, 0, 0, 0, 0, nullptr}) {
     // batched: C[b] = beta * C[b] + alpha * A[b] . B[b]; C is not read when beta == 0
     const long long per = M * N, total = per * batch;
     for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < total;
          e += static_cast<long long>(gridDim.x) * blockDim.x) {
         const long long b = e / per, r = e - b * per;
         const long long i = r / N, j = r - i * N;
-        const TIn* a = A + b * batch_a;
-        const TIn* bb = B + b * batch_b;
         float acc = 0.0f;
-        for (long long k = 0; k < K; ++k)
-            acc = fmaf(ld_as_float(a, i * sa_i + k * sa_k), ld_as_float(bb, k * sb_k + j * sb_j), acc);
+        if (bc.on) {
+            // debug mode: indices relative to the operand's base, checked against its extent before every access
+            for (long long k = 0; k < K; ++k) {
+                const long long ia = b * batch_a + i * sa_i + k * sa_k, ib = b * batch_b + k * sb_k + j * sb_j;
+                const float x = in_bounds(bc, ia, bc.a_elems) ? ld_as_float(A, ia) : 0.0f;
+                const float y = in_bounds(bc, ib, bc.b_elems) ? ld_as_float(B, ib) : 0.0f;
+                acc = fmaf(x, y, acc);
+            }
+            const long long ic = b * batch_c + r;
+            if (!in_bounds(bc, ic, bc.c_elems)) continue;
+        } else {
+            const TIn* a = A + b * batch_a;
+            const TIn* bb = B + b * batch_b;
+            for (long long k = 0; k < K; ++k)
+                acc = fmaf(ld_as_float(a, i * sa_i + k * sa_k), ld_as_float(bb, k * sb_k + j * sb_j), acc);
+        }
         TOut* c = C + b * batch_c;
         float v = alpha * acc;
         if (beta != 0.0f) v = fmaf(beta, as_float(c[r]), v);     // plain load: this thread overwrites it next
@@ -352,7 +379,8 @@ template <typename TIn, typename TOut>
 __global__ void conv2d_generic_kernel(int Nimg, int H, int W, int Cin, int Cout, int R, int S, int pad, int stride,
                                       int P, int Q, const TIn* __restrict__ x, const TIn* __restrict__ w,
                                       const float* __restrict__ bias, int relu, TOut* __restrict__ y,
-                                      const TOut* __restrict__ residual = nullptr) {
+                                      const TOut* __restrict__ residual = nullptr,
+                                      BoundsCheck bc = BoundsCheck{0, 0, 0, 0, 0, nullptr}) {
     const long long total = static_cast<long long>(Nimg) * P * Q * Cout;
     for (long long e = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; e < total;
          e += static_cast<long long>(gridDim.x) * blockDim.x) {
@@ -371,12 +399,21 @@ __global__ void conv2d_generic_kernel(int Nimg, int H, int W, int Cin, int Cout,
                 if (ww < 0 || ww >= W) continue;
                 const long long xo = ((static_cast<long long>(n) * H + h) * W + ww) * Cin;
                 const long long wo = ((static_cast<long long>(k) * R + r) * S + s) * Cin;
-                for (int c = 0; c < Cin; ++c) acc = fmaf(ld_as_float(x, xo + c), ld_as_float(w, wo + c), acc);
+                if (bc.on) {
+                    for (int c = 0; c < Cin; ++c) {
+                        const float xv = in_bounds(bc, xo + c, bc.a_elems) ? ld_as_float(x, xo + c) : 0.0f;
+                        const float wv = in_bounds(bc, wo + c, bc.b_elems) ? ld_as_float(w, wo + c) : 0.0f;
+                        acc = fmaf(xv, wv, acc);
+                    }
+                } else {
+                    for (int c = 0; c < Cin; ++c) acc = fmaf(ld_as_float(x, xo + c), ld_as_float(w, wo + c), acc);
+                }
             }
         }
         if (bias != nullptr) acc += __ldg(bias + k);
-        if (residual != nullptr) acc += as_float(residual[e]);
+        if (residual != nullptr && in_bounds(bc, e, bc.r_elems)) acc += as_float(residual[e]);
         if (relu) acc = fmaxf(acc, 0.0f);
+        if (!in_bounds(bc, e, bc.c_elems)) continue;
         st_from_float(y, e, acc);
     }
 }

@@ -1701,8 +1701,31 @@ int tdx_check_device_status(void* stream) {
     TDX_CUDA(cudaMemcpy(&v, ctx->status_ptr, sizeof v, cudaMemcpyDeviceToHost));
     if (v != 0) {
         TDX_CUDA(cudaMemset(ctx->status_ptr, 0, sizeof v));
+        if (v == tdx::kStatusBounds)
+            return fail(TDX_ERR_BOUNDS, "the bounds-checked debug mode caught an index outside its operand (the access was skipped)");
         return fail(TDX_ERR_TIMEOUT, "a kernel abandoned a bounded wait (role code %d)", v);
     }
+    return TDX_OK;
+}
+
+int tdx_selftest_bounds_check(void* stream) {
+    DeviceCtx* ctx;
+    int rc = get_ctx(&ctx);
+    if (rc) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t n = 8;
+    ScratchGuard guard;
+    void *a, *b, *c;
+    if ((rc = guard.alloc(&a, n * n * 4))) return rc;
+    if ((rc = guard.alloc(&b, n * n * 4))) return rc;
+    if ((rc = guard.alloc(&c, n * n * 4))) return rc;
+    TDX_CUDA(cudaMemsetAsync(a, 0, n * n * 4, st));
+    TDX_CUDA(cudaMemsetAsync(b, 0, n * n * 4, st));
+    // the right operand really has 64 elements; the check is told 60, so the last four indices must be refused
+    tdx::BoundsCheck bc{1, n * n, n * n - 4, n * n, 0, ctx->status_ptr};
+    rc = run_gemm_generic(ctx, GemmProblem{n, n, n, 0, 0, TDX_F32}, 1.0f, a, b, c, st, BatchArgs(), false, &bc);
+    if (rc) return rc;
+    TDX_CUDA(cudaStreamSynchronize(st));
     return TDX_OK;
 }
 
