@@ -85,9 +85,15 @@ typedef struct {
                     /*     CTA stages its 128 rows of A and half of the B slice, one thread issues MMAs    */
                     /*     over both, and each CTA keeps a 128 x tile_n accumulator half                  */
     int split_k;    /* >= 1; > 1 needs a workspace and runs a fixed-order reduction afterwards  */
+                    /*     (store_mode 3: neither, see there)                                    */
     int store_mode; /* 1 = 16-byte stores from registers; 2 = 32 x 32 blocks staged in shared     */
                     /*     memory and written by TMA store (needs N % 8 == 0, split_k = 1,         */
                     /*     16-byte aligned C; falls back to 1 if C is misaligned)                  */
+                    /*     3 = (GEMM, tile_m = 128, split_k in 2..8, tile_n a multiple of 32 * split_k) the   */
+                    /*     split_k CTAs of a tile form a thread-block cluster, exchange column slices of     */
+                    /*     their fp32 partial tiles through distributed shared memory and each writes its    */
+                    /*     slice of the result, summed over the K slices in ascending order: no workspace,   */
+                    /*     no reduction launch.  One CTA per (tile, K slice).                                */
     int raster;     /* width, in tiles along M, of the panels the tile order walks; 0 = all     */
     int patch_w;    /* conv only: output-pixel patch that forms the rows of a tile (w x h,      */
     int patch_h;    /*   w*h a power of two <= 128, w >= 8; tile_m / (w*h) patches per tile); 0 = choose */

@@ -11,9 +11,11 @@ int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensor
     const long long items = static_cast<long long>(p_in.tiles_m) * p_in.tiles_n * p_in.split_k * (p_in.batch > 1 ? p_in.batch : 1);
     UmmaParams p = p_in;
     if (p.b_box == 0) p.b_box = p.bn;
-    const int grid = p.tiles != nullptr ? plan_grid : static_cast<int>(std::min<long long>(items, ctx->sm_count));
+    // cluster reduction: one CTA per (tile, K slice), the split_k CTAs of a tile forming one cluster
+    const int grid = p.tiles != nullptr ? plan_grid
+                                        : static_cast<int>(p.cluster_reduce ? items : std::min<long long>(items, ctx->sm_count));
     size_t smem = static_cast<size_t>(p.stages) * ((p.bm + p.bn) * 128) + 1024 +
-                  staging_bytes_for(p.bm, p.tma_store ? 2 : 1) + (p.partial_tma ? partial_staging_bytes(p.bm) : 0);
+                  staging_bytes_for(p.bm, p.tma_store ? 2 : p.cluster_reduce ? 3 : 1) + (p.partial_tma ? partial_staging_bytes(p.bm) : 0);
     if (halo)
         smem = static_cast<size_t>(p.a_stages) * (p.bm / 128) * p.halo_bytes + static_cast<size_t>(p.stages) * p.bn * 128 +
                1024 + staging_bytes_for(p.bm, p.tma_store ? 2 : 1);
@@ -27,11 +29,18 @@ int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensor
     lc.blockDim = dim3(static_cast<unsigned>(halo ? threads + 32 : threads));   // halo: one more warp, the halo producer
     lc.dynamicSmemBytes = smem;
     lc.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = 1;
+    if (p.cluster_reduce) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = static_cast<unsigned>(p.split_k);
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        lc.numAttrs = 2;
+    }
     if (halo)
         TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_conv_halo_kernel, ma, ma_row ? *ma_row : ma, mb, mc, mc_row ? *mc_row : mc, p));
     else if (conv)
@@ -190,7 +199,14 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         p.rounds = kplan.rounds;
         p.b_box = 64;
     }
-    if (cfg.split_k > 1) {
+    // split-K summed inside clusters: neither workspace nor reduction kernel
+    const bool cluster_reduce = cfg.store_mode == 3 && cfg.split_k > 1;
+    if (cluster_reduce) {
+        if (static_cast<long long>(nbatch) * p.tiles_m * p.tiles_n * cfg.split_k >= (1LL << 31))
+            return fail(TDX_ERR_UNSUPPORTED, "too many tiles for one launch");
+        p.cluster_reduce = 1;
+    }
+    if (cfg.split_k > 1 && !cluster_reduce) {
         const size_t need = static_cast<size_t>(cfg.split_k) * g.M * g.N * sizeof(float) * nbatch;
         if (internal_ws) {
             int rc = ensure_ws(ctx, need, &ws);
@@ -272,6 +288,19 @@ int run_gemm_umma(DeviceCtx* ctx, const GemmProblem& g, float alpha, const void*
         if (rc) return rc;
     }
     if (k_balanced) plan_grid = kplan.grid;
+    if (cluster_reduce) {
+        // the summed slices leave through the copy engine when the result is bf16 with 16-byte aligned rows and there is
+        // no accumulate term; else 16-byte (or element-wise) stores from registers
+        if (p.vec_store && beta == 0.0f && !f32_result && nbatch == 1) {
+            uint64_t dims[2] = {static_cast<uint64_t>(g.N), static_cast<uint64_t>(g.M)};
+            uint64_t str[1] = {static_cast<uint64_t>(g.N) * 2};
+            uint32_t box[2] = {32, 32};
+            rc = get_tensor_map(ctx, C, 2, dims, str, box, &mc, 64);
+            if (rc) return rc;
+            p.cluster_tma = 1;
+        }
+        return launch_umma(ctx, false, ma, mb, mc, p, st, false, nullptr, nullptr, 0);
+    }
     if (p.partial != nullptr && p.split_k > 1) {
         // fp32 partial tiles leave through shared memory and the copy engine (whole 128-byte lines) when the workspace
         // rows allow it and the pipeline leaves room for the staging blocks; else straight from registers

@@ -301,6 +301,14 @@ double model_gemm_us(const GemmProblem& g, const tdx_config& c, int sm_count) {
         const double per_tile = overlapped ? std::max(main_loop, epi) : main_loop + epi;
         cycles = 5500.0 + rounds * per_tile + (overlapped ? epi : 0.0) + (pair ? 4000.0 : 0.0);
     }
+    // split-K summed inside clusters: one CTA per (tile, K slice), nothing overlaps; after the main loop the ranks
+    // exchange (split - 1) / split of a 128 x bn fp32 tile each way through distributed shared memory and store their
+    // slice (measured: 6.7 k cycles for 32 KB sent, 9.9 k for 64 KB)
+    const bool in_cluster = c.store_mode == 3 && split > 1 && !pair;
+    if (in_cluster) {
+        const double sent = 128.0 * bn * 4.0 * (split - 1) / split;
+        cycles = 5500.0 + rounds * (main_loop + 3400.0 + 0.1 * sent);
+    }
     int kbal_slots = 0;
     if (c.fit == 3 && !pair) {
         // K-balanced: every CTA walks its even share of the tiles x K blocks units; a CTA's run touches one or two
@@ -320,7 +328,7 @@ double model_gemm_us(const GemmProblem& g, const tdx_config& c, int sm_count) {
     }
     // split-K: the reduction kernel's launch hides behind the GEMM's tail and the partial sums are still in L2 when it
     // reads them (128 x 8192 x 8192 in three splits: about 4 us on top of the GEMM kernel)
-    if (split > 1) us += 2.0 + (static_cast<double>(split) * g.M * g.N * 4.0 * 2.0 + g.M * g.N * 2.0) / 8.0e6;
+    if (split > 1 && !in_cluster) us += 2.0 + (static_cast<double>(split) * g.M * g.N * 4.0 * 2.0 + g.M * g.N * 2.0) / 8.0e6;
     const double hbm_us = (static_cast<double>(g.M) * g.K + static_cast<double>(g.K) * g.N + static_cast<double>(g.M) * g.N) * 2.0 / 5.0e6;
     return std::max(us, hbm_us);
 }

@@ -174,7 +174,7 @@ int resolve_gemm_config(const GemmProblem& g, const tdx_config* user, int sm_cou
         c.stages = c.cta_pair == 2 ? std::max(2, pair_max_stages(c.tile_n, smem_limit, c.store_mode))
                                    : std::max(2, umma_max_stages(c.tile_m, c.tile_n, smem_limit, c.store_mode));
         // partial tiles (split-K, K-balanced plan): leave room for their staging blocks when that still leaves a pipeline
-        if (c.cta_pair != 2 && (c.split_k > 1 || c.fit == 3) && umma_max_stages_partial(c.tile_m, c.tile_n, smem_limit) >= 3)
+        if (c.cta_pair != 2 && c.store_mode != 3 && (c.split_k > 1 || c.fit == 3) && umma_max_stages_partial(c.tile_m, c.tile_n, smem_limit) >= 3)
             c.stages = std::min(c.stages, umma_max_stages_partial(c.tile_m, c.tile_n, smem_limit));
     }
     if (!user && !from_cache) c.raster = d.raster;
@@ -422,8 +422,9 @@ void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int 
                 for (int s : {2, 3, 4, 6, 8, 16})
                     if (num_kb / s >= 2 && tiles * s <= 4LL * sm_count) splits.push_back(s);
             for (int sk : splits)
-                for (int sm : {2, 1}) {
+                for (int sm : {2, 1, 3}) {
                     if (sm == 2 && (sk > 1 || N % 8)) continue;
+                    if (sm == 3 && (sk == 1 || conv)) continue;     // split-K summed inside a cluster of sk CTAs
                     if (sm == 1 && sk == 1 && N % 8 == 0 && tiles * tm * bn > (1 << 22))
                         continue;                          // large outputs: 16-byte scattered stores never win
                     const int max_st = umma_max_stages(tm, bn, smem_limit, sm);
@@ -433,7 +434,7 @@ void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int 
                     if (max_st - 2 >= 3) stage_opts.push_back(max_st - 2);
                     // split-K: also the deepest pipeline that leaves room for staging the partial tiles
                     const int staged_st = umma_max_stages_partial(tm, bn, smem_limit);
-                    if (sk > 1 && staged_st >= 3 && std::find(stage_opts.begin(), stage_opts.end(), staged_st) == stage_opts.end())
+                    if (sk > 1 && sm == 1 && staged_st >= 3 && std::find(stage_opts.begin(), stage_opts.end(), staged_st) == stage_opts.end())
                         stage_opts.push_back(staged_st);
                     for (int st : stage_opts)
                         for (int raster : {0, 8, 2, 4, 16})
@@ -960,6 +961,7 @@ int tdx_gemm_workspace_size(int64_t M, int64_t N, int64_t K, int dtype, const td
     if (dtype != TDX_F32 && dtype != TDX_BF16) return fail(TDX_ERR_INVALID_ARG, "unknown dtype %d", dtype);
     const int split = cfg ? std::max(cfg->split_k, 1) : 1;
     *bytes = split > 1 ? static_cast<size_t>(split) * M * N * sizeof(float) : 0;
+    if (cfg && cfg->store_mode == 3) *bytes = 0;       // summed inside clusters: no partial tiles in global memory
     if (cfg && cfg->fit == 3 && M > 0 && N > 0 && K > 0) {
         // K-balanced plan: as many slots as the most finely cut tile has pieces (depends on the SM count)
         int sm_count, smem_limit;

@@ -61,6 +61,13 @@ struct UmmaParams {
     int tma_store;            // final output leaves through shared memory + TMA store (needs bn % 64 == 0)
     int partial_tma;          // split-K: fp32 partial tiles leave through shared memory + TMA store (tmC then maps the
                               // workspace as (N, M, batch * split) floats; two 32 x 32 fp32 blocks per epilogue warp)
+    int cluster_reduce;       // split-K summed inside a thread-block cluster of split_k CTAs (GEMM, 128-row tiles, one
+                              // tile per CTA): CTA rank s of a cluster reduces K slice s of the cluster's tile, then
+                              // the ranks exchange column slices of their partial tiles through distributed shared
+                              // memory and rank q writes columns [q, q + 1) * bn / split_k of the result -- no
+                              // workspace and no reduction kernel.  The sum runs over the slices in ascending order.
+    int cluster_tma;          // cluster reduction: the summed slice leaves as 32 x 32 bf16 blocks through shared memory and
+                              // the copy engine (tmC maps C as for the staged epilogue); else 16-byte stores from registers
     int sbx, sby;             // conv TMA-store box: sbx x sby output pixels (sbx * sby = 32)
     // convolution geometry (kConv only)
     int bw, bh, nb;           // spatial patch (bw x bh output pixels), patches per tile = bm / (bw*bh)
@@ -269,6 +276,13 @@ __device__ __forceinline__ void issue_kblock(const UmmaParams& p, const CUtensor
     }
 }
 
+// Slot layout of the cluster reduction: a slot holds one rank's 128 x slice partial sums for the rank that owns the
+// slice, as [lane quarter][4-column group][row within the quarter][16 bytes]: the 32 rows of a warp lie side by side
+// (no bank conflicts on either end) and a warp's 32-column step is one contiguous 4 KB piece.
+__device__ __forceinline__ uint32_t cluster_slot_offset(int quarter, int slice, int c_in_slice, int lane) {
+    return (static_cast<uint32_t>(quarter * (slice >> 2) + (c_in_slice >> 2)) * 32u + static_cast<uint32_t>(lane)) * 16u;
+}
+
 // Epilogue role (all warps from the third on).  With the staged epilogue there are 16 of them (4 per TMEM
 // lane quarter) and the warps of a quarter take the 32-column steps round robin; the direct epilogue has one
 // warp per quarter and 128-row half.
@@ -278,7 +292,12 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                                               volatile int* abort_flag, int mh, int warp, int lane, int total_items,
                                               int first_item = -1, int item_stride = 0, int m_mul = 1, int m_add = 0,
                                               uint32_t tempty_cluster_addr = 0, const CUtensorMap* tmC_row = nullptr,
-                                              const TileCoord* t_first = nullptr, bool have_first = false) {
+                                              const TileCoord* t_first = nullptr, bool have_first = false,
+                                              const uint8_t* recv = nullptr, int my_rank = 0) {
+    // recv != nullptr (cluster reduction): `t_first` is this rank's column slice of the cluster's tile, its accumulator
+    // columns start my_rank * t.bn into the slot, and the other ranks' partial sums of the slice lie in `recv`
+    const bool reduce_here = recv != nullptr;
+    const int tmem_col_off = reduce_here ? my_rank * t_first->bn : 0;
     // CTA pairs: the pair walks tiles of 256 rows, this CTA owns rows [128 * (2 m + rank), +128) of tile m, and the
     // accumulator-free signal goes to the leader CTA's barrier (tempty_cluster_addr, a shared::cluster address)
     if (first_item < 0) {
@@ -481,11 +500,35 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
         for (int c0 = 0; c0 < t.bn; c0 += 32) {
             uint32_t r[32];
             const uint32_t taddr =
-                tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * p.bn + c0);
+                tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(buf * p.bn + tmem_col_off + c0);
             ptx::tmem_ld_32x32b_x32(taddr, r);
             ptx::tmem_ld_wait();
             const int col0 = t.n0 + c0;
-            if (p.split_k > 1 && p.partial_tma) {
+            if (reduce_here) {
+                // slices in ascending order, this rank's own (from tensor memory) in its place: the result does not
+                // depend on which rank writes it
+                float sum[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) sum[j] = 0.0f;
+                const uint32_t slot_bytes = static_cast<uint32_t>(kHalfM) * static_cast<uint32_t>(t.bn) * 4u;
+                const uint32_t in_slot = cluster_slot_offset(quarter, t.bn, c0, lane);
+                for (int s = 0; s < p.split_k; ++s) {
+                    if (s == my_rank) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) sum[j] += __uint_as_float(r[j]);
+                    } else {
+                        const uint8_t* src = recv + static_cast<uint32_t>(s < my_rank ? s : s - 1) * slot_bytes + in_slot;
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            const float4 v = *reinterpret_cast<const float4*>(src + g * 512);
+                            sum[4 * g] += v.x; sum[4 * g + 1] += v.y; sum[4 * g + 2] += v.z; sum[4 * g + 3] += v.w;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(sum[j]);
+            }
+            if (p.split_k > 1 && p.partial_tma && !reduce_here) {
                 // fp32 partial tile through shared memory: the thread writes its row's 32 values (128 bytes, 16-byte
                 // chunk c at chunk c ^ (row % 8): the 128-byte swizzle of the copy engine) and the copy engine stores
                 // the 32 x 32 block as whole 128-byte lines, clipped at the matrix edge; stores straight from registers
@@ -510,7 +553,7 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                 continue;
             }
             if (valid && col0 < p.N) {
-            if (p.split_k > 1) {
+            if (p.split_k > 1 && !reduce_here) {
                 float* dst = p.partial + ((static_cast<long long>(t.batch) * p.split_k + t.split) * p.M + grow) * p.N + col0;
                 if (p.vec_store) {
 #pragma unroll
@@ -602,6 +645,91 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
     if ((p.tma_store || p.partial_tma) && lane < 4) ptx::tma_store_wait_all<0>();
 }
 
+// Cluster reduction, first half: every epilogue warp sends its 32 rows of the column slices that other ranks own into
+// those ranks' receive slots (slot of this rank) with 16-byte stores through distributed shared memory.  (Staging the
+// slices in this CTA's shared memory and sending 4 KB pieces with the copy engine, counted on the receiver's barrier,
+// was built and measured too: 29.8 against 28.9 us on the 128 x 8192 x 8192 GEMM, so the stores stayed.)
+__device__ __forceinline__ void cluster_push_partials(const UmmaParams& p, uint8_t* recv_base, uint32_t tmem_base, int warp,
+                                                      int lane, int me) {
+    const int quarter = warp & 3;
+    const int slice = p.bn / p.split_k;
+    const uint32_t slot_bytes = static_cast<uint32_t>(kHalfM) * static_cast<uint32_t>(slice) * 4u;
+    for (int c0 = 0; c0 < p.bn; c0 += 32) {
+        const int owner = c0 / slice;
+        if (owner == me) continue;
+        uint32_t r[32];
+        ptx::tmem_ld_32x32b_x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(c0), r);
+        ptx::tmem_ld_wait();
+        const uint32_t in_slot = cluster_slot_offset(quarter, slice, c0 - owner * slice, lane);
+        const uint32_t there = ptx::smem_u32(recv_base) + static_cast<uint32_t>(me < owner ? me : me - 1) * slot_bytes + in_slot;
+        const uint32_t remote = ptx::mapa_u32(there, static_cast<uint32_t>(owner));
+#pragma unroll
+        for (int g = 0; g < 8; ++g)
+            ptx::st_cluster_v4(remote + g * 512, r[4 * g], r[4 * g + 1], r[4 * g + 2], r[4 * g + 3]);
+    }
+}
+
+// Cluster reduction, second half (bf16 result, rows of C 16-byte aligned): each epilogue warp sums its 32 rows of this
+// rank's column slice over the K slices in ascending order -- its own from tensor memory, the others' from the receive
+// slots -- and hands 32 x 32 bf16 blocks to the copy engine (64-byte swizzle, as in the staged epilogue; two blocks per
+// warp take turns).  Stores straight from registers reach the same lines 16 bytes at a time and cost about ten times more.
+__device__ __forceinline__ void cluster_reduce_store(const UmmaParams& p, const CUtensorMap* tmC, const uint8_t* recv,
+                                                     uint8_t* staging, uint32_t tmem_base, const TileCoord& t, int warp,
+                                                     int lane, int me) {
+    const int quarter = warp & 3;
+    const int slice = p.bn / p.split_k;
+    const uint32_t slot_bytes = static_cast<uint32_t>(kHalfM) * static_cast<uint32_t>(slice) * 4u;
+    const int row0 = t.m_blk * p.bm + quarter * 32;
+    uint8_t* blocks = staging + (warp - 2) * 4096;
+    const int sw = (lane >> 1) & 3;
+    int step = 0;
+    for (int c0 = 0; c0 < slice; c0 += 32, ++step) {
+        uint32_t r[32];
+        ptx::tmem_ld_32x32b_x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(me * slice + c0), r);
+        ptx::tmem_ld_wait();
+        float sum[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) sum[j] = 0.0f;
+        const uint32_t in_slot = cluster_slot_offset(quarter, slice, c0, lane);
+        for (int s = 0; s < p.split_k; ++s) {
+            if (s == me) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) sum[j] += __uint_as_float(r[j]);
+            } else {
+                const uint8_t* src = recv + static_cast<uint32_t>(s < me ? s : s - 1) * slot_bytes + in_slot;
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    const float4 v = *reinterpret_cast<const float4*>(src + g * 512);
+                    sum[4 * g] += v.x; sum[4 * g + 1] += v.y; sum[4 * g + 2] += v.z; sum[4 * g + 3] += v.w;
+                }
+            }
+        }
+        uint32_t pk[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+            __nv_bfloat162 h2 = __floats2bfloat162_rn(p.alpha * sum[2 * e], p.alpha * sum[2 * e + 1]);
+            pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+        }
+        uint8_t* blk = blocks + (step & 1) * 2048;
+        if (lane == 0) ptx::tma_store_wait_read<1>();      // the store issued two steps ago has read this block
+        __syncwarp();
+        uint8_t* my_row = blk + lane * 64;
+#pragma unroll
+        for (int g = 0; g < 4; ++g)
+            *reinterpret_cast<uint4*>(my_row + ((g ^ sw) << 4)) = make_uint4(pk[4 * g], pk[4 * g + 1], pk[4 * g + 2], pk[4 * g + 3]);
+        ptx::fence_proxy_async_smem();
+        __syncwarp();
+        const int col0 = t.n0 + me * slice + c0;
+        if (lane == 0 && row0 < p.M && col0 < p.N) {
+            ptx::tma_store_2d(tmC, blk, col0, row0);
+            ptx::tma_store_commit();
+        }
+        __syncwarp();
+    }
+    // shared memory must stay alive until the copy engine has drained this warp's last store
+    if (lane == 0) ptx::tma_store_wait_all<0>();
+}
+
 template <bool kConv>
 __global__ void __launch_bounds__(576, 1)
 umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -636,7 +764,7 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
         ptx::fence_barrier_init();
         ptx::tma_prefetch_desc(&tmA);
         ptx::tma_prefetch_desc(&tmB);
-        if (p.tma_store) ptx::tma_prefetch_desc(&tmC);
+        if (p.tma_store || p.cluster_tma) ptx::tma_prefetch_desc(&tmC);
     }
     if (warp == 1) {
         __syncwarp();
@@ -768,9 +896,32 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
                 }
             }
         }
+    } else if (!kConv && p.cluster_reduce) {
+        // the partial tile of this CTA's K slice is complete once the accumulator barrier flips
+        if (have_first) wait_bounded(&tfull_bar[0], 0u, abort_flag, p.status, kTimeoutEpilogue);
+        ptx::tc_fence_after_sync();
     } else {
         epilogue_role<kConv>(p, &tmC, smem + static_cast<size_t>(p.stages) * stage_bytes, tmem_base, tfull_bar,
                              tempty_bar, abort_flag, mh, warp, lane, total_items, -1, 0, 1, 0, 0, nullptr, &t_first, have_first);
+    }
+    if (!kConv && p.cluster_reduce) {
+        // Every thread of every CTA of the cluster takes part in both barriers, whatever happened in its role.
+        // (1) all partial tiles are complete, so every CTA's pipeline stages are free: they become the receive slots;
+        // (2) all slices have arrived where they are summed.  After (2) a CTA touches only its own shared memory.
+        const int me = static_cast<int>(ptx::cluster_ctarank());
+        const bool good = have_first && !*abort_flag;
+        ptx::cluster_sync_all();
+        if (warp >= 2 && good) cluster_push_partials(p, smem, tmem_base, warp, lane, me);
+        ptx::cluster_sync_all();
+        if (warp >= 2 && good && p.cluster_tma) {
+            cluster_reduce_store(p, &tmC, smem, smem + static_cast<size_t>(p.stages) * stage_bytes, tmem_base, t_first, warp, lane, me);
+        } else if (warp >= 2 && good) {
+            TileCoord slice = t_first;
+            slice.bn = p.bn / p.split_k;
+            slice.n0 = t_first.n0 + me * slice.bn;
+            epilogue_role<kConv>(p, &tmC, smem + static_cast<size_t>(p.stages) * stage_bytes, tmem_base, tfull_bar, tempty_bar,
+                                 abort_flag, mh, warp, lane, total_items, -1, 0, 1, 0, 0, nullptr, &slice, true, smem, me);
+        }
     }
 
     ptx::tc_fence_before_sync();

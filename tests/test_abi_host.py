@@ -144,20 +144,27 @@ def test_gemm_search_space_obeys_constraints(shape):
         assert c["kernel"] == tdx.TDX_KERNEL_UMMA and c["tile_m"] in (128, 256) and c["tile_k"] == 64
         assert c["tile_n"] % 64 == 0                          # B is read N-major here
         assert 2 <= c["stages"] <= 8
-        assert c["store_mode"] in (1, 2)
-        staging = 16 * 2048 if c["store_mode"] == 2 else 0
+        assert c["store_mode"] in (1, 2, 3)
+        staging = {1: 0, 2: 16 * 2048, 3: 8 * 2048}[c["store_mode"]]
         rows_per_cta = 128 + c["tile_n"] // 2 if c["cta_pair"] == 2 else c["tile_m"] + c["tile_n"]
         assert c["stages"] * rows_per_cta * 128 + 1024 + 512 + staging <= SMEM_LIMIT
         if c["cta_pair"] == 2:
             assert c["tile_m"] == 256 and c["split_k"] == 1 and c["tile_n"] % 128 == 0
         if c["store_mode"] == 2:
             assert c["split_k"] == 1
+        if c["store_mode"] == 3:
+            # split-K summed inside a cluster: cluster size = split_k, slices of whole 32-column steps, and the receive
+            # slots for the other ranks' slices fit the pipeline stages
+            assert 2 <= c["split_k"] <= 8 and c["tile_m"] == 128 and c["cta_pair"] == 1 and c["fit"] == 1
+            assert c["tile_n"] % (32 * c["split_k"]) == 0
+            assert (c["split_k"] - 1) * 128 * (c["tile_n"] // c["split_k"]) * 4 <= c["stages"] * rows_per_cta * 128
         halves = 1 if c["cta_pair"] == 2 else c["tile_m"] // 128
         assert halves * c["tile_n"] <= 512                     # one tile's accumulators fit in a CTA's TMEM
         per = -(-num_kb // c["split_k"])
         assert (c["split_k"] - 1) * per < num_kb               # no empty K slice
     if M * N <= 128 * 8192:
         assert any(c["split_k"] > 1 for c in cfgs)             # skinny shapes get split-K candidates
+        assert any(c["store_mode"] == 3 for c in cfgs)         # ... with the sum in a workspace and inside clusters
     if shape == (8192, 8192, 8192):
         assert all(c["split_k"] == 1 for c in cfgs)
 
@@ -300,6 +307,26 @@ def test_k_balanced_plan_covers_every_unit_once_and_evenly(shape, ctas):
     assert sum(loads) == units
     share = units / used
     assert max(loads) <= share + 5 and min(loads) >= share - 5                # even up to the snapping length
+
+
+def test_cluster_reduction_config_constraints_and_workspace_size():
+    # store_mode 3 (split-K summed inside a cluster of split_k CTAs): no workspace; constraints checked before any launch
+    M, N, K = 128, 8192, 8192
+    ok = tdx.tdx_config(kernel=tdx.TDX_KERNEL_UMMA, tile_m=128, tile_n=192, split_k=3, store_mode=3)
+    st, need = tdx.tdx_gemm_workspace_size(M, N, K, tdx.TDX_BF16, ok)
+    assert st == 0 and need == 0
+    base = dict(M=M, N=N, K=K, transA=0, transB=0, alpha=1.0, dtype=tdx.TDX_BF16, A=256, B=512, C=1024)
+    for kw in [dict(tile_m=128, tile_n=192, split_k=1),              # nothing to sum
+               dict(tile_m=128, tile_n=192, split_k=4),              # 192 columns do not cut into four slices of 32-column steps
+               dict(tile_m=128, tile_n=128, split_k=16),             # larger than a cluster
+               dict(tile_m=256, tile_n=128, split_k=2),              # 128-row tiles only
+               dict(tile_m=128, tile_n=256, split_k=2, fit=2),       # uniform grid only
+               dict(tile_m=256, tile_n=256, split_k=2, cta_pair=2)]:
+        cfg = tdx.tdx_config(kernel=tdx.TDX_KERNEL_UMMA, store_mode=3, **kw)
+        assert tdx.tdx_gemm_ex(**base, cfg=cfg) == tdx.TDX_ERR_CONFIG, kw
+    # the convolution has no split-K, hence no cluster reduction
+    cfg = tdx.tdx_config(kernel=tdx.TDX_KERNEL_UMMA, store_mode=3, split_k=2, tile_m=128, tile_n=64)
+    assert tdx.tdx_conv2d_bias_relu_ex(1, 16, 16, 64, 64, 3, 3, 1, 1, tdx.TDX_BF16, 256, 512, 1024, 1, 2048, None, cfg) == tdx.TDX_ERR_CONFIG
 
 
 def test_k_balanced_config_constraints_and_workspace_size():
