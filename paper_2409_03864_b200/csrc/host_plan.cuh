@@ -282,10 +282,13 @@ double model_gemm_us(const GemmProblem& g, const tdx_config& c, int sm_count) {
     const int64_t kb = ceil_div(num_kb, split);
     const int64_t tiles = ceil_div(g.M, tm) * ceil_div(g.N, bn) * split;
     const int halves = pair ? 1 : tm / 128;                                 // 128-row halves one CTA computes
-    const double mma = 4.0 * halves * std::max(bn / 2.0, 60.0);
-    // operand slices of tiles narrower than 128 columns arrive at about 46 bytes per cycle (measured: 128 x 64 tiles,
-    // 533 cycles per 24 KB K block), wider ones at about 70
-    const double l2 = (pair ? (128.0 + bn / 2.0) : (tm + static_cast<double>(bn))) * 128.0 / (bn < 128 ? 46.0 : 70.0);
+    // a pair's MMA over 256 rows takes 115 cycles or more however narrow it is (measured at 128 columns)
+    const double mma = 4.0 * halves * std::max(bn / 2.0, pair ? 115.0 : 60.0);
+    // the smaller a K block's copies, the slower the SM takes its operand slices in from L2: about 46 bytes per cycle for
+    // 24 KB blocks (128 x 64 tiles: 533 cycles per block), 50 for 32 KB (128 x 128: 655), about 70 from 48 KB on; a pair's
+    // CTAs keep up with their MMAs at 32 KB per block (511 cycles measured at 256 columns)
+    const double kb_rows = pair ? (128.0 + bn / 2.0) : (tm + static_cast<double>(bn));
+    const double l2 = kb_rows * 128.0 / (pair ? 70.0 : kb_rows < 256.0 ? 46.0 : kb_rows < 384.0 ? 50.0 : 70.0);
     const double main_loop = static_cast<double>(kb) * std::max(mma, l2);
     const double blocks = halves * 4.0 * (bn / 32.0);                       // 32 x 32 output blocks per CTA and tile
     double epi = (c.store_mode == 2 ? 600.0 * std::ceil(blocks / 16.0) : 1200.0 * std::ceil(blocks / (4.0 * halves)));

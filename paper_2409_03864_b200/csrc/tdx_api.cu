@@ -56,9 +56,10 @@ int enum_gemm(const GemmProblem& g, int sm_count, int smem_limit, std::vector<td
 // The automatic choice for a bf16 shape the tuning cache does not know: the candidate of the search space that the
 // cost model ranks first.  On eleven shapes outside the tuned set that candidate measured within 12 % of the exhaustive
 // search's winner on ten (29 % on 2048 x 512 x 8192) and well ahead of the size heuristic it replaces (2048^3: 19.4
-// vs 27.5 us, search 17.7; 4096 x 1024 x 4096: 32.3 vs 49.4 us, search 28.9).  CTA pairs are left out (the model does
-// not see their fixed costs).  Ranking a few hundred candidates costs milliseconds, so the answer is kept per shape,
-// and the last one per thread.
+// vs 27.5 us, search 17.7; 4096 x 1024 x 4096: 32.3 vs 49.4 us, search 28.9).  CTA pairs and the split-K summed inside
+// clusters compete too, now that the model carries their measured costs (2048^3: 17.0 us; 4096 x 1024 x 4096: 26.9;
+// 512 x 4096 x 4096: 28.4 -> 22.6).  Ranking a few hundred candidates costs milliseconds, so the answer is kept per
+// shape, and the last one per thread.
 bool model_default_gemm(const GemmProblem& g, int sm_count, int smem_limit, tdx_config* out) {
     typedef std::array<int64_t, 7> Key;
     const Key key = {g.M, g.N, g.K, g.transA, g.transB, sm_count, smem_limit};
@@ -77,7 +78,7 @@ bool model_default_gemm(const GemmProblem& g, int sm_count, int smem_limit, tdx_
             pick.first = false;
             std::memset(&pick.second, 0, sizeof pick.second);
             for (const tdx_config& c : cands) {
-                if (c.cta_pair == 2 || c.fit == 3) continue;      // chosen by measurement only (tuning cache, search)
+                if (c.fit == 3) continue;      // chosen by measurement only (tuning cache, search)
                 const double us = model_gemm_us(g, c, sm_count);
                 if (!pick.first || us < best_us) { pick.first = true; pick.second = c; best_us = us; }
             }
@@ -874,7 +875,8 @@ int tdx_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int transA,
         tdx_config cfg;
         rc = resolve_gemm_config(g, beta != 0.0f ? &want : nullptr, ctx->sm_count, ctx->smem_optin, &cfg);
         if (rc) return rc;
-        if (cfg.kernel != TDX_KERNEL_UMMA || cfg.cta_pair == 2) return run_gemm_generic(ctx, g, alpha, A, B, C, st, ba);
+        if (cfg.kernel != TDX_KERNEL_UMMA) return run_gemm_generic(ctx, g, alpha, A, B, C, st, ba);
+        if (cfg.cta_pair == 2) return run_gemm_pair(ctx, g, alpha, A, B, C, cfg, st);      // automatic choice, beta = 0 only
         return run_gemm_umma(ctx, g, alpha, A, B, C, cfg, nullptr, 0, true, st, beta);
     }
     rc = run_gemm_batched_bf16(ctx, g, alpha, beta, A, strideA, B, strideB, C, strideC, batch, direct, st);

@@ -187,3 +187,25 @@ def test_batched_fp32_on_the_tensor_cores_in_one_launch(shape, tA, tB):
     assert tdx.tdx_kernel_launch_count() - n0 <= 3
     err = error(batch, M, N, K, tA, tB, 0.5, -1.0, "f32", A, B, C, got)
     assert err < TIGHT["f32"], err
+
+
+def test_one_batch_without_accumulate_takes_the_automatic_configuration():
+    # batch = 1, beta = 0 is the plain GEMM: whatever configuration the library picks for tdx_gemm (for this shape,
+    # which the shipped tuning cache does not list, the cost model's: a CTA pair) runs, in one launch, same bits
+    batch, M, N, K = 1, 2048, 2048, 2048
+    st, cfg = tdx.tdx_default_gemm_config(M, N, K, 0, 1, tdx.TDX_BF16)
+    assert st == 0 and cfg.kernel == tdx.TDX_KERNEL_UMMA
+    A, B, C = operands(batch, M, N, K, "bf16", seed=97, transB=1)
+    n0 = tdx.tdx_kernel_launch_count()
+    st, got = run(batch, M, N, K, 0, 1, 1.0, 0.0, "bf16", A, B, C)
+    assert st == 0, tdx.tdx_last_error()
+    assert tdx.tdx_kernel_launch_count() - n0 == 1
+    dA, dB = to_dev(A), to_dev(B)
+    dC = torch.zeros(M * N, dtype=torch.int16, device="cuda")
+    assert tdx.tdx_gemm(M, N, K, 0, 1, 1.0, tdx.TDX_BF16, dA, dB, dC) == 0
+    torch.cuda.synchronize()
+    assert np.array_equal(got.reshape(-1), dC.cpu().numpy().view(np.uint16))
+    rows = [0, 1, 127, 128, 1000, 2047]
+    ref = oracle.gemm(M, N, K, 0, 1, 1.0, "bf16", A[0], B[0], rows=rows)
+    sc = oracle.gemm_row_scales(M, N, K, 0, 1, 1.0, "bf16", A[0], B[0], rows=rows)
+    assert oracle.max_normalised_error(oracle.decode(got, "bf16")[rows], ref, sc) < TIGHT["bf16"]
