@@ -89,7 +89,7 @@ typedef struct {
     int store_mode; /* 1 = 16-byte stores from registers; 2 = 32 x 32 blocks staged in shared     */
                     /*     memory and written by TMA store (needs N % 8 == 0, split_k = 1,         */
                     /*     16-byte aligned C; falls back to 1 if C is misaligned)                  */
-                    /*     3 = (GEMM, tile_m = 128, split_k in 2..8, tile_n a multiple of 32 * split_k) the   */
+                    /*     3 = (GEMM, cta_pair = 1, split_k in 2..8, tile_n a multiple of 32 * split_k) the   */
                     /*     split_k CTAs of a tile form a thread-block cluster, exchange column slices of     */
                     /*     their fp32 partial tiles through distributed shared memory and each writes its    */
                     /*     slice of the result, summed over the K slices in ascending order: no workspace,   */

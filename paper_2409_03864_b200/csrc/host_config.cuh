@@ -40,8 +40,9 @@ bool conv_umma_layout_ok(const ConvProblem& c) {
 }
 
 // Shared memory the staged (TMA-store) epilogue needs: one 32 x 32 bf16 block for each of its 16 warps.
-// The cluster reduction (store_mode 3) stages its summed slice the same way: two blocks for each of its four warps.
-int staging_bytes_for(int /*tile_m*/, int store_mode) { return store_mode == 2 ? 16 * 2048 : store_mode == 3 ? 8 * 2048 : 0; }
+// The cluster reduction (store_mode 3) stages its summed slice the same way: two blocks for each of its four warps per
+// 128-row half.
+int staging_bytes_for(int tile_m, int store_mode) { return store_mode == 2 ? 16 * 2048 : store_mode == 3 ? (tile_m / 128) * 8 * 2048 : 0; }
 
 // Shared memory for fp32 partial tiles that leave through the copy engine (split-K, K-balanced plan): two 32 x 32 fp32
 // blocks for each of the four epilogue warps per 128-row half.  Optional: a configuration whose stages leave no room for
@@ -118,12 +119,11 @@ const char* umma_config_reason(const tdx_config& c, bool b_mn_major, int64_t num
         return "store_mode must be 1 (direct), 2 (TMA store) or 3 (split-K summed inside a thread-block cluster)";
     if (c.store_mode == 3) {
         if (conv || c.cta_pair == 2) return "the cluster reduction is implemented for the single-CTA GEMM only";
-        if (c.tile_m != 128) return "the cluster reduction works on 128-row tiles";
         if (c.split_k < 2 || c.split_k > 8) return "the cluster reduction needs split_k in [2, 8] (the cluster size)";
         if (c.tile_n % (32 * c.split_k)) return "the cluster reduction cuts the tile into split_k column slices of a multiple of 32 columns";
         if (c.fit > 1) return "the cluster reduction runs the uniform grid: fit must be 0 or 1";
         // the other ranks' slices are received in the pipeline stages, free by then
-        if (static_cast<int64_t>(c.stages) * (128 + c.tile_n) * 128 < static_cast<int64_t>(c.split_k - 1) * 128 * (c.tile_n / c.split_k) * 4)
+        if (static_cast<int64_t>(c.stages) * (c.tile_m + c.tile_n) * 128 < static_cast<int64_t>(c.split_k - 1) * c.tile_m * (c.tile_n / c.split_k) * 4)
             return "the pipeline stages are too small to receive the other ranks' slices";
     }
     if (c.store_mode == 2) {

@@ -309,7 +309,7 @@ double model_gemm_us(const GemmProblem& g, const tdx_config& c, int sm_count) {
     // slice (measured: 6.7 k cycles for 32 KB sent, 9.9 k for 64 KB)
     const bool in_cluster = c.store_mode == 3 && split > 1 && !pair;
     if (in_cluster) {
-        const double sent = 128.0 * bn * 4.0 * (split - 1) / split;
+        const double sent = static_cast<double>(tm) * bn * 4.0 * (split - 1) / split;
         cycles = 5500.0 + rounds * (main_loop + 3400.0 + 0.1 * sent);
     }
     int kbal_slots = 0;

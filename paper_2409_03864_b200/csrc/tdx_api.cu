@@ -108,7 +108,7 @@ bool model_pick_direct_store(const GemmProblem& g, int sm_count, int smem_limit,
         double best_us = 0.0;
         for (tdx_config c : cands) {
             if (c.cta_pair == 2 || c.k_stagger != 0 || c.fit == 3) continue;
-            c.store_mode = 1;
+            if (c.store_mode != 3) c.store_mode = 1;      // (a K split summed inside clusters stores through the copy engine)
             c.fit = 1;
             const double us = model_gemm_us(g, c, sm_count);
             if (!pick.first || us < best_us) { pick.first = true; pick.second = c; best_us = us; }
@@ -815,10 +815,12 @@ int tdx_gemm_f32out(int64_t M, int64_t N, int64_t K, int transA, int transB, flo
         want.tile_n = ranked.tile_n;
         want.split_k = ranked.split_k;
         want.raster = ranked.raster;
+        if (ranked.store_mode == 3) want.store_mode = 3;
     }
     tdx_config cfg;
     rc = resolve_gemm_config(g, &want, ctx->sm_count, ctx->smem_optin, &cfg);
     if (rc) return rc;
+    prefer_cluster_reduce(g, ctx->smem_optin, &cfg);
     return run_gemm_umma(ctx, g, alpha, A, B, C, cfg, nullptr, 0, true, st, 0.0f, nullptr, true);
 }
 
@@ -870,6 +872,7 @@ int tdx_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int transA,
                 want.tile_n = ranked.tile_n;
                 want.split_k = ranked.split_k;
                 want.raster = ranked.raster;
+                if (ranked.store_mode == 3) want.store_mode = 3;
             }
         }
         tdx_config cfg;
@@ -877,6 +880,7 @@ int tdx_gemm_batched(int64_t batch, int64_t M, int64_t N, int64_t K, int transA,
         if (rc) return rc;
         if (cfg.kernel != TDX_KERNEL_UMMA) return run_gemm_generic(ctx, g, alpha, A, B, C, st, ba);
         if (cfg.cta_pair == 2) return run_gemm_pair(ctx, g, alpha, A, B, C, cfg, st);      // automatic choice, beta = 0 only
+        if (beta != 0.0f) prefer_cluster_reduce(g, ctx->smem_optin, &cfg);
         return run_gemm_umma(ctx, g, alpha, A, B, C, cfg, nullptr, 0, true, st, beta);
     }
     rc = run_gemm_batched_bf16(ctx, g, alpha, beta, A, strideA, B, strideB, C, strideC, batch, direct, st);

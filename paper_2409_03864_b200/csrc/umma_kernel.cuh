@@ -61,13 +61,13 @@ struct UmmaParams {
     int tma_store;            // final output leaves through shared memory + TMA store (needs bn % 64 == 0)
     int partial_tma;          // split-K: fp32 partial tiles leave through shared memory + TMA store (tmC then maps the
                               // workspace as (N, M, batch * split) floats; two 32 x 32 fp32 blocks per epilogue warp)
-    int cluster_reduce;       // split-K summed inside a thread-block cluster of split_k CTAs (GEMM, 128-row tiles, one
+    int cluster_reduce;       // split-K summed inside a thread-block cluster of split_k CTAs (GEMM, one
                               // tile per CTA): CTA rank s of a cluster reduces K slice s of the cluster's tile, then
                               // the ranks exchange column slices of their partial tiles through distributed shared
                               // memory and rank q writes columns [q, q + 1) * bn / split_k of the result -- no
                               // workspace and no reduction kernel.  The sum runs over the slices in ascending order.
-    int cluster_tma;          // cluster reduction: the summed slice leaves as 32 x 32 bf16 blocks through shared memory and
-                              // the copy engine (tmC maps C as for the staged epilogue); else 16-byte stores from registers
+    int cluster_tma;          // cluster reduction: the summed slice leaves as 32 x 32 blocks through shared memory and the
+                              // copy engine (1: bf16, 2: fp32; tmC maps C as (N, M) or (N, M, batch)); 0: stores from registers
     int sbx, sby;             // conv TMA-store box: sbx x sby output pixels (sbx * sby = 32)
     // convolution geometry (kConv only)
     int bw, bh, nb;           // spatial patch (bw x bh output pixels), patches per tile = bm / (bw*bh)
@@ -276,9 +276,9 @@ __device__ __forceinline__ void issue_kblock(const UmmaParams& p, const CUtensor
     }
 }
 
-// Slot layout of the cluster reduction: a slot holds one rank's 128 x slice partial sums for the rank that owns the
-// slice, as [lane quarter][4-column group][row within the quarter][16 bytes]: the 32 rows of a warp lie side by side
-// (no bank conflicts on either end) and a warp's 32-column step is one contiguous 4 KB piece.
+// Slot layout of the cluster reduction: a slot holds one rank's bm x slice partial sums for the rank that owns the
+// slice, as [32-row group][4-column group][row within the group][16 bytes] (`quarter` = 4 * half + lane quarter): the
+// 32 rows of a warp lie side by side (no bank conflicts on either end) and a warp's 32-column step is one contiguous 4 KB.
 __device__ __forceinline__ uint32_t cluster_slot_offset(int quarter, int slice, int c_in_slice, int lane) {
     return (static_cast<uint32_t>(quarter * (slice >> 2) + (c_in_slice >> 2)) * 32u + static_cast<uint32_t>(lane)) * 16u;
 }
@@ -510,8 +510,8 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
                 float sum[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) sum[j] = 0.0f;
-                const uint32_t slot_bytes = static_cast<uint32_t>(kHalfM) * static_cast<uint32_t>(t.bn) * 4u;
-                const uint32_t in_slot = cluster_slot_offset(quarter, t.bn, c0, lane);
+                const uint32_t slot_bytes = static_cast<uint32_t>(p.bm) * static_cast<uint32_t>(t.bn) * 4u;
+                const uint32_t in_slot = cluster_slot_offset(half * 4 + quarter, t.bn, c0, lane);
                 for (int s = 0; s < p.split_k; ++s) {
                     if (s == my_rank) {
 #pragma unroll
@@ -652,15 +652,16 @@ __device__ __forceinline__ void epilogue_role(const UmmaParams& p, const CUtenso
 __device__ __forceinline__ void cluster_push_partials(const UmmaParams& p, uint8_t* recv_base, uint32_t tmem_base, int warp,
                                                       int lane, int me) {
     const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;                  // 256-row tiles: warps 6..9 drain the second accumulator slot
     const int slice = p.bn / p.split_k;
-    const uint32_t slot_bytes = static_cast<uint32_t>(kHalfM) * static_cast<uint32_t>(slice) * 4u;
+    const uint32_t slot_bytes = static_cast<uint32_t>(p.bm) * static_cast<uint32_t>(slice) * 4u;
     for (int c0 = 0; c0 < p.bn; c0 += 32) {
         const int owner = c0 / slice;
         if (owner == me) continue;
         uint32_t r[32];
-        ptx::tmem_ld_32x32b_x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(c0), r);
+        ptx::tmem_ld_32x32b_x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(half * p.bn + c0), r);
         ptx::tmem_ld_wait();
-        const uint32_t in_slot = cluster_slot_offset(quarter, slice, c0 - owner * slice, lane);
+        const uint32_t in_slot = cluster_slot_offset(half * 4 + quarter, slice, c0 - owner * slice, lane);
         const uint32_t there = ptx::smem_u32(recv_base) + static_cast<uint32_t>(me < owner ? me : me - 1) * slot_bytes + in_slot;
         const uint32_t remote = ptx::mapa_u32(there, static_cast<uint32_t>(owner));
 #pragma unroll
@@ -669,28 +670,33 @@ __device__ __forceinline__ void cluster_push_partials(const UmmaParams& p, uint8
     }
 }
 
-// Cluster reduction, second half (bf16 result, rows of C 16-byte aligned): each epilogue warp sums its 32 rows of this
-// rank's column slice over the K slices in ascending order -- its own from tensor memory, the others' from the receive
-// slots -- and hands 32 x 32 bf16 blocks to the copy engine (64-byte swizzle, as in the staged epilogue; two blocks per
-// warp take turns).  Stores straight from registers reach the same lines 16 bytes at a time and cost about ten times more.
+// Cluster reduction, second half: each epilogue warp sums its 32 rows of this rank's column slice over the K slices in
+// ascending order -- its own from tensor memory, the others' from the receive slots --, applies alpha and the accumulate
+// term (beta times what C held, read straight from global memory: a thread's 32 columns are one or two whole lines) and
+// hands 32 x 32 blocks to the copy engine: bf16 with the 64-byte swizzle of the staged epilogue, two 2 KB blocks per warp
+// taking turns (p.cluster_tma == 1), or fp32 with the 128-byte swizzle, one 4 KB block per warp (== 2).  tmC maps C as
+// (N, M) or, batched, (N, M, batch).  Stores straight from registers reach the same lines 16 bytes at a time and cost
+// about ten times more.
 __device__ __forceinline__ void cluster_reduce_store(const UmmaParams& p, const CUtensorMap* tmC, const uint8_t* recv,
                                                      uint8_t* staging, uint32_t tmem_base, const TileCoord& t, int warp,
                                                      int lane, int me) {
     const int quarter = warp & 3;
+    const int half = (warp - 2) >> 2;
     const int slice = p.bn / p.split_k;
-    const uint32_t slot_bytes = static_cast<uint32_t>(kHalfM) * static_cast<uint32_t>(slice) * 4u;
-    const int row0 = t.m_blk * p.bm + quarter * 32;
+    const uint32_t slot_bytes = static_cast<uint32_t>(p.bm) * static_cast<uint32_t>(slice) * 4u;
+    const int row0 = t.m_blk * p.bm + half * kHalfM + quarter * 32;
+    const long long grow = static_cast<long long>(row0) + lane;
+    const bool f32 = p.cluster_tma == 2;
     uint8_t* blocks = staging + (warp - 2) * 4096;
-    const int sw = (lane >> 1) & 3;
     int step = 0;
     for (int c0 = 0; c0 < slice; c0 += 32, ++step) {
         uint32_t r[32];
-        ptx::tmem_ld_32x32b_x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(me * slice + c0), r);
+        ptx::tmem_ld_32x32b_x32(tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + static_cast<uint32_t>(half * p.bn + me * slice + c0), r);
         ptx::tmem_ld_wait();
         float sum[32];
 #pragma unroll
         for (int j = 0; j < 32; ++j) sum[j] = 0.0f;
-        const uint32_t in_slot = cluster_slot_offset(quarter, slice, c0, lane);
+        const uint32_t in_slot = cluster_slot_offset(half * 4 + quarter, slice, c0, lane);
         for (int s = 0; s < p.split_k; ++s) {
             if (s == me) {
 #pragma unroll
@@ -704,24 +710,64 @@ __device__ __forceinline__ void cluster_reduce_store(const UmmaParams& p, const 
                 }
             }
         }
-        uint32_t pk[16];
+        const int col0 = t.n0 + me * slice + c0;
 #pragma unroll
-        for (int e = 0; e < 16; ++e) {
-            __nv_bfloat162 h2 = __floats2bfloat162_rn(p.alpha * sum[2 * e], p.alpha * sum[2 * e + 1]);
-            pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+        for (int j = 0; j < 32; ++j) sum[j] *= p.alpha;
+        if (p.beta != 0.0f && grow < p.M) {
+            // (rows are 16-byte aligned and N is a multiple of 8 (bf16) or 4 (fp32) here, so groups are all in or all out)
+            if (f32) {
+                const float* old = p.Cf + t.batch * p.batch_c + grow * p.ldc + col0;
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    if (col0 + g * 4 < p.N) {
+                        const float4 o = *reinterpret_cast<const float4*>(old + g * 4);
+                        sum[4 * g] = fmaf(p.beta, o.x, sum[4 * g]); sum[4 * g + 1] = fmaf(p.beta, o.y, sum[4 * g + 1]);
+                        sum[4 * g + 2] = fmaf(p.beta, o.z, sum[4 * g + 2]); sum[4 * g + 3] = fmaf(p.beta, o.w, sum[4 * g + 3]);
+                    }
+                }
+            } else {
+                const __nv_bfloat16* old = p.C + t.batch * p.batch_c + grow * p.ldc + col0;
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                    if (col0 + g * 8 < p.N) {
+                        const uint4 o = *reinterpret_cast<const uint4*>(old + g * 8);
+                        const uint32_t ow[4] = {o.x, o.y, o.z, o.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            sum[8 * g + 2 * e] = fmaf(p.beta, __uint_as_float(ow[e] << 16), sum[8 * g + 2 * e]);
+                            sum[8 * g + 2 * e + 1] = fmaf(p.beta, __uint_as_float(ow[e] & 0xFFFF0000u), sum[8 * g + 2 * e + 1]);
+                        }
+                    }
+                }
+            }
         }
-        uint8_t* blk = blocks + (step & 1) * 2048;
-        if (lane == 0) ptx::tma_store_wait_read<1>();      // the store issued two steps ago has read this block
+        uint8_t* blk = f32 ? blocks : blocks + (step & 1) * 2048;
+        // the store that last read this block (the previous one; for bf16 the one before it) must be done with it
+        if (lane == 0) { if (f32) ptx::tma_store_wait_read<0>(); else ptx::tma_store_wait_read<1>(); }
         __syncwarp();
-        uint8_t* my_row = blk + lane * 64;
+        if (f32) {
+            uint8_t* my_row = blk + lane * 128;
 #pragma unroll
-        for (int g = 0; g < 4; ++g)
-            *reinterpret_cast<uint4*>(my_row + ((g ^ sw) << 4)) = make_uint4(pk[4 * g], pk[4 * g + 1], pk[4 * g + 2], pk[4 * g + 3]);
+            for (int g = 0; g < 8; ++g)
+                *reinterpret_cast<float4*>(my_row + ((g ^ (lane & 7)) << 4)) = make_float4(sum[4 * g], sum[4 * g + 1], sum[4 * g + 2], sum[4 * g + 3]);
+        } else {
+            uint32_t pk[16];
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+                __nv_bfloat162 h2 = __floats2bfloat162_rn(sum[2 * e], sum[2 * e + 1]);
+                pk[e] = *reinterpret_cast<uint32_t*>(&h2);
+            }
+            uint8_t* my_row = blk + lane * 64;
+            const int sw = (lane >> 1) & 3;
+#pragma unroll
+            for (int g = 0; g < 4; ++g)
+                *reinterpret_cast<uint4*>(my_row + ((g ^ sw) << 4)) = make_uint4(pk[4 * g], pk[4 * g + 1], pk[4 * g + 2], pk[4 * g + 3]);
+        }
         ptx::fence_proxy_async_smem();
         __syncwarp();
-        const int col0 = t.n0 + me * slice + c0;
         if (lane == 0 && row0 < p.M && col0 < p.N) {
-            ptx::tma_store_2d(tmC, blk, col0, row0);
+            if (p.batch > 1) ptx::tma_store_3d(tmC, blk, col0, row0, t.batch);
+            else ptx::tma_store_2d(tmC, blk, col0, row0);
             ptx::tma_store_commit();
         }
         __syncwarp();
@@ -897,8 +943,8 @@ umma_contract_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_const
             }
         }
     } else if (!kConv && p.cluster_reduce) {
-        // the partial tile of this CTA's K slice is complete once the accumulator barrier flips
-        if (have_first) wait_bounded(&tfull_bar[0], 0u, abort_flag, p.status, kTimeoutEpilogue);
+        // the partial tile of this CTA's K slice is complete once the accumulator barrier (of this warp's 128-row half) flips
+        if (have_first) wait_bounded(&tfull_bar[((warp - 2) >> 2) % mh], 0u, abort_flag, p.status, kTimeoutEpilogue);
         ptx::tc_fence_after_sync();
     } else {
         epilogue_role<kConv>(p, &tmC, smem + static_cast<size_t>(p.stages) * stage_bytes, tmem_base, tfull_bar,

@@ -145,7 +145,7 @@ def test_gemm_search_space_obeys_constraints(shape):
         assert c["tile_n"] % 64 == 0                          # B is read N-major here
         assert 2 <= c["stages"] <= 8
         assert c["store_mode"] in (1, 2, 3)
-        staging = {1: 0, 2: 16 * 2048, 3: 8 * 2048}[c["store_mode"]]
+        staging = {1: 0, 2: 16 * 2048, 3: (c["tile_m"] // 128) * 8 * 2048}[c["store_mode"]]
         rows_per_cta = 128 + c["tile_n"] // 2 if c["cta_pair"] == 2 else c["tile_m"] + c["tile_n"]
         assert c["stages"] * rows_per_cta * 128 + 1024 + 512 + staging <= SMEM_LIMIT
         if c["cta_pair"] == 2:
@@ -155,9 +155,9 @@ def test_gemm_search_space_obeys_constraints(shape):
         if c["store_mode"] == 3:
             # split-K summed inside a cluster: cluster size = split_k, slices of whole 32-column steps, and the receive
             # slots for the other ranks' slices fit the pipeline stages
-            assert 2 <= c["split_k"] <= 8 and c["tile_m"] == 128 and c["cta_pair"] == 1 and c["fit"] == 1
+            assert 2 <= c["split_k"] <= 8 and c["cta_pair"] == 1 and c["fit"] == 1
             assert c["tile_n"] % (32 * c["split_k"]) == 0
-            assert (c["split_k"] - 1) * 128 * (c["tile_n"] // c["split_k"]) * 4 <= c["stages"] * rows_per_cta * 128
+            assert (c["split_k"] - 1) * c["tile_m"] * (c["tile_n"] // c["split_k"]) * 4 <= c["stages"] * rows_per_cta * 128
         halves = 1 if c["cta_pair"] == 2 else c["tile_m"] // 128
         assert halves * c["tile_n"] <= 512                     # one tile's accumulators fit in a CTA's TMEM
         per = -(-num_kb // c["split_k"])
@@ -319,7 +319,6 @@ def test_cluster_reduction_config_constraints_and_workspace_size():
     for kw in [dict(tile_m=128, tile_n=192, split_k=1),              # nothing to sum
                dict(tile_m=128, tile_n=192, split_k=4),              # 192 columns do not cut into four slices of 32-column steps
                dict(tile_m=128, tile_n=128, split_k=16),             # larger than a cluster
-               dict(tile_m=256, tile_n=128, split_k=2),              # 128-row tiles only
                dict(tile_m=128, tile_n=256, split_k=2, fit=2),       # uniform grid only
                dict(tile_m=256, tile_n=256, split_k=2, cta_pair=2)]:
         cfg = tdx.tdx_config(kernel=tdx.TDX_KERNEL_UMMA, store_mode=3, **kw)

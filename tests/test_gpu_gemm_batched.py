@@ -40,13 +40,16 @@ def error(batch, M, N, K, tA, tB, alpha, beta, dtype, A, B, C, got):
 def test_the_papers_batch_matmul_workload(dtype):
     # Case Study 4's loop nest as printed: 6 batches of 196 x 256 x 2305, C += A . B.  K = 2305 breaks every 16-byte
     # rule of the copy engine, so both types first repack their operands K-major with K padded (fp32: as three bf16
-    # pieces), then ONE tensor-core launch covers all batches and one reduction adds the K splits and the old C.
+    # pieces), then ONE tensor-core launch covers all batches; bf16 sums its K slices inside thread-block clusters, where
+    # the old C is added too; fp32 in a reduction launch.
     batch, M, N, K = 6, 196, 256, 2305
     A, B, C = operands(batch, M, N, K, dtype, seed=90)
     n0 = tdx.tdx_kernel_launch_count()
     st, got = run(batch, M, N, K, 0, 0, 1.0, 1.0, dtype, A, B, C)
     assert st == 0, tdx.tdx_last_error()
-    assert tdx.tdx_kernel_launch_count() - n0 <= 3          # repack, GEMM over all batches, reduction: no generic kernel
+    # repack, GEMM over all batches, and for fp32 (whose K split of six does not cut the 128 columns into 32-column
+    # slices) a reduction launch: no generic kernel
+    assert tdx.tdx_kernel_launch_count() - n0 == (2 if dtype == "bf16" else 3)
     err = error(batch, M, N, K, 0, 0, 1.0, 1.0, dtype, A, B, C, got)
     assert err < TOL[dtype] and err < TIGHT[dtype], err
 
