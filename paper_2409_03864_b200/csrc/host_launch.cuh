@@ -40,6 +40,28 @@ int launch_umma(DeviceCtx* ctx, bool conv, const CUtensorMap& ma, const CUtensor
         attr[1].val.clusterDim.y = 1;
         attr[1].val.clusterDim.z = 1;
         lc.numAttrs = 2;
+        // a cluster must fit one GPC with this much shared memory per CTA: ask once per shape of launch, so that a
+        // configuration the device cannot schedule is refused as a configuration, not as a failed launch
+        static std::mutex mu;
+        static std::map<std::array<long long, 4>, int> known;
+        const std::array<long long, 4> key = {ctx->dev, p.split_k, static_cast<long long>(smem), threads};
+        int clusters = -1;
+        {
+            std::lock_guard<std::mutex> lk(mu);
+            auto it = known.find(key);
+            if (it != known.end()) clusters = it->second;
+        }
+        if (clusters < 0) {
+            cudaLaunchConfig_t q = lc;
+            q.numAttrs = 2;
+            q.gridDim = dim3(static_cast<unsigned>(p.split_k));
+            TDX_CUDA(cudaOccupancyMaxActiveClusters(&clusters, tdx::umma_contract_kernel<false>, &q));
+            std::lock_guard<std::mutex> lk(mu);
+            known[key] = clusters;
+        }
+        if (clusters < 1)
+            return fail(TDX_ERR_CONFIG, "a cluster of %d CTAs with %zu bytes of shared memory each cannot be scheduled on this device",
+                        p.split_k, smem);
     }
     if (halo)
         TDX_CUDA(cudaLaunchKernelEx(&lc, tdx::umma_conv_halo_kernel, ma, ma_row ? *ma_row : ma, mb, mc, mc_row ? *mc_row : mc, p));
