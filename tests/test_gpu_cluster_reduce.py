@@ -131,3 +131,33 @@ def test_cluster_reduction_batched_with_accumulate_term():
     assert out.returncode == 0, out.stdout + out.stderr
     line = [l for l in out.stdout.splitlines() if l.startswith("FORCED_OK")][0].split()
     assert int(line[1]) == 1 and float(line[2]) < 1.0, line
+
+
+@pytest.mark.parametrize("shape", [(384, 512, 2048, 0, 0), (520, 392, 1536, 1, 1), (128, 2048, 4096, 0, 1)])
+def test_every_family_of_the_search_space_matches_the_oracle(shape):
+    """Whatever the search may time must also be right: one candidate of every (tile, split, store mode, pair, fit,
+    K order) family that the library enumerates for the shape runs and is compared with the oracle -- the in-cluster
+    split-K of every legal cluster size among them."""
+    M, N, K, tA, tB = shape
+    st, cands = tdx.tdx_enum_gemm_configs(M, N, K, tA, tB, tdx.TDX_BF16)
+    assert st == 0 and cands
+    A, B = si.gemm_bf16_normal(M, N, K, seed=98, transA=tA, transB=tB)
+    ref = oracle.gemm(M, N, K, tA, tB, 1.0, "bf16", A, B)
+    sc = oracle.gemm_row_scales(M, N, K, tA, tB, 1.0, "bf16", A, B)
+    seen, in_cluster = set(), 0
+    for c in cands:
+        fam = (c["tile_m"], c["tile_n"], c["split_k"], c["store_mode"], c["cta_pair"], c["fit"], c["k_stagger"])
+        if fam in seen:
+            continue
+        seen.add(fam)
+        cfg = tdx.tdx_config(**c)
+        ws = None
+        if c["split_k"] > 1 and c["store_mode"] != 3:
+            ws = torch.empty(c["split_k"] * M * N * 4, dtype=torch.uint8, device="cuda")
+        st, C, ok = run_gemm(M, N, K, tA, tB, 1.0, "bf16", A, B, cfg=cfg, workspace=ws)
+        assert st == 0 and ok, (fam, tdx.tdx_last_error())
+        err = oracle.max_normalised_error(oracle.decode(C, "bf16").reshape(M, N), ref, sc)
+        assert err < TIGHT["bf16"], (fam, err)
+        in_cluster += c["store_mode"] == 3
+    assert len(seen) >= 10 and in_cluster >= 1
+    assert tdx.tdx_check_device_status() == 0
