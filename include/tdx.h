@@ -104,7 +104,7 @@ typedef struct {
                     /*     (8 x 16 patches, stride 1, more than one tap); 3 = as 2, but the 16-row patches */
                     /*     are cut from the column formed by all images of the batch, H + pad rows apart, so */
                     /*     that an image height that is no multiple of 16 wastes no rows; 0 = choose        */
-    int fit;        /* GEMM, split_k = 1, tile_n >= 192 (CTA pairs: transB = 1 only): 2 = some row blocks are cut into narrower tiles */
+    int fit;        /* GEMM (split_k = 1; CTA pairs: transB = 1 only) and convolutions whose filter is streamed, tile_n >= 192: 2 = some row blocks are cut into narrower tiles */
                     /*     (multiples of 64 columns) so that all CTAs finish together when the uniform grid  */
                     /*     would leave the last wave of CTAs partly idle; 1 = uniform grid; 0 = fitted when  */
                     /*     the cost model predicts a gain of at least 3 %.  The first call for a shape on a  */

@@ -585,10 +585,10 @@ int run_conv_umma(DeviceCtx* ctx, const ConvProblem& c, const void* x, const voi
     p.cchunks = cchunks;
     p.status = ctx->status_ptr;
 
-    // tile widths fitted to the CTA count, as for the GEMM (halo kernel, streamed filter): the filter slices then
-    // arrive in 64-row copies
+    // tile widths fitted to the CTA count, as for the GEMM (streamed filter): the filter slices then arrive in 64-row
+    // copies
     int plan_grid = 0;
-    if (halo && !p.b_resident && cfg.fit != 1 && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0) {
+    if (!p.b_resident && cfg.fit != 1 && cfg.tile_n >= 192 && cfg.tile_n % 64 == 0) {
         DevicePlan dp;
         int rcp = get_tile_plan(ctx, static_cast<int64_t>(p.tiles_m) * cfg.tile_m, c.Cout, p.num_kb, cfg.tile_m, cfg.tile_n,
                                 cfg.raster, cfg.fit == 2 ? 0.0 : 0.03, &dp);

@@ -371,8 +371,16 @@ double model_conv_us(const ConvProblem& cp, const tdx_config& c, int sm_count, i
     const double blocks = halves * 4.0 * (bn / 32.0);
     const double epi = c.store_mode == 2 ? 600.0 * std::ceil(blocks / 16.0) : 1200.0 * std::ceil(blocks / (4.0 * halves));
     const bool overlapped = tmem_slots_for(tm, bn) > halves;
-    const double rounds = std::ceil(static_cast<double>(tiles) / sm_count);
+    double rounds = std::ceil(static_cast<double>(tiles) / sm_count);
     const double per_tile = overlapped ? std::max(main_loop, epi) : main_loop + epi;
+    // tile widths fitted to the CTA count (streamed filter, tiles of 192 columns or more): the planner's own ratio of
+    // the fitted makespan to the uniform grid's
+    if (c.fit != 1 && bn >= 192 && bn % 64 == 0 && !(c.halo >= 2 && bytes_per_kb < bn * 128.0)) {
+        TilePlan plan;
+        if (plan_fitted_tiles(ceil_div(halves_total, halves) * tm, cp.Cout, num_kb, tm, bn, c.raster, sm_count, c.fit == 2 ? 0.0 : 0.03, &plan) &&
+            plan.uniform > 0.0)
+            rounds *= plan.makespan / plan.uniform;
+    }
     // between configurations with the same number of rounds, the one with less work in total (fewer wasted rows) wins
     const double cycles = 5500.0 + rounds * per_tile + (overlapped ? epi : 0.0) + 1e-3 * static_cast<double>(tiles) * per_tile / sm_count;
     const double hbm_us = (static_cast<double>(cp.N) * cp.H * cp.W * cp.Cin + static_cast<double>(cp.Cout) * taps * cp.Cin +

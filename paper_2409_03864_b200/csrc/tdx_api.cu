@@ -448,13 +448,13 @@ void enum_umma_space(bool b_mn, int64_t tiles_m, int64_t N, int64_t num_kb, int 
                                 c.split_k = sk; c.store_mode = sm; c.raster = raster; c.k_stagger = stagger;
                                 c.patch_w = patch_w; c.patch_h = patch_h;
                                 c.halo = conv ? 1 : 0;
-                                c.fit = conv ? 0 : 1;
+                                c.fit = 1;
                                 if (umma_config_reason(c, b_mn, num_kb, smem_limit, conv, N, 3, 3, stride) != nullptr) continue;
                                 out->push_back(c);
-                                if (!conv && sk == 1 && bn >= 192 && bn % 64 == 0 && stagger == 0) {
+                                if (sk == 1 && bn >= 192 && bn % 64 == 0 && stagger == 0) {
                                     // the same tile with widths fitted to the CTA count, where that changes anything
                                     TilePlan plan;
-                                    if (plan_fitted_tiles(tiles_m * 128, N, num_kb, tm, bn, raster, sm_count, 0.0, &plan)) {
+                                    if (plan_fitted_tiles(tiles_m_t * tm, N, num_kb, tm, bn, raster, sm_count, 0.0, &plan)) {
                                         c.fit = 2;
                                         out->push_back(c);
                                     }

@@ -239,7 +239,8 @@ __device__ __forceinline__ void issue_kblock(const UmmaParams& p, const CUtensor
             const int pw = rem - ph * p.patches_w;
             ld4(a_dst + i * patch_bytes, tmA, cc * kBK, pw * p.bw * p.stride + s - p.pad, ph * p.bh * p.stride + r - p.pad, n);
         }
-        ld3(b_dst, tmB, cc * kBK, tap, t.n0);
+        // (tiles from a fitted table arrive in 64-row copies, like the GEMM's)
+        for (int r0 = 0; r0 < t.bn; r0 += p.b_box) ld3(b_dst + r0 * 128, tmB, cc * kBK, tap, t.n0 + r0);
         return;
     }
     int ka = kb, kbb = kb;                  // K block of A and of B

@@ -333,3 +333,22 @@ def test_conv_halo_with_tile_widths_fitted_to_the_cta_count(tile_m):
     st, y1, ok = run_conv(N, H, W, Cin, Cout, 3, 3, 1, 1, "bf16", x, w, b, 1, cfg=umma(halo=3, tile_m=tile_m, tile_n=256, fit=1))
     assert st == 0 and ok, tdx.tdx_last_error()
     assert np.array_equal(y, y1)          # the reduction order inside an output does not depend on the tile width
+
+
+@pytest.mark.parametrize("case", [(8, 56, 56, 64, 512, 3, 3, 1, 2), (4, 28, 28, 128, 384, 1, 1, 0, 1), (6, 30, 26, 64, 256, 3, 3, 1, 2)])
+@pytest.mark.parametrize("tile_m", [128, 256])
+def test_conv_per_tap_with_tile_widths_fitted_to_the_cta_count(case, tile_m):
+    # fit = 2 on the per-tap kernel (strided layers, 1 x 1 filters): some row blocks are cut into narrower tiles so that
+    # all CTAs finish together; filter slices arrive in 64-row copies.  Same bits as the uniform grid.
+    N, H, W, Cin, Cout, R, S, pad, stride = case
+    x, w, b = si.conv_bf16(N, H, W, Cin, Cout, R, S, seed=87)
+    st, y, ok = run_conv(N, H, W, Cin, Cout, R, S, pad, stride, "bf16", x, w, b, 1, cfg=umma(halo=1, tile_m=tile_m, tile_n=256, fit=2))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    P, Q = oracle.conv_out_dim(H, R, pad, stride), oracle.conv_out_dim(W, S, pad, stride)
+    rows = structured_rows(N * P * Q, max_blocks=24)
+    err = conv_error(N, H, W, Cin, Cout, R, S, pad, stride, "bf16", x, w, b, 1, y, rows=rows)
+    assert err < TIGHT["bf16"], err
+    st, y1, ok = run_conv(N, H, W, Cin, Cout, R, S, pad, stride, "bf16", x, w, b, 1, cfg=umma(halo=1, tile_m=tile_m, tile_n=256, fit=1))
+    assert st == 0 and ok, tdx.tdx_last_error()
+    assert np.array_equal(y, y1)
+    assert tdx.tdx_check_device_status() == 0
