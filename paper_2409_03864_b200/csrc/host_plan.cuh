@@ -333,7 +333,7 @@ double model_gemm_us(const GemmProblem& g, const tdx_config& c, int sm_count) {
     // reads them (128 x 8192 x 8192 in three splits: about 4 us on top of the GEMM kernel)
     if (split > 1 && !in_cluster) us += 2.0 + (static_cast<double>(split) * g.M * g.N * 4.0 * 2.0 + g.M * g.N * 2.0) / 8.0e6;
     const double hbm_us = (static_cast<double>(g.M) * g.K + static_cast<double>(g.K) * g.N + static_cast<double>(g.M) * g.N) * 2.0 / 5.0e6;
-    return std::max(us, hbm_us);
+    return std::max(us, hbm_us) + 1e-3 * us;      // candidates that all sit on the HBM floor keep the order of their compute estimates
 }
 
 // The same kind of model for a convolution configuration (ranks the candidates of the guided convolution search).
@@ -383,9 +383,14 @@ double model_conv_us(const ConvProblem& cp, const tdx_config& c, int sm_count, i
     }
     // between configurations with the same number of rounds, the one with less work in total (fewer wasted rows) wins
     const double cycles = 5500.0 + rounds * per_tile + (overlapped ? epi : 0.0) + 1e-3 * static_cast<double>(tiles) * per_tile / sm_count;
-    const double hbm_us = (static_cast<double>(cp.N) * cp.H * cp.W * cp.Cin + static_cast<double>(cp.Cout) * taps * cp.Cin +
+    // (a strided filter smaller than its stride touches only part of the input.  Candidates that all sit on the HBM floor
+    // -- short reductions, where the model's per-tile figures are least reliable -- are told apart only by what is
+    // known to matter there: fewer copies per K block and fewer rounds; otherwise the first enumerated, the largest
+    // tile, stands: 56 x 56 x 64 -> 256 1 x 1 measured 22.3 us with 256 x 256 tiles, 32.3 with 128 x 128.)
+    const double touched = std::min(1.0, static_cast<double>(cp.R) / cp.stride) * std::min(1.0, static_cast<double>(cp.S) / cp.stride);
+    const double hbm_us = (static_cast<double>(cp.N) * cp.H * cp.W * cp.Cin * touched + static_cast<double>(cp.Cout) * taps * cp.Cin +
                            static_cast<double>(cp.N) * cp.P * cp.Q * cp.Cout) * 2.0 / 5.0e6;
-    return std::max(cycles / clk_mhz, hbm_us);
+    return std::max(cycles / clk_mhz, hbm_us) + 1e-3 * (rounds * (1.0 + static_cast<double>(num_kb) * copy_issue / 1000.0));
 }
 
 }  // namespace
